@@ -1,0 +1,234 @@
+"""Seeded synthetic inputs for the graded KV-cache decode path.
+
+This module only *draws data*: keys, values, queries, prompt attention masses
+and ladder widths shaped like the paper's workloads (Qwen/Llama GQA shapes,
+64-token blocks, outlier key channels, planted heavy tokens, slow drift,
+topical clusters for the page scorer).  It holds none of the method's
+arithmetic (no quantiser, no allocator, no attention over the graded cache)
+and is imported by both the CPU oracle's tests and the CUDA path's tests and
+benchmark, so that both sides see byte-identical inputs.
+
+All tensors are torch tensors; random draws come from one ``torch.Generator``
+per (config, layer) seeded with ``1000 * config_id + layer`` in a fixed order
+(K base, V base, q, outlier permutation, drift, planting, masses), so a given
+(config, layer, device type) always produces the same bytes.
+
+Layouts: K, V ``[B][T][Hkv][d]`` bf16; q ``[B][Hq][d_k]`` bf16; token mass
+``[B][Hkv][T]`` fp32.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from typing import Optional
+
+import torch
+
+BLOCK = 64
+GROUP = 32
+
+POLICY_STAIRCASE = 0
+POLICY_RD = 1
+POLICY_EXTERNAL = 2
+
+
+@dataclasses.dataclass
+class Workload:
+    """Shape + policy description of one benchmark/parity configuration."""
+
+    name: str
+    config_id: int
+    n_layers: int
+    batch: int
+    n_q_heads: int
+    n_kv_heads: int
+    d_k: int
+    d_v: int
+    ctx: int                      # tokens ingested in bulk before decode
+    max_ctx: int
+    v_aliases_k: int = 0
+    page_tokens: int = 0          # 0 = no page scorer
+    policy: int = POLICY_STAIRCASE
+    stair_tokens: tuple = (-1, 0, 0, 0)   # widths of the 16/8/4/2 rungs, newest first
+    n_sink_blocks: int = 0
+    retire_after: int = 0
+    rd_budget_bpv: float = 0.0
+    residual_fraction: float = 0.0
+    softmax_scale: float = 0.0    # 0 -> 1/sqrt(d_k)
+    decode_steps: int = 0
+    quest_budget_tokens: int = 0
+    # data recipe
+    n_outlier: int = 4
+    outlier_gain: float = 8.0
+    n_heavy: int = 16
+    drift_std: float = 0.0
+    n_clusters: int = 0
+
+    @property
+    def group_size(self) -> int:
+        return self.n_q_heads // self.n_kv_heads
+
+
+def config(cid: int, scale: str = "full") -> Workload:
+    """The five benchmark configurations; ``scale='small'`` keeps the structure
+    (every rung populated, ragged tail, several splits) at a size the CPU
+    oracle finishes in seconds."""
+    small = scale == "small"
+    if cid == 0:
+        # tiny single-layer decode: newest 512 exact, 1024 int8, 1536 int4, oldest 1024 int2
+        return Workload("cfg0_tiny_gqa", 0, 1, 1, 8, 2, 128, 128, 4096, 4096 + 128,
+                        stair_tokens=(512, 1024, 1536, 1024))
+    if cid == 1:
+        T = 2048 if small else 16384
+        return Workload("cfg1_qwen3b_rd5", 1, 2 if small else 36, 1, 16, 2, 128, 128, T, T + 128,
+                        policy=POLICY_RD, retire_after=512 if not small else 128,
+                        rd_budget_bpv=4.84, residual_fraction=0.01, drift_std=0.05)
+    if cid == 2:
+        if small:
+            return Workload("cfg2_llama8b_append_small", 2, 2, 2, 8, 2, 128, 128, 2048, 2048 + 256,
+                            stair_tokens=(128, 384, 768, 512), drift_std=0.05, decode_steps=130)
+        return Workload("cfg2_llama8b_append", 2, 32, 8, 32, 8, 128, 128, 32768, 32768 + 256,
+                        stair_tokens=(1024, 4096, 16384, 8192), drift_std=0.05, decode_steps=256)
+    if cid == 3:
+        if small:
+            return Workload("cfg3_quest_small", 3, 1, 2, 8, 2, 128, 128, 2048 + 24, 2048 + 128,
+                            page_tokens=16, policy=POLICY_RD, rd_budget_bpv=4.0, retire_after=64,
+                            n_clusters=16, n_heavy=0, quest_budget_tokens=256)
+        return Workload("cfg3_quest_llama8b", 3, 32, 4, 32, 8, 128, 128, 32768, 32768 + 128,
+                        page_tokens=16, policy=POLICY_RD, rd_budget_bpv=4.0, retire_after=64,
+                        n_clusters=64, n_heavy=0, quest_budget_tokens=2048)
+    if cid == 4:
+        T = 8192 if small else 1048576
+        nb = T // BLOCK
+        w16 = 4096 if not small else 256
+        cen = (nb // 4) * BLOCK
+        rest = T - w16 - cen
+        # 5.000 bits/value: int8 width x and int4 width y with 9x + 5y = 5T - 16*w16 - 0.25*cen
+        # solved in whole blocks in stair_for_cfg4()
+        w8, w4 = _cfg4_split(T, w16, cen)
+        assert w8 + w4 == rest
+        return Workload("cfg4_mla_1m" if not small else "cfg4_mla_small", 4, 1 if small else 27, 1,
+                        16, 1, 576, 512, T, T + 128, v_aliases_k=1,
+                        stair_tokens=(w16, w8, w4, 0), softmax_scale=1.0 / math.sqrt(192.0),
+                        n_outlier=8, outlier_gain=6.0, n_heavy=0)
+    raise ValueError(cid)
+
+
+def _cfg4_split(T: int, w16: int, cen: int):
+    """Whole-block int8/int4 widths that land the MLA ladder on 5.0 bits/value
+    (16, 9, 5 and 0.25 bits/value per rung incl. scale overhead)."""
+    rest_blocks = (T - w16 - cen) // BLOCK
+    target = 5.0 * T - 16.0 * w16 - 0.25 * cen
+    best = None
+    for b8 in range(rest_blocks + 1):
+        b4 = rest_blocks - b8
+        bits = (9 * b8 + 5 * b4) * BLOCK
+        if bits <= target and (best is None or bits > best[0]):
+            best = (bits, b8, b4)
+    return best[1] * BLOCK, best[2] * BLOCK
+
+
+def _gen(device, seed: int) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    return g
+
+
+def _randn(shape, g, device):
+    return torch.randn(shape, generator=g, device=device, dtype=torch.float32)
+
+
+def make_layer(w: Workload, layer: int, device="cpu", ctx: Optional[int] = None,
+               with_mass: Optional[bool] = None):
+    """Draw one layer's prompt K/V, one decode query and (for RD policies) the
+    prompt attention masses.  Returns a dict of tensors on ``device``."""
+    device = torch.device(device)
+    T = w.ctx if ctx is None else ctx
+    B, Hq, Hkv, dk, dv = w.batch, w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v
+    g = _gen(device, 1000 * w.config_id + layer)
+    grp = w.group_size
+
+    q = _randn((B, Hq, dk), g, device)
+    if w.n_clusters > 0:
+        centres = _randn((w.n_clusters, dk), g, device)
+        page = w.page_tokens if w.page_tokens > 0 else BLOCK
+        n_pages = (T + page - 1) // page
+        # topic segments of geometric length (mean 8 pages), one cluster each
+        cont = torch.rand((B, Hkv, n_pages), generator=g, device=device) < (1.0 - 1.0 / 8.0)
+        cont[..., 0] = False
+        seg_id = torch.cumsum((~cont).to(torch.int64), dim=-1) - 1
+        seg_cluster = torch.randint(0, w.n_clusters, (B, Hkv, n_pages), generator=g, device=device)
+        page_cluster = torch.gather(seg_cluster, -1, seg_id)
+        tok_cluster = page_cluster.repeat_interleave(page, dim=-1)[..., :T]      # [B][Hkv][T]
+        K = centres[tok_cluster] + 0.3 * _randn((B, Hkv, T, dk), g, device)       # [B][Hkv][T][dk]
+        K = K.permute(0, 2, 1, 3).contiguous()
+        qc = torch.randint(0, w.n_clusters, (B, Hq), generator=g, device=device)
+        q = centres[qc] + 0.5 * q
+    else:
+        K = _randn((B, T, Hkv, dk), g, device)
+    V = None if w.v_aliases_k else _randn((B, T, Hkv, dv), g, device)
+
+    # outlier channels: first n_outlier entries of a seeded permutation, per KV head
+    for h in range(Hkv):
+        perm = torch.randperm(dk, generator=g, device=device)[: w.n_outlier]
+        K[:, :, h, perm] *= w.outlier_gain
+
+    if w.drift_std > 0:
+        K += torch.cumsum(w.drift_std * _randn((B, T, Hkv, dk), g, device), dim=1)
+        if V is not None:
+            V += torch.cumsum(w.drift_std * _randn((B, T, Hkv, dv), g, device), dim=1)
+
+    if w.n_heavy > 0:
+        n_closed_tok = (T // BLOCK) * BLOCK
+        for b in range(B):
+            for h in range(Hkv):
+                pos = torch.randperm(n_closed_tok, generator=g, device=device)[: w.n_heavy]
+                for i in range(w.n_heavy):
+                    qh = q[b, h * grp + (i % grp)]
+                    qhat = qh / qh.norm()
+                    k = K[b, pos[i], h]
+                    u = k - (k @ qhat) * qhat
+                    u = u / u.norm()
+                    K[b, pos[i], h] = k.norm() * (0.6 * qhat + 0.8 * u)
+
+    out = {
+        "k": K.to(torch.bfloat16),
+        "v": None if V is None else V.to(torch.bfloat16),
+        "q": q.to(torch.bfloat16),
+    }
+
+    want_mass = (w.policy == POLICY_RD) if with_mass is None else with_mass
+    if want_mass:
+        # prompt attention mass per token: softmax weights of 16 synthetic observation
+        # queries per head, averaged over the queries and the g heads of the KV head
+        n_obs = 16
+        scale = w.softmax_scale if w.softmax_scale > 0 else 1.0 / math.sqrt(dk)
+        Kd = out["k"].to(torch.float64)                                  # [B][T][Hkv][dk]
+        qd = out["q"].to(torch.float64).view(B, Hkv, grp, dk)
+        obs = qd[:, :, :, None, :] + 0.5 * torch.randn(
+            (B, Hkv, grp, n_obs, dk), generator=g, device=device, dtype=torch.float64)
+        mass = torch.zeros((B, Hkv, T), dtype=torch.float64, device=device)
+        for b in range(B):
+            for h in range(Hkv):
+                logits = torch.einsum("gnd,td->gnt", obs[b, h], Kd[b, :, h]) * scale
+                mass[b, h] = torch.softmax(logits, dim=-1).mean(dim=(0, 1))
+        out["mass"] = mass.to(torch.float32)
+    return out
+
+
+def make_decode_tokens(w: Workload, layer: int, step: int, device="cpu"):
+    """One decode step's new K/V row per sequence and the step's query
+    (``[B][1][Hkv][d]`` bf16 and ``[B][Hq][d_k]`` bf16)."""
+    device = torch.device(device)
+    g = _gen(device, 7_000_000 + 100_000 * w.config_id + 1000 * layer + step)
+    B, Hq, Hkv, dk, dv = w.batch, w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v
+    k = _randn((B, 1, Hkv, dk), g, device)
+    v = None if w.v_aliases_k else _randn((B, 1, Hkv, dv), g, device)
+    q = _randn((B, Hq, dk), g, device)
+    return {"k": k.to(torch.bfloat16), "v": None if v is None else v.to(torch.bfloat16),
+            "q": q.to(torch.bfloat16)}
+
+
+def bf16_to_f32_numpy(t: torch.Tensor):
+    """bf16 tensor -> float32 numpy array holding the same (bf16-representable) values."""
+    return t.detach().to("cpu").to(torch.float32).numpy()
