@@ -1,0 +1,174 @@
+/*
+ * gkv.h - C ABI of the graded KV-cache decode-attention library (Geodesia-KV hot path).
+ *
+ * One cache object holds, for every (layer, sequence, KV head) "stream", a sequence of
+ * 64-token blocks, each on one rung of the precision ladder {16, 8, 4, 2, centroid}
+ * (paper Sec. 3.2), an always-exact partial tail block, optional exact residual tokens
+ * (Sec. 3.4) and optional exact per-page key min/max boxes (Sec. 3.5).  All compute runs
+ * in CUDA kernels for sm_100a; there is no CPU fallback.
+ *
+ * Conventions
+ *  - "device" pointers are CUDA device memory owned by the caller; "host" pointers are
+ *    ordinary host memory.  The library never allocates device memory: everything it
+ *    keeps on the device lives in the caller's arena.
+ *  - `stream` is a cudaStream_t passed as void*.  All calls on one cache must be issued
+ *    in order on one stream (or externally ordered).  Calls are asynchronous unless the
+ *    function's comment says it synchronises.
+ *  - Every function returns 0 (GKV_OK) or a negative gkv_status.  Arguments are validated
+ *    on the host before anything is launched; nothing traps or asserts on the device.
+ *  - bf16 / fp16 data are raw 16-bit patterns.  Values must be finite and, for blocks
+ *    below level 16 and for queries, within +-65504 (fp16 range).
+ */
+#ifndef GKV_H_
+#define GKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GKV_ABI_VERSION 1u
+#if defined(__GNUC__)
+#define GKV_API __attribute__((visibility("default")))
+#else
+#define GKV_API
+#endif
+
+typedef enum gkv_status {
+  GKV_OK = 0,
+  GKV_ERR_INVALID_ARG = -1,     /* null pointer, bad shape, bad index */
+  GKV_ERR_ARENA_TOO_SMALL = -2, /* arena cannot hold the metadata or a needed block slot */
+  GKV_ERR_CTX_FULL = -3,        /* append would exceed max_ctx */
+  GKV_ERR_BAD_STATE = -4,       /* e.g. page selection without page_tokens, ingest on a non-empty stream */
+  GKV_ERR_UNSUPPORTED = -5,     /* shape or combination not compiled */
+  GKV_ERR_RANGE = -6,           /* a scale/zero saturated at +-65504 (result stored, flag returned) */
+  GKV_ERR_BUDGET = -7,          /* RD budget unreachable even with every free block at centroid (plan applied) */
+  GKV_ERR_CUDA = -8             /* CUDA runtime error; see gkv_last_cuda_error */
+} gkv_status;
+
+enum { GKV_POLICY_STAIRCASE = 0, GKV_POLICY_RD = 1, GKV_POLICY_EXTERNAL = 2 };
+enum { GKV_REDUCE_MAX = 0, GKV_REDUCE_SUM = 1 };
+enum { GKV_TENSOR_K = 0, GKV_TENSOR_V = 1 };
+
+typedef struct gkv_cache gkv_cache; /* opaque; host object owned by the library */
+
+/* Shape and policy of a cache.  Zero-initialise, then set struct_size / abi_version. */
+typedef struct gkv_config {
+  uint32_t struct_size;  /* sizeof(gkv_config) */
+  uint32_t abi_version;  /* GKV_ABI_VERSION */
+  int32_t n_layers, batch, n_q_heads, n_kv_heads; /* n_q_heads % n_kv_heads == 0 */
+  int32_t d_k, d_v;      /* head dims; this build: 128 / 128 */
+  int32_t v_aliases_k;   /* 1: values are channels [0, d_v) of the key row (latent attention) */
+  int32_t max_ctx;       /* capacity in tokens per sequence */
+  int32_t block_tokens;  /* 64 (Sec. 3.2) */
+  int32_t group;         /* 32: keys 32 tokens x 1 channel, values 1 token x 32 channels */
+  int32_t page_tokens;   /* 0 = no page scorer; else 16, 32 or 64 (Sec. 3.5) */
+  int32_t policy;        /* GKV_POLICY_* */
+  int32_t stair_tokens[4]; /* STAIRCASE: widths in tokens of the 16/8/4/2 rungs, newest first;
+                              -1 = unbounded; older blocks are centroid */
+  int32_t n_sink_blocks; /* oldest blocks kept at 16 bits (Fig. 1) */
+  int32_t retire_after;  /* RD: newest retire_after tokens' blocks stay at 16 bits (Sec. 3.2) */
+  float rd_budget_bpv;   /* RD: bits/value incl. scales over all ingested tokens (Eq. 4) */
+  float residual_fraction; /* exact residual tokens per stream = floor(fraction * ctx) (Sec. 3.4) */
+  int32_t quest_reduce;  /* GKV_REDUCE_*: page score over the query heads of a KV head */
+  int32_t monotone_in_age; /* RD: 1 = levels never rise toward older blocks */
+  float softmax_scale;   /* 0 -> 1/sqrt(d_k) */
+} gkv_config;
+
+/* Exact integer accounting of resident and read bits (Sec. 3.5 Eq. 7-8, Sec. 4.4). */
+typedef struct gkv_bits {
+  uint64_t values;        /* K and V values addressed: ctx * (d_k + d_v) per stream, summed */
+  uint64_t code_bits, param_bits, exact_bits, centroid_bits, tail_bits;
+  uint64_t residual_bits, residual_index_bits, box_bits;
+  uint64_t resident_bits; /* sum of the eight categories above */
+  uint64_t meta_bits;     /* block table, residual masks, work descriptors (not in resident_bits) */
+  uint64_t last_read_bits;/* graded bits touched by the last gkv_decode_attn, plus all boxes if a
+                             gkv_quest_select preceded it on that layer */
+  uint64_t blocks_by_level[5]; /* closed blocks at 16, 8, 4, 2, centroid */
+  double bpv_resident, bpv_paper /* without residual index bits */, bpv_read;
+} gkv_bits;
+
+/* Bytes of device arena that are certainly enough for `cfg` (metadata + block slots).
+ * A smaller arena is accepted by gkv_create as long as the metadata fits; appends then
+ * fail with GKV_ERR_ARENA_TOO_SMALL when slots run out.  bytes: host out. */
+GKV_API int gkv_query_arena_bytes(const gkv_config* cfg, size_t* bytes);
+
+/* Create a cache inside `arena` (device, 256-byte aligned, arena_bytes long, owned by the
+ * caller and kept alive until gkv_destroy).  The arena's metadata region is initialised on
+ * the default ordering of `stream`-less cudaMemset, so the call synchronises.  out: host. */
+GKV_API int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache** out);
+
+/* Free the host object (synchronises the device first).  The arena is not touched. */
+GKV_API int gkv_destroy(gkv_cache* c);
+
+/* Append n_new tokens to every sequence of `layer`, then move full blocks down the ladder
+ * (Sec. 3.2: monotone demotion, never upward, requantised from the block's current
+ * representation).  The only mutating call.
+ *   k_new  device bf16 [batch][n_new][n_kv_heads][d_k]
+ *   v_new  device bf16 [batch][n_new][n_kv_heads][d_v]; NULL iff v_aliases_k
+ *   n_new  1 = decode step; >1 only on an empty layer (bulk ingest: each full block is
+ *          encoded once, directly at its planned level)
+ *   token_mass  device fp32 [batch][n_kv_heads][n_new], prompt attention mass per token already
+ *          aggregated over observed queries and the KV head's query heads (Sec. 3.1);
+ *          required for GKV_POLICY_RD and for residual_fraction > 0 at bulk ingest, else NULL
+ *   level_plan  HOST int8 [batch][n_kv_heads][n_new/64], values in {16,8,4,2,1};
+ *          required for GKV_POLICY_EXTERNAL at bulk ingest, else NULL
+ * Bulk ingest under GKV_POLICY_RD (and residual selection) synchronises the stream once, to
+ * run the allocator (Sec. 3.3) on the host.  Decode-step appends never synchronise.
+ * May return GKV_ERR_RANGE / GKV_ERR_BUDGET as warnings after completing the work. */
+GKV_API int gkv_append_demote(gkv_cache* c, int32_t layer, const void* k_new, const void* v_new, int32_t n_new,
+                      const float* token_mass, const int8_t* level_plan, void* stream);
+
+/* Single-query attention of every query head over the graded cache of `layer`
+ * (Sec. 3.7; Eq. 1 over the reconstructed keys/values; split-context partials reduced
+ * separately).
+ *   q        device bf16 [batch][n_q_heads][d_k]
+ *   page_idx device int32 [batch][n_kv_heads][n_sel] ascending closed-page indices, or NULL with
+ *            n_sel = 0 for a full read.  With a list, only those pages and the partial tail block
+ *            are read; every other token is hard-masked (Sec. 3.5)
+ *   out      device fp32 [batch][n_q_heads][d_v]
+ *   lse      device fp32 [batch][n_q_heads] natural-log sum of exp(logit), or NULL */
+GKV_API int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_idx, int32_t n_sel,
+                    float* out, float* lse, void* stream);
+
+/* Compressed-Quest page selection (Sec. 3.5): score every page of every closed block with the
+ * box upper bound sum_d max(q_d * min_d, q_d * max_d), reduce over the KV head's query heads,
+ * keep the k = min(budget_tokens / page_tokens, closed pages) best per (sequence, KV head).
+ *   q            device bf16 [batch][n_q_heads][d_k]
+ *   page_idx_out device int32 [batch][n_kv_heads][k], ascending
+ *   n_sel_out    host int32, receives k */
+GKV_API int gkv_quest_select(gkv_cache* c, int32_t layer, const void* q, int32_t budget_tokens,
+                     int32_t* page_idx_out, int32_t* n_sel_out, void* stream);
+
+/* Resident / read bit accounting of `layer` (-1 = all layers).  Synchronises when the last
+ * read used a page list (it is fetched to count the bits touched).  out: host. */
+GKV_API int gkv_bits_report(gkv_cache* c, int32_t layer, gkv_bits* out);
+
+/* Parity helpers (synchronise).  Logical contents of one closed block of one tensor:
+ *   level       host int32: 16, 8, 4, 2 or 1
+ *   codes       host uint8 [64][d] (levels 8/4/2)
+ *   scale/zero  host fp16 bits; K: [2][d_k] (32-token halves), V: [64][d_v/32]
+ *   rows_bf16   host bf16 bits; level 16: [64][d]; level 1: [d] centroid
+ * Unused outputs may be NULL.  block == number of closed blocks addresses the tail (level 16,
+ * n_rows receives its token count). */
+GKV_API int gkv_debug_export_block(gkv_cache* c, int32_t layer, int32_t b, int32_t kv_head, int32_t block,
+                           int32_t which, int32_t* level, uint8_t* codes, uint16_t* scale_fp16,
+                           uint16_t* zero_fp16, uint16_t* rows_bf16, int32_t* n_rows);
+/* Residual token indices of one stream, ascending.  idx: host int32 [cap]; n: host. */
+GKV_API int gkv_debug_export_residual(gkv_cache* c, int32_t layer, int32_t b, int32_t kv_head, int32_t* idx,
+                              int32_t cap, int32_t* n);
+/* Levels of all closed blocks of one stream.  levels: host int8 [cap]; n: host. */
+GKV_API int gkv_debug_export_levels(gkv_cache* c, int32_t layer, int32_t b, int32_t kv_head, int8_t* levels,
+                            int32_t cap, int32_t* n);
+/* Current context length (tokens) of a layer. */
+GKV_API int gkv_ctx_len(gkv_cache* c, int32_t layer, int32_t* ctx);
+
+GKV_API const char* gkv_strerror(int status);
+GKV_API int gkv_last_cuda_error(gkv_cache* c); /* cudaError_t of the last GKV_ERR_CUDA */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GKV_H_ */

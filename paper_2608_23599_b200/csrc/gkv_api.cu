@@ -1,0 +1,1029 @@
+// Host side of the graded KV-cache library: arena layout, slot allocator, ladder policies and the
+// extern "C" entry points declared in include/gkv.h.  All tensor work is done by the kernels in
+// gkv_decode.cu / gkv_pack.cu / gkv_quest.cu; this file only decides *which* block sits on which
+// rung (paper Sec. 3.2-3.3), where it lives in the arena, and which warp reads what.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/gkv.h"
+#include "gkv_internal.h"
+
+using namespace gkv;
+
+namespace {
+
+constexpr int kTargetWarps = 148 * 2 * kDecodeWarps;   // one resident wave: 2 CTAs x 8 warps per SM
+constexpr int kSparseWarpsPerStream = 16;
+constexpr size_t kMinWarpBytes = 8192;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int level_index(int level) { return level == 16 ? 0 : level == 8 ? 1 : level == 4 ? 2 : level == 2 ? 3 : 4; }
+constexpr int kLevels[5] = {16, 8, 4, 2, 1};
+inline uint32_t slot_units(int level) { return static_cast<uint32_t>(slot_bytes(level) / 256); }
+inline uint64_t block_bits(int level) { return static_cast<uint64_t>(slot_bytes(level)) * 8; }
+
+// Segregated free lists over one heap of 256-byte units.  Slots are freed and reallocated by
+// size class; when the bump region is exhausted a larger free slot is split.
+struct SlotHeap {
+  uint32_t begin = 0, end = 0, bump = 0;
+  std::vector<uint32_t> free_list[5];
+  bool alloc(int level, uint32_t* off) {
+    const int ci = level_index(level);
+    if (!free_list[ci].empty()) {
+      *off = free_list[ci].back();
+      free_list[ci].pop_back();
+      return true;
+    }
+    const uint32_t need = slot_units(level);
+    if (bump + need <= end) {
+      *off = bump;
+      bump += need;
+      return true;
+    }
+    for (int cj = ci - 1; cj >= 0; --cj) {      // split a larger free slot
+      if (free_list[cj].empty()) continue;
+      const uint32_t base = free_list[cj].back();
+      free_list[cj].pop_back();
+      uint32_t rest_off = base + need, rest = slot_units(kLevels[cj]) - need;
+      *off = base;
+      for (int ck = 0; ck < 5 && rest > 0; ++ck) {
+        const uint32_t u = slot_units(kLevels[ck]);
+        while (rest >= u) {
+          free_list[ck].push_back(rest_off);
+          rest_off += u;
+          rest -= u;
+        }
+      }
+      return true;
+    }
+    return false;
+  }
+  void release(int level, uint32_t off) { free_list[level_index(level)].push_back(off); }
+};
+
+struct LayerState {
+  int n_closed = 0, n_tail = 0;
+  bool has_tail_slot = false;
+  std::vector<int8_t> level;            // [n_streams][max_blocks]
+  TableEntry* table_h = nullptr;        // pinned [n_streams][table_stride]
+  WarpDesc* warps_h = nullptr;          // pinned [max_warps]
+  StreamParts* parts_h = nullptr;       // pinned [n_streams]
+  uint32_t* res_off_h = nullptr;        // pinned [n_streams]
+  int32_t* res_count_h = nullptr;       // pinned [n_streams]
+  std::vector<std::vector<int32_t>> res_idx;
+  bool desc_dirty = true;
+  int n_warps = 0;
+  cudaEvent_t ev = nullptr;             // last upload from this layer's pinned mirrors
+  // device regions
+  TableEntry* table_d = nullptr;
+  WarpDesc* warps_d = nullptr;
+  StreamParts* parts_d = nullptr;
+  uint32_t* res_off_d = nullptr;
+  int32_t* res_count_d = nullptr;
+  int32_t* res_idx_d = nullptr;         // [n_streams][res_cap]
+  uint16_t* boxes_d = nullptr;
+  // accounting of the last read
+  int last_mode = 0;                    // 0 none, 1 full, 2 page list
+  const int32_t* last_pages = nullptr;
+  int last_n_sel = 0;
+  bool quest_ran = false;
+  bool budget_flag = false;
+};
+
+}  // namespace
+
+struct gkv_cache {
+  gkv_config cfg;
+  uint8_t* arena = nullptr;
+  size_t arena_bytes = 0;
+  int n_streams = 0, group = 0, max_blocks = 0, table_stride = 0, max_warps = 0, res_cap = 0, box_stride = 0;
+  float scale = 0.f;
+  SlotHeap heap;
+  std::vector<LayerState> layers;
+  // shared device scratch
+  uint32_t* status_d = nullptr;
+  uint8_t* debug_d = nullptr;
+  float* partial_d = nullptr;
+  float* range_d = nullptr;
+  float* mass_d = nullptr;
+  int8_t* levels_d = nullptr;
+  float* scores_d = nullptr;            // residual scores [n_streams][max_ctx] or page scores
+  int32_t* kper_d = nullptr;
+  EncodeJob* jobs_d = nullptr;
+  size_t jobs_cap = 0;
+  // shared pinned staging (jobs | levels | k-per-stream), guarded by ev_stage
+  uint8_t* stage_h = nullptr;
+  size_t stage_bytes = 0;
+  cudaEvent_t ev_stage = nullptr;
+  int last_cuda = 0;
+};
+
+namespace {
+
+struct ArenaPlan {
+  size_t status, debug, partial, range, mass, levels, scores, kper, jobs, per_layer, heap_begin, total_meta;
+  size_t l_table, l_warps, l_parts, l_resoff, l_rescount, l_residx, l_respool, l_boxes, layer_bytes;
+};
+
+struct Derived {
+  int n_streams, group, max_blocks, table_stride, max_warps, res_cap, box_stride;
+};
+
+int validate_config(const gkv_config* c) {
+  if (!c) return GKV_ERR_INVALID_ARG;
+  if (c->struct_size != sizeof(gkv_config) || c->abi_version != GKV_ABI_VERSION) return GKV_ERR_INVALID_ARG;
+  if (c->n_layers <= 0 || c->batch <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0) return GKV_ERR_INVALID_ARG;
+  if (c->n_q_heads % c->n_kv_heads != 0) return GKV_ERR_INVALID_ARG;
+  if (c->max_ctx <= 0) return GKV_ERR_INVALID_ARG;
+  if (c->block_tokens != kBlock || c->group != kGroup) return GKV_ERR_UNSUPPORTED;
+  if (c->d_k != kD || c->d_v != kD || c->v_aliases_k != 0) return GKV_ERR_UNSUPPORTED;
+  if (c->n_q_heads / c->n_kv_heads > kMaxHeadsPerKv) return GKV_ERR_UNSUPPORTED;
+  if (c->page_tokens != 0 && c->page_tokens != 16 && c->page_tokens != 32 && c->page_tokens != 64)
+    return GKV_ERR_INVALID_ARG;
+  if (c->policy < GKV_POLICY_STAIRCASE || c->policy > GKV_POLICY_EXTERNAL) return GKV_ERR_INVALID_ARG;
+  if (c->residual_fraction < 0.f || c->residual_fraction > 1.f) return GKV_ERR_INVALID_ARG;
+  if (c->n_sink_blocks < 0 || c->retire_after < 0) return GKV_ERR_INVALID_ARG;
+  if (c->quest_reduce != GKV_REDUCE_MAX && c->quest_reduce != GKV_REDUCE_SUM) return GKV_ERR_INVALID_ARG;
+  if (c->policy == GKV_POLICY_STAIRCASE)
+    for (int i = 0; i < 4; ++i)
+      if (c->stair_tokens[i] < -1 || (c->stair_tokens[i] > 0 && c->stair_tokens[i] % kBlock)) return GKV_ERR_INVALID_ARG;
+  return GKV_OK;
+}
+
+Derived derive(const gkv_config& c) {
+  Derived d;
+  d.n_streams = c.batch * c.n_kv_heads;
+  d.group = c.n_q_heads / c.n_kv_heads;
+  d.max_blocks = (c.max_ctx + kBlock - 1) / kBlock;
+  d.table_stride = d.max_blocks + 2;
+  d.max_warps = static_cast<int>(align_up(kTargetWarps + 2 * d.n_streams, kDecodeWarps));
+  d.max_warps = std::max(d.max_warps, static_cast<int>(align_up(d.n_streams * kSparseWarpsPerStream, kDecodeWarps)));
+  d.res_cap = c.residual_fraction > 0.f
+                  ? static_cast<int>(align_up(static_cast<size_t>(std::floor(static_cast<double>(c.residual_fraction) * c.max_ctx)) + 16, 16))
+                  : 0;
+  d.box_stride = c.page_tokens > 0 ? static_cast<int>(align_up((c.max_ctx + c.page_tokens - 1) / c.page_tokens, 8)) : 0;
+  return d;
+}
+
+ArenaPlan plan_arena(const gkv_config& c, const Derived& d) {
+  ArenaPlan a;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  a.status = take(256);
+  a.debug = take(kBlock * kD + 2 * 1024 + kBlock * kD * 2);
+  a.partial = take(static_cast<size_t>(d.max_warps) * kPartialFloats * sizeof(float));
+  a.range = take(static_cast<size_t>(d.n_streams) * d.max_blocks * sizeof(float));
+  a.mass = take(static_cast<size_t>(d.n_streams) * d.max_blocks * sizeof(float));
+  a.levels = take(static_cast<size_t>(d.n_streams) * d.max_blocks);
+  const size_t score_elems = std::max<size_t>(c.residual_fraction > 0.f ? c.max_ctx : 0, d.box_stride);
+  a.scores = take(static_cast<size_t>(d.n_streams) * score_elems * sizeof(float));
+  a.kper = take(static_cast<size_t>(d.n_streams) * sizeof(int32_t));
+  a.jobs = take(static_cast<size_t>(d.n_streams) * d.max_blocks * sizeof(EncodeJob));
+  a.per_layer = off;
+  size_t lo = 0;
+  auto ltake = [&](size_t bytes) { size_t o = lo; lo = align_up(lo + bytes, 256); return o; };
+  a.l_table = ltake(static_cast<size_t>(d.n_streams) * d.table_stride * sizeof(TableEntry));
+  a.l_warps = ltake(static_cast<size_t>(d.max_warps) * sizeof(WarpDesc));
+  a.l_parts = ltake(static_cast<size_t>(d.n_streams) * sizeof(StreamParts));
+  a.l_resoff = ltake(static_cast<size_t>(d.n_streams) * sizeof(uint32_t));
+  a.l_rescount = ltake(static_cast<size_t>(d.n_streams) * sizeof(int32_t));
+  a.l_residx = ltake(static_cast<size_t>(d.n_streams) * std::max(d.res_cap, 1) * sizeof(int32_t));
+  a.l_respool = ltake(static_cast<size_t>(d.n_streams) * d.res_cap * 2 * kRowBytes);
+  a.l_boxes = ltake(static_cast<size_t>(d.n_streams) * kD * 2 * d.box_stride * sizeof(uint16_t));
+  a.layer_bytes = lo;
+  a.heap_begin = align_up(a.per_layer + static_cast<size_t>(c.n_layers) * a.layer_bytes, 256);
+  a.total_meta = a.heap_begin;
+  return a;
+}
+
+// Level per closed block (0 = oldest) from rung widths, newest first (Sec. 3.2: blocks leave the
+// recent window and walk down the ladder; sinks stay exact, Fig. 1).
+void staircase_levels(const gkv_config& c, int n_closed, int8_t* lv) {
+  long long edge[4];
+  long long acc = 0;
+  bool unbounded = false;
+  for (int i = 0; i < 4; ++i) {
+    if (c.stair_tokens[i] < 0) unbounded = true;
+    if (!unbounded) acc += c.stair_tokens[i] / kBlock;
+    edge[i] = unbounded ? -1 : acc;
+  }
+  static const int8_t rung[4] = {16, 8, 4, 2};
+  for (int i = 0; i < n_closed; ++i) {
+    const long long age = n_closed - 1 - i;
+    int8_t L = 1;
+    for (int k = 0; k < 4; ++k) {
+      if (edge[k] < 0 || age < edge[k]) {
+        L = rung[k];
+        break;
+      }
+    }
+    if (i < c.n_sink_blocks) L = 16;
+    lv[i] = L;
+  }
+}
+
+// Worst-case slot bytes of one stream under the configured policy at max_ctx.
+size_t worst_stream_bytes(const gkv_config& c, const Derived& d) {
+  size_t bytes = 0;
+  if (c.policy == GKV_POLICY_STAIRCASE) {
+    // the population of each rung is bounded by its width (or by max_blocks when unbounded)
+    std::vector<int8_t> lv(d.max_blocks);
+    staircase_levels(c, d.max_blocks, lv.data());
+    for (int i = 0; i < d.max_blocks; ++i) bytes += slot_bytes(lv[i]);
+    for (int L : kLevels) bytes += 2 * slot_bytes(L);     // allocate-before-free slack + tail
+  } else {
+    bytes = static_cast<size_t>(d.max_blocks + 2) * slot_bytes(16);
+  }
+  return bytes;
+}
+
+int cuda_fail(gkv_cache* c, cudaError_t e) {
+  if (c) c->last_cuda = static_cast<int>(e);
+  return GKV_ERR_CUDA;
+}
+#define CK(c, expr)                                   \
+  do {                                                \
+    cudaError_t e__ = (expr);                         \
+    if (e__ != cudaSuccess) return cuda_fail(c, e__); \
+  } while (0)
+
+// Upload from a pinned mirror; the caller must have waited for `ev` before modifying the mirror.
+int upload(gkv_cache* c, void* dst, const void* src, size_t bytes, cudaStream_t st, cudaEvent_t ev) {
+  if (bytes == 0) return GKV_OK;
+  CK(c, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st));
+  CK(c, cudaEventRecord(ev, st));
+  return GKV_OK;
+}
+
+// ---- RD allocator (Sec. 3.3) -------------------------------------------------------------------
+// The paper's bit depth b* = ceil(log2(c|q| e_b / (2 eps_t) + 1)) with eps_t = tau / (N_b m_b)
+// means "b bits suffice iff y_b = m_b e_b <= tau (2^b - 1)" once constants are folded into tau.
+// Levels snap up to the ladder (b* <= 1 -> centroid); tau is the smallest breakpoint whose plan,
+// after the projections (pinned exact, never above the previous level, never rising toward older
+// blocks), fits the bit budget.
+void rd_levels_for_tau(const std::vector<double>& y, double tau, const std::vector<char>& pinned,
+                       const int8_t* prev, bool mono, std::vector<int8_t>& lv) {
+  const int n = static_cast<int>(y.size());
+  for (int b = 0; b < n; ++b) {
+    int8_t L;
+    if (y[b] <= tau) L = 1;
+    else if (y[b] <= tau * 3.0) L = 2;
+    else if (y[b] <= tau * 15.0) L = 4;
+    else if (y[b] <= tau * 255.0) L = 8;
+    else L = 16;
+    if (pinned[b]) L = 16;
+    if (prev && prev[b] < L) L = prev[b];
+    lv[b] = L;
+  }
+  if (mono) {
+    int nxt = -1;
+    for (int b = n - 1; b >= 0; --b) {
+      if (pinned[b]) continue;
+      if (nxt >= 0 && nxt < lv[b]) lv[b] = static_cast<int8_t>(nxt);
+      nxt = lv[b];
+    }
+  }
+}
+
+bool rd_allocate(const gkv_config& c, const float* mass, const float* range, int n, int n_tail, int8_t* out) {
+  std::vector<double> y(n);
+  std::vector<char> pinned(n, 0);
+  const int recent = c.retire_after / kBlock;
+  for (int b = 0; b < n; ++b) {
+    y[b] = static_cast<double>(mass[b]) * static_cast<double>(range[b]);
+    if (b < c.n_sink_blocks || (n - 1 - b) < recent) pinned[b] = 1;
+  }
+  const long long nval_tok = c.d_k + c.d_v;
+  const long long T = static_cast<long long>(n) * kBlock + n_tail;
+  const long long budget_bits = static_cast<long long>(std::floor(static_cast<double>(c.rd_budget_bpv) * static_cast<double>(T * nval_tok)));
+  const long long tail_bits = static_cast<long long>(n_tail) * 16 * nval_tok;
+  std::vector<double> cands;
+  cands.reserve(4 * n + 1);
+  cands.push_back(0.0);
+  static const double ks[4] = {1.0, 3.0, 15.0, 255.0};
+  for (int b = 0; b < n; ++b)
+    for (double k : ks) cands.push_back(y[b] / k);
+  std::sort(cands.begin(), cands.end());
+  cands.erase(std::unique(cands.begin(), cands.end()), cands.end());
+  std::vector<int8_t> lv(n);
+  auto feasible = [&](double tau) {
+    rd_levels_for_tau(y, tau, pinned, nullptr, c.monotone_in_age != 0, lv);
+    long long bits = tail_bits;
+    for (int b = 0; b < n; ++b) bits += static_cast<long long>(block_bits(lv[b]));
+    return bits <= budget_bits;
+  };
+  // bits(tau) never increases with tau, so the smallest feasible candidate is found by bisection
+  size_t lo = 0, hi = cands.size();
+  while (lo < hi) {
+    const size_t mid = (lo + hi) / 2;
+    if (feasible(cands[mid])) hi = mid;
+    else lo = mid + 1;
+  }
+  bool budget_miss = false;
+  if (lo == cands.size()) {
+    budget_miss = true;
+    lo = cands.size() - 1;
+  }
+  rd_levels_for_tau(y, cands[lo], pinned, nullptr, c.monotone_in_age != 0, lv);
+  std::memcpy(out, lv.data(), n);
+  return budget_miss;
+}
+
+// ---- decode work split ---------------------------------------------------------------------------
+size_t item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) {
+  if (item < L.n_closed) return slot_bytes(L.level[static_cast<size_t>(stream) * c->max_blocks + item]);
+  if (item == L.n_closed) return 16 * 2 * kRowBytes + 1;      // tail: mid-fill estimate (its size changes every step)
+  return 16 * 2 * kRowBytes;                                   // residual group of 16 rows
+}
+
+void build_descs(gkv_cache* c, LayerState& L) {
+  const int ns = c->n_streams;
+  std::vector<int> n_items(ns);
+  std::vector<size_t> bytes(ns, 0);
+  size_t total = 0;
+  for (int s = 0; s < ns; ++s) {
+    const int groups = (L.res_count_h[s] + 15) / 16;
+    n_items[s] = L.n_closed + 1 + groups;
+    for (int i = 0; i < n_items[s]; ++i) bytes[s] += item_cost(c, L, s, i);
+    total += bytes[s];
+  }
+  const size_t target = std::max(kMinWarpBytes, (total + kTargetWarps - 1) / kTargetWarps);
+  int w = 0;
+  for (int s = 0; s < ns; ++s) {
+    int nw = static_cast<int>((bytes[s] + target / 2) / target);
+    nw = std::max(1, std::min(nw, n_items[s]));
+    nw = std::min(nw, c->max_warps - w - (ns - 1 - s));
+    L.parts_h[s].begin = w;
+    size_t acc = 0;
+    int item = 0;
+    for (int k = 0; k < nw; ++k) {
+      const size_t limit = bytes[s] * (k + 1) / nw;
+      const int begin = item;
+      const int max_end = n_items[s] - (nw - 1 - k);     // leave one item for each later warp
+      do {
+        acc += item_cost(c, L, s, item);
+        ++item;
+      } while (item < max_end && acc < limit);
+      WarpDesc& d = L.warps_h[w];
+      d.stream = s;
+      d.item_begin = begin;
+      d.item_end = item;
+      d.partial = w;
+      ++w;
+    }
+    L.warps_h[w - 1].item_end = n_items[s];
+    L.parts_h[s].end = w;
+  }
+  const int padded = static_cast<int>(align_up(w, kDecodeWarps));
+  for (int i = w; i < padded; ++i) L.warps_h[i] = WarpDesc{-1, 0, 0, 0};
+  L.n_warps = padded;
+  L.desc_dirty = false;
+}
+
+void set_entry(gkv_cache* c, LayerState& L, int stream, int block, uint32_t off, int level) {
+  TableEntry& e = L.table_h[static_cast<size_t>(stream) * c->table_stride + block];
+  e.off256 = off;
+  e.level = static_cast<uint32_t>(level);
+}
+
+int wait_event(gkv_cache* c, cudaEvent_t ev) {
+  CK(c, cudaEventSynchronize(ev));
+  return GKV_OK;
+}
+
+int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v_new, int n_new,
+                const float* token_mass, const int8_t* level_plan, cudaStream_t st) {
+  const gkv_config& cfg = c->cfg;
+  LayerState& L = c->layers[layer];
+  const int ns = c->n_streams, n_closed = n_new / kBlock, n_tail = n_new % kBlock;
+  int warn = GKV_OK;
+  int rc;
+  if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
+  if ((rc = wait_event(c, c->ev_stage)) != GKV_OK) return rc;
+
+  // 1. boxes / range / mass of every closed block
+  const bool need_rd = cfg.policy == GKV_POLICY_RD;
+  if ((cfg.page_tokens > 0 || need_rd) && n_closed > 0) {
+    StatsParams sp{};
+    sp.arena = c->arena;
+    sp.k_in = k_new;
+    sp.token_mass = token_mass;
+    sp.n_tok = n_new;
+    sp.n_kv_heads = cfg.n_kv_heads;
+    sp.first_block = 0;
+    sp.n_blocks = n_closed;
+    sp.n_streams = ns;
+    sp.page_tokens = cfg.page_tokens;
+    sp.boxes = L.boxes_d;
+    sp.box_stride = c->box_stride;
+    sp.block_range = need_rd ? c->range_d : nullptr;
+    sp.block_mass = need_rd ? c->mass_d : nullptr;
+    CK(c, launch_stats(sp, st));
+  }
+
+  // 2. level plan
+  std::fill(L.level.begin(), L.level.end(), 0);
+  if (cfg.policy == GKV_POLICY_STAIRCASE) {
+    std::vector<int8_t> lv(std::max(n_closed, 1));
+    staircase_levels(cfg, n_closed, lv.data());
+    for (int s = 0; s < ns; ++s) std::memcpy(&L.level[static_cast<size_t>(s) * c->max_blocks], lv.data(), n_closed);
+  } else if (cfg.policy == GKV_POLICY_EXTERNAL) {
+    for (int s = 0; s < ns; ++s)
+      for (int b = 0; b < n_closed; ++b) {
+        const int8_t v = level_plan[static_cast<size_t>(s) * n_closed + b];
+        if (v != 16 && v != 8 && v != 4 && v != 2 && v != 1) return GKV_ERR_INVALID_ARG;
+        L.level[static_cast<size_t>(s) * c->max_blocks + b] = v;
+      }
+  } else if (n_closed > 0) {
+    std::vector<float> range(static_cast<size_t>(ns) * n_closed), mass(static_cast<size_t>(ns) * n_closed);
+    CK(c, cudaMemcpyAsync(range.data(), c->range_d, range.size() * sizeof(float), cudaMemcpyDeviceToHost, st));
+    CK(c, cudaMemcpyAsync(mass.data(), c->mass_d, mass.size() * sizeof(float), cudaMemcpyDeviceToHost, st));
+    CK(c, cudaStreamSynchronize(st));
+    for (int s = 0; s < ns; ++s) {
+      const bool miss = rd_allocate(cfg, &mass[static_cast<size_t>(s) * n_closed], &range[static_cast<size_t>(s) * n_closed],
+                                    n_closed, n_tail, &L.level[static_cast<size_t>(s) * c->max_blocks]);
+      if (miss) {
+        L.budget_flag = true;
+        warn = GKV_ERR_BUDGET;
+      }
+    }
+  }
+
+  // 3. slots + table mirror
+  for (int s = 0; s < ns; ++s) {
+    for (int b = 0; b <= n_closed; ++b) {
+      const int lvl = b < n_closed ? L.level[static_cast<size_t>(s) * c->max_blocks + b] : 16;
+      uint32_t off;
+      if (!c->heap.alloc(lvl, &off)) return GKV_ERR_ARENA_TOO_SMALL;
+      set_entry(c, L, s, b, off, lvl);
+      L.table_h[static_cast<size_t>(s) * c->table_stride + b].resmask = 0;
+    }
+    L.res_count_h[s] = 0;
+    L.res_idx[s].clear();
+  }
+  L.has_tail_slot = true;
+
+  // 4. exact residual (Sec. 3.4): score, top fraction per stream, gather rows, mask the blocks
+  uint8_t* stage = c->stage_h;
+  size_t stage_off = 0;
+  if (cfg.residual_fraction > 0.f && token_mass && n_closed > 0) {
+    const int n_res_nom = static_cast<int>(std::floor(static_cast<double>(cfg.residual_fraction) * static_cast<double>(n_new)));
+    int8_t* lv_stage = reinterpret_cast<int8_t*>(stage + stage_off);
+    std::memcpy(lv_stage, L.level.data(), L.level.size());
+    stage_off = align_up(stage_off + L.level.size(), 256);
+    int32_t* k_stage = reinterpret_cast<int32_t*>(stage + stage_off);
+    stage_off = align_up(stage_off + ns * sizeof(int32_t), 256);
+    int max_k = 0;
+    for (int s = 0; s < ns; ++s) {
+      int eligible = 0;
+      for (int b = 0; b < n_closed; ++b)
+        if (b >= cfg.n_sink_blocks && L.level[static_cast<size_t>(s) * c->max_blocks + b] != 16) eligible += kBlock;
+      k_stage[s] = std::min(std::min(n_res_nom, eligible), c->res_cap);
+      max_k = std::max(max_k, k_stage[s]);
+      L.res_count_h[s] = k_stage[s];
+    }
+    CK(c, cudaMemcpyAsync(c->levels_d, lv_stage, L.level.size(), cudaMemcpyHostToDevice, st));
+    CK(c, cudaMemcpyAsync(c->kper_d, k_stage, ns * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CK(c, launch_residual_scores(v_new, token_mass, c->levels_d, c->max_blocks, cfg.n_sink_blocks, ns,
+                                 cfg.n_kv_heads, n_new, n_closed, c->scores_d, st));
+    CK(c, launch_topk(c->scores_d, n_new, n_closed * kBlock, c->kper_d, 0, L.res_idx_d, c->res_cap, ns, st));
+    if (max_k > 0) {
+      std::vector<int32_t> idx(static_cast<size_t>(ns) * c->res_cap);
+      CK(c, cudaMemcpyAsync(idx.data(), L.res_idx_d, idx.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+      CK(c, cudaStreamSynchronize(st));
+      for (int s = 0; s < ns; ++s) {
+        L.res_idx[s].assign(idx.begin() + static_cast<size_t>(s) * c->res_cap,
+                            idx.begin() + static_cast<size_t>(s) * c->res_cap + L.res_count_h[s]);
+        for (int32_t tok : L.res_idx[s]) {
+          if (tok < 0 || tok >= n_closed * kBlock) return GKV_ERR_BAD_STATE;
+          L.table_h[static_cast<size_t>(s) * c->table_stride + tok / kBlock].resmask |= 1ull << (tok % kBlock);
+        }
+      }
+    }
+  }
+
+  // 5. uploads, then encode every closed block once at its planned level, copy the tail rows
+  if ((rc = upload(c, L.table_d, L.table_h, static_cast<size_t>(ns) * c->table_stride * sizeof(TableEntry), st, L.ev)) != GKV_OK) return rc;
+  if ((rc = upload(c, L.res_count_d, L.res_count_h, ns * sizeof(int32_t), st, L.ev)) != GKV_OK) return rc;
+  if (L.res_count_d && cfg.residual_fraction > 0.f) {
+    int max_k = 0;
+    for (int s = 0; s < ns; ++s) max_k = std::max(max_k, L.res_count_h[s]);
+    CK(c, launch_residual_gather(c->arena, k_new, v_new, n_new, cfg.n_kv_heads, L.res_idx_d, c->res_cap,
+                                 L.res_count_d, L.res_off_d, max_k, ns, st));
+  }
+  const size_t n_jobs = static_cast<size_t>(ns) * n_closed;
+  if (n_jobs > 0) {
+    EncodeJob* jobs = reinterpret_cast<EncodeJob*>(stage + stage_off);
+    size_t j = 0;
+    for (int s = 0; s < ns; ++s)
+      for (int b = 0; b < n_closed; ++b) {
+        EncodeJob& job = jobs[j++];
+        job.src_off256 = 0;
+        job.dst_off256 = L.table_h[static_cast<size_t>(s) * c->table_stride + b].off256;
+        job.src_level = 0;
+        job.dst_level = L.level[static_cast<size_t>(s) * c->max_blocks + b];
+        job.stream = s;
+        job.block = b;
+        job.pad = 0;
+      }
+    CK(c, cudaMemcpyAsync(c->jobs_d, jobs, n_jobs * sizeof(EncodeJob), cudaMemcpyHostToDevice, st));
+    EncodeParams ep{};
+    ep.arena = c->arena;
+    ep.jobs = c->jobs_d;
+    ep.n_jobs = static_cast<int32_t>(n_jobs);
+    ep.k_in = k_new;
+    ep.v_in = v_new;
+    ep.n_tok = n_new;
+    ep.n_kv_heads = cfg.n_kv_heads;
+    ep.status = c->status_d;
+    CK(c, launch_encode(ep, st));
+  }
+  CK(c, cudaEventRecord(c->ev_stage, st));
+  CK(c, launch_append_rows(c->arena, L.table_d, c->table_stride, n_closed, ns, cfg.n_kv_heads, k_new, v_new, n_new,
+                           n_closed * kBlock, n_tail, 0, st));
+  L.n_closed = n_closed;
+  L.n_tail = n_tail;
+  L.desc_dirty = true;
+  L.last_mode = 0;
+  L.quest_ran = false;
+  return warn;
+}
+
+int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v_new, cudaStream_t st) {
+  const gkv_config& cfg = c->cfg;
+  LayerState& L = c->layers[layer];
+  const int ns = c->n_streams;
+  int rc;
+  const size_t table_bytes = static_cast<size_t>(ns) * c->table_stride * sizeof(TableEntry);
+  if (!L.has_tail_slot) {
+    // a new tail block starts: give every stream an exact slot for it
+    if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
+    for (int s = 0; s < ns; ++s) {
+      uint32_t off;
+      if (!c->heap.alloc(16, &off)) return GKV_ERR_ARENA_TOO_SMALL;
+      set_entry(c, L, s, L.n_closed, off, 16);
+      L.table_h[static_cast<size_t>(s) * c->table_stride + L.n_closed].resmask = 0;
+    }
+    L.has_tail_slot = true;
+    if ((rc = upload(c, L.table_d, L.table_h, table_bytes, st, L.ev)) != GKV_OK) return rc;
+    L.desc_dirty = true;
+  }
+  CK(c, launch_append_rows(c->arena, L.table_d, c->table_stride, L.n_closed, ns, cfg.n_kv_heads, k_new, v_new, 1, 0, 1,
+                           L.n_tail, st));
+  L.n_tail += 1;
+  if (L.n_tail < kBlock) return GKV_OK;
+
+  // the tail block closes (still level 16, in place): boxes from its unquantised keys, then the
+  // staircase moves every block that crossed a rung boundary one or more rungs down
+  const int closed_block = L.n_closed;
+  if (cfg.page_tokens > 0) {
+    StatsParams sp{};
+    sp.arena = c->arena;
+    sp.k_in = nullptr;
+    sp.table = L.table_d;
+    sp.table_stride = c->table_stride;
+    sp.n_tok = 0;
+    sp.n_kv_heads = cfg.n_kv_heads;
+    sp.first_block = closed_block;
+    sp.n_blocks = 1;
+    sp.n_streams = ns;
+    sp.page_tokens = cfg.page_tokens;
+    sp.boxes = L.boxes_d;
+    sp.box_stride = c->box_stride;
+    CK(c, launch_stats(sp, st));
+  }
+  for (int s = 0; s < ns; ++s) L.level[static_cast<size_t>(s) * c->max_blocks + closed_block] = 16;
+  L.n_closed += 1;
+  L.n_tail = 0;
+  L.has_tail_slot = false;
+  L.desc_dirty = true;
+  if (cfg.policy != GKV_POLICY_STAIRCASE) return GKV_OK;
+
+  std::vector<int8_t> target(L.n_closed);
+  staircase_levels(cfg, L.n_closed, target.data());
+  if ((rc = wait_event(c, c->ev_stage)) != GKV_OK) return rc;
+  if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
+  EncodeJob* jobs = reinterpret_cast<EncodeJob*>(c->stage_h);
+  size_t n_jobs = 0;
+  std::vector<std::pair<int, uint32_t>> to_free;
+  for (int s = 0; s < ns; ++s)
+    for (int b = 0; b < L.n_closed; ++b) {
+      int8_t& cur = L.level[static_cast<size_t>(s) * c->max_blocks + b];
+      if (target[b] >= cur) continue;                    // monotone: levels only fall
+      TableEntry& e = L.table_h[static_cast<size_t>(s) * c->table_stride + b];
+      uint32_t off;
+      if (!c->heap.alloc(target[b], &off)) return GKV_ERR_ARENA_TOO_SMALL;
+      EncodeJob& job = jobs[n_jobs++];
+      job.src_off256 = e.off256;
+      job.dst_off256 = off;
+      job.src_level = cur;
+      job.dst_level = target[b];
+      job.stream = s;
+      job.block = b;
+      job.pad = 0;
+      to_free.emplace_back(cur, e.off256);
+      e.off256 = off;
+      e.level = static_cast<uint32_t>(target[b]);
+      cur = target[b];
+    }
+  if (n_jobs > 0) {
+    CK(c, cudaMemcpyAsync(c->jobs_d, jobs, n_jobs * sizeof(EncodeJob), cudaMemcpyHostToDevice, st));
+    CK(c, cudaEventRecord(c->ev_stage, st));
+    EncodeParams ep{};
+    ep.arena = c->arena;
+    ep.jobs = c->jobs_d;
+    ep.n_jobs = static_cast<int32_t>(n_jobs);
+    ep.n_kv_heads = cfg.n_kv_heads;
+    ep.status = c->status_d;
+    CK(c, launch_encode(ep, st));
+    for (auto& f : to_free) c->heap.release(f.first, f.second);
+    if ((rc = upload(c, L.table_d, L.table_h, table_bytes, st, L.ev)) != GKV_OK) return rc;
+  }
+  return GKV_OK;
+}
+
+uint64_t full_read_bits(const gkv_cache* c, const LayerState& L) {
+  const uint64_t nval_tok = c->cfg.d_k + c->cfg.d_v;
+  uint64_t bits = 0;
+  for (int s = 0; s < c->n_streams; ++s) {
+    for (int b = 0; b < L.n_closed; ++b) bits += block_bits(L.level[static_cast<size_t>(s) * c->max_blocks + b]);
+    bits += static_cast<uint64_t>(L.n_tail) * 16 * nval_tok;
+    bits += static_cast<uint64_t>(L.res_count_h[s]) * 16 * nval_tok;
+  }
+  return bits;
+}
+
+}  // namespace
+
+// ================================================================================================
+extern "C" {
+
+const char* gkv_strerror(int status) {
+  switch (status) {
+    case GKV_OK: return "ok";
+    case GKV_ERR_INVALID_ARG: return "invalid argument";
+    case GKV_ERR_ARENA_TOO_SMALL: return "arena too small";
+    case GKV_ERR_CTX_FULL: return "context full";
+    case GKV_ERR_BAD_STATE: return "bad state";
+    case GKV_ERR_UNSUPPORTED: return "unsupported shape or combination";
+    case GKV_ERR_RANGE: return "scale or zero saturated at fp16 range";
+    case GKV_ERR_BUDGET: return "rate-distortion budget unreachable";
+    case GKV_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown status";
+  }
+}
+
+int gkv_last_cuda_error(gkv_cache* c) { return c ? c->last_cuda : 0; }
+
+int gkv_query_arena_bytes(const gkv_config* cfg, size_t* bytes) {
+  int rc = validate_config(cfg);
+  if (rc != GKV_OK) return rc;
+  if (!bytes) return GKV_ERR_INVALID_ARG;
+  const Derived d = derive(*cfg);
+  const ArenaPlan a = plan_arena(*cfg, d);
+  const size_t heap = static_cast<size_t>(cfg->n_layers) * d.n_streams * worst_stream_bytes(*cfg, d);
+  *bytes = a.heap_begin + align_up(heap, 256) + 4096;
+  return GKV_OK;
+}
+
+int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache** out) {
+  int rc = validate_config(cfg);
+  if (rc != GKV_OK) return rc;
+  if (!arena || !out || (reinterpret_cast<uintptr_t>(arena) & 255)) return GKV_ERR_INVALID_ARG;
+  const Derived d = derive(*cfg);
+  const ArenaPlan a = plan_arena(*cfg, d);
+  if (arena_bytes < a.heap_begin + slot_bytes(16)) return GKV_ERR_ARENA_TOO_SMALL;
+  if ((arena_bytes / 256) > 0xffffffffull) return GKV_ERR_UNSUPPORTED;
+  gkv_cache* c = new (std::nothrow) gkv_cache();
+  if (!c) return GKV_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->arena = static_cast<uint8_t*>(arena);
+  c->arena_bytes = arena_bytes;
+  c->n_streams = d.n_streams;
+  c->group = d.group;
+  c->max_blocks = d.max_blocks;
+  c->table_stride = d.table_stride;
+  c->max_warps = d.max_warps;
+  c->res_cap = d.res_cap;
+  c->box_stride = d.box_stride;
+  c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : static_cast<float>(1.0 / std::sqrt(static_cast<double>(cfg->d_k)));
+  c->heap.begin = c->heap.bump = static_cast<uint32_t>(a.heap_begin / 256);
+  c->heap.end = static_cast<uint32_t>(arena_bytes / 256);
+  c->status_d = reinterpret_cast<uint32_t*>(c->arena + a.status);
+  c->debug_d = c->arena + a.debug;
+  c->partial_d = reinterpret_cast<float*>(c->arena + a.partial);
+  c->range_d = reinterpret_cast<float*>(c->arena + a.range);
+  c->mass_d = reinterpret_cast<float*>(c->arena + a.mass);
+  c->levels_d = reinterpret_cast<int8_t*>(c->arena + a.levels);
+  c->scores_d = reinterpret_cast<float*>(c->arena + a.scores);
+  c->kper_d = reinterpret_cast<int32_t*>(c->arena + a.kper);
+  c->jobs_d = reinterpret_cast<EncodeJob*>(c->arena + a.jobs);
+  c->jobs_cap = static_cast<size_t>(d.n_streams) * d.max_blocks;
+
+  auto fail = [&](cudaError_t e) {
+    c->last_cuda = static_cast<int>(e);
+    gkv_destroy(c);
+    return GKV_ERR_CUDA;
+  };
+  cudaError_t e = cudaMemset(c->arena, 0, a.heap_begin);
+  if (e != cudaSuccess) return fail(e);
+  c->stage_bytes = align_up(c->jobs_cap * sizeof(EncodeJob), 256) + align_up(static_cast<size_t>(d.n_streams) * d.max_blocks, 256) +
+                   align_up(d.n_streams * sizeof(int32_t), 256) + 1024;
+  if ((e = cudaHostAlloc(reinterpret_cast<void**>(&c->stage_h), c->stage_bytes, cudaHostAllocDefault)) != cudaSuccess) return fail(e);
+  if ((e = cudaEventCreateWithFlags(&c->ev_stage, cudaEventDisableTiming)) != cudaSuccess) return fail(e);
+  c->layers.resize(cfg->n_layers);
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    LayerState& L = c->layers[l];
+    uint8_t* lb = c->arena + a.per_layer + static_cast<size_t>(l) * a.layer_bytes;
+    L.table_d = reinterpret_cast<TableEntry*>(lb + a.l_table);
+    L.warps_d = reinterpret_cast<WarpDesc*>(lb + a.l_warps);
+    L.parts_d = reinterpret_cast<StreamParts*>(lb + a.l_parts);
+    L.res_off_d = reinterpret_cast<uint32_t*>(lb + a.l_resoff);
+    L.res_count_d = reinterpret_cast<int32_t*>(lb + a.l_rescount);
+    L.res_idx_d = reinterpret_cast<int32_t*>(lb + a.l_residx);
+    L.boxes_d = reinterpret_cast<uint16_t*>(lb + a.l_boxes);
+    L.level.assign(static_cast<size_t>(d.n_streams) * d.max_blocks, 0);
+    L.res_idx.resize(d.n_streams);
+    const size_t tb = static_cast<size_t>(d.n_streams) * d.table_stride * sizeof(TableEntry);
+    if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.table_h), tb, cudaHostAllocDefault)) != cudaSuccess) return fail(e);
+    std::memset(L.table_h, 0, tb);
+    if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.warps_h), d.max_warps * sizeof(WarpDesc), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
+    if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.parts_h), d.n_streams * sizeof(StreamParts), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
+    if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.res_off_h), d.n_streams * sizeof(uint32_t), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
+    if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.res_count_h), d.n_streams * sizeof(int32_t), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
+    for (int s = 0; s < d.n_streams; ++s) {
+      L.res_count_h[s] = 0;
+      L.res_off_h[s] = static_cast<uint32_t>((a.per_layer + static_cast<size_t>(l) * a.layer_bytes + a.l_respool +
+                                              static_cast<size_t>(s) * d.res_cap * 2 * kRowBytes) / 256);
+    }
+    if ((e = cudaEventCreateWithFlags(&L.ev, cudaEventDisableTiming)) != cudaSuccess) return fail(e);
+    if ((e = cudaMemcpy(L.res_off_d, L.res_off_h, d.n_streams * sizeof(uint32_t), cudaMemcpyHostToDevice)) != cudaSuccess) return fail(e);
+  }
+  if ((e = cudaDeviceSynchronize()) != cudaSuccess) return fail(e);
+  *out = c;
+  return GKV_OK;
+}
+
+int gkv_destroy(gkv_cache* c) {
+  if (!c) return GKV_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  for (LayerState& L : c->layers) {
+    if (L.table_h) cudaFreeHost(L.table_h);
+    if (L.warps_h) cudaFreeHost(L.warps_h);
+    if (L.parts_h) cudaFreeHost(L.parts_h);
+    if (L.res_off_h) cudaFreeHost(L.res_off_h);
+    if (L.res_count_h) cudaFreeHost(L.res_count_h);
+    if (L.ev) cudaEventDestroy(L.ev);
+  }
+  if (c->stage_h) cudaFreeHost(c->stage_h);
+  if (c->ev_stage) cudaEventDestroy(c->ev_stage);
+  delete c;
+  return GKV_OK;
+}
+
+int gkv_ctx_len(gkv_cache* c, int32_t layer, int32_t* ctx) {
+  if (!c || !ctx || layer < 0 || layer >= c->cfg.n_layers) return GKV_ERR_INVALID_ARG;
+  const LayerState& L = c->layers[layer];
+  *ctx = L.n_closed * kBlock + L.n_tail;
+  return GKV_OK;
+}
+
+int gkv_append_demote(gkv_cache* c, int32_t layer, const void* k_new, const void* v_new, int32_t n_new,
+                      const float* token_mass, const int8_t* level_plan, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !k_new || !v_new || n_new <= 0) return GKV_ERR_INVALID_ARG;
+  LayerState& L = c->layers[layer];
+  const int ctx = L.n_closed * kBlock + L.n_tail;
+  if (static_cast<long long>(ctx) + n_new > c->cfg.max_ctx) return GKV_ERR_CTX_FULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (n_new == 1) return append_one(c, layer, static_cast<const uint16_t*>(k_new), static_cast<const uint16_t*>(v_new), st);
+  if (ctx != 0) return GKV_ERR_BAD_STATE;
+  if (c->cfg.policy == GKV_POLICY_RD && !token_mass) return GKV_ERR_INVALID_ARG;
+  if (c->cfg.policy == GKV_POLICY_EXTERNAL && !level_plan && n_new >= kBlock) return GKV_ERR_INVALID_ARG;
+  return bulk_ingest(c, layer, static_cast<const uint16_t*>(k_new), static_cast<const uint16_t*>(v_new), n_new,
+                     token_mass, level_plan, st);
+}
+
+int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_idx, int32_t n_sel,
+                    float* out, float* lse, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !out) return GKV_ERR_INVALID_ARG;
+  if (!page_idx && n_sel != 0) return GKV_ERR_INVALID_ARG;
+  LayerState& L = c->layers[layer];
+  if (L.n_closed * kBlock + L.n_tail == 0) return GKV_ERR_BAD_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const gkv_config& cfg = c->cfg;
+  DecodeParams p{};
+  p.arena = c->arena;
+  p.table = L.table_d;
+  p.q = static_cast<const uint16_t*>(q);
+  p.partial = c->partial_d;
+  p.res_off256 = L.res_off_d;
+  p.res_count = L.res_count_d;
+  p.table_stride = c->table_stride;
+  p.n_closed = L.n_closed;
+  p.n_tail = L.n_tail;
+  p.n_kv_heads = cfg.n_kv_heads;
+  p.group = c->group;
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  p.status = c->status_d;
+  CombineParams cp{};
+  cp.partial = c->partial_d;
+  cp.out = out;
+  cp.lse = lse;
+  cp.n_kv_heads = cfg.n_kv_heads;
+  cp.group = c->group;
+  int n_ctas;
+  if (page_idx) {
+    if (cfg.page_tokens <= 0) return GKV_ERR_BAD_STATE;
+    if (n_sel < 0 || n_sel > L.n_closed * (kBlock / cfg.page_tokens)) return GKV_ERR_INVALID_ARG;
+    for (int s = 0; s < c->n_streams; ++s)
+      if (L.res_count_h[s] > 0) return GKV_ERR_UNSUPPORTED;
+    p.page_idx = page_idx;
+    p.n_sel = n_sel;
+    p.page_tokens = cfg.page_tokens;
+    p.warps_per_stream = kSparseWarpsPerStream;
+    p.n_warps = c->n_streams * kSparseWarpsPerStream;
+    p.warps = nullptr;
+    cp.parts = nullptr;
+    cp.warps_per_stream = kSparseWarpsPerStream;
+    n_ctas = (p.n_warps + kDecodeWarps - 1) / kDecodeWarps;
+    L.last_mode = 2;
+    L.last_pages = page_idx;
+    L.last_n_sel = n_sel;
+  } else {
+    if (L.desc_dirty) {
+      int rc = wait_event(c, L.ev);
+      if (rc != GKV_OK) return rc;
+      build_descs(c, L);
+      if ((rc = upload(c, L.warps_d, L.warps_h, static_cast<size_t>(L.n_warps) * sizeof(WarpDesc), st, L.ev)) != GKV_OK) return rc;
+      if ((rc = upload(c, L.parts_d, L.parts_h, static_cast<size_t>(c->n_streams) * sizeof(StreamParts), st, L.ev)) != GKV_OK) return rc;
+    }
+    p.warps = L.warps_d;
+    p.n_warps = L.n_warps;
+    cp.parts = L.parts_d;
+    n_ctas = L.n_warps / kDecodeWarps;
+    L.last_mode = 1;
+    L.quest_ran = false;
+  }
+  CK(c, launch_decode(p, n_ctas, st));
+  CK(c, launch_combine(cp, c->n_streams, st));
+  return GKV_OK;
+}
+
+int gkv_quest_select(gkv_cache* c, int32_t layer, const void* q, int32_t budget_tokens, int32_t* page_idx_out,
+                     int32_t* n_sel_out, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !page_idx_out || !n_sel_out || budget_tokens < 0)
+    return GKV_ERR_INVALID_ARG;
+  const gkv_config& cfg = c->cfg;
+  if (cfg.page_tokens <= 0) return GKV_ERR_BAD_STATE;
+  LayerState& L = c->layers[layer];
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_pages = L.n_closed * (kBlock / cfg.page_tokens);
+  const int k = std::min(budget_tokens / cfg.page_tokens, n_pages);
+  *n_sel_out = k;
+  L.quest_ran = true;
+  if (k <= 0) return GKV_OK;
+  CK(c, launch_quest_scores(L.boxes_d, c->box_stride, n_pages, static_cast<const uint16_t*>(q), c->n_streams,
+                            cfg.n_kv_heads, c->group, cfg.quest_reduce, c->scores_d, c->box_stride, st));
+  CK(c, launch_topk(c->scores_d, c->box_stride, n_pages, nullptr, k, page_idx_out, k, c->n_streams, st));
+  return GKV_OK;
+}
+
+int gkv_bits_report(gkv_cache* c, int32_t layer, gkv_bits* out) {
+  if (!c || !out || layer < -1 || layer >= c->cfg.n_layers) return GKV_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  const gkv_config& cfg = c->cfg;
+  const uint64_t nval_tok = cfg.d_k + cfg.d_v;
+  const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? cfg.n_layers : layer + 1;
+  int warn = GKV_OK;
+  for (int l = l0; l < l1; ++l) {
+    LayerState& L = c->layers[l];
+    const int ctx = L.n_closed * kBlock + L.n_tail;
+    for (int s = 0; s < c->n_streams; ++s) {
+      out->values += static_cast<uint64_t>(ctx) * nval_tok;
+      for (int b = 0; b < L.n_closed; ++b) {
+        const int lv = L.level[static_cast<size_t>(s) * c->max_blocks + b];
+        out->blocks_by_level[level_index(lv)] += 1;
+        if (lv == 16) out->exact_bits += 16ull * kBlock * nval_tok;
+        else if (lv == 1) out->centroid_bits += 16ull * nval_tok;
+        else {
+          out->code_bits += static_cast<uint64_t>(lv) * kBlock * nval_tok;
+          out->param_bits += (kBlock * nval_tok / kGroup) * 32ull;
+        }
+      }
+      out->tail_bits += static_cast<uint64_t>(L.n_tail) * 16 * nval_tok;
+      out->residual_bits += static_cast<uint64_t>(L.res_count_h[s]) * 16 * nval_tok;
+      out->residual_index_bits += static_cast<uint64_t>(L.res_count_h[s]) * 32;
+      if (cfg.page_tokens > 0) out->box_bits += static_cast<uint64_t>(L.n_closed) * (kBlock / cfg.page_tokens) * 2 * cfg.d_k * 16;
+      out->meta_bits += static_cast<uint64_t>(L.n_closed + 1) * sizeof(TableEntry) * 8;
+    }
+    out->meta_bits += static_cast<uint64_t>(L.n_warps) * sizeof(WarpDesc) * 8;
+    if (L.last_mode == 1) out->last_read_bits += full_read_bits(c, L);
+    if (L.last_mode == 2) {
+      // fetch the page list that was used and count what it touched
+      std::vector<int32_t> pages(static_cast<size_t>(c->n_streams) * std::max(L.last_n_sel, 1));
+      if (L.last_n_sel > 0) {
+        cudaError_t e = cudaMemcpy(pages.data(), L.last_pages, static_cast<size_t>(c->n_streams) * L.last_n_sel * sizeof(int32_t), cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+      }
+      const int page = cfg.page_tokens, ppb = kBlock / page;
+      for (int s = 0; s < c->n_streams; ++s) {
+        std::vector<char> group_seen(static_cast<size_t>(L.n_closed) * 2, 0), cent_seen(L.n_closed, 0);
+        for (int i = 0; i < L.last_n_sel; ++i) {
+          const int pg = pages[static_cast<size_t>(s) * L.last_n_sel + i];
+          if (pg < 0 || pg >= L.n_closed * ppb) return GKV_ERR_BAD_STATE;
+          const int blk = pg / ppb;
+          const int lv = L.level[static_cast<size_t>(s) * c->max_blocks + blk];
+          if (lv == 16) out->last_read_bits += static_cast<uint64_t>(page) * 16 * nval_tok;
+          else if (lv == 1) cent_seen[blk] = 1;
+          else {
+            out->last_read_bits += static_cast<uint64_t>(page) * nval_tok * lv;
+            out->last_read_bits += static_cast<uint64_t>(page) * (cfg.d_v / kGroup) * 32;
+            for (int t0 = pg * page; t0 < (pg + 1) * page; t0 += kGroup) group_seen[t0 / kGroup] = 1;
+          }
+        }
+        for (char g : group_seen) if (g) out->last_read_bits += static_cast<uint64_t>(cfg.d_k) * 32;
+        for (char g : cent_seen) if (g) out->last_read_bits += 16ull * nval_tok;
+        out->last_read_bits += static_cast<uint64_t>(L.n_tail) * 16 * nval_tok;
+      }
+    }
+    if (L.quest_ran && L.last_mode == 2)
+      out->last_read_bits += static_cast<uint64_t>(c->n_streams) * L.n_closed * (kBlock / cfg.page_tokens) * 2 * cfg.d_k * 16;
+    if (L.budget_flag) warn = GKV_ERR_BUDGET;
+  }
+  out->resident_bits = out->code_bits + out->param_bits + out->exact_bits + out->centroid_bits + out->tail_bits +
+                       out->residual_bits + out->residual_index_bits + out->box_bits;
+  const double v = static_cast<double>(std::max<uint64_t>(out->values, 1));
+  out->bpv_resident = static_cast<double>(out->resident_bits) / v;
+  out->bpv_paper = static_cast<double>(out->resident_bits - out->residual_index_bits) / v;
+  out->bpv_read = static_cast<double>(out->last_read_bits) / v;
+  // device-detected conditions surface here (this call may synchronise)
+  uint32_t status = 0;
+  cudaError_t e = cudaMemcpy(&status, c->status_d, sizeof(status), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  if (status & kStatusInternal) return GKV_ERR_BAD_STATE;
+  if (status & kStatusRange) warn = GKV_ERR_RANGE;
+  return warn;
+}
+
+int gkv_debug_export_levels(gkv_cache* c, int32_t layer, int32_t b, int32_t kv_head, int8_t* levels, int32_t cap,
+                            int32_t* n) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || b < 0 || b >= c->cfg.batch || kv_head < 0 ||
+      kv_head >= c->cfg.n_kv_heads || !levels || !n)
+    return GKV_ERR_INVALID_ARG;
+  const LayerState& L = c->layers[layer];
+  const int s = b * c->cfg.n_kv_heads + kv_head;
+  *n = L.n_closed;
+  for (int i = 0; i < std::min(cap, L.n_closed); ++i) levels[i] = L.level[static_cast<size_t>(s) * c->max_blocks + i];
+  return GKV_OK;
+}
+
+int gkv_debug_export_residual(gkv_cache* c, int32_t layer, int32_t b, int32_t kv_head, int32_t* idx, int32_t cap,
+                              int32_t* n) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || b < 0 || b >= c->cfg.batch || kv_head < 0 ||
+      kv_head >= c->cfg.n_kv_heads || !idx || !n)
+    return GKV_ERR_INVALID_ARG;
+  const LayerState& L = c->layers[layer];
+  const int s = b * c->cfg.n_kv_heads + kv_head;
+  *n = static_cast<int32_t>(L.res_idx[s].size());
+  for (int i = 0; i < std::min<int>(cap, *n); ++i) idx[i] = L.res_idx[s][i];
+  return GKV_OK;
+}
+
+int gkv_debug_export_block(gkv_cache* c, int32_t layer, int32_t b, int32_t kv_head, int32_t block, int32_t which,
+                           int32_t* level, uint8_t* codes, uint16_t* scale_fp16, uint16_t* zero_fp16,
+                           uint16_t* rows_bf16, int32_t* n_rows) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || b < 0 || b >= c->cfg.batch || kv_head < 0 ||
+      kv_head >= c->cfg.n_kv_heads || (which != GKV_TENSOR_K && which != GKV_TENSOR_V))
+    return GKV_ERR_INVALID_ARG;
+  LayerState& L = c->layers[layer];
+  if (block < 0 || block > L.n_closed || (block == L.n_closed && !L.has_tail_slot)) return GKV_ERR_INVALID_ARG;
+  const int s = b * c->cfg.n_kv_heads + kv_head;
+  const TableEntry& e = L.table_h[static_cast<size_t>(s) * c->table_stride + block];
+  const int lv = block == L.n_closed ? 16 : static_cast<int>(e.level);
+  if (level) *level = lv;
+  if (n_rows) *n_rows = block == L.n_closed ? L.n_tail : (lv == 1 ? 1 : kBlock);
+  CK(c, cudaDeviceSynchronize());
+  uint8_t* d_codes = c->debug_d;
+  uint16_t* d_scale = reinterpret_cast<uint16_t*>(c->debug_d + kBlock * kD);
+  uint16_t* d_zero = reinterpret_cast<uint16_t*>(c->debug_d + kBlock * kD + 1024);
+  uint16_t* d_rows = reinterpret_cast<uint16_t*>(c->debug_d + kBlock * kD + 2048);
+  CK(c, launch_export_block(c->arena, e.off256, lv, which, d_codes, d_scale, d_zero, d_rows, 0));
+  CK(c, cudaDeviceSynchronize());
+  if (lv == 16) {
+    if (rows_bf16) CK(c, cudaMemcpy(rows_bf16, d_rows, kBlock * kD * 2, cudaMemcpyDeviceToHost));
+  } else if (lv == 1) {
+    if (rows_bf16) CK(c, cudaMemcpy(rows_bf16, d_rows, kD * 2, cudaMemcpyDeviceToHost));
+  } else {
+    const size_t np = which == GKV_TENSOR_K ? 2 * kD : kBlock * (kD / kGroup);
+    if (codes) CK(c, cudaMemcpy(codes, d_codes, kBlock * kD, cudaMemcpyDeviceToHost));
+    if (scale_fp16) CK(c, cudaMemcpy(scale_fp16, d_scale, np * 2, cudaMemcpyDeviceToHost));
+    if (zero_fp16) CK(c, cudaMemcpy(zero_fp16, d_zero, np * 2, cudaMemcpyDeviceToHost));
+  }
+  return GKV_OK;
+}
+
+}  // extern "C"

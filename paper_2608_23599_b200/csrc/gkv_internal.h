@@ -1,0 +1,129 @@
+// Structures shared by the host library (gkv_api.cu) and the kernels, and the launch
+// prototypes of every kernel file.  Nothing here is part of the public ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gkv_layout.cuh"
+
+namespace gkv {
+
+// One entry of a stream's block table (device + pinned host mirror).  Index i < n_closed is a
+// closed block, index n_closed is the tail block (level 16, partially filled).
+struct alignas(16) TableEntry {
+  uint32_t off256;   // slot offset from the arena base in 256-byte units
+  uint32_t level;    // 16, 8, 4, 2, 1
+  uint64_t resmask;  // bit t set: token t of the block is served from the residual pool instead
+};
+
+// Work of one warp of the decode kernel: a contiguous range of items of one stream.
+// Items: [0, n_closed) closed blocks, n_closed = tail block, n_closed + 1 + j = residual group j
+// (16 residual rows each).
+struct alignas(16) WarpDesc {
+  int32_t stream;      // -1 = idle warp
+  int32_t item_begin;
+  int32_t item_end;
+  int32_t partial;     // row of the partial buffer this warp writes
+};
+
+struct alignas(8) StreamParts {
+  int32_t begin, end;  // partial rows [begin, end) belong to this stream
+};
+
+constexpr int kDecodeWarps = 8;             // warps per CTA of the decode kernel
+constexpr int kStageBytes = 6144;           // per-warp pipeline stage
+constexpr int kStages = 2;
+constexpr int kMaxHeadsPerKv = 8;           // one n=8 tensor-core tile of query heads
+constexpr int kPartialFloats = kMaxHeadsPerKv * (kD + 2);   // per partial row: m, l, o[128] per head
+
+struct DecodeParams {
+  const uint8_t* arena;
+  const TableEntry* table;      // [n_streams][table_stride]
+  const WarpDesc* warps;        // [n_warps]
+  const uint16_t* q;            // bf16 [batch][n_q_heads][128]
+  float* partial;               // [n_partials][kPartialFloats]
+  const uint32_t* res_off256;   // [n_streams] residual pool offset (rows of 512 B: K row | V row)
+  const int32_t* res_count;     // [n_streams]
+  int32_t table_stride;
+  int32_t n_warps;
+  int32_t n_closed, n_tail;
+  int32_t n_kv_heads, group;    // group = query heads per KV head
+  float scale_log2;             // softmax scale * log2(e)
+  // sparse (page list) mode
+  const int32_t* page_idx;      // [n_streams][n_sel] or nullptr
+  int32_t n_sel, page_tokens, warps_per_stream;
+  uint32_t* status;             // device status word (bit flags)
+};
+
+struct CombineParams {
+  const float* partial;
+  const StreamParts* parts;     // [n_streams]; nullptr in sparse mode (then fixed warps_per_stream)
+  float* out;                   // [batch][n_q_heads][128]
+  float* lse;                   // nullable
+  int32_t n_kv_heads, group, warps_per_stream;
+};
+
+// One block to encode: read 64 tokens from `src`, write level `dst_level` at dst.
+struct alignas(16) EncodeJob {
+  uint32_t src_off256;   // source slot (when src_level != 0)
+  uint32_t dst_off256;
+  int16_t src_level;     // 0 = bf16 input rows (bulk ingest); else level of the source slot
+  int16_t dst_level;
+  int32_t stream;        // for src_level == 0: which (b, kv head); token base = block * 64
+  int32_t block;
+  int32_t pad;
+};
+
+struct EncodeParams {
+  uint8_t* arena;
+  const EncodeJob* jobs;
+  int32_t n_jobs;
+  const uint16_t* k_in;   // bf16 [batch][n_tok][n_kv_heads][128] (src_level == 0)
+  const uint16_t* v_in;
+  int32_t n_tok, n_kv_heads;
+  uint32_t* status;
+};
+
+// Statistics of freshly closed blocks: page boxes, key range proxy, block mass.
+struct StatsParams {
+  uint8_t* arena;
+  const uint16_t* k_in;        // bf16 input rows, or nullptr to read the block's exact slot
+  const float* token_mass;     // [n_streams][n_tok] or nullptr
+  const TableEntry* table;
+  int32_t table_stride;
+  int32_t n_tok, n_kv_heads;
+  int32_t first_block, n_blocks;     // blocks [first_block, first_block + n_blocks) of every stream
+  int32_t n_streams;
+  int32_t page_tokens;               // 0 = no boxes
+  uint16_t* boxes;                   // [n_streams][128][2][box_stride] bf16
+  int32_t box_stride;                // pages (padded)
+  float* block_range;                // [n_streams][n_blocks] or nullptr
+  float* block_mass;                 // [n_streams][n_blocks] or nullptr
+};
+
+constexpr uint32_t kStatusRange = 1u;      // a scale or zero saturated
+constexpr uint32_t kStatusInternal = 2u;   // an index check failed inside a kernel
+
+cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st);
+cudaError_t launch_combine(const CombineParams& p, int n_streams, cudaStream_t st);
+cudaError_t launch_encode(const EncodeParams& p, cudaStream_t st);
+cudaError_t launch_stats(const StatsParams& p, cudaStream_t st);
+cudaError_t launch_append_rows(uint8_t* arena, const TableEntry* table, int table_stride, int tail_index,
+                               int n_streams, int n_kv_heads, const uint16_t* k_in, const uint16_t* v_in,
+                               int n_tok, int first_tok, int n_rows, int dst_row0, cudaStream_t st);
+cudaError_t launch_residual_scores(const uint16_t* v_in, const float* token_mass, const int8_t* levels,
+                                   int levels_stride, int n_sink_blocks, int n_streams, int n_kv_heads, int n_tok,
+                                   int n_closed, float* scores, cudaStream_t st);
+cudaError_t launch_topk(const float* scores, int score_stride, int n, const int32_t* k_per_stream, int k_uniform,
+                        int32_t* idx_out, int idx_stride, int n_streams, cudaStream_t st);
+cudaError_t launch_residual_gather(uint8_t* arena, const uint16_t* k_in, const uint16_t* v_in, int n_tok,
+                                   int n_kv_heads, const int32_t* idx, int idx_stride, const int32_t* count,
+                                   const uint32_t* res_off256, int max_count, int n_streams, cudaStream_t st);
+cudaError_t launch_quest_scores(const uint16_t* boxes, int box_stride, int n_pages, const uint16_t* q,
+                                int n_streams, int n_kv_heads, int group, int reduce, float* scores,
+                                int score_stride, cudaStream_t st);
+cudaError_t launch_export_block(const uint8_t* arena, uint32_t off256, int level, int which, uint8_t* codes,
+                                uint16_t* scale, uint16_t* zero, uint16_t* rows, cudaStream_t st);
+size_t decode_smem_bytes();
+
+}  // namespace gkv

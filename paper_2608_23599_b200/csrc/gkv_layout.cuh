@@ -1,0 +1,103 @@
+// Physical layout of graded blocks in the arena and the logical<->physical index maps.
+//
+// A block is 64 tokens of one (layer, sequence, KV head) stream (paper Sec. 3.2).  Head dim
+// D = 128 in this build.  Slots are multiples of 512 bytes:
+//
+//   level 16 : [K rows 64 x 128 bf16][V rows 64 x 128 bf16]                    32768 B
+//   level 1  : [K centroid 128 bf16][V centroid 128 bf16]                        512 B
+//   level b in {8,4,2}: two halves (tokens 0-31, 32-63), each
+//       Kp   512 B     key scale/zero per channel for this half (keys are grouped along time)
+//       Kc   2 x CB    key codes of the half's two 16-token tiles, CB = 256*b bytes each
+//       Vp   2 x 256 B value scale/zero per (token, 32-channel group) of each tile
+//       Vc   2 x CB    value codes of the two tiles
+//     slot = 2 * (1024 + 4*CB) = 18432 / 10240 / 6144 B
+//
+// Codes are stored in the order the attention kernel's tensor-core fragments consume them, so
+// that a 16-byte load per lane feeds mma.m16n8k16 A operands without any shuffle:
+//   tile (16 tokens), lane = 4*r + c4, mma index s in 0..7, A register a in 0..3, half hlf in 0..1
+//   K role (A = K tile [16 tokens x 16 channels]):
+//       token = 16*tile + r + 8*(a&1),  channel = 16*s + 8*(a>>1) + 2*c4 + hlf
+//   V role (A = V^T tile [16 channels x 16 tokens]):
+//       channel = 16*s + r + 8*(a&1),   token = 16*tile + 8*(a>>1) + 2*c4 + hlf
+// A lane's 64 values of a tile form 32 pairs rho = 4*s + a (lo = hlf 0, hi = hlf 1).  With b-bit
+// codes a 32-bit word holds ppw = 16/b pairs: word = rho / ppw, pos = rho % ppw, lo code at bit
+// b*pos, hi code at bit 16 + b*pos.  Word w of a lane lives at byte
+// ((w/4)*32 + lane)*16 + (w%4)*4 of the tile's code region (chunk-major, 512 B per warp load).
+#pragma once
+#include <stdint.h>
+
+#if defined(__CUDACC__)
+#define GKV_HD __host__ __device__ __forceinline__
+#else
+#define GKV_HD inline
+#endif
+
+namespace gkv {
+
+constexpr int kBlock = 64;     // tokens per block
+constexpr int kGroup = 32;     // quantisation group
+constexpr int kD = 128;        // head dim of this build
+constexpr int kTile = 16;      // tokens per tensor-core tile
+constexpr int kRowBytes = kD * 2;
+
+// Item levels as stored in the block table.
+constexpr int kLvlExact = 16, kLvlCentroid = 1;
+
+GKV_HD int code_bytes_per_tile(int bits) { return 256 * bits; }
+GKV_HD int half_bytes(int bits) { return 1024 + 4 * code_bytes_per_tile(bits); }
+GKV_HD int slot_bytes(int level) {
+  return level == 16 ? 2 * kBlock * kRowBytes : (level == 1 ? 2 * kRowBytes : 2 * half_bytes(level));
+}
+// Offsets inside one half of a quantised slot.
+GKV_HD int off_kp() { return 0; }
+GKV_HD int off_kc(int bits, int t) { return 512 + t * code_bytes_per_tile(bits); }
+GKV_HD int off_vp(int bits, int t) { return 512 + 2 * code_bytes_per_tile(bits) + t * 256; }
+GKV_HD int off_vc(int bits, int t) { return 1024 + (2 + t) * code_bytes_per_tile(bits); }
+
+// Where code (lane, s, a, hlf) of a tile sits: byte offset of its 32-bit word inside the tile's
+// code region, and the bit position inside the word.
+GKV_HD void code_pos(int bits, int lane, int s, int a, int hlf, int* byte_off, int* bit) {
+  const int rho = 4 * s + a;
+  const int ppw = 16 / bits;
+  const int w = rho / ppw, pos = rho % ppw;
+  *byte_off = ((w >> 2) * 32 + lane) * 16 + (w & 3) * 4;
+  *bit = bits * pos + 16 * hlf;
+}
+
+// K role: logical (token in block, channel) -> (tile, lane, s, a, hlf)
+GKV_HD void k_coord(int tok, int ch, int* tile, int* lane, int* s, int* a, int* hlf) {
+  *tile = tok >> 4;
+  const int t16 = tok & 15, c16 = ch & 15;
+  const int r = t16 & 7, c4 = (c16 & 7) >> 1;
+  *lane = 4 * r + c4;
+  *s = ch >> 4;
+  *a = (t16 >> 3) | ((c16 >> 3) << 1);
+  *hlf = c16 & 1;
+}
+// V role: logical (token in block, channel) -> (tile, lane, s, a, hlf)
+GKV_HD void v_coord(int tok, int ch, int* tile, int* lane, int* s, int* a, int* hlf) {
+  *tile = tok >> 4;
+  const int t16 = tok & 15, c16 = ch & 15;
+  const int r = c16 & 7, c4 = (t16 & 7) >> 1;
+  *lane = 4 * r + c4;
+  *s = ch >> 4;
+  *a = (c16 >> 3) | ((t16 >> 3) << 1);
+  *hlf = t16 & 1;
+}
+// Key params of a half: 16-byte records [s][c4] = {scale c0, scale c1, zero c0, zero c1,
+// scale c2, scale c3, zero c2, zero c3} with c0 = 16 s + 2 c4, c1 = c0 + 1, c2 = c0 + 8, c3 = c2 + 1.
+// Returns the index (in fp16 units) of channel ch's scale inside the 512-byte record array;
+// its zero sits 2 entries later.
+GKV_HD int kp_index(int ch) {
+  const int s = ch >> 4, c16 = ch & 15;
+  const int c4 = (c16 & 7) >> 1;
+  return (s * 4 + c4) * 8 + (c16 >> 3) * 4 + (c16 & 1);
+}
+// Value params of a tile: 16-byte records [group][c4] = {scale tA0, scale tA1, zero tA0, zero tA1,
+// scale tB0, scale tB1, zero tB0, zero tB1} with tA0 = 2 c4, tB0 = 8 + 2 c4 (tokens of the tile).
+GKV_HD int vp_index(int t16, int grp) {
+  const int c4 = (t16 & 7) >> 1;
+  return (grp * 4 + c4) * 8 + (t16 >> 3) * 4 + (t16 & 1);
+}
+
+}  // namespace gkv

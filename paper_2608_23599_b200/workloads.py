@@ -178,8 +178,8 @@ def make_layer(w: Workload, layer: int, device="cpu", ctx: Optional[int] = None,
         if V is not None:
             V += torch.cumsum(w.drift_std * _randn((B, T, Hkv, dv), g, device), dim=1)
 
-    if w.n_heavy > 0:
-        n_closed_tok = (T // BLOCK) * BLOCK
+    n_closed_tok = (T // BLOCK) * BLOCK
+    if w.n_heavy > 0 and n_closed_tok >= w.n_heavy:
         for b in range(B):
             for h in range(Hkv):
                 pos = torch.randperm(n_closed_tok, generator=g, device=device)[: w.n_heavy]

@@ -1,0 +1,233 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+Discrete state (levels, codes, scale/zero, centroids, exact rows, residual indices, selected
+pages, bit counts) must match bit for bit; fp32 attention outputs within max-abs 2e-3 and
+relative L2 1e-2."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import gkv_oracle as O
+from paper_2608_23599_b200 import workloads as W
+import parity_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _binding():
+    from paper_2608_23599_b200 import binding as B
+    B.build()
+    return B
+
+
+def _pair(w, n_layers=None):
+    B = _binding()
+    ocache = O.GradedCache(U.oracle_config(w, n_layers))
+    gcache = B.Cache(B.config_from_workload(w, n_layers))
+    return ocache, gcache
+
+
+def _tiny(T, **kw):
+    base = dict(name="tiny", config_id=9, n_layers=1, batch=1, n_q_heads=8, n_kv_heads=2, d_k=128, d_v=128,
+                ctx=T, max_ctx=T + 256)
+    base.update(kw)
+    return W.Workload(**base)
+
+
+@pytest.mark.parametrize("level", [16, 8, 4, 2, 1])
+@pytest.mark.parametrize("T", [64, 200, 1000])
+def test_single_tier(level, T):
+    """Every rung on its own: external plan puts all closed blocks on one level; ragged tail."""
+    w = _tiny(T, policy=W.POLICY_EXTERNAL)
+    ocache, gcache = _pair(w)
+    data = W.make_layer(w, 0, "cpu")
+    plan = np.full((w.batch, w.n_kv_heads, T // 64), level, dtype=np.int8)
+    U.ingest_both(w, 0, data, ocache, gcache, level_plan=plan)
+    U.assert_state_equal(ocache, gcache, 0)
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
+    U.assert_outputs_close(out, o_out, f"level {level} T {T}")
+    assert np.max(np.abs(lse.cpu().numpy() - o_lse)) < 5e-3
+    rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
+    assert rep_g.resident_bits == rep_o["resident_bits"] and rep_g.last_read_bits == rep_o["last_read_bits"]
+    gcache.close()
+
+
+def test_tail_only_and_single_token():
+    """Contexts shorter than one block: only the exact tail exists."""
+    for T in (1, 17, 63):
+        w = _tiny(T)
+        ocache, gcache = _pair(w)
+        data = W.make_layer(w, 0, "cpu")
+        U.ingest_both(w, 0, data, ocache, gcache)
+        U.assert_state_equal(ocache, gcache, 0)
+        out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
+        U.assert_outputs_close(out, o_out, f"tail only T {T}")
+        gcache.close()
+
+
+def test_cfg0_full_parity():
+    """Config 0: 8 query / 2 KV heads, context 4096, ladder 512 exact / 1024 int8 / 1536 int4 / 1024 int2,
+    outlier key channels, planted heavy tokens.  Everything, all blocks."""
+    w = W.config(0)
+    ocache, gcache = _pair(w)
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    U.assert_state_equal(ocache, gcache, 0)
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
+    err, rel = U.assert_outputs_close(out, o_out, "cfg0")
+    rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
+    assert rep_g.bpv_resident == rep_o["bpv_resident"] == 6.875
+    assert rep_g.last_read_bits == rep_o["last_read_bits"]
+    assert list(rep_g.blocks_by_level) == [16, 32, 48, 32, 0]
+    # run to run determinism: bitwise identical outputs
+    out2 = torch.empty_like(out)
+    gcache.gkv_decode_attn(0, data["q"].to(gcache.device), out2)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+    gcache.close()
+
+
+def test_cfg2_small_append_and_demotion():
+    """Config 2 structure at small size: bulk ingest, then one token per step with staircase
+    demotion (16 -> 8 -> 4 -> 2 -> centroid) at every block fill; state bit-exact at checkpoints."""
+    w = W.config(2, "small")
+    ocache, gcache = _pair(w)
+    dev = gcache.device
+    for layer in range(w.n_layers):
+        data = W.make_layer(w, layer, "cpu")
+        U.ingest_both(w, layer, data, ocache, gcache)
+    U.assert_state_equal(ocache, gcache, 0)
+    check_out = {0, 1, 63, 64, 65, 127, 128, 129}
+    check_state = {64, 128}
+    for step in range(w.decode_steps):
+        for layer in range(w.n_layers):
+            tok = W.make_decode_tokens(w, layer, step, "cpu")
+            ocache.append_demote(layer, U.f32(tok["k"]), U.f32(tok["v"]))
+            gcache.gkv_append_demote(layer, tok["k"].to(dev), tok["v"].to(dev))
+            if step in check_out:
+                out, lse, o_out, o_lse = U.decode_both(ocache, gcache, layer, tok["q"])
+                U.assert_outputs_close(out, o_out, f"cfg2-small step {step} layer {layer}")
+        if step + 1 in check_state:
+            for layer in range(w.n_layers):
+                U.assert_state_equal(ocache, gcache, layer)
+                rep_g, rep_o = gcache.gkv_bits_report(layer), ocache.bits_report(layer)
+                assert rep_g.resident_bits == rep_o["resident_bits"]
+    # monotonicity: no block ever rose (oracle history) and the GPU agrees with the final levels
+    for key, st in ocache.streams.items():
+        for blk in st.blocks:
+            assert all(a >= b for a, b in zip(blk.history, blk.history[1:]))
+    gcache.close()
+
+
+def test_cfg1_small_rd_allocator_and_residual():
+    """Config 1 structure: RD allocator at 4.84 bits/value + 1 % exact residual, drifted K/V."""
+    w = W.config(1, "small")
+    ocache, gcache = _pair(w)
+    for layer in range(w.n_layers):
+        data = W.make_layer(w, layer, "cpu")
+        U.ingest_both(w, layer, data, ocache, gcache)
+        U.assert_state_equal(ocache, gcache, layer)
+        lv = ocache.levels(layer, 0, 0)
+        assert len(set(lv.tolist())) >= 3, f"allocator produced a flat plan: {lv}"
+        out, lse, o_out, o_lse = U.decode_both(ocache, gcache, layer, data["q"])
+        U.assert_outputs_close(out, o_out, f"cfg1-small layer {layer}")
+        rep_g, rep_o = gcache.gkv_bits_report(layer), ocache.bits_report(layer)
+        assert rep_g.resident_bits == rep_o["resident_bits"]
+        assert rep_g.last_read_bits == rep_o["last_read_bits"]
+        assert rep_g.bpv_paper <= 4.84 + 16 * 0.01 + 1e-9
+    gcache.close()
+
+
+def test_cfg3_small_quest_select_and_sparse_attention():
+    """Config 3 structure: exact page boxes, box upper-bound scores, top-k pages, attention over
+    the selected graded pages plus the partial tail block."""
+    w = W.config(3, "small")
+    ocache, gcache = _pair(w)
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    U.assert_state_equal(ocache, gcache, 0)
+    k = w.quest_budget_tokens // w.page_tokens
+    pages = torch.full((w.batch, w.n_kv_heads, k), -1, dtype=torch.int32, device=dev)
+    n_sel = gcache.gkv_quest_select(0, data["q"].to(dev), w.quest_budget_tokens, pages)
+    torch.cuda.synchronize()
+    sel_o = ocache.quest_select(0, U.f32(data["q"]), w.quest_budget_tokens)
+    assert n_sel == k
+    pg = pages.cpu().numpy()
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            assert np.array_equal(pg[b, h], sel_o[b][h]), f"selected pages differ for stream {(b, h)}"
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"], page_idx_gpu=pages, n_sel=n_sel,
+                                           page_idx_oracle=sel_o)
+    U.assert_outputs_close(out, o_out, "cfg3-small sparse")
+    rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
+    assert rep_g.resident_bits == rep_o["resident_bits"]
+    assert rep_g.last_read_bits == rep_o["last_read_bits"]
+    # a full read on the same cache still matches
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
+    U.assert_outputs_close(out, o_out, "cfg3-small full")
+    gcache.close()
+
+
+def test_quest_selecting_every_page_equals_full_read():
+    w = dataclasses.replace(W.config(3, "small"), quest_budget_tokens=1 << 20)
+    ocache, gcache = _pair(w)
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    n_pages = (w.ctx // 64) * 4
+    pages = torch.zeros((w.batch, w.n_kv_heads, n_pages), dtype=torch.int32, device=dev)
+    n_sel = gcache.gkv_quest_select(0, data["q"].to(dev), w.quest_budget_tokens, pages)
+    assert n_sel == n_pages
+    out_s = torch.empty((w.batch, w.n_q_heads, w.d_v), dtype=torch.float32, device=dev)
+    out_f = torch.empty_like(out_s)
+    gcache.gkv_decode_attn(0, data["q"].to(dev), out_s, page_idx=pages, n_sel=n_sel)
+    gcache.gkv_decode_attn(0, data["q"].to(dev), out_f)
+    torch.cuda.synchronize()
+    assert torch.allclose(out_s, out_f, atol=2e-4, rtol=0)
+    assert torch.equal(pages.cpu(), torch.arange(n_pages, dtype=torch.int32).expand(w.batch, w.n_kv_heads, n_pages))
+    gcache.close()
+
+
+def test_host_side_errors():
+    B = _binding()
+    w = _tiny(200)
+    gcache = B.Cache(B.config_from_workload(w))
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    out = torch.empty((1, 8, 128), dtype=torch.float32, device=dev)
+    with pytest.raises(B.GkvError) as e:
+        gcache.gkv_decode_attn(0, data["q"].to(dev), out)            # empty layer
+    assert e.value.status == -4
+    gcache.gkv_append_demote(0, data["k"].to(dev), data["v"].to(dev))
+    with pytest.raises(B.GkvError) as e:
+        gcache.gkv_append_demote(0, data["k"].to(dev), data["v"].to(dev))   # bulk ingest on a non-empty layer
+    assert e.value.status == -4
+    with pytest.raises(B.GkvError) as e:
+        gcache.gkv_append_demote(3, data["k"].to(dev), data["v"].to(dev))   # bad layer
+    assert e.value.status == -1
+    pages = torch.zeros((1, 2, 4), dtype=torch.int32, device=dev)
+    with pytest.raises(B.GkvError) as e:
+        gcache.gkv_quest_select(0, data["q"].to(dev), 64, pages)            # no page scorer configured
+    assert e.value.status == -4
+    gcache.close()
+    # an arena that holds the metadata but not the blocks reports ARENA_TOO_SMALL at append time
+    cfg = B.config_from_workload(_tiny(4096))
+    small = B.Cache(cfg, arena_bytes=B.gkv_query_arena_bytes(cfg) - 3 * 1024 * 1024)
+    big = W.make_layer(_tiny(4096), 0, "cpu")
+    with pytest.raises(B.GkvError) as e:
+        small.gkv_append_demote(0, big["k"].to(dev), big["v"].to(dev))
+    assert e.value.status == -2
+    small.close()
+    # context capacity
+    w2 = _tiny(200)
+    w2 = dataclasses.replace(w2, max_ctx=200)
+    full = B.Cache(B.config_from_workload(w2))
+    d2 = W.make_layer(w2, 0, "cpu")
+    full.gkv_append_demote(0, d2["k"].to(dev), d2["v"].to(dev))
+    tok = W.make_decode_tokens(w2, 0, 0, "cpu")
+    with pytest.raises(B.GkvError) as e:
+        full.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
+    assert e.value.status == -3
+    full.close()
