@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the graded decode-attention hot path.
+
+A step = one decode step of the whole hot path over all layers of the workload:
+per layer, gkv_append_demote (append one token per sequence, close/demote blocks) followed by
+gkv_decode_attn over the graded cache (config 3 adds gkv_quest_select and reads the selected
+pages).  Metric: effective context tokens/s = batch * context / step time, plus achieved HBM GB/s
+of the decode kernel against the measured copy bandwidth.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+
+N > 1 runs N independent replicas (the path has no exchange step), one process per GPU under
+torchrun; `value` sums the replicas' tokens over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_23599_b200 import workloads as W  # noqa: E402
+
+METRIC = "graded decode-attn effective ctx tokens/s and HBM GB/s as % of 8 TB/s roofline"
+UNIT = "ctx tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch from an ncu capture
+# (profiles/ holds the summary); None = not captured for that workload.
+DRAM_TRAFFIC_PER_LAUNCH = {}
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled during the timed region."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=self.f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return res
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        os.unlink(self.path)
+        if sm:
+            res.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return res
+
+
+def dist_setup(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return rank, local, world
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def max_over_ranks(x: float, world: int) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# --------------------------------------------------------------------------------------------------
+def build_cache(w: W.Workload, n_layers: int, extra_ctx: int, device):
+    """Generate each layer on the GPU, ingest it, free it."""
+    from paper_2608_23599_b200 import binding as B
+    import dataclasses
+    wl = dataclasses.replace(w, max_ctx=w.ctx + extra_ctx, n_layers=n_layers)
+    cache = B.Cache(B.config_from_workload(wl, n_layers), device=device)
+    qs = []
+    for layer in range(n_layers):
+        data = W.make_layer(wl, layer, device)
+        cache.gkv_append_demote(layer, data["k"], data["v"], token_mass=data.get("mass"))
+        qs.append(data["q"])
+        del data
+    torch.cuda.synchronize()
+    return wl, cache, qs
+
+
+def run_ours(args, rank, local, world):
+    from paper_2608_23599_b200 import binding as B
+    B.build()
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    w = W.config(args.config)
+    n_layers = args.layers or w.n_layers
+    K, Wm = args.steps, args.warmup
+    total_steps = 2 * (K + Wm) + 8
+    wl, cache, q0 = build_cache(w, n_layers, total_steps + 64, device)
+    Bsz, Hq, Hkv, d = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.d_k
+    gen = torch.Generator(device=device)
+    gen.manual_seed(4242 + rank)
+    # per-step decode inputs, resident in HBM for the device-timed region
+    k_new = torch.randn((total_steps, n_layers, Bsz, 1, Hkv, d), generator=gen, device=device).to(torch.bfloat16)
+    v_new = torch.randn((total_steps, n_layers, Bsz, 1, Hkv, d), generator=gen, device=device).to(torch.bfloat16)
+    q_new = torch.randn((total_steps, n_layers, Bsz, Hq, d), generator=gen, device=device).to(torch.bfloat16)
+    out = torch.empty((n_layers, Bsz, Hq, d), dtype=torch.float32, device=device)
+    quest = wl.page_tokens > 0 and wl.quest_budget_tokens > 0
+    k_sel = wl.quest_budget_tokens // wl.page_tokens if quest else 0
+    pages = torch.zeros((Bsz, Hkv, max(k_sel, 1)), dtype=torch.int32, device=device) if quest else None
+
+    def step_device(s):
+        for l in range(n_layers):
+            cache.gkv_append_demote(l, k_new[s, l], v_new[s, l])
+            if quest:
+                n_sel = cache.gkv_quest_select(l, q_new[s, l], wl.quest_budget_tokens, pages)
+                cache.gkv_decode_attn(l, q_new[s, l], out[l], page_idx=pages, n_sel=n_sel)
+            else:
+                cache.gkv_decode_attn(l, q_new[s, l], out[l])
+
+    # ---- device-resident timing -------------------------------------------------------------------
+    s = 0
+    for _ in range(Wm):
+        step_device(s)
+        s += 1
+    ctx_start = cache.gkv_ctx_len(0)
+    sampler = ClockSampler(local)
+    barrier(world)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    closes = 0
+    for _ in range(K):
+        step_device(s)
+        s += 1
+        if cache.gkv_ctx_len(0) % 64 == 0:
+            closes += 1
+    ev1.record()
+    barrier(world)
+    clocks = sampler.stop()
+    ms_step = max_over_ranks(ev0.elapsed_time(ev1) / K, world)
+    value = world * Bsz * ctx_start / (ms_step * 1e-3)
+
+    # ---- dominant kernel: decode_attn alone, per launch -------------------------------------------
+    rep = cache.gkv_bits_report(0)
+    algo_bytes = rep.last_read_bits / 8 + Bsz * Hq * d * 2 + Bsz * Hq * d * 4
+    if quest:
+        algo_bytes = (rep.last_read_bits - rep.box_bits) / 8 + Bsz * Hq * d * 6
+    reps = max(3, min(20, int(2e10 / max(algo_bytes * n_layers, 1))))
+    for l in range(n_layers):
+        if quest:
+            cache.gkv_decode_attn(l, q_new[0, l], out[l], page_idx=pages, n_sel=k_sel)
+        else:
+            cache.gkv_decode_attn(l, q_new[0, l], out[l])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for r in range(reps):
+        for l in range(n_layers):
+            if quest:
+                cache.gkv_decode_attn(l, q_new[r % total_steps, l], out[l], page_idx=pages, n_sel=k_sel)
+            else:
+                cache.gkv_decode_attn(l, q_new[r % total_steps, l], out[l])
+    e1.record()
+    torch.cuda.synchronize()
+    us_launch = e0.elapsed_time(e1) * 1e3 / (reps * n_layers)
+    achieved = algo_bytes / (us_launch * 1e-6) / 1e9
+    peak, peak_kind = measured_hbm_peak()
+    traffic = DRAM_TRAFFIC_PER_LAUNCH.get(wl.name)
+
+    # ---- end to end: host buffers, H2D of the step's inputs and D2H of its result inside the region
+    hk = torch.randn((n_layers, Bsz, 1, Hkv, d)).to(torch.bfloat16).pin_memory()
+    hv = torch.randn((n_layers, Bsz, 1, Hkv, d)).to(torch.bfloat16).pin_memory()
+    hq = torch.randn((n_layers, Bsz, Hq, d)).to(torch.bfloat16).pin_memory()
+    hout = torch.empty((n_layers, Bsz, Hq, d), dtype=torch.float32).pin_memory()
+    dk, dv, dq = torch.empty_like(hk, device=device), torch.empty_like(hv, device=device), torch.empty_like(hq, device=device)
+
+    def step_e2e():
+        dk.copy_(hk, non_blocking=True)
+        dv.copy_(hv, non_blocking=True)
+        dq.copy_(hq, non_blocking=True)
+        for l in range(n_layers):
+            cache.gkv_append_demote(l, dk[l], dv[l])
+            if quest:
+                n_sel = cache.gkv_quest_select(l, dq[l], wl.quest_budget_tokens, pages)
+                cache.gkv_decode_attn(l, dq[l], out[l], page_idx=pages, n_sel=n_sel)
+            else:
+                cache.gkv_decode_attn(l, dq[l], out[l])
+        hout.copy_(out, non_blocking=True)
+        torch.cuda.current_stream().synchronize()      # the caller consumes the step's result
+
+    for _ in range(Wm):
+        step_e2e()
+    ctx_e2e = cache.gkv_ctx_len(0)
+    barrier(world)
+    t0 = time.perf_counter()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()
+    for _ in range(K):
+        step_e2e()
+    g1.record()
+    barrier(world)
+    wall_ms = (time.perf_counter() - t0) * 1e3 / K
+    e2e_ms = max_over_ranks(g0.elapsed_time(g1) / K, world)
+    e2e_value = world * Bsz * ctx_e2e / (e2e_ms * 1e-3)
+    h2d = hk.numel() * 2 + hv.numel() * 2 + hq.numel() * 2
+    d2h = hout.numel() * 4
+
+    launches_per_layer = 3 + (2 if quest else 0)
+    gpu_launches = K * n_layers * launches_per_layer + closes * n_layers * (1 + (1 if wl.page_tokens else 0))
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 exact rows / int8-int4-int2 codes dequantised to f16, f32 accumulate",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "batch": Bsz, "context": ctx_start, "n_layers": n_layers,
+                   "n_q_heads": Hq, "n_kv_heads": Hkv, "head_dim": d, "resident_bpv": rep.bpv_resident,
+                   "l2": "inputs larger than L2: each layer call streams %.0f MB" % (algo_bytes / 1e6),
+                   "parallelism": "replicas x%d" % world, "block_fills_in_timed_region": closes},
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"]},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms, "host_wall_ms_per_step": wall_ms},
+        "gpu_launches": gpu_launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": traffic, "peak_kind": peak_kind + " copy bandwidth",
+                     "kernel": "decode_kernel (+ its combine_kernel, timed per gkv_decode_attn call)",
+                     "us_per_launch": us_launch, "algorithmic_bytes_per_launch": algo_bytes,
+                     "frac_of_8TBs": achieved / NOMINAL_HBM_GBS},
+        "ctx_tokens_per_s_per_layer_call": Bsz * ctx_start / (us_launch * 1e-6),
+    }
+    if rank == 0:
+        line["cpu_baseline"] = cpu_baseline(wl, n_layers, budget_s=args.cpu_seconds)
+    cache.close()
+    return line
+
+
+# --------------------------------------------------------------------------------------------------
+def cpu_baseline(w: W.Workload, n_layers: int, budget_s: float = 20.0, steps: int = 1):
+    """The oracle as it stands, timed on the host cores on a bounded sample: S streams of one layer
+    (ingest untimed), one decode step = append one token + graded attention; scaled to the whole
+    workload (all streams, all layers)."""
+    import dataclasses
+    from oracle import gkv_oracle as O
+    S = 1
+    ws = dataclasses.replace(w, batch=1, n_kv_heads=S, n_q_heads=S * w.group_size, n_layers=1)
+    data = W.make_layer(ws, 0, "cpu")
+    cfg = O.Config(n_layers=1, batch=1, n_q_heads=ws.n_q_heads, n_kv_heads=S, d_k=w.d_k, d_v=w.d_v,
+                   page_tokens=w.page_tokens, policy=w.policy, stair_tokens=tuple(w.stair_tokens),
+                   n_sink_blocks=w.n_sink_blocks, retire_after=w.retire_after, rd_budget_bpv=w.rd_budget_bpv,
+                   residual_fraction=w.residual_fraction, softmax_scale=w.softmax_scale)
+    oc = O.GradedCache(cfg)
+    f32 = lambda t: t.to(torch.float32).numpy()
+    mass = data.get("mass")
+    oc.append_demote(0, f32(data["k"]), f32(data["v"]), token_mass=None if mass is None else mass.numpy())
+    times = []
+    t_begin = time.perf_counter()
+    i = 0
+    while i < max(1, steps) or (time.perf_counter() - t_begin < budget_s and i < 8):
+        tok = W.make_decode_tokens(ws, 0, i, "cpu")
+        kk, vv, qq = f32(tok["k"]), f32(tok["v"]), f32(tok["q"])
+        t0 = time.perf_counter()
+        oc.append_demote(0, kk, vv)
+        if w.page_tokens > 0 and w.quest_budget_tokens > 0:
+            sel = oc.quest_select(0, qq, w.quest_budget_tokens)
+            oc.decode_attn(0, qq, sel)
+        else:
+            oc.decode_attn(0, qq)
+        times.append(time.perf_counter() - t0)
+        i += 1
+    t_stream = float(np.median(times))
+    n_streams = w.batch * w.n_kv_heads
+    t_step = t_stream * n_streams / S * n_layers
+    return {"value": w.batch * w.ctx / t_step, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+            "sample": "%d of %d streams of 1 of %d layers, %d decode steps (append + attention), median, "
+                      "scaled linearly to all streams and layers" % (S, n_streams, n_layers, len(times)),
+            "seconds_per_stream_step": t_stream}
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return None
+    w = W.config(args.config)
+    n_layers = args.layers or w.n_layers
+    t0 = time.perf_counter()
+    base = cpu_baseline(w, n_layers, budget_s=0.0, steps=args.warmup + args.steps)
+    ms = (time.perf_counter() - t0) * 1e3
+    return {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": w.batch * w.ctx / base["value"] * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "batch": w.batch, "context": w.ctx, "n_layers": n_layers},
+            "cpu_baseline": {"value": base["value"], "unit": UNIT, "cores": base["cores"], "kind": "oracle",
+                             "sample": base["sample"]},
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "wall_ms_total": ms}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=2, help="workload: 0..3 (default 2: Llama-8B-like batched decode)")
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (0 = as defined)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        rank = int(os.environ.get("RANK", "0"))
+        world = int(os.environ.get("WORLD_SIZE", "1"))
+        line = run_reference(args, rank, world)
+        if line is not None:
+            print(json.dumps(line))
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    rank, local, world = dist_setup(args.gpus)
+    line = run_ours(args, rank, local, world)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
