@@ -5,14 +5,17 @@
 // blocks of any level, the exact tail block, groups of exact residual rows) and keeps its own
 // online-softmax state for the g <= 8 query heads of the KV head (one read of the KV bytes serves
 // the whole GQA group, Sec. 3.1).  Warps never wait on each other: each one runs a private
-// double-buffered cp.async pipeline (global -> shared, 16 B per lane, 512 B per instruction) and
-// reads back only what it staged, so there are no block-level barriers and no spin waits.
+// double-buffered pipeline of TMA bulk copies (cp.async.bulk global -> shared, completion on a
+// per-warp mbarrier) and consumes only what it staged; every mbarrier wait is bounded.
 //
 // Math: S^T[tokens x heads] = K[tokens x ch] Q^T and O^T[ch x heads] += V^T[ch x tokens] P^T on
 // mma.m16n8k16 with the query heads as the n = 8 dimension.  Quantised codes are stored in
-// A-fragment order (gkv_layout.cuh), unpacked with the fp16 magic-number trick (0x6400 | code),
-// dequantised with one hfma2 per pair and fed to f16 MMAs; exact rows go through ldmatrix and
-// bf16 MMAs with P split into hi + lo bf16 parts so that its rounding stays below 2^-16.
+// A-fragment order (gkv_layout.cuh) at bit positions where one LOP3 turns a code into the fp16
+// number "bias + code".  Scales are folded into the B operands (q' = q * s_k per 32-token key
+// group, P' = p * s_v per 32-channel value group); zero points and the biases are handled by
+// extra MMAs (A = zero-point pattern or all ones) instead of per-value arithmetic, so the ALU
+// cost is ~5 instructions per 8 values.  Exact rows go through ldmatrix and bf16 MMAs with P
+// split into hi + lo bf16 parts so that its rounding stays below 2^-16.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -23,17 +26,37 @@ namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
 constexpr float kNegInf = -__builtin_huge_valf();
+constexpr int kRowPitch = kRowBytes + 16;       // staged exact rows: 272 B pitch -> conflict-free ldmatrix
+constexpr uint32_t kOnesH2 = 0x3C003C00u;       // half2(1, 1)
+constexpr int kWaitSpins = 1 << 22;             // bound of every mbarrier wait
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&a)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
@@ -56,11 +79,12 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                        uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ uint32_t lop3_and_or(uint32_t x, uint32_t mask, uint32_t orv) {
   uint32_t r;
@@ -74,6 +98,7 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 }
 __device__ __forceinline__ uint32_t h2_as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
+__device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) { return h2_as_u32(__hmul2(u32_as_h2(a), u32_as_h2(b))); }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -81,85 +106,73 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
-// Unpack the four A registers of one MMA from packed codes and dequantise them:
-// a0,a1 use (scA, zrA), a2,a3 use (scB, zrB).  `w` is the 32-bit word holding the pairs and
-// `odd` tells (for 2-bit codes) whether the MMA index is odd (pairs 4..7 of the word).
+// ---- code unpack: the four A registers of MMA index s as fp16 "bias + code" ------------------
+// Biases (rows r / rows r + 8 of the MMA): 8-bit 1024 / 1024; 4-bit 256 / 16; 2-bit 256 / 64 for
+// even s and 16 / 4 for odd s.  `mid` is the centre of the code range: products are formed with
+// (code - mid) so that the fp16 rounding of the folded scale acts on a centred value; the term
+// mid * sum(q s) is added back from an exact MMA.
 template <int BITS>
-__device__ __forceinline__ void unpack_dequant(uint32_t w0, uint32_t w1, bool odd, __half2 scA, __half2 zrA,
-                                               __half2 scB, __half2 zrB, uint32_t (&a)[4]) {
-  constexpr uint32_t kMagic = 0x64006400u;   // half2(1024, 1024)
-  __half2 c0, c1, c2, c3;
-  if constexpr (BITS == 8) {
-    // w0 = pairs (a0, a1), w1 = pairs (a2, a3); pair pos 0: bytes 0/2, pos 1: bytes 1/3;
-    // selector 5 picks the 0x64 byte of the magic word as the high byte of each half
-    const __half2 k1024 = __float2half2_rn(1024.f);
-    c0 = __hsub2(u32_as_h2(prmt(w0, kMagic, 0x5250u)), k1024);
-    c1 = __hsub2(u32_as_h2(prmt(w0, kMagic, 0x5351u)), k1024);
-    c2 = __hsub2(u32_as_h2(prmt(w1, kMagic, 0x5250u)), k1024);
-    c3 = __hsub2(u32_as_h2(prmt(w1, kMagic, 0x5351u)), k1024);
-  } else if constexpr (BITS == 4) {
-    // w0 holds the four pairs: pos p at bits 4p / 16 + 4p
-    const __half2 k1024 = __float2half2_rn(1024.f);
-    const __half2 k16th = __float2half2_rn(0.0625f), km64 = __float2half2_rn(-64.f);
-    const uint32_t hi = w0 >> 8;
-    c0 = __hsub2(u32_as_h2(lop3_and_or(w0, 0x000F000Fu, kMagic)), k1024);
-    c1 = __hfma2(u32_as_h2(lop3_and_or(w0, 0x00F000F0u, kMagic)), k16th, km64);
-    c2 = __hsub2(u32_as_h2(lop3_and_or(hi, 0x000F000Fu, kMagic)), k1024);
-    c3 = __hfma2(u32_as_h2(lop3_and_or(hi, 0x00F000F0u, kMagic)), k16th, km64);
-  } else {
-    // 2-bit: the word holds eight pairs; an odd MMA index uses pairs 4..7 (bits 8.. / 24..)
-    const uint32_t v = odd ? (w0 >> 8) : w0;
-    c0 = __hsub2(u32_as_h2(lop3_and_or(v, 0x00030003u, kMagic)), __float2half2_rn(1024.f));
-    c1 = __hfma2(u32_as_h2(lop3_and_or(v, 0x000C000Cu, kMagic)), __float2half2_rn(0.25f), __float2half2_rn(-256.f));
-    c2 = __hfma2(u32_as_h2(lop3_and_or(v, 0x00300030u, kMagic)), __float2half2_rn(0.0625f), __float2half2_rn(-64.f));
-    c3 = __hfma2(u32_as_h2(lop3_and_or(v, 0x00C000C0u, kMagic)), __float2half2_rn(0.015625f), __float2half2_rn(-16.f));
-  }
-  a[0] = h2_as_u32(__hfma2(c0, scA, zrA));
-  a[1] = h2_as_u32(__hfma2(c1, scA, zrA));
-  a[2] = h2_as_u32(__hfma2(c2, scB, zrB));
-  a[3] = h2_as_u32(__hfma2(c3, scB, zrB));
-}
+struct Bias;
+template <>
+struct Bias<8> {
+  static constexpr float lo_even = 1024.f, hi_even = 1024.f, lo_odd = 1024.f, hi_odd = 1024.f, mid = 127.5f;
+};
+template <>
+struct Bias<4> {
+  static constexpr float lo_even = 256.f, hi_even = 16.f, lo_odd = 256.f, hi_odd = 16.f, mid = 7.5f;
+};
+template <>
+struct Bias<2> {
+  static constexpr float lo_even = 256.f, hi_even = 64.f, lo_odd = 16.f, hi_odd = 4.f, mid = 1.5f;
+};
 
-// Fetch the code word(s) of MMA index s from a lane's preloaded chunk(s) of a tile.
+// Words of one lane for MMA indices [s0, s0 + NS): 8-bit 2 words per s, 4-bit 1, 2-bit 1 per 2.
 template <int BITS>
-struct TileCodes {
-  // 8-bit: 16 words (4 chunks); 4-bit: 8 words (2 chunks); 2-bit: 4 words (1 chunk)
-  static constexpr int kChunks = BITS / 2;
-  uint4 ch[kChunks];
-  __device__ __forceinline__ void load(const uint8_t* tile_codes, int lane) {
-#pragma unroll
-    for (int j = 0; j < kChunks; ++j) ch[j] = *reinterpret_cast<const uint4*>(tile_codes + (j * 32 + lane) * 16);
-  }
-  __device__ __forceinline__ uint32_t word(int w) const {
-    const uint4& c = ch[w >> 2];
-    switch (w & 3) {
-      case 0: return c.x;
-      case 1: return c.y;
-      case 2: return c.z;
-      default: return c.w;
+__device__ __forceinline__ void unpack(const uint32_t* w, int s_local, uint32_t (&a)[4]) {
+  if constexpr (BITS == 8) {
+    constexpr uint32_t kMagic = 0x64006400u;            // selector 5 picks the 0x64 byte
+    const uint32_t w0 = w[2 * s_local], w1 = w[2 * s_local + 1];
+    a[0] = prmt(w0, kMagic, 0x5250u);
+    a[1] = prmt(w0, kMagic, 0x5351u);
+    a[2] = prmt(w1, kMagic, 0x5250u);
+    a[3] = prmt(w1, kMagic, 0x5351u);
+  } else if constexpr (BITS == 4) {
+    const uint32_t v0 = w[s_local] << 2, v1 = w[s_local] >> 6;
+    a[0] = lop3_and_or(v0, 0x003C003Cu, 0x5C005C00u);   // 256 + code
+    a[1] = lop3_and_or(v0, 0x03C003C0u, 0x4C004C00u);   // 16 + code
+    a[2] = lop3_and_or(v1, 0x003C003Cu, 0x5C005C00u);
+    a[3] = lop3_and_or(v1, 0x03C003C0u, 0x4C004C00u);
+  } else {
+    const uint32_t v0 = w[s_local >> 1] << 2, v1 = w[s_local >> 1] >> 6;
+    if ((s_local & 1) == 0) {
+      a[0] = lop3_and_or(v0, 0x000C000Cu, 0x5C005C00u);  // 256 + code
+      a[1] = lop3_and_or(v0, 0x00300030u, 0x54005400u);  // 64 + code
+      a[2] = lop3_and_or(v1, 0x000C000Cu, 0x5C005C00u);
+      a[3] = lop3_and_or(v1, 0x00300030u, 0x54005400u);
+    } else {
+      a[0] = lop3_and_or(v0, 0x00C000C0u, 0x4C004C00u);  // 16 + code
+      a[1] = lop3_and_or(v0, 0x03000300u, 0x44004400u);  // 4 + code
+      a[2] = lop3_and_or(v1, 0x00C000C0u, 0x4C004C00u);
+      a[3] = lop3_and_or(v1, 0x03000300u, 0x44004400u);
     }
   }
-};
+}
 
 struct SoftmaxState {
   float m0, m1;        // running max (log2 domain) of heads 2*c4, 2*c4+1
   float l0, l1;        // lane-partial sums of exp2 (reduced over the r lanes at the end)
   float o[8][4];       // O^T accumulators: tile u rows (16u + r, 16u + 8 + r) x heads (2c4, 2c4+1)
+  float zc[4];         // value zero-point term: rows = 32-channel groups (lanes r < 4), same heads
 };
 
-// Online-softmax update for NT token tiles.  On entry S holds raw dot products; bias is additive
-// in the log2 domain (0, -inf for masked tokens, log2(count) for centroid rows).  On exit S holds
-// the probabilities relative to the new running max.
+// Online-softmax update for NT token tiles.  On entry S holds logits in the log2 domain (bias
+// already added: 0, -inf for masked tokens, log2(count) for centroid rows).  On exit S holds the
+// probabilities relative to the new running max.
 template <int NT>
-__device__ __forceinline__ void softmax_update(float (&S)[NT][4], const float (&bias)[NT][2], float scale_log2,
-                                               SoftmaxState& st) {
+__device__ __forceinline__ void softmax_update(float (&S)[NT][4], SoftmaxState& st) {
   float mx0 = kNegInf, mx1 = kNegInf;
 #pragma unroll
   for (int t = 0; t < NT; ++t) {
-    S[t][0] = fmaf(S[t][0], scale_log2, bias[t][0]);
-    S[t][1] = fmaf(S[t][1], scale_log2, bias[t][0]);
-    S[t][2] = fmaf(S[t][2], scale_log2, bias[t][1]);
-    S[t][3] = fmaf(S[t][3], scale_log2, bias[t][1]);
     mx0 = fmaxf(mx0, fmaxf(S[t][0], S[t][2]));
     mx1 = fmaxf(mx1, fmaxf(S[t][1], S[t][3]));
   }
@@ -170,17 +183,21 @@ __device__ __forceinline__ void softmax_update(float (&S)[NT][4], const float (&
   }
   const float mn0 = fmaxf(st.m0, mx0), mn1 = fmaxf(st.m1, mx1);
   const float ms0 = (mn0 == kNegInf) ? 0.f : mn0, ms1 = (mn1 == kNegInf) ? 0.f : mn1;
-  const float al0 = exp2f(st.m0 - ms0), al1 = exp2f(st.m1 - ms1);
-  st.m0 = mn0;
-  st.m1 = mn1;
-  st.l0 *= al0;
-  st.l1 *= al1;
+  if (__any_sync(kFull, mn0 != st.m0 || mn1 != st.m1)) {
+    const float al0 = exp2f(st.m0 - ms0), al1 = exp2f(st.m1 - ms1);
+    st.m0 = mn0;
+    st.m1 = mn1;
+    st.l0 *= al0;
+    st.l1 *= al1;
 #pragma unroll
-  for (int u = 0; u < 8; ++u) {
-    st.o[u][0] *= al0;
-    st.o[u][1] *= al1;
-    st.o[u][2] *= al0;
-    st.o[u][3] *= al1;
+    for (int u = 0; u < 8; ++u) {
+      st.o[u][0] *= al0;
+      st.o[u][1] *= al1;
+      st.o[u][2] *= al0;
+      st.o[u][3] *= al1;
+    }
+    st.zc[0] *= al0;
+    st.zc[1] *= al1;
   }
 #pragma unroll
   for (int t = 0; t < NT; ++t) {
@@ -214,11 +231,8 @@ __device__ __forceinline__ void make_p_bf16(const float (&S)[4], uint32_t (&pf)[
 }
 
 // ---- item cursor ---------------------------------------------------------------------------
-enum StepKind : int { kRowsK = 0, kRowsV = 1, kQ8K = 2, kQ8V = 3, kQ4 = 4, kQ2 = 5 };
-enum RowSrc : int { kSrcBlock = 0, kSrcCentroid = 1, kSrcResidual = 2 };
-
 struct Cursor {
-  int item;          // full mode: item index; sparse mode: position in the warp's page range
+  int item;          // dense: item index; sparse: position in the warp's slice of the page list
   int sub;           // step inside the item
   int nsub;          // steps of the item
   int adv;           // items consumed when the item is done (centroid runs consume several)
@@ -233,18 +247,37 @@ struct WarpCtx {
   const DecodeParams* p;
   const TableEntry* table;   // this stream's table
   int lane;
-  int item_end;              // full mode: one past the last item; sparse: one past the last page position
+  int item_end;              // dense: one past the last item; sparse: one past the last page position
   int stream;
-  bool sparse, has_tail;
-  int page_lo;               // sparse: first page position
+  bool has_tail;
   uint32_t stage[kStages];   // shared-memory addresses of the stages
   const uint8_t* stage_ptr[kStages];
+  uint32_t bar[kStages];
+  // prefetched window of table entries (dense mode): lane i holds entry win_base + i
+  uint4 win;
+  int win_base;
 };
 
 __device__ __forceinline__ int popc4(int m) { return __popc(m & 15); }
 
-// Set up cursor fields for item index `it` (full mode).  Returns false when past the end.
-__device__ __forceinline__ bool load_item_full(const WarpCtx& w, int it, Cursor& c) {
+__device__ __forceinline__ TableEntry window_entry(WarpCtx& w, int item) {
+  const int last = w.p->n_closed;            // the tail entry is the last valid one
+  if (item < w.win_base || item >= w.win_base + 32) {
+    w.win_base = item;
+    const int idx = min(item + w.lane, last);
+    w.win = *reinterpret_cast<const uint4*>(w.table + idx);
+  }
+  const int src = item - w.win_base;
+  TableEntry e;
+  e.off256 = __shfl_sync(kFull, w.win.x, src);
+  e.level = __shfl_sync(kFull, w.win.y, src);
+  const uint32_t lo = __shfl_sync(kFull, w.win.z, src), hi = __shfl_sync(kFull, w.win.w, src);
+  e.resmask = (static_cast<uint64_t>(hi) << 32) | lo;
+  return e;
+}
+
+// Dense mode: set up the cursor for item index `it`.  Returns false when past the end.
+__device__ __forceinline__ bool load_item_dense(WarpCtx& w, int it, Cursor& c) {
   const DecodeParams& p = *w.p;
   while (true) {
     if (it >= w.item_end) return false;
@@ -252,7 +285,7 @@ __device__ __forceinline__ bool load_item_full(const WarpCtx& w, int it, Cursor&
     c.sub = 0;
     c.adv = 1;
     if (it <= p.n_closed) {
-      const TableEntry e = w.table[it];
+      const TableEntry e = window_entry(w, it);
       c.off256 = e.off256;
       c.resmask = e.resmask;
       c.level = static_cast<int>(e.level);
@@ -263,7 +296,10 @@ __device__ __forceinline__ bool load_item_full(const WarpCtx& w, int it, Cursor&
         c.ntok = p.n_tail;
         const int nt = (p.n_tail + 15) >> 4;
         c.tmask = (1 << nt) - 1;
-        if (nt == 0) { ++it; continue; }
+        if (nt == 0) {
+          ++it;
+          continue;
+        }
       }
       switch (c.level) {
         case 16: c.nsub = 2 * popc4(c.tmask); break;
@@ -271,9 +307,10 @@ __device__ __forceinline__ bool load_item_full(const WarpCtx& w, int it, Cursor&
         case 4: c.nsub = 2; break;
         case 2: c.nsub = 1; break;
         default: {   // centroid run: up to 16 consecutive centroid blocks inside this warp's range
-          int run = 1;
           const int lim = min(min(w.item_end, p.n_closed) - it, 16);
-          while (run < lim && w.table[it + run].level == 1u) ++run;
+          const bool is_c = (w.lane < lim) && (w.table[it + w.lane].level == 1u);
+          const unsigned m = __ballot_sync(kFull, is_c);
+          const int run = __ffs(~m) - 1;      // consecutive centroid blocks starting at `it`
           c.adv = run;
           c.ntok = run;
           c.nsub = 2;
@@ -291,7 +328,7 @@ __device__ __forceinline__ bool load_item_full(const WarpCtx& w, int it, Cursor&
     c.ntok = rows;
     c.nsub = 2;
     c.tmask = 1;
-    c.off256 = p.res_off256[w.stream] + 2u * 16u * static_cast<uint32_t>(j);   // 512 B per row = 2 units
+    c.off256 = p.res_off256[w.stream] + 32u * static_cast<uint32_t>(j);   // 16 rows x 512 B = 32 units
     c.resmask = 0;
     return true;
   }
@@ -299,7 +336,7 @@ __device__ __forceinline__ bool load_item_full(const WarpCtx& w, int it, Cursor&
 
 // Sparse mode: position `pos` in the warp's slice of the ascending page list; pages that fall in
 // the same block are merged into one visit.  Position item_end stands for the tail block.
-__device__ __forceinline__ bool load_item_sparse(const WarpCtx& w, int pos, Cursor& c) {
+__device__ __forceinline__ bool load_item_sparse(WarpCtx& w, int pos, Cursor& c) {
   const DecodeParams& p = *w.p;
   const int tiles_per_page = p.page_tokens >> 4;
   const int pages_per_block = kBlock / p.page_tokens;
@@ -350,12 +387,15 @@ __device__ __forceinline__ bool load_item_sparse(const WarpCtx& w, int pos, Curs
   return false;
 }
 
-__device__ __forceinline__ bool load_item(const WarpCtx& w, int it, Cursor& c) {
-  return w.sparse ? load_item_sparse(w, it, c) : load_item_full(w, it, c);
+template <bool SPARSE>
+__device__ __forceinline__ bool load_item(WarpCtx& w, int it, Cursor& c) {
+  if constexpr (SPARSE) return load_item_sparse(w, it, c);
+  else return load_item_dense(w, it, c);
 }
-__device__ __forceinline__ bool advance(const WarpCtx& w, Cursor& c) {
+template <bool SPARSE>
+__device__ __forceinline__ bool advance(WarpCtx& w, Cursor& c) {
   if (++c.sub < c.nsub) return true;
-  return load_item(w, c.item + c.adv, c);
+  return load_item<SPARSE>(w, c.item + c.adv, c);
 }
 
 // k-th set bit (0-based) of a 4-bit mask
@@ -370,84 +410,74 @@ __device__ __forceinline__ int nth_set_bit(int mask, int k) {
   }
   return idx;
 }
-// For quantised levels in sparse mode: which half does step `sub` address (levels 8 and 4)?
+// idx-th half that has an active tile (levels 8 and 4, sparse visits)
 __device__ __forceinline__ int half_of_step(const Cursor& c, int idx) {
-  // idx-th active half
   const bool h0 = (c.tmask & 3) != 0;
   return (idx == 0) ? (h0 ? 0 : 1) : 1;
 }
 
-// Contiguous copy of `bytes` (multiple of 512) from global to a stage offset.
-__device__ __forceinline__ void copy_span(uint32_t sdst, const uint8_t* gsrc, int bytes, int lane) {
-  for (int o = lane * 16; o < bytes; o += 512) cp_async16(sdst + o, gsrc + o, 16);
-}
-
-// Issue the loads of the cursor's current step into stage `sidx`.
+// Issue the TMA bulk copies of the cursor's current step into stage `sidx`.  The warp must have
+// finished reading that stage (callers __syncwarp() before).
+template <bool SPARSE>
 __device__ __forceinline__ void issue_step(const WarpCtx& w, const Cursor& c, int sidx) {
   const DecodeParams& p = *w.p;
-  const uint32_t sdst = w.stage[sidx];
+  const uint32_t sdst = w.stage[sidx], bar = w.bar[sidx];
   const int lane = w.lane;
   if (c.level == 16 || c.level == 1 || c.level == 17) {
-    // 16 rows of 256 B, row r chunk q stored at r*256 + ((q ^ (r & 7)) << 4)
+    // up to 16 rows of 256 B, staged at a 272-byte pitch; one bulk copy per row
     const bool is_v = (c.sub & 1) != 0;
-    const uint8_t* base;
-    size_t row_stride;
-    int row0 = 0, nrows;
+    const uint8_t* src = nullptr;
+    int nrows;
     if (c.level == 16) {
       const int tile = nth_set_bit(c.tmask, c.sub >> 1);
-      base = p.arena + static_cast<size_t>(c.off256) * 256 + (is_v ? kBlock * kRowBytes : 0);
-      row_stride = kRowBytes;
-      row0 = tile * 16;
-      nrows = min(16, c.ntok - row0);
+      nrows = min(16, c.ntok - tile * 16);
+      src = p.arena + static_cast<size_t>(c.off256) * 256 + (is_v ? kBlock * kRowBytes : 0) +
+            static_cast<size_t>(tile * 16 + lane) * kRowBytes;
     } else if (c.level == 17) {
-      base = p.arena + static_cast<size_t>(c.off256) * 256 + (is_v ? kRowBytes : 0);
-      row_stride = 2 * kRowBytes;
       nrows = c.ntok;
+      src = p.arena + static_cast<size_t>(c.off256) * 256 + (is_v ? kRowBytes : 0) +
+            static_cast<size_t>(lane) * 2 * kRowBytes;
     } else {
-      base = nullptr;   // centroid rows live in separate slots
-      row_stride = 0;
       nrows = c.ntok;
-    }
-    // per-row source pointer for centroid runs: lane r < nrows looks up block (item + r)
-    const uint8_t* myrow = p.arena;
-    if (c.level == 1) {
       if (lane < nrows) {
-        const int blk = w.sparse ? (p.page_idx[static_cast<size_t>(w.stream) * p.n_sel + c.item] /
-                                    (kBlock / p.page_tokens))
-                                 : (c.item + lane);
-        myrow = p.arena + static_cast<size_t>(w.table[blk].off256) * 256 + (is_v ? kRowBytes : 0);
+        int blk;
+        if constexpr (SPARSE) blk = p.page_idx[static_cast<size_t>(w.stream) * p.n_sel + c.item] / (kBlock / p.page_tokens);
+        else blk = c.item + lane;
+        src = p.arena + static_cast<size_t>(w.table[blk].off256) * 256 + (is_v ? kRowBytes : 0);
       }
     }
+    if (lane == 0) mbar_expect_tx(bar, static_cast<uint32_t>(nrows) * kRowBytes);
+    __syncwarp();
+    if (lane < nrows) {
+      bulk_g2s(sdst + lane * kRowPitch, src, kRowBytes, bar);
+    } else if (lane < 16) {
+      // rows past the end are zero so that 0 * garbage never produces a NaN
+      uint4* z = reinterpret_cast<uint4*>(const_cast<uint8_t*>(w.stage_ptr[sidx]) + lane * kRowPitch);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int row = 2 * j + (lane >> 4), q = lane & 15;
-      const uint8_t* src;
-      if (c.level == 1) {
-        const unsigned long long ptr = __shfl_sync(kFull, reinterpret_cast<unsigned long long>(myrow), row);
-        src = reinterpret_cast<const uint8_t*>(ptr);
-      } else {
-        src = base + static_cast<size_t>(row0 + row) * row_stride;
-      }
-      const bool valid = row < nrows;
-      cp_async16(sdst + row * 256 + ((q ^ (row & 7)) << 4), valid ? (src + q * 16) : p.arena, valid ? 16 : 0);
+      for (int i = 0; i < kRowBytes / 16; ++i) z[i] = make_uint4(0, 0, 0, 0);
     }
     return;
   }
+  if (lane != 0) return;
   const int bits = c.level;
   const int cb = code_bytes_per_tile(bits);
   const uint8_t* slot = p.arena + static_cast<size_t>(c.off256) * 256;
-  if (c.tmask == 15) {
+  if (!SPARSE || c.tmask == 15) {
     // full block: every step is one contiguous span of the slot
+    const uint8_t* src;
+    uint32_t bytes;
     if (bits == 8) {
-      const int half = c.sub >> 1;
-      const uint8_t* hb = slot + half * half_bytes(8);
-      if ((c.sub & 1) == 0) copy_span(sdst, hb, 512 + 2 * cb, lane);
-      else copy_span(sdst, hb + 512 + 2 * cb, 512 + 2 * cb, lane);
+      bytes = 512 + 2 * cb;
+      src = slot + (c.sub >> 1) * half_bytes(8) + (c.sub & 1) * bytes;
     } else if (bits == 4) {
-      copy_span(sdst, slot + c.sub * half_bytes(4), half_bytes(4), lane);
+      bytes = half_bytes(4);
+      src = slot + c.sub * bytes;
     } else {
-      copy_span(sdst, slot, 2 * half_bytes(2), lane);
+      bytes = 2 * half_bytes(2);
+      src = slot;
     }
+    mbar_expect_tx(bar, bytes);
+    bulk_g2s(sdst, src, bytes, bar);
     return;
   }
   // sparse visit: copy only the pieces of the selected tiles (same stage offsets as a full copy)
@@ -455,130 +485,222 @@ __device__ __forceinline__ void issue_step(const WarpCtx& w, const Cursor& c, in
     const int half = half_of_step(c, c.sub >> 1);
     const int tm = (c.tmask >> (2 * half)) & 3;
     const uint8_t* hb = slot + half * half_bytes(8);
+    const int nt = popc4(tm);
     if ((c.sub & 1) == 0) {
-      copy_span(sdst, hb, 512, lane);
+      mbar_expect_tx(bar, 512 + nt * cb);
+      bulk_g2s(sdst, hb, 512, bar);
       for (int t = 0; t < 2; ++t)
-        if (tm & (1 << t)) copy_span(sdst + 512 + t * cb, hb + off_kc(8, t), cb, lane);
+        if (tm & (1 << t)) bulk_g2s(sdst + 512 + t * cb, hb + off_kc(8, t), cb, bar);
     } else {
-      const int vbase = 512 + 2 * cb;
+      mbar_expect_tx(bar, nt * (256 + cb));
       for (int t = 0; t < 2; ++t)
         if (tm & (1 << t)) {
-          if (lane < 16) cp_async16(sdst + t * 256 + lane * 16, hb + off_vp(8, t) + lane * 16, 16);
-          copy_span(sdst + 512 + t * cb, hb + off_vc(8, t), cb, lane);
+          bulk_g2s(sdst + t * 256, hb + off_vp(8, t), 256, bar);
+          bulk_g2s(sdst + 512 + t * cb, hb + off_vc(8, t), cb, bar);
         }
-      (void)vbase;
     }
   } else {
     const int nh = (bits == 4) ? 1 : 2;
+    uint32_t total = 0;
+    for (int hh = 0; hh < nh; ++hh) {
+      const int half = (bits == 4) ? half_of_step(c, c.sub) : hh;
+      const int tm = (c.tmask >> (2 * half)) & 3;
+      if (tm) total += 512 + popc4(tm) * (2 * cb + 256);
+    }
+    mbar_expect_tx(bar, total);
     for (int hh = 0; hh < nh; ++hh) {
       const int half = (bits == 4) ? half_of_step(c, c.sub) : hh;
       const int tm = (c.tmask >> (2 * half)) & 3;
       if (tm == 0) continue;
       const uint8_t* hb = slot + half * half_bytes(bits);
       const uint32_t sd = sdst + ((bits == 4) ? 0 : hh * half_bytes(2));
-      copy_span(sd, hb, 512, lane);
+      bulk_g2s(sd, hb, 512, bar);
       for (int t = 0; t < 2; ++t)
         if (tm & (1 << t)) {
-          copy_span(sd + off_kc(bits, t), hb + off_kc(bits, t), cb, lane);
-          if (lane < 16) cp_async16(sd + off_vp(bits, t) + lane * 16, hb + off_vp(bits, t) + lane * 16, 16);
-          copy_span(sd + off_vc(bits, t), hb + off_vc(bits, t), cb, lane);
+          bulk_g2s(sd + off_kc(bits, t), hb + off_kc(bits, t), cb, bar);
+          bulk_g2s(sd + off_vp(bits, t), hb + off_vp(bits, t), 256, bar);
+          bulk_g2s(sd + off_vc(bits, t), hb + off_vc(bits, t), cb, bar);
         }
     }
   }
 }
 
 // ---- compute ---------------------------------------------------------------------------------
-// QK^T of the active tiles of one half from staged key params + codes.
-template <int BITS>
+// Logits of the active tiles of one half (32 tokens): S = scale * (q . k~) + token bias, with
+// k~ = s * code + z.  Data MMAs use A = bias + code and B = q' = q * s; the bias is removed with a
+// "ones" MMA on the same q' and the zero points enter through an MMA with A = z and B = q.
+template <int BITS, bool FULL>
 __device__ __forceinline__ void qk_half(const uint8_t* kp, const uint8_t* kc0, const uint8_t* kc1, int tm,
-                                        const uint32_t (&qh)[16], int lane, float (&S)[2][4]) {
-  const int c4 = lane & 3;
-  TileCodes<BITS> t0, t1;
-  if (tm & 1) t0.load(kc0, lane);
-  if (tm & 2) t1.load(kc1, lane);
+                                        const uint32_t (&qh)[16], int lane, float scale_log2, uint64_t resmask,
+                                        int half, float (&S)[2][4]) {
+  const int c4 = lane & 3, r = lane >> 2;
+  constexpr int kWords = 2 * BITS;               // words per lane and tile
+  uint32_t w0[kWords], w1[kWords];
+  if (FULL || (tm & 1)) {
+#pragma unroll
+    for (int j = 0; j < kWords / 4; ++j) {
+      const uint4 v = *reinterpret_cast<const uint4*>(kc0 + (j * 32 + lane) * 16);
+      w0[4 * j] = v.x; w0[4 * j + 1] = v.y; w0[4 * j + 2] = v.z; w0[4 * j + 3] = v.w;
+    }
+  }
+  if (FULL || (tm & 2)) {
+#pragma unroll
+    for (int j = 0; j < kWords / 4; ++j) {
+      const uint4 v = *reinterpret_cast<const uint4*>(kc1 + (j * 32 + lane) * 16);
+      w1[4 * j] = v.x; w1[4 * j + 1] = v.y; w1[4 * j + 2] = v.z; w1[4 * j + 3] = v.w;
+    }
+  }
+  float zd[4] = {0.f, 0.f, 0.f, 0.f};        // rows r: sum_c q_c z_c; rows r + 8: sum_c q_c s_c (exact products)
+  float qe[4] = {0.f, 0.f, 0.f, 0.f};        // sum_c q'_c over even MMA indices (all rows equal)
+  float qo[4] = {0.f, 0.f, 0.f, 0.f};        // ... over odd MMA indices (2-bit only)
+#pragma unroll
+  for (int t = 0; t < 2; ++t) S[t][0] = S[t][1] = S[t][2] = S[t][3] = 0.f;
 #pragma unroll
   for (int s = 0; s < 8; ++s) {
-    const uint4 pr = *reinterpret_cast<const uint4*>(kp + (s * 4 + c4) * 16);
-    const __half2 scA = u32_as_h2(pr.x), zrA = u32_as_h2(pr.y), scB = u32_as_h2(pr.z), zrB = u32_as_h2(pr.w);
+    const uint4 pr = *reinterpret_cast<const uint4*>(kp + (s * 4 + c4) * 16);   // s01, z01, s23, z23
+    const uint32_t q0 = hmul2_u32(qh[2 * s], pr.x), q1 = hmul2_u32(qh[2 * s + 1], pr.z);
+    mma_f16(zd, pr.y, pr.x, pr.w, pr.z, qh[2 * s], qh[2 * s + 1]);
+    if (BITS == 2 && (s & 1)) mma_f16(qo, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
+    else mma_f16(qe, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
     uint32_t a[4];
-    if (tm & 1) {
-      if constexpr (BITS == 8) unpack_dequant<8>(t0.word(2 * s), t0.word(2 * s + 1), false, scA, zrA, scB, zrB, a);
-      else if constexpr (BITS == 4) unpack_dequant<4>(t0.word(s), 0u, false, scA, zrA, scB, zrB, a);
-      else unpack_dequant<2>(t0.word(s >> 1), 0u, (s & 1) != 0, scA, zrA, scB, zrB, a);
-      mma_f16(S[0], a, qh[2 * s], qh[2 * s + 1]);
+    if (FULL || (tm & 1)) {
+      unpack<BITS>(w0, s, a);
+      mma_f16(S[0], a[0], a[1], a[2], a[3], q0, q1);
     }
-    if (tm & 2) {
-      if constexpr (BITS == 8) unpack_dequant<8>(t1.word(2 * s), t1.word(2 * s + 1), false, scA, zrA, scB, zrB, a);
-      else if constexpr (BITS == 4) unpack_dequant<4>(t1.word(s), 0u, false, scA, zrA, scB, zrB, a);
-      else unpack_dequant<2>(t1.word(s >> 1), 0u, (s & 1) != 0, scA, zrA, scB, zrB, a);
-      mma_f16(S[1], a, qh[2 * s], qh[2 * s + 1]);
+    if (FULL || (tm & 2)) {
+      unpack<BITS>(w1, s, a);
+      mma_f16(S[1], a[0], a[1], a[2], a[3], q0, q1);
     }
   }
-}
-
-// O^T += V^T P^T for the active tiles of one half from staged value params + codes.
-template <int BITS>
-__device__ __forceinline__ void pv_half(const uint8_t* vp0, const uint8_t* vp1, const uint8_t* vc0,
-                                        const uint8_t* vc1, int tm, const uint32_t (&pf)[2][2], int lane,
-                                        SoftmaxState& st) {
-  const int c4 = lane & 3;
-  TileCodes<BITS> t0, t1;
-  if (tm & 1) t0.load(vc0, lane);
-  if (tm & 2) t1.load(vc1, lane);
-#pragma unroll
-  for (int grp = 0; grp < 4; ++grp) {
-    uint4 pr0 = make_uint4(0, 0, 0, 0), pr1 = make_uint4(0, 0, 0, 0);
-    if (tm & 1) pr0 = *reinterpret_cast<const uint4*>(vp0 + (grp * 4 + c4) * 16);
-    if (tm & 2) pr1 = *reinterpret_cast<const uint4*>(vp1 + (grp * 4 + c4) * 16);
-#pragma unroll
-    for (int uu = 0; uu < 2; ++uu) {
-      const int u = 2 * grp + uu;
-      uint32_t a[4];
-      if (tm & 1) {
-        const __half2 scA = u32_as_h2(pr0.x), zrA = u32_as_h2(pr0.y), scB = u32_as_h2(pr0.z), zrB = u32_as_h2(pr0.w);
-        if constexpr (BITS == 8) unpack_dequant<8>(t0.word(2 * u), t0.word(2 * u + 1), false, scA, zrA, scB, zrB, a);
-        else if constexpr (BITS == 4) unpack_dequant<4>(t0.word(u), 0u, false, scA, zrA, scB, zrB, a);
-        else unpack_dequant<2>(t0.word(u >> 1), 0u, (u & 1) != 0, scA, zrA, scB, zrB, a);
-        mma_f16(st.o[u], a, pf[0][0], pf[0][1]);
-      }
-      if (tm & 2) {
-        const __half2 scA = u32_as_h2(pr1.x), zrA = u32_as_h2(pr1.y), scB = u32_as_h2(pr1.z), zrB = u32_as_h2(pr1.w);
-        if constexpr (BITS == 8) unpack_dequant<8>(t1.word(2 * u), t1.word(2 * u + 1), false, scA, zrA, scB, zrB, a);
-        else if constexpr (BITS == 4) unpack_dequant<4>(t1.word(u), 0u, false, scA, zrA, scB, zrB, a);
-        else unpack_dequant<2>(t1.word(u >> 1), 0u, (u & 1) != 0, scA, zrA, scB, zrB, a);
-        mma_f16(st.o[u], a, pf[1][0], pf[1][1]);
-      }
-    }
-  }
-}
-
-// Token validity bias of a half for the lane's rows: tokens 32*half + 16*t + r (+8).
-__device__ __forceinline__ void half_bias(uint64_t resmask, int half, int tm, int lane, float (&bias)[2][2]) {
-  const int r = lane >> 2;
+  // rows r carry bias lo, rows r + 8 carry bias hi (per parity of the MMA index)
+  constexpr float kMid = Bias<BITS>::mid;
+  const float z0 = fmaf(kMid, zd[2], zd[0]), z1 = fmaf(kMid, zd[3], zd[1]);     // sum q (z + mid s)
+  const float c_lo0 = z0 - (Bias<BITS>::lo_even + kMid) * qe[0] - (Bias<BITS>::lo_odd + kMid) * qo[0];
+  const float c_lo1 = z1 - (Bias<BITS>::lo_even + kMid) * qe[1] - (Bias<BITS>::lo_odd + kMid) * qo[1];
+  const float c_hi0 = z0 - (Bias<BITS>::hi_even + kMid) * qe[0] - (Bias<BITS>::hi_odd + kMid) * qo[0];
+  const float c_hi1 = z1 - (Bias<BITS>::hi_even + kMid) * qe[1] - (Bias<BITS>::hi_odd + kMid) * qo[1];
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
     const int tok = 32 * half + 16 * t + r;
-    const bool on = (tm >> t) & 1;
-    bias[t][0] = (on && !((resmask >> tok) & 1ull)) ? 0.f : kNegInf;
-    bias[t][1] = (on && !((resmask >> (tok + 8)) & 1ull)) ? 0.f : kNegInf;
+    const bool on = FULL || ((tm >> t) & 1);
+    const float b_lo = (on && !((resmask >> tok) & 1ull)) ? 0.f : kNegInf;
+    const float b_hi = (on && !((resmask >> (tok + 8)) & 1ull)) ? 0.f : kNegInf;
+    S[t][0] = fmaf(S[t][0] + c_lo0, scale_log2, b_lo);
+    S[t][1] = fmaf(S[t][1] + c_lo1, scale_log2, b_lo);
+    S[t][2] = fmaf(S[t][2] + c_hi0, scale_log2, b_hi);
+    S[t][3] = fmaf(S[t][3] + c_hi1, scale_log2, b_hi);
   }
 }
 
-template <int BITS>
+// O^T += V~^T P^T for the active tiles of one half, v~ = s * code + z per (token, 32-channel group).
+// pf holds the raw fp16 P^T fragments of the two tiles.
+template <int BITS, bool FULL>
+__device__ __forceinline__ void pv_half(const uint8_t* vp0, const uint8_t* vp1, const uint8_t* vc0,
+                                        const uint8_t* vc1, int tm, const uint32_t (&pf)[2][2], int lane,
+                                        SoftmaxState& st) {
+  const int c4 = lane & 3, r = lane >> 2;
+  constexpr int kWordsPerGrp = BITS / 2;          // words of a lane covering MMA indices 2g, 2g+1
+  // per-lane scales of its token pairs, all four groups: {sA, sB} x 4 per tile
+  uint32_t sc0[8], sc1[8];
+  float tz[4] = {0.f, 0.f, 0.f, 0.f};
+  if (FULL || (tm & 1)) {
+    const uint4 x = *reinterpret_cast<const uint4*>(vp0 + c4 * 32), y = *reinterpret_cast<const uint4*>(vp0 + c4 * 32 + 16);
+    sc0[0] = x.x; sc0[1] = x.y; sc0[2] = x.z; sc0[3] = x.w; sc0[4] = y.x; sc0[5] = y.y; sc0[6] = y.z; sc0[7] = y.w;
+    // rows g < 4: sum_tok p z[tok][g]; rows 8 + g: sum_tok p s[tok][g] (exact products)
+    uint2 z = make_uint2(0, 0), sg = make_uint2(0, 0);
+    if (r < 4) {
+      z = *reinterpret_cast<const uint2*>(vp0 + 128 + (r * 4 + c4) * 8);
+      sg = make_uint2(sc0[0], sc0[1]);
+      if (r == 1) sg = make_uint2(sc0[2], sc0[3]);
+      if (r == 2) sg = make_uint2(sc0[4], sc0[5]);
+      if (r == 3) sg = make_uint2(sc0[6], sc0[7]);
+    }
+    mma_f16(tz, z.x, sg.x, z.y, sg.y, pf[0][0], pf[0][1]);
+  }
+  if (FULL || (tm & 2)) {
+    const uint4 x = *reinterpret_cast<const uint4*>(vp1 + c4 * 32), y = *reinterpret_cast<const uint4*>(vp1 + c4 * 32 + 16);
+    sc1[0] = x.x; sc1[1] = x.y; sc1[2] = x.z; sc1[3] = x.w; sc1[4] = y.x; sc1[5] = y.y; sc1[6] = y.z; sc1[7] = y.w;
+    uint2 z = make_uint2(0, 0), sg = make_uint2(0, 0);
+    if (r < 4) {
+      z = *reinterpret_cast<const uint2*>(vp1 + 128 + (r * 4 + c4) * 8);
+      sg = make_uint2(sc1[0], sc1[1]);
+      if (r == 1) sg = make_uint2(sc1[2], sc1[3]);
+      if (r == 2) sg = make_uint2(sc1[4], sc1[5]);
+      if (r == 3) sg = make_uint2(sc1[6], sc1[7]);
+    }
+    mma_f16(tz, z.x, sg.x, z.y, sg.y, pf[1][0], pf[1][1]);
+  }
+  st.zc[0] += fmaf(Bias<BITS>::mid, tz[2], tz[0]);
+  st.zc[1] += fmaf(Bias<BITS>::mid, tz[3], tz[1]);
+#pragma unroll
+  for (int grp = 0; grp < 4; ++grp) {
+    float ps[4] = {0.f, 0.f, 0.f, 0.f};          // sum over tokens of P' (all rows equal)
+    float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};   // this step's O for u = 2g, 2g+1
+    uint32_t wd[kWordsPerGrp];
+    uint32_t a[4];
+    if (FULL || (tm & 1)) {
+      const uint32_t p0 = hmul2_u32(pf[0][0], sc0[2 * grp]), p1 = hmul2_u32(pf[0][1], sc0[2 * grp + 1]);
+      mma_f16(ps, kOnesH2, kOnesH2, kOnesH2, kOnesH2, p0, p1);
+      // words of MMA indices 2 grp and 2 grp + 1: 8-bit words 4g..4g+3, 4-bit 2g..2g+1, 2-bit g
+      const uint8_t* base = vc0 + ((grp * kWordsPerGrp >> 2) * 32 + lane) * 16 + ((grp * kWordsPerGrp) & 3) * 4;
+      if constexpr (BITS == 8) {
+        const uint4 v = *reinterpret_cast<const uint4*>(base);
+        wd[0] = v.x; wd[1] = v.y; wd[2] = v.z; wd[3] = v.w;
+      } else if constexpr (BITS == 4) {
+        const uint2 v = *reinterpret_cast<const uint2*>(base);
+        wd[0] = v.x; wd[1] = v.y;
+      } else {
+        wd[0] = *reinterpret_cast<const uint32_t*>(base);
+      }
+      unpack<BITS>(wd, 0, a);
+      mma_f16(acc0, a[0], a[1], a[2], a[3], p0, p1);
+      unpack<BITS>(wd, 1, a);
+      mma_f16(acc1, a[0], a[1], a[2], a[3], p0, p1);
+    }
+    if (FULL || (tm & 2)) {
+      const uint32_t p0 = hmul2_u32(pf[1][0], sc1[2 * grp]), p1 = hmul2_u32(pf[1][1], sc1[2 * grp + 1]);
+      mma_f16(ps, kOnesH2, kOnesH2, kOnesH2, kOnesH2, p0, p1);
+      const uint8_t* base = vc1 + ((grp * kWordsPerGrp >> 2) * 32 + lane) * 16 + ((grp * kWordsPerGrp) & 3) * 4;
+      if constexpr (BITS == 8) {
+        const uint4 v = *reinterpret_cast<const uint4*>(base);
+        wd[0] = v.x; wd[1] = v.y; wd[2] = v.z; wd[3] = v.w;
+      } else if constexpr (BITS == 4) {
+        const uint2 v = *reinterpret_cast<const uint2*>(base);
+        wd[0] = v.x; wd[1] = v.y;
+      } else {
+        wd[0] = *reinterpret_cast<const uint32_t*>(base);
+      }
+      unpack<BITS>(wd, 0, a);
+      mma_f16(acc0, a[0], a[1], a[2], a[3], p0, p1);
+      unpack<BITS>(wd, 1, a);
+      mma_f16(acc1, a[0], a[1], a[2], a[3], p0, p1);
+    }
+    // remove the biases: u = 2g is an even MMA index, u = 2g + 1 an odd one
+    st.o[2 * grp][0] += acc0[0] - (Bias<BITS>::lo_even + Bias<BITS>::mid) * ps[0];
+    st.o[2 * grp][1] += acc0[1] - (Bias<BITS>::lo_even + Bias<BITS>::mid) * ps[1];
+    st.o[2 * grp][2] += acc0[2] - (Bias<BITS>::hi_even + Bias<BITS>::mid) * ps[0];
+    st.o[2 * grp][3] += acc0[3] - (Bias<BITS>::hi_even + Bias<BITS>::mid) * ps[1];
+    st.o[2 * grp + 1][0] += acc1[0] - (Bias<BITS>::lo_odd + Bias<BITS>::mid) * ps[0];
+    st.o[2 * grp + 1][1] += acc1[1] - (Bias<BITS>::lo_odd + Bias<BITS>::mid) * ps[1];
+    st.o[2 * grp + 1][2] += acc1[2] - (Bias<BITS>::hi_odd + Bias<BITS>::mid) * ps[0];
+    st.o[2 * grp + 1][3] += acc1[3] - (Bias<BITS>::hi_odd + Bias<BITS>::mid) * ps[1];
+  }
+}
+
+template <int BITS, bool FULL>
 __device__ __forceinline__ void qk_softmax_half(const uint8_t* half_k, int half, int tm, uint64_t resmask,
                                                 const uint32_t (&qh)[16], int lane, float scale_log2,
                                                 SoftmaxState& st, uint32_t (&pf)[2][2]) {
   constexpr int cb = 256 * BITS;
-  float S[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-  qk_half<BITS>(half_k, half_k + 512, half_k + 512 + cb, tm, qh, lane, S);
-  float bias[2][2];
-  half_bias(resmask, half, tm, lane, bias);
-  softmax_update<2>(S, bias, scale_log2, st);
+  float S[2][4];
+  qk_half<BITS, FULL>(half_k, half_k + 512, half_k + 512 + cb, tm, qh, lane, scale_log2, resmask, half, S);
+  softmax_update<2>(S, st);
   make_p_f16(S[0], pf[0], st);
   make_p_f16(S[1], pf[1], st);
 }
 
 // Process a staged step.  pf carries P fragments from a key step to the following value step.
+template <bool SPARSE>
 __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, int sidx, const uint32_t (&qb)[16],
                                              const uint32_t (&qh)[16], SoftmaxState& st, uint32_t (&pf)[4]) {
   const DecodeParams& p = *w.p;
@@ -590,48 +712,50 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
       // key rows: S^T = K Q^T
       float S[1][4] = {{0.f, 0.f, 0.f, 0.f}};
       const int mi = lane >> 3;
-      const int row = (lane & 7) + (mi & 1) * 8;
+      const uint32_t base = sa + ((lane & 7) + (mi & 1) * 8) * kRowPitch + (mi >> 1) * 16;
 #pragma unroll
       for (int s = 0; s < 8; ++s) {
         uint32_t a[4];
-        const int q = 2 * s + (mi >> 1);
-        ldmatrix_x4(a, sa + row * 256 + ((q ^ (row & 7)) << 4));
+        ldmatrix_x4(a, base + s * 32);
         mma_bf16(S[0], a, qb[2 * s], qb[2 * s + 1]);
       }
       // validity / weight of the lane's rows r and r + 8
       const int r = lane >> 2;
-      float bias[1][2];
+      float b_lo, b_hi;
       if (c.level == 16) {
         const int tile = nth_set_bit(c.tmask, c.sub >> 1);
         const int t0 = tile * 16 + r;
-        bias[0][0] = (t0 < c.ntok && !((c.resmask >> t0) & 1ull)) ? 0.f : kNegInf;
-        bias[0][1] = (t0 + 8 < c.ntok && !((c.resmask >> (t0 + 8)) & 1ull)) ? 0.f : kNegInf;
+        b_lo = (t0 < c.ntok && !((c.resmask >> t0) & 1ull)) ? 0.f : kNegInf;
+        b_hi = (t0 + 8 < c.ntok && !((c.resmask >> (t0 + 8)) & 1ull)) ? 0.f : kNegInf;
       } else if (c.level == 17) {
-        bias[0][0] = (r < c.ntok) ? 0.f : kNegInf;
-        bias[0][1] = (r + 8 < c.ntok) ? 0.f : kNegInf;
+        b_lo = (r < c.ntok) ? 0.f : kNegInf;
+        b_hi = (r + 8 < c.ntok) ? 0.f : kNegInf;
       } else {
         // centroid rows: each stands for the block's readable tokens -> add log2(count)
         float myb = kNegInf;
         if (lane < c.ntok) {
           int cnt;
-          if (w.sparse) cnt = 16 * popc4(c.tmask);
+          if constexpr (SPARSE) cnt = 16 * popc4(c.tmask);
           else cnt = kBlock - __popcll(w.table[c.item + lane].resmask);
           myb = cnt > 0 ? log2f(static_cast<float>(cnt)) : kNegInf;
         }
-        bias[0][0] = __shfl_sync(kFull, myb, r);
-        bias[0][1] = __shfl_sync(kFull, myb, r + 8);
+        b_lo = __shfl_sync(kFull, myb, r);
+        b_hi = __shfl_sync(kFull, myb, r + 8);
       }
-      softmax_update<1>(S, bias, p.scale_log2, st);
+      S[0][0] = fmaf(S[0][0], p.scale_log2, b_lo);
+      S[0][1] = fmaf(S[0][1], p.scale_log2, b_lo);
+      S[0][2] = fmaf(S[0][2], p.scale_log2, b_hi);
+      S[0][3] = fmaf(S[0][3], p.scale_log2, b_hi);
+      softmax_update<1>(S, st);
       make_p_bf16(S[0], pf, st);
     } else {
       // value rows: O^T += V^T P^T with P = hi + lo
       const int mi = lane >> 3;
-      const int row = (lane & 7) + (mi >> 1) * 8;
+      const uint32_t base = sa + ((lane & 7) + (mi >> 1) * 8) * kRowPitch + (mi & 1) * 16;
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         uint32_t a[4];
-        const int q = 2 * u + (mi & 1);
-        ldmatrix_x4_trans(a, sa + row * 256 + ((q ^ (row & 7)) << 4));
+        ldmatrix_x4_trans(a, base + u * 32);
         mma_bf16(st.o[u], a, pf[0], pf[1]);
         mma_bf16(st.o[u], a, pf[2], pf[3]);
       }
@@ -639,31 +763,30 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
     return;
   }
   uint32_t (&pf2)[2][2] = *reinterpret_cast<uint32_t (*)[2][2]>(&pf);
+  constexpr bool FULL = !SPARSE;
   if (c.level == 8) {
-    const int half = (c.tmask == 15) ? (c.sub >> 1) : half_of_step(c, c.sub >> 1);
+    const int half = FULL ? (c.sub >> 1) : ((c.tmask == 15) ? (c.sub >> 1) : half_of_step(c, c.sub >> 1));
     const int tm = (c.tmask >> (2 * half)) & 3;
-    if ((c.sub & 1) == 0) {
-      qk_softmax_half<8>(sp, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
-    } else {
-      pv_half<8>(sp, sp + 256, sp + 512, sp + 512 + 2048, tm, pf2, lane, st);
-    }
+    if ((c.sub & 1) == 0) qk_softmax_half<8, FULL>(sp, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
+    else pv_half<8, FULL>(sp, sp + 256, sp + 512, sp + 512 + 2048, tm, pf2, lane, st);
   } else if (c.level == 4) {
-    const int half = (c.tmask == 15) ? c.sub : half_of_step(c, c.sub);
+    const int half = FULL ? c.sub : ((c.tmask == 15) ? c.sub : half_of_step(c, c.sub));
     const int tm = (c.tmask >> (2 * half)) & 3;
-    qk_softmax_half<4>(sp, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
-    pv_half<4>(sp + off_vp(4, 0), sp + off_vp(4, 1), sp + off_vc(4, 0), sp + off_vc(4, 1), tm, pf2, lane, st);
+    qk_softmax_half<4, FULL>(sp, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
+    pv_half<4, FULL>(sp + off_vp(4, 0), sp + off_vp(4, 1), sp + off_vc(4, 0), sp + off_vc(4, 1), tm, pf2, lane, st);
   } else {
 #pragma unroll 1
     for (int half = 0; half < 2; ++half) {
       const int tm = (c.tmask >> (2 * half)) & 3;
-      if (tm == 0) continue;
+      if (!FULL && tm == 0) continue;
       const uint8_t* hb = sp + half * half_bytes(2);
-      qk_softmax_half<2>(hb, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
-      pv_half<2>(hb + off_vp(2, 0), hb + off_vp(2, 1), hb + off_vc(2, 0), hb + off_vc(2, 1), tm, pf2, lane, st);
+      qk_softmax_half<2, FULL>(hb, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
+      pv_half<2, FULL>(hb + off_vp(2, 0), hb + off_vp(2, 1), hb + off_vc(2, 0), hb + off_vc(2, 1), tm, pf2, lane, st);
     }
   }
 }
 
+template <bool SPARSE>
 __global__ void __launch_bounds__(kDecodeWarps * 32, 2) decode_kernel(const __grid_constant__ DecodeParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -673,9 +796,10 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 2) decode_kernel(const __gr
   WarpCtx w;
   w.p = &p;
   w.lane = lane;
-  w.sparse = p.page_idx != nullptr;
+  w.win_base = -(1 << 30);
+  w.win = make_uint4(0, 0, 0, 0);
   int partial_row, first;
-  if (!w.sparse) {
+  if constexpr (!SPARSE) {
     const WarpDesc wd = p.warps[gw];
     if (wd.stream < 0) return;
     w.stream = wd.stream;
@@ -694,11 +818,19 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 2) decode_kernel(const __gr
   }
   w.table = p.table + static_cast<size_t>(w.stream) * p.table_stride;
   uint8_t* sbase = smem + warp * (kStages * kStageBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kDecodeWarps * kStages * kStageBytes) + warp * kStages;
 #pragma unroll
   for (int s = 0; s < kStages; ++s) {
     w.stage_ptr[s] = sbase + s * kStageBytes;
     w.stage[s] = smem_u32(sbase + s * kStageBytes);
+    w.bar[s] = smem_u32(bars + s);
   }
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) mbar_init(w.bar[s], 1);
+    fence_proxy_async();
+  }
+  __syncwarp();
 
   // Query fragments: B operand Q^T[16 channels x 8 heads]; lane (r, c4) holds head r, channels
   // 16 s + 2 c4 (+1) and 16 s + 8 + 2 c4 (+1), in bf16 (exact rows) and fp16 (quantised tiers).
@@ -727,35 +859,55 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 2) decode_kernel(const __gr
   st.l0 = st.l1 = 0.f;
 #pragma unroll
   for (int u = 0; u < 8; ++u) st.o[u][0] = st.o[u][1] = st.o[u][2] = st.o[u][3] = 0.f;
+  st.zc[0] = st.zc[1] = st.zc[2] = st.zc[3] = 0.f;
   uint32_t pf[4] = {0, 0, 0, 0};
 
   Cursor cur;
-  bool have = load_item(w, first, cur);
+  bool have = load_item<SPARSE>(w, first, cur);
   int sidx = 0;
-  if (have) {
-    issue_step(w, cur, 0);
-    cp_async_commit();
-  }
+  uint32_t phase = 0;             // bit s = parity to wait for on stage s
+  bool failed = false;
+  if (have) issue_step<SPARSE>(w, cur, 0);
   while (have) {
     Cursor nxt = cur;
-    const bool more = advance(w, nxt);
-    if (more) issue_step(w, nxt, sidx ^ 1);
-    cp_async_commit();
-    cp_async_wait<1>();
+    const bool more = advance<SPARSE>(w, nxt);
+    if (more) issue_step<SPARSE>(w, nxt, sidx ^ 1);
+    // bounded wait for this step's bytes
+    int spins = 0;
+    while (!mbar_try_wait(w.bar[sidx], (phase >> sidx) & 1u)) {
+      if (++spins > kWaitSpins) {
+        failed = true;
+        break;
+      }
+    }
+    if (__any_sync(kFull, failed)) break;
+    phase ^= 1u << sidx;
     __syncwarp();
-    compute_step(w, cur, sidx, qb, qh, st, pf);
+    compute_step<SPARSE>(w, cur, sidx, qb, qh, st, pf);
     __syncwarp();
     cur = nxt;
     have = more;
     sidx ^= 1;
   }
-  cp_async_wait<0>();
+  if (failed) {
+    // a copy never completed: flag it and publish an empty partial (the host reports BAD_STATE)
+    if (lane == 0) atomicOr(p.status, kStatusInternal);
+    st.m0 = st.m1 = kNegInf;
+    st.l0 = st.l1 = 0.f;
+  }
 
   // lane-partial sums -> per-head sums (reduce over the 8 r lanes that share c4)
 #pragma unroll
   for (int d = 4; d <= 16; d <<= 1) {
     st.l0 += __shfl_xor_sync(kFull, st.l0, d);
     st.l1 += __shfl_xor_sync(kFull, st.l1, d);
+  }
+  // value zero-point term: row g of zc (lane 4 g + c4) belongs to channels [32 g, 32 g + 32)
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    const float z0 = __shfl_sync(kFull, st.zc[0], 4 * g + c4), z1 = __shfl_sync(kFull, st.zc[1], 4 * g + c4);
+    st.o[2 * g][0] += z0; st.o[2 * g][1] += z1; st.o[2 * g][2] += z0; st.o[2 * g][3] += z1;
+    st.o[2 * g + 1][0] += z0; st.o[2 * g + 1][1] += z1; st.o[2 * g + 1][2] += z0; st.o[2 * g + 1][3] += z1;
   }
   float* out = p.partial + static_cast<size_t>(partial_row) * kPartialFloats;
   const int h0 = 2 * c4, h1 = 2 * c4 + 1;
@@ -808,18 +960,24 @@ __global__ void __launch_bounds__(kD) combine_kernel(const __grid_constant__ Com
 
 }  // namespace
 
-size_t decode_smem_bytes() { return static_cast<size_t>(kDecodeWarps) * kStages * kStageBytes; }
+size_t decode_smem_bytes() {
+  return static_cast<size_t>(kDecodeWarps) * kStages * kStageBytes + kDecodeWarps * kStages * sizeof(uint64_t);
+}
 
 cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(decode_smem_bytes()));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(decode_smem_bytes()));
     if (e != cudaSuccess) return e;
     configured = true;
   }
   if (n_ctas <= 0) return cudaSuccess;
-  decode_kernel<<<n_ctas, kDecodeWarps * 32, decode_smem_bytes(), st>>>(p);
+  if (p.page_idx) decode_kernel<true><<<n_ctas, kDecodeWarps * 32, decode_smem_bytes(), st>>>(p);
+  else decode_kernel<false><<<n_ctas, kDecodeWarps * 32, decode_smem_bytes(), st>>>(p);
   return cudaGetLastError();
 }
 

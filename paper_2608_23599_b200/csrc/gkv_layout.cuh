@@ -19,10 +19,17 @@
 //       token = 16*tile + r + 8*(a&1),  channel = 16*s + 8*(a>>1) + 2*c4 + hlf
 //   V role (A = V^T tile [16 channels x 16 tokens]):
 //       channel = 16*s + r + 8*(a&1),   token = 16*tile + 8*(a>>1) + 2*c4 + hlf
-// A lane's 64 values of a tile form 32 pairs rho = 4*s + a (lo = hlf 0, hi = hlf 1).  With b-bit
-// codes a 32-bit word holds ppw = 16/b pairs: word = rho / ppw, pos = rho % ppw, lo code at bit
-// b*pos, hi code at bit 16 + b*pos.  Word w of a lane lives at byte
-// ((w/4)*32 + lane)*16 + (w%4)*4 of the tile's code region (chunk-major, 512 B per warp load).
+// A lane's 64 values of a tile form 32 pairs (s, a) (lo = hlf 0 in bits 0-15, hi = hlf 1 in bits
+// 16-31 of a 32-bit word).  The bit position of a pair is chosen so that the kernel can turn a
+// code into an fp16 number "bias + code" with one shift per word and one LOP3 per pair (the code
+// is OR-ed into the mantissa of 2^E; a field at mantissa bit p with E = 10 - p has weight 1):
+//   8-bit: word = 2 s + (a >> 1); pair at byte (a & 1) and byte 2 + (a & 1)      bias 1024
+//   4-bit: word = s;              pair at bit 4 a                    bias 256 (a even) / 16 (a odd)
+//   2-bit: word = s >> 1;         pair at bit 4 (s & 1) + 2 (a & 1) + 8 (a >> 1)
+//                                 bias 256 / 64 (s even, a even / odd), 16 / 4 (s odd)
+// so that within one MMA the bias depends only on the A-row half (a & 1) and can be removed after
+// the MMA with one extra "ones" MMA.  Word w of a lane lives at byte ((w/4)*32 + lane)*16 + (w%4)*4
+// of the tile's code region (chunk-major: 512 contiguous bytes per warp-wide 16-byte load).
 #pragma once
 #include <stdint.h>
 
@@ -57,11 +64,19 @@ GKV_HD int off_vc(int bits, int t) { return 1024 + (2 + t) * code_bytes_per_tile
 // Where code (lane, s, a, hlf) of a tile sits: byte offset of its 32-bit word inside the tile's
 // code region, and the bit position inside the word.
 GKV_HD void code_pos(int bits, int lane, int s, int a, int hlf, int* byte_off, int* bit) {
-  const int rho = 4 * s + a;
-  const int ppw = 16 / bits;
-  const int w = rho / ppw, pos = rho % ppw;
+  int w, b;
+  if (bits == 8) {
+    w = 2 * s + (a >> 1);
+    b = 8 * (a & 1);
+  } else if (bits == 4) {
+    w = s;
+    b = 4 * a;
+  } else {
+    w = s >> 1;
+    b = 4 * (s & 1) + 2 * (a & 1) + 8 * (a >> 1);
+  }
   *byte_off = ((w >> 2) * 32 + lane) * 16 + (w & 3) * 4;
-  *bit = bits * pos + 16 * hlf;
+  *bit = b + 16 * hlf;
 }
 
 // K role: logical (token in block, channel) -> (tile, lane, s, a, hlf)
@@ -93,11 +108,18 @@ GKV_HD int kp_index(int ch) {
   const int c4 = (c16 & 7) >> 1;
   return (s * 4 + c4) * 8 + (c16 >> 3) * 4 + (c16 & 1);
 }
-// Value params of a tile: 16-byte records [group][c4] = {scale tA0, scale tA1, zero tA0, zero tA1,
-// scale tB0, scale tB1, zero tB0, zero tB1} with tA0 = 2 c4, tB0 = 8 + 2 c4 (tokens of the tile).
-GKV_HD int vp_index(int t16, int grp) {
+// Value params of a tile (256 B): scales first, then zeros, both as fp16 pairs of the lane's
+// token pairs tA = (2 c4, 2 c4 + 1) and tB = (8 + 2 c4, 9 + 2 c4):
+//   scales [c4][group] = {s tA0, s tA1, s tB0, s tB1}   (one lane reads its 4 groups as 32 contiguous bytes)
+//   zeros  [group][c4] = {z tA0, z tA1, z tB0, z tB1}   at byte 128 (lane r < 4 reads group r)
+// Returns the fp16 index of the scale / of the zero of (token t16 of the tile, group grp).
+GKV_HD int vp_scale_index(int t16, int grp) {
   const int c4 = (t16 & 7) >> 1;
-  return (grp * 4 + c4) * 8 + (t16 >> 3) * 4 + (t16 & 1);
+  return (c4 * 4 + grp) * 4 + (t16 >> 3) * 2 + (t16 & 1);
+}
+GKV_HD int vp_zero_index(int t16, int grp) {
+  const int c4 = (t16 & 7) >> 1;
+  return 64 + (grp * 4 + c4) * 4 + (t16 >> 3) * 2 + (t16 & 1);
 }
 
 }  // namespace gkv

@@ -76,9 +76,8 @@ __device__ void load_tile(float* tile, const uint8_t* arena, const EncodeParams&
       z = fp16_bits_to_f32(kp[idx + 2]);
     } else {
       const uint16_t* vp = reinterpret_cast<const uint16_t*>(hb + off_vp(bits, (t >> 4) & 1));
-      const int idx = vp_index(t & 15, c >> 5);
-      s = fp16_bits_to_f32(vp[idx]);
-      z = fp16_bits_to_f32(vp[idx + 2]);
+      s = fp16_bits_to_f32(vp[vp_scale_index(t & 15, c >> 5)]);
+      z = fp16_bits_to_f32(vp[vp_zero_index(t & 15, c >> 5)]);
     }
     tile[t * kTileLd + c] = __fmaf_rn(static_cast<float>(code), s, z);
   }
@@ -106,8 +105,7 @@ __device__ __forceinline__ uint8_t quant_code(float x, float s32, float z32, flo
 
 // Pack the logical codes [64][128] (shared) of one tensor into the slot's fragment-ordered words.
 __device__ void pack_codes(uint8_t* slot, const uint8_t* codes, int bits, bool is_v) {
-  const int ppw = 16 / bits;
-  const int words_per_lane = 32 / ppw;
+  const int words_per_lane = 2 * bits;           // 64 codes of `bits` bits per lane and tile
   const int total = 4 * 32 * words_per_lane;
   for (int i = threadIdx.x; i < total; i += blockDim.x) {
     const int w = i % words_per_lane;
@@ -115,21 +113,23 @@ __device__ void pack_codes(uint8_t* slot, const uint8_t* codes, int bits, bool i
     const int tile = i / (words_per_lane * 32);
     const int r = lane >> 2, c4 = lane & 3;
     uint32_t word = 0;
-    for (int pos = 0; pos < ppw; ++pos) {
-      const int rho = w * ppw + pos;
-      const int s = rho >> 2, a = rho & 3;
-      for (int hlf = 0; hlf < 2; ++hlf) {
-        int tok, ch;
-        if (!is_v) {
-          tok = 16 * tile + r + 8 * (a & 1);
-          ch = 16 * s + 8 * (a >> 1) + 2 * c4 + hlf;
-        } else {
-          ch = 16 * s + r + 8 * (a & 1);
-          tok = 16 * tile + 8 * (a >> 1) + 2 * c4 + hlf;
+    // every (s, a, hlf) whose code lives in word w of this lane
+    for (int s = 0; s < 8; ++s)
+      for (int a = 0; a < 4; ++a)
+        for (int hlf = 0; hlf < 2; ++hlf) {
+          int boff, bit;
+          code_pos(bits, lane, s, a, hlf, &boff, &bit);
+          if (boff != ((w >> 2) * 32 + lane) * 16 + (w & 3) * 4) continue;
+          int tok, ch;
+          if (!is_v) {
+            tok = 16 * tile + r + 8 * (a & 1);
+            ch = 16 * s + 8 * (a >> 1) + 2 * c4 + hlf;
+          } else {
+            ch = 16 * s + r + 8 * (a & 1);
+            tok = 16 * tile + 8 * (a >> 1) + 2 * c4 + hlf;
+          }
+          word |= static_cast<uint32_t>(codes[tok * kD + ch]) << bit;
         }
-        word |= static_cast<uint32_t>(codes[tok * kD + ch]) << (bits * pos + 16 * hlf);
-      }
-    }
     const int half = tile >> 1, t = tile & 1;
     uint8_t* region = slot + half * half_bytes(bits) + (is_v ? off_vc(bits, t) : off_kc(bits, t));
     *reinterpret_cast<uint32_t*>(region + ((w >> 2) * 32 + lane) * 16 + (w & 3) * 4) = word;
@@ -199,9 +199,8 @@ __global__ void __launch_bounds__(256) encode_kernel(const __grid_constant__ Enc
           for (int c = 0; c < kGroup; ++c)
             codes[t * kD + 32 * g + c] = quant_code(tile[t * kTileLd + 32 * g + c], s32, z32, inv, qmax);
           uint16_t* vp = reinterpret_cast<uint16_t*>(dst + (t >> 5) * half_bytes(L) + off_vp(L, (t >> 4) & 1));
-          const int idx = vp_index(t & 15, g);
-          vp[idx] = q.s_bits;
-          vp[idx + 2] = q.z_bits;
+          vp[vp_scale_index(t & 15, g)] = q.s_bits;
+          vp[vp_zero_index(t & 15, g)] = q.z_bits;
         }
         if (range) atomicOr(p.status, kStatusRange);
         __syncthreads();
@@ -368,8 +367,8 @@ __global__ void __launch_bounds__(256) export_kernel(const uint8_t* arena, uint3
     // [64][4]
     const int t = tid >> 2, g = tid & 3;
     const uint16_t* vp = reinterpret_cast<const uint16_t*>(slot + (t >> 5) * half_bytes(level) + off_vp(level, (t >> 4) & 1));
-    scale[t * 4 + g] = vp[vp_index(t & 15, g)];
-    zero[t * 4 + g] = vp[vp_index(t & 15, g) + 2];
+    scale[t * 4 + g] = vp[vp_scale_index(t & 15, g)];
+    zero[t * 4 + g] = vp[vp_zero_index(t & 15, g)];
   }
 }
 
