@@ -34,6 +34,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     objs = []
     flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
+    flags += os.environ.get("GKV_NVCC_DEFS", "").split()      # e.g. -DGKV_DECODE_WARPS=12 (tuning experiments)
     procs = []
     for src in SOURCES:
         obj = os.path.join(CSRC, src.replace(".cu", ".o"))

@@ -16,7 +16,7 @@ using namespace gkv;
 
 namespace {
 
-constexpr int kTargetWarps = 148 * 2 * kDecodeWarps;   // one resident wave: 2 CTAs x 8 warps per SM
+constexpr int kTargetWarps = 148 * kDecodeCtasPerSm * kDecodeWarps;   // one resident wave of CTAs
 constexpr int kSparseWarpsPerStream = 16;
 constexpr size_t kMinWarpBytes = 8192;
 

@@ -158,6 +158,8 @@ __device__ __forceinline__ void unpack(const uint32_t* w, int s_local, uint32_t 
   }
 }
 
+__device__ __forceinline__ float fast_exp2(float x);
+
 struct SoftmaxState {
   float m0, m1;        // running max (log2 domain) of heads 2*c4, 2*c4+1
   float l0, l1;        // lane-partial sums of exp2 (reduced over the r lanes at the end)
@@ -184,7 +186,7 @@ __device__ __forceinline__ void softmax_update(float (&S)[NT][4], SoftmaxState& 
   const float mn0 = fmaxf(st.m0, mx0), mn1 = fmaxf(st.m1, mx1);
   const float ms0 = (mn0 == kNegInf) ? 0.f : mn0, ms1 = (mn1 == kNegInf) ? 0.f : mn1;
   if (__any_sync(kFull, mn0 != st.m0 || mn1 != st.m1)) {
-    const float al0 = exp2f(st.m0 - ms0), al1 = exp2f(st.m1 - ms1);
+    const float al0 = fast_exp2(st.m0 - ms0), al1 = fast_exp2(st.m1 - ms1);
     st.m0 = mn0;
     st.m1 = mn1;
     st.l0 *= al0;
@@ -201,10 +203,10 @@ __device__ __forceinline__ void softmax_update(float (&S)[NT][4], SoftmaxState& 
   }
 #pragma unroll
   for (int t = 0; t < NT; ++t) {
-    S[t][0] = exp2f(S[t][0] - ms0);
-    S[t][1] = exp2f(S[t][1] - ms1);
-    S[t][2] = exp2f(S[t][2] - ms0);
-    S[t][3] = exp2f(S[t][3] - ms1);
+    S[t][0] = fast_exp2(S[t][0] - ms0);
+    S[t][1] = fast_exp2(S[t][1] - ms1);
+    S[t][2] = fast_exp2(S[t][2] - ms0);
+    S[t][3] = fast_exp2(S[t][3] - ms1);
   }
 }
 
@@ -250,9 +252,10 @@ struct WarpCtx {
   int item_end;              // dense: one past the last item; sparse: one past the last page position
   int stream;
   bool has_tail;
-  uint32_t stage[kStages];   // shared-memory addresses of the stages
-  const uint8_t* stage_ptr[kStages];
-  uint32_t bar[kStages];
+  uint32_t stage0;           // shared-memory address of stage 0 (stage s at + s * kStageBytes)
+  const uint8_t* stage_ptr0; // the same as a generic pointer
+  uint32_t bar0;             // mbarrier of stage 0 (stage s at + 8 s)
+  uint32_t qb_addr;          // this lane's bf16 query fragments in shared memory (16 words)
   // prefetched window of table entries (dense mode): lane i holds entry win_base + i
   uint4 win;
   int win_base;
@@ -421,7 +424,7 @@ __device__ __forceinline__ int half_of_step(const Cursor& c, int idx) {
 template <bool SPARSE>
 __device__ __forceinline__ void issue_step(const WarpCtx& w, const Cursor& c, int sidx) {
   const DecodeParams& p = *w.p;
-  const uint32_t sdst = w.stage[sidx], bar = w.bar[sidx];
+  const uint32_t sdst = w.stage0 + sidx * kStageBytes, bar = w.bar0 + sidx * 8;
   const int lane = w.lane;
   if (c.level == 16 || c.level == 1 || c.level == 17) {
     // up to 16 rows of 256 B, staged at a 272-byte pitch; one bulk copy per row
@@ -452,7 +455,7 @@ __device__ __forceinline__ void issue_step(const WarpCtx& w, const Cursor& c, in
       bulk_g2s(sdst + lane * kRowPitch, src, kRowBytes, bar);
     } else if (lane < 16) {
       // rows past the end are zero so that 0 * garbage never produces a NaN
-      uint4* z = reinterpret_cast<uint4*>(const_cast<uint8_t*>(w.stage_ptr[sidx]) + lane * kRowPitch);
+      uint4* z = reinterpret_cast<uint4*>(const_cast<uint8_t*>(w.stage_ptr0) + sidx * kStageBytes + lane * kRowPitch);
 #pragma unroll
       for (int i = 0; i < kRowBytes / 16; ++i) z[i] = make_uint4(0, 0, 0, 0);
     }
@@ -526,51 +529,99 @@ __device__ __forceinline__ void issue_step(const WarpCtx& w, const Cursor& c, in
 }
 
 // ---- compute ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+// D = A B (no accumulator input: the first MMA of a chain)
+__device__ __forceinline__ void mma_f16_first(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};\n"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+}
+
+// Code words of MMA indices (2 j, 2 j + 1) of one lane: 8-bit 4 words, 4-bit 2 words, 2-bit 1 word.
+template <int BITS>
+__device__ __forceinline__ void load_words(uint32_t codes, int j, int lane, uint32_t (&w)[BITS / 2]) {
+  constexpr int kW = BITS / 2;
+  const uint32_t a = codes + ((j * kW >> 2) * 32 + lane) * 16 + ((j * kW) & 3) * 4;
+  if constexpr (BITS == 8) {
+    const uint4 v = lds128(a);
+    w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+  } else if constexpr (BITS == 4) {
+    const uint2 v = lds64(a);
+    w[0] = v.x; w[1] = v.y;
+  } else {
+    w[0] = lds32(a);
+  }
+}
+
 // Logits of the active tiles of one half (32 tokens): S = scale * (q . k~) + token bias, with
-// k~ = s * code + z.  Data MMAs use A = bias + code and B = q' = q * s; the bias is removed with a
-// "ones" MMA on the same q' and the zero points enter through an MMA with A = z and B = q.
+// k~ = s * code + z.  Data MMAs use A = bias + code and B = q' = q * s; the bias (and the code
+// centre) is removed with a "ones" MMA on the same q' and the zero points enter through an MMA
+// with A = (z | s) and B = q.  All arguments that address shared memory are 32-bit addresses.
 template <int BITS, bool FULL>
-__device__ __forceinline__ void qk_half(const uint8_t* kp, const uint8_t* kc0, const uint8_t* kc1, int tm,
-                                        const uint32_t (&qh)[16], int lane, float scale_log2, uint64_t resmask,
-                                        int half, float (&S)[2][4]) {
+__device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, uint32_t kc1, int tm, const uint32_t (&qh)[16],
+                                        int lane, float scale_log2, uint64_t resmask, int half, float (&S)[2][4]) {
   const int c4 = lane & 3, r = lane >> 2;
-  constexpr int kWords = 2 * BITS;               // words per lane and tile
-  uint32_t w0[kWords], w1[kWords];
-  if (FULL || (tm & 1)) {
+  float zd[4];        // rows r: sum_c q_c z_c; rows r + 8: sum_c q_c s_c (exact products)
+  float qe[4];        // sum_c q'_c over even MMA indices (all rows equal)
+  float qo[4] = {0.f, 0.f, 0.f, 0.f};   // ... over odd MMA indices (2-bit only)
+  constexpr int kW = BITS / 2;
+  kp += c4 * 16;
 #pragma unroll
-    for (int j = 0; j < kWords / 4; ++j) {
-      const uint4 v = *reinterpret_cast<const uint4*>(kc0 + (j * 32 + lane) * 16);
-      w0[4 * j] = v.x; w0[4 * j + 1] = v.y; w0[4 * j + 2] = v.z; w0[4 * j + 3] = v.w;
+  for (int j = 0; j < 4; ++j) {
+    uint32_t w0[kW], w1[kW];
+    if (FULL || (tm & 1)) load_words<BITS>(kc0, j, lane, w0);
+    if (FULL || (tm & 2)) load_words<BITS>(kc1, j, lane, w1);
+#pragma unroll
+    for (int ss = 0; ss < 2; ++ss) {
+      const int s = 2 * j + ss;
+      const uint4 pr = lds128(kp + s * 64);   // s01, z01, s23, z23
+      const uint32_t q0 = hmul2_u32(qh[2 * s], pr.x), q1 = hmul2_u32(qh[2 * s + 1], pr.z);
+      if (s == 0) mma_f16_first(zd, pr.y, pr.x, pr.w, pr.z, qh[0], qh[1]);
+      else mma_f16(zd, pr.y, pr.x, pr.w, pr.z, qh[2 * s], qh[2 * s + 1]);
+      if (BITS == 2 && ss == 1) {
+        if (s == 1) mma_f16_first(qo, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
+        else mma_f16(qo, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
+      } else {
+        if (s == 0) mma_f16_first(qe, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
+        else mma_f16(qe, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
+      }
+      uint32_t a[4];
+      if (FULL || (tm & 1)) {
+        unpack<BITS>(w0, ss, a);
+        if (s == 0) mma_f16_first(S[0], a[0], a[1], a[2], a[3], q0, q1);
+        else mma_f16(S[0], a[0], a[1], a[2], a[3], q0, q1);
+      }
+      if (FULL || (tm & 2)) {
+        unpack<BITS>(w1, ss, a);
+        if (s == 0) mma_f16_first(S[1], a[0], a[1], a[2], a[3], q0, q1);
+        else mma_f16(S[1], a[0], a[1], a[2], a[3], q0, q1);
+      }
     }
   }
-  if (FULL || (tm & 2)) {
-#pragma unroll
-    for (int j = 0; j < kWords / 4; ++j) {
-      const uint4 v = *reinterpret_cast<const uint4*>(kc1 + (j * 32 + lane) * 16);
-      w1[4 * j] = v.x; w1[4 * j + 1] = v.y; w1[4 * j + 2] = v.z; w1[4 * j + 3] = v.w;
-    }
-  }
-  float zd[4] = {0.f, 0.f, 0.f, 0.f};        // rows r: sum_c q_c z_c; rows r + 8: sum_c q_c s_c (exact products)
-  float qe[4] = {0.f, 0.f, 0.f, 0.f};        // sum_c q'_c over even MMA indices (all rows equal)
-  float qo[4] = {0.f, 0.f, 0.f, 0.f};        // ... over odd MMA indices (2-bit only)
-#pragma unroll
-  for (int t = 0; t < 2; ++t) S[t][0] = S[t][1] = S[t][2] = S[t][3] = 0.f;
-#pragma unroll
-  for (int s = 0; s < 8; ++s) {
-    const uint4 pr = *reinterpret_cast<const uint4*>(kp + (s * 4 + c4) * 16);   // s01, z01, s23, z23
-    const uint32_t q0 = hmul2_u32(qh[2 * s], pr.x), q1 = hmul2_u32(qh[2 * s + 1], pr.z);
-    mma_f16(zd, pr.y, pr.x, pr.w, pr.z, qh[2 * s], qh[2 * s + 1]);
-    if (BITS == 2 && (s & 1)) mma_f16(qo, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
-    else mma_f16(qe, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
-    uint32_t a[4];
-    if (FULL || (tm & 1)) {
-      unpack<BITS>(w0, s, a);
-      mma_f16(S[0], a[0], a[1], a[2], a[3], q0, q1);
-    }
-    if (FULL || (tm & 2)) {
-      unpack<BITS>(w1, s, a);
-      mma_f16(S[1], a[0], a[1], a[2], a[3], q0, q1);
-    }
+  if (!FULL) {
+    if (!(tm & 1)) S[0][0] = S[0][1] = S[0][2] = S[0][3] = 0.f;
+    if (!(tm & 2)) S[1][0] = S[1][1] = S[1][2] = S[1][3] = 0.f;
   }
   // rows r carry bias lo, rows r + 8 carry bias hi (per parity of the MMA index)
   constexpr float kMid = Bias<BITS>::mid;
@@ -579,12 +630,23 @@ __device__ __forceinline__ void qk_half(const uint8_t* kp, const uint8_t* kc0, c
   const float c_lo1 = z1 - (Bias<BITS>::lo_even + kMid) * qe[1] - (Bias<BITS>::lo_odd + kMid) * qo[1];
   const float c_hi0 = z0 - (Bias<BITS>::hi_even + kMid) * qe[0] - (Bias<BITS>::hi_odd + kMid) * qo[0];
   const float c_hi1 = z1 - (Bias<BITS>::hi_even + kMid) * qe[1] - (Bias<BITS>::hi_odd + kMid) * qo[1];
+  if (FULL && resmask == 0) {
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      S[t][0] = (S[t][0] + c_lo0) * scale_log2;
+      S[t][1] = (S[t][1] + c_lo1) * scale_log2;
+      S[t][2] = (S[t][2] + c_hi0) * scale_log2;
+      S[t][3] = (S[t][3] + c_hi1) * scale_log2;
+    }
+    return;
+  }
+  const uint32_t rm = static_cast<uint32_t>(resmask >> (32 * half));      // this half's 32 tokens
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
-    const int tok = 32 * half + 16 * t + r;
+    const int tok = 16 * t + r;
     const bool on = FULL || ((tm >> t) & 1);
-    const float b_lo = (on && !((resmask >> tok) & 1ull)) ? 0.f : kNegInf;
-    const float b_hi = (on && !((resmask >> (tok + 8)) & 1ull)) ? 0.f : kNegInf;
+    const float b_lo = (on && !((rm >> tok) & 1u)) ? 0.f : kNegInf;
+    const float b_hi = (on && !((rm >> (tok + 8)) & 1u)) ? 0.f : kNegInf;
     S[t][0] = fmaf(S[t][0] + c_lo0, scale_log2, b_lo);
     S[t][1] = fmaf(S[t][1] + c_lo1, scale_log2, b_lo);
     S[t][2] = fmaf(S[t][2] + c_hi0, scale_log2, b_hi);
@@ -592,103 +654,86 @@ __device__ __forceinline__ void qk_half(const uint8_t* kp, const uint8_t* kc0, c
   }
 }
 
+// One tile's share of O^T += V~^T P^T for group grp: data MMAs accumulate (bias + code) * P' straight
+// into O; `ps` collects sum P' so that the bias can be taken out afterwards.
+template <int BITS>
+__device__ __forceinline__ void pv_tile_group(uint32_t vc, int grp, int lane, uint32_t p0, uint32_t p1, bool first,
+                                              float (&ps)[4], float (&o0)[4], float (&o1)[4]) {
+  uint32_t wd[BITS / 2];
+  uint32_t a[4];
+  load_words<BITS>(vc, grp, lane, wd);
+  if (first) mma_f16_first(ps, kOnesH2, kOnesH2, kOnesH2, kOnesH2, p0, p1);
+  else mma_f16(ps, kOnesH2, kOnesH2, kOnesH2, kOnesH2, p0, p1);
+  unpack<BITS>(wd, 0, a);
+  mma_f16(o0, a[0], a[1], a[2], a[3], p0, p1);
+  unpack<BITS>(wd, 1, a);
+  mma_f16(o1, a[0], a[1], a[2], a[3], p0, p1);
+}
+
 // O^T += V~^T P^T for the active tiles of one half, v~ = s * code + z per (token, 32-channel group).
 // pf holds the raw fp16 P^T fragments of the two tiles.
 template <int BITS, bool FULL>
-__device__ __forceinline__ void pv_half(const uint8_t* vp0, const uint8_t* vp1, const uint8_t* vc0,
-                                        const uint8_t* vc1, int tm, const uint32_t (&pf)[2][2], int lane,
-                                        SoftmaxState& st) {
+__device__ __forceinline__ void pv_half(uint32_t vp0, uint32_t vp1, uint32_t vc0, uint32_t vc1, int tm,
+                                        const uint32_t (&pf)[2][2], int lane, SoftmaxState& st) {
   const int c4 = lane & 3, r = lane >> 2;
-  constexpr int kWordsPerGrp = BITS / 2;          // words of a lane covering MMA indices 2g, 2g+1
   // per-lane scales of its token pairs, all four groups: {sA, sB} x 4 per tile
-  uint32_t sc0[8], sc1[8];
-  float tz[4] = {0.f, 0.f, 0.f, 0.f};
-  if (FULL || (tm & 1)) {
-    const uint4 x = *reinterpret_cast<const uint4*>(vp0 + c4 * 32), y = *reinterpret_cast<const uint4*>(vp0 + c4 * 32 + 16);
-    sc0[0] = x.x; sc0[1] = x.y; sc0[2] = x.z; sc0[3] = x.w; sc0[4] = y.x; sc0[5] = y.y; sc0[6] = y.z; sc0[7] = y.w;
+  uint4 x0, y0, x1, y1;
+  float tz[4];
+  const bool t0 = FULL || (tm & 1), t1 = FULL || (tm & 2);
+  if (t0) {
+    x0 = lds128(vp0 + c4 * 32);
+    y0 = lds128(vp0 + c4 * 32 + 16);
     // rows g < 4: sum_tok p z[tok][g]; rows 8 + g: sum_tok p s[tok][g] (exact products)
     uint2 z = make_uint2(0, 0), sg = make_uint2(0, 0);
     if (r < 4) {
-      z = *reinterpret_cast<const uint2*>(vp0 + 128 + (r * 4 + c4) * 8);
-      sg = make_uint2(sc0[0], sc0[1]);
-      if (r == 1) sg = make_uint2(sc0[2], sc0[3]);
-      if (r == 2) sg = make_uint2(sc0[4], sc0[5]);
-      if (r == 3) sg = make_uint2(sc0[6], sc0[7]);
+      z = lds64(vp0 + 128 + (r * 4 + c4) * 8);
+      sg = lds64(vp0 + c4 * 32 + r * 8);
     }
-    mma_f16(tz, z.x, sg.x, z.y, sg.y, pf[0][0], pf[0][1]);
+    mma_f16_first(tz, z.x, sg.x, z.y, sg.y, pf[0][0], pf[0][1]);
   }
-  if (FULL || (tm & 2)) {
-    const uint4 x = *reinterpret_cast<const uint4*>(vp1 + c4 * 32), y = *reinterpret_cast<const uint4*>(vp1 + c4 * 32 + 16);
-    sc1[0] = x.x; sc1[1] = x.y; sc1[2] = x.z; sc1[3] = x.w; sc1[4] = y.x; sc1[5] = y.y; sc1[6] = y.z; sc1[7] = y.w;
+  if (t1) {
+    x1 = lds128(vp1 + c4 * 32);
+    y1 = lds128(vp1 + c4 * 32 + 16);
     uint2 z = make_uint2(0, 0), sg = make_uint2(0, 0);
     if (r < 4) {
-      z = *reinterpret_cast<const uint2*>(vp1 + 128 + (r * 4 + c4) * 8);
-      sg = make_uint2(sc1[0], sc1[1]);
-      if (r == 1) sg = make_uint2(sc1[2], sc1[3]);
-      if (r == 2) sg = make_uint2(sc1[4], sc1[5]);
-      if (r == 3) sg = make_uint2(sc1[6], sc1[7]);
+      z = lds64(vp1 + 128 + (r * 4 + c4) * 8);
+      sg = lds64(vp1 + c4 * 32 + r * 8);
     }
-    mma_f16(tz, z.x, sg.x, z.y, sg.y, pf[1][0], pf[1][1]);
+    if (t0) mma_f16(tz, z.x, sg.x, z.y, sg.y, pf[1][0], pf[1][1]);
+    else mma_f16_first(tz, z.x, sg.x, z.y, sg.y, pf[1][0], pf[1][1]);
   }
   st.zc[0] += fmaf(Bias<BITS>::mid, tz[2], tz[0]);
   st.zc[1] += fmaf(Bias<BITS>::mid, tz[3], tz[1]);
 #pragma unroll
   for (int grp = 0; grp < 4; ++grp) {
-    float ps[4] = {0.f, 0.f, 0.f, 0.f};          // sum over tokens of P' (all rows equal)
-    float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};   // this step's O for u = 2g, 2g+1
-    uint32_t wd[kWordsPerGrp];
-    uint32_t a[4];
-    if (FULL || (tm & 1)) {
-      const uint32_t p0 = hmul2_u32(pf[0][0], sc0[2 * grp]), p1 = hmul2_u32(pf[0][1], sc0[2 * grp + 1]);
-      mma_f16(ps, kOnesH2, kOnesH2, kOnesH2, kOnesH2, p0, p1);
-      // words of MMA indices 2 grp and 2 grp + 1: 8-bit words 4g..4g+3, 4-bit 2g..2g+1, 2-bit g
-      const uint8_t* base = vc0 + ((grp * kWordsPerGrp >> 2) * 32 + lane) * 16 + ((grp * kWordsPerGrp) & 3) * 4;
-      if constexpr (BITS == 8) {
-        const uint4 v = *reinterpret_cast<const uint4*>(base);
-        wd[0] = v.x; wd[1] = v.y; wd[2] = v.z; wd[3] = v.w;
-      } else if constexpr (BITS == 4) {
-        const uint2 v = *reinterpret_cast<const uint2*>(base);
-        wd[0] = v.x; wd[1] = v.y;
-      } else {
-        wd[0] = *reinterpret_cast<const uint32_t*>(base);
-      }
-      unpack<BITS>(wd, 0, a);
-      mma_f16(acc0, a[0], a[1], a[2], a[3], p0, p1);
-      unpack<BITS>(wd, 1, a);
-      mma_f16(acc1, a[0], a[1], a[2], a[3], p0, p1);
+    float ps[4];          // sum over tokens of P' (all rows equal)
+    if (t0) {
+      const uint32_t sa = grp == 0 ? x0.x : grp == 1 ? x0.z : grp == 2 ? y0.x : y0.z;
+      const uint32_t sb = grp == 0 ? x0.y : grp == 1 ? x0.w : grp == 2 ? y0.y : y0.w;
+      pv_tile_group<BITS>(vc0, grp, lane, hmul2_u32(pf[0][0], sa), hmul2_u32(pf[0][1], sb), true, ps,
+                          st.o[2 * grp], st.o[2 * grp + 1]);
     }
-    if (FULL || (tm & 2)) {
-      const uint32_t p0 = hmul2_u32(pf[1][0], sc1[2 * grp]), p1 = hmul2_u32(pf[1][1], sc1[2 * grp + 1]);
-      mma_f16(ps, kOnesH2, kOnesH2, kOnesH2, kOnesH2, p0, p1);
-      const uint8_t* base = vc1 + ((grp * kWordsPerGrp >> 2) * 32 + lane) * 16 + ((grp * kWordsPerGrp) & 3) * 4;
-      if constexpr (BITS == 8) {
-        const uint4 v = *reinterpret_cast<const uint4*>(base);
-        wd[0] = v.x; wd[1] = v.y; wd[2] = v.z; wd[3] = v.w;
-      } else if constexpr (BITS == 4) {
-        const uint2 v = *reinterpret_cast<const uint2*>(base);
-        wd[0] = v.x; wd[1] = v.y;
-      } else {
-        wd[0] = *reinterpret_cast<const uint32_t*>(base);
-      }
-      unpack<BITS>(wd, 0, a);
-      mma_f16(acc0, a[0], a[1], a[2], a[3], p0, p1);
-      unpack<BITS>(wd, 1, a);
-      mma_f16(acc1, a[0], a[1], a[2], a[3], p0, p1);
+    if (t1) {
+      const uint32_t sa = grp == 0 ? x1.x : grp == 1 ? x1.z : grp == 2 ? y1.x : y1.z;
+      const uint32_t sb = grp == 0 ? x1.y : grp == 1 ? x1.w : grp == 2 ? y1.y : y1.w;
+      pv_tile_group<BITS>(vc1, grp, lane, hmul2_u32(pf[1][0], sa), hmul2_u32(pf[1][1], sb), !t0, ps,
+                          st.o[2 * grp], st.o[2 * grp + 1]);
     }
-    // remove the biases: u = 2g is an even MMA index, u = 2g + 1 an odd one
-    st.o[2 * grp][0] += acc0[0] - (Bias<BITS>::lo_even + Bias<BITS>::mid) * ps[0];
-    st.o[2 * grp][1] += acc0[1] - (Bias<BITS>::lo_even + Bias<BITS>::mid) * ps[1];
-    st.o[2 * grp][2] += acc0[2] - (Bias<BITS>::hi_even + Bias<BITS>::mid) * ps[0];
-    st.o[2 * grp][3] += acc0[3] - (Bias<BITS>::hi_even + Bias<BITS>::mid) * ps[1];
-    st.o[2 * grp + 1][0] += acc1[0] - (Bias<BITS>::lo_odd + Bias<BITS>::mid) * ps[0];
-    st.o[2 * grp + 1][1] += acc1[1] - (Bias<BITS>::lo_odd + Bias<BITS>::mid) * ps[1];
-    st.o[2 * grp + 1][2] += acc1[2] - (Bias<BITS>::hi_odd + Bias<BITS>::mid) * ps[0];
-    st.o[2 * grp + 1][3] += acc1[3] - (Bias<BITS>::hi_odd + Bias<BITS>::mid) * ps[1];
+    // remove bias + centre: u = 2g is an even MMA index, u = 2g + 1 an odd one
+    constexpr float kMid = Bias<BITS>::mid;
+    st.o[2 * grp][0] = fmaf(-(Bias<BITS>::lo_even + kMid), ps[0], st.o[2 * grp][0]);
+    st.o[2 * grp][1] = fmaf(-(Bias<BITS>::lo_even + kMid), ps[1], st.o[2 * grp][1]);
+    st.o[2 * grp][2] = fmaf(-(Bias<BITS>::hi_even + kMid), ps[0], st.o[2 * grp][2]);
+    st.o[2 * grp][3] = fmaf(-(Bias<BITS>::hi_even + kMid), ps[1], st.o[2 * grp][3]);
+    st.o[2 * grp + 1][0] = fmaf(-(Bias<BITS>::lo_odd + kMid), ps[0], st.o[2 * grp + 1][0]);
+    st.o[2 * grp + 1][1] = fmaf(-(Bias<BITS>::lo_odd + kMid), ps[1], st.o[2 * grp + 1][1]);
+    st.o[2 * grp + 1][2] = fmaf(-(Bias<BITS>::hi_odd + kMid), ps[0], st.o[2 * grp + 1][2]);
+    st.o[2 * grp + 1][3] = fmaf(-(Bias<BITS>::hi_odd + kMid), ps[1], st.o[2 * grp + 1][3]);
   }
 }
 
 template <int BITS, bool FULL>
-__device__ __forceinline__ void qk_softmax_half(const uint8_t* half_k, int half, int tm, uint64_t resmask,
+__device__ __forceinline__ void qk_softmax_half(uint32_t half_k, int half, int tm, uint64_t resmask,
                                                 const uint32_t (&qh)[16], int lane, float scale_log2,
                                                 SoftmaxState& st, uint32_t (&pf)[2][2]) {
   constexpr int cb = 256 * BITS;
@@ -701,12 +746,11 @@ __device__ __forceinline__ void qk_softmax_half(const uint8_t* half_k, int half,
 
 // Process a staged step.  pf carries P fragments from a key step to the following value step.
 template <bool SPARSE>
-__device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, int sidx, const uint32_t (&qb)[16],
+__device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, int sidx,
                                              const uint32_t (&qh)[16], SoftmaxState& st, uint32_t (&pf)[4]) {
   const DecodeParams& p = *w.p;
   const int lane = w.lane;
-  const uint8_t* sp = w.stage_ptr[sidx];
-  const uint32_t sa = w.stage[sidx];
+  const uint32_t sa = w.stage0 + sidx * kStageBytes;
   if (c.level == 16 || c.level == 1 || c.level == 17) {
     if ((c.sub & 1) == 0) {
       // key rows: S^T = K Q^T
@@ -717,7 +761,8 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
       for (int s = 0; s < 8; ++s) {
         uint32_t a[4];
         ldmatrix_x4(a, base + s * 32);
-        mma_bf16(S[0], a, qb[2 * s], qb[2 * s + 1]);
+        const uint2 b = lds64(w.qb_addr + s * 256);
+        mma_bf16(S[0], a, b.x, b.y);
       }
       // validity / weight of the lane's rows r and r + 8
       const int r = lane >> 2;
@@ -767,19 +812,19 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
   if (c.level == 8) {
     const int half = FULL ? (c.sub >> 1) : ((c.tmask == 15) ? (c.sub >> 1) : half_of_step(c, c.sub >> 1));
     const int tm = (c.tmask >> (2 * half)) & 3;
-    if ((c.sub & 1) == 0) qk_softmax_half<8, FULL>(sp, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
-    else pv_half<8, FULL>(sp, sp + 256, sp + 512, sp + 512 + 2048, tm, pf2, lane, st);
+    if ((c.sub & 1) == 0) qk_softmax_half<8, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
+    else pv_half<8, FULL>(sa, sa + 256, sa + 512, sa + 512 + 2048, tm, pf2, lane, st);
   } else if (c.level == 4) {
     const int half = FULL ? c.sub : ((c.tmask == 15) ? c.sub : half_of_step(c, c.sub));
     const int tm = (c.tmask >> (2 * half)) & 3;
-    qk_softmax_half<4, FULL>(sp, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
-    pv_half<4, FULL>(sp + off_vp(4, 0), sp + off_vp(4, 1), sp + off_vc(4, 0), sp + off_vc(4, 1), tm, pf2, lane, st);
+    qk_softmax_half<4, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
+    pv_half<4, FULL>(sa + off_vp(4, 0), sa + off_vp(4, 1), sa + off_vc(4, 0), sa + off_vc(4, 1), tm, pf2, lane, st);
   } else {
 #pragma unroll 1
     for (int half = 0; half < 2; ++half) {
       const int tm = (c.tmask >> (2 * half)) & 3;
       if (!FULL && tm == 0) continue;
-      const uint8_t* hb = sp + half * half_bytes(2);
+      const uint32_t hb = sa + half * half_bytes(2);
       qk_softmax_half<2, FULL>(hb, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
       pv_half<2, FULL>(hb + off_vp(2, 0), hb + off_vp(2, 1), hb + off_vc(2, 0), hb + off_vc(2, 1), tm, pf2, lane, st);
     }
@@ -787,7 +832,7 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
 }
 
 template <bool SPARSE>
-__global__ void __launch_bounds__(kDecodeWarps * 32, 2) decode_kernel(const __grid_constant__ DecodeParams p) {
+__global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_kernel(const __grid_constant__ DecodeParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gw = blockIdx.x * kDecodeWarps + warp;
@@ -819,15 +864,14 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 2) decode_kernel(const __gr
   w.table = p.table + static_cast<size_t>(w.stream) * p.table_stride;
   uint8_t* sbase = smem + warp * (kStages * kStageBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kDecodeWarps * kStages * kStageBytes) + warp * kStages;
-#pragma unroll
-  for (int s = 0; s < kStages; ++s) {
-    w.stage_ptr[s] = sbase + s * kStageBytes;
-    w.stage[s] = smem_u32(sbase + s * kStageBytes);
-    w.bar[s] = smem_u32(bars + s);
-  }
+  uint8_t* qb_smem = smem + kDecodeWarps * (kStages * kStageBytes + kStages * 8) + warp * 2048;
+  w.stage_ptr0 = sbase;
+  w.stage0 = smem_u32(sbase);
+  w.bar0 = smem_u32(bars);
+  w.qb_addr = smem_u32(qb_smem) + lane * 8;       // word pair s at + 256 s (conflict-free 8-byte accesses)
   if (lane == 0) {
 #pragma unroll
-    for (int s = 0; s < kStages; ++s) mbar_init(w.bar[s], 1);
+    for (int s = 0; s < kStages; ++s) mbar_init(w.bar0 + 8 * s, 1);
     fence_proxy_async();
   }
   __syncwarp();
@@ -835,7 +879,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 2) decode_kernel(const __gr
   // Query fragments: B operand Q^T[16 channels x 8 heads]; lane (r, c4) holds head r, channels
   // 16 s + 2 c4 (+1) and 16 s + 8 + 2 c4 (+1), in bf16 (exact rows) and fp16 (quantised tiers).
   const int r = lane >> 2, c4 = lane & 3;
-  uint32_t qb[16], qh[16];
+  uint32_t qh[16];
   {
     const int b = w.stream / p.n_kv_heads, kvh = w.stream - b * p.n_kv_heads;
     const int n_q_heads = p.n_kv_heads * p.group;
@@ -847,8 +891,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 2) decode_kernel(const __gr
         v0 = *reinterpret_cast<const uint32_t*>(qrow + 16 * s + 2 * c4);
         v1 = *reinterpret_cast<const uint32_t*>(qrow + 16 * s + 8 + 2 * c4);
       }
-      qb[2 * s] = v0;
-      qb[2 * s + 1] = v1;
+      asm volatile("st.shared.v2.u32 [%0], {%1,%2};\n" ::"r"(w.qb_addr + s * 256), "r"(v0), "r"(v1) : "memory");
       qh[2 * s] = h2_as_u32(__floats2half2_rn(bf16lo_to_f32(v0), bf16hi_to_f32(v0)));
       qh[2 * s + 1] = h2_as_u32(__floats2half2_rn(bf16lo_to_f32(v1), bf16hi_to_f32(v1)));
     }
@@ -874,7 +917,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 2) decode_kernel(const __gr
     if (more) issue_step<SPARSE>(w, nxt, sidx ^ 1);
     // bounded wait for this step's bytes
     int spins = 0;
-    while (!mbar_try_wait(w.bar[sidx], (phase >> sidx) & 1u)) {
+    while (!mbar_try_wait(w.bar0 + 8 * sidx, (phase >> sidx) & 1u)) {
       if (++spins > kWaitSpins) {
         failed = true;
         break;
@@ -883,7 +926,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 2) decode_kernel(const __gr
     if (__any_sync(kFull, failed)) break;
     phase ^= 1u << sidx;
     __syncwarp();
-    compute_step<SPARSE>(w, cur, sidx, qb, qh, st, pf);
+    compute_step<SPARSE>(w, cur, sidx, qh, st, pf);
     __syncwarp();
     cur = nxt;
     have = more;
@@ -961,7 +1004,8 @@ __global__ void __launch_bounds__(kD) combine_kernel(const __grid_constant__ Com
 }  // namespace
 
 size_t decode_smem_bytes() {
-  return static_cast<size_t>(kDecodeWarps) * kStages * kStageBytes + kDecodeWarps * kStages * sizeof(uint64_t);
+  // per warp: pipeline stages, their mbarriers, and the bf16 query fragments (2 KiB)
+  return static_cast<size_t>(kDecodeWarps) * (kStages * kStageBytes + kStages * sizeof(uint64_t) + 2048);
 }
 
 cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st) {

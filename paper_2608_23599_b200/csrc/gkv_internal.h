@@ -30,9 +30,16 @@ struct alignas(8) StreamParts {
   int32_t begin, end;  // partial rows [begin, end) belong to this stream
 };
 
-constexpr int kDecodeWarps = 8;             // warps per CTA of the decode kernel
+#ifndef GKV_DECODE_WARPS
+#define GKV_DECODE_WARPS 8
+#endif
+#ifndef GKV_DECODE_CTAS_PER_SM
+#define GKV_DECODE_CTAS_PER_SM 2
+#endif
+constexpr int kDecodeWarps = GKV_DECODE_WARPS;               // warps per CTA of the decode kernel
 constexpr int kStageBytes = 6144;           // per-warp pipeline stage
 constexpr int kStages = 2;
+constexpr int kDecodeCtasPerSm = GKV_DECODE_CTAS_PER_SM;
 constexpr int kMaxHeadsPerKv = 8;           // one n=8 tensor-core tile of query heads
 constexpr int kPartialFloats = kMaxHeadsPerKv * (kD + 2);   // per partial row: m, l, o[128] per head
 
