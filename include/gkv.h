@@ -142,6 +142,25 @@ GKV_API int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const in
 GKV_API int gkv_quest_select(gkv_cache* c, int32_t layer, const void* q, int32_t budget_tokens,
                      int32_t* page_idx_out, int32_t* n_sel_out, void* stream);
 
+/* The same page selection as gkv_quest_select for callers that cannot have any device memory
+ * allocated on their behalf while they run: a plug-in that was handed a fixed arena by a serving
+ * engine whose pool is fully committed, a real-time loop that forbids allocation after start-up,
+ * or code that runs where cudaMalloc is not allowed.  (The paper has no counterpart; this is a
+ * packaging variant of the Sec. 3.5 selection.)  The page scores, which gkv_quest_select keeps in
+ * the arena, go to a fixed 4 MiB array that is part of the library image, so the call performs no
+ * cudaMalloc / cudaFree and uses no allocating library routine.
+ *   - Limit: batch * n_kv_heads * round_up(closed pages, 8) <= 1,048,576 scores; larger caches get
+ *     GKV_ERR_UNSUPPORTED (use gkv_quest_select).
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress);
+ *     make that first call before any stream capture begins.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.  Each
+ *     call overwrites every score it later reads, so stale contents are harmless, but two calls
+ *     whose kernels overlap on the GPU (different streams, or different caches) race: issue them
+ *     on one stream or order them yourself.
+ * Arguments and results are exactly those of gkv_quest_select. */
+GKV_API int gkv_quest_select_static(gkv_cache* c, int32_t layer, const void* q, int32_t budget_tokens,
+                                    int32_t* page_idx_out, int32_t* n_sel_out, void* stream);
+
 /* Resident / read bit accounting of `layer` (-1 = all layers).  Synchronises when the last
  * read used a page list (it is fetched to count the bits touched).  out: host. */
 GKV_API int gkv_bits_report(gkv_cache* c, int32_t layer, gkv_bits* out);

@@ -23,7 +23,7 @@ ERR_RANGE, ERR_BUDGET = -6, -7
 
 EXPORTS = [
     "gkv_query_arena_bytes", "gkv_create", "gkv_destroy", "gkv_append_demote", "gkv_decode_attn",
-    "gkv_quest_select", "gkv_bits_report", "gkv_debug_export_block", "gkv_debug_export_residual",
+    "gkv_quest_select", "gkv_quest_select_static", "gkv_bits_report", "gkv_debug_export_block", "gkv_debug_export_residual",
     "gkv_debug_export_levels", "gkv_ctx_len", "gkv_strerror", "gkv_last_cuda_error",
 ]
 
@@ -79,6 +79,7 @@ def load():
     lib.gkv_append_demote.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp]
     lib.gkv_decode_attn.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp]
     lib.gkv_quest_select.argtypes = [vp, i32, vp, i32, vp, C.POINTER(i32), vp]
+    lib.gkv_quest_select_static.argtypes = [vp, i32, vp, i32, vp, C.POINTER(i32), vp]
     lib.gkv_bits_report.argtypes = [vp, i32, C.POINTER(GkvBits)]
     lib.gkv_debug_export_block.argtypes = [vp, i32, i32, i32, i32, i32, C.POINTER(i32), vp, vp, vp, vp, C.POINTER(i32)]
     lib.gkv_debug_export_residual.argtypes = [vp, i32, i32, i32, vp, i32, C.POINTER(i32)]
@@ -192,6 +193,14 @@ class Cache:
         n = C.c_int32(0)
         _check(load().gkv_quest_select(self.handle, layer, _ptr(q), budget_tokens, _ptr(page_idx_out), C.byref(n),
                                        _stream()), "gkv_quest_select")
+        return n.value
+
+    def gkv_quest_select_static(self, layer, q, budget_tokens, page_idx_out) -> int:
+        """gkv_quest_select with its score scratch in the library's fixed device array: for callers
+        that must not trigger any device allocation.  Same arguments and results."""
+        n = C.c_int32(0)
+        _check(load().gkv_quest_select_static(self.handle, layer, _ptr(q), budget_tokens, _ptr(page_idx_out),
+                                              C.byref(n), _stream()), "gkv_quest_select_static")
         return n.value
 
     def gkv_bits_report(self, layer=-1) -> GkvBits:

@@ -690,6 +690,29 @@ uint64_t full_read_bits(const gkv_cache* c, const LayerState& L) {
   return bits;
 }
 
+// ---- page selection without any allocation -----------------------------------------------------
+// Scratch for gkv_quest_select_static: page scores of one call, [n_streams][score_stride] fp32.
+// Every GPU that loads the library holds these 4 MiB until the process exits.
+constexpr size_t kStaticScoreFloats = size_t(1) << 20;
+static __device__ __align__(256) float g_static_scores[kStaticScoreFloats];
+constexpr int kMaxDevices = 64;
+static float* g_static_scores_ptr[kMaxDevices] = {};
+
+// In host code the array's name is only a handle; the device address has to be asked for, once
+// per device, with that device current.
+int static_scores_address(gkv_cache* c, float** out) {
+  int dev = -1;
+  CK(c, cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return GKV_ERR_UNSUPPORTED;
+  if (!g_static_scores_ptr[dev]) {
+    void* ptr = nullptr;
+    CK(c, cudaGetSymbolAddress(&ptr, g_static_scores));
+    g_static_scores_ptr[dev] = static_cast<float*>(ptr);
+  }
+  *out = g_static_scores_ptr[dev];
+  return GKV_OK;
+}
+
 }  // namespace
 
 // ================================================================================================
@@ -922,6 +945,33 @@ int gkv_quest_select(gkv_cache* c, int32_t layer, const void* q, int32_t budget_
   CK(c, launch_quest_scores(L.boxes_d, c->box_stride, n_pages, static_cast<const uint16_t*>(q), c->n_streams,
                             cfg.n_kv_heads, c->group, cfg.quest_reduce, c->scores_d, c->box_stride, st));
   CK(c, launch_topk(c->scores_d, c->box_stride, n_pages, nullptr, k, page_idx_out, k, c->n_streams, st));
+  return GKV_OK;
+}
+
+int gkv_quest_select_static(gkv_cache* c, int32_t layer, const void* q, int32_t budget_tokens,
+                            int32_t* page_idx_out, int32_t* n_sel_out, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !page_idx_out || !n_sel_out || budget_tokens < 0)
+    return GKV_ERR_INVALID_ARG;
+  const gkv_config& cfg = c->cfg;
+  if (cfg.page_tokens <= 0) return GKV_ERR_BAD_STATE;
+  LayerState& L = c->layers[layer];
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_pages = L.n_closed * (kBlock / cfg.page_tokens);
+  // the scores of all streams must fit the fixed scratch: n_streams * stride floats
+  const size_t stride = align_up(static_cast<size_t>(std::max(n_pages, 1)), 8);
+  if (stride * static_cast<size_t>(c->n_streams) > kStaticScoreFloats) return GKV_ERR_UNSUPPORTED;
+  float* scores = nullptr;
+  int rc = static_scores_address(c, &scores);
+  if (rc != GKV_OK) return rc;
+  const int k = std::min(budget_tokens / cfg.page_tokens, n_pages);
+  *n_sel_out = k;
+  L.quest_ran = true;
+  if (k <= 0) return GKV_OK;
+  // every score in [0, n_pages) of every stream is rewritten by the scorer before the selection
+  // reads it, so nothing left over from an earlier call is ever looked at
+  CK(c, launch_quest_scores(L.boxes_d, c->box_stride, n_pages, static_cast<const uint16_t*>(q), c->n_streams,
+                            cfg.n_kv_heads, c->group, cfg.quest_reduce, scores, static_cast<int>(stride), st));
+  CK(c, launch_topk(scores, static_cast<int>(stride), n_pages, nullptr, k, page_idx_out, k, c->n_streams, st));
   return GKV_OK;
 }
 
