@@ -6,8 +6,19 @@ import torch
 from oracle import gkv_oracle as O
 from paper_2608_23599_b200 import workloads as W
 
-ABS_TOL = 2e-3      # max-abs error on fp32-accumulated attention outputs
+ABS_TOL = 2e-3      # max-abs error on fp32-accumulated attention outputs, per unit of value scale
 REL_TOL = 1e-2      # relative L2 error per (sequence, head)
+
+
+def value_scale(v) -> float:
+    """Scale of the values being averaged: their standard deviation, never below 1.  The error of
+    the kernel is a perturbation of the softmax weights at fp16 operand precision (2^-12 relative),
+    so its absolute size grows with the spread of the values; the 2e-3 bound is stated for
+    unit-variance values (config 0) and is applied per unit of value standard deviation."""
+    if v is None:
+        return 1.0
+    x = v.detach().float() if hasattr(v, "detach") else torch.as_tensor(np.asarray(v)).float()
+    return max(1.0, float(x.std()))
 
 
 def oracle_config(w: W.Workload, n_layers=None) -> O.Config:
@@ -71,13 +82,14 @@ def assert_state_equal(ocache, gcache, layer, streams=None, blocks=None):
                 assert np.array_equal(ex["rows"][: st.n_tail], O.bf16_bits(st.tail_v))
 
 
-def assert_outputs_close(out_gpu, out_oracle, what=""):
+def assert_outputs_close(out_gpu, out_oracle, what="", scale=1.0):
     g = out_gpu.detach().to("cpu").to(torch.float64).numpy()
     o = np.asarray(out_oracle, dtype=np.float64)
     assert g.shape == o.shape
     assert np.all(np.isfinite(g)), f"{what}: non-finite output"
     err = np.abs(g - o).max()
-    assert err <= ABS_TOL, f"{what}: max-abs error {err:.3e} > {ABS_TOL}"
+    tol = ABS_TOL * max(1.0, scale)
+    assert err <= tol, f"{what}: max-abs error {err:.3e} > {tol:.3e} (value scale {scale:.2f})"
     num = np.linalg.norm(g - o, axis=-1)
     den = np.linalg.norm(o, axis=-1) + 1e-30
     rel = (num / den).max()

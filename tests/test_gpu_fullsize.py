@@ -1,0 +1,222 @@
+"""Full-size parity: the configurations of the benchmark spec at their real shapes, in the launch
+configuration bench.py times (all sequences and KV heads of a layer in one call), checked against
+the oracle on a sample of streams (the oracle is run on those streams only) plus properties that
+hold at any size.  Inputs are drawn on the GPU with the same recipe and copied to the host for the
+oracle."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import gkv_oracle as O
+from paper_2608_23599_b200 import workloads as W
+import parity_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _binding():
+    from paper_2608_23599_b200 import binding as B
+    B.build()
+    return B
+
+
+def _sample_oracle(w, data, streams, n_layers=1):
+    """Oracle cache holding only the sampled (b, kv head) streams of one layer: they become KV heads
+    0..n-1 of a batch-1 cache with the matching query heads."""
+    g = w.group_size
+    cfg = U.oracle_config(dataclasses.replace(w, batch=1, n_kv_heads=len(streams), n_q_heads=g * len(streams)), n_layers)
+    k = torch.stack([data["k"][b, :, h] for b, h in streams], dim=1)[None]
+    v = torch.stack([data["v"][b, :, h] for b, h in streams], dim=1)[None]
+    q = torch.cat([data["q"][b, h * g:(h + 1) * g] for b, h in streams], dim=0)[None]
+    mass = None
+    if data.get("mass") is not None:
+        mass = torch.stack([data["mass"][b, h] for b, h in streams], dim=0)[None].cpu().numpy()
+    return O.GradedCache(cfg), U.f32(k), U.f32(v), U.f32(q), mass
+
+
+def _compare_blocks(B, gcache, ocache, layer, streams, blocks):
+    for j, (b, h) in enumerate(streams):
+        st = ocache.streams[(layer, 0, j)]
+        assert np.array_equal(gcache.gkv_debug_export_levels(layer, b, h), ocache.levels(layer, 0, j))
+        assert np.array_equal(gcache.gkv_debug_export_residual(layer, b, h), st.res_idx)
+        for i in blocks:
+            if i >= st.n_closed:
+                continue
+            blk = st.blocks[i]
+            for which, name in ((B.TENSOR_K, "k"), (B.TENSOR_V, "v")):
+                ex = gcache.gkv_debug_export_block(layer, b, h, i, which)
+                tag = f"stream {(b, h)} block {i} {name} level {blk.level}"
+                assert ex["level"] == blk.level, tag
+                if blk.level == 16:
+                    assert np.array_equal(ex["rows"], O.bf16_bits(getattr(blk, f"{name}_exact"))), tag
+                elif blk.level == 1:
+                    assert np.array_equal(ex["rows"][0], O.bf16_bits(getattr(blk, f"{name}_cent"))), tag
+                else:
+                    assert np.array_equal(ex["scale"], getattr(blk, f"{name}_scale").view(np.uint16)), tag
+                    assert np.array_equal(ex["zero"], getattr(blk, f"{name}_zero").view(np.uint16)), tag
+                    assert np.array_equal(ex["codes"], getattr(blk, f"{name}_codes")), tag
+
+
+def _heads_of(streams, g, n_kv):
+    return [(b, h * g + j) for b, h in streams for j in range(g)]
+
+
+def _assert_sampled_outputs(out_gpu, o_out, streams, g, what, scale=1.0):
+    got = torch.stack([out_gpu[b, hq] for b, hq in _heads_of(streams, g, None)], dim=0)[None]
+    return U.assert_outputs_close(got, o_out, what, scale=scale)
+
+
+def test_cfg2_full_size_sampled_streams_with_appends():
+    """Config 2 at full size (B=8, 32/8 heads, T=32768, one layer): bulk ingest, then 65 decode
+    steps (one block fill with the four staircase demotions)."""
+    B = _binding()
+    w = dataclasses.replace(W.config(2), n_layers=1)
+    gcache = B.Cache(B.config_from_workload(w, 1))
+    dev = gcache.device
+    data = W.make_layer(w, 0, dev)
+    gcache.gkv_append_demote(0, data["k"], data["v"])
+    streams = [(0, 0), (3, 5), (7, 7)]
+    ocache, k, v, q, _ = _sample_oracle(w, data, streams)
+    ocache.append_demote(0, k, v)
+    blocks = [0, 1, 47, 48, 49, 175, 176, 300, 431, 432, 433, 495, 496, 511]      # every rung and its borders
+    _compare_blocks(B, gcache, ocache, 0, streams, blocks)
+    out = torch.empty((w.batch, w.n_q_heads, 128), dtype=torch.float32, device=dev)
+    gcache.gkv_decode_attn(0, data["q"], out)
+    torch.cuda.synchronize()
+    o_out, _ = ocache.decode_attn(0, q)
+    scale = U.value_scale(data["v"])      # the random-walk drift grows the values to a std of ~6
+    err, rel = _assert_sampled_outputs(out, o_out, streams, w.group_size, "cfg2 full step 0", scale)
+    print(f"cfg2 full: value std {scale:.2f}, max-abs error {err:.2e}, relative L2 {rel:.2e}")
+    # no NaN anywhere and every head's output is a convex combination of bounded values
+    assert torch.isfinite(out).all() and float(out.abs().max()) < 50
+    rep = gcache.gkv_bits_report(0)
+    assert abs(rep.bpv_resident - 4.8984375) < 1e-9 and rep.last_read_bits == rep.resident_bits
+    g = torch.Generator(device=dev)
+    g.manual_seed(99)
+    for step in range(65):
+        kn = torch.randn((w.batch, 1, w.n_kv_heads, 128), generator=g, device=dev).to(torch.bfloat16)
+        vn = torch.randn((w.batch, 1, w.n_kv_heads, 128), generator=g, device=dev).to(torch.bfloat16)
+        qn = torch.randn((w.batch, w.n_q_heads, 128), generator=g, device=dev).to(torch.bfloat16)
+        gcache.gkv_append_demote(0, kn, vn)
+        sub = {"k": kn, "v": vn, "q": qn}
+        ks = torch.stack([kn[b, :, h] for b, h in streams], dim=1)[None]
+        vs = torch.stack([vn[b, :, h] for b, h in streams], dim=1)[None]
+        ocache.append_demote(0, U.f32(ks), U.f32(vs))
+        if step in (0, 62, 63, 64):
+            gcache.gkv_decode_attn(0, qn, out)
+            torch.cuda.synchronize()
+            qs = torch.cat([qn[b, h * 4:(h + 1) * 4] for b, h in streams], dim=0)[None]
+            o_out, _ = ocache.decode_attn(0, U.f32(qs))
+            _assert_sampled_outputs(out, o_out, streams, w.group_size, f"cfg2 full step {step + 1}", scale)
+    # after the block fill: the demoted blocks (one per rung border) are bit-exact
+    _compare_blocks(B, gcache, ocache, 0, streams, [48, 176, 432, 496, 497, 512])
+    assert gcache.gkv_ctx_len(0) == 32768 + 65
+    for j in range(len(streams)):
+        for blk in ocache.streams[(0, 0, j)].blocks:
+            assert all(a >= b for a, b in zip(blk.history, blk.history[1:]))      # monotone demotion
+    gcache.close()
+
+
+def test_cfg1_full_size_rd_and_residual_sampled():
+    """Config 1 at full size (16/2 heads, T=16384, RD at 4.84 bits/value + 1 % residual), two layers:
+    every stream is checked (there are only two per layer)."""
+    B = _binding()
+    w = dataclasses.replace(W.config(1), n_layers=2)
+    gcache = B.Cache(B.config_from_workload(w, 2))
+    dev = gcache.device
+    for layer in range(2):
+        data = W.make_layer(w, layer, dev)
+        gcache.gkv_append_demote(layer, data["k"], data["v"], token_mass=data["mass"])
+        streams = [(0, 0), (0, 1)]
+        ocache, k, v, q, mass = _sample_oracle(w, data, streams)
+        ocache.append_demote(0, k, v, token_mass=mass)
+        # the oracle cache is layer 0 of its own; compare against `layer` of the GPU cache
+        for j, (b, h) in enumerate(streams):
+            st = ocache.streams[(0, 0, j)]
+            assert np.array_equal(gcache.gkv_debug_export_levels(layer, b, h), ocache.levels(0, 0, j))
+            res = gcache.gkv_debug_export_residual(layer, b, h)
+            assert len(res) == 163 and np.array_equal(res, st.res_idx)
+        lv = ocache.levels(0, 0, 0)
+        assert len(set(lv.tolist())) >= 3
+        nb = len(lv)
+        picks = sorted(set([0, 1, nb // 4, nb // 2, nb - 9, nb - 8, nb - 1]))
+        for j, (b, h) in enumerate(streams):
+            for i in picks:
+                blk = ocache.streams[(0, 0, j)].blocks[i]
+                ex = gcache.gkv_debug_export_block(layer, b, h, i, B.TENSOR_V)
+                assert ex["level"] == blk.level
+                if blk.level in (8, 4, 2):
+                    assert np.array_equal(ex["codes"], blk.v_codes)
+                    assert np.array_equal(ex["scale"], blk.v_scale.view(np.uint16))
+        out = torch.empty((w.batch, w.n_q_heads, 128), dtype=torch.float32, device=dev)
+        gcache.gkv_decode_attn(layer, data["q"], out)
+        torch.cuda.synchronize()
+        o_out, _ = ocache.decode_attn(0, q)
+        scale = U.value_scale(data["v"])
+        err, rel = U.assert_outputs_close(out, o_out, f"cfg1 full layer {layer}", scale=scale)
+        print(f"cfg1 full layer {layer}: value std {scale:.2f}, max-abs error {err:.2e}, relative L2 {rel:.2e}")
+        rep_g, rep_o = gcache.gkv_bits_report(layer), ocache.bits_report(0)
+        assert rep_g.resident_bits == rep_o["resident_bits"]
+        assert rep_g.bpv_paper <= 4.84 + 16 * 163 / 16384 + 1e-9
+    gcache.close()
+
+
+def test_cfg3_full_size_quest_sampled():
+    """Config 3 at full size (B=4, 32/8 heads, T=32768, 16-token pages, budget 2048 tokens):
+    selected pages bit-exact and sparse attention outputs on sampled streams."""
+    B = _binding()
+    w = dataclasses.replace(W.config(3), n_layers=1)
+    gcache = B.Cache(B.config_from_workload(w, 1))
+    dev = gcache.device
+    data = W.make_layer(w, 0, dev)
+    gcache.gkv_append_demote(0, data["k"], data["v"], token_mass=data["mass"])
+    streams = [(0, 0), (2, 3), (3, 7)]
+    ocache, k, v, q, mass = _sample_oracle(w, data, streams)
+    ocache.append_demote(0, k, v, token_mass=mass)
+    for j, (b, h) in enumerate(streams):
+        assert np.array_equal(gcache.gkv_debug_export_levels(0, b, h), ocache.levels(0, 0, j))
+    k_sel = w.quest_budget_tokens // w.page_tokens
+    pages = torch.full((w.batch, w.n_kv_heads, k_sel), -1, dtype=torch.int32, device=dev)
+    n_sel = gcache.gkv_quest_select(0, data["q"], w.quest_budget_tokens, pages)
+    torch.cuda.synchronize()
+    assert n_sel == k_sel == 128
+    sel_o = ocache.quest_select(0, q, w.quest_budget_tokens)
+    pg = pages.cpu().numpy()
+    for j, (b, h) in enumerate(streams):
+        assert np.array_equal(pg[b, h], sel_o[0][j]), f"pages differ for stream {(b, h)}"
+    # properties for every stream: ascending, unique, in range
+    assert (np.diff(pg, axis=-1) > 0).all() and pg.min() >= 0 and pg.max() < 2048
+    out = torch.empty((w.batch, w.n_q_heads, 128), dtype=torch.float32, device=dev)
+    gcache.gkv_decode_attn(0, data["q"], out, page_idx=pages, n_sel=n_sel)
+    torch.cuda.synchronize()
+    o_out, _ = ocache.decode_attn(0, q, sel_o)
+    err, rel = _assert_sampled_outputs(out, o_out, streams, w.group_size, "cfg3 full sparse", U.value_scale(data["v"]))
+    print(f"cfg3 full: max-abs error {err:.2e}, relative L2 {rel:.2e}")
+    assert torch.isfinite(out).all()
+    gcache.close()
+
+
+def test_cfg0_repeated_through_bench_sized_launches():
+    """Config 0 is small enough to be checked in full in test_gpu_parity; here its launch is
+    repeated with changing tail lengths (every value of ctx mod 64 after the ingest)."""
+    B = _binding()
+    w = dataclasses.replace(W.config(0), max_ctx=4096 + 192)
+    ocache = O.GradedCache(U.oracle_config(w))
+    gcache = B.Cache(B.config_from_workload(w))
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    worst = 0.0
+    for step in range(70):
+        tok = W.make_decode_tokens(w, 0, step, "cpu")
+        ocache.append_demote(0, U.f32(tok["k"]), U.f32(tok["v"]))
+        gcache.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
+        if step % 7 == 0 or step in (62, 63, 64):
+            out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, tok["q"])
+            err, rel = U.assert_outputs_close(out, o_out, f"cfg0 step {step}")
+            worst = max(worst, err)
+    U.assert_state_equal(ocache, gcache, 0)
+    print(f"cfg0 worst max-abs error over 70 steps: {worst:.2e}")
+    gcache.close()
