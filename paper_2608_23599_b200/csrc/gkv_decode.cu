@@ -973,8 +973,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
 }
 
 // Merge the partials of one (stream, query head): fixed ascending order, so results are
-// reproducible run to run.
+// reproducible run to run.  The (m, l) pairs are staged in shared memory with one round trip,
+// then every thread (one per channel) accumulates its column with independent, unrolled loads.
+constexpr int kCombineChunk = 128;
 __global__ void __launch_bounds__(kD) combine_kernel(const __grid_constant__ CombineParams p) {
+  __shared__ float sm_m[kCombineChunk], sm_w[kCombineChunk];
   const int stream = blockIdx.x, h = blockIdx.y, c = threadIdx.x;
   int begin, end;
   if (p.parts) {
@@ -984,16 +987,34 @@ __global__ void __launch_bounds__(kD) combine_kernel(const __grid_constant__ Com
     begin = stream * p.warps_per_stream;
     end = begin + p.warps_per_stream;
   }
+  const float* base = p.partial + h * (kD + 2);
+  // pass 1: global maximum of the partial maxima
+  float mloc = kNegInf;
+  for (int i = begin + c; i < end; i += kD) mloc = fmaxf(mloc, __ldcg(base + static_cast<size_t>(i) * kPartialFloats));
+  sm_m[c] = mloc;
+  __syncthreads();
   float M = kNegInf;
-  for (int i = begin; i < end; ++i) M = fmaxf(M, p.partial[static_cast<size_t>(i) * kPartialFloats + h * (kD + 2)]);
+#pragma unroll 8
+  for (int i = 0; i < kD; ++i) M = fmaxf(M, sm_m[i]);
+  // pass 2: chunks of up to 128 partials, weights in shared memory, columns in registers
   float L = 0.f, acc = 0.f;
-  for (int i = begin; i < end; ++i) {
-    const float* row = p.partial + static_cast<size_t>(i) * kPartialFloats + h * (kD + 2);
-    const float m = row[0];
-    if (m == kNegInf) continue;
-    const float wgt = exp2f(m - M);
-    L = fmaf(wgt, row[1], L);
-    acc = fmaf(wgt, row[2 + c], acc);
+  for (int c0 = begin; c0 < end; c0 += kCombineChunk) {
+    const int n = min(kCombineChunk, end - c0);
+    __syncthreads();
+    if (c < n) {
+      const float* row = base + static_cast<size_t>(c0 + c) * kPartialFloats;
+      const float m = __ldcg(row);
+      const float wgt = (m == kNegInf) ? 0.f : exp2f(m - M);
+      sm_w[c] = wgt;
+      sm_m[c] = wgt * __ldcg(row + 1);
+    }
+    __syncthreads();
+    const float* col = base + static_cast<size_t>(c0) * kPartialFloats + 2 + c;
+#pragma unroll 8
+    for (int i = 0; i < n; ++i) {
+      L += sm_m[i];
+      acc = fmaf(sm_w[i], __ldcg(col + static_cast<size_t>(i) * kPartialFloats), acc);
+    }
   }
   const int b = stream / p.n_kv_heads, kvh = stream - b * p.n_kv_heads;
   const size_t hq = static_cast<size_t>(b) * p.n_kv_heads * p.group + static_cast<size_t>(kvh) * p.group + h;
