@@ -393,26 +393,9 @@ void build_descs(gkv_cache* c, LayerState& L) {
   }
   const int padded = static_cast<int>(align_up(w, kDecodeWarps));
   for (int i = w; i < padded; ++i) L.warps_h[i] = WarpDesc{-1, 0, 0, 0};
-  // Deal the warps over the CTAs like cards, ordered by bytes per unit of cost: exact rows are
-  // bound by bytes, low-bit blocks by instruction issue, so every CTA (and SM) should hold a mix
-  // of both and overlap them instead of running one kind only.
-  const int n_ctas = padded / kDecodeWarps;
-  std::vector<std::pair<double, int>> order(padded);
-  for (int i = 0; i < padded; ++i) {
-    const WarpDesc& d = L.warps_h[i];
-    double bytes = 0, cost = 1;
-    if (d.stream >= 0)
-      for (int it = d.item_begin; it < d.item_end; ++it) {
-        cost += static_cast<double>(item_cost(c, L, d.stream, it));
-        bytes += it < L.n_closed ? slot_bytes(L.level[static_cast<size_t>(d.stream) * c->max_blocks + it]) : 8192;
-      }
-    order[i] = {d.stream >= 0 ? -bytes / cost : 1.0, i};
-  }
-  std::stable_sort(order.begin(), order.end());
-  std::vector<WarpDesc> dealt(padded);
-  for (int rank = 0; rank < padded; ++rank)
-    dealt[(rank % n_ctas) * kDecodeWarps + rank / n_ctas] = L.warps_h[order[rank].second];
-  std::memcpy(L.warps_h, dealt.data(), padded * sizeof(WarpDesc));
+  // Warps stay in stream order: the warps of a CTA then work on neighbouring blocks of the same
+  // level and share one code path, which keeps the instruction cache warm (dealing the levels
+  // across CTAs was measured to be slower).
   L.n_warps = padded;
   L.desc_dirty = false;
 }

@@ -28,7 +28,14 @@ constexpr unsigned kFull = 0xffffffffu;
 constexpr float kNegInf = -__builtin_huge_valf();
 constexpr int kRowPitch = kRowBytes + 16;       // staged exact rows: 272 B pitch -> conflict-free ldmatrix
 constexpr uint32_t kOnesH2 = 0x3C003C00u;       // half2(1, 1)
-constexpr int kWaitSpins = 1 << 22;             // bound of every mbarrier wait
+constexpr int kWaitSpins = 1 << 20;             // bound of every mbarrier wait (each poll may sleep up to the hint)
+#ifndef GKV_WAIT_HINT_NS
+#define GKV_WAIT_HINT_NS 2000
+#endif
+constexpr uint32_t kWaitHintNs = GKV_WAIT_HINT_NS;
+#ifndef GKV_L2_PREFETCH_AHEAD
+#define GKV_L2_PREFETCH_AHEAD 0
+#endif    // suspend-time hint of one poll, nanoseconds
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -45,16 +52,19 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(src), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n"
       ".reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
       "selp.u32 %0, 1, 0, p;\n"
       "}\n"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(kWaitHintNs)
       : "memory");
   return ok != 0;
 }
@@ -294,6 +304,19 @@ __device__ __forceinline__ bool load_item_dense(WarpCtx& w, int it, Cursor& c) {
       c.level = static_cast<int>(e.level);
       c.tmask = 15;
       c.ntok = kBlock;
+#if GKV_L2_PREFETCH_AHEAD > 0
+      {
+        // Pull a later item of this warp's range into L2 now: shared memory holds only two steps
+        // per warp, far less than HBM's bandwidth-delay product, so the DRAM latency is taken here,
+        // ahead of time, and the staged copies then hit L2.
+        const int ahead = it + GKV_L2_PREFETCH_AHEAD;
+        if (ahead < w.item_end && ahead < p.n_closed) {
+          const TableEntry pe = window_entry(w, ahead);
+          if (w.lane == 0 && pe.level != 1u)
+            bulk_prefetch_l2(p.arena + static_cast<size_t>(pe.off256) * 256, slot_bytes(static_cast<int>(pe.level)));
+        }
+      }
+#endif
       if (it == p.n_closed) {           // tail block: exact rows, n_tail of them
         c.level = 16;
         c.ntok = p.n_tail;
@@ -910,10 +933,13 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   int sidx = 0;
   uint32_t phase = 0;             // bit s = parity to wait for on stage s
   bool failed = false;
+#ifndef GKV_EXP_SKIP_COPY
   if (have) issue_step<SPARSE>(w, cur, 0);
+#endif
   while (have) {
     Cursor nxt = cur;
     const bool more = advance<SPARSE>(w, nxt);
+#ifndef GKV_EXP_SKIP_COPY
     if (more) issue_step<SPARSE>(w, nxt, sidx ^ 1);
     // bounded wait for this step's bytes
     int spins = 0;
@@ -923,10 +949,13 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
         break;
       }
     }
+#endif
     if (__any_sync(kFull, failed)) break;
     phase ^= 1u << sidx;
     __syncwarp();
+#ifndef GKV_EXP_SKIP_COMPUTE
     compute_step<SPARSE>(w, cur, sidx, qh, st, pf);
+#endif
     __syncwarp();
     cur = nxt;
     have = more;
