@@ -11,6 +11,7 @@
 
 #include "../../include/gkv.h"
 #include "gkv_internal.h"
+#include "gkv_mla.h"
 
 using namespace gkv;
 
@@ -23,14 +24,21 @@ constexpr size_t kMinWarpCost = 300;      // do not split below about one block 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int level_index(int level) { return level == 16 ? 0 : level == 8 ? 1 : level == 4 ? 2 : level == 2 ? 3 : 4; }
 constexpr int kLevels[5] = {16, 8, 4, 2, 1};
-inline uint32_t slot_units(int level) { return static_cast<uint32_t>(slot_bytes(level) / 256); }
-inline uint64_t block_bits(int level) { return static_cast<uint64_t>(slot_bytes(level)) * 8; }
+// Logical bits of one closed block (codes + fp16 scale/zero per group of 32, or one centroid row
+// per tensor, or exact rows); nval_tok = values per token (d_k + d_v, or d_k when V aliases K).
+inline uint64_t block_bits(int level, uint64_t nval_tok) {
+  if (level == 16) return 16ull * kBlock * nval_tok;
+  if (level == 1) return 16ull * nval_tok;
+  return static_cast<uint64_t>(level) * kBlock * nval_tok + (kBlock * nval_tok / kGroup) * 32ull;
+}
 
 // Segregated free lists over one heap of 256-byte units.  Slots are freed and reallocated by
 // size class; when the bump region is exhausted a larger free slot is split.
 struct SlotHeap {
   uint32_t begin = 0, end = 0, bump = 0;
+  uint32_t units[5] = {0, 0, 0, 0, 0};          // slot size per level (16, 8, 4, 2, 1) in 256-byte units
   std::vector<uint32_t> free_list[5];
+  uint32_t slot_units(int level) const { return units[level_index(level)]; }
   bool alloc(int level, uint32_t* off) {
     const int ci = level_index(level);
     if (!free_list[ci].empty()) {
@@ -124,6 +132,11 @@ struct gkv_cache {
 
 namespace {
 
+inline bool is_mla(const gkv_config& c) { return c.v_aliases_k != 0; }
+inline int geo_slot_bytes(const gkv_config& c, int level) { return is_mla(c) ? mla_slot_bytes(level) : slot_bytes(level); }
+inline uint64_t nval_per_token(const gkv_config& c) { return is_mla(c) ? c.d_k : c.d_k + c.d_v; }
+constexpr int kMlaTargetCtas = 148 * 2;
+
 struct ArenaPlan {
   size_t status, debug, partial, range, mass, levels, scores, kper, jobs, per_layer, heap_begin, total_meta;
   size_t l_table, l_warps, l_parts, l_resoff, l_rescount, l_residx, l_respool, l_boxes, layer_bytes;
@@ -140,8 +153,15 @@ int validate_config(const gkv_config* c) {
   if (c->n_q_heads % c->n_kv_heads != 0) return GKV_ERR_INVALID_ARG;
   if (c->max_ctx <= 0) return GKV_ERR_INVALID_ARG;
   if (c->block_tokens != kBlock || c->group != kGroup) return GKV_ERR_UNSUPPORTED;
-  if (c->d_k != kD || c->d_v != kD || c->v_aliases_k != 0) return GKV_ERR_UNSUPPORTED;
-  if (c->n_q_heads / c->n_kv_heads > kMaxHeadsPerKv) return GKV_ERR_UNSUPPORTED;
+  if (c->v_aliases_k) {
+    // latent attention: one 576-wide stream per sequence, 16 heads, values = channels [0, 512)
+    if (c->d_k != kMlaDk || c->d_v != kMlaDv || c->n_kv_heads != 1 || c->n_q_heads != kMlaHeads) return GKV_ERR_UNSUPPORTED;
+    if (c->page_tokens != 0 || c->residual_fraction != 0.f || c->policy == GKV_POLICY_RD) return GKV_ERR_UNSUPPORTED;
+    if (c->policy == GKV_POLICY_STAIRCASE && c->stair_tokens[3] != 0) return GKV_ERR_UNSUPPORTED;   // no 2-bit rung
+  } else {
+    if (c->d_k != kD || c->d_v != kD) return GKV_ERR_UNSUPPORTED;
+    if (c->n_q_heads / c->n_kv_heads > kMaxHeadsPerKv) return GKV_ERR_UNSUPPORTED;
+  }
   if (c->page_tokens != 0 && c->page_tokens != 16 && c->page_tokens != 32 && c->page_tokens != 64)
     return GKV_ERR_INVALID_ARG;
   if (c->policy < GKV_POLICY_STAIRCASE || c->policy > GKV_POLICY_EXTERNAL) return GKV_ERR_INVALID_ARG;
@@ -174,8 +194,9 @@ ArenaPlan plan_arena(const gkv_config& c, const Derived& d) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   a.status = take(256);
-  a.debug = take(kBlock * kD + 2 * 1024 + kBlock * kD * 2);
-  a.partial = take(static_cast<size_t>(d.max_warps) * kPartialFloats * sizeof(float));
+  a.debug = take(kBlock * kMlaDk + 2 * 4096 + kBlock * kMlaDk * 2);
+  a.partial = take(is_mla(c) ? static_cast<size_t>(kMlaTargetCtas + 2 * d.n_streams) * kMlaPartialFloats * sizeof(float)
+                             : static_cast<size_t>(d.max_warps) * kPartialFloats * sizeof(float));
   a.range = take(static_cast<size_t>(d.n_streams) * d.max_blocks * sizeof(float));
   a.mass = take(static_cast<size_t>(d.n_streams) * d.max_blocks * sizeof(float));
   a.levels = take(static_cast<size_t>(d.n_streams) * d.max_blocks);
@@ -233,10 +254,10 @@ size_t worst_stream_bytes(const gkv_config& c, const Derived& d) {
     // the population of each rung is bounded by its width (or by max_blocks when unbounded)
     std::vector<int8_t> lv(d.max_blocks);
     staircase_levels(c, d.max_blocks, lv.data());
-    for (int i = 0; i < d.max_blocks; ++i) bytes += slot_bytes(lv[i]);
-    for (int L : kLevels) bytes += 2 * slot_bytes(L);     // allocate-before-free slack + tail
+    for (int i = 0; i < d.max_blocks; ++i) bytes += geo_slot_bytes(c, lv[i]);
+    for (int L : kLevels) bytes += 2 * geo_slot_bytes(c, L);     // allocate-before-free slack + tail
   } else {
-    bytes = static_cast<size_t>(d.max_blocks + 2) * slot_bytes(16);
+    bytes = static_cast<size_t>(d.max_blocks + 2) * geo_slot_bytes(c, 16);
   }
   return bytes;
 }
@@ -313,7 +334,7 @@ bool rd_allocate(const gkv_config& c, const float* mass, const float* range, int
   auto feasible = [&](double tau) {
     rd_levels_for_tau(y, tau, pinned, nullptr, c.monotone_in_age != 0, lv);
     long long bits = tail_bits;
-    for (int b = 0; b < n; ++b) bits += static_cast<long long>(block_bits(lv[b]));
+    for (int b = 0; b < n; ++b) bits += static_cast<long long>(block_bits(lv[b], nval_tok));
     return bits <= budget_bits;
   };
   // bits(tau) never increases with tau, so the smallest feasible candidate is found by bisection
@@ -662,11 +683,223 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
   return GKV_OK;
 }
 
+
+// ---- latent-attention (MLA) host paths -----------------------------------------------------------
+// One stream per sequence; staircase or external plans only.  The block table, slot heap and
+// staging are shared with the GQA path; the kernels are those of gkv_mla.cu.
+size_t mla_item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) {
+  if (item < L.n_closed) {
+    switch (L.level[static_cast<size_t>(stream) * c->max_blocks + item]) {
+      case 16: return 1400;       // measured shares of a block's time on B200 (exact rows are byte-bound)
+      case 8: return 1000;
+      case 4: return 800;
+      default: return 60;
+    }
+  }
+  return 700;                     // tail
+}
+
+void mla_build_descs(gkv_cache* c, LayerState& L) {
+  const int ns = c->n_streams;
+  std::vector<size_t> cost(ns, 0);
+  size_t total = 0;
+  const int n_items = L.n_closed + 1;
+  for (int s = 0; s < ns; ++s) {
+    for (int i = 0; i < n_items; ++i) cost[s] += mla_item_cost(c, L, s, i);
+    total += cost[s];
+  }
+  const size_t target = std::max<size_t>(800, (total + kMlaTargetCtas - 1) / kMlaTargetCtas);
+  int w = 0;
+  for (int s = 0; s < ns; ++s) {
+    int nw = static_cast<int>((cost[s] + target / 2) / target);
+    nw = std::max(1, std::min(nw, n_items));
+    nw = std::min(nw, kMlaTargetCtas + 2 * ns - w - (ns - 1 - s));
+    L.parts_h[s].begin = w;
+    size_t acc = 0;
+    int item = 0;
+    for (int k = 0; k < nw; ++k) {
+      const size_t limit = cost[s] * (k + 1) / nw;
+      const int begin = item;
+      const int max_end = n_items - (nw - 1 - k);
+      do {
+        acc += mla_item_cost(c, L, s, item);
+        ++item;
+      } while (item < max_end && acc < limit);
+      L.warps_h[w] = WarpDesc{s, begin, item, w};
+      ++w;
+    }
+    L.warps_h[w - 1].item_end = n_items;
+    L.parts_h[s].end = w;
+  }
+  L.n_warps = w;                  // here: number of CTAs
+  L.desc_dirty = false;
+}
+
+int mla_bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, int n_new, const int8_t* level_plan, cudaStream_t st) {
+  const gkv_config& cfg = c->cfg;
+  LayerState& L = c->layers[layer];
+  const int ns = c->n_streams, n_closed = n_new / kBlock, n_tail = n_new % kBlock;
+  int rc;
+  if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
+  if ((rc = wait_event(c, c->ev_stage)) != GKV_OK) return rc;
+  std::fill(L.level.begin(), L.level.end(), 0);
+  if (cfg.policy == GKV_POLICY_STAIRCASE) {
+    std::vector<int8_t> lv(std::max(n_closed, 1));
+    staircase_levels(cfg, n_closed, lv.data());
+    for (int s = 0; s < ns; ++s) std::memcpy(&L.level[static_cast<size_t>(s) * c->max_blocks], lv.data(), n_closed);
+  } else {
+    for (int s = 0; s < ns; ++s)
+      for (int b = 0; b < n_closed; ++b) {
+        const int8_t v = level_plan[static_cast<size_t>(s) * n_closed + b];
+        if (v != 16 && v != 8 && v != 4 && v != 1) return v == 2 ? GKV_ERR_UNSUPPORTED : GKV_ERR_INVALID_ARG;
+        L.level[static_cast<size_t>(s) * c->max_blocks + b] = v;
+      }
+  }
+  for (int s = 0; s < ns; ++s) {
+    for (int b = 0; b <= n_closed; ++b) {
+      const int lvl = b < n_closed ? L.level[static_cast<size_t>(s) * c->max_blocks + b] : 16;
+      uint32_t off;
+      if (!c->heap.alloc(lvl, &off)) return GKV_ERR_ARENA_TOO_SMALL;
+      set_entry(c, L, s, b, off, lvl);
+      L.table_h[static_cast<size_t>(s) * c->table_stride + b].resmask = 0;
+    }
+    L.res_count_h[s] = 0;
+  }
+  L.has_tail_slot = true;
+  if ((rc = upload(c, L.table_d, L.table_h, static_cast<size_t>(ns) * c->table_stride * sizeof(TableEntry), st, L.ev)) != GKV_OK) return rc;
+  const size_t n_jobs = static_cast<size_t>(ns) * n_closed;
+  if (n_jobs > 0) {
+    EncodeJob* jobs = reinterpret_cast<EncodeJob*>(c->stage_h);
+    size_t j = 0;
+    for (int s = 0; s < ns; ++s)
+      for (int b = 0; b < n_closed; ++b) {
+        EncodeJob& job = jobs[j++];
+        job.src_off256 = 0;
+        job.dst_off256 = L.table_h[static_cast<size_t>(s) * c->table_stride + b].off256;
+        job.src_level = 0;
+        job.dst_level = L.level[static_cast<size_t>(s) * c->max_blocks + b];
+        job.stream = s;
+        job.block = b;
+        job.pad = 0;
+      }
+    CK(c, cudaMemcpyAsync(c->jobs_d, jobs, n_jobs * sizeof(EncodeJob), cudaMemcpyHostToDevice, st));
+    MlaEncodeParams ep{};
+    ep.arena = c->arena;
+    ep.jobs = c->jobs_d;
+    ep.n_jobs = static_cast<int32_t>(n_jobs);
+    ep.k_in = k_new;
+    ep.n_tok = n_new;
+    ep.status = c->status_d;
+    CK(c, launch_mla_encode(ep, st));
+  }
+  CK(c, cudaEventRecord(c->ev_stage, st));
+  CK(c, launch_mla_append_rows(c->arena, L.table_d, c->table_stride, n_closed, ns, k_new, n_new, n_closed * kBlock, n_tail, 0, st));
+  L.n_closed = n_closed;
+  L.n_tail = n_tail;
+  L.desc_dirty = true;
+  L.last_mode = 0;
+  return GKV_OK;
+}
+
+int mla_append_one(gkv_cache* c, int layer, const uint16_t* k_new, cudaStream_t st) {
+  const gkv_config& cfg = c->cfg;
+  LayerState& L = c->layers[layer];
+  const int ns = c->n_streams;
+  int rc;
+  const size_t table_bytes = static_cast<size_t>(ns) * c->table_stride * sizeof(TableEntry);
+  if (!L.has_tail_slot) {
+    if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
+    for (int s = 0; s < ns; ++s) {
+      uint32_t off;
+      if (!c->heap.alloc(16, &off)) return GKV_ERR_ARENA_TOO_SMALL;
+      set_entry(c, L, s, L.n_closed, off, 16);
+      L.table_h[static_cast<size_t>(s) * c->table_stride + L.n_closed].resmask = 0;
+    }
+    L.has_tail_slot = true;
+    if ((rc = upload(c, L.table_d, L.table_h, table_bytes, st, L.ev)) != GKV_OK) return rc;
+    L.desc_dirty = true;
+  }
+  CK(c, launch_mla_append_rows(c->arena, L.table_d, c->table_stride, L.n_closed, ns, k_new, 1, 0, 1, L.n_tail, st));
+  L.n_tail += 1;
+  if (L.n_tail < kBlock) return GKV_OK;
+  const int closed_block = L.n_closed;
+  for (int s = 0; s < ns; ++s) L.level[static_cast<size_t>(s) * c->max_blocks + closed_block] = 16;
+  L.n_closed += 1;
+  L.n_tail = 0;
+  L.has_tail_slot = false;
+  L.desc_dirty = true;
+  if (cfg.policy != GKV_POLICY_STAIRCASE) return GKV_OK;
+  std::vector<int8_t> target(L.n_closed);
+  staircase_levels(cfg, L.n_closed, target.data());
+  if ((rc = wait_event(c, c->ev_stage)) != GKV_OK) return rc;
+  if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
+  EncodeJob* jobs = reinterpret_cast<EncodeJob*>(c->stage_h);
+  size_t n_jobs = 0;
+  std::vector<std::pair<int, uint32_t>> to_free;
+  for (int s = 0; s < ns; ++s)
+    for (int b = 0; b < L.n_closed; ++b) {
+      int8_t& cur = L.level[static_cast<size_t>(s) * c->max_blocks + b];
+      if (target[b] >= cur) continue;
+      TableEntry& e = L.table_h[static_cast<size_t>(s) * c->table_stride + b];
+      uint32_t off;
+      if (!c->heap.alloc(target[b], &off)) return GKV_ERR_ARENA_TOO_SMALL;
+      EncodeJob& job = jobs[n_jobs++];
+      job.src_off256 = e.off256;
+      job.dst_off256 = off;
+      job.src_level = cur;
+      job.dst_level = target[b];
+      job.stream = s;
+      job.block = b;
+      job.pad = 0;
+      to_free.emplace_back(cur, e.off256);
+      e.off256 = off;
+      e.level = static_cast<uint32_t>(target[b]);
+      cur = target[b];
+    }
+  if (n_jobs > 0) {
+    CK(c, cudaMemcpyAsync(c->jobs_d, jobs, n_jobs * sizeof(EncodeJob), cudaMemcpyHostToDevice, st));
+    CK(c, cudaEventRecord(c->ev_stage, st));
+    MlaEncodeParams ep{};
+    ep.arena = c->arena;
+    ep.jobs = c->jobs_d;
+    ep.n_jobs = static_cast<int32_t>(n_jobs);
+    ep.status = c->status_d;
+    CK(c, launch_mla_encode(ep, st));
+    for (auto& f : to_free) c->heap.release(f.first, f.second);
+    if ((rc = upload(c, L.table_d, L.table_h, table_bytes, st, L.ev)) != GKV_OK) return rc;
+  }
+  return GKV_OK;
+}
+
+int mla_decode(gkv_cache* c, LayerState& L, const void* q, float* out, float* lse, cudaStream_t st) {
+  if (L.desc_dirty) {
+    int rc = wait_event(c, L.ev);
+    if (rc != GKV_OK) return rc;
+    mla_build_descs(c, L);
+    if ((rc = upload(c, L.warps_d, L.warps_h, static_cast<size_t>(L.n_warps) * sizeof(WarpDesc), st, L.ev)) != GKV_OK) return rc;
+    if ((rc = upload(c, L.parts_d, L.parts_h, static_cast<size_t>(c->n_streams) * sizeof(StreamParts), st, L.ev)) != GKV_OK) return rc;
+  }
+  MlaDecodeParams p{};
+  p.arena = c->arena;
+  p.table = L.table_d;
+  p.ctas = L.warps_d;
+  p.q = static_cast<const uint16_t*>(q);
+  p.partial = c->partial_d;
+  p.table_stride = c->table_stride;
+  p.n_closed = L.n_closed;
+  p.n_tail = L.n_tail;
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  p.status = c->status_d;
+  L.last_mode = 1;
+  CK(c, launch_mla_decode(p, L.n_warps, L.parts_d, c->n_streams, out, lse, st));
+  return GKV_OK;
+}
+
 uint64_t full_read_bits(const gkv_cache* c, const LayerState& L) {
-  const uint64_t nval_tok = c->cfg.d_k + c->cfg.d_v;
+  const uint64_t nval_tok = nval_per_token(c->cfg);
   uint64_t bits = 0;
   for (int s = 0; s < c->n_streams; ++s) {
-    for (int b = 0; b < L.n_closed; ++b) bits += block_bits(L.level[static_cast<size_t>(s) * c->max_blocks + b]);
+    for (int b = 0; b < L.n_closed; ++b) bits += block_bits(L.level[static_cast<size_t>(s) * c->max_blocks + b], nval_tok);
     bits += static_cast<uint64_t>(L.n_tail) * 16 * nval_tok;
     bits += static_cast<uint64_t>(L.res_count_h[s]) * 16 * nval_tok;
   }
@@ -735,7 +968,7 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
   if (!arena || !out || (reinterpret_cast<uintptr_t>(arena) & 255)) return GKV_ERR_INVALID_ARG;
   const Derived d = derive(*cfg);
   const ArenaPlan a = plan_arena(*cfg, d);
-  if (arena_bytes < a.heap_begin + slot_bytes(16)) return GKV_ERR_ARENA_TOO_SMALL;
+  if (arena_bytes < a.heap_begin + geo_slot_bytes(*cfg, 16)) return GKV_ERR_ARENA_TOO_SMALL;
   if ((arena_bytes / 256) > 0xffffffffull) return GKV_ERR_UNSUPPORTED;
   gkv_cache* c = new (std::nothrow) gkv_cache();
   if (!c) return GKV_ERR_INVALID_ARG;
@@ -750,6 +983,7 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
   c->res_cap = d.res_cap;
   c->box_stride = d.box_stride;
   c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : static_cast<float>(1.0 / std::sqrt(static_cast<double>(cfg->d_k)));
+  for (int i = 0; i < 5; ++i) c->heap.units[i] = static_cast<uint32_t>(geo_slot_bytes(*cfg, kLevels[i]) / 256);
   c->heap.begin = c->heap.bump = static_cast<uint32_t>(a.heap_begin / 256);
   c->heap.end = static_cast<uint32_t>(arena_bytes / 256);
   c->status_d = reinterpret_cast<uint32_t*>(c->arena + a.status);
@@ -833,11 +1067,18 @@ int gkv_ctx_len(gkv_cache* c, int32_t layer, int32_t* ctx) {
 
 int gkv_append_demote(gkv_cache* c, int32_t layer, const void* k_new, const void* v_new, int32_t n_new,
                       const float* token_mass, const int8_t* level_plan, void* stream) {
-  if (!c || layer < 0 || layer >= c->cfg.n_layers || !k_new || !v_new || n_new <= 0) return GKV_ERR_INVALID_ARG;
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !k_new || n_new <= 0) return GKV_ERR_INVALID_ARG;
+  if (is_mla(c->cfg) ? (v_new != nullptr) : (v_new == nullptr)) return GKV_ERR_INVALID_ARG;
   LayerState& L = c->layers[layer];
   const int ctx = L.n_closed * kBlock + L.n_tail;
   if (static_cast<long long>(ctx) + n_new > c->cfg.max_ctx) return GKV_ERR_CTX_FULL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (is_mla(c->cfg)) {
+    if (n_new == 1) return mla_append_one(c, layer, static_cast<const uint16_t*>(k_new), st);
+    if (ctx != 0) return GKV_ERR_BAD_STATE;
+    if (c->cfg.policy == GKV_POLICY_EXTERNAL && !level_plan && n_new >= kBlock) return GKV_ERR_INVALID_ARG;
+    return mla_bulk_ingest(c, layer, static_cast<const uint16_t*>(k_new), n_new, level_plan, st);
+  }
   if (n_new == 1) return append_one(c, layer, static_cast<const uint16_t*>(k_new), static_cast<const uint16_t*>(v_new), st);
   if (ctx != 0) return GKV_ERR_BAD_STATE;
   if (c->cfg.policy == GKV_POLICY_RD && !token_mass) return GKV_ERR_INVALID_ARG;
@@ -854,6 +1095,10 @@ int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* p
   if (L.n_closed * kBlock + L.n_tail == 0) return GKV_ERR_BAD_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const gkv_config& cfg = c->cfg;
+  if (is_mla(cfg)) {
+    if (page_idx) return GKV_ERR_BAD_STATE;
+    return mla_decode(c, L, q, out, lse, st);
+  }
   DecodeParams p{};
   p.arena = c->arena;
   p.table = L.table_d;
@@ -962,7 +1207,7 @@ int gkv_bits_report(gkv_cache* c, int32_t layer, gkv_bits* out) {
   if (!c || !out || layer < -1 || layer >= c->cfg.n_layers) return GKV_ERR_INVALID_ARG;
   std::memset(out, 0, sizeof(*out));
   const gkv_config& cfg = c->cfg;
-  const uint64_t nval_tok = cfg.d_k + cfg.d_v;
+  const uint64_t nval_tok = nval_per_token(cfg);
   const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? cfg.n_layers : layer + 1;
   int warn = GKV_OK;
   for (int l = l0; l < l1; ++l) {
@@ -1073,6 +1318,25 @@ int gkv_debug_export_block(gkv_cache* c, int32_t layer, int32_t b, int32_t kv_he
   if (level) *level = lv;
   if (n_rows) *n_rows = block == L.n_closed ? L.n_tail : (lv == 1 ? 1 : kBlock);
   CK(c, cudaDeviceSynchronize());
+  if (is_mla(c->cfg)) {
+    if (which != GKV_TENSOR_K) return GKV_ERR_INVALID_ARG;     // values are channels [0, 512) of the key row
+    uint8_t* m_codes = c->debug_d;
+    uint16_t* m_scale = reinterpret_cast<uint16_t*>(c->debug_d + kBlock * kMlaDk);
+    uint16_t* m_zero = reinterpret_cast<uint16_t*>(c->debug_d + kBlock * kMlaDk + 4096);
+    uint16_t* m_rows = reinterpret_cast<uint16_t*>(c->debug_d + kBlock * kMlaDk + 8192);
+    CK(c, launch_mla_export(c->arena, e.off256, lv, m_codes, m_scale, m_zero, m_rows, 0));
+    CK(c, cudaDeviceSynchronize());
+    if (lv == 16) {
+      if (rows_bf16) CK(c, cudaMemcpy(rows_bf16, m_rows, kBlock * kMlaDk * 2, cudaMemcpyDeviceToHost));
+    } else if (lv == 1) {
+      if (rows_bf16) CK(c, cudaMemcpy(rows_bf16, m_rows, kMlaDk * 2, cudaMemcpyDeviceToHost));
+    } else {
+      if (codes) CK(c, cudaMemcpy(codes, m_codes, kBlock * kMlaDk, cudaMemcpyDeviceToHost));
+      if (scale_fp16) CK(c, cudaMemcpy(scale_fp16, m_scale, 2 * kMlaDk * 2, cudaMemcpyDeviceToHost));
+      if (zero_fp16) CK(c, cudaMemcpy(zero_fp16, m_zero, 2 * kMlaDk * 2, cudaMemcpyDeviceToHost));
+    }
+    return GKV_OK;
+  }
   uint8_t* d_codes = c->debug_d;
   uint16_t* d_scale = reinterpret_cast<uint16_t*>(c->debug_d + kBlock * kD);
   uint16_t* d_zero = reinterpret_cast<uint16_t*>(c->debug_d + kBlock * kD + 1024);

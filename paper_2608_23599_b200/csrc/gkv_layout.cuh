@@ -123,3 +123,31 @@ GKV_HD int vp_zero_index(int t16, int grp) {
 }
 
 }  // namespace gkv
+
+// ---- latent-attention (MLA) streams: one 576-wide row per token, values = channels [0, 512) ----
+// The row is quantised once with the key rule (32 tokens x 1 channel per group).  Codes are stored
+// in the K-role fragment order above with 36 MMA indices (16 channels each); the value role reads
+// the same codes and transposes the 8x8 fragments in registers.  Words are stored word-major:
+// word w of a lane lives at byte (w * 32 + lane) * 4 of the tile's code region.
+namespace gkv {
+constexpr int kMlaDk = 576, kMlaDv = 512, kMlaHeads = 16, kMlaKSteps = kMlaDk / 16;   // 36
+constexpr int kMlaRowBytes = kMlaDk * 2;                                              // 1152
+GKV_HD int mla_code_bytes_per_tile(int bits) { return kMlaKSteps * 8 * bits * 32 / 8; }   // 1152 * bits
+GKV_HD int mla_kp_bytes() { return kMlaKSteps * 4 * 16; }                                 // 2304 per half
+GKV_HD int mla_half_bytes(int bits) { return mla_kp_bytes() + 2 * mla_code_bytes_per_tile(bits); }
+GKV_HD int mla_slot_bytes(int level) {
+  return level == 16 ? kBlock * kMlaRowBytes : (level == 1 ? 1280 : 2 * mla_half_bytes(level));
+}
+GKV_HD void mla_code_pos(int bits, int lane, int s, int a, int hlf, int* byte_off, int* bit) {
+  int w, b;
+  if (bits == 8) {
+    w = 2 * s + (a >> 1);
+    b = 8 * (a & 1);
+  } else {
+    w = s;
+    b = 4 * a;
+  }
+  *byte_off = (w * 32 + lane) * 4;
+  *bit = b + 16 * hlf;
+}
+}  // namespace gkv

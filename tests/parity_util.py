@@ -10,15 +10,18 @@ ABS_TOL = 2e-3      # max-abs error on fp32-accumulated attention outputs, per u
 REL_TOL = 1e-2      # relative L2 error per (sequence, head)
 
 
-def value_scale(v) -> float:
-    """Scale of the values being averaged: their standard deviation, never below 1.  The error of
-    the kernel is a perturbation of the softmax weights at fp16 operand precision (2^-12 relative),
-    so its absolute size grows with the spread of the values; the 2e-3 bound is stated for
-    unit-variance values (config 0) and is applied per unit of value standard deviation."""
+def value_scale(v):
+    """Scale of the values being averaged, per output channel: the standard deviation of that
+    channel over all tokens and streams, never below 1.  The error of the kernel is a perturbation
+    of the softmax weights at fp16 operand precision (2^-12 relative), so on every channel its
+    absolute size grows with the spread of that channel's values; the 2e-3 bound is stated for
+    unit-variance values (config 0) and is applied per unit of value standard deviation.
+    v: [..., channels] (torch or numpy); returns a numpy vector [channels]."""
     if v is None:
         return 1.0
-    x = v.detach().float() if hasattr(v, "detach") else torch.as_tensor(np.asarray(v)).float()
-    return max(1.0, float(x.std()))
+    x = v.detach().float().cpu() if hasattr(v, "detach") else torch.as_tensor(np.asarray(v)).float()
+    sd = x.reshape(-1, x.shape[-1]).std(dim=0).numpy().astype(np.float64)
+    return np.maximum(1.0, sd)
 
 
 def oracle_config(w: W.Workload, n_layers=None) -> O.Config:
@@ -36,10 +39,10 @@ def f32(t):
 def ingest_both(w, layer, data, ocache, gcache, level_plan=None):
     """data: dict from workloads.make_layer on CPU."""
     mass = data.get("mass")
-    ocache.append_demote(layer, f32(data["k"]), f32(data["v"]),
+    ocache.append_demote(layer, f32(data["k"]), f32(data.get("v")),
                          token_mass=None if mass is None else mass.numpy(), level_plan=level_plan)
     dev = gcache.device
-    gcache.gkv_append_demote(layer, data["k"].to(dev), data["v"].to(dev),
+    gcache.gkv_append_demote(layer, data["k"].to(dev), None if data.get("v") is None else data["v"].to(dev),
                              token_mass=None if mass is None else mass.to(dev).contiguous(),
                              level_plan=level_plan)
 
@@ -60,7 +63,8 @@ def assert_state_equal(ocache, gcache, layer, streams=None, blocks=None):
             todo = range(st.n_closed) if blocks is None else [i for i in blocks if i < st.n_closed]
             for i in todo:
                 blk = st.blocks[i]
-                for which, name in ((B.TENSOR_K, "k"), (B.TENSOR_V, "v")):
+                tensors = ((B.TENSOR_K, "k"),) if cfg.v_aliases_k else ((B.TENSOR_K, "k"), (B.TENSOR_V, "v"))
+                for which, name in tensors:
                     ex = gcache.gkv_debug_export_block(layer, b, h, i, which)
                     assert ex["level"] == blk.level
                     tag = f"layer {layer} stream {(b, h)} block {i} {name} level {blk.level}"
@@ -78,8 +82,9 @@ def assert_state_equal(ocache, gcache, layer, streams=None, blocks=None):
                 ex = gcache.gkv_debug_export_block(layer, b, h, st.n_closed, B.TENSOR_K)
                 assert ex["n_rows"] == st.n_tail
                 assert np.array_equal(ex["rows"][: st.n_tail], O.bf16_bits(st.tail_k))
-                ex = gcache.gkv_debug_export_block(layer, b, h, st.n_closed, B.TENSOR_V)
-                assert np.array_equal(ex["rows"][: st.n_tail], O.bf16_bits(st.tail_v))
+                if not cfg.v_aliases_k:
+                    ex = gcache.gkv_debug_export_block(layer, b, h, st.n_closed, B.TENSOR_V)
+                    assert np.array_equal(ex["rows"][: st.n_tail], O.bf16_bits(st.tail_v))
 
 
 def assert_outputs_close(out_gpu, out_oracle, what="", scale=1.0):
@@ -87,9 +92,11 @@ def assert_outputs_close(out_gpu, out_oracle, what="", scale=1.0):
     o = np.asarray(out_oracle, dtype=np.float64)
     assert g.shape == o.shape
     assert np.all(np.isfinite(g)), f"{what}: non-finite output"
+    scale = np.maximum(1.0, np.asarray(scale, dtype=np.float64))        # scalar or per channel
+    nerr = (np.abs(g - o) / scale).max()
     err = np.abs(g - o).max()
-    tol = ABS_TOL * max(1.0, scale)
-    assert err <= tol, f"{what}: max-abs error {err:.3e} > {tol:.3e} (value scale {scale:.2f})"
+    assert nerr <= ABS_TOL, (f"{what}: max-abs error per unit of value scale {nerr:.3e} > {ABS_TOL} "
+                             f"(raw max-abs {err:.3e}, value scale up to {float(np.max(scale)):.2f})")
     num = np.linalg.norm(g - o, axis=-1)
     den = np.linalg.norm(o, axis=-1) + 1e-30
     rel = (num / den).max()

@@ -231,3 +231,55 @@ def test_host_side_errors():
         full.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
     assert e.value.status == -3
     full.close()
+
+
+# ---- latent attention (MLA): 576-wide stream, 16 heads, values = key channels [0, 512) --------------
+def _mla(T, **kw):
+    base = dict(name="mla_tiny", config_id=14, n_layers=1, batch=2, n_q_heads=16, n_kv_heads=1, d_k=576, d_v=512,
+                ctx=T, max_ctx=T + 256, v_aliases_k=1, softmax_scale=1.0 / 192 ** 0.5, n_outlier=8, outlier_gain=6.0,
+                n_heavy=0)
+    base.update(kw)
+    return W.Workload(**base)
+
+
+@pytest.mark.parametrize("level", [16, 8, 4, 1])
+@pytest.mark.parametrize("T", [64, 200, 1100])
+def test_mla_single_tier(level, T):
+    w = _mla(T, policy=W.POLICY_EXTERNAL)
+    ocache, gcache = _pair(w)
+    data = W.make_layer(w, 0, "cpu")
+    plan = np.full((w.batch, 1, T // 64), level, dtype=np.int8)
+    U.ingest_both(w, 0, data, ocache, gcache, level_plan=plan)
+    U.assert_state_equal(ocache, gcache, 0)
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
+    U.assert_outputs_close(out, o_out, f"mla level {level} T {T}", scale=U.value_scale(data["k"][..., :512]))
+    assert np.max(np.abs(lse.cpu().numpy() - o_lse)) < 5e-3
+    rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
+    assert rep_g.resident_bits == rep_o["resident_bits"] and rep_g.last_read_bits == rep_o["last_read_bits"]
+    gcache.close()
+
+
+def test_cfg4_small_mla_ladder_with_appends():
+    """Config 4 structure at small size: exact newest rung, int8, int4, centroid for the oldest
+    quarter (5.0 bits/value), then appends with staircase demotion."""
+    w = W.config(4, "small")
+    ocache, gcache = _pair(w)
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    U.assert_state_equal(ocache, gcache, 0)
+    rep = gcache.gkv_bits_report(0)
+    assert abs(rep.bpv_resident - 5.0) < 0.01 and rep.blocks_by_level[3] == 0 and rep.blocks_by_level[4] == 32
+    scale = U.value_scale(data["k"][..., :512])
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
+    err, rel = U.assert_outputs_close(out, o_out, "cfg4-small", scale=scale)
+    for step in range(66):
+        tok = W.make_decode_tokens(w, 0, step, "cpu")
+        ocache.append_demote(0, U.f32(tok["k"]), None)
+        gcache.gkv_append_demote(0, tok["k"].to(dev), None)
+        if step in (0, 31, 62, 63, 64, 65):
+            out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, tok["q"])
+            U.assert_outputs_close(out, o_out, f"cfg4-small step {step}", scale=scale)
+    U.assert_state_equal(ocache, gcache, 0)
+    assert gcache.gkv_bits_report(0).resident_bits == ocache.bits_report(0)["resident_bits"]
+    gcache.close()
