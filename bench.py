@@ -141,7 +141,7 @@ def build_cache(w: W.Workload, n_layers: int, extra_ctx: int, device):
     qs = []
     for layer in range(n_layers):
         data = W.make_layer(wl, layer, device)
-        cache.gkv_append_demote(layer, data["k"], data["v"], token_mass=data.get("mass"))
+        cache.gkv_append_demote(layer, data["k"], data.get("v"), token_mass=data.get("mass"))
         qs.append(data["q"])
         del data
     torch.cuda.synchronize()
@@ -158,21 +158,22 @@ def run_ours(args, rank, local, world):
     K, Wm = args.steps, args.warmup
     total_steps = 2 * (K + Wm) + 8
     wl, cache, q0 = build_cache(w, n_layers, total_steps + 64, device)
-    Bsz, Hq, Hkv, d = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.d_k
+    Bsz, Hq, Hkv, d, dv = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.d_k, wl.d_v
+    alias = bool(wl.v_aliases_k)
     gen = torch.Generator(device=device)
     gen.manual_seed(4242 + rank)
     # per-step decode inputs, resident in HBM for the device-timed region
     k_new = torch.randn((total_steps, n_layers, Bsz, 1, Hkv, d), generator=gen, device=device).to(torch.bfloat16)
-    v_new = torch.randn((total_steps, n_layers, Bsz, 1, Hkv, d), generator=gen, device=device).to(torch.bfloat16)
+    v_new = None if alias else torch.randn((total_steps, n_layers, Bsz, 1, Hkv, dv), generator=gen, device=device).to(torch.bfloat16)
     q_new = torch.randn((total_steps, n_layers, Bsz, Hq, d), generator=gen, device=device).to(torch.bfloat16)
-    out = torch.empty((n_layers, Bsz, Hq, d), dtype=torch.float32, device=device)
+    out = torch.empty((n_layers, Bsz, Hq, dv), dtype=torch.float32, device=device)
     quest = wl.page_tokens > 0 and wl.quest_budget_tokens > 0
     k_sel = wl.quest_budget_tokens // wl.page_tokens if quest else 0
     pages = torch.zeros((Bsz, Hkv, max(k_sel, 1)), dtype=torch.int32, device=device) if quest else None
 
     def step_device(s):
         for l in range(n_layers):
-            cache.gkv_append_demote(l, k_new[s, l], v_new[s, l])
+            cache.gkv_append_demote(l, k_new[s, l], None if alias else v_new[s, l])
             if quest:
                 n_sel = cache.gkv_quest_select(l, q_new[s, l], wl.quest_budget_tokens, pages)
                 cache.gkv_decode_attn(l, q_new[s, l], out[l], page_idx=pages, n_sel=n_sel)
@@ -204,7 +205,7 @@ def run_ours(args, rank, local, world):
 
     # ---- dominant kernel: decode_attn alone, per launch -------------------------------------------
     rep = cache.gkv_bits_report(0)
-    algo_bytes = rep.last_read_bits / 8 + Bsz * Hq * d * 2 + Bsz * Hq * d * 4
+    algo_bytes = rep.last_read_bits / 8 + Bsz * Hq * d * 2 + Bsz * Hq * dv * 4
     if quest:
         algo_bytes = (rep.last_read_bits - rep.box_bits) / 8 + Bsz * Hq * d * 6
     reps = max(3, min(20, int(2e10 / max(algo_bytes * n_layers, 1))))
@@ -231,17 +232,18 @@ def run_ours(args, rank, local, world):
 
     # ---- end to end: host buffers, H2D of the step's inputs and D2H of its result inside the region
     hk = torch.randn((n_layers, Bsz, 1, Hkv, d)).to(torch.bfloat16).pin_memory()
-    hv = torch.randn((n_layers, Bsz, 1, Hkv, d)).to(torch.bfloat16).pin_memory()
+    hv = torch.randn((n_layers, Bsz, 1, Hkv, dv)).to(torch.bfloat16).pin_memory()
     hq = torch.randn((n_layers, Bsz, Hq, d)).to(torch.bfloat16).pin_memory()
-    hout = torch.empty((n_layers, Bsz, Hq, d), dtype=torch.float32).pin_memory()
-    dk, dv, dq = torch.empty_like(hk, device=device), torch.empty_like(hv, device=device), torch.empty_like(hq, device=device)
+    hout = torch.empty((n_layers, Bsz, Hq, dv), dtype=torch.float32).pin_memory()
+    dk, dvv, dq = torch.empty_like(hk, device=device), torch.empty_like(hv, device=device), torch.empty_like(hq, device=device)
 
     def step_e2e():
         dk.copy_(hk, non_blocking=True)
-        dv.copy_(hv, non_blocking=True)
+        if not alias:
+            dvv.copy_(hv, non_blocking=True)
         dq.copy_(hq, non_blocking=True)
         for l in range(n_layers):
-            cache.gkv_append_demote(l, dk[l], dv[l])
+            cache.gkv_append_demote(l, dk[l], None if alias else dvv[l])
             if quest:
                 n_sel = cache.gkv_quest_select(l, dq[l], wl.quest_budget_tokens, pages)
                 cache.gkv_decode_attn(l, dq[l], out[l], page_idx=pages, n_sel=n_sel)
@@ -264,10 +266,10 @@ def run_ours(args, rank, local, world):
     wall_ms = (time.perf_counter() - t0) * 1e3 / K
     e2e_ms = max_over_ranks(g0.elapsed_time(g1) / K, world)
     e2e_value = world * Bsz * ctx_e2e / (e2e_ms * 1e-3)
-    h2d = hk.numel() * 2 + hv.numel() * 2 + hq.numel() * 2
+    h2d = hk.numel() * 2 + (0 if alias else hv.numel() * 2) + hq.numel() * 2
     d2h = hout.numel() * 4
 
-    launches_per_layer = 3 + (2 if quest else 0)
+    launches_per_layer = 3 + (2 if quest else 0)      # append, decode, combine (+ score, top-k)
     gpu_launches = K * n_layers * launches_per_layer + closes * n_layers * (1 + (1 if wl.page_tokens else 0))
 
     line = {
@@ -304,22 +306,30 @@ def cpu_baseline(w: W.Workload, n_layers: int, budget_s: float = 20.0, steps: in
     import dataclasses
     from oracle import gkv_oracle as O
     S = 1
+    ctx_scale = 1
+    if w.ctx > 131072:
+        # a million-token stream takes the numpy oracle minutes: time a 1/16 context with the same
+        # ladder proportions and scale linearly (the oracle's cost is linear in the context)
+        ctx_scale = 16
+        w = dataclasses.replace(w, ctx=w.ctx // ctx_scale, max_ctx=w.ctx // ctx_scale + 128,
+                                stair_tokens=tuple((t // ctx_scale) // 64 * 64 for t in w.stair_tokens))
     ws = dataclasses.replace(w, batch=1, n_kv_heads=S, n_q_heads=S * w.group_size, n_layers=1)
     data = W.make_layer(ws, 0, "cpu")
     cfg = O.Config(n_layers=1, batch=1, n_q_heads=ws.n_q_heads, n_kv_heads=S, d_k=w.d_k, d_v=w.d_v,
-                   page_tokens=w.page_tokens, policy=w.policy, stair_tokens=tuple(w.stair_tokens),
+                   v_aliases_k=w.v_aliases_k, page_tokens=w.page_tokens, policy=w.policy, stair_tokens=tuple(w.stair_tokens),
                    n_sink_blocks=w.n_sink_blocks, retire_after=w.retire_after, rd_budget_bpv=w.rd_budget_bpv,
                    residual_fraction=w.residual_fraction, softmax_scale=w.softmax_scale)
     oc = O.GradedCache(cfg)
     f32 = lambda t: t.to(torch.float32).numpy()
     mass = data.get("mass")
-    oc.append_demote(0, f32(data["k"]), f32(data["v"]), token_mass=None if mass is None else mass.numpy())
+    oc.append_demote(0, f32(data["k"]), None if data.get("v") is None else f32(data["v"]),
+                     token_mass=None if mass is None else mass.numpy())
     times = []
     t_begin = time.perf_counter()
     i = 0
     while i < max(1, steps) or (time.perf_counter() - t_begin < budget_s and i < 8):
         tok = W.make_decode_tokens(ws, 0, i, "cpu")
-        kk, vv, qq = f32(tok["k"]), f32(tok["v"]), f32(tok["q"])
+        kk, vv, qq = f32(tok["k"]), (None if tok["v"] is None else f32(tok["v"])), f32(tok["q"])
         t0 = time.perf_counter()
         oc.append_demote(0, kk, vv)
         if w.page_tokens > 0 and w.quest_budget_tokens > 0:
@@ -331,10 +341,12 @@ def cpu_baseline(w: W.Workload, n_layers: int, budget_s: float = 20.0, steps: in
         i += 1
     t_stream = float(np.median(times))
     n_streams = w.batch * w.n_kv_heads
-    t_step = t_stream * n_streams / S * n_layers
-    return {"value": w.batch * w.ctx / t_step, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
-            "sample": "%d of %d streams of 1 of %d layers, %d decode steps (append + attention), median, "
-                      "scaled linearly to all streams and layers" % (S, n_streams, n_layers, len(times)),
+    t_step = t_stream * n_streams / S * n_layers * ctx_scale
+    return {"value": w.batch * w.ctx * ctx_scale / t_step, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+            "sample": "%d of %d streams of 1 of %d layers%s, %d decode steps (append + attention), median, "
+                      "scaled linearly to all streams and layers" % (S, n_streams, n_layers,
+                                                                      " at 1/%d of the context" % ctx_scale if ctx_scale > 1 else "",
+                                                                      len(times)),
             "seconds_per_stream_step": t_stream}
 
 
@@ -361,7 +373,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", type=int, default=2, help="workload: 0..3 (default 2: Llama-8B-like batched decode)")
+    ap.add_argument("--config", type=int, default=2, help="workload: 0..4 (default 2: Llama-8B-like batched decode)")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (0 = as defined)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

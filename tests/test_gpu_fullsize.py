@@ -220,3 +220,81 @@ def test_cfg0_repeated_through_bench_sized_launches():
     U.assert_state_equal(ocache, gcache, 0)
     print(f"cfg0 worst max-abs error over 70 steps: {worst:.2e}")
     gcache.close()
+
+
+def test_cfg4_full_size_mla_one_million_tokens():
+    """Config 4 at full size: MLA 576/512, 16 heads, 1,048,576 tokens, 5.0 bits/value ladder
+    (newest 4096 exact, int8, int4, oldest quarter centroid).
+    (a) sampled blocks of every rung are bit-exact against the oracle's per-block encoder;
+    (b) property that holds at any size: the million-token result equals the log-sum-exp merge of
+        four quarter caches that hold the same blocks at the same levels;
+    (c) the newest quarter (exact + int8 rungs, 262,144 tokens, 4096 blocks) matches the oracle."""
+    B = _binding()
+    w = dataclasses.replace(W.config(4), n_layers=1)
+    gcache = B.Cache(B.config_from_workload(w, 1))
+    dev = gcache.device
+    data = W.make_layer(w, 0, dev)
+    k = data["k"]                                                    # [1][T][1][576]
+    gcache.gkv_append_demote(0, k, None)
+    T = w.ctx
+    levels = gcache.gkv_debug_export_levels(0, 0, 0)
+    assert len(levels) == T // 64
+    rep = gcache.gkv_bits_report(0)
+    assert abs(rep.bpv_resident - 5.0) < 1e-3
+    assert list(rep.blocks_by_level) == [64, int((levels == 8).sum()), int((levels == 4).sum()), 0, 4096]
+    out_full = torch.empty((1, 16, 512), dtype=torch.float32, device=dev)
+    lse_full = torch.empty((1, 16), dtype=torch.float32, device=dev)
+    gcache.gkv_decode_attn(0, data["q"], out_full, lse_full)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out_full).all()
+    # (a) sampled blocks, every rung and its borders
+    nb = len(levels)
+    b8 = int(np.argmax(levels == 8)); b4 = int(np.argmax(levels == 4))
+    picks = sorted(set([0, 1, 4095, 4096, b4, b4 + 1, b8 - 1, b8, b8 + 1, nb - 65, nb - 64, nb - 1] +
+                       list(range(37, nb, nb // 97))))
+    kh = k[0, :, 0].cpu()
+    for i in picks:
+        blk, _ = O.make_block(int(levels[i]), U.f32(kh[i * 64:(i + 1) * 64]), None)
+        ex = gcache.gkv_debug_export_block(0, 0, 0, i, B.TENSOR_K)
+        assert ex["level"] == levels[i]
+        if blk.level == 16:
+            assert np.array_equal(ex["rows"], O.bf16_bits(blk.k_exact)), f"block {i}"
+        elif blk.level == 1:
+            assert np.array_equal(ex["rows"][0], O.bf16_bits(blk.k_cent)), f"block {i}"
+        else:
+            assert np.array_equal(ex["codes"], blk.k_codes), f"block {i} codes"
+            assert np.array_equal(ex["scale"], blk.k_scale.view(np.uint16)) and np.array_equal(ex["zero"], blk.k_zero.view(np.uint16))
+    # (b) four quarter caches with the same per-block levels, merged by their log-sum-exp
+    Tq = T // 4
+    wq = dataclasses.replace(w, ctx=Tq, max_ctx=Tq + 64, policy=W.POLICY_EXTERNAL)
+    outs, lses = [], []
+    newest = None
+    for qi in range(4):
+        qc = B.Cache(B.config_from_workload(wq, 1))
+        plan = levels[qi * (Tq // 64):(qi + 1) * (Tq // 64)].astype(np.int8).reshape(1, 1, -1)
+        qc.gkv_append_demote(0, k[:, qi * Tq:(qi + 1) * Tq].contiguous(), None, level_plan=plan)
+        o = torch.empty_like(out_full); l = torch.empty_like(lse_full)
+        qc.gkv_decode_attn(0, data["q"], o, l)
+        torch.cuda.synchronize()
+        outs.append(o.double()); lses.append(l.double())
+        if qi == 3:
+            newest = (o.clone(), l.clone())
+        qc.close()
+    L = torch.stack(lses); Mx = L.max(dim=0).values
+    wts = torch.exp(L - Mx)
+    merged = (torch.stack(outs) * wts[..., None]).sum(0) / wts.sum(0)[..., None]
+    scale = U.value_scale(k[0, :, 0, :512])
+    gap = ((merged - out_full.double()).abs().cpu().numpy() / scale).max()
+    assert gap < 2e-4, f"million-token result differs from the merge of its quarters by {gap:.2e} per unit of value scale"
+    lse_merged = Mx + torch.log(wts.sum(0))
+    assert float((lse_merged - lse_full.double()).abs().max()) < 1e-3
+    # (c) oracle on the newest quarter (exact + int8 rungs)
+    ocfg = U.oracle_config(wq, 1)
+    oc = O.GradedCache(ocfg)
+    plan = levels[3 * (Tq // 64):].astype(np.int8).reshape(1, 1, -1)
+    oc.append_demote(0, U.f32(k[:, 3 * Tq:].cpu()), None, level_plan=plan)
+    o_out, o_lse = oc.decode_attn(0, U.f32(data["q"]))
+    err, rel = U.assert_outputs_close(newest[0], o_out, "cfg4 newest quarter", scale=scale)
+    assert np.max(np.abs(newest[1].cpu().numpy() - o_lse)) < 5e-3
+    print(f"cfg4 full: quarter-merge gap {gap:.2e}, newest-quarter max-abs error {err:.2e}, relative L2 {rel:.2e}")
+    gcache.close()
