@@ -19,7 +19,7 @@ namespace {
 
 constexpr int kTargetWarps = 148 * kDecodeCtasPerSm * kDecodeWarps;   // one resident wave of CTAs
 constexpr int kSparseWarpsPerStream = 16;
-constexpr size_t kMinWarpCost = 300;      // do not split below about one block per warp
+constexpr size_t kMinWarpCost = 1000;     // do not split below about one block per warp
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int level_index(int level) { return level == 16 ? 0 : level == 8 ? 1 : level == 4 ? 2 : level == 2 ? 3 : 4; }
@@ -79,6 +79,8 @@ struct LayerState {
   std::vector<int8_t> level;            // [n_streams][max_blocks]
   TableEntry* table_h = nullptr;        // pinned [n_streams][table_stride]
   WarpDesc* warps_h = nullptr;          // pinned [max_warps]
+  uint32_t* units_h = nullptr;          // pinned [n_streams][unit_stride]
+  int n_units = 0;
   StreamParts* parts_h = nullptr;       // pinned [n_streams]
   uint32_t* res_off_h = nullptr;        // pinned [n_streams]
   int32_t* res_count_h = nullptr;       // pinned [n_streams]
@@ -89,6 +91,7 @@ struct LayerState {
   // device regions
   TableEntry* table_d = nullptr;
   WarpDesc* warps_d = nullptr;
+  uint32_t* units_d = nullptr;
   StreamParts* parts_d = nullptr;
   uint32_t* res_off_d = nullptr;
   int32_t* res_count_d = nullptr;
@@ -139,11 +142,11 @@ constexpr int kMlaTargetCtas = 148 * 2;
 
 struct ArenaPlan {
   size_t status, debug, partial, range, mass, levels, scores, kper, jobs, per_layer, heap_begin, total_meta;
-  size_t l_table, l_warps, l_parts, l_resoff, l_rescount, l_residx, l_respool, l_boxes, layer_bytes;
+  size_t l_table, l_warps, l_units, l_parts, l_resoff, l_rescount, l_residx, l_respool, l_boxes, layer_bytes;
 };
 
 struct Derived {
-  int n_streams, group, max_blocks, table_stride, max_warps, res_cap, box_stride;
+  int n_streams, group, max_blocks, table_stride, max_warps, res_cap, box_stride, unit_stride;
 };
 
 int validate_config(const gkv_config* c) {
@@ -185,6 +188,7 @@ Derived derive(const gkv_config& c) {
   d.res_cap = c.residual_fraction > 0.f
                   ? static_cast<int>(align_up(static_cast<size_t>(std::floor(static_cast<double>(c.residual_fraction) * c.max_ctx)) + 16, 16))
                   : 0;
+  d.unit_stride = d.max_blocks + 1 + d.res_cap / 16;
   d.box_stride = c.page_tokens > 0 ? static_cast<int>(align_up((c.max_ctx + c.page_tokens - 1) / c.page_tokens, 8)) : 0;
   return d;
 }
@@ -209,6 +213,7 @@ ArenaPlan plan_arena(const gkv_config& c, const Derived& d) {
   auto ltake = [&](size_t bytes) { size_t o = lo; lo = align_up(lo + bytes, 256); return o; };
   a.l_table = ltake(static_cast<size_t>(d.n_streams) * d.table_stride * sizeof(TableEntry));
   a.l_warps = ltake(static_cast<size_t>(d.max_warps) * sizeof(WarpDesc));
+  a.l_units = ltake(static_cast<size_t>(d.n_streams) * d.unit_stride * sizeof(uint32_t));
   a.l_parts = ltake(static_cast<size_t>(d.n_streams) * sizeof(StreamParts));
   a.l_resoff = ltake(static_cast<size_t>(d.n_streams) * sizeof(uint32_t));
   a.l_rescount = ltake(static_cast<size_t>(d.n_streams) * sizeof(int32_t));
@@ -355,69 +360,94 @@ bool rd_allocate(const gkv_config& c, const float* mass, const float* range, int
 }
 
 // ---- decode work split ---------------------------------------------------------------------------
-// Cost of one item for the work split, in units of 10 ps of whole-GPU time per block, measured
-// on B200 with single-level caches (a 64-token block costs 6.5 ns exact, 4.2 ns at 8 bits, 3.1 ns
-// at 4 bits, 2.9 ns at 2 bits, 0.9 ns as a centroid).  Bytes alone are the wrong weight: below
-// 8 bits the kernel is bound by instruction issue and a block costs about the same whatever its
-// code width, while exact blocks are bound by bytes.
+// Cost of one item for the work split: cycles a warp needs for it while the whole GPU runs the
+// mixed workload (measured on B200 by timing individual warps of the config-2 launch: an exact
+// block ~26 K cycles, 8-bit ~11.5 K, 4-bit ~10 K, 2-bit ~6.7 K, a centroid block ~0.6 K).  Bytes
+// alone are the wrong weight: below 8 bits the kernel is bound by instruction issue and a block
+// costs about the same whatever its code width.
 size_t item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) {
   if (item < L.n_closed) {
     switch (L.level[static_cast<size_t>(stream) * c->max_blocks + item]) {
-      case 16: return 653;
-      case 8: return 422;
-      case 4: return 309;
-      case 2: return 291;
-      default: return 91;
+      case 16: return 2600;
+      case 8: return 1150;
+      case 4: return 1000;
+      case 2: return 670;
+      default: return 60;
     }
   }
-  if (item == L.n_closed) return 330;      // tail: mid-fill estimate (its size changes every step)
-  return 165;                              // residual group of 16 exact rows
+  if (item == L.n_closed) return 1300;     // tail: mid-fill estimate (its size changes every step)
+  return 650;                              // residual group of 16 exact rows
 }
 
+// Units of a stream (a block, a run of up to 16 neighbouring centroid blocks, the tail, a residual
+// group) are dealt to the stream's warps longest-first onto the least loaded warp, so that every
+// warp ends up with the same cost whatever the order of levels along the context; each warp then
+// walks its units in ascending token order.
 void build_descs(gkv_cache* c, LayerState& L) {
   const int ns = c->n_streams;
-  std::vector<int> n_items(ns);
-  std::vector<size_t> bytes(ns, 0);
+  struct Unit { uint32_t word; size_t cost; };
+  std::vector<std::vector<Unit>> units(ns);
+  std::vector<size_t> cost(ns, 0);
   size_t total = 0;
   for (int s = 0; s < ns; ++s) {
+    const int8_t* lv = L.level.data() + static_cast<size_t>(s) * c->max_blocks;
     const int groups = (L.res_count_h[s] + 15) / 16;
-    n_items[s] = L.n_closed + 1 + groups;
-    for (int i = 0; i < n_items[s]; ++i) bytes[s] += item_cost(c, L, s, i);
-    total += bytes[s];
+    const int n_items = L.n_closed + 1 + groups;
+    std::vector<Unit>& u = units[s];
+    u.reserve(n_items);
+    for (int i = 0; i < n_items;) {
+      int run = 1;
+      if (i < L.n_closed && lv[i] != 16 && lv[i] != 8 && lv[i] != 4 && lv[i] != 2) {
+        while (run < 16 && i + run < L.n_closed) {
+          const int8_t l2 = lv[i + run];
+          if (l2 == 16 || l2 == 8 || l2 == 4 || l2 == 2) break;
+          ++run;
+        }
+      }
+      size_t k = 0;
+      for (int j = 0; j < run; ++j) k += item_cost(c, L, s, i + j);
+      u.push_back(Unit{static_cast<uint32_t>(i) | (static_cast<uint32_t>(run) << 24), k});
+      cost[s] += k;
+      i += run;
+    }
+    total += cost[s];
   }
   const size_t target = std::max(kMinWarpCost, (total + kTargetWarps - 1) / kTargetWarps);
-  int w = 0;
+  int w = 0, pos = 0;
+  std::vector<size_t> load;
+  std::vector<std::vector<uint32_t>> mine;
   for (int s = 0; s < ns; ++s) {
-    int nw = static_cast<int>((bytes[s] + target / 2) / target);
-    nw = std::max(1, std::min(nw, n_items[s]));
+    std::vector<Unit>& u = units[s];
+    int nw = static_cast<int>((cost[s] + target / 2) / target);
+    nw = std::max(1, std::min(nw, static_cast<int>(u.size())));
     nw = std::min(nw, c->max_warps - w - (ns - 1 - s));
+    std::stable_sort(u.begin(), u.end(), [](const Unit& a, const Unit& b) { return a.cost > b.cost; });
+    load.assign(nw, 0);
+    mine.assign(nw, {});
+    for (const Unit& x : u) {
+      int best = 0;
+      for (int k = 1; k < nw; ++k)
+        if (load[k] < load[best]) best = k;
+      load[best] += x.cost;
+      mine[best].push_back(x.word);
+    }
     L.parts_h[s].begin = w;
-    size_t acc = 0;
-    int item = 0;
     for (int k = 0; k < nw; ++k) {
-      const size_t limit = bytes[s] * (k + 1) / nw;
-      const int begin = item;
-      const int max_end = n_items[s] - (nw - 1 - k);     // leave one item for each later warp
-      do {
-        acc += item_cost(c, L, s, item);
-        ++item;
-      } while (item < max_end && acc < limit);
+      std::sort(mine[k].begin(), mine[k].end(), [](uint32_t a, uint32_t b) { return (a & 0xffffffu) < (b & 0xffffffu); });
       WarpDesc& d = L.warps_h[w];
       d.stream = s;
-      d.item_begin = begin;
-      d.item_end = item;
+      d.item_begin = pos;
+      for (uint32_t x : mine[k]) L.units_h[pos++] = x;
+      d.item_end = pos;
       d.partial = w;
       ++w;
     }
-    L.warps_h[w - 1].item_end = n_items[s];
     L.parts_h[s].end = w;
   }
   const int padded = static_cast<int>(align_up(w, kDecodeWarps));
   for (int i = w; i < padded; ++i) L.warps_h[i] = WarpDesc{-1, 0, 0, 0};
-  // Warps stay in stream order: the warps of a CTA then work on neighbouring blocks of the same
-  // level and share one code path, which keeps the instruction cache warm (dealing the levels
-  // across CTAs was measured to be slower).
   L.n_warps = padded;
+  L.n_units = pos;
   L.desc_dirty = false;
 }
 
@@ -1014,6 +1044,7 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
     uint8_t* lb = c->arena + a.per_layer + static_cast<size_t>(l) * a.layer_bytes;
     L.table_d = reinterpret_cast<TableEntry*>(lb + a.l_table);
     L.warps_d = reinterpret_cast<WarpDesc*>(lb + a.l_warps);
+    L.units_d = reinterpret_cast<uint32_t*>(lb + a.l_units);
     L.parts_d = reinterpret_cast<StreamParts*>(lb + a.l_parts);
     L.res_off_d = reinterpret_cast<uint32_t*>(lb + a.l_resoff);
     L.res_count_d = reinterpret_cast<int32_t*>(lb + a.l_rescount);
@@ -1025,6 +1056,8 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
     if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.table_h), tb, cudaHostAllocDefault)) != cudaSuccess) return fail(e);
     std::memset(L.table_h, 0, tb);
     if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.warps_h), d.max_warps * sizeof(WarpDesc), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
+    if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.units_h), static_cast<size_t>(d.n_streams) * d.unit_stride * sizeof(uint32_t),
+                           cudaHostAllocDefault)) != cudaSuccess) return fail(e);
     if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.parts_h), d.n_streams * sizeof(StreamParts), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
     if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.res_off_h), d.n_streams * sizeof(uint32_t), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
     if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.res_count_h), d.n_streams * sizeof(int32_t), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
@@ -1047,6 +1080,7 @@ int gkv_destroy(gkv_cache* c) {
   for (LayerState& L : c->layers) {
     if (L.table_h) cudaFreeHost(L.table_h);
     if (L.warps_h) cudaFreeHost(L.warps_h);
+    if (L.units_h) cudaFreeHost(L.units_h);
     if (L.parts_h) cudaFreeHost(L.parts_h);
     if (L.res_off_h) cudaFreeHost(L.res_off_h);
     if (L.res_count_h) cudaFreeHost(L.res_count_h);
@@ -1143,9 +1177,11 @@ int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* p
       if (rc != GKV_OK) return rc;
       build_descs(c, L);
       if ((rc = upload(c, L.warps_d, L.warps_h, static_cast<size_t>(L.n_warps) * sizeof(WarpDesc), st, L.ev)) != GKV_OK) return rc;
+      if ((rc = upload(c, L.units_d, L.units_h, static_cast<size_t>(L.n_units) * sizeof(uint32_t), st, L.ev)) != GKV_OK) return rc;
       if ((rc = upload(c, L.parts_d, L.parts_h, static_cast<size_t>(c->n_streams) * sizeof(StreamParts), st, L.ev)) != GKV_OK) return rc;
     }
     p.warps = L.warps_d;
+    p.units = L.units_d;
     p.n_warps = L.n_warps;
     cp.parts = L.parts_d;
     n_ctas = L.n_warps / kDecodeWarps;
@@ -1231,7 +1267,7 @@ int gkv_bits_report(gkv_cache* c, int32_t layer, gkv_bits* out) {
       if (cfg.page_tokens > 0) out->box_bits += static_cast<uint64_t>(L.n_closed) * (kBlock / cfg.page_tokens) * 2 * cfg.d_k * 16;
       out->meta_bits += static_cast<uint64_t>(L.n_closed + 1) * sizeof(TableEntry) * 8;
     }
-    out->meta_bits += static_cast<uint64_t>(L.n_warps) * sizeof(WarpDesc) * 8;
+    out->meta_bits += static_cast<uint64_t>(L.n_warps) * sizeof(WarpDesc) * 8 + static_cast<uint64_t>(L.n_units) * 32;
     if (L.last_mode == 1) out->last_read_bits += full_read_bits(c, L);
     if (L.last_mode == 2) {
       // fetch the page list that was used and count what it touched

@@ -19,6 +19,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <cstdio>
+
 #include "gkv_internal.h"
 
 namespace gkv {
@@ -244,7 +246,8 @@ __device__ __forceinline__ void make_p_bf16(const float (&S)[4], uint32_t (&pf)[
 
 // ---- item cursor ---------------------------------------------------------------------------
 struct Cursor {
-  int item;          // dense: item index; sparse: position in the warp's slice of the page list
+  int item;          // dense: position in the warp's unit list; sparse: position in its slice of the page list
+  int first;         // dense: first item (block index) of the unit
   int sub;           // step inside the item
   int nsub;          // steps of the item
   int adv;           // items consumed when the item is done (centroid runs consume several)
@@ -266,64 +269,65 @@ struct WarpCtx {
   const uint8_t* stage_ptr0; // the same as a generic pointer
   uint32_t bar0;             // mbarrier of stage 0 (stage s at + 8 s)
   uint32_t qb_addr;          // this lane's bf16 query fragments in shared memory (16 words)
-  // prefetched window of table entries (dense mode): lane i holds entry win_base + i
-  uint4 win;
-  int win_base;
+  // dense mode: this warp's unit list and the prefetched entry of the unit after the current one
+  const uint32_t* units;     // unit = first item | run length << 24
+  uint32_t pf_unit;
+  uint4 pf_entry;
+  int pf_pos;
 };
 
 __device__ __forceinline__ int popc4(int m) { return __popc(m & 15); }
 
-__device__ __forceinline__ TableEntry window_entry(WarpCtx& w, int item) {
-  const int last = w.p->n_closed;            // the tail entry is the last valid one
-  if (item < w.win_base || item >= w.win_base + 32) {
-    w.win_base = item;
-    const int idx = min(item + w.lane, last);
-    w.win = *reinterpret_cast<const uint4*>(w.table + idx);
+// Unit at list position `pos` and the table entry of its first item; the pair for pos + 1 is
+// requested right away so that its two dependent loads are in flight while this unit is processed.
+__device__ __forceinline__ void unit_at(WarpCtx& w, int pos, uint32_t* unit, TableEntry* e) {
+  uint32_t u;
+  uint4 raw;
+  if (pos == w.pf_pos) {
+    u = w.pf_unit;
+    raw = w.pf_entry;
+  } else {
+    u = w.units[pos];
+    raw = *reinterpret_cast<const uint4*>(w.table + min(static_cast<int>(u & 0xffffffu), w.p->n_closed));
   }
-  const int src = item - w.win_base;
-  TableEntry e;
-  e.off256 = __shfl_sync(kFull, w.win.x, src);
-  e.level = __shfl_sync(kFull, w.win.y, src);
-  const uint32_t lo = __shfl_sync(kFull, w.win.z, src), hi = __shfl_sync(kFull, w.win.w, src);
-  e.resmask = (static_cast<uint64_t>(hi) << 32) | lo;
-  return e;
+  if (pos + 1 < w.item_end) {
+    w.pf_unit = w.units[pos + 1];
+    w.pf_entry = *reinterpret_cast<const uint4*>(w.table + min(static_cast<int>(w.pf_unit & 0xffffffu), w.p->n_closed));
+    w.pf_pos = pos + 1;
+  }
+  *unit = u;
+  e->off256 = raw.x;
+  e->level = raw.y;
+  e->resmask = (static_cast<uint64_t>(raw.w) << 32) | raw.z;
 }
 
-// Dense mode: set up the cursor for item index `it`.  Returns false when past the end.
-__device__ __forceinline__ bool load_item_dense(WarpCtx& w, int it, Cursor& c) {
+// Dense mode: set up the cursor for position `pos` of the warp's unit list (c.item holds the
+// position, c.adv = 1).  Returns false when past the end.
+__device__ __forceinline__ bool load_item_dense(WarpCtx& w, int pos, Cursor& c) {
   const DecodeParams& p = *w.p;
   while (true) {
-    if (it >= w.item_end) return false;
-    c.item = it;
+    if (pos >= w.item_end) return false;
+    uint32_t unit;
+    TableEntry e;
+    unit_at(w, pos, &unit, &e);
+    const int it = static_cast<int>(unit & 0xffffffu), run = static_cast<int>(unit >> 24);
+    c.item = pos;
+    c.first = it;
     c.sub = 0;
     c.adv = 1;
     if (it <= p.n_closed) {
-      const TableEntry e = window_entry(w, it);
       c.off256 = e.off256;
       c.resmask = e.resmask;
       c.level = static_cast<int>(e.level);
       c.tmask = 15;
       c.ntok = kBlock;
-#if GKV_L2_PREFETCH_AHEAD > 0
-      {
-        // Pull a later item of this warp's range into L2 now: shared memory holds only two steps
-        // per warp, far less than HBM's bandwidth-delay product, so the DRAM latency is taken here,
-        // ahead of time, and the staged copies then hit L2.
-        const int ahead = it + GKV_L2_PREFETCH_AHEAD;
-        if (ahead < w.item_end && ahead < p.n_closed) {
-          const TableEntry pe = window_entry(w, ahead);
-          if (w.lane == 0 && pe.level != 1u)
-            bulk_prefetch_l2(p.arena + static_cast<size_t>(pe.off256) * 256, slot_bytes(static_cast<int>(pe.level)));
-        }
-      }
-#endif
       if (it == p.n_closed) {           // tail block: exact rows, n_tail of them
         c.level = 16;
         c.ntok = p.n_tail;
         const int nt = (p.n_tail + 15) >> 4;
         c.tmask = (1 << nt) - 1;
         if (nt == 0) {
-          ++it;
+          ++pos;
           continue;
         }
       }
@@ -332,16 +336,10 @@ __device__ __forceinline__ bool load_item_dense(WarpCtx& w, int it, Cursor& c) {
         case 8: c.nsub = 4; break;
         case 4: c.nsub = 2; break;
         case 2: c.nsub = 1; break;
-        default: {   // centroid run: up to 16 consecutive centroid blocks inside this warp's range
-          const int lim = min(min(w.item_end, p.n_closed) - it, 16);
-          const bool is_c = (w.lane < lim) && (w.table[it + w.lane].level == 1u);
-          const unsigned m = __ballot_sync(kFull, is_c);
-          const int run = __ffs(~m) - 1;      // consecutive centroid blocks starting at `it`
-          c.adv = run;
+        default:     // run of up to 16 consecutive centroid blocks (merged by the host)
           c.ntok = run;
           c.nsub = 2;
           c.level = 1;
-        }
       }
       return true;
     }
@@ -349,7 +347,10 @@ __device__ __forceinline__ bool load_item_dense(WarpCtx& w, int it, Cursor& c) {
     const int j = it - p.n_closed - 1;
     const int n_res = p.res_count ? p.res_count[w.stream] : 0;
     const int rows = min(16, n_res - 16 * j);
-    if (rows <= 0) return false;
+    if (rows <= 0) {
+      ++pos;
+      continue;
+    }
     c.level = 17;
     c.ntok = rows;
     c.nsub = 2;
@@ -468,7 +469,7 @@ __device__ __forceinline__ void issue_step(const WarpCtx& w, const Cursor& c, in
       if (lane < nrows) {
         int blk;
         if constexpr (SPARSE) blk = p.page_idx[static_cast<size_t>(w.stream) * p.n_sel + c.item] / (kBlock / p.page_tokens);
-        else blk = c.item + lane;
+        else blk = c.first + lane;
         src = p.arena + static_cast<size_t>(w.table[blk].off256) * 256 + (is_v ? kRowBytes : 0);
       }
     }
@@ -804,7 +805,7 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
         if (lane < c.ntok) {
           int cnt;
           if constexpr (SPARSE) cnt = 16 * popc4(c.tmask);
-          else cnt = kBlock - __popcll(w.table[c.item + lane].resmask);
+          else cnt = kBlock - __popcll(w.table[c.first + lane].resmask);
           myb = cnt > 0 ? log2f(static_cast<float>(cnt)) : kNegInf;
         }
         b_lo = __shfl_sync(kFull, myb, r);
@@ -864,8 +865,10 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   WarpCtx w;
   w.p = &p;
   w.lane = lane;
-  w.win_base = -(1 << 30);
-  w.win = make_uint4(0, 0, 0, 0);
+  w.units = p.units;
+  w.pf_pos = -1;
+  w.pf_unit = 0;
+  w.pf_entry = make_uint4(0, 0, 0, 0);
   int partial_row, first;
   if constexpr (!SPARSE) {
     const WarpDesc wd = p.warps[gw];
@@ -928,6 +931,10 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   st.zc[0] = st.zc[1] = st.zc[2] = st.zc[3] = 0.f;
   uint32_t pf[4] = {0, 0, 0, 0};
 
+#ifdef GKV_EXP_PROFILE
+  long long prof_wait = 0, prof_steps = 0;
+  const long long prof_t0 = clock64();
+#endif
   Cursor cur;
   bool have = load_item<SPARSE>(w, first, cur);
   int sidx = 0;
@@ -941,6 +948,9 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     const bool more = advance<SPARSE>(w, nxt);
 #ifndef GKV_EXP_SKIP_COPY
     if (more) issue_step<SPARSE>(w, nxt, sidx ^ 1);
+#ifdef GKV_EXP_PROFILE
+    const long long tw0 = clock64();
+#endif
     // bounded wait for this step's bytes
     int spins = 0;
     while (!mbar_try_wait(w.bar0 + 8 * sidx, (phase >> sidx) & 1u)) {
@@ -951,6 +961,10 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     }
 #endif
     if (__any_sync(kFull, failed)) break;
+#ifdef GKV_EXP_PROFILE
+    prof_wait += clock64() - tw0;
+    prof_steps += 1;
+#endif
     phase ^= 1u << sidx;
     __syncwarp();
 #ifndef GKV_EXP_SKIP_COMPUTE
@@ -961,6 +975,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     have = more;
     sidx ^= 1;
   }
+#ifdef GKV_EXP_PROFILE
+  if (lane == 0 && (gw % 97) == 0)
+    printf("PROF warp %d stream %d items %d steps %lld total %lld wait %lld\n", gw, w.stream, w.item_end - first, prof_steps,
+           clock64() - prof_t0, prof_wait);
+#endif
   if (failed) {
     // a copy never completed: flag it and publish an empty partial (the host reports BAD_STATE)
     if (lane == 0) atomicOr(p.status, kStatusInternal);

@@ -16,9 +16,11 @@ struct alignas(16) TableEntry {
   uint64_t resmask;  // bit t set: token t of the block is served from the residual pool instead
 };
 
-// Work of one warp of the decode kernel: a contiguous range of items of one stream.
-// Items: [0, n_closed) closed blocks, n_closed = tail block, n_closed + 1 + j = residual group j
-// (16 residual rows each).
+// Work of one warp of the decode kernel: positions [item_begin, item_end) of the layer's unit
+// list, all of one stream.  A unit is one item or a run of consecutive centroid blocks:
+// `first item | run << 24`.  Items: [0, n_closed) closed blocks, n_closed = tail block,
+// n_closed + 1 + j = residual group j (16 residual rows each).  (The MLA kernel uses the same
+// struct per CTA with item_begin / item_end as a plain item range.)
 struct alignas(16) WarpDesc {
   int32_t stream;      // -1 = idle warp
   int32_t item_begin;
@@ -47,6 +49,7 @@ struct DecodeParams {
   const uint8_t* arena;
   const TableEntry* table;      // [n_streams][table_stride]
   const WarpDesc* warps;        // [n_warps]
+  const uint32_t* units;        // the layer's unit list (dense mode)
   const uint16_t* q;            // bf16 [batch][n_q_heads][128]
   float* partial;               // [n_partials][kPartialFloats]
   const uint32_t* res_off256;   // [n_streams] residual pool offset (rows of 512 B: K row | V row)
