@@ -5,6 +5,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -424,10 +425,13 @@ void build_descs(gkv_cache* c, LayerState& L) {
     std::stable_sort(u.begin(), u.end(), [](const Unit& a, const Unit& b) { return a.cost > b.cost; });
     load.assign(nw, 0);
     mine.assign(nw, {});
+    static const double wave2 = std::getenv("GKV_WAVE2_SPEED") ? std::atof(std::getenv("GKV_WAVE2_SPEED")) : 1.0;
+    std::vector<double> inv(nw);
+    for (int k = 0; k < nw; ++k) inv[k] = ((w + k) / kDecodeWarps >= 148) ? 1.0 / wave2 : 1.0;
     for (const Unit& x : u) {
       int best = 0;
       for (int k = 1; k < nw; ++k)
-        if (load[k] < load[best]) best = k;
+        if ((load[k] + x.cost) * inv[k] < (load[best] + x.cost) * inv[best]) best = k;
       load[best] += x.cost;
       mine[best].push_back(x.word);
     }

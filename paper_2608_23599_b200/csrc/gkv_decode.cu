@@ -119,10 +119,13 @@ __device__ __forceinline__ float bf16lo_to_f32(uint32_t u) { return __uint_as_fl
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
 // ---- code unpack: the four A registers of MMA index s as fp16 "bias + code" ------------------
-// Biases (rows r / rows r + 8 of the MMA): 8-bit 1024 / 1024; 4-bit 256 / 16; 2-bit 256 / 64 for
-// even s and 16 / 4 for odd s.  `mid` is the centre of the code range: products are formed with
-// (code - mid) so that the fp16 rounding of the folded scale acts on a centred value; the term
-// mid * sum(q s) is added back from an exact MMA.
+// Biases (rows r / rows r + 8 of the MMA): 8-bit 1024 / 1024; 4-bit 1024 / 64; 2-bit 1024 / 256 for
+// even s and 64 / 16 for odd s: a code that sits at mantissa bit b of an fp16 with exponent 2^E has
+// the value code * 2^(E - 10 + b), so picking E = 10 - b makes "mask, or in the exponent" a complete
+// conversion with no shift; only the upper byte of each 16-bit half needs one shift by 8.  `mid`
+// is the centre of the code range: products are formed with (code - mid) so that the fp16
+// rounding of the folded scale acts on a centred value; the term mid * sum(q s) is added back
+// from an exact MMA.
 template <int BITS>
 struct Bias;
 template <>
@@ -131,11 +134,11 @@ struct Bias<8> {
 };
 template <>
 struct Bias<4> {
-  static constexpr float lo_even = 256.f, hi_even = 16.f, lo_odd = 256.f, hi_odd = 16.f, mid = 7.5f;
+  static constexpr float lo_even = 1024.f, hi_even = 64.f, lo_odd = 1024.f, hi_odd = 64.f, mid = 7.5f;
 };
 template <>
 struct Bias<2> {
-  static constexpr float lo_even = 256.f, hi_even = 64.f, lo_odd = 16.f, hi_odd = 4.f, mid = 1.5f;
+  static constexpr float lo_even = 1024.f, hi_even = 256.f, lo_odd = 64.f, hi_odd = 16.f, mid = 1.5f;
 };
 
 // Words of one lane for MMA indices [s0, s0 + NS): 8-bit 2 words per s, 4-bit 1, 2-bit 1 per 2.
@@ -149,23 +152,23 @@ __device__ __forceinline__ void unpack(const uint32_t* w, int s_local, uint32_t 
     a[2] = prmt(w1, kMagic, 0x5250u);
     a[3] = prmt(w1, kMagic, 0x5351u);
   } else if constexpr (BITS == 4) {
-    const uint32_t v0 = w[s_local] << 2, v1 = w[s_local] >> 6;
-    a[0] = lop3_and_or(v0, 0x003C003Cu, 0x5C005C00u);   // 256 + code
-    a[1] = lop3_and_or(v0, 0x03C003C0u, 0x4C004C00u);   // 16 + code
-    a[2] = lop3_and_or(v1, 0x003C003Cu, 0x5C005C00u);
-    a[3] = lop3_and_or(v1, 0x03C003C0u, 0x4C004C00u);
+    const uint32_t v0 = w[s_local], v1 = w[s_local] >> 8;
+    a[0] = lop3_and_or(v0, 0x000F000Fu, 0x64006400u);   // 1024 + code
+    a[1] = lop3_and_or(v0, 0x00F000F0u, 0x54005400u);   // 64 + code
+    a[2] = lop3_and_or(v1, 0x000F000Fu, 0x64006400u);
+    a[3] = lop3_and_or(v1, 0x00F000F0u, 0x54005400u);
   } else {
-    const uint32_t v0 = w[s_local >> 1] << 2, v1 = w[s_local >> 1] >> 6;
+    const uint32_t v0 = w[s_local >> 1], v1 = w[s_local >> 1] >> 8;
     if ((s_local & 1) == 0) {
-      a[0] = lop3_and_or(v0, 0x000C000Cu, 0x5C005C00u);  // 256 + code
-      a[1] = lop3_and_or(v0, 0x00300030u, 0x54005400u);  // 64 + code
-      a[2] = lop3_and_or(v1, 0x000C000Cu, 0x5C005C00u);
-      a[3] = lop3_and_or(v1, 0x00300030u, 0x54005400u);
+      a[0] = lop3_and_or(v0, 0x00030003u, 0x64006400u);  // 1024 + code
+      a[1] = lop3_and_or(v0, 0x000C000Cu, 0x5C005C00u);  // 256 + code
+      a[2] = lop3_and_or(v1, 0x00030003u, 0x64006400u);
+      a[3] = lop3_and_or(v1, 0x000C000Cu, 0x5C005C00u);
     } else {
-      a[0] = lop3_and_or(v0, 0x00C000C0u, 0x4C004C00u);  // 16 + code
-      a[1] = lop3_and_or(v0, 0x03000300u, 0x44004400u);  // 4 + code
-      a[2] = lop3_and_or(v1, 0x00C000C0u, 0x4C004C00u);
-      a[3] = lop3_and_or(v1, 0x03000300u, 0x44004400u);
+      a[0] = lop3_and_or(v0, 0x00300030u, 0x54005400u);  // 64 + code
+      a[1] = lop3_and_or(v0, 0x00C000C0u, 0x4C004C00u);  // 16 + code
+      a[2] = lop3_and_or(v1, 0x00300030u, 0x54005400u);
+      a[3] = lop3_and_or(v1, 0x00C000C0u, 0x4C004C00u);
     }
   }
 }
@@ -269,6 +272,7 @@ struct WarpCtx {
   const uint8_t* stage_ptr0; // the same as a generic pointer
   uint32_t bar0;             // mbarrier of stage 0 (stage s at + 8 s)
   uint32_t qb_addr;          // this lane's bf16 query fragments in shared memory (16 words)
+  uint32_t qh_addr;          // the same in fp16
   // dense mode: this warp's unit list and the prefetched entry of the unit after the current one
   const uint32_t* units;     // unit = first item | run length << 24
   uint32_t pf_unit;
@@ -335,7 +339,7 @@ __device__ __forceinline__ bool load_item_dense(WarpCtx& w, int pos, Cursor& c) 
         case 16: c.nsub = 2 * popc4(c.tmask); break;
         case 8: c.nsub = 4; break;
         case 4: c.nsub = 2; break;
-        case 2: c.nsub = 1; break;
+        case 2: c.nsub = 2; break;
         default:     // run of up to 16 consecutive centroid blocks (merged by the host)
           c.ntok = run;
           c.nsub = 2;
@@ -391,8 +395,8 @@ __device__ __forceinline__ bool load_item_sparse(WarpCtx& w, int pos, Cursor& c)
     switch (c.level) {
       case 16: c.nsub = 2 * popc4(mask); break;
       case 8: c.nsub = 2 * (((mask & 3) != 0) + ((mask & 12) != 0)); break;
-      case 4: c.nsub = ((mask & 3) != 0) + ((mask & 12) != 0); break;
-      case 2: c.nsub = 1; break;
+      case 4:
+      case 2: c.nsub = ((mask & 3) != 0) + ((mask & 12) != 0); break;
       default: c.nsub = 2; c.ntok = 1; break;     // a single centroid row weighted by the selected tokens
     }
     return true;
@@ -496,12 +500,9 @@ __device__ __forceinline__ void issue_step(const WarpCtx& w, const Cursor& c, in
     if (bits == 8) {
       bytes = 512 + 2 * cb;
       src = slot + (c.sub >> 1) * half_bytes(8) + (c.sub & 1) * bytes;
-    } else if (bits == 4) {
-      bytes = half_bytes(4);
-      src = slot + c.sub * bytes;
     } else {
-      bytes = 2 * half_bytes(2);
-      src = slot;
+      bytes = half_bytes(bits);
+      src = slot + c.sub * bytes;
     }
     mbar_expect_tx(bar, bytes);
     bulk_g2s(sdst, src, bytes, bar);
@@ -527,28 +528,17 @@ __device__ __forceinline__ void issue_step(const WarpCtx& w, const Cursor& c, in
         }
     }
   } else {
-    const int nh = (bits == 4) ? 1 : 2;
-    uint32_t total = 0;
-    for (int hh = 0; hh < nh; ++hh) {
-      const int half = (bits == 4) ? half_of_step(c, c.sub) : hh;
-      const int tm = (c.tmask >> (2 * half)) & 3;
-      if (tm) total += 512 + popc4(tm) * (2 * cb + 256);
-    }
-    mbar_expect_tx(bar, total);
-    for (int hh = 0; hh < nh; ++hh) {
-      const int half = (bits == 4) ? half_of_step(c, c.sub) : hh;
-      const int tm = (c.tmask >> (2 * half)) & 3;
-      if (tm == 0) continue;
-      const uint8_t* hb = slot + half * half_bytes(bits);
-      const uint32_t sd = sdst + ((bits == 4) ? 0 : hh * half_bytes(2));
-      bulk_g2s(sd, hb, 512, bar);
-      for (int t = 0; t < 2; ++t)
-        if (tm & (1 << t)) {
-          bulk_g2s(sd + off_kc(bits, t), hb + off_kc(bits, t), cb, bar);
-          bulk_g2s(sd + off_vp(bits, t), hb + off_vp(bits, t), 256, bar);
-          bulk_g2s(sd + off_vc(bits, t), hb + off_vc(bits, t), cb, bar);
-        }
-    }
+    const int half = half_of_step(c, c.sub);
+    const int tm = (c.tmask >> (2 * half)) & 3;
+    const uint8_t* hb = slot + half * half_bytes(bits);
+    mbar_expect_tx(bar, 512 + popc4(tm) * (2 * cb + 256));
+    bulk_g2s(sdst, hb, 512, bar);
+    for (int t = 0; t < 2; ++t)
+      if (tm & (1 << t)) {
+        bulk_g2s(sdst + off_kc(bits, t), hb + off_kc(bits, t), cb, bar);
+        bulk_g2s(sdst + off_vp(bits, t), hb + off_vp(bits, t), 256, bar);
+        bulk_g2s(sdst + off_vc(bits, t), hb + off_vc(bits, t), cb, bar);
+      }
   }
 }
 
@@ -602,47 +592,57 @@ __device__ __forceinline__ void load_words(uint32_t codes, int j, int lane, uint
 // k~ = s * code + z.  Data MMAs use A = bias + code and B = q' = q * s; the bias (and the code
 // centre) is removed with a "ones" MMA on the same q' and the zero points enter through an MMA
 // with A = (z | s) and B = q.  All arguments that address shared memory are 32-bit addresses.
+// The loop over channel slabs is kept rolled: the kernel is bound by instruction fetch, and a
+// compact body that stays in the instruction caches is worth more than the scheduling freedom
+// of straight-line code.
+// Channel slab j (MMA indices 2 j and 2 j + 1) of qk_half; FIRST starts the accumulation chains.
+template <int BITS, bool FULL, bool FIRST>
+__device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm, uint32_t qh_addr, int lane,
+                                        float (&zd)[4], float (&qe)[4], float (&qo)[4], float (&S)[2][4]) {
+  constexpr int cb = 256 * BITS;
+  constexpr int kW = BITS / 2;
+  uint32_t w0[kW], w1[kW];
+  if (FULL || (tm & 1)) load_words<BITS>(kc0, j, lane, w0);
+  if (FULL || (tm & 2)) load_words<BITS>(kc0 + cb, j, lane, w1);
+#pragma unroll
+  for (int ss = 0; ss < 2; ++ss) {
+    const uint4 pr = lds128(kp + j * 128 + ss * 64);   // s01, z01, s23, z23
+    const uint2 q = lds64(qh_addr + j * 512 + ss * 256);
+    const uint32_t q0 = hmul2_u32(q.x, pr.x), q1 = hmul2_u32(q.y, pr.z);
+    if (FIRST && ss == 0) mma_f16_first(zd, pr.y, pr.x, pr.w, pr.z, q.x, q.y);
+    else mma_f16(zd, pr.y, pr.x, pr.w, pr.z, q.x, q.y);
+    if (BITS == 2 && ss == 1) {
+      if (FIRST) mma_f16_first(qo, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
+      else mma_f16(qo, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
+    } else {
+      if (FIRST && ss == 0) mma_f16_first(qe, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
+      else mma_f16(qe, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
+    }
+    uint32_t a[4];
+    if (FULL || (tm & 1)) {
+      unpack<BITS>(w0, ss, a);
+      if (FIRST && ss == 0) mma_f16_first(S[0], a[0], a[1], a[2], a[3], q0, q1);
+      else mma_f16(S[0], a[0], a[1], a[2], a[3], q0, q1);
+    }
+    if (FULL || (tm & 2)) {
+      unpack<BITS>(w1, ss, a);
+      if (FIRST && ss == 0) mma_f16_first(S[1], a[0], a[1], a[2], a[3], q0, q1);
+      else mma_f16(S[1], a[0], a[1], a[2], a[3], q0, q1);
+    }
+  }
+}
+
 template <int BITS, bool FULL>
-__device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, uint32_t kc1, int tm, const uint32_t (&qh)[16],
-                                        int lane, float scale_log2, uint64_t resmask, int half, float (&S)[2][4]) {
+__device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, int tm, uint32_t qh_addr, int lane, float scale_log2,
+                                        uint64_t resmask, int half, float (&S)[2][4]) {
   const int c4 = lane & 3, r = lane >> 2;
   float zd[4];        // rows r: sum_c q_c z_c; rows r + 8: sum_c q_c s_c (exact products)
   float qe[4];        // sum_c q'_c over even MMA indices (all rows equal)
   float qo[4] = {0.f, 0.f, 0.f, 0.f};   // ... over odd MMA indices (2-bit only)
-  constexpr int kW = BITS / 2;
   kp += c4 * 16;
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    uint32_t w0[kW], w1[kW];
-    if (FULL || (tm & 1)) load_words<BITS>(kc0, j, lane, w0);
-    if (FULL || (tm & 2)) load_words<BITS>(kc1, j, lane, w1);
-#pragma unroll
-    for (int ss = 0; ss < 2; ++ss) {
-      const int s = 2 * j + ss;
-      const uint4 pr = lds128(kp + s * 64);   // s01, z01, s23, z23
-      const uint32_t q0 = hmul2_u32(qh[2 * s], pr.x), q1 = hmul2_u32(qh[2 * s + 1], pr.z);
-      if (s == 0) mma_f16_first(zd, pr.y, pr.x, pr.w, pr.z, qh[0], qh[1]);
-      else mma_f16(zd, pr.y, pr.x, pr.w, pr.z, qh[2 * s], qh[2 * s + 1]);
-      if (BITS == 2 && ss == 1) {
-        if (s == 1) mma_f16_first(qo, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
-        else mma_f16(qo, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
-      } else {
-        if (s == 0) mma_f16_first(qe, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
-        else mma_f16(qe, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
-      }
-      uint32_t a[4];
-      if (FULL || (tm & 1)) {
-        unpack<BITS>(w0, ss, a);
-        if (s == 0) mma_f16_first(S[0], a[0], a[1], a[2], a[3], q0, q1);
-        else mma_f16(S[0], a[0], a[1], a[2], a[3], q0, q1);
-      }
-      if (FULL || (tm & 2)) {
-        unpack<BITS>(w1, ss, a);
-        if (s == 0) mma_f16_first(S[1], a[0], a[1], a[2], a[3], q0, q1);
-        else mma_f16(S[1], a[0], a[1], a[2], a[3], q0, q1);
-      }
-    }
-  }
+  qk_slab<BITS, FULL, true>(kp, kc0, 0, tm, qh_addr, lane, zd, qe, qo, S);
+#pragma unroll 1
+  for (int j = 1; j < 4; ++j) qk_slab<BITS, FULL, false>(kp, kc0, j, tm, qh_addr, lane, zd, qe, qo, S);
   if (!FULL) {
     if (!(tm & 1)) S[0][0] = S[0][1] = S[0][2] = S[0][3] = 0.f;
     if (!(tm & 2)) S[1][0] = S[1][1] = S[1][2] = S[1][3] = 0.f;
@@ -655,12 +655,13 @@ __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, uint32_t kc1,
   const float c_hi0 = z0 - (Bias<BITS>::hi_even + kMid) * qe[0] - (Bias<BITS>::hi_odd + kMid) * qo[0];
   const float c_hi1 = z1 - (Bias<BITS>::hi_even + kMid) * qe[1] - (Bias<BITS>::hi_odd + kMid) * qo[1];
   if (FULL && resmask == 0) {
+    const float d_lo0 = c_lo0 * scale_log2, d_lo1 = c_lo1 * scale_log2, d_hi0 = c_hi0 * scale_log2, d_hi1 = c_hi1 * scale_log2;
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
-      S[t][0] = (S[t][0] + c_lo0) * scale_log2;
-      S[t][1] = (S[t][1] + c_lo1) * scale_log2;
-      S[t][2] = (S[t][2] + c_hi0) * scale_log2;
-      S[t][3] = (S[t][3] + c_hi1) * scale_log2;
+      S[t][0] = fmaf(S[t][0], scale_log2, d_lo0);
+      S[t][1] = fmaf(S[t][1], scale_log2, d_lo1);
+      S[t][2] = fmaf(S[t][2], scale_log2, d_hi0);
+      S[t][3] = fmaf(S[t][3], scale_log2, d_hi1);
     }
     return;
   }
@@ -681,13 +682,12 @@ __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, uint32_t kc1,
 // One tile's share of O^T += V~^T P^T for group grp: data MMAs accumulate (bias + code) * P' straight
 // into O; `ps` collects sum P' so that the bias can be taken out afterwards.
 template <int BITS>
-__device__ __forceinline__ void pv_tile_group(uint32_t vc, int grp, int lane, uint32_t p0, uint32_t p1, bool first,
-                                              float (&ps)[4], float (&o0)[4], float (&o1)[4]) {
+__device__ __forceinline__ void pv_tile_group(uint32_t vc, int grp, int lane, uint32_t p0, uint32_t p1, float (&ps)[4],
+                                              float (&o0)[4], float (&o1)[4]) {
   uint32_t wd[BITS / 2];
   uint32_t a[4];
   load_words<BITS>(vc, grp, lane, wd);
-  if (first) mma_f16_first(ps, kOnesH2, kOnesH2, kOnesH2, kOnesH2, p0, p1);
-  else mma_f16(ps, kOnesH2, kOnesH2, kOnesH2, kOnesH2, p0, p1);
+  mma_f16(ps, kOnesH2, kOnesH2, kOnesH2, kOnesH2, p0, p1);
   unpack<BITS>(wd, 0, a);
   mma_f16(o0, a[0], a[1], a[2], a[3], p0, p1);
   unpack<BITS>(wd, 1, a);
@@ -695,74 +695,61 @@ __device__ __forceinline__ void pv_tile_group(uint32_t vc, int grp, int lane, ui
 }
 
 // O^T += V~^T P^T for the active tiles of one half, v~ = s * code + z per (token, 32-channel group).
-// pf holds the raw fp16 P^T fragments of the two tiles.
+// pf holds the raw fp16 P^T fragments of the two tiles; tile t has its parameters at vp + 256 t and
+// its codes at vc + 256 BITS t.  The loop over the two tiles is kept rolled (see qk_half).
 template <int BITS, bool FULL>
-__device__ __forceinline__ void pv_half(uint32_t vp0, uint32_t vp1, uint32_t vc0, uint32_t vc1, int tm,
-                                        const uint32_t (&pf)[2][2], int lane, SoftmaxState& st) {
+__device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const uint32_t (&pf)[2][2], int lane,
+                                        SoftmaxState& st) {
+  constexpr int cb = 256 * BITS;
   const int c4 = lane & 3, r = lane >> 2;
-  // per-lane scales of its token pairs, all four groups: {sA, sB} x 4 per tile
-  uint4 x0, y0, x1, y1;
-  float tz[4];
-  const bool t0 = FULL || (tm & 1), t1 = FULL || (tm & 2);
-  if (t0) {
-    x0 = lds128(vp0 + c4 * 32);
-    y0 = lds128(vp0 + c4 * 32 + 16);
-    // rows g < 4: sum_tok p z[tok][g]; rows 8 + g: sum_tok p s[tok][g] (exact products)
+  float tz[4] = {0.f, 0.f, 0.f, 0.f};   // rows g < 4: sum_tok p z[tok][g]; rows 8 + g: sum_tok p s[tok][g]
+  float ps[4][4];                       // per group: sum over tokens of P' (all rows equal)
+#pragma unroll
+  for (int g = 0; g < 4; ++g) ps[g][0] = ps[g][1] = ps[g][2] = ps[g][3] = 0.f;
+#ifdef GKV_PV_ROLL
+#pragma unroll 1
+#else
+#pragma unroll
+#endif
+  for (int t = 0; t < 2; ++t) {
+    if (!FULL && !((tm >> t) & 1)) continue;
+    const uint32_t p0 = t ? pf[1][0] : pf[0][0], p1 = t ? pf[1][1] : pf[0][1];
+    const uint32_t vpt = vp + t * 256, vct = vc + t * cb;
+    // per-lane scales of its token pairs, all four groups: {sA, sB} x 4
+    const uint4 x = lds128(vpt + c4 * 32), y = lds128(vpt + c4 * 32 + 16);
     uint2 z = make_uint2(0, 0), sg = make_uint2(0, 0);
     if (r < 4) {
-      z = lds64(vp0 + 128 + (r * 4 + c4) * 8);
-      sg = lds64(vp0 + c4 * 32 + r * 8);
+      z = lds64(vpt + 128 + (r * 4 + c4) * 8);
+      sg = lds64(vpt + c4 * 32 + r * 8);
     }
-    mma_f16_first(tz, z.x, sg.x, z.y, sg.y, pf[0][0], pf[0][1]);
-  }
-  if (t1) {
-    x1 = lds128(vp1 + c4 * 32);
-    y1 = lds128(vp1 + c4 * 32 + 16);
-    uint2 z = make_uint2(0, 0), sg = make_uint2(0, 0);
-    if (r < 4) {
-      z = lds64(vp1 + 128 + (r * 4 + c4) * 8);
-      sg = lds64(vp1 + c4 * 32 + r * 8);
-    }
-    if (t0) mma_f16(tz, z.x, sg.x, z.y, sg.y, pf[1][0], pf[1][1]);
-    else mma_f16_first(tz, z.x, sg.x, z.y, sg.y, pf[1][0], pf[1][1]);
+    mma_f16(tz, z.x, sg.x, z.y, sg.y, p0, p1);
+    pv_tile_group<BITS>(vct, 0, lane, hmul2_u32(p0, x.x), hmul2_u32(p1, x.y), ps[0], st.o[0], st.o[1]);
+    pv_tile_group<BITS>(vct, 1, lane, hmul2_u32(p0, x.z), hmul2_u32(p1, x.w), ps[1], st.o[2], st.o[3]);
+    pv_tile_group<BITS>(vct, 2, lane, hmul2_u32(p0, y.x), hmul2_u32(p1, y.y), ps[2], st.o[4], st.o[5]);
+    pv_tile_group<BITS>(vct, 3, lane, hmul2_u32(p0, y.z), hmul2_u32(p1, y.w), ps[3], st.o[6], st.o[7]);
   }
   st.zc[0] += fmaf(Bias<BITS>::mid, tz[2], tz[0]);
   st.zc[1] += fmaf(Bias<BITS>::mid, tz[3], tz[1]);
+  // remove bias + centre: u = 2g is an even MMA index, u = 2g + 1 an odd one
+  constexpr float kMid = Bias<BITS>::mid;
 #pragma unroll
   for (int grp = 0; grp < 4; ++grp) {
-    float ps[4];          // sum over tokens of P' (all rows equal)
-    if (t0) {
-      const uint32_t sa = grp == 0 ? x0.x : grp == 1 ? x0.z : grp == 2 ? y0.x : y0.z;
-      const uint32_t sb = grp == 0 ? x0.y : grp == 1 ? x0.w : grp == 2 ? y0.y : y0.w;
-      pv_tile_group<BITS>(vc0, grp, lane, hmul2_u32(pf[0][0], sa), hmul2_u32(pf[0][1], sb), true, ps,
-                          st.o[2 * grp], st.o[2 * grp + 1]);
-    }
-    if (t1) {
-      const uint32_t sa = grp == 0 ? x1.x : grp == 1 ? x1.z : grp == 2 ? y1.x : y1.z;
-      const uint32_t sb = grp == 0 ? x1.y : grp == 1 ? x1.w : grp == 2 ? y1.y : y1.w;
-      pv_tile_group<BITS>(vc1, grp, lane, hmul2_u32(pf[1][0], sa), hmul2_u32(pf[1][1], sb), !t0, ps,
-                          st.o[2 * grp], st.o[2 * grp + 1]);
-    }
-    // remove bias + centre: u = 2g is an even MMA index, u = 2g + 1 an odd one
-    constexpr float kMid = Bias<BITS>::mid;
-    st.o[2 * grp][0] = fmaf(-(Bias<BITS>::lo_even + kMid), ps[0], st.o[2 * grp][0]);
-    st.o[2 * grp][1] = fmaf(-(Bias<BITS>::lo_even + kMid), ps[1], st.o[2 * grp][1]);
-    st.o[2 * grp][2] = fmaf(-(Bias<BITS>::hi_even + kMid), ps[0], st.o[2 * grp][2]);
-    st.o[2 * grp][3] = fmaf(-(Bias<BITS>::hi_even + kMid), ps[1], st.o[2 * grp][3]);
-    st.o[2 * grp + 1][0] = fmaf(-(Bias<BITS>::lo_odd + kMid), ps[0], st.o[2 * grp + 1][0]);
-    st.o[2 * grp + 1][1] = fmaf(-(Bias<BITS>::lo_odd + kMid), ps[1], st.o[2 * grp + 1][1]);
-    st.o[2 * grp + 1][2] = fmaf(-(Bias<BITS>::hi_odd + kMid), ps[0], st.o[2 * grp + 1][2]);
-    st.o[2 * grp + 1][3] = fmaf(-(Bias<BITS>::hi_odd + kMid), ps[1], st.o[2 * grp + 1][3]);
+    st.o[2 * grp][0] = fmaf(-(Bias<BITS>::lo_even + kMid), ps[grp][0], st.o[2 * grp][0]);
+    st.o[2 * grp][1] = fmaf(-(Bias<BITS>::lo_even + kMid), ps[grp][1], st.o[2 * grp][1]);
+    st.o[2 * grp][2] = fmaf(-(Bias<BITS>::hi_even + kMid), ps[grp][0], st.o[2 * grp][2]);
+    st.o[2 * grp][3] = fmaf(-(Bias<BITS>::hi_even + kMid), ps[grp][1], st.o[2 * grp][3]);
+    st.o[2 * grp + 1][0] = fmaf(-(Bias<BITS>::lo_odd + kMid), ps[grp][0], st.o[2 * grp + 1][0]);
+    st.o[2 * grp + 1][1] = fmaf(-(Bias<BITS>::lo_odd + kMid), ps[grp][1], st.o[2 * grp + 1][1]);
+    st.o[2 * grp + 1][2] = fmaf(-(Bias<BITS>::hi_odd + kMid), ps[grp][0], st.o[2 * grp + 1][2]);
+    st.o[2 * grp + 1][3] = fmaf(-(Bias<BITS>::hi_odd + kMid), ps[grp][1], st.o[2 * grp + 1][3]);
   }
 }
 
 template <int BITS, bool FULL>
-__device__ __forceinline__ void qk_softmax_half(uint32_t half_k, int half, int tm, uint64_t resmask,
-                                                const uint32_t (&qh)[16], int lane, float scale_log2,
-                                                SoftmaxState& st, uint32_t (&pf)[2][2]) {
-  constexpr int cb = 256 * BITS;
+__device__ __forceinline__ void qk_softmax_half(uint32_t half_k, int half, int tm, uint64_t resmask, uint32_t qh_addr,
+                                                int lane, float scale_log2, SoftmaxState& st, uint32_t (&pf)[2][2]) {
   float S[2][4];
-  qk_half<BITS, FULL>(half_k, half_k + 512, half_k + 512 + cb, tm, qh, lane, scale_log2, resmask, half, S);
+  qk_half<BITS, FULL>(half_k, half_k + 512, tm, qh_addr, lane, scale_log2, resmask, half, S);
   softmax_update<2>(S, st);
   make_p_f16(S[0], pf[0], st);
   make_p_f16(S[1], pf[1], st);
@@ -770,8 +757,8 @@ __device__ __forceinline__ void qk_softmax_half(uint32_t half_k, int half, int t
 
 // Process a staged step.  pf carries P fragments from a key step to the following value step.
 template <bool SPARSE>
-__device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, int sidx,
-                                             const uint32_t (&qh)[16], SoftmaxState& st, uint32_t (&pf)[4]) {
+__device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, int sidx, SoftmaxState& st,
+                                             uint32_t (&pf)[4]) {
   const DecodeParams& p = *w.p;
   const int lane = w.lane;
   const uint32_t sa = w.stage0 + sidx * kStageBytes;
@@ -833,24 +820,21 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
   }
   uint32_t (&pf2)[2][2] = *reinterpret_cast<uint32_t (*)[2][2]>(&pf);
   constexpr bool FULL = !SPARSE;
+  const uint32_t qh = w.qh_addr;
   if (c.level == 8) {
     const int half = FULL ? (c.sub >> 1) : ((c.tmask == 15) ? (c.sub >> 1) : half_of_step(c, c.sub >> 1));
     const int tm = (c.tmask >> (2 * half)) & 3;
     if ((c.sub & 1) == 0) qk_softmax_half<8, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
-    else pv_half<8, FULL>(sa, sa + 256, sa + 512, sa + 512 + 2048, tm, pf2, lane, st);
-  } else if (c.level == 4) {
+    else pv_half<8, FULL>(sa, sa + 512, tm, pf2, lane, st);
+  } else {
     const int half = FULL ? c.sub : ((c.tmask == 15) ? c.sub : half_of_step(c, c.sub));
     const int tm = (c.tmask >> (2 * half)) & 3;
-    qk_softmax_half<4, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
-    pv_half<4, FULL>(sa + off_vp(4, 0), sa + off_vp(4, 1), sa + off_vc(4, 0), sa + off_vc(4, 1), tm, pf2, lane, st);
-  } else {
-#pragma unroll 1
-    for (int half = 0; half < 2; ++half) {
-      const int tm = (c.tmask >> (2 * half)) & 3;
-      if (!FULL && tm == 0) continue;
-      const uint32_t hb = sa + half * half_bytes(2);
-      qk_softmax_half<2, FULL>(hb, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
-      pv_half<2, FULL>(hb + off_vp(2, 0), hb + off_vp(2, 1), hb + off_vc(2, 0), hb + off_vc(2, 1), tm, pf2, lane, st);
+    if (c.level == 4) {
+      qk_softmax_half<4, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
+      pv_half<4, FULL>(sa + off_vp(4, 0), sa + off_vc(4, 0), tm, pf2, lane, st);
+    } else {
+      qk_softmax_half<2, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
+      pv_half<2, FULL>(sa + off_vp(2, 0), sa + off_vc(2, 0), tm, pf2, lane, st);
     }
   }
 }
@@ -895,6 +879,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   w.stage0 = smem_u32(sbase);
   w.bar0 = smem_u32(bars);
   w.qb_addr = smem_u32(qb_smem) + lane * 8;       // word pair s at + 256 s (conflict-free 8-byte accesses)
+  w.qh_addr = w.qb_addr + kDecodeWarps * 2048;
   if (lane == 0) {
 #pragma unroll
     for (int s = 0; s < kStages; ++s) mbar_init(w.bar0 + 8 * s, 1);
@@ -905,7 +890,6 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   // Query fragments: B operand Q^T[16 channels x 8 heads]; lane (r, c4) holds head r, channels
   // 16 s + 2 c4 (+1) and 16 s + 8 + 2 c4 (+1), in bf16 (exact rows) and fp16 (quantised tiers).
   const int r = lane >> 2, c4 = lane & 3;
-  uint32_t qh[16];
   {
     const int b = w.stream / p.n_kv_heads, kvh = w.stream - b * p.n_kv_heads;
     const int n_q_heads = p.n_kv_heads * p.group;
@@ -918,10 +902,12 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
         v1 = *reinterpret_cast<const uint32_t*>(qrow + 16 * s + 8 + 2 * c4);
       }
       asm volatile("st.shared.v2.u32 [%0], {%1,%2};\n" ::"r"(w.qb_addr + s * 256), "r"(v0), "r"(v1) : "memory");
-      qh[2 * s] = h2_as_u32(__floats2half2_rn(bf16lo_to_f32(v0), bf16hi_to_f32(v0)));
-      qh[2 * s + 1] = h2_as_u32(__floats2half2_rn(bf16lo_to_f32(v1), bf16hi_to_f32(v1)));
+      const uint32_t h0 = h2_as_u32(__floats2half2_rn(bf16lo_to_f32(v0), bf16hi_to_f32(v0)));
+      const uint32_t h1 = h2_as_u32(__floats2half2_rn(bf16lo_to_f32(v1), bf16hi_to_f32(v1)));
+      asm volatile("st.shared.v2.u32 [%0], {%1,%2};\n" ::"r"(w.qh_addr + s * 256), "r"(h0), "r"(h1) : "memory");
     }
   }
+  __syncwarp();
 
   SoftmaxState st;
   st.m0 = st.m1 = kNegInf;
@@ -934,6 +920,8 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
 #ifdef GKV_EXP_PROFILE
   long long prof_wait = 0, prof_steps = 0;
   const long long prof_t0 = clock64();
+  unsigned long long prof_g0;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(prof_g0));
 #endif
   Cursor cur;
   bool have = load_item<SPARSE>(w, first, cur);
@@ -968,7 +956,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     phase ^= 1u << sidx;
     __syncwarp();
 #ifndef GKV_EXP_SKIP_COMPUTE
-    compute_step<SPARSE>(w, cur, sidx, qh, st, pf);
+    compute_step<SPARSE>(w, cur, sidx, st, pf);
 #endif
     __syncwarp();
     cur = nxt;
@@ -976,9 +964,12 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     sidx ^= 1;
   }
 #ifdef GKV_EXP_PROFILE
-  if (lane == 0 && (gw % 97) == 0)
-    printf("PROF warp %d stream %d items %d steps %lld total %lld wait %lld\n", gw, w.stream, w.item_end - first, prof_steps,
-           clock64() - prof_t0, prof_wait);
+  if (lane == 0 && (gw % 13) == 0) {
+    unsigned long long prof_g1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(prof_g1));
+    printf("PROF warp %d stream %d items %d steps %lld total %lld wait %lld g0 %llu g1 %llu\n", gw, w.stream, w.item_end - first,
+           prof_steps, clock64() - prof_t0, prof_wait, prof_g0 % 1000000000ull, prof_g1 % 1000000000ull);
+  }
 #endif
   if (failed) {
     // a copy never completed: flag it and publish an empty partial (the host reports BAD_STATE)
@@ -1074,7 +1065,7 @@ __global__ void __launch_bounds__(kD) combine_kernel(const __grid_constant__ Com
 
 size_t decode_smem_bytes() {
   // per warp: pipeline stages, their mbarriers, and the bf16 query fragments (2 KiB)
-  return static_cast<size_t>(kDecodeWarps) * (kStages * kStageBytes + kStages * sizeof(uint64_t) + 2048);
+  return static_cast<size_t>(kDecodeWarps) * (kStages * kStageBytes + kStages * sizeof(uint64_t) + 2 * 2048);
 }
 
 cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st) {

@@ -39,7 +39,7 @@ struct alignas(8) StreamParts {
 #define GKV_DECODE_CTAS_PER_SM 2
 #endif
 constexpr int kDecodeWarps = GKV_DECODE_WARPS;               // warps per CTA of the decode kernel
-constexpr int kStageBytes = 6144;           // per-warp pipeline stage
+constexpr int kStageBytes = 5120;           // per-warp pipeline stage
 constexpr int kStages = 2;
 constexpr int kDecodeCtasPerSm = GKV_DECODE_CTAS_PER_SM;
 constexpr int kMaxHeadsPerKv = 8;           // one n=8 tensor-core tile of query heads
