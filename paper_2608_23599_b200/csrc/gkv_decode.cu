@@ -598,7 +598,7 @@ __device__ __forceinline__ void load_words(uint32_t codes, int j, int lane, uint
 // Channel slab j (MMA indices 2 j and 2 j + 1) of qk_half; FIRST starts the accumulation chains.
 template <int BITS, bool FULL, bool FIRST>
 __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm, uint32_t qh_addr, int lane,
-                                        float (&zd)[4], float (&qe)[4], float (&qo)[4], float (&S)[2][4]) {
+                                        const uint32_t (&ones)[4], float (&zd)[4], float (&qe)[4], float (&qo)[4], float (&S)[2][4]) {
   constexpr int cb = 256 * BITS;
   constexpr int kW = BITS / 2;
   uint32_t w0[kW], w1[kW];
@@ -609,14 +609,14 @@ __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm
     const uint4 pr = lds128(kp + j * 128 + ss * 64);   // s01, z01, s23, z23
     const uint2 q = lds64(qh_addr + j * 512 + ss * 256);
     const uint32_t q0 = hmul2_u32(q.x, pr.x), q1 = hmul2_u32(q.y, pr.z);
-    if (FIRST && ss == 0) mma_f16_first(zd, pr.y, pr.x, pr.w, pr.z, q.x, q.y);
-    else mma_f16(zd, pr.y, pr.x, pr.w, pr.z, q.x, q.y);
+    if (FIRST && ss == 0) mma_f16_first(zd, pr.x, pr.y, pr.z, pr.w, q.x, q.y);
+    else mma_f16(zd, pr.x, pr.y, pr.z, pr.w, q.x, q.y);
     if (BITS == 2 && ss == 1) {
-      if (FIRST) mma_f16_first(qo, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
-      else mma_f16(qo, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
+      if (FIRST) mma_f16_first(qo, ones[0], ones[1], ones[2], ones[3], q0, q1);
+      else mma_f16(qo, ones[0], ones[1], ones[2], ones[3], q0, q1);
     } else {
-      if (FIRST && ss == 0) mma_f16_first(qe, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
-      else mma_f16(qe, kOnesH2, kOnesH2, kOnesH2, kOnesH2, q0, q1);
+      if (FIRST && ss == 0) mma_f16_first(qe, ones[0], ones[1], ones[2], ones[3], q0, q1);
+      else mma_f16(qe, ones[0], ones[1], ones[2], ones[3], q0, q1);
     }
     uint32_t a[4];
     if (FULL || (tm & 1)) {
@@ -634,22 +634,22 @@ __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm
 
 template <int BITS, bool FULL>
 __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, int tm, uint32_t qh_addr, int lane, float scale_log2,
-                                        uint64_t resmask, int half, float (&S)[2][4]) {
+                                        uint64_t resmask, int half, const uint32_t (&ones)[4], float (&S)[2][4]) {
   const int c4 = lane & 3, r = lane >> 2;
-  float zd[4];        // rows r: sum_c q_c z_c; rows r + 8: sum_c q_c s_c (exact products)
+  float zd[4];        // rows r: sum_c q_c s_c; rows r + 8: sum_c q_c z_c (exact products)
   float qe[4];        // sum_c q'_c over even MMA indices (all rows equal)
   float qo[4] = {0.f, 0.f, 0.f, 0.f};   // ... over odd MMA indices (2-bit only)
   kp += c4 * 16;
-  qk_slab<BITS, FULL, true>(kp, kc0, 0, tm, qh_addr, lane, zd, qe, qo, S);
+  qk_slab<BITS, FULL, true>(kp, kc0, 0, tm, qh_addr, lane, ones, zd, qe, qo, S);
 #pragma unroll 1
-  for (int j = 1; j < 4; ++j) qk_slab<BITS, FULL, false>(kp, kc0, j, tm, qh_addr, lane, zd, qe, qo, S);
+  for (int j = 1; j < 4; ++j) qk_slab<BITS, FULL, false>(kp, kc0, j, tm, qh_addr, lane, ones, zd, qe, qo, S);
   if (!FULL) {
     if (!(tm & 1)) S[0][0] = S[0][1] = S[0][2] = S[0][3] = 0.f;
     if (!(tm & 2)) S[1][0] = S[1][1] = S[1][2] = S[1][3] = 0.f;
   }
   // rows r carry bias lo, rows r + 8 carry bias hi (per parity of the MMA index)
   constexpr float kMid = Bias<BITS>::mid;
-  const float z0 = fmaf(kMid, zd[2], zd[0]), z1 = fmaf(kMid, zd[3], zd[1]);     // sum q (z + mid s)
+  const float z0 = fmaf(kMid, zd[0], zd[2]), z1 = fmaf(kMid, zd[1], zd[3]);     // sum q (z + mid s)
   const float c_lo0 = z0 - (Bias<BITS>::lo_even + kMid) * qe[0] - (Bias<BITS>::lo_odd + kMid) * qo[0];
   const float c_lo1 = z1 - (Bias<BITS>::lo_even + kMid) * qe[1] - (Bias<BITS>::lo_odd + kMid) * qo[1];
   const float c_hi0 = z0 - (Bias<BITS>::hi_even + kMid) * qe[0] - (Bias<BITS>::hi_odd + kMid) * qo[0];
@@ -682,12 +682,12 @@ __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, int tm, uint3
 // One tile's share of O^T += V~^T P^T for group grp: data MMAs accumulate (bias + code) * P' straight
 // into O; `ps` collects sum P' so that the bias can be taken out afterwards.
 template <int BITS>
-__device__ __forceinline__ void pv_tile_group(uint32_t vc, int grp, int lane, uint32_t p0, uint32_t p1, float (&ps)[4],
-                                              float (&o0)[4], float (&o1)[4]) {
+__device__ __forceinline__ void pv_tile_group(uint32_t vc, int grp, int lane, uint32_t p0, uint32_t p1,
+                                              const uint32_t (&ones)[4], float (&ps)[4], float (&o0)[4], float (&o1)[4]) {
   uint32_t wd[BITS / 2];
   uint32_t a[4];
   load_words<BITS>(vc, grp, lane, wd);
-  mma_f16(ps, kOnesH2, kOnesH2, kOnesH2, kOnesH2, p0, p1);
+  mma_f16(ps, ones[0], ones[1], ones[2], ones[3], p0, p1);
   unpack<BITS>(wd, 0, a);
   mma_f16(o0, a[0], a[1], a[2], a[3], p0, p1);
   unpack<BITS>(wd, 1, a);
@@ -699,7 +699,7 @@ __device__ __forceinline__ void pv_tile_group(uint32_t vc, int grp, int lane, ui
 // its codes at vc + 256 BITS t.  The loop over the two tiles is kept rolled (see qk_half).
 template <int BITS, bool FULL>
 __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const uint32_t (&pf)[2][2], int lane,
-                                        SoftmaxState& st) {
+                                        const uint32_t (&ones)[4], SoftmaxState& st) {
   constexpr int cb = 256 * BITS;
   const int c4 = lane & 3, r = lane >> 2;
   float tz[4] = {0.f, 0.f, 0.f, 0.f};   // rows g < 4: sum_tok p z[tok][g]; rows 8 + g: sum_tok p s[tok][g]
@@ -723,10 +723,10 @@ __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const 
       sg = lds64(vpt + c4 * 32 + r * 8);
     }
     mma_f16(tz, z.x, sg.x, z.y, sg.y, p0, p1);
-    pv_tile_group<BITS>(vct, 0, lane, hmul2_u32(p0, x.x), hmul2_u32(p1, x.y), ps[0], st.o[0], st.o[1]);
-    pv_tile_group<BITS>(vct, 1, lane, hmul2_u32(p0, x.z), hmul2_u32(p1, x.w), ps[1], st.o[2], st.o[3]);
-    pv_tile_group<BITS>(vct, 2, lane, hmul2_u32(p0, y.x), hmul2_u32(p1, y.y), ps[2], st.o[4], st.o[5]);
-    pv_tile_group<BITS>(vct, 3, lane, hmul2_u32(p0, y.z), hmul2_u32(p1, y.w), ps[3], st.o[6], st.o[7]);
+    pv_tile_group<BITS>(vct, 0, lane, hmul2_u32(p0, x.x), hmul2_u32(p1, x.y), ones, ps[0], st.o[0], st.o[1]);
+    pv_tile_group<BITS>(vct, 1, lane, hmul2_u32(p0, x.z), hmul2_u32(p1, x.w), ones, ps[1], st.o[2], st.o[3]);
+    pv_tile_group<BITS>(vct, 2, lane, hmul2_u32(p0, y.x), hmul2_u32(p1, y.y), ones, ps[2], st.o[4], st.o[5]);
+    pv_tile_group<BITS>(vct, 3, lane, hmul2_u32(p0, y.z), hmul2_u32(p1, y.w), ones, ps[3], st.o[6], st.o[7]);
   }
   st.zc[0] += fmaf(Bias<BITS>::mid, tz[2], tz[0]);
   st.zc[1] += fmaf(Bias<BITS>::mid, tz[3], tz[1]);
@@ -747,9 +747,10 @@ __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const 
 
 template <int BITS, bool FULL>
 __device__ __forceinline__ void qk_softmax_half(uint32_t half_k, int half, int tm, uint64_t resmask, uint32_t qh_addr,
-                                                int lane, float scale_log2, SoftmaxState& st, uint32_t (&pf)[2][2]) {
+                                                int lane, float scale_log2, const uint32_t (&ones)[4], SoftmaxState& st,
+                                                uint32_t (&pf)[2][2]) {
   float S[2][4];
-  qk_half<BITS, FULL>(half_k, half_k + 512, tm, qh_addr, lane, scale_log2, resmask, half, S);
+  qk_half<BITS, FULL>(half_k, half_k + 512, tm, qh_addr, lane, scale_log2, resmask, half, ones, S);
   softmax_update<2>(S, st);
   make_p_f16(S[0], pf[0], st);
   make_p_f16(S[1], pf[1], st);
@@ -757,8 +758,8 @@ __device__ __forceinline__ void qk_softmax_half(uint32_t half_k, int half, int t
 
 // Process a staged step.  pf carries P fragments from a key step to the following value step.
 template <bool SPARSE>
-__device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, int sidx, SoftmaxState& st,
-                                             uint32_t (&pf)[4]) {
+__device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, int sidx, const uint32_t (&ones)[4],
+                                             SoftmaxState& st, uint32_t (&pf)[4]) {
   const DecodeParams& p = *w.p;
   const int lane = w.lane;
   const uint32_t sa = w.stage0 + sidx * kStageBytes;
@@ -824,17 +825,17 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
   if (c.level == 8) {
     const int half = FULL ? (c.sub >> 1) : ((c.tmask == 15) ? (c.sub >> 1) : half_of_step(c, c.sub >> 1));
     const int tm = (c.tmask >> (2 * half)) & 3;
-    if ((c.sub & 1) == 0) qk_softmax_half<8, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
-    else pv_half<8, FULL>(sa, sa + 512, tm, pf2, lane, st);
+    if ((c.sub & 1) == 0) qk_softmax_half<8, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, ones, st, pf2);
+    else pv_half<8, FULL>(sa, sa + 512, tm, pf2, lane, ones, st);
   } else {
     const int half = FULL ? c.sub : ((c.tmask == 15) ? c.sub : half_of_step(c, c.sub));
     const int tm = (c.tmask >> (2 * half)) & 3;
     if (c.level == 4) {
-      qk_softmax_half<4, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
-      pv_half<4, FULL>(sa + off_vp(4, 0), sa + off_vc(4, 0), tm, pf2, lane, st);
+      qk_softmax_half<4, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, ones, st, pf2);
+      pv_half<4, FULL>(sa + off_vp(4, 0), sa + off_vc(4, 0), tm, pf2, lane, ones, st);
     } else {
-      qk_softmax_half<2, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
-      pv_half<2, FULL>(sa + off_vp(2, 0), sa + off_vc(2, 0), tm, pf2, lane, st);
+      qk_softmax_half<2, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, ones, st, pf2);
+      pv_half<2, FULL>(sa + off_vp(2, 0), sa + off_vc(2, 0), tm, pf2, lane, ones, st);
     }
   }
 }
@@ -916,6 +917,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   for (int u = 0; u < 8; ++u) st.o[u][0] = st.o[u][1] = st.o[u][2] = st.o[u][3] = 0.f;
   st.zc[0] = st.zc[1] = st.zc[2] = st.zc[3] = 0.f;
   uint32_t pf[4] = {0, 0, 0, 0};
+  // half2(1, 1) four times: the A operand of the column-sum MMAs.  Produced by opaque moves so that
+  // the compiler keeps one register quad for the whole kernel instead of rebuilding it per MMA.
+  uint32_t ones[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) asm volatile("mov.b32 %0, %1;\n" : "=r"(ones[i]) : "r"(kOnesH2));
 
 #ifdef GKV_EXP_PROFILE
   long long prof_wait = 0, prof_steps = 0;
@@ -956,7 +962,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     phase ^= 1u << sidx;
     __syncwarp();
 #ifndef GKV_EXP_SKIP_COMPUTE
-    compute_step<SPARSE>(w, cur, sidx, st, pf);
+    compute_step<SPARSE>(w, cur, sidx, ones, st, pf);
 #endif
     __syncwarp();
     cur = nxt;
