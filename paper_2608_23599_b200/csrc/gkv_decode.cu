@@ -641,7 +641,11 @@ __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, int tm, uint3
   float qo[4] = {0.f, 0.f, 0.f, 0.f};   // ... over odd MMA indices (2-bit only)
   kp += c4 * 16;
   qk_slab<BITS, FULL, true>(kp, kc0, 0, tm, qh_addr, lane, ones, zd, qe, qo, S);
+#ifdef GKV_QK_ROLL
 #pragma unroll 1
+#else
+#pragma unroll
+#endif
   for (int j = 1; j < 4; ++j) qk_slab<BITS, FULL, false>(kp, kc0, j, tm, qh_addr, lane, ones, zd, qe, qo, S);
   if (!FULL) {
     if (!(tm & 1)) S[0][0] = S[0][1] = S[0][2] = S[0][3] = 0.f;
@@ -929,42 +933,55 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   unsigned long long prof_g0;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(prof_g0));
 #endif
+  // Software pipeline over steps: while step k is computed, step k + 1 is in flight.  The loop
+  // starts on an empty pseudo-unit (level 0) so that the cursor and copy code exists once.
   Cursor cur;
-  bool have = load_item<SPARSE>(w, first, cur);
-  int sidx = 0;
+  cur.item = first - 1;
+  cur.first = 0;
+  cur.sub = 0;
+  cur.nsub = 1;
+  cur.adv = 1;
+  cur.level = 0;
+  cur.ntok = 0;
+  cur.tmask = 0;
+  cur.off256 = 0;
+  cur.resmask = 0;
+  bool have = true;
+  int sidx = 1;
   uint32_t phase = 0;             // bit s = parity to wait for on stage s
   bool failed = false;
-#ifndef GKV_EXP_SKIP_COPY
-  if (have) issue_step<SPARSE>(w, cur, 0);
-#endif
   while (have) {
     Cursor nxt = cur;
     const bool more = advance<SPARSE>(w, nxt);
 #ifndef GKV_EXP_SKIP_COPY
     if (more) issue_step<SPARSE>(w, nxt, sidx ^ 1);
-#ifdef GKV_EXP_PROFILE
-    const long long tw0 = clock64();
 #endif
-    // bounded wait for this step's bytes
-    int spins = 0;
-    while (!mbar_try_wait(w.bar0 + 8 * sidx, (phase >> sidx) & 1u)) {
-      if (++spins > kWaitSpins) {
-        failed = true;
-        break;
+    if (cur.level != 0) {
+#ifndef GKV_EXP_SKIP_COPY
+#ifdef GKV_EXP_PROFILE
+      const long long tw0 = clock64();
+#endif
+      // bounded wait for this step's bytes
+      int spins = 0;
+      while (!mbar_try_wait(w.bar0 + 8 * sidx, (phase >> sidx) & 1u)) {
+        if (++spins > kWaitSpins) {
+          failed = true;
+          break;
+        }
       }
-    }
-#endif
-    if (__any_sync(kFull, failed)) break;
+      if (__any_sync(kFull, failed)) break;
 #ifdef GKV_EXP_PROFILE
-    prof_wait += clock64() - tw0;
-    prof_steps += 1;
+      prof_wait += clock64() - tw0;
+      prof_steps += 1;
 #endif
-    phase ^= 1u << sidx;
-    __syncwarp();
+      phase ^= 1u << sidx;
+#endif
+      __syncwarp();
 #ifndef GKV_EXP_SKIP_COMPUTE
-    compute_step<SPARSE>(w, cur, sidx, ones, st, pf);
+      compute_step<SPARSE>(w, cur, sidx, ones, st, pf);
 #endif
-    __syncwarp();
+      __syncwarp();
+    }
     cur = nxt;
     have = more;
     sidx ^= 1;
