@@ -33,10 +33,10 @@ struct alignas(8) StreamParts {
 };
 
 #ifndef GKV_DECODE_WARPS
-#define GKV_DECODE_WARPS 8
+#define GKV_DECODE_WARPS 16
 #endif
 #ifndef GKV_DECODE_CTAS_PER_SM
-#define GKV_DECODE_CTAS_PER_SM 2
+#define GKV_DECODE_CTAS_PER_SM 1
 #endif
 constexpr int kDecodeWarps = GKV_DECODE_WARPS;               // warps per CTA of the decode kernel
 constexpr int kStageBytes = 5120;           // per-warp pipeline stage
