@@ -19,7 +19,7 @@ using namespace gkv;
 namespace {
 
 constexpr int kTargetWarps = 148 * kDecodeCtasPerSm * kDecodeWarps;   // one resident wave of CTAs
-constexpr int kSparseWarpsPerStream = 16;
+constexpr int kSparseWarpsPerStream = kDecodeWarps;   // page-list reads: one CTA per stream
 constexpr size_t kMinWarpCost = 1000;     // do not split below about one block per warp
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -414,7 +414,7 @@ void build_descs(gkv_cache* c, LayerState& L) {
     total += cost[s];
   }
   const size_t target = std::max(kMinWarpCost, (total + kTargetWarps - 1) / kTargetWarps);
-  int w = 0, pos = 0;
+  int w = 0, pos = 0, row = 0;
   std::vector<size_t> load;
   std::vector<std::vector<uint32_t>> mine;
   for (int s = 0; s < ns; ++s) {
@@ -435,7 +435,8 @@ void build_descs(gkv_cache* c, LayerState& L) {
       load[best] += x.cost;
       mine[best].push_back(x.word);
     }
-    L.parts_h[s].begin = w;
+    // one partial row per (CTA, stream): the kernel merges the warps of a CTA that share a stream
+    L.parts_h[s].begin = row;
     for (int k = 0; k < nw; ++k) {
       std::sort(mine[k].begin(), mine[k].end(), [](uint32_t a, uint32_t b) { return (a & 0xffffffu) < (b & 0xffffffu); });
       WarpDesc& d = L.warps_h[w];
@@ -443,10 +444,12 @@ void build_descs(gkv_cache* c, LayerState& L) {
       d.item_begin = pos;
       for (uint32_t x : mine[k]) L.units_h[pos++] = x;
       d.item_end = pos;
-      d.partial = w;
+      if (k > 0 && w % kDecodeWarps == 0) ++row;
+      d.partial = row;
       ++w;
     }
-    L.parts_h[s].end = w;
+    ++row;
+    L.parts_h[s].end = row;
   }
   const int padded = static_cast<int>(align_up(w, kDecodeWarps));
   for (int i = w; i < padded; ++i) L.warps_h[i] = WarpDesc{-1, 0, 0, 0};
@@ -1170,7 +1173,7 @@ int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* p
     p.n_warps = c->n_streams * kSparseWarpsPerStream;
     p.warps = nullptr;
     cp.parts = nullptr;
-    cp.warps_per_stream = kSparseWarpsPerStream;
+    cp.warps_per_stream = 1;            // the kernel leaves one merged row per stream
     n_ctas = (p.n_warps + kDecodeWarps - 1) / kDecodeWarps;
     L.last_mode = 2;
     L.last_pages = page_idx;

@@ -849,7 +849,6 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gw = blockIdx.x * kDecodeWarps + warp;
-  if (gw >= p.n_warps) return;
 
   WarpCtx w;
   w.p = &p;
@@ -858,24 +857,34 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   w.pf_pos = -1;
   w.pf_unit = 0;
   w.pf_entry = make_uint4(0, 0, 0, 0);
-  int partial_row, first;
-  if constexpr (!SPARSE) {
-    const WarpDesc wd = p.warps[gw];
-    if (wd.stream < 0) return;
-    w.stream = wd.stream;
-    w.item_end = wd.item_end;
-    w.has_tail = false;
-    first = wd.item_begin;
-    partial_row = wd.partial;
-  } else {
-    const int wps = p.warps_per_stream;
-    w.stream = gw / wps;
-    const int wi = gw - w.stream * wps;
-    first = static_cast<int>((static_cast<long long>(wi) * p.n_sel) / wps);
-    w.item_end = static_cast<int>((static_cast<long long>(wi + 1) * p.n_sel) / wps);
-    w.has_tail = (wi == wps - 1);
-    partial_row = gw;
+  w.stream = -1;
+  w.item_end = 0;
+  w.has_tail = false;
+  int partial_row = 0, first = 0;
+  if (gw < p.n_warps) {
+    if constexpr (!SPARSE) {
+      const WarpDesc wd = p.warps[gw];
+      w.stream = wd.stream;
+      w.item_end = wd.item_end;
+      first = wd.item_begin;
+      partial_row = wd.partial;
+    } else {
+      const int wps = p.warps_per_stream;
+      w.stream = gw / wps;
+      const int wi = gw - w.stream * wps;
+      first = static_cast<int>((static_cast<long long>(wi) * p.n_sel) / wps);
+      w.item_end = static_cast<int>((static_cast<long long>(wi + 1) * p.n_sel) / wps);
+      w.has_tail = (wi == wps - 1);
+      partial_row = blockIdx.x;      // kDecodeWarps warps per stream: one CTA, one partial row
+    }
   }
+  // per-warp (stream, partial row) for the merge at the end
+  int* s_group = reinterpret_cast<int*>(smem + kDecodeWarps * (kStages * kStageBytes + kStages * 8 + 2 * 2048));
+  if (lane == 0) {
+    s_group[warp] = w.stream;
+    s_group[kDecodeWarps + warp] = partial_row;
+  }
+  if (w.stream >= 0) {
   w.table = p.table + static_cast<size_t>(w.stream) * p.table_stride;
   uint8_t* sbase = smem + warp * (kStages * kStageBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kDecodeWarps * kStages * kStageBytes) + warp * kStages;
@@ -987,7 +996,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     sidx ^= 1;
   }
 #ifdef GKV_EXP_PROFILE
-  if (lane == 0 && (gw % 13) == 0) {
+  if (lane == 0 && (blockIdx.x % 10) == 0) {
     unsigned long long prof_g1;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(prof_g1));
     printf("PROF warp %d stream %d items %d steps %lld total %lld wait %lld g0 %llu g1 %llu\n", gw, w.stream, w.item_end - first,
@@ -1014,23 +1023,60 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     st.o[2 * g][0] += z0; st.o[2 * g][1] += z1; st.o[2 * g][2] += z0; st.o[2 * g][3] += z1;
     st.o[2 * g + 1][0] += z0; st.o[2 * g + 1][1] += z1; st.o[2 * g + 1][2] += z0; st.o[2 * g + 1][3] += z1;
   }
-  float* out = p.partial + static_cast<size_t>(partial_row) * kPartialFloats;
+  // the warp's partial row goes to its own (now idle) stage memory
+  float* out = reinterpret_cast<float*>(sbase);
   const int h0 = 2 * c4, h1 = 2 * c4 + 1;
   if (r == 0) {
-    if (h0 < p.group) { out[h0 * (kD + 2)] = st.m0; out[h0 * (kD + 2) + 1] = st.l0; }
-    if (h1 < p.group) { out[h1 * (kD + 2)] = st.m1; out[h1 * (kD + 2) + 1] = st.l1; }
+    out[h0 * (kD + 2)] = st.m0; out[h0 * (kD + 2) + 1] = st.l0;
+    out[h1 * (kD + 2)] = st.m1; out[h1 * (kD + 2) + 1] = st.l1;
   }
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
     const int ch = 16 * u + r;
-    if (h0 < p.group) {
-      out[h0 * (kD + 2) + 2 + ch] = st.o[u][0];
-      out[h0 * (kD + 2) + 2 + ch + 8] = st.o[u][2];
+    out[h0 * (kD + 2) + 2 + ch] = st.o[u][0];
+    out[h0 * (kD + 2) + 2 + ch + 8] = st.o[u][2];
+    out[h1 * (kD + 2) + 2 + ch] = st.o[u][1];
+    out[h1 * (kD + 2) + 2 + ch + 8] = st.o[u][3];
+  }
+  }   // w.stream >= 0
+
+  // Merge the rows of the CTA's warps that share a stream (they are neighbours) into one global
+  // partial row per (CTA, stream), in warp order; every warp of the CTA arrives here exactly once.
+  __syncthreads();
+  constexpr int kRowFloats = kStages * kStageBytes / 4;     // distance between two warps' rows
+  const float* rows = reinterpret_cast<const float*>(smem);
+  const int n_elem = p.group * (kD + 2);
+  int gb = 0;
+#pragma unroll 1
+  while (gb < kDecodeWarps) {
+    const int sid = s_group[gb];
+    int ge = gb + 1;
+#pragma unroll 1
+    while (ge < kDecodeWarps && s_group[ge] == sid) ++ge;
+    if (sid >= 0) {
+      float* dst = p.partial + static_cast<size_t>(s_group[kDecodeWarps + gb]) * kPartialFloats;
+#pragma unroll 1
+      for (int e = threadIdx.x; e < n_elem; e += kDecodeWarps * 32) {
+        const int h = e / (kD + 2), j = e - h * (kD + 2);
+        const float* col = rows + h * (kD + 2);
+        float M = kNegInf;
+#pragma unroll 1
+        for (int i = gb; i < ge; ++i) M = fmaxf(M, col[i * kRowFloats]);
+        float acc = 0.f;
+        if (j == 0) {
+          acc = M;
+        } else {
+#pragma unroll 2
+          for (int i = gb; i < ge; ++i) {
+            const float m = col[i * kRowFloats];
+            const float wgt = (m == kNegInf) ? 0.f : fast_exp2(m - M);
+            acc = fmaf(wgt, col[i * kRowFloats + j], acc);
+          }
+        }
+        dst[e] = acc;
+      }
     }
-    if (h1 < p.group) {
-      out[h1 * (kD + 2) + 2 + ch] = st.o[u][1];
-      out[h1 * (kD + 2) + 2 + ch + 8] = st.o[u][3];
-    }
+    gb = ge;
   }
 }
 
@@ -1088,7 +1134,7 @@ __global__ void __launch_bounds__(kD) combine_kernel(const __grid_constant__ Com
 
 size_t decode_smem_bytes() {
   // per warp: pipeline stages, their mbarriers, and the bf16 query fragments (2 KiB)
-  return static_cast<size_t>(kDecodeWarps) * (kStages * kStageBytes + kStages * sizeof(uint64_t) + 2 * 2048);
+  return static_cast<size_t>(kDecodeWarps) * (kStages * kStageBytes + kStages * sizeof(uint64_t) + 2 * 2048 + 2 * sizeof(int));
 }
 
 cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st) {
