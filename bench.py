@@ -269,7 +269,7 @@ def run_ours(args, rank, local, world):
     h2d = hk.numel() * 2 + (0 if alias else hv.numel() * 2) + hq.numel() * 2
     d2h = hout.numel() * 4
 
-    launches_per_layer = 3 + (2 if quest else 0)      # append, decode, combine (+ score, top-k)
+    launches_per_layer = 2 + (2 if quest else 0)      # append, decode with fused merge (+ score, top-k)
     gpu_launches = K * n_layers * launches_per_layer + closes * n_layers * (1 + (1 if wl.page_tokens else 0))
 
     line = {
@@ -287,7 +287,7 @@ def run_ours(args, rank, local, world):
         "gpu_launches": gpu_launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_kind": peak_kind + " copy bandwidth",
-                     "kernel": "decode_kernel (+ its combine_kernel, timed per gkv_decode_attn call)",
+                     "kernel": "decode_kernel (split-K partials merged in the same launch; timed per gkv_decode_attn call)",
                      "us_per_launch": us_launch, "algorithmic_bytes_per_launch": algo_bytes,
                      "frac_of_8TBs": achieved / NOMINAL_HBM_GBS},
         "ctx_tokens_per_s_per_layer_call": Bsz * ctx_start / (us_launch * 1e-6),

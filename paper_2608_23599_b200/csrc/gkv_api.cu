@@ -125,6 +125,7 @@ struct gkv_cache {
   int8_t* levels_d = nullptr;
   float* scores_d = nullptr;            // residual scores [n_streams][max_ctx] or page scores
   int32_t* kper_d = nullptr;
+  int32_t* tickets_d = nullptr;         // per-stream arrival counters of the decode kernel's final merge
   EncodeJob* jobs_d = nullptr;
   size_t jobs_cap = 0;
   // shared pinned staging (jobs | levels | k-per-stream), guarded by ev_stage
@@ -142,7 +143,7 @@ inline uint64_t nval_per_token(const gkv_config& c) { return is_mla(c) ? c.d_k :
 constexpr int kMlaTargetCtas = 148 * 2;
 
 struct ArenaPlan {
-  size_t status, debug, partial, range, mass, levels, scores, kper, jobs, per_layer, heap_begin, total_meta;
+  size_t status, debug, partial, range, mass, levels, scores, kper, tickets, jobs, per_layer, heap_begin, total_meta;
   size_t l_table, l_warps, l_units, l_parts, l_resoff, l_rescount, l_residx, l_respool, l_boxes, layer_bytes;
 };
 
@@ -208,6 +209,7 @@ ArenaPlan plan_arena(const gkv_config& c, const Derived& d) {
   const size_t score_elems = std::max<size_t>(c.residual_fraction > 0.f ? c.max_ctx : 0, d.box_stride);
   a.scores = take(static_cast<size_t>(d.n_streams) * score_elems * sizeof(float));
   a.kper = take(static_cast<size_t>(d.n_streams) * sizeof(int32_t));
+  a.tickets = take(static_cast<size_t>(d.n_streams) * sizeof(int32_t));
   a.jobs = take(static_cast<size_t>(d.n_streams) * d.max_blocks * sizeof(EncodeJob));
   a.per_layer = off;
   size_t lo = 0;
@@ -1031,6 +1033,7 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
   c->levels_d = reinterpret_cast<int8_t*>(c->arena + a.levels);
   c->scores_d = reinterpret_cast<float*>(c->arena + a.scores);
   c->kper_d = reinterpret_cast<int32_t*>(c->arena + a.kper);
+  c->tickets_d = reinterpret_cast<int32_t*>(c->arena + a.tickets);
   c->jobs_d = reinterpret_cast<EncodeJob*>(c->arena + a.jobs);
   c->jobs_cap = static_cast<size_t>(d.n_streams) * d.max_blocks;
 
@@ -1154,12 +1157,9 @@ int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* p
   p.group = c->group;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.status = c->status_d;
-  CombineParams cp{};
-  cp.partial = c->partial_d;
-  cp.out = out;
-  cp.lse = lse;
-  cp.n_kv_heads = cfg.n_kv_heads;
-  cp.group = c->group;
+  p.tickets = c->tickets_d;
+  p.out = out;
+  p.lse = lse;
   int n_ctas;
   if (page_idx) {
     if (cfg.page_tokens <= 0) return GKV_ERR_BAD_STATE;
@@ -1172,8 +1172,7 @@ int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* p
     p.warps_per_stream = kSparseWarpsPerStream;
     p.n_warps = c->n_streams * kSparseWarpsPerStream;
     p.warps = nullptr;
-    cp.parts = nullptr;
-    cp.warps_per_stream = 1;            // the kernel leaves one merged row per stream
+    p.parts = nullptr;
     n_ctas = (p.n_warps + kDecodeWarps - 1) / kDecodeWarps;
     L.last_mode = 2;
     L.last_pages = page_idx;
@@ -1190,13 +1189,12 @@ int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* p
     p.warps = L.warps_d;
     p.units = L.units_d;
     p.n_warps = L.n_warps;
-    cp.parts = L.parts_d;
+    p.parts = L.parts_d;
     n_ctas = L.n_warps / kDecodeWarps;
     L.last_mode = 1;
     L.quest_ran = false;
   }
   CK(c, launch_decode(p, n_ctas, st));
-  CK(c, launch_combine(cp, c->n_streams, st));
   return GKV_OK;
 }
 

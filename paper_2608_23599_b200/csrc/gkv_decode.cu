@@ -1075,66 +1075,63 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
         }
         dst[e] = acc;
       }
+      // The CTA that delivers the stream's last row normalises and writes the output: rows are
+      // published with a fence before the ticket is taken, and read back through L2.  Nobody
+      // waits for anybody; the order of summation is the row order, whichever CTA does it.
+      __threadfence();
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        int begin = sid, end = sid + 1;
+        if (p.parts) {
+          begin = p.parts[sid].begin;
+          end = p.parts[sid].end;
+        }
+        const int n = end - begin;
+        bool is_last = true;
+        if (n > 1) {
+          is_last = atomicAdd(&p.tickets[sid], 1) == n - 1;
+          if (is_last) p.tickets[sid] = 0;        // ready for the next launch
+        }
+        s_group[2 * kDecodeWarps] = is_last ? begin : -1;
+        s_group[2 * kDecodeWarps + 1] = end;
+      }
+      __syncthreads();
+      const int begin = s_group[2 * kDecodeWarps], end = s_group[2 * kDecodeWarps + 1];
+      if (begin >= 0) {
+        __threadfence();
+        const int b = sid / p.n_kv_heads, kvh = sid - b * p.n_kv_heads;
+#pragma unroll 1
+        for (int e = threadIdx.x; e < p.group * kD; e += kDecodeWarps * 32) {
+          const int h = e / kD, ch = e - h * kD;
+          const float* col = p.partial + static_cast<size_t>(begin) * kPartialFloats + h * (kD + 2);
+          float M = kNegInf;
+#pragma unroll 4
+          for (int i = 0; i < end - begin; ++i) M = fmaxf(M, __ldcg(col + static_cast<size_t>(i) * kPartialFloats));
+          float L = 0.f, acc = 0.f;
+#pragma unroll 4
+          for (int i = 0; i < end - begin; ++i) {
+            const float* row = col + static_cast<size_t>(i) * kPartialFloats;
+            const float m = __ldcg(row);
+            const float wgt = (m == kNegInf) ? 0.f : exp2f(m - M);
+            L = fmaf(wgt, __ldcg(row + 1), L);
+            acc = fmaf(wgt, __ldcg(row + 2 + ch), acc);
+          }
+          const size_t hq = static_cast<size_t>(b) * p.n_kv_heads * p.group + static_cast<size_t>(kvh) * p.group + h;
+          p.out[hq * kD + ch] = (L > 0.f) ? acc / L : 0.f;
+          if (p.lse && ch == 0) p.lse[hq] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : kNegInf;
+        }
+      }
+      __syncthreads();
     }
     gb = ge;
   }
-}
-
-// Merge the partials of one (stream, query head): fixed ascending order, so results are
-// reproducible run to run.  The (m, l) pairs are staged in shared memory with one round trip,
-// then every thread (one per channel) accumulates its column with independent, unrolled loads.
-constexpr int kCombineChunk = 128;
-__global__ void __launch_bounds__(kD) combine_kernel(const __grid_constant__ CombineParams p) {
-  __shared__ float sm_m[kCombineChunk], sm_w[kCombineChunk];
-  const int stream = blockIdx.x, h = blockIdx.y, c = threadIdx.x;
-  int begin, end;
-  if (p.parts) {
-    begin = p.parts[stream].begin;
-    end = p.parts[stream].end;
-  } else {
-    begin = stream * p.warps_per_stream;
-    end = begin + p.warps_per_stream;
-  }
-  const float* base = p.partial + h * (kD + 2);
-  // pass 1: global maximum of the partial maxima
-  float mloc = kNegInf;
-  for (int i = begin + c; i < end; i += kD) mloc = fmaxf(mloc, __ldcg(base + static_cast<size_t>(i) * kPartialFloats));
-  sm_m[c] = mloc;
-  __syncthreads();
-  float M = kNegInf;
-#pragma unroll 8
-  for (int i = 0; i < kD; ++i) M = fmaxf(M, sm_m[i]);
-  // pass 2: chunks of up to 128 partials, weights in shared memory, columns in registers
-  float L = 0.f, acc = 0.f;
-  for (int c0 = begin; c0 < end; c0 += kCombineChunk) {
-    const int n = min(kCombineChunk, end - c0);
-    __syncthreads();
-    if (c < n) {
-      const float* row = base + static_cast<size_t>(c0 + c) * kPartialFloats;
-      const float m = __ldcg(row);
-      const float wgt = (m == kNegInf) ? 0.f : exp2f(m - M);
-      sm_w[c] = wgt;
-      sm_m[c] = wgt * __ldcg(row + 1);
-    }
-    __syncthreads();
-    const float* col = base + static_cast<size_t>(c0) * kPartialFloats + 2 + c;
-#pragma unroll 8
-    for (int i = 0; i < n; ++i) {
-      L += sm_m[i];
-      acc = fmaf(sm_w[i], __ldcg(col + static_cast<size_t>(i) * kPartialFloats), acc);
-    }
-  }
-  const int b = stream / p.n_kv_heads, kvh = stream - b * p.n_kv_heads;
-  const size_t hq = static_cast<size_t>(b) * p.n_kv_heads * p.group + static_cast<size_t>(kvh) * p.group + h;
-  p.out[hq * kD + c] = (L > 0.f) ? acc / L : 0.f;
-  if (p.lse && c == 0) p.lse[hq] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : kNegInf;
 }
 
 }  // namespace
 
 size_t decode_smem_bytes() {
   // per warp: pipeline stages, their mbarriers, and the bf16 query fragments (2 KiB)
-  return static_cast<size_t>(kDecodeWarps) * (kStages * kStageBytes + kStages * sizeof(uint64_t) + 2 * 2048 + 2 * sizeof(int));
+  return static_cast<size_t>(kDecodeWarps) * (kStages * kStageBytes + kStages * sizeof(uint64_t) + 2 * 2048 + 2 * sizeof(int)) + 2 * sizeof(int);
 }
 
 cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st) {
@@ -1151,11 +1148,6 @@ cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st) {
   if (n_ctas <= 0) return cudaSuccess;
   if (p.page_idx) decode_kernel<true><<<n_ctas, kDecodeWarps * 32, decode_smem_bytes(), st>>>(p);
   else decode_kernel<false><<<n_ctas, kDecodeWarps * 32, decode_smem_bytes(), st>>>(p);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_combine(const CombineParams& p, int n_streams, cudaStream_t st) {
-  combine_kernel<<<dim3(n_streams, p.group), kD, 0, st>>>(p);
   return cudaGetLastError();
 }
 

@@ -63,14 +63,11 @@ struct DecodeParams {
   const int32_t* page_idx;      // [n_streams][n_sel] or nullptr
   int32_t n_sel, page_tokens, warps_per_stream;
   uint32_t* status;             // device status word (bit flags)
-};
-
-struct CombineParams {
-  const float* partial;
-  const StreamParts* parts;     // [n_streams]; nullptr in sparse mode (then fixed warps_per_stream)
+  // final merge: the CTA that completes a stream's last partial row normalises and writes it
+  const StreamParts* parts;     // [n_streams]; nullptr in sparse mode (one row per stream, row = stream)
+  int32_t* tickets;             // [n_streams] arrival counters, zero between launches
   float* out;                   // [batch][n_q_heads][128]
   float* lse;                   // nullable
-  int32_t n_kv_heads, group, warps_per_stream;
 };
 
 // One block to encode: read 64 tokens from `src`, write level `dst_level` at dst.
@@ -115,7 +112,6 @@ constexpr uint32_t kStatusRange = 1u;      // a scale or zero saturated
 constexpr uint32_t kStatusInternal = 2u;   // an index check failed inside a kernel
 
 cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st);
-cudaError_t launch_combine(const CombineParams& p, int n_streams, cudaStream_t st);
 cudaError_t launch_encode(const EncodeParams& p, cudaStream_t st);
 cudaError_t launch_stats(const StatsParams& p, cudaStream_t st);
 cudaError_t launch_append_rows(uint8_t* arena, const TableEntry* table, int table_stride, int tail_index,
