@@ -54,6 +54,17 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
+// 16-byte asynchronous copy; src_bytes = 0 writes zeros instead
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+// the mbarrier gets one more pending arrival now, delivered when this thread's copies above are done
+__device__ __forceinline__ void cp_async_mbar_arrive(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
   asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(src), "r"(bytes) : "memory");
 }
@@ -454,60 +465,69 @@ __device__ __forceinline__ void issue_step(const WarpCtx& w, const Cursor& c, in
   const DecodeParams& p = *w.p;
   const uint32_t sdst = w.stage0 + sidx * kStageBytes, bar = w.bar0 + sidx * 8;
   const int lane = w.lane;
-  if (c.level == 16 || c.level == 1 || c.level == 17) {
-    // up to 16 rows of 256 B, staged at a 272-byte pitch; one bulk copy per row
+  if (c.level == 16 || c.level == 17) {
+    // 16 rows of 256 B at a regular stride, staged at a 272-byte pitch: 256 16-byte pieces, eight per
+    // lane (piece q = lane + 32 i is row q / 16, column q % 16).  Rows past the end are written as
+    // zeros so that 0 * garbage never produces a NaN.  The warp's copies complete the barrier
+    // phase through one tracked arrival per lane plus the plain arrival that matches the
+    // barrier's count of one.
     const bool is_v = (c.sub & 1) != 0;
-    const uint8_t* src = nullptr;
-    int nrows;
+    const int row0 = lane >> 4, col = lane & 15;
+    const uint8_t* g = p.arena + static_cast<size_t>(c.off256) * 256 + col * 16;
+    const uint32_t d = sdst + row0 * kRowPitch + col * 16;
     if (c.level == 16) {
       const int tile = nth_set_bit(c.tmask, c.sub >> 1);
-      nrows = min(16, c.ntok - tile * 16);
-      src = p.arena + static_cast<size_t>(c.off256) * 256 + (is_v ? kBlock * kRowBytes : 0) +
-            static_cast<size_t>(tile * 16 + lane) * kRowBytes;
-    } else if (c.level == 17) {
-      nrows = c.ntok;
-      src = p.arena + static_cast<size_t>(c.off256) * 256 + (is_v ? kRowBytes : 0) +
-            static_cast<size_t>(lane) * 2 * kRowBytes;
+      const int nrows = c.ntok - tile * 16;
+      g += (is_v ? kBlock * kRowBytes : 0) + static_cast<size_t>(tile * 16 + row0) * kRowBytes;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) cp_async16(d + i * 2 * kRowPitch, g + i * 2 * kRowBytes, (row0 + 2 * i < nrows) ? 16u : 0u);
     } else {
-      nrows = c.ntok;
-      if (lane < nrows) {
-        int blk;
-        if constexpr (SPARSE) blk = p.page_idx[static_cast<size_t>(w.stream) * p.n_sel + c.item] / (kBlock / p.page_tokens);
-        else blk = c.first + lane;
-        src = p.arena + static_cast<size_t>(w.table[blk].off256) * 256 + (is_v ? kRowBytes : 0);
-      }
+      g += (is_v ? kRowBytes : 0) + static_cast<size_t>(row0) * 2 * kRowBytes;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) cp_async16(d + i * 2 * kRowPitch, g + i * 4 * kRowBytes, (row0 + 2 * i < c.ntok) ? 16u : 0u);
+    }
+    cp_async_mbar_arrive(bar);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+    return;
+  }
+  if (c.level == 1) {
+    // up to 16 centroid rows gathered from their blocks; one bulk copy per row
+    const bool is_v = (c.sub & 1) != 0;
+    const uint8_t* src = nullptr;
+    const int nrows = c.ntok;
+    if (lane < nrows) {
+      int blk;
+      if constexpr (SPARSE) blk = p.page_idx[static_cast<size_t>(w.stream) * p.n_sel + c.item] / (kBlock / p.page_tokens);
+      else blk = c.first + lane;
+      src = p.arena + static_cast<size_t>(w.table[blk].off256) * 256 + (is_v ? kRowBytes : 0);
     }
     if (lane == 0) mbar_expect_tx(bar, static_cast<uint32_t>(nrows) * kRowBytes);
     __syncwarp();
     if (lane < nrows) {
       bulk_g2s(sdst + lane * kRowPitch, src, kRowBytes, bar);
     } else if (lane < 16) {
-      // rows past the end are zero so that 0 * garbage never produces a NaN
       uint4* z = reinterpret_cast<uint4*>(const_cast<uint8_t*>(w.stage_ptr0) + sidx * kStageBytes + lane * kRowPitch);
 #pragma unroll
       for (int i = 0; i < kRowBytes / 16; ++i) z[i] = make_uint4(0, 0, 0, 0);
     }
     return;
   }
-  if (lane != 0) return;
   const int bits = c.level;
   const int cb = code_bytes_per_tile(bits);
   const uint8_t* slot = p.arena + static_cast<size_t>(c.off256) * 256;
   if (!SPARSE || c.tmask == 15) {
-    // full block: every step is one contiguous span of the slot
-    const uint8_t* src;
-    uint32_t bytes;
-    if (bits == 8) {
-      bytes = 512 + 2 * cb;
-      src = slot + (c.sub >> 1) * half_bytes(8) + (c.sub & 1) * bytes;
-    } else {
-      bytes = half_bytes(bits);
-      src = slot + c.sub * bytes;
+    // full block: every step is one contiguous span of the slot, all steps of a level alike
+    // (8-bit: key part and value part of each half, 4608 B; 4- and 2-bit: one half)
+    const uint32_t bytes = (bits == 8) ? 512 + 2 * 2048 : (bits == 4 ? half_bytes(4) : half_bytes(2));
+    const uint8_t* src = slot + c.sub * bytes;
+    if (lane == 0) {
+      mbar_expect_tx(bar, bytes);
+      bulk_g2s(sdst, src, bytes, bar);
     }
-    mbar_expect_tx(bar, bytes);
-    bulk_g2s(sdst, src, bytes, bar);
     return;
   }
+  if (lane != 0) return;
   // sparse visit: copy only the pieces of the selected tiles (same stage offsets as a full copy)
   if (bits == 8) {
     const int half = half_of_step(c, c.sub >> 1);
@@ -985,7 +1005,6 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
 #endif
       phase ^= 1u << sidx;
 #endif
-      __syncwarp();
 #ifndef GKV_EXP_SKIP_COMPUTE
       compute_step<SPARSE>(w, cur, sidx, ones, st, pf);
 #endif
