@@ -140,7 +140,7 @@ namespace {
 inline bool is_mla(const gkv_config& c) { return c.v_aliases_k != 0; }
 inline int geo_slot_bytes(const gkv_config& c, int level) { return is_mla(c) ? mla_slot_bytes(level) : slot_bytes(level); }
 inline uint64_t nval_per_token(const gkv_config& c) { return is_mla(c) ? c.d_k : c.d_k + c.d_v; }
-constexpr int kMlaTargetCtas = 148 * 2;
+constexpr int kMlaTargetCtas = 148;          // one CTA per SM (213 KB of shared memory, tensor memory)
 
 struct ArenaPlan {
   size_t status, debug, partial, range, mass, levels, scores, kper, tickets, jobs, per_layer, heap_begin, total_meta;
@@ -727,15 +727,17 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
 // One stream per sequence; staircase or external plans only.  The block table, slot heap and
 // staging are shared with the GQA path; the kernels are those of gkv_mla.cu.
 size_t mla_item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) {
+  // a tile costs about the same whatever its level (the dequantised tile is what the tensor
+  // cores and the shared-memory pipes see); 64 centroid blocks share one tile
   if (item < L.n_closed) {
     switch (L.level[static_cast<size_t>(stream) * c->max_blocks + item]) {
-      case 16: return 1400;       // measured shares of a block's time on B200 (exact rows are byte-bound)
+      case 16: return 1200;
       case 8: return 1000;
-      case 4: return 800;
-      default: return 60;
+      case 4: return 950;
+      default: return 20;
     }
   }
-  return 700;                     // tail
+  return 600;                     // tail
 }
 
 void mla_build_descs(gkv_cache* c, LayerState& L) {

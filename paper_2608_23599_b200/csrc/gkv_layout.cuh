@@ -125,29 +125,35 @@ GKV_HD int vp_zero_index(int t16, int grp) {
 }  // namespace gkv
 
 // ---- latent-attention (MLA) streams: one 576-wide row per token, values = channels [0, 512) ----
-// The row is quantised once with the key rule (32 tokens x 1 channel per group).  Codes are stored
-// in the K-role fragment order above with 36 MMA indices (16 channels each); the value role reads
-// the same codes and transposes the 8x8 fragments in registers.  Words are stored word-major:
-// word w of a lane lives at byte (w * 32 + lane) * 4 of the tile's code region.
+// The row is quantised once with the key rule (32 tokens x 1 channel per group).  A quantised slot
+// is two halves of 32 tokens: [params 2304 B][codes 32 rows x 72 chunks]; a chunk is 8 neighbouring
+// channels of one token (8 bytes at 8 bits, one 32-bit word at 4 bits).  The params of chunk j are
+// 32 bytes: eight fp16 scales, then eight fp16 zero points.  Inside a chunk the codes are placed so
+// that one "mask, or in an exponent" (4 bits) or one byte permute (8 bits) yields the fp16 pair
+// of two neighbouring channels: 4-bit channel c sits at bit 4 (c >> 1) + 16 (c & 1); 8-bit channel c
+// sits in word c >> 2 at byte ((c & 3) >> 1) + 2 (c & 1).
 namespace gkv {
 constexpr int kMlaDk = 576, kMlaDv = 512, kMlaHeads = 16, kMlaKSteps = kMlaDk / 16;   // 36
+constexpr int kMlaChunks = kMlaDk / 8;                                                // 72
 constexpr int kMlaRowBytes = kMlaDk * 2;                                              // 1152
-GKV_HD int mla_code_bytes_per_tile(int bits) { return kMlaKSteps * 8 * bits * 32 / 8; }   // 1152 * bits
-GKV_HD int mla_kp_bytes() { return kMlaKSteps * 4 * 16; }                                 // 2304 per half
-GKV_HD int mla_half_bytes(int bits) { return mla_kp_bytes() + 2 * mla_code_bytes_per_tile(bits); }
+GKV_HD int mla_kp_bytes() { return kMlaChunks * 32; }                                     // 2304 per half
+GKV_HD int mla_code_row_bytes(int bits) { return kMlaChunks * bits; }                     // 576 / 288
+GKV_HD int mla_half_bytes(int bits) { return mla_kp_bytes() + 32 * mla_code_row_bytes(bits); }
 GKV_HD int mla_slot_bytes(int level) {
   return level == 16 ? kBlock * kMlaRowBytes : (level == 1 ? 1280 : 2 * mla_half_bytes(level));
 }
-GKV_HD void mla_code_pos(int bits, int lane, int s, int a, int hlf, int* byte_off, int* bit) {
-  int w, b;
+// fp16 index of channel ch's scale inside a half's params; its zero point sits 8 entries later
+GKV_HD int mla_kp_index(int ch) { return (ch >> 3) * 16 + (ch & 7); }
+// position of the code of (token t32 of the half, channel ch): byte offset of its 32-bit word from
+// the start of the half's code rows, and the bit inside that word
+GKV_HD void mla_code_pos(int bits, int t32, int ch, int* byte_off, int* bit) {
+  const int j = ch >> 3, c = ch & 7;
   if (bits == 8) {
-    w = 2 * s + (a >> 1);
-    b = 8 * (a & 1);
+    *byte_off = t32 * mla_code_row_bytes(8) + j * 8 + (c >> 2) * 4;
+    *bit = 8 * (((c & 3) >> 1) + 2 * (c & 1));
   } else {
-    w = s;
-    b = 4 * a;
+    *byte_off = t32 * mla_code_row_bytes(4) + j * 4;
+    *bit = 4 * (c >> 1) + 16 * (c & 1);
   }
-  *byte_off = (w * 32 + lane) * 4;
-  *bit = b + 16 * hlf;
 }
 }  // namespace gkv
