@@ -727,17 +727,19 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
 // One stream per sequence; staircase or external plans only.  The block table, slot heap and
 // staging are shared with the GQA path; the kernels are those of gkv_mla.cu.
 size_t mla_item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) {
-  // a tile costs about the same whatever its level (the dequantised tile is what the tensor
-  // cores and the shared-memory pipes see); 64 centroid blocks share one tile
+  // cycles of a CTA per block, measured inside the config-4 mixture on B200 (in units where a
+  // 4-bit block is 1000): the dequantised tile is what the tensor cores and the shared-memory
+  // pipes see, so quantised levels cost about the same; an exact block streams 3.2x the bytes
+  // through the two raw stages; 64 centroid blocks share one tile but are gathered row by row
   if (item < L.n_closed) {
     switch (L.level[static_cast<size_t>(stream) * c->max_blocks + item]) {
-      case 16: return 1200;
-      case 8: return 1000;
-      case 4: return 950;
-      default: return 20;
+      case 16: return 1700;
+      case 8: return 1100;
+      case 4: return 1000;
+      default: return 36;
     }
   }
-  return 600;                     // tail
+  return 900;                     // tail
 }
 
 void mla_build_descs(gkv_cache* c, LayerState& L) {

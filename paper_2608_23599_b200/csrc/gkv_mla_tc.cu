@@ -47,8 +47,8 @@ constexpr int kOffRaw = kOffP + 2 * kTcPBytes;         // 169984
 constexpr int kOffMisc = kOffRaw + 2 * kTcRawBytes;    // 211456
 constexpr int kTcSmem = kOffMisc + 2048 + 1024;        // + misc + alignment slack
 // misc: 16 mbarriers (128 B) | tmem base (4 B) @128 | abort flag @132 | bias[2][64] floats @256 |
-//       head maxima [2][4 warps][16] floats @768 | row sums [4][16] @1280
-constexpr int kMiscTmem = 128, kMiscAbort = 132, kMiscBias = 256, kMiscMax = 768, kMiscSum = 1280;
+//       head maxima [2][4 warps][16] floats @768, rescale flags [2][4] ints @1280 | row sums [4][16] @1344
+constexpr int kMiscTmem = 128, kMiscAbort = 132, kMiscBias = 256, kMiscMax = 768, kMiscSum = 1344;
 enum { kBarRawFull = 0, kBarRawEmpty = 2, kBarKtFull = 4, kBarSFull = 6, kBarPFull = 8, kBarPvDone = 10, kBarMax = 12, kBarSum = 14 };
 constexpr int kTcWaitSpins = 1 << 20;
 constexpr float kNegInfT = -INFINITY;
@@ -191,19 +191,21 @@ __device__ __forceinline__ void t_st16(uint32_t taddr, const float (&v)[16]) {
   asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle (Blackwell version bit set).  Strides in bytes.
-__device__ __forceinline__ uint64_t t_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+// Shared-memory matrix descriptor (Blackwell version bit set), 128-byte swizzle unless told otherwise.
+// Strides in bytes.
+__device__ __forceinline__ uint64_t t_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint64_t layout = 2) {
   uint64_t d = 0;
   d |= static_cast<uint64_t>((saddr >> 4) & 0x3fffu);
   d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3fffu) << 16;
   d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3fffu) << 32;
   d |= 1ull << 46;                 // descriptor version
-  d |= 2ull << 61;                 // SWIZZLE_128B
+  d |= layout << 61;               // 2 = SWIZZLE_128B, 6 = SWIZZLE_32B
   return d;
 }
 // Instruction descriptor for kind::f16 with fp16 operands and an fp32 accumulator.
-__host__ __device__ constexpr uint32_t t_idesc(int m, int n, bool a_mn_major) {
-  return (1u << 4) | (static_cast<uint32_t>(a_mn_major) << 15) | (static_cast<uint32_t>(n >> 3) << 17) |
+__host__ __device__ constexpr uint32_t t_idesc(int m, int n, bool a_mn_major, bool b_mn_major = false) {
+  return (1u << 4) | (static_cast<uint32_t>(a_mn_major) << 15) | (static_cast<uint32_t>(b_mn_major) << 16) |
+         (static_cast<uint32_t>(n >> 3) << 17) |
          (static_cast<uint32_t>(m >> 4) << 24);
 }
 
@@ -220,7 +222,7 @@ struct TcTile {
   uint32_t off256;
 };
 
-__device__ __forceinline__ bool tc_next(const MlaDecodeParams& p, const TableEntry* table, int item_end, int it, TcTile& t) {
+__device__ __noinline__ bool tc_next(const MlaDecodeParams& p, const TableEntry* table, int item_end, int it, TcTile& t) {
   if (it >= item_end) return false;
   const TableEntry e = table[it];
   t.item = it;
@@ -298,41 +300,38 @@ __device__ __forceinline__ uint32_t tc_tile_addr(uint32_t tile, int row, int j) 
 
 // dequantise one half (32 tokens) of a quantised block: thread = (chunk j, 8 tokens)
 template <int BITS>
-__device__ __forceinline__ void tc_dequant_half(uint32_t raw, uint32_t tile, int half, int tid) {
-  const int j = tid % kMlaChunks, tg = tid / kMlaChunks;
+__device__ __forceinline__ void tc_dequant_half(uint32_t raw, uint32_t tile, int half, int j, int tg) {
   const uint4 sv = t_lds128(raw + j * 32), zv = t_lds128(raw + j * 32 + 16);
   const __half2 s0 = t_h2(sv.x), s1 = t_h2(sv.y), s2 = t_h2(sv.z), s3 = t_h2(sv.w);
   const __half2 z0 = t_h2(zv.x), z1 = t_h2(zv.y), z2 = t_h2(zv.z), z3 = t_h2(zv.w);
-  const uint32_t codes = raw + mla_kp_bytes() + j * BITS;
+  const uint32_t codes = raw + mla_kp_bytes() + j * BITS + tg * 8 * (kMlaChunks * BITS);
+  // rows 32 half + 8 tg + i: row & 7 = i, so the swizzled 16-byte slot is (j & 7) ^ i
+  const uint32_t out = tile + (j >> 3) * kTcPanelBytes + (32 * half + 8 * tg) * 128;
+  const uint32_t jx = (j & 7) << 4;
+  const __half2 b0 = __float2half2_rn(1024.f), b1 = __float2half2_rn(BITS == 4 ? 64.f : 1024.f);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    const int tok = tg * 8 + i;
     uint32_t x0, x1, x2, x3;
-    __half2 b0, b1;
     if constexpr (BITS == 4) {
-      const uint32_t w = t_lds32(codes + tok * (kMlaChunks * 4));
+      const uint32_t w = t_lds32(codes + i * (kMlaChunks * 4));
       const uint32_t v = w >> 8;
       x0 = t_lop_ao(w, 0x000F000Fu, 0x64006400u);      // 1024 + code (channels 0, 1)
       x1 = t_lop_ao(w, 0x00F000F0u, 0x54005400u);      // 64 + code   (channels 2, 3)
       x2 = t_lop_ao(v, 0x000F000Fu, 0x64006400u);
       x3 = t_lop_ao(v, 0x00F000F0u, 0x54005400u);
-      b0 = __float2half2_rn(1024.f);
-      b1 = __float2half2_rn(64.f);
     } else {
-      const uint2 w = t_lds64(codes + tok * (kMlaChunks * 8));
+      const uint2 w = t_lds64(codes + i * (kMlaChunks * 8));
       x0 = t_prmt(w.x, 0x64006400u, 0x5250u);
       x1 = t_prmt(w.x, 0x64006400u, 0x5351u);
       x2 = t_prmt(w.y, 0x64006400u, 0x5250u);
       x3 = t_prmt(w.y, 0x64006400u, 0x5351u);
-      b0 = __float2half2_rn(1024.f);
-      b1 = b0;
     }
     // code = x - bias exactly; k~ = code * s + z with one rounding
     const uint32_t y0 = t_u(__hfma2(__hsub2(t_h2(x0), b0), s0, z0));
     const uint32_t y1 = t_u(__hfma2(__hsub2(t_h2(x1), b1), s1, z1));
     const uint32_t y2 = t_u(__hfma2(__hsub2(t_h2(x2), b0), s2, z2));
     const uint32_t y3 = t_u(__hfma2(__hsub2(t_h2(x3), b1), s3, z3));
-    t_sts128(tc_tile_addr(tile, 32 * half + tok, j), y0, y1, y2, y3);
+    t_sts128(out + i * 128 + (jx ^ (i << 4)), y0, y1, y2, y3);
   }
 }
 
@@ -427,78 +426,88 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
   } else if (warp == kTcMmaWarp) {
     // ---------------- tensor-core issue (whole warp, one elected lane per instruction) ----------------
     {
-      constexpr uint32_t kIdQK = t_idesc(64, 16, false), kIdPV = t_idesc(128, 16, true);
+      constexpr uint32_t kIdQK = t_idesc(64, 16, false), kIdPV = t_idesc(128, 16, true, true);
       // descriptors differ only in the start-address field (16-byte units in the low word)
       const uint64_t dq = t_desc(base + kOffQ, 16, 1024);
       auto issue_qk = [&](int tg) {
         const int b = tg & 1;
         const uint64_t da = t_desc(base + kOffTile + b * kTcTileBytes, 16, 1024);
         const uint32_t d = tmem + kTmemS + 16 * b;
+#ifdef GKV_TC_ROLL_MMA
+#pragma unroll 1
+#else
 #pragma unroll
+#endif
         for (int pn = 0; pn < 9; ++pn)
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
             t_mma_f16(d, da + ((pn * kTcPanelBytes + kk * 32) >> 4), dq + ((pn * 2048 + kk * 32) >> 4), kIdQK, (pn | kk) != 0);
         t_commit(bar(kBarSFull, b));
       };
-#ifdef GKV_TC_PROFILE
-      long long m_kt = 0, m_qk = 0, m_p = 0, m_pv = 0, m_t0 = clock64(), c_x = clock64();
+      auto issue_pv = [&](int tg) {
+        const int b = tg & 1;
+        const uint64_t da = t_desc(base + kOffTile + b * kTcTileBytes, kTcPanelBytes, 1024);
+        // P: [64 tokens][16 heads] fp16, heads contiguous (MN-major), 32-byte swizzle, 8-token groups of 256 B
+        const uint64_t dp = t_desc(base + kOffP + b * kTcPBytes, 256, 256, 6);
+        const uint32_t first = tg != 0;
+#ifdef GKV_TC_ROLL_MMA
+#pragma unroll 1
+#else
+#pragma unroll
 #endif
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            t_mma_f16(tmem + kTmemO + 16 * i, da + ((2 * i * kTcPanelBytes + kk * 2048) >> 4), dp + ((kk * 512) >> 4), kIdPV,
+                      kk != 0 ? 1u : first);
+        t_commit(bar(kBarPvDone, b));
+      };
+      // Event-driven order: the value MMAs of tile pv go out as soon as its P is there, the key MMAs
+      // of tile qk as soon as its tile is there (qk runs at most two tiles ahead of pv: S and the
+      // tile buffers are double).  n_tiles is not known in advance: the iterator tells.
       TcTile t;
-      int it = cd.item_begin, tg = 0;
-      bool ok = true, have = tc_next(p, table, cd.item_end, it, t);
-      if (have) {
-        ok = t_wait_warp(bar(kBarKtFull, 0), 0, abort_flag);
-        t_fence_after();
-        if (ok) issue_qk(0);
-      }
-      while (ok && have) {
-        it = t.item + t.adv;
-        TcTile nt;
-        const bool more = tc_next(p, table, cd.item_end, it, nt);
-        if (more) {                                         // logits of the next tile while this one is in softmax
-#ifdef GKV_TC_PROFILE
-          c_x = clock64();
-#endif
-          ok = t_wait_warp(bar(kBarKtFull, (tg + 1) & 1), ((tg + 1) >> 1) & 1, abort_flag);
-          TCP(m_kt);
-          t_fence_after();
-          if (ok) issue_qk(tg + 1);
-          TCP(m_qk);
+      int it = cd.item_begin;
+      bool more_tiles = tc_next(p, table, cd.item_end, it, t);
+      int qk = 0, pv = 0, n_known = more_tiles ? 1 : 0;      // tiles [0, n_known) exist so far
+      bool ok = true;
+      int spins = 0;
+      while (ok && (pv < n_known || more_tiles)) {
+        bool progress = false;
+        // key MMAs of tile qk: S[qk & 1] is free once the softmax of tile qk - 2 has published its P
+        if (qk < n_known && qk < pv + 2) {
+          const bool ready = __all_sync(kFullT, t_try_wait(bar(kBarKtFull, qk & 1), (qk >> 1) & 1));
+          if (ready) {
+            t_fence_after();
+            issue_qk(qk);
+            ++qk;
+            // look one tile further
+            it = t.item + t.adv;
+            more_tiles = tc_next(p, table, cd.item_end, it, t);
+            if (more_tiles) ++n_known;
+            progress = true;
+          }
         }
-#ifdef GKV_TC_PROFILE
-        c_x = clock64();
-#endif
-        if (ok) ok = t_wait_warp(bar(kBarPFull, tg & 1), (tg >> 1) & 1, abort_flag);
-        TCP(m_p);
-        if (ok) {
-          t_fence_after();
-          const int b = tg & 1;
-          const uint64_t da = t_desc(base + kOffTile + b * kTcTileBytes, kTcPanelBytes, 1024);
-          const uint64_t dp = t_desc(base + kOffP + b * kTcPBytes, 16, 1024);
-          const uint32_t first = tg != 0;
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              t_mma_f16(tmem + kTmemO + 16 * i, da + ((2 * i * kTcPanelBytes + kk * 2048) >> 4), dp + ((kk * 32) >> 4), kIdPV,
-                        kk != 0 ? 1u : first);
-          t_commit(bar(kBarPvDone, b));
-          TCP(m_pv);
+        if (pv < qk) {
+          const bool ready = __all_sync(kFullT, t_try_wait(bar(kBarPFull, pv & 1), (pv >> 1) & 1));
+          if (ready) {
+            t_fence_after();
+            issue_pv(pv);
+            ++pv;
+            progress = true;
+          }
         }
-        t = nt;
-        have = more;
-        ++tg;
+        if (progress) spins = 0;
+        else if (++spins > kTcWaitSpins || *abort_flag) {
+          *abort_flag = 1;
+          ok = false;
+        }
+        ok = __all_sync(kFullT, ok);
       }
-#ifdef GKV_TC_PROFILE
-      if (blockIdx.x % 37 == 0 && lane == 0)
-        printf("TCM cta %d tiles %d total %lld wait_kt %lld issue_qk %lld wait_p %lld issue_pv %lld\n", blockIdx.x, tg, clock64() - m_t0,
-               m_kt, m_qk, m_p, m_pv);
-#endif
     }
   } else if (warp >= kTcFirstDequantWarp) {
     // ---------------- dequantisation ----------------
     const int dt = tid - kTcFirstDequantWarp * 32;          // 0 .. 287
+    const int dj = dt % kMlaChunks, dg = dt / kMlaChunks;   // chunk of 8 channels, token group
     TcTile t;
     int it = cd.item_begin, tg = 0, sg = 0;
     bool ok = true;
@@ -527,8 +536,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
           if (!ok) break;
           const uint32_t raw = base + kOffRaw + rb * kTcRawBytes;
           if (t.kind == 0) {
-            if (t.level == 8) tc_dequant_half<8>(raw, tile, s, dt);
-            else tc_dequant_half<4>(raw, tile, s, dt);
+            if (t.level == 8) tc_dequant_half<8>(raw, tile, s, dj, dg);
+            else tc_dequant_half<4>(raw, tile, s, dj, dg);
           } else {
             tc_rows_quarter(raw, tile, s, min(16, t.nrows - 16 * s), dt);
           }
@@ -561,7 +570,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       l_part[h] = 0.f;
     }
     TcTile t;
-    int it = cd.item_begin, ts = 0;
+    int it = cd.item_begin, ts = 0, xph = 0;                // xph: exchanges done so far (phase of the exchange barrier)
     bool ok = true;
     const uint32_t tlane = tmem + (static_cast<uint32_t>(32 * warp) << 16);
 #ifdef GKV_TC_PROFILE
@@ -579,43 +588,53 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       t_ld16(tlane + kTmemS + 16 * b, s);
       const int row = 16 * warp + (lane & 15);
       const float bs = (lane < 16) ? bias_sm[b * 64 + row] : kNegInfT;
-      float mx[16];
+      // Common case: no logit of the tile exceeds its head's running max by more than the slack;
+      // then the (stale) max stays and nothing is reduced.  The four warps agree through one flag
+      // exchange; only when a flag is up are the head maxima reduced and O rescaled.
+      bool mine = false;
 #pragma unroll
       for (int h = 0; h < 16; ++h) {
         s[h] = (bs == kNegInfT) ? kNegInfT : fmaf(s[h], p.scale_log2, bs);
-        mx[h] = s[h];
+        mine |= s[h] > m_run[h] + kRescaleSlack;            // also true for the first finite logit (max = -inf)
       }
-#pragma unroll
-      for (int d = 8; d >= 1; d >>= 1)
-#pragma unroll
-        for (int h = 0; h < 16; ++h) mx[h] = fmaxf(mx[h], __shfl_xor_sync(kFullT, mx[h], d));
-      float* mrow = max_sm + (b * 4 + warp) * 16;
-      if (lane == 0) {
-#pragma unroll
-        for (int h = 0; h < 16; ++h) mrow[h] = mx[h];
-      }
-      __syncwarp();
-      if (lane == 0) t_bar_arrive(bar(kBarMax, b));
       TCP(s_c);
-      ok = t_wait_warp(bar(kBarMax, b), (ts >> 1) & 1, abort_flag) && ok;
+      uint32_t need_u;
+      asm volatile(
+          "{\n"
+          ".reg .pred pi, po;\n"
+          "setp.ne.u32 pi, %1, 0;\n"
+          "bar.red.or.pred po, 1, 128, pi;\n"
+          "selp.u32 %0, 1, 0, po;\n"
+          "}\n"
+          : "=r"(need_u)
+          : "r"(static_cast<uint32_t>(mine))
+          : "memory");
+      const bool need = need_u != 0;
       TCP(s_x);
-      bool need = false;
-      float m_new[16];
-#pragma unroll
-      for (int h = 0; h < 16; ++h) {
-        const float* mm = max_sm + b * 64 + h;
-        const float bm = fmaxf(fmaxf(mm[0], mm[16]), fmaxf(mm[32], mm[48]));
-        m_new[h] = fmaxf(m_run[h], bm);
-        need |= bm > m_run[h] + kRescaleSlack || (m_run[h] == kNegInfT && bm != kNegInfT);
-      }
       if (need) {                                           // uniform over the 128 softmax threads
+        float mx[16];
+#pragma unroll
+        for (int h = 0; h < 16; ++h) mx[h] = s[h];
+#pragma unroll
+        for (int d = 8; d >= 1; d >>= 1)
+#pragma unroll
+          for (int h = 0; h < 16; ++h) mx[h] = fmaxf(mx[h], __shfl_xor_sync(kFullT, mx[h], d));
+        float* mbuf = max_sm + (xph & 1) * 64;
+        if (lane == 0) {
+#pragma unroll
+          for (int h = 0; h < 16; ++h) mbuf[warp * 16 + h] = mx[h];
+        }
+        asm volatile("bar.sync 1, 128;\n" ::: "memory");
         float alpha[16];
 #pragma unroll
         for (int h = 0; h < 16; ++h) {
-          alpha[h] = (m_run[h] == kNegInfT) ? 0.f : t_ex2(m_run[h] - m_new[h]);
-          m_run[h] = m_new[h];
+          const float bm = fmaxf(fmaxf(mbuf[h], mbuf[16 + h]), fmaxf(mbuf[32 + h], mbuf[48 + h]));
+          const float mn = fmaxf(m_run[h], bm);
+          alpha[h] = (m_run[h] == kNegInfT) ? 0.f : t_ex2(m_run[h] - mn);
+          m_run[h] = mn;
           l_part[h] *= alpha[h];
         }
+        ++xph;
         if (ts > 0) {                                       // O holds the tiles before ts: rescale it
           ok = t_wait_warp(bar(kBarPvDone, (ts - 1) & 1), ((ts - 1) >> 1) & 1, abort_flag) && ok;
           t_fence_after();
@@ -631,15 +650,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       }
       // probabilities relative to the (possibly stale) running max; the rounded value is what is summed
       if (lane < 16) {
-        const uint32_t prow = base + kOffP + b * kTcPBytes + (row & 7) * 2;
+        uint32_t pk[8];
 #pragma unroll
-        for (int h = 0; h < 16; ++h) {
-          const float pr = (s[h] == kNegInfT) ? 0.f : t_ex2(s[h] - m_run[h]);
-          const __half ph = __float2half_rn(pr);
-          l_part[h] += __half2float(ph);
-          const uint32_t a = prow + h * 128 + ((((row >> 3) ^ (h & 7))) << 4);
-          asm volatile("st.shared.u16 [%0], %1;\n" ::"r"(a), "h"(__half_as_ushort(ph)) : "memory");
+        for (int h = 0; h < 16; h += 2) {
+          const float p0 = (s[h] == kNegInfT) ? 0.f : t_ex2(s[h] - m_run[h]);
+          const float p1 = (s[h + 1] == kNegInfT) ? 0.f : t_ex2(s[h + 1] - m_run[h + 1]);
+          const __half2 ph = __floats2half2_rn(p0, p1);
+          l_part[h] += __low2float(ph);
+          l_part[h + 1] += __high2float(ph);
+          pk[h >> 1] = t_u(ph);
         }
+        // row of 16 heads (32 B) of token `row`; 32-byte swizzle: the 16-byte halves swap on bit 7
+        const uint32_t prow = base + kOffP + b * kTcPBytes + row * 32;
+        const uint32_t sw = ((row >> 2) & 1) << 4;
+        t_sts128(prow + sw, pk[0], pk[1], pk[2], pk[3]);
+        t_sts128(prow + (sw ^ 16), pk[4], pk[5], pk[6], pk[7]);
       }
       t_fence_async();
       t_fence_before();
@@ -666,9 +691,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
 #pragma unroll
       for (int h = 0; h < 16; ++h) sum_sm[warp * 16 + h] = l_part[h];
     }
-    __syncwarp();
-    if (lane == 0) t_bar_arrive(bar(kBarSum, 0));
-    ok = t_wait_warp(bar(kBarSum, 0), 0, abort_flag) && ok;
+    asm volatile("bar.sync 1, 128;\n" ::: "memory");
     const bool good = __all_sync(kFullT, ok && ts > 0 && !*abort_flag);
     if (warp == 0 && lane == 0) {
 #pragma unroll
@@ -701,28 +724,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
 // (stream, head), one thread per value channel.
 __global__ void __launch_bounds__(kMlaDv) mla_combine_kernel(const float* partial, const StreamParts* parts, float* out,
                                                              float* lse) {
-  __shared__ float sm_w[128], sm_l[128];
+  __shared__ float sm_m[kMlaDv], sm_w[kMlaDv];
   const int stream = blockIdx.x, h = blockIdx.y, c = threadIdx.x;
   const int begin = parts[stream].begin, end = parts[stream].end;
   const float* base = partial + h * (kMlaDv + 2);
+  // pass 1: the maximum of the rows' maxima (one row per thread, then a shared-memory sweep)
   float M = kNegInfT;
-  for (int i = begin; i < end; ++i) M = fmaxf(M, __ldcg(base + static_cast<size_t>(i) * kMlaPartialFloats));
+  for (int c0 = begin; c0 < end; c0 += kMlaDv) {
+    const int n = min(kMlaDv, end - c0);
+    __syncthreads();
+    sm_m[c] = c < n ? __ldcg(base + static_cast<size_t>(c0 + c) * kMlaPartialFloats) : kNegInfT;
+    __syncthreads();
+#pragma unroll 8
+    for (int i = 0; i < n; ++i) M = fmaxf(M, sm_m[i]);
+  }
+  // pass 2: weights per row in shared memory, then every thread sums its channel over the rows
   float L = 0.f, acc = 0.f;
-  for (int c0 = begin; c0 < end; c0 += 128) {
-    const int n = min(128, end - c0);
+  for (int c0 = begin; c0 < end; c0 += kMlaDv) {
+    const int n = min(kMlaDv, end - c0);
     __syncthreads();
     if (c < n) {
       const float* row = base + static_cast<size_t>(c0 + c) * kMlaPartialFloats;
       const float m = __ldcg(row);
       const float w = (m == kNegInfT) ? 0.f : exp2f(m - M);
       sm_w[c] = w;
-      sm_l[c] = w * __ldcg(row + 1);
+      sm_m[c] = w * __ldcg(row + 1);
     }
     __syncthreads();
     const float* col = base + static_cast<size_t>(c0) * kMlaPartialFloats + 2 + c;
-#pragma unroll 4
+#pragma unroll 8
     for (int i = 0; i < n; ++i) {
-      L += sm_l[i];
+      L += sm_m[i];
       acc = fmaf(sm_w[i], __ldcg(col + static_cast<size_t>(i) * kMlaPartialFloats), acc);
     }
   }
@@ -730,7 +762,6 @@ __global__ void __launch_bounds__(kMlaDv) mla_combine_kernel(const float* partia
   out[hq * kMlaDv + c] = (L > 0.f) ? acc / L : 0.f;
   if (lse && c == 0) lse[hq] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : kNegInfT;
 }
-
 
 }  // namespace
 
