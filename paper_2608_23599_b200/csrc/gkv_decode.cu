@@ -31,13 +31,7 @@ constexpr float kNegInf = -__builtin_huge_valf();
 constexpr int kRowPitch = kRowBytes + 16;       // staged exact rows: 272 B pitch -> conflict-free ldmatrix
 constexpr uint32_t kOnesH2 = 0x3C003C00u;       // half2(1, 1)
 constexpr int kWaitSpins = 1 << 20;             // bound of every mbarrier wait (each poll may sleep up to the hint)
-#ifndef GKV_WAIT_HINT_NS
-#define GKV_WAIT_HINT_NS 2000
-#endif
-constexpr uint32_t kWaitHintNs = GKV_WAIT_HINT_NS;
-#ifndef GKV_L2_PREFETCH_AHEAD
-#define GKV_L2_PREFETCH_AHEAD 0
-#endif    // suspend-time hint of one poll, nanoseconds
+constexpr uint32_t kWaitHintNs = 2000;          // suspend-time hint of one mbarrier poll, nanoseconds
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -64,9 +58,6 @@ __device__ __forceinline__ void cp_async_mbar_arrive(uint32_t bar) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -661,11 +652,7 @@ __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, int tm, uint3
   float qo[4] = {0.f, 0.f, 0.f, 0.f};   // ... over odd MMA indices (2-bit only)
   kp += c4 * 16;
   qk_slab<BITS, FULL, true>(kp, kc0, 0, tm, qh_addr, lane, ones, zd, qe, qo, S);
-#ifdef GKV_QK_ROLL
-#pragma unroll 1
-#else
 #pragma unroll
-#endif
   for (int j = 1; j < 4; ++j) qk_slab<BITS, FULL, false>(kp, kc0, j, tm, qh_addr, lane, ones, zd, qe, qo, S);
   if (!FULL) {
     if (!(tm & 1)) S[0][0] = S[0][1] = S[0][2] = S[0][3] = 0.f;
@@ -730,11 +717,7 @@ __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const 
   float ps[4][4];                       // per group: sum over tokens of P' (all rows equal)
 #pragma unroll
   for (int g = 0; g < 4; ++g) ps[g][0] = ps[g][1] = ps[g][2] = ps[g][3] = 0.f;
-#ifdef GKV_PV_ROLL
-#pragma unroll 1
-#else
 #pragma unroll
-#endif
   for (int t = 0; t < 2; ++t) {
     if (!FULL && !((tm >> t) & 1)) continue;
     const uint32_t p0 = t ? pf[1][0] : pf[0][0], p1 = t ? pf[1][1] : pf[0][1];
@@ -956,12 +939,6 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
 #pragma unroll
   for (int i = 0; i < 4; ++i) asm volatile("mov.b32 %0, %1;\n" : "=r"(ones[i]) : "r"(kOnesH2));
 
-#ifdef GKV_EXP_PROFILE
-  long long prof_wait = 0, prof_steps = 0;
-  const long long prof_t0 = clock64();
-  unsigned long long prof_g0;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(prof_g0));
-#endif
   // Software pipeline over steps: while step k is computed, step k + 1 is in flight.  The loop
   // starts on an empty pseudo-unit (level 0) so that the cursor and copy code exists once.
   Cursor cur;
@@ -982,14 +959,8 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   while (have) {
     Cursor nxt = cur;
     const bool more = advance<SPARSE>(w, nxt);
-#ifndef GKV_EXP_SKIP_COPY
     if (more) issue_step<SPARSE>(w, nxt, sidx ^ 1);
-#endif
     if (cur.level != 0) {
-#ifndef GKV_EXP_SKIP_COPY
-#ifdef GKV_EXP_PROFILE
-      const long long tw0 = clock64();
-#endif
       // bounded wait for this step's bytes
       int spins = 0;
       while (!mbar_try_wait(w.bar0 + 8 * sidx, (phase >> sidx) & 1u)) {
@@ -999,29 +970,14 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
         }
       }
       if (__any_sync(kFull, failed)) break;
-#ifdef GKV_EXP_PROFILE
-      prof_wait += clock64() - tw0;
-      prof_steps += 1;
-#endif
       phase ^= 1u << sidx;
-#endif
-#ifndef GKV_EXP_SKIP_COMPUTE
       compute_step<SPARSE>(w, cur, sidx, ones, st, pf);
-#endif
       __syncwarp();
     }
     cur = nxt;
     have = more;
     sidx ^= 1;
   }
-#ifdef GKV_EXP_PROFILE
-  if (lane == 0 && (blockIdx.x % 10) == 0) {
-    unsigned long long prof_g1;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(prof_g1));
-    printf("PROF warp %d stream %d items %d steps %lld total %lld wait %lld g0 %llu g1 %llu\n", gw, w.stream, w.item_end - first,
-           prof_steps, clock64() - prof_t0, prof_wait, prof_g0 % 1000000000ull, prof_g1 % 1000000000ull);
-  }
-#endif
   if (failed) {
     // a copy never completed: flag it and publish an empty partial (the host reports BAD_STATE)
     if (lane == 0) atomicOr(p.status, kStatusInternal);

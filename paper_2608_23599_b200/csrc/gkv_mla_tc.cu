@@ -19,9 +19,6 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
-#ifdef GKV_TC_PROFILE
-#include <cstdio>
-#endif
 
 #include "gkv_internal.h"
 #include "gkv_layout.cuh"
@@ -357,11 +354,6 @@ __device__ __forceinline__ void tc_rows_quarter(uint32_t raw, uint32_t tile, int
 }
 
 // ---- kernel ------------------------------------------------------------------------------------
-#ifdef GKV_TC_PROFILE
-#define TCP(acc) do { const long long c_y = clock64(); acc += c_y - c_x; c_x = c_y; } while (0)
-#else
-#define TCP(acc)
-#endif
 // Warp roles: 0-3 softmax (warp w owns tensor-memory lanes 32 w .. 32 w + 31), 4-12 dequantisation,
 // 13 producer, 14 tensor-core issue.
 __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __grid_constant__ MlaDecodeParams p) {
@@ -433,11 +425,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
         const int b = tg & 1;
         const uint64_t da = t_desc(base + kOffTile + b * kTcTileBytes, 16, 1024);
         const uint32_t d = tmem + kTmemS + 16 * b;
-#ifdef GKV_TC_ROLL_MMA
-#pragma unroll 1
-#else
 #pragma unroll
-#endif
         for (int pn = 0; pn < 9; ++pn)
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
@@ -450,11 +438,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
         // P: [64 tokens][16 heads] fp16, heads contiguous (MN-major), 32-byte swizzle, 8-token groups of 256 B
         const uint64_t dp = t_desc(base + kOffP + b * kTcPBytes, 256, 256, 6);
         const uint32_t first = tg != 0;
-#ifdef GKV_TC_ROLL_MMA
-#pragma unroll 1
-#else
 #pragma unroll
-#endif
         for (int i = 0; i < 4; ++i)
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
@@ -511,20 +495,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     TcTile t;
     int it = cd.item_begin, tg = 0, sg = 0;
     bool ok = true;
-#ifdef GKV_TC_PROFILE
-    long long c_pv = 0, c_raw = 0, c_deq = 0, c_t0 = clock64(), c_x = 0;
-    int n_cent = 0;
-#endif
     while (ok && tc_next(p, table, cd.item_end, it, t)) {
       const int b = tg & 1;
       const uint32_t tile = base + kOffTile + b * kTcTileBytes;
-#ifdef GKV_TC_PROFILE
-      c_x = clock64();
-      n_cent += t.kind == 2;
-#endif
       // the tile buffer is free once the value MMAs of tile tg - 2 are done
       if (tg >= 2) ok = t_wait_warp(bar(kBarPvDone, b), ((tg - 2) >> 1) & 1, abort_flag);
-      TCP(c_pv);
       if (!ok) break;
       if (dt < 64) bias_sm[b * 64 + dt] = dt < t.nrows ? (t.kind == 2 ? 6.0f : 0.f) : kNegInfT;   // log2(64) per centroid row
       const int nq = (t.kind == 0) ? 2 : 4;
@@ -532,7 +507,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
         if (s < t.nstages) {
           const int rb = sg & 1;
           ok = t_wait_warp(bar(kBarRawFull, rb), (sg >> 1) & 1, abort_flag);
-          TCP(c_raw);
           if (!ok) break;
           const uint32_t raw = base + kOffRaw + rb * kTcRawBytes;
           if (t.kind == 0) {
@@ -552,15 +526,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       t_fence_async();
       __syncwarp();
       if (lane == 0) t_bar_arrive(bar(kBarKtFull, b));
-      TCP(c_deq);
       it = t.item + t.adv;
       ++tg;
     }
-#ifdef GKV_TC_PROFILE
-    if (lane == 0 && warp == 4 && (blockIdx.x % 37 == 0 || blockIdx.x < 3))
-      printf("TCP cta %d tiles %d (centroid %d) total %lld pvwait %lld rawwait %lld dequant %lld\n", blockIdx.x, tg, n_cent,
-             clock64() - c_t0, c_pv, c_raw, c_deq);
-#endif
   } else {
     // ---------------- softmax (warps 0-3) and the result ----------------
     float m_run[16], l_part[16];
@@ -573,16 +541,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     int it = cd.item_begin, ts = 0, xph = 0;                // xph: exchanges done so far (phase of the exchange barrier)
     bool ok = true;
     const uint32_t tlane = tmem + (static_cast<uint32_t>(32 * warp) << 16);
-#ifdef GKV_TC_PROFILE
-    long long s_w = 0, s_x = 0, s_r = 0, s_c = 0, s_t0 = clock64(), c_x = 0;
-#endif
     while (tc_next(p, table, cd.item_end, it, t)) {
       const int b = ts & 1;
-#ifdef GKV_TC_PROFILE
-      c_x = clock64();
-#endif
       ok = t_wait_warp(bar(kBarSFull, b), (ts >> 1) & 1, abort_flag) && ok;
-      TCP(s_w);
       t_fence_after();
       float s[16];
       t_ld16(tlane + kTmemS + 16 * b, s);
@@ -597,7 +558,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
         s[h] = (bs == kNegInfT) ? kNegInfT : fmaf(s[h], p.scale_log2, bs);
         mine |= s[h] > m_run[h] + kRescaleSlack;            // also true for the first finite logit (max = -inf)
       }
-      TCP(s_c);
       uint32_t need_u;
       asm volatile(
           "{\n"
@@ -610,7 +570,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
           : "r"(static_cast<uint32_t>(mine))
           : "memory");
       const bool need = need_u != 0;
-      TCP(s_x);
       if (need) {                                           // uniform over the 128 softmax threads
         float mx[16];
 #pragma unroll
@@ -670,15 +629,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       t_fence_before();
       __syncwarp();
       if (lane == 0) t_bar_arrive(bar(kBarPFull, b));
-      TCP(s_r);
       it = t.item + t.adv;
       ++ts;
     }
-#ifdef GKV_TC_PROFILE
-    if (lane == 0 && warp == 0 && blockIdx.x % 37 == 0)
-      printf("TCS cta %d tiles %d total %lld wait_s %lld load_max %lld exchange %lld rest %lld\n", blockIdx.x, ts, clock64() - s_t0, s_w,
-             s_c, s_x, s_r);
-#endif
     // ---------------- result ----------------
     float* out = p.partial + static_cast<size_t>(cd.partial) * kMlaPartialFloats;
     if (ts > 0) ok = t_wait_warp(bar(kBarPvDone, (ts - 1) & 1), ((ts - 1) >> 1) & 1, abort_flag) && ok;
