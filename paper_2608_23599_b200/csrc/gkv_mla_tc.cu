@@ -673,47 +673,61 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
   if (warp == 0) t_tmem_dealloc(tmem, kTmemCols);
 }
 
-// Merge the partial rows of a stream's CTAs in CTA order (bitwise reproducible), one block per
-// (stream, head), one thread per value channel.
-__global__ void __launch_bounds__(kMlaDv) mla_combine_kernel(const float* partial, const StreamParts* parts, float* out,
-                                                             float* lse) {
-  __shared__ float sm_m[kMlaDv], sm_w[kMlaDv];
-  const int stream = blockIdx.x, h = blockIdx.y, c = threadIdx.x;
+// Merge the partial rows of a stream's CTAs.  One block per (stream, head, slice of 64 value
+// channels); its 512 threads are 8 row groups x 64 channels, row group g sums rows g, g + 8, ...
+// in that order and the 8 sums are added in group order, so the result is bitwise reproducible.
+constexpr int kCombSlice = 64, kCombGroups = 8, kCombThreads = kCombSlice * kCombGroups;
+__global__ void __launch_bounds__(kCombThreads) mla_combine_kernel(const float* partial, const StreamParts* parts, float* out,
+                                                                   float* lse) {
+  __shared__ float sm_m[kCombThreads], sm_w[kCombThreads], sm_acc[kCombGroups][kCombSlice];
+  const int stream = blockIdx.x, h = blockIdx.y, slice = blockIdx.z, tid = threadIdx.x;
+  const int c = tid % kCombSlice, g = tid / kCombSlice;
   const int begin = parts[stream].begin, end = parts[stream].end;
   const float* base = partial + h * (kMlaDv + 2);
   // pass 1: the maximum of the rows' maxima (one row per thread, then a shared-memory sweep)
   float M = kNegInfT;
-  for (int c0 = begin; c0 < end; c0 += kMlaDv) {
-    const int n = min(kMlaDv, end - c0);
+  for (int c0 = begin; c0 < end; c0 += kCombThreads) {
+    const int n = min(kCombThreads, end - c0);
     __syncthreads();
-    sm_m[c] = c < n ? __ldcg(base + static_cast<size_t>(c0 + c) * kMlaPartialFloats) : kNegInfT;
+    sm_m[tid] = tid < n ? __ldcg(base + static_cast<size_t>(c0 + tid) * kMlaPartialFloats) : kNegInfT;
     __syncthreads();
 #pragma unroll 8
     for (int i = 0; i < n; ++i) M = fmaxf(M, sm_m[i]);
   }
-  // pass 2: weights per row in shared memory, then every thread sums its channel over the rows
+  // pass 2: weights per row in shared memory, then every thread sums its channel over its rows
   float L = 0.f, acc = 0.f;
-  for (int c0 = begin; c0 < end; c0 += kMlaDv) {
-    const int n = min(kMlaDv, end - c0);
+  for (int c0 = begin; c0 < end; c0 += kCombThreads) {
+    const int n = min(kCombThreads, end - c0);
     __syncthreads();
-    if (c < n) {
-      const float* row = base + static_cast<size_t>(c0 + c) * kMlaPartialFloats;
+    if (tid < n) {
+      const float* row = base + static_cast<size_t>(c0 + tid) * kMlaPartialFloats;
       const float m = __ldcg(row);
       const float w = (m == kNegInfT) ? 0.f : exp2f(m - M);
-      sm_w[c] = w;
-      sm_m[c] = w * __ldcg(row + 1);
+      sm_w[tid] = w;
+      sm_m[tid] = w * __ldcg(row + 1);
     }
     __syncthreads();
-    const float* col = base + static_cast<size_t>(c0) * kMlaPartialFloats + 2 + c;
+    const float* col = base + static_cast<size_t>(c0) * kMlaPartialFloats + 2 + slice * kCombSlice + c;
 #pragma unroll 8
-    for (int i = 0; i < n; ++i) {
-      L += sm_m[i];
-      acc = fmaf(sm_w[i], __ldcg(col + static_cast<size_t>(i) * kMlaPartialFloats), acc);
-    }
+    for (int i = g; i < n; i += kCombGroups) acc = fmaf(sm_w[i], __ldcg(col + static_cast<size_t>(i) * kMlaPartialFloats), acc);
+    if (g == 0 && c == 0)
+      for (int i = 0; i < n; ++i) L += sm_m[i];
   }
-  const size_t hq = static_cast<size_t>(stream) * kMlaHeads + h;
-  out[hq * kMlaDv + c] = (L > 0.f) ? acc / L : 0.f;
-  if (lse && c == 0) lse[hq] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : kNegInfT;
+  sm_acc[g][c] = acc;
+  __syncthreads();
+  if (g == 0) {
+    if (c == 0) sm_m[0] = L;
+  }
+  __syncthreads();
+  L = sm_m[0];
+  if (g == 0) {
+    float tot = 0.f;
+#pragma unroll
+    for (int k = 0; k < kCombGroups; ++k) tot += sm_acc[k][c];
+    const size_t hq = static_cast<size_t>(stream) * kMlaHeads + h;
+    out[hq * kMlaDv + slice * kCombSlice + c] = (L > 0.f) ? tot / L : 0.f;
+    if (lse && slice == 0 && c == 0) lse[hq] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : kNegInfT;
+  }
 }
 
 }  // namespace
@@ -730,7 +744,7 @@ cudaError_t launch_mla_decode(const MlaDecodeParams& p, int n_ctas, const Stream
   mla_tc_decode_kernel<<<n_ctas, kTcThreads, kTcSmem, st>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  mla_combine_kernel<<<dim3(n_streams, kMlaHeads), kMlaDv, 0, st>>>(p.partial, parts, out, lse);
+  mla_combine_kernel<<<dim3(n_streams, kMlaHeads, kMlaDv / kCombSlice), kCombThreads, 0, st>>>(p.partial, parts, out, lse);
   return cudaGetLastError();
 }
 
