@@ -219,9 +219,10 @@ struct TcTile {
   uint32_t off256;
 };
 
-__device__ __noinline__ bool tc_next(const MlaDecodeParams& p, const TableEntry* table, int item_end, int it, TcTile& t) {
+// `e` is the caller's copy of table[it] (it fetches the next one while a tile is being worked on).
+__device__ __noinline__ bool tc_next(const MlaDecodeParams& p, const TableEntry* table, int item_end, int it, const TableEntry e,
+                                     TcTile& t) {
   if (it >= item_end) return false;
-  const TableEntry e = table[it];
   t.item = it;
   t.adv = 1;
   t.off256 = e.off256;
@@ -259,6 +260,11 @@ __device__ __noinline__ bool tc_next(const MlaDecodeParams& p, const TableEntry*
     t.nstages = 2;
   }
   return true;
+}
+
+// table[it] for the iterator, clamped to the stream's last entry (the tail)
+__device__ __forceinline__ TableEntry tc_entry(const MlaDecodeParams& p, const TableEntry* table, int it) {
+  return table[min(it, p.n_closed)];
 }
 
 // producer warp: copies of stage s of tile t into raw buffer `raw`.  Lane 0 posts the byte count
@@ -407,7 +413,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     TcTile t;
     int it = cd.item_begin, sg = 0;
     bool ok = true;
-    while (ok && tc_next(p, table, cd.item_end, it, t)) {
+    TableEntry pre = tc_entry(p, table, it);
+    while (ok && tc_next(p, table, cd.item_end, it, pre, t)) {
+      pre = tc_entry(p, table, t.item + t.adv);
       for (int s = 0; s < t.nstages && ok; ++s, ++sg) {
         const int b = sg & 1;
         ok = t_wait_warp(bar(kBarRawEmpty, b), ((sg >> 1) & 1) ^ 1, abort_flag);        // fresh barriers pass
@@ -451,7 +459,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       // tile buffers are double).  n_tiles is not known in advance: the iterator tells.
       TcTile t;
       int it = cd.item_begin;
-      bool more_tiles = tc_next(p, table, cd.item_end, it, t);
+      TableEntry pre = tc_entry(p, table, it);
+      bool more_tiles = tc_next(p, table, cd.item_end, it, pre, t);
+      pre = tc_entry(p, table, t.item + t.adv);
       int qk = 0, pv = 0, n_known = more_tiles ? 1 : 0;      // tiles [0, n_known) exist so far
       bool ok = true;
       int spins = 0;
@@ -466,8 +476,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
             ++qk;
             // look one tile further
             it = t.item + t.adv;
-            more_tiles = tc_next(p, table, cd.item_end, it, t);
-            if (more_tiles) ++n_known;
+            more_tiles = tc_next(p, table, cd.item_end, it, pre, t);
+            if (more_tiles) {
+              ++n_known;
+              pre = tc_entry(p, table, t.item + t.adv);
+            }
             progress = true;
           }
         }
@@ -495,7 +508,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     TcTile t;
     int it = cd.item_begin, tg = 0, sg = 0;
     bool ok = true;
-    while (ok && tc_next(p, table, cd.item_end, it, t)) {
+    TableEntry pre = tc_entry(p, table, it);
+    while (ok && tc_next(p, table, cd.item_end, it, pre, t)) {
+      pre = tc_entry(p, table, t.item + t.adv);
       const int b = tg & 1;
       const uint32_t tile = base + kOffTile + b * kTcTileBytes;
       // the tile buffer is free once the value MMAs of tile tg - 2 are done
@@ -541,7 +556,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     int it = cd.item_begin, ts = 0, xph = 0;                // xph: exchanges done so far (phase of the exchange barrier)
     bool ok = true;
     const uint32_t tlane = tmem + (static_cast<uint32_t>(32 * warp) << 16);
-    while (tc_next(p, table, cd.item_end, it, t)) {
+    TableEntry pre = tc_entry(p, table, it);
+    while (tc_next(p, table, cd.item_end, it, pre, t)) {
+      pre = tc_entry(p, table, t.item + t.adv);
       const int b = ts & 1;
       ok = t_wait_warp(bar(kBarSFull, b), (ts >> 1) & 1, abort_flag) && ok;
       t_fence_after();
