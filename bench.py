@@ -373,7 +373,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", type=int, default=2, help="workload: 0..4 (default 2: Llama-8B-like batched decode)")
+    ap.add_argument("--config", type=int, default=2, help="workload: 0..4 (default 2: Llama-8B-like batched decode); 5 = RD-V2 operating point")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (0 = as defined)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

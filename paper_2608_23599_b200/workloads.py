@@ -70,7 +70,7 @@ class Workload:
 
 
 def config(cid: int, scale: str = "full") -> Workload:
-    """The five benchmark configurations; ``scale='small'`` keeps the structure
+    """The five benchmark configurations (0-4) and the RD-V2 operating point (5); ``scale='small'`` keeps the structure
     (every rung populated, ragged tail, several splits) at a size the CPU
     oracle finishes in seconds."""
     small = scale == "small"
@@ -111,6 +111,15 @@ def config(cid: int, scale: str = "full") -> Workload:
                         16, 1, 576, 512, T, T + 128, v_aliases_k=1,
                         stair_tokens=(w16, w8, w4, 0), softmax_scale=1.0 / math.sqrt(192.0),
                         n_outlier=8, outlier_gain=6.0, n_heavy=0)
+    if cid == 5:
+        # not one of the five headline configurations: the paper's RD-V2 operating point
+        # (Sec. 3.3 / Table 2: a near-centroid-only base plus ~10 % exact residual tokens chosen by
+        # attention mass x squared value error, ~2 bits/value) on the config-2 shapes
+        if small:
+            return Workload("cfg5_rdv2_small", 5, 1, 2, 8, 2, 128, 128, 2048 + 40, 2048 + 128,
+                            stair_tokens=(128, 0, 0, 0), residual_fraction=0.10, drift_std=0.05)
+        return Workload("cfg5_rdv2", 5, 32, 8, 32, 8, 128, 128, 32768, 32768 + 128,
+                        stair_tokens=(256, 0, 0, 0), residual_fraction=0.10, drift_std=0.05)
     raise ValueError(cid)
 
 
@@ -197,7 +206,7 @@ def make_layer(w: Workload, layer: int, device="cpu", ctx: Optional[int] = None,
         "q": q.to(torch.bfloat16),
     }
 
-    want_mass = (w.policy == POLICY_RD) if with_mass is None else with_mass
+    want_mass = (w.policy == POLICY_RD or w.residual_fraction > 0) if with_mass is None else with_mass
     if want_mass:
         # prompt attention mass per token: softmax weights of 16 synthetic observation
         # queries per head, averaged over the queries and the g heads of the KV head

@@ -139,6 +139,33 @@ def test_cfg1_small_rd_allocator_and_residual():
     gcache.close()
 
 
+def test_rdv2_operating_point_small():
+    """The paper's RD-V2 operating point (Table 2): every closed block outside a short exact window
+    is a centroid, 10 % of the tokens stay exact as residual rows; then decode steps with appends."""
+    w = W.config(5, "small")
+    ocache, gcache = _pair(w)
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    U.assert_state_equal(ocache, gcache, 0)
+    lv = ocache.levels(0, 0, 0)
+    assert set(lv.tolist()) <= {16, 1} and (lv == 1).sum() >= len(lv) - 3
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
+    U.assert_outputs_close(out, o_out, "rdv2-small", scale=U.value_scale(data["v"]))
+    rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
+    assert rep_g.resident_bits == rep_o["resident_bits"] and rep_g.last_read_bits == rep_o["last_read_bits"]
+    assert 1.5 < rep_g.bpv_paper < 3.5
+    for step in range(30):
+        tok = W.make_decode_tokens(w, 0, step, "cpu")
+        ocache.append_demote(0, U.f32(tok["k"]), U.f32(tok["v"]))
+        gcache.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
+        if step in (0, 23, 24, 29):
+            out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, tok["q"])
+            U.assert_outputs_close(out, o_out, f"rdv2-small step {step}", scale=U.value_scale(data["v"]))
+    U.assert_state_equal(ocache, gcache, 0)
+    gcache.close()
+
+
 def test_cfg3_small_quest_select_and_sparse_attention():
     """Config 3 structure: exact page boxes, box upper-bound scores, top-k pages, attention over
     the selected graded pages plus the partial tail block."""
