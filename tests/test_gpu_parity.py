@@ -197,6 +197,34 @@ def test_cfg3_small_quest_select_and_sparse_attention():
     gcache.close()
 
 
+@pytest.mark.parametrize("page", [32, 64])
+def test_quest_larger_pages(page):
+    """Page sizes 32 and 64 (the paper's own Quest setting is page = block = 64 tokens with a
+    12.5 % page budget): boxes, scores, selection and the page-sparse read."""
+    w = dataclasses.replace(W.config(3, "small"), page_tokens=page, quest_budget_tokens=256)
+    ocache, gcache = _pair(w)
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    U.assert_state_equal(ocache, gcache, 0)
+    k = w.quest_budget_tokens // page
+    pages = torch.full((w.batch, w.n_kv_heads, k), -1, dtype=torch.int32, device=dev)
+    n_sel = gcache.gkv_quest_select(0, data["q"].to(dev), w.quest_budget_tokens, pages)
+    torch.cuda.synchronize()
+    sel_o = ocache.quest_select(0, U.f32(data["q"]), w.quest_budget_tokens)
+    assert n_sel == k
+    pg = pages.cpu().numpy()
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            assert np.array_equal(pg[b, h], sel_o[b][h]), f"selected pages differ for stream {(b, h)}"
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"], page_idx_gpu=pages, n_sel=n_sel,
+                                           page_idx_oracle=sel_o)
+    U.assert_outputs_close(out, o_out, f"page {page} sparse")
+    rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
+    assert rep_g.resident_bits == rep_o["resident_bits"] and rep_g.last_read_bits == rep_o["last_read_bits"]
+    gcache.close()
+
+
 def test_quest_selecting_every_page_equals_full_read():
     w = dataclasses.replace(W.config(3, "small"), quest_budget_tokens=1 << 20)
     ocache, gcache = _pair(w)
