@@ -119,16 +119,25 @@ def barrier(world):
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
-    torch.cuda.synchronize()
+    if torch.cuda.is_available():
+        torch.cuda.synchronize()
 
 
 def max_over_ranks(x: float, world: int) -> float:
+    """Replicas do not exchange data; the only collective is this maximum of the per-rank times
+    (NCCL on the GPUs; the CPU tests run it over gloo)."""
     if world == 1:
         return x
     import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([x], dtype=torch.float64, device=dev)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def aggregate_value(world: int, batch: int, ctx: int, ms_step: float) -> float:
+    """Whole-job context tokens/s of `world` replicas whose slowest rank took ms_step per step."""
+    return world * batch * ctx / (ms_step * 1e-3)
 
 
 # --------------------------------------------------------------------------------------------------
@@ -201,7 +210,7 @@ def run_ours(args, rank, local, world):
     barrier(world)
     clocks = sampler.stop()
     ms_step = max_over_ranks(ev0.elapsed_time(ev1) / K, world)
-    value = world * Bsz * ctx_start / (ms_step * 1e-3)
+    value = aggregate_value(world, Bsz, ctx_start, ms_step)
 
     # ---- dominant kernel: decode_attn alone, per launch -------------------------------------------
     rep = cache.gkv_bits_report(0)
