@@ -181,6 +181,15 @@ GKV_API int gkv_debug_export_residual(gkv_cache* c, int32_t layer, int32_t b, in
 /* Levels of all closed blocks of one stream.  levels: host int8 [cap]; n: host. */
 GKV_API int gkv_debug_export_levels(gkv_cache* c, int32_t layer, int32_t b, int32_t kv_head, int8_t* levels,
                             int32_t cap, int32_t* n);
+/* The host-side level plan on its own, without a cache or a device (all pointers host): what
+ * gkv_append_demote decides for one stream whose n_closed blocks are closed and whose tail holds
+ * n_tail tokens.  Staircase policy (Sec. 3.2, Fig. 1): from cfg->stair_tokens / n_sink_blocks;
+ * mass and range are ignored and may be NULL.  RD policy (Sec. 3.3, the monotone allocator):
+ * mass / range are fp32 [n_closed] per-block attention mass and range proxy; *budget_miss is set
+ * when even the cheapest plan exceeds rd_budget_bpv.  levels: int8 [n_closed], index 0 = oldest.
+ * Used by the CPU tests to hold the host logic against the oracle. */
+GKV_API int gkv_debug_plan_levels(const gkv_config* cfg, int32_t n_closed, int32_t n_tail, const float* mass,
+                                  const float* range, int8_t* levels, int32_t* budget_miss);
 /* Current context length (tokens) of a layer. */
 GKV_API int gkv_ctx_len(gkv_cache* c, int32_t layer, int32_t* ctx);
 

@@ -10,6 +10,7 @@ import ctypes as C
 import os
 from typing import Optional
 
+import numpy as np
 import torch
 
 from . import build as _build
@@ -24,7 +25,7 @@ ERR_RANGE, ERR_BUDGET = -6, -7
 EXPORTS = [
     "gkv_query_arena_bytes", "gkv_create", "gkv_destroy", "gkv_append_demote", "gkv_decode_attn",
     "gkv_quest_select", "gkv_quest_select_static", "gkv_bits_report", "gkv_debug_export_block", "gkv_debug_export_residual",
-    "gkv_debug_export_levels", "gkv_ctx_len", "gkv_strerror", "gkv_last_cuda_error",
+    "gkv_debug_export_levels", "gkv_debug_plan_levels", "gkv_ctx_len", "gkv_strerror", "gkv_last_cuda_error",
 ]
 
 
@@ -144,6 +145,21 @@ def gkv_query_arena_bytes(cfg: GkvConfig) -> int:
     out = C.c_size_t(0)
     _check(load().gkv_query_arena_bytes(C.byref(cfg), C.byref(out)), "gkv_query_arena_bytes")
     return out.value
+
+
+def gkv_debug_plan_levels(cfg: GkvConfig, n_closed: int, n_tail: int = 0, mass=None, rng=None):
+    """Host-only level plan of one stream (no device needed): (levels int8 [n_closed], budget_miss)."""
+    levels = np.zeros(max(n_closed, 1), dtype=np.int8)
+    miss = C.c_int32(0)
+    fp = C.POINTER(C.c_float)
+    m = None if mass is None else np.ascontiguousarray(mass, dtype=np.float32)
+    r = None if rng is None else np.ascontiguousarray(rng, dtype=np.float32)
+    _check(load().gkv_debug_plan_levels(C.byref(cfg), n_closed, n_tail,
+                                        None if m is None else m.ctypes.data_as(fp),
+                                        None if r is None else r.ctypes.data_as(fp),
+                                        levels.ctypes.data_as(C.POINTER(C.c_int8)), C.byref(miss)),
+           "gkv_debug_plan_levels")
+    return levels[:n_closed], bool(miss.value)
 
 
 class Cache:

@@ -1088,6 +1088,26 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
   return GKV_OK;
 }
 
+int gkv_debug_plan_levels(const gkv_config* cfg, int32_t n_closed, int32_t n_tail, const float* mass, const float* range,
+                          int8_t* levels, int32_t* budget_miss) {
+  int rc = validate_config(cfg);
+  if (rc != GKV_OK) return rc;
+  if (n_closed < 0 || n_tail < 0 || n_tail >= kBlock || (n_closed > 0 && !levels)) return GKV_ERR_INVALID_ARG;
+  if (budget_miss) *budget_miss = 0;
+  if (n_closed == 0) return GKV_OK;
+  if (cfg->policy == GKV_POLICY_STAIRCASE) {
+    staircase_levels(*cfg, n_closed, levels);
+    return GKV_OK;
+  }
+  if (cfg->policy == GKV_POLICY_RD) {
+    if (!mass || !range) return GKV_ERR_INVALID_ARG;
+    const bool miss = rd_allocate(*cfg, mass, range, n_closed, n_tail, levels);
+    if (budget_miss) *budget_miss = miss ? 1 : 0;
+    return GKV_OK;
+  }
+  return GKV_ERR_UNSUPPORTED;      // external plans are the caller's
+}
+
 int gkv_destroy(gkv_cache* c) {
   if (!c) return GKV_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
