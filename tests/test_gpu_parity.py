@@ -338,3 +338,41 @@ def test_cfg4_small_mla_ladder_with_appends():
     U.assert_state_equal(ocache, gcache, 0)
     assert gcache.gkv_bits_report(0).resident_bits == ocache.bits_report(0)["resident_bits"]
     gcache.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("hq,hkv", [(2, 2), (4, 2), (16, 2), (8, 1)])
+def test_query_group_sizes(hq, hkv):
+    """1, 2, 8 query heads per KV head (the tensor-core tile holds up to 8) on a full ladder."""
+    w = _tiny(1000, n_q_heads=hq, n_kv_heads=hkv, stair_tokens=(192, 192, 256, 192))
+    ocache, gcache = _pair(w)
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    U.assert_state_equal(ocache, gcache, 0)
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
+    U.assert_outputs_close(out, o_out, f"group {hq // hkv}")
+    assert np.max(np.abs(lse.cpu().numpy() - o_lse)) < 5e-3
+    gcache.close()
+
+
+@pytest.mark.gpu
+def test_decode_is_bitwise_reproducible():
+    """The split-K merge runs in a fixed order whichever CTA finishes last: the same call twice,
+    and the same cache read through a second handle, give identical bits."""
+    w = W.config(2, "small")
+    outs = []
+    for _ in range(2):
+        _, gcache = _pair(w)
+        dev = gcache.device
+        data = W.make_layer(w, 0, "cpu")
+        gcache.gkv_append_demote(0, data["k"].to(dev), data["v"].to(dev))
+        q = data["q"].to(dev)
+        for _rep in range(3):
+            out = torch.empty((w.batch, w.n_q_heads, w.d_v), dtype=torch.float32, device=dev)
+            lse = torch.empty((w.batch, w.n_q_heads), dtype=torch.float32, device=dev)
+            gcache.gkv_decode_attn(0, q, out, lse=lse)
+            torch.cuda.synchronize()
+            outs.append((out.cpu().numpy().copy(), lse.cpu().numpy().copy()))
+        gcache.close()
+    for o, l in outs[1:]:
+        assert np.array_equal(o, outs[0][0]) and np.array_equal(l, outs[0][1])
