@@ -903,6 +903,12 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     fence_proxy_async();
   }
   __syncwarp();
+  // Launched with programmatic stream serialisation: what is above (descriptor fetch, barrier
+  // set-up) may overlap the tail of the previous kernel in the stream.  Nothing that a previous
+  // kernel may have written (the query, appended rows, partial rows, tickets) is touched before
+  // this wait, which returns once that kernel has completed and its writes are visible.
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
 
   // Query fragments: B operand Q^T[16 channels x 8 heads]; lane (r, c4) holds head r, channels
   // 16 s + 2 c4 (+1) and 16 s + 8 + 2 c4 (+1), in bf16 (exact rows) and fp16 (quantised tiers).
@@ -1121,9 +1127,18 @@ cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st) {
     configured = true;
   }
   if (n_ctas <= 0) return cudaSuccess;
-  if (p.page_idx) decode_kernel<true><<<n_ctas, kDecodeWarps * 32, decode_smem_bytes(), st>>>(p);
-  else decode_kernel<false><<<n_ctas, kDecodeWarps * 32, decode_smem_bytes(), st>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_ctas);
+  cfg.blockDim = dim3(kDecodeWarps * 32);
+  cfg.dynamicSmemBytes = decode_smem_bytes();
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (p.page_idx) return cudaLaunchKernelEx(&cfg, decode_kernel<true>, p);
+  return cudaLaunchKernelEx(&cfg, decode_kernel<false>, p);
 }
 
 }  // namespace gkv
