@@ -281,6 +281,10 @@ __global__ void __launch_bounds__(128) append_rows_kernel(uint8_t* arena, const 
       in + ((static_cast<size_t>(b) * n_tok + first_tok + row) * n_kv_heads + kvh) * kD);
   uint32_t* dst = reinterpret_cast<uint32_t*>(slot + (is_v ? kBlock * kRowBytes : 0) +
                                               static_cast<size_t>(dst_row0 + row) * kRowBytes);
+  // launched with programmatic stream serialisation: the address set-up above overlaps the tail
+  // of the previous kernel; the new rows are read, and the slot written, only after it completed
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
   dst[i] = src[i];
 }
 
@@ -398,9 +402,17 @@ cudaError_t launch_append_rows(uint8_t* arena, const TableEntry* table, int tabl
                                int n_streams, int n_kv_heads, const uint16_t* k_in, const uint16_t* v_in,
                                int n_tok, int first_tok, int n_rows, int dst_row0, cudaStream_t st) {
   if (n_rows <= 0) return cudaSuccess;
-  append_rows_kernel<<<dim3(n_streams, n_rows), 128, 0, st>>>(arena, table, table_stride, tail_index, n_kv_heads,
-                                                             k_in, v_in, n_tok, first_tok, dst_row0);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_streams, n_rows);
+  cfg.blockDim = dim3(128);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, append_rows_kernel, arena, table, table_stride, tail_index, n_kv_heads, k_in, v_in, n_tok,
+                            first_tok, dst_row0);
 }
 
 cudaError_t launch_residual_scores(const uint16_t* v_in, const float* token_mass, const int8_t* levels,
