@@ -8,6 +8,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <numeric>
 #include <vector>
 
 #include "../../include/gkv.h"
@@ -364,22 +365,22 @@ bool rd_allocate(const gkv_config& c, const float* mass, const float* range, int
 
 // ---- decode work split ---------------------------------------------------------------------------
 // Cost of one item for the work split: cycles a warp needs for it while the whole GPU runs the
-// mixed workload (measured on B200 by timing individual warps of the config-2 launch: an exact
-// block ~26 K cycles, 8-bit ~11.5 K, 4-bit ~10 K, 2-bit ~6.7 K, a centroid block ~0.6 K).  Bytes
-// alone are the wrong weight: below 8 bits the kernel is bound by instruction issue and a block
-// costs about the same whatever its code width.
+// mixed workload, measured on B200 by timing every step of individual warps of the config-2 launch
+// (in units where a 4-bit block is 1000): an exact block 1590, 8-bit 1070, 4-bit 1000, 2-bit 1015, a
+// centroid block 47 (a run of 16 costs 745).  Bytes are the wrong weight: below 8 bits the kernel
+// is bound by instruction issue and a block costs the same whatever its code width.
 size_t item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) {
   if (item < L.n_closed) {
     switch (L.level[static_cast<size_t>(stream) * c->max_blocks + item]) {
-      case 16: return 2600;
-      case 8: return 1150;
+      case 16: return 1590;
+      case 8: return 1070;
       case 4: return 1000;
-      case 2: return 670;
-      default: return 60;
+      case 2: return 1015;
+      default: return 47;
     }
   }
-  if (item == L.n_closed) return 1300;     // tail: mid-fill estimate (its size changes every step)
-  return 650;                              // residual group of 16 exact rows
+  if (item == L.n_closed) return 800;      // tail: mid-fill estimate (its size changes every step)
+  return 550;                              // residual group of 16 exact rows
 }
 
 // Units of a stream (a block, a run of up to 16 neighbouring centroid blocks, the tail, a residual
@@ -427,24 +428,30 @@ void build_descs(gkv_cache* c, LayerState& L) {
     std::stable_sort(u.begin(), u.end(), [](const Unit& a, const Unit& b) { return a.cost > b.cost; });
     load.assign(nw, 0);
     mine.assign(nw, {});
-    static const double wave2 = std::getenv("GKV_WAVE2_SPEED") ? std::atof(std::getenv("GKV_WAVE2_SPEED")) : 1.0;
-    std::vector<double> inv(nw);
-    for (int k = 0; k < nw; ++k) inv[k] = ((w + k) / kDecodeWarps >= 148) ? 1.0 / wave2 : 1.0;
     for (const Unit& x : u) {
       int best = 0;
       for (int k = 1; k < nw; ++k)
-        if ((load[k] + x.cost) * inv[k] < (load[best] + x.cost) * inv[best]) best = k;
+        if (load[k] < load[best]) best = k;
       load[best] += x.cost;
       mine[best].push_back(x.word);
     }
+    // Longest-first dealing hands the costliest units (exact blocks, then 8-bit ones) to the first
+    // warps, and a CTA is a window of consecutive warps: walk the warps with a golden-ratio stride so
+    // that every window holds the same mixture of levels.  Warps of one SM share its issue slots, and
+    // a CTA whose warps all run the issue-heavy levels would finish last.
+    int stride = std::max(1, static_cast<int>(nw * 0.6180339887 + 0.5));
+    while (std::gcd(stride, nw) != 1) ++stride;
+    std::vector<int> order(nw);
+    for (int k = 0; k < nw; ++k) order[k] = static_cast<int>((static_cast<long long>(k) * stride) % nw);
     // one partial row per (CTA, stream): the kernel merges the warps of a CTA that share a stream
     L.parts_h[s].begin = row;
     for (int k = 0; k < nw; ++k) {
-      std::sort(mine[k].begin(), mine[k].end(), [](uint32_t a, uint32_t b) { return (a & 0xffffffu) < (b & 0xffffffu); });
+      std::vector<uint32_t>& m = mine[order[k]];
+      std::sort(m.begin(), m.end(), [](uint32_t a, uint32_t b) { return (a & 0xffffffu) < (b & 0xffffffu); });
       WarpDesc& d = L.warps_h[w];
       d.stream = s;
       d.item_begin = pos;
-      for (uint32_t x : mine[k]) L.units_h[pos++] = x;
+      for (uint32_t x : m) L.units_h[pos++] = x;
       d.item_end = pos;
       if (k > 0 && w % kDecodeWarps == 0) ++row;
       d.partial = row;
