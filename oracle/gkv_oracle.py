@@ -18,6 +18,9 @@ What it follows (paper sections / equations):
   readable, cold pages hard-masked; resident / read accounting (Sec. 3.5,
   Eq. 7-8).
 * Attention error certificate (Sec. 3.6, Eq. 9) - used as a pin in the tests.
+* Block attention mass m_b (Sec. 3.1, Eq. 2): the summed softmax weight of a
+  block's tokens, averaged over the KV head's query heads, and its running
+  update m_b <- 0.9 m_b + 0.1 m_b_new at every observed decode query.
 * Dense softmax attention over the reconstructed cache (Sec. 3.1, Eq. 1;
   Sec. 3.7) evaluated in float64.
 
@@ -249,6 +252,7 @@ class Stream:
     res_v: Optional[np.ndarray] = None
     range_flag: bool = False
     budget_flag: bool = False
+    ema_mass: np.ndarray = field(default_factory=lambda: np.zeros(0, np.float64))   # running m_b, one per block (+ partial block)
 
     @property
     def n_closed(self) -> int:
@@ -490,6 +494,7 @@ class GradedCache:
                                               cfg.rd_budget_bpv, cfg.n_sink_blocks, cfg.retire_after,
                                               None, cfg.monotone_in_age)
             st.budget_flag = bflag
+            st.ema_mass = mass_b.astype(np.float64)        # the prefill observer's masses start the running average
         if cfg.residual_fraction > 0 and token_mass is not None:
             vsrc = kk[:, :cfg.d_v] if self.alias else vv
             st.res_idx = rd_residual_select(token_mass, vsrc[:n_closed * P], levels, cfg.n_sink_blocks,
@@ -611,6 +616,35 @@ class GradedCache:
         if return_weights:
             return out, lse, weights
         return out, lse
+
+    def decode_attn_observe(self, layer: int, q):
+        """decode_attn over the full context that also observes block attention mass (Sec. 3.1).
+
+        For every stream: a_b = (1/g) sum over the KV head's g query heads of sum_{j in b} w_{h,j}
+        (Eq. 2 with the current query as the observed one; the heads that share the KV head are
+        aggregated, Sec. 3.1 last paragraph), b = 0 .. n_closed with the last entry the partial
+        block (absent when it is empty).  Tokens served from the exact residual count for the
+        block they sit in.  Then the running mass: m_b <- 0.9 m_b + 0.1 a_b (a block seen for the
+        first time starts from 0).  Returns out, lse, {(b, kv head): a}."""
+        cfg = self.cfg
+        g = cfg.n_q_heads // cfg.n_kv_heads
+        out, lse, weights = self.decode_attn(layer, q, None, return_weights=True)
+        observed = {}
+        for b in range(cfg.batch):
+            for h in range(cfg.n_kv_heads):
+                st = self.streams[(layer, b, h)]
+                nb = st.n_closed + (1 if st.n_tail else 0)
+                a = np.zeros(nb, dtype=np.float64)
+                for j in range(g):
+                    w = weights[(b, h * g + j)]
+                    for blk in range(nb):
+                        a[blk] += w[blk * P:(blk + 1) * P].sum()
+                a /= g
+                old = np.zeros(nb, dtype=np.float64)
+                old[:min(nb, len(st.ema_mass))] = st.ema_mass[:nb]
+                st.ema_mass = 0.9 * old + 0.1 * a
+                observed[(b, h)] = a
+        return out, lse, observed
 
     # -- page scorer -------------------------------------------------------------------
     def quest_scores(self, layer: int, q):

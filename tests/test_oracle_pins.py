@@ -515,3 +515,86 @@ def test_staircase_levels():
     lv = O.staircase_levels(10, (128, 128, 64, 128), 2)
     assert list(lv[:2]) == [16, 16]
     assert list(O.staircase_levels(3, (-1, 0, 0, 0), 0)) == [16, 16, 16]
+
+
+# ---- block attention mass and its running average (Sec. 3.1, Eq. 2) ---------------------------
+def test_block_mass_bruteforce_and_partition_of_unity():
+    """a_b against softmax written out with scalar loops; masses of a stream sum to one; with
+    identical keys a block's mass is its share of the tokens (closed form)."""
+    cfg = small_cfg(n_q_heads=4, n_kv_heads=2, d_k=32, d_v=32, stair_tokens=(64, 64, 0, 0))
+    T = 3 * 64 + 17                                   # exact, 8-bit, centroid blocks and a partial block
+    k, v, q = rand_kv(cfg, T)
+    c = O.GradedCache(cfg)
+    c.append_demote(0, k, v)
+    assert list(c.levels(0, 0, 0)) == [1, 8, 16]
+    _, _, obs = c.decode_attn_observe(0, q)
+    sc = float(np.float32(1.0 / math.sqrt(32)))
+    for h_kv in range(2):
+        a = obs[(0, h_kv)]
+        assert a.shape == (4,)
+        assert abs(a.sum() - 1.0) < 1e-12
+        K, _ = c.reconstruct(c.streams[(0, 0, h_kv)])
+        want = [0.0] * 4
+        for j in range(2):                            # the two query heads of this KV head
+            hq = 2 * h_kv + j
+            logits = [sc * math.fsum(float(q[0, hq, d]) * float(K[t, d]) for d in range(32)) for t in range(T)]
+            m = max(logits)
+            e = [math.exp(x - m) for x in logits]
+            z = math.fsum(e)
+            for t in range(T):
+                want[t // 64] += e[t] / z / 2
+        assert np.max(np.abs(a - np.array(want))) < 1e-13
+    # identical keys -> uniform weights -> mass = tokens of the block / T
+    k2 = np.repeat(k[:, :1], T, axis=1)
+    c2 = O.GradedCache(small_cfg(n_q_heads=4, n_kv_heads=2, d_k=32, d_v=32, stair_tokens=(-1, 0, 0, 0)))
+    c2.append_demote(0, k2, v)
+    _, _, obs2 = c2.decode_attn_observe(0, q)
+    assert np.max(np.abs(obs2[(0, 1)] - np.array([64, 64, 64, 17]) / T)) < 1e-13
+
+
+def test_block_mass_counts_residual_tokens_for_their_block_and_ema_closed_form():
+    cfg = small_cfg(n_q_heads=2, n_kv_heads=1, d_k=32, d_v=32, policy=O.POLICY_RD, rd_budget_bpv=4.0,
+                    residual_fraction=0.05, retire_after=64)
+    T = 4 * 64
+    k, v, q = rand_kv(cfg, T)
+    mass = np.abs(RNG.standard_normal((1, 1, T))).astype(np.float32)
+    mass /= mass.sum()
+    c = O.GradedCache(cfg)
+    c.append_demote(0, k, v, token_mass=mass)
+    st = c.streams[(0, 0, 0)]
+    assert len(st.res_idx) == int(0.05 * T)
+    # the running mass starts from the prefill observer's block masses
+    m0 = st.ema_mass.copy()
+    assert np.allclose(m0, mass[0, 0].reshape(4, 64).sum(axis=1), rtol=1e-6)
+    out, lse, w = c.decode_attn(0, q, None, return_weights=True)
+    _, _, obs = c.decode_attn_observe(0, q)
+    a = obs[(0, 0)]
+    # residual tokens are part of the dense weights, so the block sums need no special case ...
+    want = sum(w[(0, j)].reshape(4, 64).sum(axis=1) for j in range(2)) / 2
+    assert np.max(np.abs(a - want)) < 1e-14
+    # ... and a block's mass includes the weight of its exact residual tokens
+    blk = int(st.res_idx[0]) // 64
+    in_blk = [int(t) for t in st.res_idx if int(t) // 64 == blk]
+    assert a[blk] >= sum(w[(0, 0)][t] + w[(0, 1)][t] for t in in_blk) / 2
+    # n identical observations: m = 0.9^n m0 + (1 - 0.9^n) a
+    for _ in range(4):
+        c.decode_attn_observe(0, q)
+    n = 5
+    assert np.max(np.abs(st.ema_mass - (0.9 ** n * m0 + (1 - 0.9 ** n) * a))) < 1e-13
+
+
+def test_block_mass_of_new_blocks_starts_from_zero():
+    cfg = small_cfg(n_q_heads=2, n_kv_heads=1, d_k=8, d_v=8, stair_tokens=(-1, 0, 0, 0))
+    k, v, q = rand_kv(cfg, 64 + 3)
+    c = O.GradedCache(cfg)
+    c.append_demote(0, k[:, :60], v[:, :60])
+    st = c.streams[(0, 0, 0)]
+    _, _, obs = c.decode_attn_observe(0, q)
+    assert obs[(0, 0)].shape == (1,) and abs(obs[(0, 0)][0] - 1.0) < 1e-13
+    assert abs(st.ema_mass[0] - 0.1) < 1e-15
+    for t in range(60, 67):
+        c.append_demote(0, k[:, t:t + 1], v[:, t:t + 1])
+    _, _, obs = c.decode_attn_observe(0, q)
+    a = obs[(0, 0)]
+    assert a.shape == (2,)
+    assert abs(st.ema_mass[0] - (0.9 * 0.1 + 0.1 * a[0])) < 1e-15 and abs(st.ema_mass[1] - 0.1 * a[1]) < 1e-15
