@@ -133,6 +133,25 @@ GKV_API int gkv_append_demote(gkv_cache* c, int32_t layer, const void* k_new, co
 GKV_API int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_idx, int32_t n_sel,
                     float* out, float* lse, void* stream);
 
+/* gkv_decode_attn over the full context that, in the same pass over the cache, observes the
+ * attention mass of every block (Sec. 3.1, Eq. 2 with this query as the observed one):
+ *   a_b = mean over the KV head's query heads of the summed softmax weight of block b's tokens,
+ * b = 0 .. n_closed - 1 and, when it holds tokens, the partial block as the last entry; tokens
+ * served from the exact residual count for the block they sit in.  The cache's running mass is
+ * then updated, m_b <- 0.9 m_b + 0.1 a_b; it starts from the prompt masses given at bulk ingest
+ * under GKV_POLICY_RD and from 0 otherwise (also for blocks that appear during decode).
+ *   q, out, lse  as for gkv_decode_attn
+ *   block_mass   device fp32 [batch][n_kv_heads][n_items], n_items = blocks that hold tokens
+ *                (ceil(ctx / 64)), or NULL: receives a_b of this call
+ * Grouped-query layout only (GKV_ERR_UNSUPPORTED with v_aliases_k).  Costs one extra small
+ * launch and 64 B of scratch writes per block and stream; the graded cache is read once. */
+GKV_API int gkv_decode_attn_observe(gkv_cache* c, int32_t layer, const void* q, float* out, float* lse,
+                                    float* block_mass, void* stream);
+
+/* Running block masses m_b of `layer` (parity checks; synchronises the device).
+ *   mass_out  HOST fp32 [batch][n_kv_heads][ceil(ctx / 64)] */
+GKV_API int gkv_debug_export_mass(gkv_cache* c, int32_t layer, float* mass_out);
+
 /* Compressed-Quest page selection (Sec. 3.5): score every page of every closed block with the
  * box upper bound sum_d max(q_d * min_d, q_d * max_d), reduce over the KV head's query heads,
  * keep the k = min(budget_tokens / page_tokens, closed pages) best per (sequence, KV head).

@@ -24,6 +24,7 @@ ERR_RANGE, ERR_BUDGET = -6, -7
 
 EXPORTS = [
     "gkv_query_arena_bytes", "gkv_create", "gkv_destroy", "gkv_append_demote", "gkv_decode_attn",
+    "gkv_decode_attn_observe", "gkv_debug_export_mass",
     "gkv_quest_select", "gkv_quest_select_static", "gkv_bits_report", "gkv_debug_export_block", "gkv_debug_export_residual",
     "gkv_debug_export_levels", "gkv_debug_plan_levels", "gkv_ctx_len", "gkv_strerror", "gkv_last_cuda_error",
 ]
@@ -79,12 +80,16 @@ def load():
     lib.gkv_destroy.argtypes = [vp]
     lib.gkv_append_demote.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp]
     lib.gkv_decode_attn.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp]
+    lib.gkv_decode_attn_observe.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    lib.gkv_debug_export_mass.argtypes = [vp, i32, vp]
     lib.gkv_quest_select.argtypes = [vp, i32, vp, i32, vp, C.POINTER(i32), vp]
     lib.gkv_quest_select_static.argtypes = [vp, i32, vp, i32, vp, C.POINTER(i32), vp]
     lib.gkv_bits_report.argtypes = [vp, i32, C.POINTER(GkvBits)]
     lib.gkv_debug_export_block.argtypes = [vp, i32, i32, i32, i32, i32, C.POINTER(i32), vp, vp, vp, vp, C.POINTER(i32)]
     lib.gkv_debug_export_residual.argtypes = [vp, i32, i32, i32, vp, i32, C.POINTER(i32)]
     lib.gkv_debug_export_levels.argtypes = [vp, i32, i32, i32, vp, i32, C.POINTER(i32)]
+    lib.gkv_debug_plan_levels.argtypes = [C.POINTER(GkvConfig), i32, i32, C.POINTER(C.c_float), C.POINTER(C.c_float),
+                                          C.POINTER(C.c_int8), C.POINTER(i32)]
     lib.gkv_ctx_len.argtypes = [vp, i32, C.POINTER(i32)]
     lib.gkv_strerror.argtypes = [C.c_int]
     lib.gkv_strerror.restype = C.c_char_p
@@ -204,6 +209,19 @@ class Cache:
     def gkv_decode_attn(self, layer, q, out, lse=None, page_idx=None, n_sel=0):
         return _check(load().gkv_decode_attn(self.handle, layer, _ptr(q), _ptr(page_idx), n_sel, _ptr(out),
                                              _ptr(lse), _stream()), "gkv_decode_attn")
+
+    def gkv_decode_attn_observe(self, layer, q, out, lse=None, block_mass=None):
+        """Full-context decode that also observes the attention mass of every block and updates the
+        cache's running masses (block_mass: device fp32 [batch][n_kv_heads][ceil(ctx / 64)] or None)."""
+        return _check(load().gkv_decode_attn_observe(self.handle, layer, _ptr(q), _ptr(out), _ptr(lse), _ptr(block_mass),
+                                                     _stream()), "gkv_decode_attn_observe")
+
+    def gkv_debug_export_mass(self, layer):
+        """Running block masses of a layer as a numpy array [batch][n_kv_heads][ceil(ctx / 64)]."""
+        n_items = (self.gkv_ctx_len(layer) + 63) // 64
+        out = np.zeros((self.cfg.batch, self.cfg.n_kv_heads, n_items), dtype=np.float32)
+        _check(load().gkv_debug_export_mass(self.handle, layer, out.ctypes.data_as(C.c_void_p)), "gkv_debug_export_mass")
+        return out
 
     def gkv_quest_select(self, layer, q, budget_tokens, page_idx_out) -> int:
         n = C.c_int32(0)

@@ -98,6 +98,7 @@ struct LayerState {
   uint32_t* res_off_d = nullptr;
   int32_t* res_count_d = nullptr;
   int32_t* res_idx_d = nullptr;         // [n_streams][res_cap]
+  float* ema_d = nullptr;               // running block mass m_b [n_streams][max_blocks + 1] (Sec. 3.1)
   uint16_t* boxes_d = nullptr;
   // accounting of the last read
   int last_mode = 0;                    // 0 none, 1 full, 2 page list
@@ -127,6 +128,9 @@ struct gkv_cache {
   float* scores_d = nullptr;            // residual scores [n_streams][max_ctx] or page scores
   int32_t* kper_d = nullptr;
   int32_t* tickets_d = nullptr;         // per-stream arrival counters of the decode kernel's final merge
+  float2* mass_raw_d = nullptr;         // scratch of an observing decode call: [n_streams][max_blocks + 1][8]
+  float2* res_raw_d = nullptr;          // [n_streams][res_cap][8]
+  float* lse2_d = nullptr;              // [n_streams][8]
   EncodeJob* jobs_d = nullptr;
   size_t jobs_cap = 0;
   // shared pinned staging (jobs | levels | k-per-stream), guarded by ev_stage
@@ -144,8 +148,8 @@ inline uint64_t nval_per_token(const gkv_config& c) { return is_mla(c) ? c.d_k :
 constexpr int kMlaTargetCtas = 148;          // one CTA per SM (213 KB of shared memory, tensor memory)
 
 struct ArenaPlan {
-  size_t status, debug, partial, range, mass, levels, scores, kper, tickets, jobs, per_layer, heap_begin, total_meta;
-  size_t l_table, l_warps, l_units, l_parts, l_resoff, l_rescount, l_residx, l_respool, l_boxes, layer_bytes;
+  size_t status, debug, partial, range, mass, levels, scores, kper, tickets, jobs, mass_raw, res_raw, lse2, per_layer, heap_begin, total_meta;
+  size_t l_table, l_warps, l_units, l_parts, l_resoff, l_rescount, l_residx, l_respool, l_boxes, l_ema, layer_bytes;
 };
 
 struct Derived {
@@ -212,6 +216,11 @@ ArenaPlan plan_arena(const gkv_config& c, const Derived& d) {
   a.kper = take(static_cast<size_t>(d.n_streams) * sizeof(int32_t));
   a.tickets = take(static_cast<size_t>(d.n_streams) * sizeof(int32_t));
   a.jobs = take(static_cast<size_t>(d.n_streams) * d.max_blocks * sizeof(EncodeJob));
+  // block-mass observation (grouped-query layout only)
+  const size_t mass_items = is_mla(c) ? 0 : static_cast<size_t>(d.n_streams) * (d.max_blocks + 1);
+  a.mass_raw = take(mass_items * kMaxHeadsPerKv * sizeof(float2));
+  a.res_raw = take(is_mla(c) ? 0 : static_cast<size_t>(d.n_streams) * d.res_cap * kMaxHeadsPerKv * sizeof(float2));
+  a.lse2 = take(static_cast<size_t>(d.n_streams) * kMaxHeadsPerKv * sizeof(float));
   a.per_layer = off;
   size_t lo = 0;
   auto ltake = [&](size_t bytes) { size_t o = lo; lo = align_up(lo + bytes, 256); return o; };
@@ -224,6 +233,7 @@ ArenaPlan plan_arena(const gkv_config& c, const Derived& d) {
   a.l_residx = ltake(static_cast<size_t>(d.n_streams) * std::max(d.res_cap, 1) * sizeof(int32_t));
   a.l_respool = ltake(static_cast<size_t>(d.n_streams) * d.res_cap * 2 * kRowBytes);
   a.l_boxes = ltake(static_cast<size_t>(d.n_streams) * kD * 2 * d.box_stride * sizeof(uint16_t));
+  a.l_ema = ltake(mass_items * sizeof(float));
   a.layer_bytes = lo;
   a.heap_begin = align_up(a.per_layer + static_cast<size_t>(c.n_layers) * a.layer_bytes, 256);
   a.total_meta = a.heap_begin;
@@ -526,6 +536,10 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
     CK(c, cudaMemcpyAsync(range.data(), c->range_d, range.size() * sizeof(float), cudaMemcpyDeviceToHost, st));
     CK(c, cudaMemcpyAsync(mass.data(), c->mass_d, mass.size() * sizeof(float), cudaMemcpyDeviceToHost, st));
     CK(c, cudaStreamSynchronize(st));
+    // the prefill observer's block masses start the running mass of the decode phase (Sec. 3.1)
+    CK(c, cudaMemcpy2DAsync(L.ema_d, static_cast<size_t>(c->max_blocks + 1) * sizeof(float), c->mass_d,
+                            static_cast<size_t>(n_closed) * sizeof(float), static_cast<size_t>(n_closed) * sizeof(float), ns,
+                            cudaMemcpyDeviceToDevice, st));
     for (int s = 0; s < ns; ++s) {
       const bool miss = rd_allocate(cfg, &mass[static_cast<size_t>(s) * n_closed], &range[static_cast<size_t>(s) * n_closed],
                                     n_closed, n_tail, &L.level[static_cast<size_t>(s) * c->max_blocks]);
@@ -1045,6 +1059,9 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
   c->scores_d = reinterpret_cast<float*>(c->arena + a.scores);
   c->kper_d = reinterpret_cast<int32_t*>(c->arena + a.kper);
   c->tickets_d = reinterpret_cast<int32_t*>(c->arena + a.tickets);
+  c->mass_raw_d = reinterpret_cast<float2*>(c->arena + a.mass_raw);
+  c->res_raw_d = reinterpret_cast<float2*>(c->arena + a.res_raw);
+  c->lse2_d = reinterpret_cast<float*>(c->arena + a.lse2);
   c->jobs_d = reinterpret_cast<EncodeJob*>(c->arena + a.jobs);
   c->jobs_cap = static_cast<size_t>(d.n_streams) * d.max_blocks;
 
@@ -1071,6 +1088,7 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
     L.res_count_d = reinterpret_cast<int32_t*>(lb + a.l_rescount);
     L.res_idx_d = reinterpret_cast<int32_t*>(lb + a.l_residx);
     L.boxes_d = reinterpret_cast<uint16_t*>(lb + a.l_boxes);
+    L.ema_d = reinterpret_cast<float*>(lb + a.l_ema);
     L.level.assign(static_cast<size_t>(d.n_streams) * d.max_blocks, 0);
     L.res_idx.resize(d.n_streams);
     const size_t tb = static_cast<size_t>(d.n_streams) * d.table_stride * sizeof(TableEntry);
@@ -1162,8 +1180,9 @@ int gkv_append_demote(gkv_cache* c, int32_t layer, const void* k_new, const void
                      token_mass, level_plan, st);
 }
 
-int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_idx, int32_t n_sel,
-                    float* out, float* lse, void* stream) {
+namespace {
+int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_idx, int32_t n_sel, float* out, float* lse,
+                bool observe, float* block_mass, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !out) return GKV_ERR_INVALID_ARG;
   if (!page_idx && n_sel != 0) return GKV_ERR_INVALID_ARG;
   LayerState& L = c->layers[layer];
@@ -1172,9 +1191,17 @@ int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* p
   const gkv_config& cfg = c->cfg;
   if (is_mla(cfg)) {
     if (page_idx) return GKV_ERR_BAD_STATE;
+    if (observe) return GKV_ERR_UNSUPPORTED;
     return mla_decode(c, L, q, out, lse, st);
   }
   DecodeParams p{};
+  if (observe) {
+    p.mass_raw = c->mass_raw_d;
+    p.res_raw = c->res_raw_d;
+    p.lse2 = c->lse2_d;
+    p.mass_stride = c->max_blocks + 1;
+    p.res_cap = c->res_cap;
+  }
   p.arena = c->arena;
   p.table = L.table_d;
   p.q = static_cast<const uint16_t*>(q);
@@ -1226,6 +1253,46 @@ int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* p
     L.quest_ran = false;
   }
   CK(c, launch_decode(p, n_ctas, st));
+  if (observe) {
+    MassFinishParams m{};
+    m.mass_raw = c->mass_raw_d;
+    m.res_raw = c->res_raw_d;
+    m.lse2 = c->lse2_d;
+    m.res_idx = L.res_idx_d;
+    m.res_count = L.res_count_d;
+    m.ema = L.ema_d;
+    m.observed = block_mass;
+    m.n_streams = c->n_streams;
+    m.n_items = L.n_closed + (L.n_tail > 0 ? 1 : 0);
+    m.mass_stride = c->max_blocks + 1;
+    m.res_cap = c->res_cap;
+    m.group = c->group;
+    CK(c, launch_mass_finish(m, st));
+  }
+  return GKV_OK;
+}
+}  // namespace
+
+int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_idx, int32_t n_sel,
+                    float* out, float* lse, void* stream) {
+  return decode_impl(c, layer, q, page_idx, n_sel, out, lse, false, nullptr, stream);
+}
+
+int gkv_decode_attn_observe(gkv_cache* c, int32_t layer, const void* q, float* out, float* lse, float* block_mass,
+                            void* stream) {
+  return decode_impl(c, layer, q, nullptr, 0, out, lse, true, block_mass, stream);
+}
+
+int gkv_debug_export_mass(gkv_cache* c, int32_t layer, float* mass_out) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !mass_out) return GKV_ERR_INVALID_ARG;
+  if (is_mla(c->cfg)) return GKV_ERR_UNSUPPORTED;
+  LayerState& L = c->layers[layer];
+  CK(c, cudaDeviceSynchronize());
+  const int n_items = L.n_closed + (L.n_tail > 0 ? 1 : 0);
+  if (n_items == 0) return GKV_OK;
+  CK(c, cudaMemcpy2D(mass_out, static_cast<size_t>(n_items) * sizeof(float), L.ema_d,
+                     static_cast<size_t>(c->max_blocks + 1) * sizeof(float), static_cast<size_t>(n_items) * sizeof(float),
+                     c->n_streams, cudaMemcpyDeviceToHost));
   return GKV_OK;
 }
 

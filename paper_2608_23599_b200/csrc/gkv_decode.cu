@@ -764,7 +764,7 @@ __device__ __forceinline__ void qk_softmax_half(uint32_t half_k, int half, int t
 }
 
 // Process a staged step.  pf carries P fragments from a key step to the following value step.
-template <bool SPARSE>
+template <bool SPARSE, bool MASS>
 __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, int sidx, const uint32_t (&ones)[4],
                                              SoftmaxState& st, uint32_t (&pf)[4]) {
   const DecodeParams& p = *w.p;
@@ -811,6 +811,24 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
       S[0][2] = fmaf(S[0][2], p.scale_log2, b_hi);
       S[0][3] = fmaf(S[0][3], p.scale_log2, b_hi);
       softmax_update<1>(S, st);
+      if constexpr (MASS) {
+        // centroid rows stand for whole blocks and residual rows belong to the block of their token:
+        // their weights are recorded row by row (relative to the running max, which goes with them)
+        if (c.level != 16) {
+          const int c4 = lane & 3;
+          float2* dst = (c.level == 1)
+                            ? p.mass_raw + (static_cast<size_t>(w.stream) * p.mass_stride + c.first) * kMaxHeadsPerKv
+                            : p.res_raw + (static_cast<size_t>(w.stream) * p.res_cap + 16 * (c.first - p.n_closed - 1)) * kMaxHeadsPerKv;
+          if (r < c.ntok) {
+            dst[r * kMaxHeadsPerKv + 2 * c4] = make_float2(st.m0, S[0][0]);
+            dst[r * kMaxHeadsPerKv + 2 * c4 + 1] = make_float2(st.m1, S[0][1]);
+          }
+          if (r + 8 < c.ntok) {
+            dst[(r + 8) * kMaxHeadsPerKv + 2 * c4] = make_float2(st.m0, S[0][2]);
+            dst[(r + 8) * kMaxHeadsPerKv + 2 * c4 + 1] = make_float2(st.m1, S[0][3]);
+          }
+        }
+      }
       make_p_bf16(S[0], pf, st);
     } else {
       // value rows: O^T += V^T P^T with P = hi + lo
@@ -847,8 +865,9 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
   }
 }
 
-template <bool SPARSE>
+template <bool SPARSE, bool MASS>
 __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_kernel(const __grid_constant__ DecodeParams p) {
+  static_assert(!(SPARSE && MASS), "block masses are observed by full reads only");
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gw = blockIdx.x * kDecodeWarps + warp;
@@ -962,6 +981,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   int sidx = 1;
   uint32_t phase = 0;             // bit s = parity to wait for on stage s
   bool failed = false;
+  float mass_l0 = 0.f, mass_l1 = 0.f, mass_m0 = kNegInf, mass_m1 = kNegInf;     // (l, m) when the current block began
   while (have) {
     Cursor nxt = cur;
     const bool more = advance<SPARSE>(w, nxt);
@@ -977,7 +997,30 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
       }
       if (__any_sync(kFull, failed)) break;
       phase ^= 1u << sidx;
-      compute_step<SPARSE>(w, cur, sidx, ones, st, pf);
+      if constexpr (MASS) {
+        if (cur.sub == 0) {
+          mass_l0 = st.l0; mass_l1 = st.l1; mass_m0 = st.m0; mass_m1 = st.m1;
+        }
+      }
+      compute_step<SPARSE, MASS>(w, cur, sidx, ones, st, pf);
+      if constexpr (MASS) {
+        // A block (or the partial block) is done: what it added to the lane's running sums is the
+        // sum now minus the sum at its start brought to the current max.
+        if (cur.sub == cur.nsub - 1 && cur.level != 1 && cur.level != 17) {
+          float d0 = st.l0 - ((mass_m0 == kNegInf) ? 0.f : mass_l0 * fast_exp2(mass_m0 - st.m0));
+          float d1 = st.l1 - ((mass_m1 == kNegInf) ? 0.f : mass_l1 * fast_exp2(mass_m1 - st.m1));
+#pragma unroll
+          for (int d = 4; d <= 16; d <<= 1) {
+            d0 += __shfl_xor_sync(kFull, d0, d);
+            d1 += __shfl_xor_sync(kFull, d1, d);
+          }
+          if (lane < 4) {
+            float2* dst = p.mass_raw + (static_cast<size_t>(w.stream) * p.mass_stride + cur.first) * kMaxHeadsPerKv + 2 * lane;
+            dst[0] = make_float2(st.m0, fmaxf(d0, 0.f));
+            dst[1] = make_float2(st.m1, fmaxf(d1, 0.f));
+          }
+        }
+      }
       __syncwarp();
     }
     cur = nxt;
@@ -1100,6 +1143,9 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
           const size_t hq = static_cast<size_t>(b) * p.n_kv_heads * p.group + static_cast<size_t>(kvh) * p.group + h;
           p.out[hq * kD + ch] = (L > 0.f) ? acc / L : 0.f;
           if (p.lse && ch == 0) p.lse[hq] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : kNegInf;
+          if constexpr (MASS) {
+            if (ch == 0) p.lse2[hq] = (L > 0.f) ? M + log2f(L) : kNegInf;
+          }
         }
       }
       __syncthreads();
@@ -1118,11 +1164,12 @@ size_t decode_smem_bytes() {
 cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(decode_smem_bytes()));
+    const int bytes = static_cast<int>(decode_smem_bytes());
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(decode_smem_bytes()));
+    e = cudaFuncSetAttribute(decode_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(decode_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -1137,8 +1184,54 @@ cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (p.page_idx) return cudaLaunchKernelEx(&cfg, decode_kernel<true>, p);
-  return cudaLaunchKernelEx(&cfg, decode_kernel<false>, p);
+  if (p.page_idx) return cudaLaunchKernelEx(&cfg, decode_kernel<true, false>, p);
+  if (p.mass_raw) return cudaLaunchKernelEx(&cfg, decode_kernel<false, true>, p);
+  return cudaLaunchKernelEx(&cfg, decode_kernel<false, false>, p);
+}
+
+namespace {
+// One thread per (stream, item).  Residual rows are ascending in token index, so the rows of a
+// block are one run found by bisection; everything is summed in a fixed order.
+__global__ void mass_finish_kernel(const MassFinishParams p) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= p.n_streams * p.n_items) return;
+  const int s = idx / p.n_items, b = idx - s * p.n_items;
+  const float* lse2 = p.lse2 + static_cast<size_t>(s) * p.group;
+  const float2* raw = p.mass_raw + (static_cast<size_t>(s) * p.mass_stride + b) * kMaxHeadsPerKv;
+  float a = 0.f;
+  for (int h = 0; h < p.group; ++h) {
+    const float2 v = raw[h];
+    if (v.y > 0.f && lse2[h] != -INFINITY) a += v.y * exp2f(v.x - lse2[h]);
+  }
+  const int n_res = p.res_count ? p.res_count[s] : 0;
+  if (n_res > 0) {
+    const int32_t* ri = p.res_idx + static_cast<size_t>(s) * p.res_cap;
+    int lo = 0, hi = n_res;
+    while (lo < hi) {                                  // first row with token >= 64 b
+      const int mid = (lo + hi) >> 1;
+      if (ri[mid] < b * kBlock) lo = mid + 1;
+      else hi = mid;
+    }
+    for (int i = lo; i < n_res && ri[i] < (b + 1) * kBlock; ++i) {
+      const float2* rr = p.res_raw + (static_cast<size_t>(s) * p.res_cap + i) * kMaxHeadsPerKv;
+      for (int h = 0; h < p.group; ++h) {
+        const float2 v = rr[h];
+        if (v.y > 0.f && lse2[h] != -INFINITY) a += v.y * exp2f(v.x - lse2[h]);
+      }
+    }
+  }
+  a /= static_cast<float>(p.group);
+  float* e = p.ema + static_cast<size_t>(s) * p.mass_stride + b;
+  *e = fmaf(0.9f, *e, 0.1f * a);
+  if (p.observed) p.observed[idx] = a;
+}
+}  // namespace
+
+cudaError_t launch_mass_finish(const MassFinishParams& p, cudaStream_t st) {
+  const int n = p.n_streams * p.n_items;
+  if (n <= 0) return cudaSuccess;
+  mass_finish_kernel<<<(n + 255) / 256, 256, 0, st>>>(p);
+  return cudaGetLastError();
 }
 
 }  // namespace gkv

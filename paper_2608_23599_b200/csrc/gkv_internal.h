@@ -68,6 +68,28 @@ struct DecodeParams {
   int32_t* tickets;             // [n_streams] arrival counters, zero between launches
   float* out;                   // [batch][n_q_heads][128]
   float* lse;                   // nullable
+  // Block attention mass (Sec. 3.1), dense mode, nullable: unnormalised (running max, sum of exp2)
+  // pairs per (stream, item, head), items = blocks 0 .. n_closed (the last is the partial block), and
+  // per (stream, residual row, head); lse2 = log2 of the softmax denominator per query head.
+  float2* mass_raw;             // [n_streams][mass_stride][8]
+  float2* res_raw;              // [n_streams][res_cap][8]
+  float* lse2;                  // [batch][n_q_heads]
+  int32_t mass_stride, res_cap;
+};
+
+// Turns the raw pairs of a decode launch into block masses a_b (mean over the KV head's query heads
+// of the block's softmax weight, residual rows added to the block they sit in) and updates the running
+// mass m_b <- 0.9 m_b + 0.1 a_b.
+struct MassFinishParams {
+  const float2* mass_raw;
+  const float2* res_raw;
+  const float* lse2;
+  const int32_t* res_idx;       // [n_streams][res_cap] ascending token indices of the residual rows
+  const int32_t* res_count;     // [n_streams]
+  float* ema;                   // [n_streams][mass_stride]
+  float* observed;              // nullable [n_streams][n_items]
+  int32_t n_streams, n_items;   // items = n_closed + (n_tail > 0)
+  int32_t mass_stride, res_cap, group;
 };
 
 // One block to encode: read 64 tokens from `src`, write level `dst_level` at dst.
@@ -112,6 +134,7 @@ constexpr uint32_t kStatusRange = 1u;      // a scale or zero saturated
 constexpr uint32_t kStatusInternal = 2u;   // an index check failed inside a kernel
 
 cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st);
+cudaError_t launch_mass_finish(const MassFinishParams& p, cudaStream_t st);
 cudaError_t launch_encode(const EncodeParams& p, cudaStream_t st);
 cudaError_t launch_stats(const StatsParams& p, cudaStream_t st);
 cudaError_t launch_append_rows(uint8_t* arena, const TableEntry* table, int table_stride, int tail_index,

@@ -37,3 +37,10 @@ def test_config_struct_matches_header_size_and_validation():
     small = B.gkv_query_arena_bytes(B.make_config(1, 1, 8, 2, 128, 128, 4096, stair_tokens=(64, 64, 64, 64)))
     large = B.gkv_query_arena_bytes(B.make_config(1, 1, 8, 2, 128, 128, 4096, stair_tokens=(-1, 0, 0, 0)))
     assert small < large
+
+
+def test_every_export_has_declared_argument_types():
+    """Without argtypes ctypes passes Python ints as 32-bit C ints, which truncates device pointers."""
+    lib = B.load()
+    for name in B.EXPORTS:
+        assert getattr(lib, name).argtypes is not None, f"{name}: argtypes not declared in binding.load()"

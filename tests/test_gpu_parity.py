@@ -376,3 +376,116 @@ def test_decode_is_bitwise_reproducible():
         gcache.close()
     for o, l in outs[1:]:
         assert np.array_equal(o, outs[0][0]) and np.array_equal(l, outs[0][1])
+
+
+# ---- block attention mass observed by the decode pass (Sec. 3.1) -------------------------------
+MASS_RTOL, MASS_ATOL = 1e-2, 2e-6     # weights carry the logit error of fp16 operands (about 1e-3 relative)
+
+
+def _observe_both(ocache, gcache, layer, q_bf16):
+    cfg = ocache.cfg
+    dev = gcache.device
+    n_items = (gcache.gkv_ctx_len(layer) + 63) // 64
+    out = torch.empty((cfg.batch, cfg.n_q_heads, cfg.d_v), dtype=torch.float32, device=dev)
+    lse = torch.empty((cfg.batch, cfg.n_q_heads), dtype=torch.float32, device=dev)
+    mass = torch.full((cfg.batch, cfg.n_kv_heads, n_items), -1.0, dtype=torch.float32, device=dev)
+    gcache.gkv_decode_attn_observe(layer, q_bf16.to(dev), out, lse, mass)
+    torch.cuda.synchronize()
+    o_out, o_lse, o_obs = ocache.decode_attn_observe(layer, U.f32(q_bf16))
+    return out, o_out, mass.cpu().numpy().astype(np.float64), o_obs
+
+
+def _assert_mass_close(got, want_by_stream, tag, unit_sum=True):
+    for (b, h), want in want_by_stream.items():
+        g = got[b, h]
+        assert g.shape == want.shape, (tag, g.shape, want.shape)
+        err = np.abs(g - want)
+        bad = err > MASS_RTOL * np.abs(want) + MASS_ATOL
+        assert not bad.any(), (tag, b, h, int(np.argmax(err)), float(err.max()), float(want[np.argmax(err)]))
+        if unit_sum:
+            assert abs(g.sum() - 1.0) < 2e-3, (tag, b, h, float(g.sum()))
+
+
+def _ema_of(ocache, layer):
+    cfg = ocache.cfg
+    return {(b, h): ocache.streams[(layer, b, h)].ema_mass for b in range(cfg.batch) for h in range(cfg.n_kv_heads)}
+
+
+def test_block_mass_all_levels_with_appends():
+    """Config 0 (every rung of the ladder, query groups of 4): the observed block masses and the
+    running masses against the oracle, across appends that grow the partial block, close it and
+    demote blocks; the attention output of the observing call equals the plain call's."""
+    w = W.config(0)
+    ocache, gcache = _pair(w)
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    out, o_out, mass, o_obs = _observe_both(ocache, gcache, 0, data["q"])
+    U.assert_outputs_close(out, o_out, "observe cfg0")
+    _assert_mass_close(mass, o_obs, "cfg0 step -1")
+    plain = torch.empty_like(out)
+    gcache.gkv_decode_attn(0, data["q"].to(dev), plain)
+    torch.cuda.synchronize()
+    assert torch.equal(plain, out)                 # observing does not change the arithmetic of the output
+    for step in range(70):
+        tok = W.make_decode_tokens(w, 0, step, "cpu")
+        ocache.append_demote(0, U.f32(tok["k"]), U.f32(tok["v"]))
+        gcache.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
+        if step in (0, 1, 62, 63, 64, 69):
+            out, o_out, mass, o_obs = _observe_both(ocache, gcache, 0, tok["q"])
+            U.assert_outputs_close(out, o_out, f"observe cfg0 step {step}")
+            _assert_mass_close(mass, o_obs, f"cfg0 step {step}")
+    _assert_mass_close(gcache.gkv_debug_export_mass(0).astype(np.float64), _ema_of(ocache, 0), "cfg0 running mass", unit_sum=False)
+    gcache.close()
+
+
+def test_block_mass_centroid_runs_and_residual_rows():
+    """RD-V2 shape: almost every block a centroid (read as runs of 16 blocks), 10 % of the tokens in
+    the exact residual whose weight counts for their block."""
+    w = W.config(5, "small")
+    ocache, gcache = _pair(w)
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    for step in range(3):
+        q = data["q"] if step == 0 else W.make_decode_tokens(w, 0, step, "cpu")["q"]
+        out, o_out, mass, o_obs = _observe_both(ocache, gcache, 0, q)
+        U.assert_outputs_close(out, o_out, f"observe rdv2 {step}", scale=U.value_scale(data["v"]))
+        _assert_mass_close(mass, o_obs, f"rdv2 {step}")
+        tok = W.make_decode_tokens(w, 0, step, "cpu")
+        ocache.append_demote(0, U.f32(tok["k"]), U.f32(tok["v"]))
+        gcache.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
+    _assert_mass_close(gcache.gkv_debug_export_mass(0).astype(np.float64), _ema_of(ocache, 0), "rdv2 running mass", unit_sum=False)
+    gcache.close()
+
+
+def test_block_mass_query_group_of_8_and_single_block():
+    w = _tiny(40, n_q_heads=16, n_kv_heads=2)
+    ocache, gcache = _pair(w)
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    out, o_out, mass, o_obs = _observe_both(ocache, gcache, 0, data["q"])
+    assert mass.shape[-1] == 1 and np.allclose(mass, 1.0, atol=1e-5)
+    _assert_mass_close(mass, o_obs, "tiny")
+    gcache.close()
+
+
+def test_block_mass_running_average_starts_from_prompt_masses():
+    """RD policy (config 1 structure): the running mass is seeded with the block sums of the prompt
+    masses given at ingest, then follows m <- 0.9 m + 0.1 a."""
+    w = W.config(1, "small")
+    ocache, gcache = _pair(w, n_layers=1)
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    seed = _ema_of(ocache, 0)
+    got0 = gcache.gkv_debug_export_mass(0).astype(np.float64)
+    for (b, h), want in seed.items():
+        assert len(want) == w.ctx // 64 and want.sum() > 0.5
+        assert np.allclose(got0[b, h, :len(want)], want, rtol=1e-6, atol=1e-9)     # the same fp32 block sums
+    for step in range(2):
+        out, o_out, mass, o_obs = _observe_both(ocache, gcache, 0, data["q"])
+        U.assert_outputs_close(out, o_out, f"observe cfg1 {step}", scale=U.value_scale(data["v"]))
+        _assert_mass_close(mass, o_obs, f"cfg1 {step}")
+    _assert_mass_close(gcache.gkv_debug_export_mass(0).astype(np.float64), _ema_of(ocache, 0), "cfg1 running mass",
+                       unit_sum=False)
+    gcache.close()
