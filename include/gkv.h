@@ -148,6 +148,21 @@ GKV_API int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const in
 GKV_API int gkv_decode_attn_observe(gkv_cache* c, int32_t layer, const void* q, float* out, float* lse,
                                     float* block_mass, void* stream);
 
+/* Decode-time re-allocation under GKV_POLICY_RD (Sec. 3.1-3.3): runs the allocator of Eq. 4 again
+ * for every stream of `layer` on the running masses m_b (gkv_decode_attn_observe) and the range
+ * proxies recorded when each block closed, at the budget rd_budget_bpv of the current context.
+ * The temporal constraint of Sec. 3.2 holds: no level rises, sink blocks and the newest
+ * retire_after tokens' blocks stay at 16 bits; blocks whose level falls are requantised from their
+ * current representation.  Reads the masses back to the host, so it synchronises `stream` once;
+ * meant to be called when a block has closed (every 64 tokens), not every step.
+ * May return GKV_ERR_BUDGET / GKV_ERR_RANGE as warnings after completing the work. */
+GKV_API int gkv_rd_reallocate(gkv_cache* c, int32_t layer, void* stream);
+
+/* Host-only (no device work): the plan gkv_rd_reallocate decides for one stream.  mass / range
+ * fp32 [n_closed]; prev int8 [n_closed] current levels; levels int8 [n_closed] out. */
+GKV_API int gkv_debug_replan_levels(const gkv_config* cfg, int32_t n_closed, int32_t n_tail, const float* mass,
+                                    const float* range, const int8_t* prev, int8_t* levels, int32_t* budget_miss);
+
 /* Running block masses m_b of `layer` (parity checks; synchronises the device).
  *   mass_out  HOST fp32 [batch][n_kv_heads][ceil(ctx / 64)] */
 GKV_API int gkv_debug_export_mass(gkv_cache* c, int32_t layer, float* mass_out);

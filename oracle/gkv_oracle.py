@@ -253,6 +253,7 @@ class Stream:
     range_flag: bool = False
     budget_flag: bool = False
     ema_mass: np.ndarray = field(default_factory=lambda: np.zeros(0, np.float64))   # running m_b, one per block (+ partial block)
+    range_b: List[float] = field(default_factory=list)       # fp32 range proxy e_b of every closed block (Sec. 3.3)
 
     @property
     def n_closed(self) -> int:
@@ -494,6 +495,7 @@ class GradedCache:
                                               cfg.rd_budget_bpv, cfg.n_sink_blocks, cfg.retire_after,
                                               None, cfg.monotone_in_age)
             st.budget_flag = bflag
+            st.range_b = [np.float32(x) for x in range_b]
             st.ema_mass = mass_b.astype(np.float64)        # the prefill observer's masses start the running average
         if cfg.residual_fraction > 0 and token_mass is not None:
             vsrc = kk[:, :cfg.d_v] if self.alias else vv
@@ -521,6 +523,8 @@ class GradedCache:
             return
         # the tail block closes: boxes from unquantised keys, block enters at level 16
         self._close_boxes(st, st.tail_k)
+        if cfg.policy == POLICY_RD:
+            st.range_b.append(np.float32(np.max(st.tail_k.max(axis=0) - st.tail_k.min(axis=0))))
         blk, _ = make_block(16, st.tail_k, st.tail_v)
         st.blocks.append(blk)
         st.tail_k = np.zeros((0, cfg.d_k), np.float32)
@@ -530,6 +534,33 @@ class GradedCache:
             for i, blk in enumerate(st.blocks):
                 if target[i] < blk.level:              # monotone: levels only fall (Sec. 3.2)
                     self._demote(st, i, int(target[i]))
+
+    def rd_reallocate(self, layer: int):
+        """Decode-time re-allocation (Sec. 3.1-3.3): the allocator of Eq. 4 run again on the running
+        block masses (rounded to fp32, the precision they are kept in) and the range proxies taken
+        when the blocks closed, at the budget of the current context, under the temporal constraint
+        of Sec. 3.2 - no level rises, sinks and the recent window stay exact.  Blocks whose level
+        falls are requantised from their current reconstruction.  Returns {(b, h): levels}."""
+        cfg = self.cfg
+        plans = {}
+        for b in range(cfg.batch):
+            for h in range(cfg.n_kv_heads):
+                st = self.streams[(layer, b, h)]
+                n = st.n_closed
+                if n == 0:
+                    continue
+                mass = np.zeros(n, dtype=np.float32)
+                mass[:min(n, len(st.ema_mass))] = np.asarray(st.ema_mass[:n], dtype=np.float32)
+                prev = np.array([blk.level for blk in st.blocks], dtype=np.int32)
+                levels, _tau, flag = rd_allocate(mass, np.asarray(st.range_b[:n], dtype=np.float32), cfg.d_k, cfg.d_v,
+                                                 self.alias, st.n_tail, cfg.rd_budget_bpv, cfg.n_sink_blocks,
+                                                 cfg.retire_after, prev, cfg.monotone_in_age)
+                st.budget_flag |= flag
+                for i in range(n):
+                    if levels[i] < st.blocks[i].level:
+                        self._demote(st, i, int(levels[i]))
+                plans[(b, h)] = np.asarray(levels, dtype=np.int32)
+        return plans
 
     def _demote(self, st: Stream, i: int, new_level: int):
         """Requantise block i from its CURRENT reconstruction (the dense data no longer

@@ -24,7 +24,7 @@ ERR_RANGE, ERR_BUDGET = -6, -7
 
 EXPORTS = [
     "gkv_query_arena_bytes", "gkv_create", "gkv_destroy", "gkv_append_demote", "gkv_decode_attn",
-    "gkv_decode_attn_observe", "gkv_debug_export_mass",
+    "gkv_decode_attn_observe", "gkv_debug_export_mass", "gkv_rd_reallocate", "gkv_debug_replan_levels",
     "gkv_quest_select", "gkv_quest_select_static", "gkv_bits_report", "gkv_debug_export_block", "gkv_debug_export_residual",
     "gkv_debug_export_levels", "gkv_debug_plan_levels", "gkv_ctx_len", "gkv_strerror", "gkv_last_cuda_error",
 ]
@@ -82,6 +82,9 @@ def load():
     lib.gkv_decode_attn.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp]
     lib.gkv_decode_attn_observe.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.gkv_debug_export_mass.argtypes = [vp, i32, vp]
+    lib.gkv_rd_reallocate.argtypes = [vp, i32, vp]
+    lib.gkv_debug_replan_levels.argtypes = [C.POINTER(GkvConfig), i32, i32, C.POINTER(C.c_float), C.POINTER(C.c_float),
+                                            C.POINTER(C.c_int8), C.POINTER(C.c_int8), C.POINTER(i32)]
     lib.gkv_quest_select.argtypes = [vp, i32, vp, i32, vp, C.POINTER(i32), vp]
     lib.gkv_quest_select_static.argtypes = [vp, i32, vp, i32, vp, C.POINTER(i32), vp]
     lib.gkv_bits_report.argtypes = [vp, i32, C.POINTER(GkvBits)]
@@ -167,6 +170,21 @@ def gkv_debug_plan_levels(cfg: GkvConfig, n_closed: int, n_tail: int = 0, mass=N
     return levels[:n_closed], bool(miss.value)
 
 
+def gkv_debug_replan_levels(cfg: GkvConfig, n_tail: int, mass, rng, prev):
+    """Host-only plan of a decode-time re-allocation of one stream: (levels int8 [n_closed], budget_miss)."""
+    m = np.ascontiguousarray(mass, dtype=np.float32)
+    r = np.ascontiguousarray(rng, dtype=np.float32)
+    pv = np.ascontiguousarray(prev, dtype=np.int8)
+    n = len(pv)
+    levels = np.zeros(n, dtype=np.int8)
+    miss = C.c_int32(0)
+    fp, bp = C.POINTER(C.c_float), C.POINTER(C.c_int8)
+    _check(load().gkv_debug_replan_levels(C.byref(cfg), n, n_tail, m.ctypes.data_as(fp), r.ctypes.data_as(fp),
+                                          pv.ctypes.data_as(bp), levels.ctypes.data_as(bp), C.byref(miss)),
+           "gkv_debug_replan_levels")
+    return levels, bool(miss.value)
+
+
 class Cache:
     """Owner of a gkv_cache handle and of the torch arena behind it."""
 
@@ -215,6 +233,11 @@ class Cache:
         cache's running masses (block_mass: device fp32 [batch][n_kv_heads][ceil(ctx / 64)] or None)."""
         return _check(load().gkv_decode_attn_observe(self.handle, layer, _ptr(q), _ptr(out), _ptr(lse), _ptr(block_mass),
                                                      _stream()), "gkv_decode_attn_observe")
+
+    def gkv_rd_reallocate(self, layer):
+        """Decode-time re-allocation of an RD-policy layer from the running block masses."""
+        return _check(load().gkv_rd_reallocate(self.handle, layer, _stream()), "gkv_rd_reallocate",
+                      allow=(ERR_RANGE, ERR_BUDGET))
 
     def gkv_debug_export_mass(self, layer):
         """Running block masses of a layer as a numpy array [batch][n_kv_heads][ceil(ctx / 64)]."""

@@ -99,6 +99,7 @@ struct LayerState {
   int32_t* res_count_d = nullptr;
   int32_t* res_idx_d = nullptr;         // [n_streams][res_cap]
   float* ema_d = nullptr;               // running block mass m_b [n_streams][max_blocks + 1] (Sec. 3.1)
+  float* range_d = nullptr;             // RD policy: range proxy e_b of every closed block [n_streams][max_blocks]
   uint16_t* boxes_d = nullptr;
   // accounting of the last read
   int last_mode = 0;                    // 0 none, 1 full, 2 page list
@@ -149,7 +150,7 @@ constexpr int kMlaTargetCtas = 148;          // one CTA per SM (213 KB of shared
 
 struct ArenaPlan {
   size_t status, debug, partial, range, mass, levels, scores, kper, tickets, jobs, mass_raw, res_raw, lse2, per_layer, heap_begin, total_meta;
-  size_t l_table, l_warps, l_units, l_parts, l_resoff, l_rescount, l_residx, l_respool, l_boxes, l_ema, layer_bytes;
+  size_t l_table, l_warps, l_units, l_parts, l_resoff, l_rescount, l_residx, l_respool, l_boxes, l_ema, l_range, layer_bytes;
 };
 
 struct Derived {
@@ -234,6 +235,7 @@ ArenaPlan plan_arena(const gkv_config& c, const Derived& d) {
   a.l_respool = ltake(static_cast<size_t>(d.n_streams) * d.res_cap * 2 * kRowBytes);
   a.l_boxes = ltake(static_cast<size_t>(d.n_streams) * kD * 2 * d.box_stride * sizeof(uint16_t));
   a.l_ema = ltake(mass_items * sizeof(float));
+  a.l_range = ltake(c.policy == GKV_POLICY_RD ? static_cast<size_t>(d.n_streams) * d.max_blocks * sizeof(float) : 0);
   a.layer_bytes = lo;
   a.heap_begin = align_up(a.per_layer + static_cast<size_t>(c.n_layers) * a.layer_bytes, 256);
   a.total_meta = a.heap_begin;
@@ -329,7 +331,8 @@ void rd_levels_for_tau(const std::vector<double>& y, double tau, const std::vect
   }
 }
 
-bool rd_allocate(const gkv_config& c, const float* mass, const float* range, int n, int n_tail, int8_t* out) {
+// prev: nullable current levels; with them no block's level rises (Sec. 3.2: demotion only).
+bool rd_allocate(const gkv_config& c, const float* mass, const float* range, int n, int n_tail, const int8_t* prev, int8_t* out) {
   std::vector<double> y(n);
   std::vector<char> pinned(n, 0);
   const int recent = c.retire_after / kBlock;
@@ -351,7 +354,7 @@ bool rd_allocate(const gkv_config& c, const float* mass, const float* range, int
   cands.erase(std::unique(cands.begin(), cands.end()), cands.end());
   std::vector<int8_t> lv(n);
   auto feasible = [&](double tau) {
-    rd_levels_for_tau(y, tau, pinned, nullptr, c.monotone_in_age != 0, lv);
+    rd_levels_for_tau(y, tau, pinned, prev, c.monotone_in_age != 0, lv);
     long long bits = tail_bits;
     for (int b = 0; b < n; ++b) bits += static_cast<long long>(block_bits(lv[b], nval_tok));
     return bits <= budget_bits;
@@ -368,7 +371,7 @@ bool rd_allocate(const gkv_config& c, const float* mass, const float* range, int
     budget_miss = true;
     lo = cands.size() - 1;
   }
-  rd_levels_for_tau(y, cands[lo], pinned, nullptr, c.monotone_in_age != 0, lv);
+  rd_levels_for_tau(y, cands[lo], pinned, prev, c.monotone_in_age != 0, lv);
   std::memcpy(out, lv.data(), n);
   return budget_miss;
 }
@@ -540,9 +543,12 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
     CK(c, cudaMemcpy2DAsync(L.ema_d, static_cast<size_t>(c->max_blocks + 1) * sizeof(float), c->mass_d,
                             static_cast<size_t>(n_closed) * sizeof(float), static_cast<size_t>(n_closed) * sizeof(float), ns,
                             cudaMemcpyDeviceToDevice, st));
+    CK(c, cudaMemcpy2DAsync(L.range_d, static_cast<size_t>(c->max_blocks) * sizeof(float), c->range_d,
+                            static_cast<size_t>(n_closed) * sizeof(float), static_cast<size_t>(n_closed) * sizeof(float), ns,
+                            cudaMemcpyDeviceToDevice, st));
     for (int s = 0; s < ns; ++s) {
       const bool miss = rd_allocate(cfg, &mass[static_cast<size_t>(s) * n_closed], &range[static_cast<size_t>(s) * n_closed],
-                                    n_closed, n_tail, &L.level[static_cast<size_t>(s) * c->max_blocks]);
+                                    n_closed, n_tail, nullptr, &L.level[static_cast<size_t>(s) * c->max_blocks]);
       if (miss) {
         L.budget_flag = true;
         warn = GKV_ERR_BUDGET;
@@ -650,6 +656,57 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
   return warn;
 }
 
+// Requantise every block whose target level lies below its current one (monotone: levels only
+// fall), each from its current representation, in one encode launch.  target: [n_closed] shared by
+// all streams (stride 0) or [n_streams][stride].
+int demote_to_targets(gkv_cache* c, LayerState& L, const int8_t* target, size_t stride, cudaStream_t st) {
+  const gkv_config& cfg = c->cfg;
+  const int ns = c->n_streams;
+  const size_t table_bytes = static_cast<size_t>(ns) * c->table_stride * sizeof(TableEntry);
+  int rc;
+  if ((rc = wait_event(c, c->ev_stage)) != GKV_OK) return rc;
+  if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
+  EncodeJob* jobs = reinterpret_cast<EncodeJob*>(c->stage_h);
+  size_t n_jobs = 0;
+  std::vector<std::pair<int, uint32_t>> to_free;
+  for (int s = 0; s < ns; ++s)
+    for (int b = 0; b < L.n_closed; ++b) {
+      const int8_t want = target[static_cast<size_t>(s) * stride + b];
+      int8_t& cur = L.level[static_cast<size_t>(s) * c->max_blocks + b];
+      if (want >= cur) continue;                         // monotone: levels only fall
+      TableEntry& e = L.table_h[static_cast<size_t>(s) * c->table_stride + b];
+      uint32_t off;
+      if (!c->heap.alloc(want, &off)) return GKV_ERR_ARENA_TOO_SMALL;
+      EncodeJob& job = jobs[n_jobs++];
+      job.src_off256 = e.off256;
+      job.dst_off256 = off;
+      job.src_level = cur;
+      job.dst_level = want;
+      job.stream = s;
+      job.block = b;
+      job.pad = 0;
+      to_free.emplace_back(cur, e.off256);
+      e.off256 = off;
+      e.level = static_cast<uint32_t>(want);
+      cur = want;
+    }
+  if (n_jobs > 0) {
+    CK(c, cudaMemcpyAsync(c->jobs_d, jobs, n_jobs * sizeof(EncodeJob), cudaMemcpyHostToDevice, st));
+    CK(c, cudaEventRecord(c->ev_stage, st));
+    EncodeParams ep{};
+    ep.arena = c->arena;
+    ep.jobs = c->jobs_d;
+    ep.n_jobs = static_cast<int32_t>(n_jobs);
+    ep.n_kv_heads = cfg.n_kv_heads;
+    ep.status = c->status_d;
+    CK(c, launch_encode(ep, st));
+    for (auto& f : to_free) c->heap.release(f.first, f.second);
+    if ((rc = upload(c, L.table_d, L.table_h, table_bytes, st, L.ev)) != GKV_OK) return rc;
+    L.desc_dirty = true;
+  }
+  return GKV_OK;
+}
+
 int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v_new, cudaStream_t st) {
   const gkv_config& cfg = c->cfg;
   LayerState& L = c->layers[layer];
@@ -677,7 +734,7 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
   // the tail block closes (still level 16, in place): boxes from its unquantised keys, then the
   // staircase moves every block that crossed a rung boundary one or more rungs down
   const int closed_block = L.n_closed;
-  if (cfg.page_tokens > 0) {
+  if (cfg.page_tokens > 0 || cfg.policy == GKV_POLICY_RD) {
     StatsParams sp{};
     sp.arena = c->arena;
     sp.k_in = nullptr;
@@ -691,6 +748,11 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
     sp.page_tokens = cfg.page_tokens;
     sp.boxes = L.boxes_d;
     sp.box_stride = c->box_stride;
+    if (cfg.policy == GKV_POLICY_RD) {       // range proxy of the closing block, kept for later re-allocation
+      sp.block_range = L.range_d;
+      sp.stat_stride = c->max_blocks;
+      sp.stat_base = closed_block;
+    }
     CK(c, launch_stats(sp, st));
   }
   for (int s = 0; s < ns; ++s) L.level[static_cast<size_t>(s) * c->max_blocks + closed_block] = 16;
@@ -702,47 +764,8 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
 
   std::vector<int8_t> target(L.n_closed);
   staircase_levels(cfg, L.n_closed, target.data());
-  if ((rc = wait_event(c, c->ev_stage)) != GKV_OK) return rc;
-  if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
-  EncodeJob* jobs = reinterpret_cast<EncodeJob*>(c->stage_h);
-  size_t n_jobs = 0;
-  std::vector<std::pair<int, uint32_t>> to_free;
-  for (int s = 0; s < ns; ++s)
-    for (int b = 0; b < L.n_closed; ++b) {
-      int8_t& cur = L.level[static_cast<size_t>(s) * c->max_blocks + b];
-      if (target[b] >= cur) continue;                    // monotone: levels only fall
-      TableEntry& e = L.table_h[static_cast<size_t>(s) * c->table_stride + b];
-      uint32_t off;
-      if (!c->heap.alloc(target[b], &off)) return GKV_ERR_ARENA_TOO_SMALL;
-      EncodeJob& job = jobs[n_jobs++];
-      job.src_off256 = e.off256;
-      job.dst_off256 = off;
-      job.src_level = cur;
-      job.dst_level = target[b];
-      job.stream = s;
-      job.block = b;
-      job.pad = 0;
-      to_free.emplace_back(cur, e.off256);
-      e.off256 = off;
-      e.level = static_cast<uint32_t>(target[b]);
-      cur = target[b];
-    }
-  if (n_jobs > 0) {
-    CK(c, cudaMemcpyAsync(c->jobs_d, jobs, n_jobs * sizeof(EncodeJob), cudaMemcpyHostToDevice, st));
-    CK(c, cudaEventRecord(c->ev_stage, st));
-    EncodeParams ep{};
-    ep.arena = c->arena;
-    ep.jobs = c->jobs_d;
-    ep.n_jobs = static_cast<int32_t>(n_jobs);
-    ep.n_kv_heads = cfg.n_kv_heads;
-    ep.status = c->status_d;
-    CK(c, launch_encode(ep, st));
-    for (auto& f : to_free) c->heap.release(f.first, f.second);
-    if ((rc = upload(c, L.table_d, L.table_h, table_bytes, st, L.ev)) != GKV_OK) return rc;
-  }
-  return GKV_OK;
+  return demote_to_targets(c, L, target.data(), 0, st);
 }
-
 
 // ---- latent-attention (MLA) host paths -----------------------------------------------------------
 // One stream per sequence; staircase or external plans only.  The block table, slot heap and
@@ -1089,6 +1112,7 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
     L.res_idx_d = reinterpret_cast<int32_t*>(lb + a.l_residx);
     L.boxes_d = reinterpret_cast<uint16_t*>(lb + a.l_boxes);
     L.ema_d = reinterpret_cast<float*>(lb + a.l_ema);
+    L.range_d = reinterpret_cast<float*>(lb + a.l_range);
     L.level.assign(static_cast<size_t>(d.n_streams) * d.max_blocks, 0);
     L.res_idx.resize(d.n_streams);
     const size_t tb = static_cast<size_t>(d.n_streams) * d.table_stride * sizeof(TableEntry);
@@ -1126,11 +1150,52 @@ int gkv_debug_plan_levels(const gkv_config* cfg, int32_t n_closed, int32_t n_tai
   }
   if (cfg->policy == GKV_POLICY_RD) {
     if (!mass || !range) return GKV_ERR_INVALID_ARG;
-    const bool miss = rd_allocate(*cfg, mass, range, n_closed, n_tail, levels);
+    const bool miss = rd_allocate(*cfg, mass, range, n_closed, n_tail, nullptr, levels);
     if (budget_miss) *budget_miss = miss ? 1 : 0;
     return GKV_OK;
   }
   return GKV_ERR_UNSUPPORTED;      // external plans are the caller's
+}
+
+int gkv_debug_replan_levels(const gkv_config* cfg, int32_t n_closed, int32_t n_tail, const float* mass, const float* range,
+                            const int8_t* prev, int8_t* levels, int32_t* budget_miss) {
+  int rc = validate_config(cfg);
+  if (rc != GKV_OK) return rc;
+  if (cfg->policy != GKV_POLICY_RD) return GKV_ERR_BAD_STATE;
+  if (n_closed <= 0 || n_tail < 0 || n_tail >= kBlock || !mass || !range || !prev || !levels) return GKV_ERR_INVALID_ARG;
+  const bool miss = rd_allocate(*cfg, mass, range, n_closed, n_tail, prev, levels);
+  if (budget_miss) *budget_miss = miss ? 1 : 0;
+  return GKV_OK;
+}
+
+int gkv_rd_reallocate(gkv_cache* c, int32_t layer, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return GKV_ERR_INVALID_ARG;
+  const gkv_config& cfg = c->cfg;
+  if (cfg.policy != GKV_POLICY_RD || is_mla(cfg)) return GKV_ERR_BAD_STATE;
+  LayerState& L = c->layers[layer];
+  const int n = L.n_closed, ns = c->n_streams;
+  if (n == 0) return GKV_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  std::vector<float> mass(static_cast<size_t>(ns) * n), range(static_cast<size_t>(ns) * n);
+  CK(c, cudaMemcpy2DAsync(mass.data(), static_cast<size_t>(n) * sizeof(float), L.ema_d,
+                          static_cast<size_t>(c->max_blocks + 1) * sizeof(float), static_cast<size_t>(n) * sizeof(float), ns,
+                          cudaMemcpyDeviceToHost, st));
+  CK(c, cudaMemcpy2DAsync(range.data(), static_cast<size_t>(n) * sizeof(float), L.range_d,
+                          static_cast<size_t>(c->max_blocks) * sizeof(float), static_cast<size_t>(n) * sizeof(float), ns,
+                          cudaMemcpyDeviceToHost, st));
+  CK(c, cudaStreamSynchronize(st));
+  std::vector<int8_t> target(static_cast<size_t>(ns) * n);
+  int warn = GKV_OK;
+  for (int s = 0; s < ns; ++s) {
+    const bool miss = rd_allocate(cfg, &mass[static_cast<size_t>(s) * n], &range[static_cast<size_t>(s) * n], n, L.n_tail,
+                                  &L.level[static_cast<size_t>(s) * c->max_blocks], &target[static_cast<size_t>(s) * n]);
+    if (miss) {
+      L.budget_flag = true;
+      warn = GKV_ERR_BUDGET;
+    }
+  }
+  const int rc = demote_to_targets(c, L, target.data(), static_cast<size_t>(n), st);
+  return rc != GKV_OK ? rc : warn;
 }
 
 int gkv_destroy(gkv_cache* c) {

@@ -128,6 +128,7 @@ struct StatsParams {
   int32_t box_stride;                // pages (padded)
   float* block_range;                // [n_streams][n_blocks] or nullptr
   float* block_mass;                 // [n_streams][n_blocks] or nullptr
+  int32_t stat_stride, stat_base;    // range / mass land at [stream * stat_stride + stat_base + i]; stride 0 = n_blocks
 };
 
 constexpr uint32_t kStatusRange = 1u;      // a scale or zero saturated

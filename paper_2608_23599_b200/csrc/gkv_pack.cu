@@ -254,13 +254,13 @@ __global__ void __launch_bounds__(kD) stats_kernel(const __grid_constant__ Stats
       if (c < s) red[c] = fmaxf(red[c], red[c + s]);
       __syncthreads();
     }
-    if (c == 0) p.block_range[static_cast<size_t>(stream) * p.n_blocks + bi] = red[0];
+    if (c == 0) p.block_range[static_cast<size_t>(stream) * (p.stat_stride ? p.stat_stride : p.n_blocks) + p.stat_base + bi] = red[0];
   }
   if (p.block_mass && c == 0) {
     const float* m = p.token_mass + static_cast<size_t>(stream) * p.n_tok + static_cast<size_t>(block) * kBlock;
     float acc = 0.f;
     for (int t = 0; t < kBlock; ++t) acc = __fadd_rn(acc, m[t]);
-    p.block_mass[static_cast<size_t>(stream) * p.n_blocks + bi] = acc;
+    p.block_mass[static_cast<size_t>(stream) * (p.stat_stride ? p.stat_stride : p.n_blocks) + p.stat_base + bi] = acc;
   }
 }
 

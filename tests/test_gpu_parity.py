@@ -489,3 +489,61 @@ def test_block_mass_running_average_starts_from_prompt_masses():
     _assert_mass_close(gcache.gkv_debug_export_mass(0).astype(np.float64), _ema_of(ocache, 0), "cfg1 running mass",
                        unit_sum=False)
     gcache.close()
+
+
+def test_decode_time_reallocation_from_running_masses():
+    """RD policy, config 1 structure: observe every decode query, append, and after each block close
+    re-run the allocator on the running masses (gkv_rd_reallocate).
+
+    The level decisions compare masses with thresholds, and the library's masses (fp32, weights at
+    fp16 operand precision) differ from the oracle's (fp64) in the third digit, so a block that sits
+    on a threshold may legitimately land on either side.  What is unique is checked exactly: the
+    decision rule on identical inputs (CPU test of gkv_debug_replan_levels against the oracle), the
+    temporal constraint, the budget, and - with the library's plan replayed as the oracle's demotion
+    plan - every code, scale, zero and centroid plus the attention outputs.  The two plans are also
+    compared directly and may differ in a few blocks only."""
+    import dataclasses
+    w = W.config(1, "small")
+    w = dataclasses.replace(w, max_ctx=w.ctx + 256)
+    ocache, gcache = _pair(w, n_layers=1)
+    ofree = O.GradedCache(U.oracle_config(w, 1))          # the oracle left to its own decisions
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    ofree.append_demote(0, U.f32(data["k"]), U.f32(data["v"]), token_mass=data["mass"].numpy())
+    cfg = ocache.cfg
+    n_changed = 0
+    differ = total = 0
+    for step in range(130):
+        tok = W.make_decode_tokens(w, 0, step, "cpu")
+        out, o_out, mass, o_obs = _observe_both(ocache, gcache, 0, tok["q"])
+        ofree.decode_attn_observe(0, U.f32(tok["q"]))
+        if step % 40 == 0:
+            _assert_mass_close(mass, o_obs, f"realloc step {step}")
+        ocache.append_demote(0, U.f32(tok["k"]), U.f32(tok["v"]))
+        ofree.append_demote(0, U.f32(tok["k"]), U.f32(tok["v"]))
+        gcache.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
+        if gcache.gkv_ctx_len(0) % 64 != 0:
+            continue
+        before = {(b, h): gcache.gkv_debug_export_levels(0, b, h).copy() for b in range(cfg.batch) for h in range(cfg.n_kv_heads)}
+        gcache.gkv_rd_reallocate(0)
+        free_plan = ofree.rd_reallocate(0)
+        recent = w.retire_after // 64
+        for (b, h), old in before.items():
+            new = gcache.gkv_debug_export_levels(0, b, h)
+            n = len(new)
+            assert np.all(new <= old)                                          # no promotion
+            assert all(new[i] == 16 for i in range(n) if n - 1 - i < recent)   # the recent window stays exact
+            differ += int(np.sum(new != free_plan[(b, h)]))
+            total += n
+            for i in np.nonzero(new < old)[0]:
+                ocache.demote_to(0, b, h, int(i), int(new[i]))
+                n_changed += 1
+        U.assert_state_equal(ocache, gcache, 0)
+        rep = gcache.gkv_bits_report(0)
+        assert rep.bpv_paper <= w.rd_budget_bpv + 16 * w.residual_fraction + 1e-6
+        out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, tok["q"])
+        U.assert_outputs_close(out, o_out, f"after reallocation at step {step}", scale=U.value_scale(data["v"]))
+    assert n_changed > 0                       # blocks that left the recent window were given a level
+    assert differ <= max(2, total // 50), (differ, total)
+    gcache.close()

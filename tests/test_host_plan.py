@@ -77,3 +77,36 @@ def test_arena_size_covers_the_worst_case_and_grows_with_context():
         B.gkv_query_arena_bytes(B.make_config(1, 1, 7, 2, 128, 128, 4096))     # heads must divide
     with pytest.raises(B.GkvError):
         B.gkv_query_arena_bytes(B.make_config(1, 1, 8, 2, 96, 96, 4096))       # head dim 128 only
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_decode_time_replan_matches_oracle_and_never_promotes(seed):
+    """The plan of gkv_rd_reallocate (host part) against the oracle's allocator run with the current
+    levels as upper bounds (Sec. 3.2: demotion only), on the plan of an earlier, shorter context."""
+    rng = np.random.default_rng(7000 + seed)
+    n0 = int(rng.integers(8, 200))
+    grow = int(rng.integers(1, 6))
+    n = n0 + grow
+    n_tail = int(rng.integers(0, 64))
+    budget = float(rng.choice([2.5, 4.0, 4.84, 7.0]))
+    retire = int(rng.choice([64, 128, 512]))
+    sinks = int(rng.integers(0, 3))
+    mono = int(seed % 2)
+    mass0 = (rng.random(n0) ** 3 / n0).astype(np.float32)
+    rge = np.exp(rng.normal(1.0, 0.5, size=n)).astype(np.float32)
+    cfg = B.make_config(1, 1, 8, 2, 128, 128, 65536, policy=B.POLICY_RD, rd_budget_bpv=budget, retire_after=retire,
+                        n_sink_blocks=sinks, monotone_in_age=mono)
+    first, _ = B.gkv_debug_plan_levels(cfg, n0, 0, mass0, rge[:n0])
+    # the context grew by `grow` exact blocks and the running masses moved
+    prev = np.concatenate([first, np.full(grow, 16, dtype=np.int8)])
+    mass = np.concatenate([0.6 * mass0 + 0.4 * (rng.random(n0) / n0), rng.random(grow) / n]).astype(np.float32)
+    got, miss = B.gkv_debug_replan_levels(cfg, n_tail, mass, rge, prev)
+    want, _tau, flag = O.rd_allocate(mass, rge, 128, 128, 0, n_tail, budget, sinks, retire, prev.astype(np.int32), mono)
+    assert np.array_equal(got.astype(np.int32), np.asarray(want, dtype=np.int32))
+    assert miss == bool(flag)
+    assert np.all(got <= prev)                                       # no promotion
+    recent = retire // 64
+    assert all(got[i] == 16 for i in range(n) if (i < sinks or n - 1 - i < recent) and prev[i] == 16)
+    if not miss:
+        bits = sum(O.block_bits(int(L), 128, 128, 0) for L in got) + n_tail * 16 * 256
+        assert bits <= np.floor(np.float32(budget) * (n * 64 + n_tail) * 256)

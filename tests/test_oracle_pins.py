@@ -598,3 +598,42 @@ def test_block_mass_of_new_blocks_starts_from_zero():
     a = obs[(0, 0)]
     assert a.shape == (2,)
     assert abs(st.ema_mass[0] - (0.9 * 0.1 + 0.1 * a[0])) < 1e-15 and abs(st.ema_mass[1] - 0.1 * a[1]) < 1e-15
+
+
+def test_decode_time_reallocation_keeps_the_temporal_constraint():
+    """Re-running the allocator on running masses (Sec. 3.1-3.3): no level rises, the recent window
+    and new blocks inside it stay exact, a block leaving the window gets a level, the budget of the
+    grown context holds, and requantisation starts from the block's current representation."""
+    cfg = small_cfg(n_q_heads=2, n_kv_heads=1, d_k=32, d_v=32, policy=O.POLICY_RD, rd_budget_bpv=5.0, retire_after=128,
+                    max_ctx=4096)
+    T = 8 * 64
+    k, v, q = rand_kv(cfg, T + 130)
+    mass = np.abs(RNG.standard_normal((1, 1, T))).astype(np.float32)
+    mass /= mass.sum()
+    c = O.GradedCache(cfg)
+    c.append_demote(0, k[:, :T], v[:, :T], token_mass=mass)
+    st = c.streams[(0, 0, 0)]
+    before = c.levels(0, 0, 0).copy()
+    assert list(before[-2:]) == [16, 16] and len(st.range_b) == 8
+    for t in range(T, T + 130):
+        c.decode_attn_observe(0, q)
+        c.append_demote(0, k[:, t:t + 1], v[:, t:t + 1])
+    assert st.n_closed == 10 and len(st.range_b) == 10
+    mid = c.levels(0, 0, 0).copy()
+    assert np.array_equal(mid[:8], before) and list(mid[8:]) == [16, 16]      # appends alone change nothing under RD
+    recon_before = st.blocks[7].recon_k().copy()
+    plans = c.rd_reallocate(0)
+    after = c.levels(0, 0, 0)
+    assert np.array_equal(after, plans[(0, 0)])
+    assert np.all(after <= mid)
+    assert list(after[-2:]) == [16, 16]                                        # the new recent window
+    assert after[6] < 16 or after[7] < 16 or st.budget_flag                    # blocks that left it were allocated
+    bits = sum(O.block_bits(int(L), 32, 32, False) for L in after) + st.n_tail * 16 * 64
+    assert st.budget_flag or bits <= math.floor(float(np.float32(5.0)) * st.ctx * 64)
+    if after[7] < 16:
+        # block 7 was exact: its new codes quantise those exact rows
+        blk, _ = O.make_block(int(after[7]), k[0, 7 * 64:8 * 64, 0], v[0, 7 * 64:8 * 64, 0])
+        assert np.array_equal(blk.recon_k(), st.blocks[7].recon_k()) and not np.array_equal(recon_before, st.blocks[7].recon_k())
+    # a second run on the same masses changes nothing (the plan is a fixed point)
+    c.rd_reallocate(0)
+    assert np.array_equal(c.levels(0, 0, 0), after)
