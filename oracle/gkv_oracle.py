@@ -203,6 +203,11 @@ class Block:
     k_cent: Optional[np.ndarray] = None      # fp32 [dk] (bf16 values)
     v_cent: Optional[np.ndarray] = None
     history: List[int] = field(default_factory=list)
+    # error bounds carried for the certificate (Sec. 3.6): kappa >= max_j |k_j - k^_j|_2 and
+    # delta >= max_j |v_j - v^_j|_2 against the ORIGINAL rows, vnorm = max_j |v_j|_2 of the originals
+    kappa: float = 0.0
+    delta: float = 0.0
+    vnorm: float = 0.0
 
     def recon_k(self) -> np.ndarray:
         if self.level == 16:
@@ -219,21 +224,36 @@ class Block:
         return dequantize_v_block(self.v_codes, self.v_scale, self.v_zero)
 
 
-def make_block(level: int, xk: np.ndarray, xv: Optional[np.ndarray], history=None) -> Tuple[Block, bool]:
-    """Encode current (fp32) block contents at ``level``.  xv None = values alias keys (MLA)."""
+def _max_row_norm(x) -> float:
+    x = np.asarray(x, dtype=np.float64)
+    return float(np.sqrt((x * x).sum(axis=1)).max())
+
+
+def make_block(level: int, xk: np.ndarray, xv: Optional[np.ndarray], history=None, parent: Optional["Block"] = None
+               ) -> Tuple[Block, bool]:
+    """Encode current (fp32) block contents at ``level``.  xv None = values alias keys (MLA).
+
+    parent = the block these contents were reconstructed from (None: xk / xv are the original
+    rows).  The error bounds of Sec. 3.6 follow the requantisation chain by the triangle
+    inequality: bound(new) = bound(parent) + max_j |x^_parent,j - x^_new,j|_2."""
     hist = list(history or []) + [level]
     flag = False
     if level == 16:
-        return Block(16, k_exact=xk.astype(np.float32), v_exact=None if xv is None else xv.astype(np.float32),
-                     history=hist), flag
-    if level == 1:
-        return Block(1, k_cent=centroid_of(xk), v_cent=None if xv is None else centroid_of(xv), history=hist), flag
-    kc, ks, kz, f1 = quantize_k_block(xk, level)
-    b = Block(level, k_codes=kc, k_scale=ks, k_zero=kz, history=hist)
+        b = Block(16, k_exact=xk.astype(np.float32), v_exact=None if xv is None else xv.astype(np.float32), history=hist)
+    elif level == 1:
+        b = Block(1, k_cent=centroid_of(xk), v_cent=None if xv is None else centroid_of(xv), history=hist)
+    else:
+        kc, ks, kz, f1 = quantize_k_block(xk, level)
+        b = Block(level, k_codes=kc, k_scale=ks, k_zero=kz, history=hist)
+        flag = f1
+        if xv is not None:
+            b.v_codes, b.v_scale, b.v_zero, f2 = quantize_v_block(xv, level)
+            flag = flag or f2
+    b.kappa = (parent.kappa if parent else 0.0) + _max_row_norm(np.asarray(xk, np.float64) - b.recon_k())
     if xv is not None:
-        b.v_codes, b.v_scale, b.v_zero, f2 = quantize_v_block(xv, level)
-        flag = f2
-    return b, (flag or f1)
+        b.delta = (parent.delta if parent else 0.0) + _max_row_norm(np.asarray(xv, np.float64) - b.recon_v())
+        b.vnorm = parent.vnorm if parent else _max_row_norm(xv)
+    return b, flag
 
 
 @dataclass
@@ -569,7 +589,7 @@ class GradedCache:
         assert new_level < old.level, "promotion is forbidden"
         xk = np.asarray(old.recon_k(), dtype=np.float32)
         xv = None if self.alias else np.asarray(old.recon_v(), dtype=np.float32)
-        st.blocks[i], flag = make_block(new_level, xk, xv, old.history)
+        st.blocks[i], flag = make_block(new_level, xk, xv, old.history, parent=old)
         st.range_flag |= flag
 
     def demote_to(self, layer: int, b: int, h: int, block: int, new_level: int):
@@ -676,6 +696,43 @@ class GradedCache:
                 st.ema_mass = 0.9 * old + 0.1 * a
                 observed[(b, h)] = a
         return out, lse, observed
+
+    def certificate(self, layer: int, q):
+        """Attention error certificate of a full-context decode query, per query head (Sec. 3.6,
+        Eq. 9): sum_b a^_b delta_b^v + min(2, M+/M- - M-/M+) max_j |v_j| with
+        M+- = sum_b a^_b exp(+-eps_b).  a^_b is the compressed-cache attention weight of block b's
+        tokens; eps_b = scale |q| kappa_b bounds the logit error of the block's tokens
+        (Cauchy-Schwarz); tokens that are exact (exact blocks, the partial block, residual rows)
+        enter with eps = delta = 0; max_j |v_j| is taken over the original value rows.
+        Returns float64 [B][Hq]."""
+        cfg = self.cfg
+        g = cfg.n_q_heads // cfg.n_kv_heads
+        _, _, weights = self.decode_attn(layer, q, None, return_weights=True)
+        cert = np.zeros((cfg.batch, cfg.n_q_heads), dtype=np.float64)
+        for b in range(cfg.batch):
+            for h in range(cfg.n_kv_heads):
+                st = self.streams[(layer, b, h)]
+                n = st.n_closed
+                exact_tok = np.zeros(st.ctx, dtype=bool)
+                exact_tok[n * P:] = True
+                if len(st.res_idx):
+                    exact_tok[st.res_idx] = True
+                vmax = max([blk.vnorm for blk in st.blocks] + ([_max_row_norm(st.tail_v)] if st.n_tail else [0.0]))
+                for j in range(g):
+                    hq = h * g + j
+                    w = weights[(b, hq)]
+                    qn = float(np.sqrt((np.asarray(q[b, hq], dtype=np.float64) ** 2).sum()))
+                    first = 0.0
+                    m_plus = m_minus = float(w[exact_tok].sum())
+                    for i, blk in enumerate(st.blocks):
+                        sel = ~exact_tok[i * P:(i + 1) * P]
+                        a = float(w[i * P:(i + 1) * P][sel].sum())
+                        eps = self.scale * qn * blk.kappa
+                        first += a * blk.delta
+                        m_plus += a * math.exp(eps)
+                        m_minus += a * math.exp(-eps)
+                    cert[b, hq] = first + min(2.0, m_plus / m_minus - m_minus / m_plus) * vmax
+        return cert
 
     # -- page scorer -------------------------------------------------------------------
     def quest_scores(self, layer: int, q):

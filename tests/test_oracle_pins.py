@@ -637,3 +637,75 @@ def test_decode_time_reallocation_keeps_the_temporal_constraint():
     # a second run on the same masses changes nothing (the plan is a fixed point)
     c.rd_reallocate(0)
     assert np.array_equal(c.levels(0, 0, 0), after)
+
+
+def test_carried_error_bounds_and_runtime_certificate():
+    """The per-block bounds carried through requantisation (Sec. 3.6) really bound the distance to
+    the ORIGINAL rows, equal it for a block encoded once, and the certificate built from them
+    (a) agrees with Eq. 9 evaluated by the stand-alone helper and (b) bounds the true output error
+    against dense attention on the original cache, with demotions and residual rows in play."""
+    cfg = small_cfg(n_q_heads=4, n_kv_heads=2, stair_tokens=(64, 64, 64, 64))
+    T = 5 * 64 + 9
+    k, v, q = rand_kv(cfg, T + 70)
+    c = O.GradedCache(cfg)
+    c.append_demote(0, k[:, :T], v[:, :T])
+    for t in range(T, T + 70):                              # one more block closes: every block moves a rung
+        c.append_demote(0, k[:, t:t + 1], v[:, t:t + 1])
+    dense = O.GradedCache(small_cfg(n_q_heads=4, n_kv_heads=2, stair_tokens=(-1, 0, 0, 0)))
+    dense.append_demote(0, k, v)
+    o_true, _ = dense.decode_attn(0, q)
+    o_hat, _, w_hat = c.decode_attn(0, q, return_weights=True)
+    cert = c.certificate(0, q)
+    for h_kv in range(2):
+        st = c.streams[(0, 0, h_kv)]
+        assert [b.level for b in st.blocks] == [1, 1, 2, 4, 8, 16]
+        for i, blk in enumerate(st.blocks):
+            k0, v0 = k[0, i * 64:(i + 1) * 64, h_kv].astype(np.float64), v[0, i * 64:(i + 1) * 64, h_kv].astype(np.float64)
+            true_k = np.linalg.norm(k0 - blk.recon_k(), axis=1).max()
+            true_v = np.linalg.norm(v0 - blk.recon_v(), axis=1).max()
+            assert true_k <= blk.kappa * (1 + 1e-12) and true_v <= blk.delta * (1 + 1e-12)
+            assert abs(blk.vnorm - np.linalg.norm(v0, axis=1).max()) < 1e-12
+            if len(blk.history) == 1:                     # encoded once from the original rows: the bound is the distance
+                assert abs(true_k - blk.kappa) < 1e-12 and abs(true_v - blk.delta) < 1e-12
+        assert st.blocks[-1].kappa == 0.0 and st.blocks[-1].delta == 0.0
+        assert st.blocks[1].history == [2, 1] and st.blocks[2].history == [4, 2] and st.blocks[1].kappa > 0
+        for j in range(2):
+            hq = 2 * h_kv + j
+            w = w_hat[(0, hq)]
+            n = st.n_closed
+            qn = np.linalg.norm(q[0, hq].astype(np.float64))
+            a_b = [w[i * 64:(i + 1) * 64].sum() for i in range(n)] + [w[n * 64:].sum()]
+            eps_b = [c.scale * qn * blk.kappa for blk in st.blocks] + [0.0]
+            dv_b = [blk.delta for blk in st.blocks] + [0.0]
+            vmax = float(np.linalg.norm(v[0, :, h_kv].astype(np.float64), axis=1).max())
+            want = O.certificate_bound(a_b, eps_b, dv_b, vmax)
+            assert abs(cert[0, hq] - want) < 1e-12 * max(1.0, want)
+            err = float(np.linalg.norm(o_true[0, hq] - o_hat[0, hq]))
+            assert 0 < err <= cert[0, hq]
+
+
+def test_certificate_is_zero_for_an_exact_cache_and_ignores_exact_residual_rows():
+    cfg = small_cfg(n_q_heads=2, n_kv_heads=1, stair_tokens=(-1, 0, 0, 0))
+    k, v, q = rand_kv(cfg, 200)
+    c = O.GradedCache(cfg)
+    c.append_demote(0, k, v)
+    assert np.all(c.certificate(0, q) == 0.0)
+    # residual rows are exact: their weight enters M+ and M- with eps = 0 and adds nothing to the first term
+    cfg2 = small_cfg(n_q_heads=2, n_kv_heads=1, policy=O.POLICY_RD, rd_budget_bpv=3.0, residual_fraction=0.25, retire_after=0)
+    mass = np.abs(RNG.standard_normal((1, 1, 256))).astype(np.float32)
+    k3, v3, q3 = rand_kv(cfg2, 256)
+    c3 = O.GradedCache(cfg2)
+    c3.append_demote(0, k3, v3, token_mass=mass)
+    st = c3.streams[(0, 0, 0)]
+    assert len(st.res_idx) == 64
+    c_with = c3.certificate(0, q3)
+    no_res = O.GradedCache(small_cfg(n_q_heads=2, n_kv_heads=1, policy=O.POLICY_EXTERNAL))
+    no_res.append_demote(0, k3, v3, level_plan=c3.levels(0, 0, 0)[None, None])
+    c_without = no_res.certificate(0, q3)
+    dense = O.GradedCache(small_cfg(n_q_heads=2, n_kv_heads=1, stair_tokens=(-1, 0, 0, 0)))
+    dense.append_demote(0, k3, v3)
+    o_true, _ = dense.decode_attn(0, q3)
+    o_hat, _ = c3.decode_attn(0, q3)
+    for h in range(2):
+        assert np.linalg.norm(o_true[0, h] - o_hat[0, h]) <= c_with[0, h]
+    assert np.all(c_with > 0) and np.all(c_without > 0)
