@@ -143,10 +143,24 @@ GKV_API int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const in
  *   q, out, lse  as for gkv_decode_attn
  *   block_mass   device fp32 [batch][n_kv_heads][n_items], n_items = blocks that hold tokens
  *                (ceil(ctx / 64)), or NULL: receives a_b of this call
- * Grouped-query layout only (GKV_ERR_UNSUPPORTED with v_aliases_k).  Costs one extra small
- * launch and 64 B of scratch writes per block and stream; the graded cache is read once. */
+ *   certificate  device fp32 [batch][n_q_heads], or NULL: the attention error certificate of this
+ *                query (Sec. 3.6, Eq. 9), a bound on |o - o^|_2 between attention over the original
+ *                rows and the output written to `out`:
+ *                  sum_b a^_b delta_b + min(2, M+/M- - M-/M+) max_j |v_j|,  M+- = sum_b a^_b exp(+-eps_b),
+ *                with a^_b the weight of block b's non-exact tokens for this head, eps_b = scale |q|
+ *                kappa_b, and kappa_b / delta_b the bounds on max_j |k_j - k^_j|_2 / max_j |v_j - v^_j|_2
+ *                that the library keeps per block: the distance itself when a block is encoded from
+ *                its original rows, grown by the distance between old and new reconstruction at every
+ *                later demotion (triangle inequality).  Exact tokens (exact blocks, the partial block,
+ *                residual rows) enter with eps = delta = 0; max_j |v_j| is over the original rows.
+ * Grouped-query layout only (GKV_ERR_UNSUPPORTED with v_aliases_k).  Costs one or two extra small
+ * launches and 64 B of scratch writes per block and stream; the graded cache is read once. */
 GKV_API int gkv_decode_attn_observe(gkv_cache* c, int32_t layer, const void* q, float* out, float* lse,
-                                    float* block_mass, void* stream);
+                                    float* block_mass, float* certificate, void* stream);
+
+/* Per-block bounds behind the certificate (parity checks; synchronises the device).
+ *   bounds_out  HOST fp32 [batch][n_kv_heads][n_closed][4]: kappa_b, delta_b, max_j |v_j|, 0 */
+GKV_API int gkv_debug_export_bounds(gkv_cache* c, int32_t layer, float* bounds_out);
 
 /* Decode-time re-allocation under GKV_POLICY_RD (Sec. 3.1-3.3): runs the allocator of Eq. 4 again
  * for every stream of `layer` on the running masses m_b (gkv_decode_attn_observe) and the range

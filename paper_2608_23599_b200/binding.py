@@ -24,7 +24,8 @@ ERR_RANGE, ERR_BUDGET = -6, -7
 
 EXPORTS = [
     "gkv_query_arena_bytes", "gkv_create", "gkv_destroy", "gkv_append_demote", "gkv_decode_attn",
-    "gkv_decode_attn_observe", "gkv_debug_export_mass", "gkv_rd_reallocate", "gkv_debug_replan_levels",
+    "gkv_decode_attn_observe", "gkv_debug_export_mass", "gkv_debug_export_bounds", "gkv_rd_reallocate",
+    "gkv_debug_replan_levels",
     "gkv_quest_select", "gkv_quest_select_static", "gkv_bits_report", "gkv_debug_export_block", "gkv_debug_export_residual",
     "gkv_debug_export_levels", "gkv_debug_plan_levels", "gkv_ctx_len", "gkv_strerror", "gkv_last_cuda_error",
 ]
@@ -80,7 +81,8 @@ def load():
     lib.gkv_destroy.argtypes = [vp]
     lib.gkv_append_demote.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp]
     lib.gkv_decode_attn.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp]
-    lib.gkv_decode_attn_observe.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    lib.gkv_decode_attn_observe.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.gkv_debug_export_bounds.argtypes = [vp, i32, vp]
     lib.gkv_debug_export_mass.argtypes = [vp, i32, vp]
     lib.gkv_rd_reallocate.argtypes = [vp, i32, vp]
     lib.gkv_debug_replan_levels.argtypes = [C.POINTER(GkvConfig), i32, i32, C.POINTER(C.c_float), C.POINTER(C.c_float),
@@ -228,11 +230,19 @@ class Cache:
         return _check(load().gkv_decode_attn(self.handle, layer, _ptr(q), _ptr(page_idx), n_sel, _ptr(out),
                                              _ptr(lse), _stream()), "gkv_decode_attn")
 
-    def gkv_decode_attn_observe(self, layer, q, out, lse=None, block_mass=None):
+    def gkv_decode_attn_observe(self, layer, q, out, lse=None, block_mass=None, certificate=None):
         """Full-context decode that also observes the attention mass of every block and updates the
-        cache's running masses (block_mass: device fp32 [batch][n_kv_heads][ceil(ctx / 64)] or None)."""
+        cache's running masses (block_mass: device fp32 [batch][n_kv_heads][ceil(ctx / 64)] or None;
+        certificate: device fp32 [batch][n_q_heads] or None, the error certificate of this query)."""
         return _check(load().gkv_decode_attn_observe(self.handle, layer, _ptr(q), _ptr(out), _ptr(lse), _ptr(block_mass),
-                                                     _stream()), "gkv_decode_attn_observe")
+                                                     _ptr(certificate), _stream()), "gkv_decode_attn_observe")
+
+    def gkv_debug_export_bounds(self, layer):
+        """Per-block certificate bounds as numpy [batch][n_kv_heads][n_closed][4] (kappa, delta, max |v|, 0)."""
+        n = self.gkv_ctx_len(layer) // 64
+        out = np.zeros((self.cfg.batch, self.cfg.n_kv_heads, n, 4), dtype=np.float32)
+        _check(load().gkv_debug_export_bounds(self.handle, layer, out.ctypes.data_as(C.c_void_p)), "gkv_debug_export_bounds")
+        return out
 
     def gkv_rd_reallocate(self, layer):
         """Decode-time re-allocation of an RD-policy layer from the running block masses."""

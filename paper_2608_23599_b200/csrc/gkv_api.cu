@@ -100,6 +100,7 @@ struct LayerState {
   int32_t* res_idx_d = nullptr;         // [n_streams][res_cap]
   float* ema_d = nullptr;               // running block mass m_b [n_streams][max_blocks + 1] (Sec. 3.1)
   float* range_d = nullptr;             // RD policy: range proxy e_b of every closed block [n_streams][max_blocks]
+  float4* err_d = nullptr;              // error bounds of every closed block for the certificate [n_streams][max_blocks]
   uint16_t* boxes_d = nullptr;
   // accounting of the last read
   int last_mode = 0;                    // 0 none, 1 full, 2 page list
@@ -150,7 +151,7 @@ constexpr int kMlaTargetCtas = 148;          // one CTA per SM (213 KB of shared
 
 struct ArenaPlan {
   size_t status, debug, partial, range, mass, levels, scores, kper, tickets, jobs, mass_raw, res_raw, lse2, per_layer, heap_begin, total_meta;
-  size_t l_table, l_warps, l_units, l_parts, l_resoff, l_rescount, l_residx, l_respool, l_boxes, l_ema, l_range, layer_bytes;
+  size_t l_table, l_warps, l_units, l_parts, l_resoff, l_rescount, l_residx, l_respool, l_boxes, l_ema, l_range, l_err, layer_bytes;
 };
 
 struct Derived {
@@ -236,6 +237,7 @@ ArenaPlan plan_arena(const gkv_config& c, const Derived& d) {
   a.l_boxes = ltake(static_cast<size_t>(d.n_streams) * kD * 2 * d.box_stride * sizeof(uint16_t));
   a.l_ema = ltake(mass_items * sizeof(float));
   a.l_range = ltake(c.policy == GKV_POLICY_RD ? static_cast<size_t>(d.n_streams) * d.max_blocks * sizeof(float) : 0);
+  a.l_err = ltake(is_mla(c) ? 0 : static_cast<size_t>(d.n_streams) * d.max_blocks * sizeof(float4));
   a.layer_bytes = lo;
   a.heap_begin = align_up(a.per_layer + static_cast<size_t>(c.n_layers) * a.layer_bytes, 256);
   a.total_meta = a.heap_begin;
@@ -643,6 +645,8 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
     ep.n_tok = n_new;
     ep.n_kv_heads = cfg.n_kv_heads;
     ep.status = c->status_d;
+    ep.err = L.err_d;
+    ep.err_stride = c->max_blocks;
     CK(c, launch_encode(ep, st));
   }
   CK(c, cudaEventRecord(c->ev_stage, st));
@@ -699,6 +703,8 @@ int demote_to_targets(gkv_cache* c, LayerState& L, const int8_t* target, size_t 
     ep.n_jobs = static_cast<int32_t>(n_jobs);
     ep.n_kv_heads = cfg.n_kv_heads;
     ep.status = c->status_d;
+    ep.err = L.err_d;
+    ep.err_stride = c->max_blocks;
     CK(c, launch_encode(ep, st));
     for (auto& f : to_free) c->heap.release(f.first, f.second);
     if ((rc = upload(c, L.table_d, L.table_h, table_bytes, st, L.ev)) != GKV_OK) return rc;
@@ -734,7 +740,7 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
   // the tail block closes (still level 16, in place): boxes from its unquantised keys, then the
   // staircase moves every block that crossed a rung boundary one or more rungs down
   const int closed_block = L.n_closed;
-  if (cfg.page_tokens > 0 || cfg.policy == GKV_POLICY_RD) {
+  {
     StatsParams sp{};
     sp.arena = c->arena;
     sp.k_in = nullptr;
@@ -748,6 +754,8 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
     sp.page_tokens = cfg.page_tokens;
     sp.boxes = L.boxes_d;
     sp.box_stride = c->box_stride;
+    sp.err = L.err_d;                        // largest value-row norm of the closing block (certificate)
+    sp.err_stride = c->max_blocks;
     if (cfg.policy == GKV_POLICY_RD) {       // range proxy of the closing block, kept for later re-allocation
       sp.block_range = L.range_d;
       sp.stat_stride = c->max_blocks;
@@ -1113,6 +1121,7 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
     L.boxes_d = reinterpret_cast<uint16_t*>(lb + a.l_boxes);
     L.ema_d = reinterpret_cast<float*>(lb + a.l_ema);
     L.range_d = reinterpret_cast<float*>(lb + a.l_range);
+    L.err_d = reinterpret_cast<float4*>(lb + a.l_err);
     L.level.assign(static_cast<size_t>(d.n_streams) * d.max_blocks, 0);
     L.res_idx.resize(d.n_streams);
     const size_t tb = static_cast<size_t>(d.n_streams) * d.table_stride * sizeof(TableEntry);
@@ -1247,7 +1256,7 @@ int gkv_append_demote(gkv_cache* c, int32_t layer, const void* k_new, const void
 
 namespace {
 int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_idx, int32_t n_sel, float* out, float* lse,
-                bool observe, float* block_mass, void* stream) {
+                bool observe, float* block_mass, float* certificate, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !out) return GKV_ERR_INVALID_ARG;
   if (!page_idx && n_sel != 0) return GKV_ERR_INVALID_ARG;
   LayerState& L = c->layers[layer];
@@ -1333,6 +1342,28 @@ int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_
     m.res_cap = c->res_cap;
     m.group = c->group;
     CK(c, launch_mass_finish(m, st));
+    if (certificate) {
+      CertificateParams cp{};
+      cp.arena = c->arena;
+      cp.table = L.table_d;
+      cp.mass_raw = c->mass_raw_d;
+      cp.res_raw = c->res_raw_d;
+      cp.lse2 = c->lse2_d;
+      cp.err = L.err_d;
+      cp.res_count = L.res_count_d;
+      cp.q = static_cast<const uint16_t*>(q);
+      cp.out = certificate;
+      cp.n_streams = c->n_streams;
+      cp.group = c->group;
+      cp.n_closed = L.n_closed;
+      cp.n_tail = L.n_tail;
+      cp.table_stride = c->table_stride;
+      cp.mass_stride = c->max_blocks + 1;
+      cp.res_cap = c->res_cap;
+      cp.err_stride = c->max_blocks;
+      cp.scale = c->scale;
+      CK(c, launch_certificate(cp, st));
+    }
   }
   return GKV_OK;
 }
@@ -1340,12 +1371,24 @@ int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_
 
 int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_idx, int32_t n_sel,
                     float* out, float* lse, void* stream) {
-  return decode_impl(c, layer, q, page_idx, n_sel, out, lse, false, nullptr, stream);
+  return decode_impl(c, layer, q, page_idx, n_sel, out, lse, false, nullptr, nullptr, stream);
 }
 
 int gkv_decode_attn_observe(gkv_cache* c, int32_t layer, const void* q, float* out, float* lse, float* block_mass,
-                            void* stream) {
-  return decode_impl(c, layer, q, nullptr, 0, out, lse, true, block_mass, stream);
+                            float* certificate, void* stream) {
+  return decode_impl(c, layer, q, nullptr, 0, out, lse, true, block_mass, certificate, stream);
+}
+
+int gkv_debug_export_bounds(gkv_cache* c, int32_t layer, float* bounds_out) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !bounds_out) return GKV_ERR_INVALID_ARG;
+  if (is_mla(c->cfg)) return GKV_ERR_UNSUPPORTED;
+  LayerState& L = c->layers[layer];
+  CK(c, cudaDeviceSynchronize());
+  if (L.n_closed == 0) return GKV_OK;
+  CK(c, cudaMemcpy2D(bounds_out, static_cast<size_t>(L.n_closed) * sizeof(float4), L.err_d,
+                     static_cast<size_t>(c->max_blocks) * sizeof(float4), static_cast<size_t>(L.n_closed) * sizeof(float4),
+                     c->n_streams, cudaMemcpyDeviceToHost));
+  return GKV_OK;
 }
 
 int gkv_debug_export_mass(gkv_cache* c, int32_t layer, float* mass_out) {

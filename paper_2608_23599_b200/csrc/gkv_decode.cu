@@ -1227,6 +1227,91 @@ __global__ void mass_finish_kernel(const MassFinishParams p) {
 }
 }  // namespace
 
+namespace {
+// One CTA of 128 threads per query head.  Every sum is taken in a fixed order (a thread's items in
+// ascending order, then a tree over the threads), so the certificate is reproducible bit for bit.
+__global__ void __launch_bounds__(128) certificate_kernel(const CertificateParams p) {
+  __shared__ float red[4][128];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int s = blockIdx.x / p.group, h = blockIdx.x - s * p.group;
+  const int hq = s * p.group + h;
+  // |q|
+  const float qc = __uint_as_float(static_cast<uint32_t>(p.q[static_cast<size_t>(hq) * kD + tid]) << 16);
+  red[0][tid] = qc * qc;
+  __syncthreads();
+  for (int w = 64; w > 0; w >>= 1) {
+    if (tid < w) red[0][tid] += red[0][tid + w];
+    __syncthreads();
+  }
+  const float qn = sqrtf(red[0][0]);
+  __syncthreads();
+  const float lse2 = p.lse2[hq];
+  const int n_items = p.n_closed + (p.n_tail > 0 ? 1 : 0);
+  float first = 0.f, mp = 0.f, mm = 0.f, vmax = 0.f;
+  for (int b = tid; b < n_items; b += 128) {
+    const float2 v = p.mass_raw[(static_cast<size_t>(s) * p.mass_stride + b) * kMaxHeadsPerKv + h];
+    const float a = (v.y > 0.f && lse2 != -INFINITY) ? v.y * exp2f(v.x - lse2) : 0.f;
+    if (b < p.n_closed) {
+      const float4 e = p.err[static_cast<size_t>(s) * p.err_stride + b];
+      const float eps = p.scale * qn * e.x;
+      first = fmaf(a, e.y, first);
+      mp = fmaf(a, expf(eps), mp);
+      mm = fmaf(a, expf(-eps), mm);
+      vmax = fmaxf(vmax, e.z);
+    } else {                                    // the partial block is exact
+      mp += a;
+      mm += a;
+    }
+  }
+  const int n_res = p.res_count ? p.res_count[s] : 0;
+  for (int i = tid; i < n_res; i += 128) {      // residual rows are exact
+    const float2 v = p.res_raw[(static_cast<size_t>(s) * p.res_cap + i) * kMaxHeadsPerKv + h];
+    const float a = (v.y > 0.f && lse2 != -INFINITY) ? v.y * exp2f(v.x - lse2) : 0.f;
+    mp += a;
+    mm += a;
+  }
+  if (p.n_tail > 0) {                           // value rows of the partial block
+    const TableEntry te = p.table[static_cast<size_t>(s) * p.table_stride + p.n_closed];
+    const uint16_t* vrows = reinterpret_cast<const uint16_t*>(p.arena + static_cast<size_t>(te.off256) * 256) + kBlock * kD;
+    for (int t = warp; t < p.n_tail; t += 4) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(vrows + t * kD + 4 * lane);
+      const float x0 = __uint_as_float(raw.x << 16), x1 = __uint_as_float(raw.x & 0xffff0000u);
+      const float x2 = __uint_as_float(raw.y << 16), x3 = __uint_as_float(raw.y & 0xffff0000u);
+      float n2 = fmaf(x0, x0, fmaf(x1, x1, fmaf(x2, x2, x3 * x3)));
+      for (int d = 1; d <= 16; d <<= 1) n2 += __shfl_xor_sync(kFull, n2, d);
+      vmax = fmaxf(vmax, sqrtf(n2));
+    }
+  }
+  red[0][tid] = first;
+  red[1][tid] = mp;
+  red[2][tid] = mm;
+  red[3][tid] = vmax;
+  __syncthreads();
+  for (int w = 64; w > 0; w >>= 1) {
+    if (tid < w) {
+      red[0][tid] += red[0][tid + w];
+      red[1][tid] += red[1][tid + w];
+      red[2][tid] += red[2][tid + w];
+      red[3][tid] = fmaxf(red[3][tid], red[3][tid + w]);
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    const float Mp = red[1][0], Mm = red[2][0];
+    float second = 0.f;
+    if (Mm > 0.f && Mp > 0.f) second = fminf(2.f, fmaxf(0.f, Mp / Mm - Mm / Mp));
+    p.out[hq] = red[0][0] + second * red[3][0];
+  }
+}
+}  // namespace
+
+cudaError_t launch_certificate(const CertificateParams& p, cudaStream_t st) {
+  const int n = p.n_streams * p.group;
+  if (n <= 0) return cudaSuccess;
+  certificate_kernel<<<n, 128, 0, st>>>(p);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_mass_finish(const MassFinishParams& p, cudaStream_t st) {
   const int n = p.n_streams * p.n_items;
   if (n <= 0) return cudaSuccess;

@@ -77,6 +77,22 @@ struct DecodeParams {
   int32_t mass_stride, res_cap;
 };
 
+// Attention error certificate of the observing decode launch that just ran (Sec. 3.6, Eq. 9).
+struct CertificateParams {
+  const uint8_t* arena;
+  const TableEntry* table;
+  const float2* mass_raw;
+  const float2* res_raw;
+  const float* lse2;
+  const float4* err;            // [n_streams][err_stride]
+  const int32_t* res_count;
+  const uint16_t* q;            // bf16 [batch][n_q_heads][128]
+  float* out;                   // [batch][n_q_heads]
+  int32_t n_streams, group, n_closed, n_tail;
+  int32_t table_stride, mass_stride, res_cap, err_stride;
+  float scale;                  // softmax scale (natural-log domain)
+};
+
 // Turns the raw pairs of a decode launch into block masses a_b (mean over the KV head's query heads
 // of the block's softmax weight, residual rows added to the block they sit in) and updates the running
 // mass m_b <- 0.9 m_b + 0.1 a_b.
@@ -111,6 +127,10 @@ struct EncodeParams {
   const uint16_t* v_in;
   int32_t n_tok, n_kv_heads;
   uint32_t* status;
+  // Error bounds for the certificate (Sec. 3.6), nullable: per (stream, block) x = bound on
+  // max_j |k_j - k^_j|, y = the same for values, z = max_j |v_j| of the original rows.
+  float4* err;            // [n_streams][err_stride]
+  int32_t err_stride;
 };
 
 // Statistics of freshly closed blocks: page boxes, key range proxy, block mass.
@@ -129,6 +149,8 @@ struct StatsParams {
   float* block_range;                // [n_streams][n_blocks] or nullptr
   float* block_mass;                 // [n_streams][n_blocks] or nullptr
   int32_t stat_stride, stat_base;    // range / mass land at [stream * stat_stride + stat_base + i]; stride 0 = n_blocks
+  float4* err;                       // nullable; with k_in == nullptr: (0, 0, max_j |v_j|, 0) of the block's exact rows
+  int32_t err_stride;
 };
 
 constexpr uint32_t kStatusRange = 1u;      // a scale or zero saturated
@@ -136,6 +158,7 @@ constexpr uint32_t kStatusInternal = 2u;   // an index check failed inside a ker
 
 cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st);
 cudaError_t launch_mass_finish(const MassFinishParams& p, cudaStream_t st);
+cudaError_t launch_certificate(const CertificateParams& p, cudaStream_t st);
 cudaError_t launch_encode(const EncodeParams& p, cudaStream_t st);
 cudaError_t launch_stats(const StatsParams& p, cudaStream_t st);
 cudaError_t launch_append_rows(uint8_t* arena, const TableEntry* table, int table_stride, int tail_index,

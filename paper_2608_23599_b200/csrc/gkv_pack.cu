@@ -140,11 +140,17 @@ __global__ void __launch_bounds__(256) encode_kernel(const __grid_constant__ Enc
   extern __shared__ __align__(16) uint8_t esm[];
   float* tile = reinterpret_cast<float*>(esm);                       // [64][kTileLd]
   uint8_t* codes = esm + kBlock * kTileLd * sizeof(float);           // [64][128]
+  float* ps = reinterpret_cast<float*>(codes + kBlock * kD);         // [256] scales (or the centroid row) of the tensor
+  float* pz = ps + 256;                                              // [256] zero points
+  float* red = pz + 256;                                             // [16] per-warp maxima
   const int tid = threadIdx.x;
   for (int j = blockIdx.x; j < p.n_jobs; j += gridDim.x) {
     const EncodeJob job = p.jobs[j];
     uint8_t* dst = p.arena + static_cast<size_t>(job.dst_off256) * 256;
     const int L = job.dst_level;
+    const bool from_original = job.src_level == 0 || job.src_level == 16;
+    float4 bound = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (p.err && !from_original && tid == 0) bound = p.err[static_cast<size_t>(job.stream) * p.err_stride + job.block];
     for (int tensor = 0; tensor < 2; ++tensor) {
       const bool is_v = tensor == 1;
       __syncthreads();
@@ -159,7 +165,9 @@ __global__ void __launch_bounds__(256) encode_kernel(const __grid_constant__ Enc
           float acc = 0.f;
           for (int t = 0; t < kBlock; ++t) acc = __fadd_rn(acc, tile[t * kTileLd + tid]);
           uint16_t* row = reinterpret_cast<uint16_t*>(dst + (is_v ? kRowBytes : 0));
-          row[tid] = f32_to_bf16_bits(__fmul_rn(acc, 1.0f / kBlock));
+          const uint16_t cb = f32_to_bf16_bits(__fmul_rn(acc, 1.0f / kBlock));
+          row[tid] = cb;
+          ps[tid] = bf16_bits_to_f32(cb);
         }
       } else {
         const float qmax = static_cast<float>((1 << L) - 1);
@@ -183,6 +191,8 @@ __global__ void __launch_bounds__(256) encode_kernel(const __grid_constant__ Enc
           const int idx = kp_index(c);
           kp[idx] = q.s_bits;
           kp[idx + 2] = q.z_bits;
+          ps[tid] = s32;                 // index = half * 128 + channel
+          pz[tid] = z32;
         } else {
           // values: group = 1 token x 32 channels; thread = (token, group)
           const int t = tid >> 2, g = tid & 3;
@@ -201,12 +211,62 @@ __global__ void __launch_bounds__(256) encode_kernel(const __grid_constant__ Enc
           uint16_t* vp = reinterpret_cast<uint16_t*>(dst + (t >> 5) * half_bytes(L) + off_vp(L, (t >> 4) & 1));
           vp[vp_scale_index(t & 15, g)] = q.s_bits;
           vp[vp_zero_index(t & 15, g)] = q.z_bits;
+          ps[tid] = s32;                 // index = token * 4 + group
+          pz[tid] = z32;
         }
         if (range) atomicOr(p.status, kStatusRange);
         __syncthreads();
         pack_codes(dst, codes, L, is_v);
       }
+      if (p.err) {
+        // Distance of the new representation from what it was made of: per token the 2-norm over
+        // the channels (thread = token x 32-channel quarter, fixed summation order), then the
+        // largest token.  The bound against the original rows grows by it (triangle inequality);
+        // for a block made from its original rows it is the distance itself.
+        __syncthreads();
+        const int t = tid >> 2, g = tid & 3;
+        float d2 = 0.f, n2 = 0.f;
+        for (int c = 32 * g; c < 32 * g + 32; ++c) {
+          const float x = tile[t * kTileLd + c];
+          float xh = x;
+          if (L == 1) xh = ps[c];
+          else if (L != 16) {
+            const int pi = is_v ? t * 4 + g : (t >> 5) * kD + c;
+            xh = __fmaf_rn(static_cast<float>(codes[t * kD + c]), ps[pi], pz[pi]);
+          }
+          const float d = x - xh;
+          d2 = fmaf(d, d, d2);
+          n2 = fmaf(x, x, n2);
+        }
+        d2 += __shfl_xor_sync(0xffffffffu, d2, 1);
+        d2 += __shfl_xor_sync(0xffffffffu, d2, 2);
+        n2 += __shfl_xor_sync(0xffffffffu, n2, 1);
+        n2 += __shfl_xor_sync(0xffffffffu, n2, 2);
+#pragma unroll
+        for (int s = 4; s <= 16; s <<= 1) {
+          d2 = fmaxf(d2, __shfl_xor_sync(0xffffffffu, d2, s));
+          n2 = fmaxf(n2, __shfl_xor_sync(0xffffffffu, n2, s));
+        }
+        if ((tid & 31) == 0) {
+          red[tid >> 5] = d2;
+          red[8 + (tid >> 5)] = n2;
+        }
+        __syncthreads();
+        if (tid == 0) {
+          float dm = red[0], nm = red[8];
+          for (int w = 1; w < 8; ++w) {
+            dm = fmaxf(dm, red[w]);
+            nm = fmaxf(nm, red[8 + w]);
+          }
+          if (!is_v) bound.x += sqrtf(dm);
+          else {
+            bound.y += sqrtf(dm);
+            if (from_original) bound.z = sqrtf(nm);
+          }
+        }
+      }
     }
+    if (p.err && tid == 0) p.err[static_cast<size_t>(job.stream) * p.err_stride + job.block] = bound;
   }
 }
 
@@ -261,6 +321,29 @@ __global__ void __launch_bounds__(kD) stats_kernel(const __grid_constant__ Stats
     float acc = 0.f;
     for (int t = 0; t < kBlock; ++t) acc = __fadd_rn(acc, m[t]);
     p.block_mass[static_cast<size_t>(stream) * (p.stat_stride ? p.stat_stride : p.n_blocks) + p.stat_base + bi] = acc;
+  }
+  if (p.err && !p.k_in) {
+    // a block that closes in place (exact rows): no error yet, largest value-row norm for the
+    // certificate.  Warp w takes tokens w, w + 4, ...; a lane sums four channels.
+    __shared__ float vred[kD / 32];
+    const uint16_t* vrows = rows + kBlock * kD;
+    const int warp = c >> 5, lane = c & 31;
+    float best = 0.f;
+    for (int t = warp; t < kBlock; t += kD / 32) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(vrows + t * kD + 4 * lane);
+      const float x0 = bf16_bits_to_f32(static_cast<uint16_t>(raw.x & 0xffffu)), x1 = bf16_bits_to_f32(static_cast<uint16_t>(raw.x >> 16));
+      const float x2 = bf16_bits_to_f32(static_cast<uint16_t>(raw.y & 0xffffu)), x3 = bf16_bits_to_f32(static_cast<uint16_t>(raw.y >> 16));
+      float n2 = fmaf(x0, x0, fmaf(x1, x1, fmaf(x2, x2, x3 * x3)));
+      for (int s = 1; s <= 16; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
+      best = fmaxf(best, n2);
+    }
+    if (lane == 0) vred[warp] = best;
+    __syncthreads();
+    if (c == 0) {
+      float m = vred[0];
+      for (int w = 1; w < kD / 32; ++w) m = fmaxf(m, vred[w]);
+      p.err[static_cast<size_t>(stream) * p.err_stride + block] = make_float4(0.f, 0.f, sqrtf(m), 0.f);
+    }
   }
 }
 
@@ -380,7 +463,7 @@ __global__ void __launch_bounds__(256) export_kernel(const uint8_t* arena, uint3
 
 cudaError_t launch_encode(const EncodeParams& p, cudaStream_t st) {
   if (p.n_jobs <= 0) return cudaSuccess;
-  const size_t smem = kBlock * kTileLd * sizeof(float) + kBlock * kD;
+  const size_t smem = kBlock * kTileLd * sizeof(float) + kBlock * kD + (256 + 256 + 16) * sizeof(float);
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(encode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));

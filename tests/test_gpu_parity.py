@@ -547,3 +547,89 @@ def test_decode_time_reallocation_from_running_masses():
     assert n_changed > 0                       # blocks that left the recent window were given a level
     assert differ <= max(2, total // 50), (differ, total)
     gcache.close()
+
+
+# ---- attention error certificate as a runtime output (Sec. 3.6, Eq. 9) ---------------------------
+def _bounds_of(ocache, layer):
+    cfg = ocache.cfg
+    out = {}
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            blocks = ocache.streams[(layer, b, h)].blocks
+            out[(b, h)] = np.array([[blk.kappa, blk.delta, blk.vnorm] for blk in blocks], dtype=np.float64).reshape(-1, 3)
+    return out
+
+
+def _check_bounds_and_certificate(w, ocache, gcache, dense, q_bf16, tag, scale=None):
+    cfg = ocache.cfg
+    dev = gcache.device
+    got = gcache.gkv_debug_export_bounds(0).astype(np.float64)
+    for (b, h), want in _bounds_of(ocache, 0).items():
+        g = got[b, h, :, :3]
+        assert g.shape == want.shape, (tag, g.shape, want.shape)
+        assert np.allclose(g, want, rtol=3e-5, atol=1e-6), (tag, b, h, float(np.abs(g - want).max()))
+        assert np.all(got[b, h, :, 3] == 0)
+    out = torch.empty((cfg.batch, cfg.n_q_heads, cfg.d_v), dtype=torch.float32, device=dev)
+    cert = torch.full((cfg.batch, cfg.n_q_heads), -1.0, dtype=torch.float32, device=dev)
+    gcache.gkv_decode_attn_observe(0, q_bf16.to(dev), out, None, None, cert)
+    torch.cuda.synchronize()
+    cert = cert.cpu().numpy().astype(np.float64)
+    want = ocache.certificate(0, U.f32(q_bf16))
+    # the weights behind the certificate carry the kernel's logit error (about 1e-3 relative)
+    assert np.allclose(cert, want, rtol=1e-2, atol=1e-5), (tag, float(np.abs(cert - want).max()), float(want.max()))
+    o_true, _ = dense.decode_attn(0, U.f32(q_bf16))
+    err = np.linalg.norm(o_true - out.cpu().numpy().astype(np.float64), axis=-1)
+    assert np.all(err <= cert * (1 + 1e-3) + 1e-4), (tag, float((err - cert).max()))
+    return cert, err
+
+
+def test_certificate_all_levels_with_demotions():
+    """Config 0: bounds of blocks encoded at ingest, then carried through a chain of demotions at
+    decode time; the certificate against the oracle's and against the true error of the library's
+    output with respect to attention over the original rows."""
+    import dataclasses
+    w = W.config(0)
+    ocache, gcache = _pair(w)
+    dense = O.GradedCache(U.oracle_config(dataclasses.replace(w, stair_tokens=(-1, 0, 0, 0))))
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    dense.append_demote(0, U.f32(data["k"]), U.f32(data["v"]))
+    cert, err = _check_bounds_and_certificate(w, ocache, gcache, dense, data["q"], "cfg0 ingest")
+    assert np.all(cert > 0) and np.all(err > 0)
+    for step in range(66):
+        tok = W.make_decode_tokens(w, 0, step, "cpu")
+        ocache.append_demote(0, U.f32(tok["k"]), U.f32(tok["v"]))
+        dense.append_demote(0, U.f32(tok["k"]), U.f32(tok["v"]))
+        gcache.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
+        if step in (5, 63, 65):
+            _check_bounds_and_certificate(w, ocache, gcache, dense, tok["q"], f"cfg0 step {step}")
+    hist = [len(b.history) for b in ocache.streams[(0, 0, 0)].blocks]
+    assert max(hist) >= 2                                   # some bounds were carried through a requantisation
+    gcache.close()
+
+
+def test_certificate_with_centroids_and_residual_rows():
+    import dataclasses
+    w = W.config(5, "small")
+    ocache, gcache = _pair(w)
+    dense = O.GradedCache(U.oracle_config(dataclasses.replace(w, stair_tokens=(-1, 0, 0, 0), residual_fraction=0.0)))
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    dense.append_demote(0, U.f32(data["k"]), U.f32(data["v"]))
+    _check_bounds_and_certificate(w, ocache, gcache, dense, data["q"], "rdv2")
+    gcache.close()
+
+
+def test_certificate_of_an_exact_cache_is_zero():
+    w = _tiny(300)
+    ocache, gcache = _pair(w)
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    dev = gcache.device
+    out = torch.empty((1, 8, 128), dtype=torch.float32, device=dev)
+    cert = torch.full((1, 8), -1.0, dtype=torch.float32, device=dev)
+    gcache.gkv_decode_attn_observe(0, data["q"].to(dev), out, None, None, cert)
+    torch.cuda.synchronize()
+    assert torch.all(cert == 0)
+    gcache.close()
