@@ -20,7 +20,8 @@ using namespace gkv;
 namespace {
 
 constexpr int kTargetWarps = 148 * kDecodeCtasPerSm * kDecodeWarps;   // one resident wave of CTAs
-constexpr int kSparseWarpsPerStream = kDecodeWarps;   // page-list reads: one CTA per stream
+// Page-list reads: a stream's pages are split over whole CTAs, as many as fill the GPU once (at most 8)
+int sparse_ctas_per_stream(int n_streams) { return std::max(1, std::min(8, 148 / std::max(n_streams, 1))); }
 constexpr size_t kMinWarpCost = 1000;     // do not split below about one block per warp
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -193,7 +194,7 @@ Derived derive(const gkv_config& c) {
   d.max_blocks = (c.max_ctx + kBlock - 1) / kBlock;
   d.table_stride = d.max_blocks + 2;
   d.max_warps = static_cast<int>(align_up(kTargetWarps + 2 * d.n_streams, kDecodeWarps));
-  d.max_warps = std::max(d.max_warps, static_cast<int>(align_up(d.n_streams * kSparseWarpsPerStream, kDecodeWarps)));
+  d.max_warps = std::max(d.max_warps, d.n_streams * sparse_ctas_per_stream(d.n_streams) * kDecodeWarps);
   d.res_cap = c.residual_fraction > 0.f
                   ? static_cast<int>(align_up(static_cast<size_t>(std::floor(static_cast<double>(c.residual_fraction) * c.max_ctx)) + 16, 16))
                   : 0;
@@ -1301,8 +1302,8 @@ int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_
     p.page_idx = page_idx;
     p.n_sel = n_sel;
     p.page_tokens = cfg.page_tokens;
-    p.warps_per_stream = kSparseWarpsPerStream;
-    p.n_warps = c->n_streams * kSparseWarpsPerStream;
+    p.warps_per_stream = sparse_ctas_per_stream(c->n_streams) * kDecodeWarps;
+    p.n_warps = c->n_streams * p.warps_per_stream;
     p.warps = nullptr;
     p.parts = nullptr;
     n_ctas = (p.n_warps + kDecodeWarps - 1) / kDecodeWarps;

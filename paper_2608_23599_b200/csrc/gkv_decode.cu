@@ -897,7 +897,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
       first = static_cast<int>((static_cast<long long>(wi) * p.n_sel) / wps);
       w.item_end = static_cast<int>((static_cast<long long>(wi + 1) * p.n_sel) / wps);
       w.has_tail = (wi == wps - 1);
-      partial_row = blockIdx.x;      // kDecodeWarps warps per stream: one CTA, one partial row
+      partial_row = blockIdx.x;      // whole CTAs per stream: one partial row per CTA
     }
   }
   // per-warp (stream, partial row) for the merge at the end
@@ -1105,7 +1105,9 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
       __threadfence();
       __syncthreads();
       if (threadIdx.x == 0) {
-        int begin = sid, end = sid + 1;
+        // sparse mode: a stream's CTAs are neighbours, one partial row each (row = CTA index)
+        const int per = p.warps_per_stream / kDecodeWarps;
+        int begin = sid * per, end = begin + per;
         if (p.parts) {
           begin = p.parts[sid].begin;
           end = p.parts[sid].end;

@@ -16,54 +16,86 @@ namespace {
 
 constexpr float kNegInfQ = -__builtin_huge_valf();
 
-__global__ void __launch_bounds__(128) quest_score_kernel(const uint16_t* __restrict__ boxes, int box_stride,
-                                                          int n_pages, const uint16_t* __restrict__ q,
-                                                          int n_kv_heads, int group, int reduce,
-                                                          float* __restrict__ scores, int score_stride) {
-  __shared__ float qs[kMaxHeadsPerKv][kD];
-  const int stream = blockIdx.y;
+// One CTA scores kQPages consecutive pages of one stream.  The 256 box rows of the stream (channel x
+// min|max, kQPages * 2 bytes of each) are streamed through shared memory in chunks of kQRows rows
+// with 16-byte cp.async copies, kQStages chunks in flight, so that the loads are wide, contiguous
+// and deep while every thread still adds its pages' channels strictly in order.
+constexpr int kQThreads = 128, kQPages = kQThreads;          // one page per thread
+constexpr int kQRows = 32;                                   // rows per chunk = 16 channels x (min, max)
+constexpr int kQStages = 4;
+constexpr int kQRowBytes = kQPages * 2;                      // 256
+constexpr int kQChunkBytes = kQRows * kQRowBytes;            // 8 KiB
+constexpr int kQPieces = kQRowBytes / 16;                    // 16-byte pieces per row
+constexpr int kQChunks = 2 * kD / kQRows;                    // 8
+
+__device__ __forceinline__ void q_cp_async16(uint32_t dst, const void* src, bool on) {
+  const uint32_t n = on ? 16u : 0u;                          // 0 source bytes: the 16 bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+
+// GROUP = query heads per KV head, a compile-time bound: a run-time bound would leave the unused
+// heads' instructions in the loop, predicated off but still issued.
+template <int GROUP>
+__global__ void __launch_bounds__(kQThreads) quest_score_kernel(const uint16_t* __restrict__ boxes, int box_stride,
+                                                                int n_pages, const uint16_t* __restrict__ q,
+                                                                int n_kv_heads, int reduce,
+                                                                float* __restrict__ scores, int score_stride) {
+  constexpr int group = GROUP;
+  extern __shared__ __align__(16) uint8_t qsm[];
+  float (*qs)[kD] = reinterpret_cast<float (*)[kD]>(qsm + kQStages * kQChunkBytes);       // [8][128]
+  const int stream = blockIdx.y, tid = threadIdx.x;
   const int b = stream / n_kv_heads, kvh = stream - b * n_kv_heads;
-  for (int i = threadIdx.x; i < group * kD; i += blockDim.x) {
+  const int page0 = blockIdx.x * kQPages;
+  const uint16_t* rows = boxes + static_cast<size_t>(stream) * kD * 2 * box_stride + page0;
+  const uint32_t stage0 = static_cast<uint32_t>(__cvta_generic_to_shared(qsm));
+  // chunk c -> stage c % kQStages: row r of the chunk is box row c * kQRows + r; a row is 32 pieces
+  // of 16 bytes (8 pages); pieces that start beyond the row's end (box_stride) are zero-filled
+  auto issue = [&](int c) {
+    const uint32_t dst = stage0 + (c % kQStages) * kQChunkBytes;
+#pragma unroll
+    for (int i = 0; i < kQRows * kQPieces / kQThreads; ++i) {
+      const int piece = tid + i * kQThreads, r = piece / kQPieces, col = piece % kQPieces;
+      const bool on = page0 + 8 * col < box_stride;
+      q_cp_async16(dst + r * kQRowBytes + col * 16, rows + static_cast<size_t>(c * kQRows + r) * box_stride + (on ? 8 * col : 0), on);
+    }
+    asm volatile("cp.async.commit_group;\n" ::: "memory");
+  };
+#pragma unroll
+  for (int c = 0; c < kQStages - 1; ++c) issue(c);
+  for (int i = tid; i < group * kD; i += kQThreads) {
     const int h = i / kD, d = i - h * kD;
     const uint16_t bits = q[(static_cast<size_t>(b) * n_kv_heads * group + static_cast<size_t>(kvh) * group + h) * kD + d];
     qs[h][d] = __uint_as_float(static_cast<uint32_t>(bits) << 16);
   }
-  __syncthreads();
-  const int p0 = (blockIdx.x * blockDim.x + threadIdx.x) * 2;     // two pages per thread (one 32-bit load)
-  if (p0 >= n_pages) return;
-  float acc[kMaxHeadsPerKv][2];
+  float acc[GROUP];
 #pragma unroll
-  for (int h = 0; h < kMaxHeadsPerKv; ++h) acc[h][0] = acc[h][1] = 0.f;
-  const uint16_t* base = boxes + static_cast<size_t>(stream) * kD * 2 * box_stride + p0;
-#pragma unroll 8
-  for (int d = 0; d < kD; ++d) {
-    const uint32_t lo2 = *reinterpret_cast<const uint32_t*>(base + static_cast<size_t>(2 * d) * box_stride);
-    const uint32_t hi2 = *reinterpret_cast<const uint32_t*>(base + static_cast<size_t>(2 * d + 1) * box_stride);
-    const float lo_a = __uint_as_float(lo2 << 16), lo_b = __uint_as_float(lo2 & 0xffff0000u);
-    const float hi_a = __uint_as_float(hi2 << 16), hi_b = __uint_as_float(hi2 & 0xffff0000u);
+  for (int h = 0; h < GROUP; ++h) acc[h] = 0.f;
+#pragma unroll 1
+  for (int c = 0; c < kQChunks; ++c) {
+    if (c + kQStages - 1 < kQChunks) issue(c + kQStages - 1);
+    else asm volatile("cp.async.commit_group;\n" ::: "memory");          // keeps the group count uniform
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(kQStages - 1) : "memory");
+    __syncthreads();                                   // chunk c (and, the first time, the query) is visible to all
+    const uint8_t* st = qsm + (c % kQStages) * kQChunkBytes + tid * 2;
 #pragma unroll
-    for (int h = 0; h < kMaxHeadsPerKv; ++h) {
-      if (h < group) {
+    for (int i = 0; i < kQRows / 2; ++i) {
+      const float lo = __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(st + (2 * i) * kQRowBytes)) << 16);
+      const float hi = __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(st + (2 * i + 1) * kQRowBytes)) << 16);
+      const int d = c * (kQRows / 2) + i;
+#pragma unroll
+      for (int h = 0; h < GROUP; ++h) {
         const float qv = qs[h][d];
-        const bool pos = qv >= 0.f;
-        acc[h][0] = __fmaf_rn(qv, pos ? hi_a : lo_a, acc[h][0]);
-        acc[h][1] = __fmaf_rn(qv, pos ? hi_b : lo_b, acc[h][1]);
+        acc[h] = __fmaf_rn(qv, qv >= 0.f ? hi : lo, acc[h]);
       }
     }
+    __syncthreads();                                   // the stage may be refilled
   }
-  float s0 = acc[0][0], s1 = acc[0][1];
-  for (int h = 1; h < group; ++h) {
-    if (reduce == 0) {
-      s0 = fmaxf(s0, acc[h][0]);
-      s1 = fmaxf(s1, acc[h][1]);
-    } else {
-      s0 = __fadd_rn(s0, acc[h][0]);
-      s1 = __fadd_rn(s1, acc[h][1]);
-    }
-  }
-  float* out = scores + static_cast<size_t>(stream) * score_stride;
-  out[p0] = s0;
-  if (p0 + 1 < n_pages) out[p0 + 1] = s1;
+  const int p0 = page0 + tid;
+  if (p0 >= n_pages) return;
+  float s0 = acc[0];
+#pragma unroll
+  for (int h = 1; h < GROUP; ++h) s0 = (reduce == 0) ? fmaxf(s0, acc[h]) : __fadd_rn(s0, acc[h]);
+  scores[static_cast<size_t>(stream) * score_stride + p0] = s0;
 }
 
 // Order-preserving key: larger score <-> larger key; -0 and +0 map to the same key.
@@ -104,15 +136,35 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
       if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
     }
     __syncthreads();
-    if (tid == 0) {
-      uint32_t rem = s_remaining;
-      int d = 255;
-      for (; d > 0; --d) {
-        if (hist[d] >= rem) break;
-        rem -= hist[d];
+    // The digit of the k-th largest is the t with c[t] >= rem > c[t + 1], c[t] = sum_{j >= t} hist[j].
+    // Warp 0: lane l owns bins 255 - 8 l .. 248 - 8 l (from the top), a shuffle scan joins the lanes.
+    if (tid < 32) {
+      const uint32_t rem = s_remaining;
+      uint32_t own[8], tot = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        own[j] = hist[255 - 8 * tid - j];
+        tot += own[j];
       }
-      s_prefix = prefix | (static_cast<uint32_t>(d) << shift);
-      s_remaining = rem;
+      uint32_t incl = tot;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xffffffffu, incl, d);
+        if (tid >= d) incl += up;
+      }
+      uint32_t above = incl - tot;                  // count in bins above this lane's eight
+      if (above < rem && incl >= rem) {             // exactly one lane
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (above < rem && above + own[j] >= rem) {
+            s_prefix = prefix | (static_cast<uint32_t>(255 - 8 * tid - j) << shift);
+            s_remaining = rem - above;
+            above = rem;                            // done: no later bin matches
+          } else {
+            above += own[j];
+          }
+        }
+      }
     }
     __syncthreads();
   }
@@ -169,10 +221,33 @@ cudaError_t launch_quest_scores(const uint16_t* boxes, int box_stride, int n_pag
                                 int n_streams, int n_kv_heads, int group, int reduce, float* scores,
                                 int score_stride, cudaStream_t st) {
   if (n_pages <= 0) return cudaSuccess;
-  const int threads = 128;
-  const int per_cta = threads * 2;
-  quest_score_kernel<<<dim3((n_pages + per_cta - 1) / per_cta, n_streams), threads, 0, st>>>(
-      boxes, box_stride, n_pages, q, n_kv_heads, group, reduce, scores, score_stride);
+  const size_t smem = kQStages * kQChunkBytes + kMaxHeadsPerKv * kD * sizeof(float);
+  const dim3 grid((n_pages + kQPages - 1) / kQPages, n_streams);
+  cudaError_t e = cudaSuccess;
+#define GKV_QUEST_CASE(G)                                                                                                \
+  case G: {                                                                                                              \
+    static bool configured = false;                                                                                      \
+    if (!configured) {                                                                                                   \
+      e = cudaFuncSetAttribute(quest_score_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)); \
+      if (e != cudaSuccess) return e;                                                                                    \
+      configured = true;                                                                                                 \
+    }                                                                                                                    \
+    quest_score_kernel<G><<<grid, kQThreads, smem, st>>>(boxes, box_stride, n_pages, q, n_kv_heads, reduce, scores,     \
+                                                         score_stride);                                                  \
+    break;                                                                                                               \
+  }
+  switch (group) {
+    GKV_QUEST_CASE(1)
+    GKV_QUEST_CASE(2)
+    GKV_QUEST_CASE(3)
+    GKV_QUEST_CASE(4)
+    GKV_QUEST_CASE(5)
+    GKV_QUEST_CASE(6)
+    GKV_QUEST_CASE(7)
+    GKV_QUEST_CASE(8)
+    default: return cudaErrorInvalidValue;
+  }
+#undef GKV_QUEST_CASE
   return cudaGetLastError();
 }
 
