@@ -238,6 +238,19 @@ def run_ours(args, rank, local, world):
     achieved = algo_bytes / (us_launch * 1e-6) / 1e9
     peak, peak_kind = measured_hbm_peak()
     traffic = DRAM_TRAFFIC_PER_LAUNCH.get(wl.name)
+    scorer = None
+    if quest:
+        # the page scorer on its own (score + top-k launches): it reads every box of the layer
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for r in range(reps):
+            for l in range(n_layers):
+                cache.gkv_quest_select(l, q_new[r % total_steps, l], wl.quest_budget_tokens, pages)
+        s1.record()
+        torch.cuda.synchronize()
+        us_sel = s0.elapsed_time(s1) * 1e3 / (reps * n_layers)
+        scorer = {"us_per_call": us_sel, "box_bytes_per_call": rep.box_bits / 8,
+                  "achieved": rep.box_bits / 8 / (us_sel * 1e-6) / 1e9, "unit": "GB/s"}
 
     # ---- end to end: host buffers, H2D of the step's inputs and D2H of its result inside the region
     hk = torch.randn((n_layers, Bsz, 1, Hkv, d)).to(torch.bfloat16).pin_memory()
@@ -301,6 +314,8 @@ def run_ours(args, rank, local, world):
                      "frac_of_8TBs": achieved / NOMINAL_HBM_GBS},
         "ctx_tokens_per_s_per_layer_call": Bsz * ctx_start / (us_launch * 1e-6),
     }
+    if scorer:
+        line["quest_select"] = scorer
     if rank == 0:
         line["cpu_baseline"] = cpu_baseline(wl, n_layers, budget_s=args.cpu_seconds)
     cache.close()
