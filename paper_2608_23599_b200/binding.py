@@ -20,7 +20,8 @@ POLICY_STAIRCASE, POLICY_RD, POLICY_EXTERNAL = 0, 1, 2
 REDUCE_MAX, REDUCE_SUM = 0, 1
 TENSOR_K, TENSOR_V = 0, 1
 OK = 0
-ERR_RANGE, ERR_BUDGET = -6, -7
+ERR_INVALID_ARG, ERR_ARENA_TOO_SMALL, ERR_CTX_FULL, ERR_BAD_STATE, ERR_UNSUPPORTED = -1, -2, -3, -4, -5
+ERR_RANGE, ERR_BUDGET, ERR_CUDA = -6, -7, -8
 
 EXPORTS = [
     "gkv_query_arena_bytes", "gkv_create", "gkv_destroy", "gkv_append_demote", "gkv_decode_attn",

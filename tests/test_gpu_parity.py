@@ -633,3 +633,42 @@ def test_certificate_of_an_exact_cache_is_zero():
     torch.cuda.synchronize()
     assert torch.all(cert == 0)
     gcache.close()
+
+
+@pytest.mark.parametrize("hq,hkv", [(2, 2), (4, 2), (16, 2)])
+def test_observe_query_group_sizes(hq, hkv):
+    """Block masses, running masses and the certificate with 1, 2 and 8 query heads per KV head."""
+    import dataclasses
+    w = _tiny(1000, n_q_heads=hq, n_kv_heads=hkv, stair_tokens=(192, 192, 256, 192))
+    ocache, gcache = _pair(w)
+    dense = O.GradedCache(U.oracle_config(dataclasses.replace(w, stair_tokens=(-1, 0, 0, 0))))
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    dense.append_demote(0, U.f32(data["k"]), U.f32(data["v"]))
+    out, o_out, mass, o_obs = _observe_both(ocache, gcache, 0, data["q"])
+    U.assert_outputs_close(out, o_out, f"observe group {hq // hkv}")
+    _assert_mass_close(mass, o_obs, f"group {hq // hkv}")
+    _check_bounds_and_certificate(w, ocache, gcache, dense, data["q"], f"group {hq // hkv}")
+    gcache.close()
+
+
+def test_observe_and_reallocate_reject_what_they_do_not_cover():
+    B = _binding()
+    # latent-attention streams: no block-mass observation
+    wm = W.config(4, "small")
+    _, gm = _pair(wm)
+    dev = gm.device
+    dm = W.make_layer(wm, 0, "cpu")
+    gm.gkv_append_demote(0, dm["k"].to(dev), None)
+    out = torch.empty((wm.batch, wm.n_q_heads, wm.d_v), dtype=torch.float32, device=dev)
+    with pytest.raises(B.GkvError) as e:
+        gm.gkv_decode_attn_observe(0, dm["q"].to(dev), out)
+    assert e.value.status == B.ERR_UNSUPPORTED
+    gm.close()
+    # re-allocation is the RD policy's
+    w = W.config(0)
+    _, g = _pair(w)
+    with pytest.raises(B.GkvError) as e:
+        g.gkv_rd_reallocate(0)
+    assert e.value.status == B.ERR_BAD_STATE
+    g.close()
