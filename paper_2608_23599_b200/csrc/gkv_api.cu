@@ -405,12 +405,28 @@ size_t item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) 
 // walks its units in ascending token order.
 void build_descs(gkv_cache* c, LayerState& L) {
   const int ns = c->n_streams;
-  struct Unit { uint32_t word; size_t cost; };
+  struct Unit { uint32_t word; uint32_t cost; };
+  // Pass 1: the units of every stream and their total cost.  Streams with the same levels and the
+  // same number of residual rows (all streams under the staircase policy) have the same units:
+  // stream s then refers to the first stream it equals (same_as[s]) and nothing is built twice.
+  std::vector<int> same_as(ns);
   std::vector<std::vector<Unit>> units(ns);
   std::vector<size_t> cost(ns, 0);
   size_t total = 0;
   for (int s = 0; s < ns; ++s) {
     const int8_t* lv = L.level.data() + static_cast<size_t>(s) * c->max_blocks;
+    same_as[s] = s;
+    if (s > 0) {
+      const int r = same_as[s - 1];
+      if (L.res_count_h[s] == L.res_count_h[r] &&
+          std::memcmp(lv, L.level.data() + static_cast<size_t>(r) * c->max_blocks, static_cast<size_t>(L.n_closed)) == 0)
+        same_as[s] = r;
+    }
+    if (same_as[s] != s) {
+      cost[s] = cost[same_as[s]];
+      total += cost[s];
+      continue;
+    }
     const int groups = (L.res_count_h[s] + 15) / 16;
     const int n_items = L.n_closed + 1 + groups;
     std::vector<Unit>& u = units[s];
@@ -426,48 +442,63 @@ void build_descs(gkv_cache* c, LayerState& L) {
       }
       size_t k = 0;
       for (int j = 0; j < run; ++j) k += item_cost(c, L, s, i + j);
-      u.push_back(Unit{static_cast<uint32_t>(i) | (static_cast<uint32_t>(run) << 24), k});
+      u.push_back(Unit{static_cast<uint32_t>(i) | (static_cast<uint32_t>(run) << 24), static_cast<uint32_t>(k)});
       cost[s] += k;
       i += run;
     }
     total += cost[s];
   }
   const size_t target = std::max(kMinWarpCost, (total + kTargetWarps - 1) / kTargetWarps);
+  // Pass 2: deal each distinct stream's units to its warps, then lay the warps out.
   int w = 0, pos = 0, row = 0;
-  std::vector<size_t> load;
-  std::vector<std::vector<uint32_t>> mine;
+  int dealt_for = -1, dealt_nw = 0;                 // the stream and warp count `lists` was dealt for
+  std::vector<std::vector<uint32_t>> lists;         // per warp (in layout order): its units, ascending
+  std::vector<std::pair<size_t, int>> heap;         // (load, warp): least loaded first, then lowest index
   for (int s = 0; s < ns; ++s) {
-    std::vector<Unit>& u = units[s];
+    const int src = same_as[s];
+    const std::vector<Unit>& u0 = units[src];
     int nw = static_cast<int>((cost[s] + target / 2) / target);
-    nw = std::max(1, std::min(nw, static_cast<int>(u.size())));
+    nw = std::max(1, std::min(nw, static_cast<int>(u0.size())));
     nw = std::min(nw, c->max_warps - w - (ns - 1 - s));
-    std::stable_sort(u.begin(), u.end(), [](const Unit& a, const Unit& b) { return a.cost > b.cost; });
-    load.assign(nw, 0);
-    mine.assign(nw, {});
-    for (const Unit& x : u) {
-      int best = 0;
-      for (int k = 1; k < nw; ++k)
-        if (load[k] < load[best]) best = k;
-      load[best] += x.cost;
-      mine[best].push_back(x.word);
+    if (dealt_for != src || dealt_nw != nw) {
+      std::vector<Unit> u(u0);
+      std::stable_sort(u.begin(), u.end(), [](const Unit& a, const Unit& b) { return a.cost > b.cost; });
+      std::vector<std::vector<uint32_t>> mine(nw);
+      heap.clear();
+      for (int k = 0; k < nw; ++k) heap.emplace_back(0, k);
+      auto later = [](const std::pair<size_t, int>& a, const std::pair<size_t, int>& b) { return a > b; };
+      std::make_heap(heap.begin(), heap.end(), later);
+      for (const Unit& x : u) {                      // longest first onto the least loaded warp
+        std::pop_heap(heap.begin(), heap.end(), later);
+        std::pair<size_t, int>& best = heap.back();
+        best.first += x.cost;
+        mine[best.second].push_back(x.word);
+        std::push_heap(heap.begin(), heap.end(), later);
+      }
+      // Longest-first dealing hands the costliest units (exact blocks, then 8-bit ones) to the first
+      // warps, and a CTA is a window of consecutive warps: walk the warps with a golden-ratio stride
+      // so that every window holds the same mixture of levels.  Warps of one SM share its issue
+      // slots, and a CTA whose warps all run the issue-heavy levels would finish last.
+      int stride = std::max(1, static_cast<int>(nw * 0.6180339887 + 0.5));
+      while (std::gcd(stride, nw) != 1) ++stride;
+      lists.assign(nw, {});
+      for (int k = 0; k < nw; ++k) {
+        std::vector<uint32_t>& m = mine[static_cast<size_t>((static_cast<long long>(k) * stride) % nw)];
+        std::sort(m.begin(), m.end(), [](uint32_t a, uint32_t b) { return (a & 0xffffffu) < (b & 0xffffffu); });
+        lists[k].swap(m);
+      }
+      dealt_for = src;
+      dealt_nw = nw;
     }
-    // Longest-first dealing hands the costliest units (exact blocks, then 8-bit ones) to the first
-    // warps, and a CTA is a window of consecutive warps: walk the warps with a golden-ratio stride so
-    // that every window holds the same mixture of levels.  Warps of one SM share its issue slots, and
-    // a CTA whose warps all run the issue-heavy levels would finish last.
-    int stride = std::max(1, static_cast<int>(nw * 0.6180339887 + 0.5));
-    while (std::gcd(stride, nw) != 1) ++stride;
-    std::vector<int> order(nw);
-    for (int k = 0; k < nw; ++k) order[k] = static_cast<int>((static_cast<long long>(k) * stride) % nw);
     // one partial row per (CTA, stream): the kernel merges the warps of a CTA that share a stream
     L.parts_h[s].begin = row;
     for (int k = 0; k < nw; ++k) {
-      std::vector<uint32_t>& m = mine[order[k]];
-      std::sort(m.begin(), m.end(), [](uint32_t a, uint32_t b) { return (a & 0xffffffu) < (b & 0xffffffu); });
+      const std::vector<uint32_t>& m = lists[k];
       WarpDesc& d = L.warps_h[w];
       d.stream = s;
       d.item_begin = pos;
-      for (uint32_t x : m) L.units_h[pos++] = x;
+      std::memcpy(L.units_h + pos, m.data(), m.size() * sizeof(uint32_t));
+      pos += static_cast<int>(m.size());
       d.item_end = pos;
       if (k > 0 && w % kDecodeWarps == 0) ++row;
       d.partial = row;
@@ -731,7 +762,8 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
     }
     L.has_tail_slot = true;
     if ((rc = upload(c, L.table_d, L.table_h, table_bytes, st, L.ev)) != GKV_OK) return rc;
-    L.desc_dirty = true;
+    // The work lists stay valid: they always hold the partial block as item n_closed (skipped by the
+    // kernel while it is empty), so a new partial block changes only its table entry.
   }
   CK(c, launch_append_rows(c->arena, L.table_d, c->table_stride, L.n_closed, ns, cfg.n_kv_heads, k_new, v_new, 1, 0, 1,
                            L.n_tail, st));
