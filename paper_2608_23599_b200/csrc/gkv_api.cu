@@ -90,7 +90,8 @@ struct LayerState {
   std::vector<std::vector<int32_t>> res_idx;
   bool desc_dirty = true;
   int n_warps = 0;
-  cudaEvent_t ev = nullptr;             // last upload from this layer's pinned mirrors
+  cudaEvent_t ev = nullptr;             // last upload from this layer's pinned table / residual mirrors
+  cudaEvent_t ev_desc = nullptr;        // last upload from its pinned work lists (warps, units, parts)
   // device regions
   TableEntry* table_d = nullptr;
   WarpDesc* warps_d = nullptr;
@@ -136,6 +137,13 @@ struct gkv_cache {
   float* lse2_d = nullptr;              // [n_streams][8]
   EncodeJob* jobs_d = nullptr;
   size_t jobs_cap = 0;
+  // Small job lists of decode-time demotions go through a ring of pinned slots with an event each,
+  // so that consecutive layers' block closes do not wait for one another's copies.
+  static constexpr int kDemoteSlots = 8;
+  EncodeJob* demote_h = nullptr;        // pinned [kDemoteSlots][demote_cap]
+  size_t demote_cap = 0;
+  int demote_next = 0;
+  cudaEvent_t ev_demote[kDemoteSlots] = {};
   // shared pinned staging (jobs | levels | k-per-stream), guarded by ev_stage
   uint8_t* stage_h = nullptr;
   size_t stage_bytes = 0;
@@ -301,6 +309,15 @@ int upload(gkv_cache* c, void* dst, const void* src, size_t bytes, cudaStream_t 
   if (bytes == 0) return GKV_OK;
   CK(c, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st));
   CK(c, cudaEventRecord(ev, st));
+  return GKV_OK;
+}
+
+// Copy the table entries of block `block` of every stream (one column of the [stream][block] table).
+int upload_table_column(gkv_cache* c, LayerState& L, int block, cudaStream_t st) {
+  const size_t pitch = static_cast<size_t>(c->table_stride) * sizeof(TableEntry);
+  CK(c, cudaMemcpy2DAsync(L.table_d + block, pitch, L.table_h + block, pitch, sizeof(TableEntry), c->n_streams,
+                          cudaMemcpyHostToDevice, st));
+  CK(c, cudaEventRecord(L.ev, st));
   return GKV_OK;
 }
 
@@ -698,50 +715,65 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
 int demote_to_targets(gkv_cache* c, LayerState& L, const int8_t* target, size_t stride, cudaStream_t st) {
   const gkv_config& cfg = c->cfg;
   const int ns = c->n_streams;
-  const size_t table_bytes = static_cast<size_t>(ns) * c->table_stride * sizeof(TableEntry);
   int rc;
-  if ((rc = wait_event(c, c->ev_stage)) != GKV_OK) return rc;
+  std::vector<std::pair<int, int>> want_list;            // (stream, block) whose level falls
+  for (int s = 0; s < ns; ++s) {
+    const int8_t* tg = target + static_cast<size_t>(s) * stride;
+    const int8_t* cur = L.level.data() + static_cast<size_t>(s) * c->max_blocks;
+    for (int b = 0; b < L.n_closed; ++b)
+      if (tg[b] < cur[b]) want_list.emplace_back(s, b);    // monotone: levels only fall
+  }
+  if (want_list.empty()) return GKV_OK;
+  EncodeJob* jobs;
+  cudaEvent_t ev_jobs;
+  if (want_list.size() <= c->demote_cap) {
+    const int slot = c->demote_next++ % gkv_cache::kDemoteSlots;
+    jobs = c->demote_h + static_cast<size_t>(slot) * c->demote_cap;
+    ev_jobs = c->ev_demote[slot];
+  } else {
+    jobs = reinterpret_cast<EncodeJob*>(c->stage_h);
+    ev_jobs = c->ev_stage;
+  }
+  if ((rc = wait_event(c, ev_jobs)) != GKV_OK) return rc;
   if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
-  EncodeJob* jobs = reinterpret_cast<EncodeJob*>(c->stage_h);
   size_t n_jobs = 0;
   std::vector<std::pair<int, uint32_t>> to_free;
-  for (int s = 0; s < ns; ++s)
-    for (int b = 0; b < L.n_closed; ++b) {
-      const int8_t want = target[static_cast<size_t>(s) * stride + b];
-      int8_t& cur = L.level[static_cast<size_t>(s) * c->max_blocks + b];
-      if (want >= cur) continue;                         // monotone: levels only fall
-      TableEntry& e = L.table_h[static_cast<size_t>(s) * c->table_stride + b];
-      uint32_t off;
-      if (!c->heap.alloc(want, &off)) return GKV_ERR_ARENA_TOO_SMALL;
-      EncodeJob& job = jobs[n_jobs++];
-      job.src_off256 = e.off256;
-      job.dst_off256 = off;
-      job.src_level = cur;
-      job.dst_level = want;
-      job.stream = s;
-      job.block = b;
-      job.pad = 0;
-      to_free.emplace_back(cur, e.off256);
-      e.off256 = off;
-      e.level = static_cast<uint32_t>(want);
-      cur = want;
-    }
-  if (n_jobs > 0) {
-    CK(c, cudaMemcpyAsync(c->jobs_d, jobs, n_jobs * sizeof(EncodeJob), cudaMemcpyHostToDevice, st));
-    CK(c, cudaEventRecord(c->ev_stage, st));
-    EncodeParams ep{};
-    ep.arena = c->arena;
-    ep.jobs = c->jobs_d;
-    ep.n_jobs = static_cast<int32_t>(n_jobs);
-    ep.n_kv_heads = cfg.n_kv_heads;
-    ep.status = c->status_d;
-    ep.err = L.err_d;
-    ep.err_stride = c->max_blocks;
-    CK(c, launch_encode(ep, st));
-    for (auto& f : to_free) c->heap.release(f.first, f.second);
-    if ((rc = upload(c, L.table_d, L.table_h, table_bytes, st, L.ev)) != GKV_OK) return rc;
-    L.desc_dirty = true;
+  to_free.reserve(want_list.size());
+  for (const auto& sb : want_list) {
+    const int s = sb.first, b = sb.second;
+    const int8_t want = target[static_cast<size_t>(s) * stride + b];
+    int8_t& cur = L.level[static_cast<size_t>(s) * c->max_blocks + b];
+    TableEntry& e = L.table_h[static_cast<size_t>(s) * c->table_stride + b];
+    uint32_t off;
+    if (!c->heap.alloc(want, &off)) return GKV_ERR_ARENA_TOO_SMALL;
+    EncodeJob& job = jobs[n_jobs++];
+    job.src_off256 = e.off256;
+    job.dst_off256 = off;
+    job.src_level = cur;
+    job.dst_level = want;
+    job.stream = s;
+    job.block = b;
+    job.pad = 0;
+    to_free.emplace_back(cur, e.off256);
+    e.off256 = off;
+    e.level = static_cast<uint32_t>(want);
+    cur = want;
   }
+  CK(c, cudaMemcpyAsync(c->jobs_d, jobs, n_jobs * sizeof(EncodeJob), cudaMemcpyHostToDevice, st));
+  CK(c, cudaEventRecord(ev_jobs, st));
+  EncodeParams ep{};
+  ep.arena = c->arena;
+  ep.jobs = c->jobs_d;
+  ep.n_jobs = static_cast<int32_t>(n_jobs);
+  ep.n_kv_heads = cfg.n_kv_heads;
+  ep.status = c->status_d;
+  ep.err = L.err_d;
+  ep.err_stride = c->max_blocks;
+  ep.table = L.table_d;             // the kernel repoints the device table; the host mirror is already updated
+  ep.table_stride = c->table_stride;
+  CK(c, launch_encode(ep, st));
+  for (auto& f : to_free) c->heap.release(f.first, f.second);
+  L.desc_dirty = true;
   return GKV_OK;
 }
 
@@ -761,7 +793,7 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
       L.table_h[static_cast<size_t>(s) * c->table_stride + L.n_closed].resmask = 0;
     }
     L.has_tail_slot = true;
-    if ((rc = upload(c, L.table_d, L.table_h, table_bytes, st, L.ev)) != GKV_OK) return rc;
+    if ((rc = upload_table_column(c, L, L.n_closed, st)) != GKV_OK) return rc;
     // The work lists stay valid: they always hold the partial block as item n_closed (skipped by the
     // kernel while it is empty), so a new partial block changes only its table entry.
   }
@@ -1001,11 +1033,11 @@ int mla_append_one(gkv_cache* c, int layer, const uint16_t* k_new, cudaStream_t 
 
 int mla_decode(gkv_cache* c, LayerState& L, const void* q, float* out, float* lse, cudaStream_t st) {
   if (L.desc_dirty) {
-    int rc = wait_event(c, L.ev);
+    int rc = wait_event(c, L.ev_desc);
     if (rc != GKV_OK) return rc;
     mla_build_descs(c, L);
-    if ((rc = upload(c, L.warps_d, L.warps_h, static_cast<size_t>(L.n_warps) * sizeof(WarpDesc), st, L.ev)) != GKV_OK) return rc;
-    if ((rc = upload(c, L.parts_d, L.parts_h, static_cast<size_t>(c->n_streams) * sizeof(StreamParts), st, L.ev)) != GKV_OK) return rc;
+    if ((rc = upload(c, L.warps_d, L.warps_h, static_cast<size_t>(L.n_warps) * sizeof(WarpDesc), st, L.ev_desc)) != GKV_OK) return rc;
+    if ((rc = upload(c, L.parts_d, L.parts_h, static_cast<size_t>(c->n_streams) * sizeof(StreamParts), st, L.ev_desc)) != GKV_OK) return rc;
   }
   MlaDecodeParams p{};
   p.arena = c->arena;
@@ -1140,6 +1172,11 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
                    align_up(d.n_streams * sizeof(int32_t), 256) + 1024;
   if ((e = cudaHostAlloc(reinterpret_cast<void**>(&c->stage_h), c->stage_bytes, cudaHostAllocDefault)) != cudaSuccess) return fail(e);
   if ((e = cudaEventCreateWithFlags(&c->ev_stage, cudaEventDisableTiming)) != cudaSuccess) return fail(e);
+  c->demote_cap = static_cast<size_t>(d.n_streams) * 8;
+  if ((e = cudaHostAlloc(reinterpret_cast<void**>(&c->demote_h), gkv_cache::kDemoteSlots * c->demote_cap * sizeof(EncodeJob),
+                         cudaHostAllocDefault)) != cudaSuccess) return fail(e);
+  for (int i = 0; i < gkv_cache::kDemoteSlots; ++i)
+    if ((e = cudaEventCreateWithFlags(&c->ev_demote[i], cudaEventDisableTiming)) != cudaSuccess) return fail(e);
   c->layers.resize(cfg->n_layers);
   for (int l = 0; l < cfg->n_layers; ++l) {
     LayerState& L = c->layers[l];
@@ -1172,6 +1209,7 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
                                               static_cast<size_t>(s) * d.res_cap * 2 * kRowBytes) / 256);
     }
     if ((e = cudaEventCreateWithFlags(&L.ev, cudaEventDisableTiming)) != cudaSuccess) return fail(e);
+    if ((e = cudaEventCreateWithFlags(&L.ev_desc, cudaEventDisableTiming)) != cudaSuccess) return fail(e);
     if ((e = cudaMemcpy(L.res_off_d, L.res_off_h, d.n_streams * sizeof(uint32_t), cudaMemcpyHostToDevice)) != cudaSuccess) return fail(e);
   }
   if ((e = cudaDeviceSynchronize()) != cudaSuccess) return fail(e);
@@ -1251,8 +1289,12 @@ int gkv_destroy(gkv_cache* c) {
     if (L.res_off_h) cudaFreeHost(L.res_off_h);
     if (L.res_count_h) cudaFreeHost(L.res_count_h);
     if (L.ev) cudaEventDestroy(L.ev);
+    if (L.ev_desc) cudaEventDestroy(L.ev_desc);
   }
   if (c->stage_h) cudaFreeHost(c->stage_h);
+  if (c->demote_h) cudaFreeHost(c->demote_h);
+  for (cudaEvent_t ev : c->ev_demote)
+    if (ev) cudaEventDestroy(ev);
   if (c->ev_stage) cudaEventDestroy(c->ev_stage);
   delete c;
   return GKV_OK;
@@ -1344,12 +1386,14 @@ int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_
     L.last_n_sel = n_sel;
   } else {
     if (L.desc_dirty) {
-      int rc = wait_event(c, L.ev);
+      // the work lists have their own event: waiting for the table's would wait for copies that
+      // the append of this very step has just queued, i.e. drain the stream
+      int rc = wait_event(c, L.ev_desc);
       if (rc != GKV_OK) return rc;
       build_descs(c, L);
-      if ((rc = upload(c, L.warps_d, L.warps_h, static_cast<size_t>(L.n_warps) * sizeof(WarpDesc), st, L.ev)) != GKV_OK) return rc;
-      if ((rc = upload(c, L.units_d, L.units_h, static_cast<size_t>(L.n_units) * sizeof(uint32_t), st, L.ev)) != GKV_OK) return rc;
-      if ((rc = upload(c, L.parts_d, L.parts_h, static_cast<size_t>(c->n_streams) * sizeof(StreamParts), st, L.ev)) != GKV_OK) return rc;
+      if ((rc = upload(c, L.warps_d, L.warps_h, static_cast<size_t>(L.n_warps) * sizeof(WarpDesc), st, L.ev_desc)) != GKV_OK) return rc;
+      if ((rc = upload(c, L.units_d, L.units_h, static_cast<size_t>(L.n_units) * sizeof(uint32_t), st, L.ev_desc)) != GKV_OK) return rc;
+      if ((rc = upload(c, L.parts_d, L.parts_h, static_cast<size_t>(c->n_streams) * sizeof(StreamParts), st, L.ev_desc)) != GKV_OK) return rc;
     }
     p.warps = L.warps_d;
     p.units = L.units_d;

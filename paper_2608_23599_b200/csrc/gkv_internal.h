@@ -131,6 +131,10 @@ struct EncodeParams {
   // max_j |k_j - k^_j|, y = the same for values, z = max_j |v_j| of the original rows.
   float4* err;            // [n_streams][err_stride]
   int32_t err_stride;
+  // Decode-time demotions: the kernel also points the block table at the new slot (nullable;
+  // offset and level of entry [stream][block], the residual mask stays).
+  TableEntry* table;
+  int32_t table_stride;
 };
 
 // Statistics of freshly closed blocks: page boxes, key range proxy, block mass.

@@ -113,23 +113,35 @@ __device__ void pack_codes(uint8_t* slot, const uint8_t* codes, int bits, bool i
     const int tile = i / (words_per_lane * 32);
     const int r = lane >> 2, c4 = lane & 3;
     uint32_t word = 0;
-    // every (s, a, hlf) whose code lives in word w of this lane
-    for (int s = 0; s < 8; ++s)
-      for (int a = 0; a < 4; ++a)
-        for (int hlf = 0; hlf < 2; ++hlf) {
-          int boff, bit;
-          code_pos(bits, lane, s, a, hlf, &boff, &bit);
-          if (boff != ((w >> 2) * 32 + lane) * 16 + (w & 3) * 4) continue;
-          int tok, ch;
-          if (!is_v) {
-            tok = 16 * tile + r + 8 * (a & 1);
-            ch = 16 * s + 8 * (a >> 1) + 2 * c4 + hlf;
-          } else {
-            ch = 16 * s + r + 8 * (a & 1);
-            tok = 16 * tile + 8 * (a >> 1) + 2 * c4 + hlf;
-          }
-          word |= static_cast<uint32_t>(codes[tok * kD + ch]) << bit;
-        }
+    // the 32 / bits codes (s, a, hlf) that live in word w of this lane (the inverse of code_pos)
+    const int per = 32 / bits;
+    for (int q = 0; q < per; ++q) {
+      int s, a, hlf;
+      if (bits == 8) {
+        s = w >> 1;
+        a = ((w & 1) << 1) | (q & 1);
+        hlf = q >> 1;
+      } else if (bits == 4) {
+        s = w;
+        a = q & 3;
+        hlf = q >> 2;
+      } else {
+        s = 2 * w + (q & 1);
+        a = (q >> 1) & 3;
+        hlf = q >> 3;
+      }
+      int boff, bit;
+      code_pos(bits, lane, s, a, hlf, &boff, &bit);
+      int tok, ch;
+      if (!is_v) {
+        tok = 16 * tile + r + 8 * (a & 1);
+        ch = 16 * s + 8 * (a >> 1) + 2 * c4 + hlf;
+      } else {
+        ch = 16 * s + r + 8 * (a & 1);
+        tok = 16 * tile + 8 * (a >> 1) + 2 * c4 + hlf;
+      }
+      word |= static_cast<uint32_t>(codes[tok * kD + ch]) << bit;
+    }
     const int half = tile >> 1, t = tile & 1;
     uint8_t* region = slot + half * half_bytes(bits) + (is_v ? off_vc(bits, t) : off_kc(bits, t));
     *reinterpret_cast<uint32_t*>(region + ((w >> 2) * 32 + lane) * 16 + (w & 3) * 4) = word;
@@ -267,6 +279,11 @@ __global__ void __launch_bounds__(256) encode_kernel(const __grid_constant__ Enc
       }
     }
     if (p.err && tid == 0) p.err[static_cast<size_t>(job.stream) * p.err_stride + job.block] = bound;
+    if (p.table && tid == 0) {
+      TableEntry* te = p.table + static_cast<size_t>(job.stream) * p.table_stride + job.block;
+      te->off256 = job.dst_off256;
+      te->level = static_cast<uint32_t>(job.dst_level);
+    }
   }
 }
 
