@@ -922,12 +922,25 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     fence_proxy_async();
   }
   __syncwarp();
+  // The start of a launch is a chain of dependent look-ups (work list -> block table -> bytes):
+  // the first unit word is asked for here, its table entry right after the wait below, so that both
+  // are on their way while the query is staged.  unit_at() picks them up as its prefetched pair.
+  if constexpr (!SPARSE) {
+    if (first < w.item_end) w.pf_unit = w.units[first];
+  }
   // Launched with programmatic stream serialisation: what is above (descriptor fetch, barrier
-  // set-up) may overlap the tail of the previous kernel in the stream.  Nothing that a previous
-  // kernel may have written (the query, appended rows, partial rows, tickets) is touched before
-  // this wait, which returns once that kernel has completed and its writes are visible.
+  // set-up, the first word of the host-written work list) may overlap the tail of the previous
+  // kernel in the stream.  Nothing that a previous kernel may have written (the block table, the
+  // query, appended rows, partial rows, tickets) is touched before this wait, which returns once
+  // that kernel has completed and its writes are visible.
   asm volatile("griddepcontrol.wait;\n" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+  if constexpr (!SPARSE) {
+    if (first < w.item_end) {
+      w.pf_entry = *reinterpret_cast<const uint4*>(w.table + min(static_cast<int>(w.pf_unit & 0xffffffu), p.n_closed));
+      w.pf_pos = first;
+    }
+  }
 
   // Query fragments: B operand Q^T[16 channels x 8 heads]; lane (r, c4) holds head r, channels
   // 16 s + 2 c4 (+1) and 16 s + 8 + 2 c4 (+1), in bf16 (exact rows) and fp16 (quantised tiers).
