@@ -1095,22 +1095,19 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
 #pragma unroll 1
       for (int e = threadIdx.x; e < n_elem; e += kDecodeWarps * 32) {
         const int h = e / (kD + 2), j = e - h * (kD + 2);
+        // one pass in warp order: running maximum M and the sum relative to it (the loads of the
+        // rows do not depend on one another; only the short rescaling chain is serial)
         const float* col = rows + h * (kD + 2);
-        float M = kNegInf;
-#pragma unroll 1
-        for (int i = gb; i < ge; ++i) M = fmaxf(M, col[i * kRowFloats]);
-        float acc = 0.f;
-        if (j == 0) {
-          acc = M;
-        } else {
+        float M = kNegInf, acc = 0.f;
 #pragma unroll 2
-          for (int i = gb; i < ge; ++i) {
-            const float m = col[i * kRowFloats];
-            const float wgt = (m == kNegInf) ? 0.f : fast_exp2(m - M);
-            acc = fmaf(wgt, col[i * kRowFloats + j], acc);
-          }
+        for (int i = gb; i < ge; ++i) {
+          const float m = col[i * kRowFloats], v = col[i * kRowFloats + j];
+          const float Mn = fmaxf(M, m);
+          const float a = (M == kNegInf) ? 0.f : fast_exp2(M - Mn), bwt = (m == kNegInf) ? 0.f : fast_exp2(m - Mn);
+          acc = fmaf(acc, a, v * bwt);
+          M = Mn;
         }
-        dst[e] = acc;
+        dst[e] = (j == 0) ? M : acc;
       }
       // The CTA that delivers the stream's last row normalises and writes the output: rows are
       // published with a fence before the ticket is taken, and read back through L2.  Nobody
@@ -1143,17 +1140,17 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
         for (int e = threadIdx.x; e < p.group * kD; e += kDecodeWarps * 32) {
           const int h = e / kD, ch = e - h * kD;
           const float* col = p.partial + static_cast<size_t>(begin) * kPartialFloats + h * (kD + 2);
-          float M = kNegInf;
-#pragma unroll 4
-          for (int i = 0; i < end - begin; ++i) M = fmaxf(M, __ldcg(col + static_cast<size_t>(i) * kPartialFloats));
-          float L = 0.f, acc = 0.f;
+          // one pass in row order (one round of independent loads instead of two dependent ones)
+          float M = kNegInf, L = 0.f, acc = 0.f;
 #pragma unroll 4
           for (int i = 0; i < end - begin; ++i) {
             const float* row = col + static_cast<size_t>(i) * kPartialFloats;
-            const float m = __ldcg(row);
-            const float wgt = (m == kNegInf) ? 0.f : exp2f(m - M);
-            L = fmaf(wgt, __ldcg(row + 1), L);
-            acc = fmaf(wgt, __ldcg(row + 2 + ch), acc);
+            const float m = __ldcg(row), l = __ldcg(row + 1), v = __ldcg(row + 2 + ch);
+            const float Mn = fmaxf(M, m);
+            const float a = (M == kNegInf) ? 0.f : exp2f(M - Mn), bwt = (m == kNegInf) ? 0.f : exp2f(m - Mn);
+            L = fmaf(L, a, l * bwt);
+            acc = fmaf(acc, a, v * bwt);
+            M = Mn;
           }
           const size_t hq = static_cast<size_t>(b) * p.n_kv_heads * p.group + static_cast<size_t>(kvh) * p.group + h;
           p.out[hq * kD + ch] = (L > 0.f) ? acc / L : 0.f;
