@@ -1092,6 +1092,19 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     while (ge < kDecodeWarps && s_group[ge] == sid) ++ge;
     if (sid >= 0) {
       float* dst = p.partial + static_cast<size_t>(s_group[kDecodeWarps + gb]) * kPartialFloats;
+      // the stream's range of partial rows, asked for now and needed when the ticket is taken
+      // (sparse mode: a stream's CTAs are neighbours, one partial row each, row = CTA index)
+      int row_begin = 0, row_end = 0;
+      if (threadIdx.x == 0) {
+        const int per = p.warps_per_stream / kDecodeWarps;
+        row_begin = sid * per;
+        row_end = row_begin + per;
+        if (p.parts) {
+          const StreamParts sp = p.parts[sid];
+          row_begin = sp.begin;
+          row_end = sp.end;
+        }
+      }
 #pragma unroll 1
       for (int e = threadIdx.x; e < n_elem; e += kDecodeWarps * 32) {
         const int h = e / (kD + 2), j = e - h * (kD + 2);
@@ -1115,13 +1128,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
       __threadfence();
       __syncthreads();
       if (threadIdx.x == 0) {
-        // sparse mode: a stream's CTAs are neighbours, one partial row each (row = CTA index)
-        const int per = p.warps_per_stream / kDecodeWarps;
-        int begin = sid * per, end = begin + per;
-        if (p.parts) {
-          begin = p.parts[sid].begin;
-          end = p.parts[sid].end;
-        }
+        const int begin = row_begin, end = row_end;
         const int n = end - begin;
         bool is_last = true;
         if (n > 1) {
