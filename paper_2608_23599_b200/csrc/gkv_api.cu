@@ -502,7 +502,17 @@ void build_descs(gkv_cache* c, LayerState& L) {
       for (int k = 0; k < nw; ++k) {
         std::vector<uint32_t>& m = mine[static_cast<size_t>((static_cast<long long>(k) * stride) % nw)];
         std::sort(m.begin(), m.end(), [](uint32_t a, uint32_t b) { return (a & 0xffffffu) < (b & 0xffffffu); });
-        lists[k].swap(m);
+        // Ascending token order runs from the oldest, narrowest blocks to the newest, widest ones, and
+        // every warp would walk it in step with all the others: a long stretch in which the whole GPU
+        // asks for half of what HBM delivers (2-bit blocks), then one in which it asks for twice that
+        // (8-bit and exact blocks).  Taking the units alternately from both ends mixes byte-light and
+        // byte-heavy blocks in every warp, so that the demand is even over the launch.
+        std::vector<uint32_t>& out = lists[k];
+        out.clear();
+        for (size_t lo = 0, hi = m.size(); lo < hi;) {
+          out.push_back(m[lo++]);
+          if (lo < hi) out.push_back(m[--hi]);
+        }
       }
       dealt_for = src;
       dealt_nw = nw;
