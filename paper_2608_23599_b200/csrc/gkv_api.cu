@@ -513,6 +513,9 @@ void build_descs(gkv_cache* c, LayerState& L) {
           out.push_back(m[lo++]);
           if (lo < hi) out.push_back(m[--hi]);
         }
+        // ... and every warp starts at a different place of its list, so that the warps are not in
+        // step with one another either
+        if (out.size() > 1) std::rotate(out.begin(), out.begin() + (static_cast<size_t>(k) * 5) % out.size(), out.end());
       }
       dealt_for = src;
       dealt_nw = nw;
