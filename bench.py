@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch from an ncu capture
 # (profiles/ holds the summary); None = not captured for that workload.
-DRAM_TRAFFIC_PER_LAUNCH = {"cfg2_llama8b_append": 333.7e6}    # 329.7 MB read + 4.0 MB written (ncu, one launch)
+DRAM_TRAFFIC_PER_LAUNCH = {"cfg2_llama8b_append": 335.9e6}    # 330.1 MB read + 5.8 MB written (ncu, one launch)
 
 
 def measured_hbm_peak():
