@@ -292,7 +292,8 @@ def run_ours(args, rank, local, world):
     d2h = hout.numel() * 4
 
     launches_per_layer = 2 + (2 if quest else 0)      # append, decode with fused merge (+ score, top-k)
-    gpu_launches = K * n_layers * launches_per_layer + closes * n_layers * (1 + (1 if wl.page_tokens else 0))
+    # a block close adds the block-statistics kernel and, under the staircase policy, one encode launch
+    gpu_launches = K * n_layers * launches_per_layer + closes * n_layers * (1 + (1 if wl.policy == W.POLICY_STAIRCASE else 0))
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
