@@ -293,7 +293,7 @@ def run_ours(args, rank, local, world):
 
     launches_per_layer = 2 + (2 if quest else 0)      # append, decode with fused merge (+ score, top-k)
     # a block close adds the block-statistics kernel and, under the staircase policy, one encode launch
-    gpu_launches = K * n_layers * launches_per_layer + closes * n_layers * (1 + (1 if wl.policy == W.POLICY_STAIRCASE else 0))
+    gpu_launches = K * n_layers * launches_per_layer + closes * n_layers * ((0 if alias else 1) + (1 if wl.policy == W.POLICY_STAIRCASE else 0))
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
