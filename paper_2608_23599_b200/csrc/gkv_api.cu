@@ -503,18 +503,18 @@ void build_descs(gkv_cache* c, LayerState& L) {
         std::vector<uint32_t>& m = mine[static_cast<size_t>((static_cast<long long>(k) * stride) % nw)];
         std::sort(m.begin(), m.end(), [](uint32_t a, uint32_t b) { return (a & 0xffffffu) < (b & 0xffffffu); });
         // Ascending token order runs from the oldest, narrowest blocks to the newest, widest ones, and
-        // every warp would walk it in step with all the others: a long stretch in which the whole GPU
-        // asks for half of what HBM delivers (2-bit blocks), then one in which it asks for twice that
-        // (8-bit and exact blocks).  Taking the units alternately from both ends mixes byte-light and
-        // byte-heavy blocks in every warp, so that the demand is even over the launch.
+        // the warps of an SM would walk it in step: all of them unpacking 2- and 4-bit codes (bound
+        // by instruction issue, memory idle), later all of them waiting for 8-bit and exact tiles
+        // (issue slots idle).  Taking the units alternately from both ends, and starting every warp
+        // at a different place of its list (below), keeps both kinds of step in every SM at all
+        // times: a warp that waits for bytes leaves its issue slots to one that unpacks.  (Shifting
+        // whole CTAs against one another instead - every SM uniform, the GPU mixed - gains nothing.)
         std::vector<uint32_t>& out = lists[k];
         out.clear();
         for (size_t lo = 0, hi = m.size(); lo < hi;) {
           out.push_back(m[lo++]);
           if (lo < hi) out.push_back(m[--hi]);
         }
-        // ... and every warp starts at a different place of its list, so that the warps are not in
-        // step with one another either
         if (out.size() > 1) std::rotate(out.begin(), out.begin() + (static_cast<size_t>(k) * 5) % out.size(), out.end());
       }
       dealt_for = src;
