@@ -505,10 +505,11 @@ void build_descs(gkv_cache* c, LayerState& L) {
         // Ascending token order runs from the oldest, narrowest blocks to the newest, widest ones, and
         // the warps of an SM would walk it in step: all of them unpacking 2- and 4-bit codes (bound
         // by instruction issue, memory idle), later all of them waiting for 8-bit and exact tiles
-        // (issue slots idle).  Taking the units alternately from both ends, and starting every warp
-        // at a different place of its list (below), keeps both kinds of step in every SM at all
-        // times: a warp that waits for bytes leaves its issue slots to one that unpacks.  (Shifting
-        // whole CTAs against one another instead - every SM uniform, the GPU mixed - gains nothing.)
+        // (issue slots idle).  Taking the units alternately from both ends makes every warp follow a
+        // byte-heavy unit with an issue-heavy one, so its two-stage pipeline always has a long
+        // compute to hide a long copy behind; starting every warp at a different place of its list
+        // (below) also keeps both kinds of step in every SM at all times.  (Shifting whole CTAs
+        // against one another instead - every SM uniform, the GPU mixed - gains nothing.)
         std::vector<uint32_t>& out = lists[k];
         out.clear();
         for (size_t lo = 0, hi = m.size(); lo < hi;) {
