@@ -419,7 +419,7 @@ size_t item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) 
 // Units of a stream (a block, a run of up to 16 neighbouring centroid blocks, the tail, a residual
 // group) are dealt to the stream's warps longest-first onto the least loaded warp, so that every
 // warp ends up with the same cost whatever the order of levels along the context; each warp then
-// walks its units in ascending token order.
+// walks its units in a mixed order (see below).
 void build_descs(gkv_cache* c, LayerState& L) {
   const int ns = c->n_streams;
   struct Unit { uint32_t word; uint32_t cost; };
