@@ -41,6 +41,10 @@ __global__ void __launch_bounds__(kQThreads) quest_score_kernel(const uint16_t* 
                                                                 int n_kv_heads, int reduce,
                                                                 float* __restrict__ scores, int score_stride) {
   constexpr int group = GROUP;
+  // launched with programmatic stream serialisation: returns once the previous kernel of the stream
+  // has completed (the launch itself overlaps that kernel's tail)
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
   extern __shared__ __align__(16) uint8_t qsm[];
   float (*qs)[kD] = reinterpret_cast<float (*)[kD]>(qsm + kQStages * kQChunkBytes);       // [8][128]
   const int stream = blockIdx.y, tid = threadIdx.x;
@@ -114,6 +118,8 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
   __shared__ uint32_t s_prefix, s_remaining;
   __shared__ uint32_t warp_sel[32], warp_eq[32];
   __shared__ uint32_t base_sel, base_eq;
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
   const int stream = blockIdx.x, tid = threadIdx.x;
   const float* sc = scores + static_cast<size_t>(stream) * score_stride;
   int32_t* out = idx_out + static_cast<size_t>(stream) * idx_stride;
@@ -222,7 +228,16 @@ cudaError_t launch_quest_scores(const uint16_t* boxes, int box_stride, int n_pag
                                 int score_stride, cudaStream_t st) {
   if (n_pages <= 0) return cudaSuccess;
   const size_t smem = kQStages * kQChunkBytes + kMaxHeadsPerKv * kD * sizeof(float);
-  const dim3 grid((n_pages + kQPages - 1) / kQPages, n_streams);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((n_pages + kQPages - 1) / kQPages, n_streams);
+  cfg.blockDim = dim3(kQThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   cudaError_t e = cudaSuccess;
 #define GKV_QUEST_CASE(G)                                                                                                \
   case G: {                                                                                                              \
@@ -232,8 +247,8 @@ cudaError_t launch_quest_scores(const uint16_t* boxes, int box_stride, int n_pag
       if (e != cudaSuccess) return e;                                                                                    \
       configured = true;                                                                                                 \
     }                                                                                                                    \
-    quest_score_kernel<G><<<grid, kQThreads, smem, st>>>(boxes, box_stride, n_pages, q, n_kv_heads, reduce, scores,     \
-                                                         score_stride);                                                  \
+    e = cudaLaunchKernelEx(&cfg, quest_score_kernel<G>, boxes, box_stride, n_pages, q, n_kv_heads, reduce, scores,       \
+                           score_stride);                                                                                \
     break;                                                                                                               \
   }
   switch (group) {
@@ -248,15 +263,22 @@ cudaError_t launch_quest_scores(const uint16_t* boxes, int box_stride, int n_pag
     default: return cudaErrorInvalidValue;
   }
 #undef GKV_QUEST_CASE
-  return cudaGetLastError();
+  return e;
 }
 
 cudaError_t launch_topk(const float* scores, int score_stride, int n, const int32_t* k_per_stream, int k_uniform,
                         int32_t* idx_out, int idx_stride, int n_streams, cudaStream_t st) {
   if (n <= 0 || n_streams <= 0) return cudaSuccess;
-  topk_kernel<<<n_streams, kTopkThreads, 0, st>>>(scores, score_stride, n, k_per_stream, k_uniform, idx_out,
-                                                   idx_stride);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_streams);
+  cfg.blockDim = dim3(kTopkThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, topk_kernel, scores, score_stride, n, k_per_stream, k_uniform, idx_out, idx_stride);
 }
 
 }  // namespace gkv
