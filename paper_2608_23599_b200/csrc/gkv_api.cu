@@ -89,6 +89,7 @@ struct LayerState {
   int32_t* res_count_h = nullptr;       // pinned [n_streams]
   std::vector<std::vector<int32_t>> res_idx;
   bool desc_dirty = true;
+  bool desc_split = false;              // the work lists hold sub-block units (never for observing calls)
   int n_warps = 0;
   cudaEvent_t ev = nullptr;             // last upload from this layer's pinned table / residual mirrors
   cudaEvent_t ev_desc = nullptr;        // last upload from its pinned work lists (warps, units, parts)
@@ -206,7 +207,7 @@ Derived derive(const gkv_config& c) {
   d.res_cap = c.residual_fraction > 0.f
                   ? static_cast<int>(align_up(static_cast<size_t>(std::floor(static_cast<double>(c.residual_fraction) * c.max_ctx)) + 16, 16))
                   : 0;
-  d.unit_stride = d.max_blocks + 1 + d.res_cap / 16;
+  d.unit_stride = d.max_blocks + 1 + d.res_cap / 16 + 3 * (kTargetWarps / 2);      // small workloads list sub-block units
   d.box_stride = c.page_tokens > 0 ? static_cast<int>(align_up((c.max_ctx + c.page_tokens - 1) / c.page_tokens, 8)) : 0;
   return d;
 }
@@ -420,7 +421,7 @@ size_t item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) 
 // group) are dealt to the stream's warps longest-first onto the least loaded warp, so that every
 // warp ends up with the same cost whatever the order of levels along the context; each warp then
 // walks its units in a mixed order (see below).
-void build_descs(gkv_cache* c, LayerState& L) {
+void build_descs(gkv_cache* c, LayerState& L, bool allow_split) {
   const int ns = c->n_streams;
   struct Unit { uint32_t word; uint32_t cost; };
   // Pass 1: the units of every stream and their total cost.  Streams with the same levels and the
@@ -430,6 +431,19 @@ void build_descs(gkv_cache* c, LayerState& L) {
   std::vector<std::vector<Unit>> units(ns);
   std::vector<size_t> cost(ns, 0);
   size_t total = 0;
+  // A small workload leaves most warps of the GPU without work, and its launch then lasts as long
+  // as its longest unit (an exact block: eight steps).  Such lists are cut finer: an exact block
+  // into its four tiles and, when the workload is smaller still, a quantised block into its two
+  // halves, a warp holding as little as one of them (more, finer units also mean more partial rows
+  // to merge at the end, which is why this stops at some size).
+  bool split = false, split_all = false;
+  if (allow_split) {
+    size_t rough = 0;
+    for (int s = 0; s < ns; ++s) rough += static_cast<size_t>(L.n_closed + 1) * 1000 + static_cast<size_t>(L.res_count_h[s] / 16) * 550;
+    split = rough < static_cast<size_t>(kTargetWarps) * kMinWarpCost / 2;          // exact blocks only
+    split_all = rough < static_cast<size_t>(kTargetWarps) * kMinWarpCost / 8;      // quantised blocks too
+  }
+  L.desc_split = split;
   for (int s = 0; s < ns; ++s) {
     const int8_t* lv = L.level.data() + static_cast<size_t>(s) * c->max_blocks;
     same_as[s] = s;
@@ -459,13 +473,22 @@ void build_descs(gkv_cache* c, LayerState& L) {
       }
       size_t k = 0;
       for (int j = 0; j < run; ++j) k += item_cost(c, L, s, i + j);
-      u.push_back(Unit{static_cast<uint32_t>(i) | (static_cast<uint32_t>(run) << 24), static_cast<uint32_t>(k)});
+      const uint32_t base = static_cast<uint32_t>(i) | (static_cast<uint32_t>(run) << 24);
+      const int8_t lvl = (run == 1 && i < L.n_closed) ? lv[i] : int8_t{0};
+      if (split && lvl == 16) {
+        for (uint32_t t = 0; t < 4; ++t) u.push_back(Unit{base | ((1u << t) << 20), static_cast<uint32_t>(k / 4)});
+      } else if (split_all && (lvl == 8 || lvl == 4 || lvl == 2)) {
+        u.push_back(Unit{base | (3u << 20), static_cast<uint32_t>(k / 2)});
+        u.push_back(Unit{base | (12u << 20), static_cast<uint32_t>(k - k / 2)});
+      } else {
+        u.push_back(Unit{base | (15u << 20), static_cast<uint32_t>(k)});
+      }
       cost[s] += k;
       i += run;
     }
     total += cost[s];
   }
-  const size_t target = std::max(kMinWarpCost, (total + kTargetWarps - 1) / kTargetWarps);
+  const size_t target = std::max(split_all ? kMinWarpCost / 4 : kMinWarpCost, (total + kTargetWarps - 1) / kTargetWarps);
   // Pass 2: deal each distinct stream's units to its warps, then lay the warps out.
   int w = 0, pos = 0, row = 0;
   int dealt_for = -1, dealt_nw = 0;                 // the stream and warp count `lists` was dealt for
@@ -501,7 +524,9 @@ void build_descs(gkv_cache* c, LayerState& L) {
       lists.assign(nw, {});
       for (int k = 0; k < nw; ++k) {
         std::vector<uint32_t>& m = mine[static_cast<size_t>((static_cast<long long>(k) * stride) % nw)];
-        std::sort(m.begin(), m.end(), [](uint32_t a, uint32_t b) { return (a & 0xffffffu) < (b & 0xffffffu); });
+        std::sort(m.begin(), m.end(), [](uint32_t a, uint32_t b) {       // by block, then by tile mask
+          return (((a & kUnitItemMask) << 4) | ((a >> 20) & 15u)) < (((b & kUnitItemMask) << 4) | ((b >> 20) & 15u));
+        });
         // Ascending token order runs from the oldest, narrowest blocks to the newest, widest ones, and
         // the warps of an SM would walk it in step: all of them unpacking 2- and 4-bit codes (bound
         // by instruction issue, memory idle), later all of them waiting for 8-bit and exact tiles
@@ -1399,12 +1424,12 @@ int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_
     L.last_pages = page_idx;
     L.last_n_sel = n_sel;
   } else {
-    if (L.desc_dirty) {
+    if (L.desc_dirty || (observe && L.desc_split)) {      // an observing call needs whole-block units
       // the work lists have their own event: waiting for the table's would wait for copies that
       // the append of this very step has just queued, i.e. drain the stream
       int rc = wait_event(c, L.ev_desc);
       if (rc != GKV_OK) return rc;
-      build_descs(c, L);
+      build_descs(c, L, !observe);
       if ((rc = upload(c, L.warps_d, L.warps_h, static_cast<size_t>(L.n_warps) * sizeof(WarpDesc), st, L.ev_desc)) != GKV_OK) return rc;
       if ((rc = upload(c, L.units_d, L.units_h, static_cast<size_t>(L.n_units) * sizeof(uint32_t), st, L.ev_desc)) != GKV_OK) return rc;
       if ((rc = upload(c, L.parts_d, L.parts_h, static_cast<size_t>(c->n_streams) * sizeof(StreamParts), st, L.ev_desc)) != GKV_OK) return rc;

@@ -276,7 +276,7 @@ struct WarpCtx {
   uint32_t qb_addr;          // this lane's bf16 query fragments in shared memory (16 words)
   uint32_t qh_addr;          // the same in fp16
   // dense mode: this warp's unit list and the prefetched entry of the unit after the current one
-  const uint32_t* units;     // unit = first item | run length << 24
+  const uint32_t* units;     // unit = first item | 16-token tile mask << 20 | run length << 24
   uint32_t pf_unit;
   uint4 pf_entry;
   int pf_pos;
@@ -294,11 +294,11 @@ __device__ __forceinline__ void unit_at(WarpCtx& w, int pos, uint32_t* unit, Tab
     raw = w.pf_entry;
   } else {
     u = w.units[pos];
-    raw = *reinterpret_cast<const uint4*>(w.table + min(static_cast<int>(u & 0xffffffu), w.p->n_closed));
+    raw = *reinterpret_cast<const uint4*>(w.table + min(static_cast<int>(u & kUnitItemMask), w.p->n_closed));
   }
   if (pos + 1 < w.item_end) {
     w.pf_unit = w.units[pos + 1];
-    w.pf_entry = *reinterpret_cast<const uint4*>(w.table + min(static_cast<int>(w.pf_unit & 0xffffffu), w.p->n_closed));
+    w.pf_entry = *reinterpret_cast<const uint4*>(w.table + min(static_cast<int>(w.pf_unit & kUnitItemMask), w.p->n_closed));
     w.pf_pos = pos + 1;
   }
   *unit = u;
@@ -316,7 +316,8 @@ __device__ __forceinline__ bool load_item_dense(WarpCtx& w, int pos, Cursor& c) 
     uint32_t unit;
     TableEntry e;
     unit_at(w, pos, &unit, &e);
-    const int it = static_cast<int>(unit & 0xffffffu), run = static_cast<int>(unit >> 24);
+    const int it = static_cast<int>(unit & kUnitItemMask), run = static_cast<int>(unit >> 24);
+    const int mask = static_cast<int>(unit >> 20) & 15;      // 16-token tiles of the block this unit covers
     c.item = pos;
     c.first = it;
     c.sub = 0;
@@ -337,11 +338,14 @@ __device__ __forceinline__ bool load_item_dense(WarpCtx& w, int pos, Cursor& c) 
           continue;
         }
       }
+      if (it < p.n_closed && c.level == 16) c.tmask = mask;
+      // a unit may cover one half of a quantised block (tile mask 3 or 12): steps [sub, nsub)
+      const int lo = (mask & 3) ? 0 : 1, hi = (mask & 12) ? 2 : 1;
       switch (c.level) {
         case 16: c.nsub = 2 * popc4(c.tmask); break;
-        case 8: c.nsub = 4; break;
-        case 4: c.nsub = 2; break;
-        case 2: c.nsub = 2; break;
+        case 8: c.sub = 2 * lo; c.nsub = 2 * hi; break;
+        case 4: c.sub = lo; c.nsub = hi; break;
+        case 2: c.sub = lo; c.nsub = hi; break;
         default:     // run of up to 16 consecutive centroid blocks (merged by the host)
           c.ntok = run;
           c.nsub = 2;
@@ -937,7 +941,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
   if constexpr (!SPARSE) {
     if (first < w.item_end) {
-      w.pf_entry = *reinterpret_cast<const uint4*>(w.table + min(static_cast<int>(w.pf_unit & 0xffffffu), p.n_closed));
+      w.pf_entry = *reinterpret_cast<const uint4*>(w.table + min(static_cast<int>(w.pf_unit & kUnitItemMask), p.n_closed));
       w.pf_pos = first;
     }
   }

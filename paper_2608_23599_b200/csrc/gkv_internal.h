@@ -28,6 +28,11 @@ struct alignas(16) WarpDesc {
   int32_t partial;     // row of the partial buffer this warp writes
 };
 
+// Unit word of the dense work lists: first item | tile mask << 20 | run length << 24.  The tile
+// mask (four 16-token tiles; 15 = the whole block) lets a unit cover part of a block: any tiles of an
+// exact block, one half (3 or 12) of a quantised one.
+constexpr uint32_t kUnitItemMask = 0xfffffu;
+
 struct alignas(8) StreamParts {
   int32_t begin, end;  // partial rows [begin, end) belong to this stream
 };
