@@ -1086,7 +1086,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   __syncthreads();
   constexpr int kRowFloats = kStages * kStageBytes / 4;     // distance between two warps' rows
   const float* rows = reinterpret_cast<const float*>(smem);
-  const int n_elem = p.group * (kD + 2);
+  const int n_pair = p.group * ((kD + 2) / 2);
   int gb = 0;
 #pragma unroll 1
   while (gb < kDecodeWarps) {
@@ -1109,22 +1109,25 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
           row_end = sp.end;
         }
       }
+      // an element is a pair of floats of the row: (m, l) of a head, or two of its channels
 #pragma unroll 1
-      for (int e = threadIdx.x; e < n_elem; e += kDecodeWarps * 32) {
-        const int h = e / (kD + 2), j = e - h * (kD + 2);
-        // one pass in warp order: running maximum M and the sum relative to it (the loads of the
+      for (int e = threadIdx.x; e < n_pair; e += kDecodeWarps * 32) {
+        const int h = e / ((kD + 2) / 2), j = e - h * ((kD + 2) / 2);
+        // one pass in warp order: running maximum M and the sums relative to it (the loads of the
         // rows do not depend on one another; only the short rescaling chain is serial)
         const float* col = rows + h * (kD + 2);
-        float M = kNegInf, acc = 0.f;
+        float M = kNegInf, acc0 = 0.f, acc1 = 0.f;
 #pragma unroll 2
         for (int i = gb; i < ge; ++i) {
-          const float m = col[i * kRowFloats], v = col[i * kRowFloats + j];
+          const float m = col[i * kRowFloats];
+          const float2 v = *reinterpret_cast<const float2*>(col + i * kRowFloats + 2 * j);
           const float Mn = fmaxf(M, m);
           const float a = (M == kNegInf) ? 0.f : fast_exp2(M - Mn), bwt = (m == kNegInf) ? 0.f : fast_exp2(m - Mn);
-          acc = fmaf(acc, a, v * bwt);
+          acc0 = fmaf(acc0, a, v.x * bwt);
+          acc1 = fmaf(acc1, a, v.y * bwt);
           M = Mn;
         }
-        dst[e] = (j == 0) ? M : acc;
+        *reinterpret_cast<float2*>(dst + h * (kD + 2) + 2 * j) = make_float2(j == 0 ? M : acc0, acc1);
       }
       // The CTA that delivers the stream's last row normalises and writes the output: rows are
       // published with a fence before the ticket is taken, and read back through L2.  Nobody
@@ -1147,24 +1150,27 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
       if (begin >= 0) {
         __threadfence();
         const int b = sid / p.n_kv_heads, kvh = sid - b * p.n_kv_heads;
+        // a thread takes two neighbouring channels of a head
 #pragma unroll 1
-        for (int e = threadIdx.x; e < p.group * kD; e += kDecodeWarps * 32) {
-          const int h = e / kD, ch = e - h * kD;
+        for (int e = threadIdx.x; e < p.group * (kD / 2); e += kDecodeWarps * 32) {
+          const int h = e / (kD / 2), ch = 2 * (e - h * (kD / 2));
           const float* col = p.partial + static_cast<size_t>(begin) * kPartialFloats + h * (kD + 2);
           // one pass in row order (one round of independent loads instead of two dependent ones)
-          float M = kNegInf, L = 0.f, acc = 0.f;
+          float M = kNegInf, L = 0.f, acc0 = 0.f, acc1 = 0.f;
 #pragma unroll 4
           for (int i = 0; i < end - begin; ++i) {
             const float* row = col + static_cast<size_t>(i) * kPartialFloats;
-            const float m = __ldcg(row), l = __ldcg(row + 1), v = __ldcg(row + 2 + ch);
-            const float Mn = fmaxf(M, m);
-            const float a = (M == kNegInf) ? 0.f : exp2f(M - Mn), bwt = (m == kNegInf) ? 0.f : exp2f(m - Mn);
-            L = fmaf(L, a, l * bwt);
-            acc = fmaf(acc, a, v * bwt);
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(row));
+            const float2 v = __ldcg(reinterpret_cast<const float2*>(row + 2 + ch));
+            const float Mn = fmaxf(M, ml.x);
+            const float a = (M == kNegInf) ? 0.f : exp2f(M - Mn), bwt = (ml.x == kNegInf) ? 0.f : exp2f(ml.x - Mn);
+            L = fmaf(L, a, ml.y * bwt);
+            acc0 = fmaf(acc0, a, v.x * bwt);
+            acc1 = fmaf(acc1, a, v.y * bwt);
             M = Mn;
           }
           const size_t hq = static_cast<size_t>(b) * p.n_kv_heads * p.group + static_cast<size_t>(kvh) * p.group + h;
-          p.out[hq * kD + ch] = (L > 0.f) ? acc / L : 0.f;
+          *reinterpret_cast<float2*>(p.out + hq * kD + ch) = (L > 0.f) ? make_float2(acc0 / L, acc1 / L) : make_float2(0.f, 0.f);
           if (p.lse && ch == 0) p.lse[hq] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : kNegInf;
           if constexpr (MASS) {
             if (ch == 0) p.lse2[hq] = (L > 0.f) ? M + log2f(L) : kNegInf;
