@@ -201,15 +201,23 @@ def run_ours(args, rank, local, world):
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     closes = 0
-    for _ in range(K):
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(K)]      # end of every step (per-step times)
+    fill_steps = []
+    for i in range(K):
         step_device(s)
         s += 1
+        marks[i].record()
         if cache.gkv_ctx_len(0) % 64 == 0:
             closes += 1
+            fill_steps.append(i)
     ev1.record()
     barrier(world)
     clocks = sampler.stop()
     ms_step = max_over_ranks(ev0.elapsed_time(ev1) / K, world)
+    per_step = [(ev0 if i == 0 else marks[i - 1]).elapsed_time(marks[i]) for i in range(K)]
+    plain = sorted(t for i, t in enumerate(per_step) if i not in fill_steps)
+    step_detail = {"ms_median_step_without_block_fill": plain[len(plain) // 2] if plain else None,
+                   "ms_block_fill_steps": [per_step[i] for i in fill_steps]}
     value = aggregate_value(world, Bsz, ctx_start, ms_step)
 
     # ---- dominant kernel: decode_attn alone, per launch -------------------------------------------
@@ -314,6 +322,11 @@ def run_ours(args, rank, local, world):
                      "us_per_launch": us_launch, "algorithmic_bytes_per_launch": algo_bytes,
                      "frac_of_8TBs": achieved / NOMINAL_HBM_GBS},
         "ctx_tokens_per_s_per_layer_call": Bsz * ctx_start / (us_launch * 1e-6),
+        # gkv_append_demote next to gkv_decode_attn: what a layer's append adds to its decode call in a
+        # plain step, and the steps in which a block fills (close, demotions, new work lists)
+        "append_demote": {"us_per_layer_in_plain_step": (step_detail["ms_median_step_without_block_fill"] or ms_step) * 1e3 / n_layers
+                          - us_launch - (scorer["us_per_call"] if scorer else 0.0),
+                          **step_detail},
     }
     if scorer:
         line["quest_select"] = scorer
