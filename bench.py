@@ -324,8 +324,8 @@ def run_ours(args, rank, local, world):
         "ctx_tokens_per_s_per_layer_call": Bsz * ctx_start / (us_launch * 1e-6),
         # gkv_append_demote next to gkv_decode_attn: what a layer's append adds to its decode call in a
         # plain step, and the steps in which a block fills (close, demotions, new work lists)
-        "append_demote": {"us_per_layer_in_plain_step": (step_detail["ms_median_step_without_block_fill"] or ms_step) * 1e3 / n_layers
-                          - us_launch - (scorer["us_per_call"] if scorer else 0.0),
+        "append_demote": {"us_per_layer_in_plain_step": max(0.0, (step_detail["ms_median_step_without_block_fill"] or ms_step) * 1e3 / n_layers
+                                                             - us_launch - (scorer["us_per_call"] if scorer else 0.0)),
                           **step_detail},
     }
     if scorer:
