@@ -116,6 +116,23 @@ def test_cfg2_full_size_sampled_streams_with_appends():
     for j in range(len(streams)):
         for blk in ocache.streams[(0, 0, j)].blocks:
             assert all(a >= b for a, b in zip(blk.history, blk.history[1:]))      # monotone demotion
+    # the observing call at full size: same output bits, block masses and certificate of the sampled streams
+    n_items = (gcache.gkv_ctx_len(0) + 63) // 64
+    mass = torch.full((w.batch, w.n_kv_heads, n_items), -1.0, dtype=torch.float32, device=dev)
+    cert = torch.full((w.batch, w.n_q_heads), -1.0, dtype=torch.float32, device=dev)
+    out2 = torch.empty_like(out)
+    gcache.gkv_decode_attn_observe(0, qn, out2, None, mass, cert)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+    mass_h, cert_h = mass.cpu().numpy().astype(np.float64), cert.cpu().numpy().astype(np.float64)
+    assert np.all(mass_h >= 0) and np.allclose(mass_h.sum(-1), 1.0, atol=2e-3)
+    assert np.all(np.isfinite(cert_h)) and np.all(cert_h > 0)
+    _, _, o_obs = ocache.decode_attn_observe(0, U.f32(qs))
+    o_cert = ocache.certificate(0, U.f32(qs))
+    for j, (b, h) in enumerate(streams):
+        want = o_obs[(0, j)]
+        assert np.allclose(mass_h[b, h], want, rtol=1e-2, atol=2e-6), (b, h, float(np.abs(mass_h[b, h] - want).max()))
+        assert np.allclose(cert_h[b, h * 4:(h + 1) * 4], o_cert[0, j * 4:(j + 1) * 4], rtol=1e-2, atol=1e-5)
     gcache.close()
 
 
