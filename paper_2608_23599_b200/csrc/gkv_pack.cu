@@ -156,14 +156,18 @@ __global__ void __launch_bounds__(256) encode_kernel(const __grid_constant__ Enc
   float* pz = ps + 256;                                              // [256] zero points
   float* red = pz + 256;                                             // [16] per-warp maxima
   const int tid = threadIdx.x;
-  for (int j = blockIdx.x; j < p.n_jobs; j += gridDim.x) {
-    const EncodeJob job = p.jobs[j];
+  // a work item is one tensor (keys or values) of one job: the two halves of a job are independent
+  // (separate regions of the slot, separate components of the error bounds) and run in different CTAs
+  for (int item = blockIdx.x; item < 2 * p.n_jobs; item += gridDim.x) {
+    const EncodeJob job = p.jobs[item >> 1];
     uint8_t* dst = p.arena + static_cast<size_t>(job.dst_off256) * 256;
     const int L = job.dst_level;
     const bool from_original = job.src_level == 0 || job.src_level == 16;
+    float* bound_out = p.err ? reinterpret_cast<float*>(p.err + static_cast<size_t>(job.stream) * p.err_stride + job.block) : nullptr;
     float4 bound = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (p.err && !from_original && tid == 0) bound = p.err[static_cast<size_t>(job.stream) * p.err_stride + job.block];
-    for (int tensor = 0; tensor < 2; ++tensor) {
+    if (p.err && !from_original && tid == 0) bound = *reinterpret_cast<const float4*>(bound_out);
+    {
+      const int tensor = item & 1;
       const bool is_v = tensor == 1;
       __syncthreads();
       load_tile(tile, p.arena, p, job, is_v);
@@ -278,8 +282,16 @@ __global__ void __launch_bounds__(256) encode_kernel(const __grid_constant__ Enc
         }
       }
     }
-    if (p.err && tid == 0) p.err[static_cast<size_t>(job.stream) * p.err_stride + job.block] = bound;
-    if (p.table && tid == 0) {
+    if (p.err && tid == 0) {
+      if ((item & 1) == 0) {
+        bound_out[0] = bound.x;            // keys: x
+      } else {
+        bound_out[1] = bound.y;            // values: y, z; w stays 0
+        bound_out[2] = bound.z;
+        bound_out[3] = 0.f;
+      }
+    }
+    if (p.table && tid == 0 && (item & 1) == 0) {
       TableEntry* te = p.table + static_cast<size_t>(job.stream) * p.table_stride + job.block;
       te->off256 = job.dst_off256;
       te->level = static_cast<uint32_t>(job.dst_level);
@@ -305,23 +317,36 @@ __global__ void __launch_bounds__(kD) stats_kernel(const __grid_constant__ Stats
   }
   float bmn = 0.f, bmx = 0.f;
   const int page = p.page_tokens > 0 ? p.page_tokens : kBlock;
-  for (int p0 = 0; p0 < kBlock; p0 += page) {
-    uint16_t lo_b = rows[static_cast<size_t>(p0) * row_stride + c], hi_b = lo_b;
-    float lo = bf16_bits_to_f32(lo_b), hi = lo;
-    for (int t = 1; t < page; ++t) {
-      const uint16_t xb = rows[static_cast<size_t>(p0 + t) * row_stride + c];
-      const float x = bf16_bits_to_f32(xb);
-      if (x < lo) { lo = x; lo_b = xb; }
-      if (x > hi) { hi = x; hi_b = xb; }
+  // The block's 64 values of this channel are fetched 16 at a time (independent loads, issued
+  // together) and folded into the running page minimum / maximum; a page is 16, 32 or 64 tokens.
+  uint16_t lo_b = 0, hi_b = 0;
+  float lo = 0.f, hi = 0.f;
+#pragma unroll 1
+  for (int t0 = 0; t0 < kBlock; t0 += 16) {
+    uint16_t xb[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) xb[i] = rows[static_cast<size_t>(t0 + i) * row_stride + c];
+    if (t0 % page == 0) {
+      lo_b = hi_b = xb[0];
+      lo = hi = bf16_bits_to_f32(xb[0]);
     }
-    if (p.page_tokens > 0) {
-      const int pg = block * (kBlock / page) + p0 / page;
-      uint16_t* bx = p.boxes + (static_cast<size_t>(stream) * kD + c) * 2 * p.box_stride;
-      bx[pg] = lo_b;
-      bx[p.box_stride + pg] = hi_b;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float x = bf16_bits_to_f32(xb[i]);
+      if (x < lo) { lo = x; lo_b = xb[i]; }
+      if (x > hi) { hi = x; hi_b = xb[i]; }
     }
-    if (p0 == 0) { bmn = lo; bmx = hi; }
-    else { bmn = fminf(bmn, lo); bmx = fmaxf(bmx, hi); }
+    if ((t0 + 16) % page == 0) {                       // the page is complete
+      const int p0 = t0 + 16 - page;
+      if (p.page_tokens > 0) {
+        const int pg = block * (kBlock / page) + p0 / page;
+        uint16_t* bx = p.boxes + (static_cast<size_t>(stream) * kD + c) * 2 * p.box_stride;
+        bx[pg] = lo_b;
+        bx[p.box_stride + pg] = hi_b;
+      }
+      if (p0 == 0) { bmn = lo; bmx = hi; }
+      else { bmn = fminf(bmn, lo); bmx = fmaxf(bmx, hi); }
+    }
   }
   if (p.block_range) {
     __shared__ float red[kD];
@@ -487,7 +512,7 @@ cudaError_t launch_encode(const EncodeParams& p, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  const int grid = p.n_jobs < 148 * 16 ? p.n_jobs : 148 * 16;
+  const int grid = 2 * p.n_jobs < 148 * 16 ? 2 * p.n_jobs : 148 * 16;
   encode_kernel<<<grid, 256, smem, st>>>(p);
   return cudaGetLastError();
 }
