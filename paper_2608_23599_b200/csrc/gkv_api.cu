@@ -712,8 +712,11 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
   if (n_jobs > 0) {
     EncodeJob* jobs = reinterpret_cast<EncodeJob*>(stage + stage_off);
     size_t j = 0;
-    for (int s = 0; s < ns; ++s)
-      for (int b = 0; b < n_closed; ++b) {
+    // order (sequence, block, KV head): CTAs that run at the same time read neighbouring rows
+    for (int sq = 0; sq < cfg.batch; ++sq)
+      for (int b = 0; b < n_closed; ++b)
+        for (int kvh = 0; kvh < cfg.n_kv_heads; ++kvh) {
+        const int s = sq * cfg.n_kv_heads + kvh;
         EncodeJob& job = jobs[j++];
         job.src_off256 = 0;
         job.dst_off256 = L.table_h[static_cast<size_t>(s) * c->table_stride + b].off256;
@@ -735,7 +738,9 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
     ep.status = c->status_d;
     ep.err = L.err_d;
     ep.err_stride = c->max_blocks;
-    CK(c, launch_encode(ep, st));
+    const bool aligned = ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new)) & 15u) == 0;
+    if (aligned && v_new) CK(c, launch_ingest(ep, st));
+    else CK(c, launch_encode(ep, st));
   }
   CK(c, cudaEventRecord(c->ev_stage, st));
   CK(c, launch_append_rows(c->arena, L.table_d, c->table_stride, n_closed, ns, cfg.n_kv_heads, k_new, v_new, n_new,

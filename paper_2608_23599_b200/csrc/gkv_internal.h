@@ -169,6 +169,7 @@ cudaError_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t st);
 cudaError_t launch_mass_finish(const MassFinishParams& p, cudaStream_t st);
 cudaError_t launch_certificate(const CertificateParams& p, cudaStream_t st);
 cudaError_t launch_encode(const EncodeParams& p, cudaStream_t st);
+cudaError_t launch_ingest(const EncodeParams& p, cudaStream_t st);   // every job reads the bf16 input rows; 16-byte aligned inputs
 cudaError_t launch_stats(const StatsParams& p, cudaStream_t st);
 cudaError_t launch_append_rows(uint8_t* arena, const TableEntry* table, int table_stride, int tail_index,
                                int n_streams, int n_kv_heads, const uint16_t* k_in, const uint16_t* v_in,
