@@ -30,7 +30,7 @@ constexpr int kInRow = kRowBytes + 16;            // padded shared-memory row: l
 constexpr int kInTensor = kBlock * kInRow;        // 17408
 constexpr int kInBuf = 2 * kInTensor;             // keys, values
 constexpr int kInThreads = 256;
-constexpr int kInSmem = 2 * kInBuf + (256 + 128 + 16) * static_cast<int>(sizeof(float));
+constexpr int kInSmem = 2 * kInBuf + (256 + 128 + 16) * static_cast<int>(sizeof(float)) + 8 * 32 * 16;   // + the warps' group parameters
 constexpr float kMagic = 12582912.f;              // 1.5 * 2^23: x + kMagic rounds x to an integer (ties to even)
 constexpr uint32_t kMagicBits = 0x4B400000u;
 constexpr uint32_t kFullI = 0xffffffffu;
@@ -114,87 +114,96 @@ __device__ __forceinline__ void i_quant2(uint32_t x, float s0, float z0, float i
   e1 = fmaf(d1, d1, e1);
 }
 
-// Keys of one half (32 tokens) x 64 channels: x[tile of the half][slice][a].  Groups are 32 tokens of
-// one channel: the lane's registers (tile, a & 1) and the eight lanes of a column (r = lane >> 2).
-// Pair k = 2 * slice + (a >> 1) names the lane's two channels 16 s + 8 (a >> 1) + 2 c4 + {0, 1}.
-// e[tile][a & 1][0 / 1]: squared error of token 16 tile + 8 (a & 1) + r over the lane's channels;
-// the two halves of a pair are summed at the end.
+// Parameters of a group as the warp keeps them in shared memory between its two passes:
+// {scale | zero << 16 (fp16 bits), reciprocal} of the low and of the high half of a register pair.
+__device__ __forceinline__ uint4 i_pack_params(const GroupParams& g0, const GroupParams& g1) {
+  return make_uint4(static_cast<uint32_t>(g0.s_bits) | (static_cast<uint32_t>(g0.z_bits) << 16), __float_as_uint(g0.inv),
+                    static_cast<uint32_t>(g1.s_bits) | (static_cast<uint32_t>(g1.z_bits) << 16), __float_as_uint(g1.inv));
+}
+__device__ __forceinline__ float i_h_lo(uint32_t u) { return __half2float(__ushort_as_half(static_cast<unsigned short>(u & 0xffffu))); }
+__device__ __forceinline__ float i_h_hi(uint32_t u) { return __half2float(__ushort_as_half(static_cast<unsigned short>(u >> 16))); }
+
+// Keys of one half (32 tokens) x 64 channels.  ldmatrix hands a lane, per 16-token tile and slice of
+// 16 channels, registers a = 0..3: token 8 (a & 1) + r, channels 16 s + 8 (a >> 1) + 2 c4 + {0, 1}
+// (r = lane >> 2, c4 = lane & 3).  Groups are 32 tokens of one channel: the lane's registers
+// (tile, a & 1) and the eight lanes r.  Pair k = 2 * slice + (a >> 1) names the lane's two channels.
+// Pass 1 finds the extremes of every pair, lane r works out the parameters of pair r; pass 2 reads
+// the rows again, quantises and stores whole words.  Both passes are rolled loops over the slices
+// (the code of all rungs together has to stay inside the instruction cache).
+// e[tile][a & 1]: squared error of token 16 tile + 8 (a & 1) + r summed over the lane's channels.
 template <int BITS>
-__device__ __forceinline__ bool ingest_keys(const uint32_t (&x)[2][4][4], uint8_t* half_base, int chh, int lane, float (&e)[2][2]) {
-  const int r = lane >> 2, c4 = lane & 3;
-  uint32_t mn[8], mx[8];
+__device__ __forceinline__ bool ingest_keys(uint32_t tile_k, uint8_t* half_base, int half, int chh, int lane, uint4* prm, float (&e)[2][2]) {
+  const int r = lane >> 2, c4 = lane & 3, mi = lane >> 3;
+  const uint32_t ld = tile_k + (32 * half + (mi & 1) * 8 + (lane & 7)) * kInRow + (64 * chh + (mi >> 1) * 8) * 2;
+  uint32_t my_mn = 0u, my_mx = 0u;
+#pragma unroll 1
+  for (int sl = 0; sl < 4; ++sl) {
+    uint32_t x0[4], x1[4];
+    i_ldm4(ld + sl * 32, x0);
+    i_ldm4(ld + 16 * kInRow + sl * 32, x1);
 #pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    const int sl = k >> 1, ah = k & 1;
-    mn[k] = i_min2(i_min2(x[0][sl][2 * ah], x[0][sl][2 * ah + 1]), i_min2(x[1][sl][2 * ah], x[1][sl][2 * ah + 1]));
-    mx[k] = i_max2(i_max2(x[0][sl][2 * ah], x[0][sl][2 * ah + 1]), i_max2(x[1][sl][2 * ah], x[1][sl][2 * ah + 1]));
+    for (int ah = 0; ah < 2; ++ah) {
+      uint32_t mn = i_min2(i_min2(x0[2 * ah], x0[2 * ah + 1]), i_min2(x1[2 * ah], x1[2 * ah + 1]));
+      uint32_t mx = i_max2(i_max2(x0[2 * ah], x0[2 * ah + 1]), i_max2(x1[2 * ah], x1[2 * ah + 1]));
 #pragma unroll
-    for (int d = 4; d <= 16; d <<= 1) {
-      mn[k] = i_min2(mn[k], __shfl_xor_sync(kFullI, mn[k], d));
-      mx[k] = i_max2(mx[k], __shfl_xor_sync(kFullI, mx[k], d));
-    }
-  }
-  // lane r works out the parameters of pair r
-  uint32_t my_mn = mn[0], my_mx = mx[0];
-#pragma unroll
-  for (int k = 1; k < 8; ++k) {
-    if (r == k) {
-      my_mn = mn[k];
-      my_mx = mx[k];
+      for (int d = 4; d <= 16; d <<= 1) {
+        mn = i_min2(mn, __shfl_xor_sync(kFullI, mn, d));
+        mx = i_max2(mx, __shfl_xor_sync(kFullI, mx, d));
+      }
+      if (r == 2 * sl + ah) {
+        my_mn = mn;
+        my_mx = mx;
+      }
     }
   }
   const GroupParams g0 = i_params<BITS>(i_lo(my_mn), i_lo(my_mx)), g1 = i_params<BITS>(i_hi(my_mn), i_hi(my_mx));
   {
-    // record [slice][c4] = {scale c0, scale c1, zero c0, zero c1, scale c0 + 8, scale c1 + 8, zero c0 + 8, zero c1 + 8}
+    // record [slice][c4] = {scale c0, scale c1, zero c0, zero c1, then the same for c0 + 8, c1 + 8}
     const int s_glob = 4 * chh + (r >> 1);
     uint2 rec;
     rec.x = static_cast<uint32_t>(g0.s_bits) | (static_cast<uint32_t>(g1.s_bits) << 16);
     rec.y = static_cast<uint32_t>(g0.z_bits) | (static_cast<uint32_t>(g1.z_bits) << 16);
     *reinterpret_cast<uint2*>(half_base + off_kp() + (s_glob * 4 + c4) * 16 + (r & 1) * 8) = rec;
   }
-  float e00 = 0.f, e01 = 0.f, e10 = 0.f, e11 = 0.f;      // [tile][a & 1], low halves
-  float f00 = 0.f, f01 = 0.f, f10 = 0.f, f11 = 0.f;      // high halves
-  uint32_t w[2][4];
+  prm[r * 4 + c4] = i_pack_params(g0, g1);
+  __syncwarp();
+  constexpr int SL = BITS == 2 ? 2 : 1;             // slices that fill whole words
+  constexpr uint32_t kOff = BITS == 8 ? 0x01010101u : (BITS == 4 ? 0x11111111u : 0x55555555u);
+  float e00 = 0.f, e01 = 0.f, e10 = 0.f, e11 = 0.f, f00 = 0.f, f01 = 0.f, f10 = 0.f, f11 = 0.f;
+#pragma unroll 1
+  for (int u = 0; u < 4 / SL; ++u) {
+    uint32_t w[2][2] = {{0u, 0u}, {0u, 0u}};        // [tile][word]: 8 bits: one word per a >> 1; else one word
 #pragma unroll
-  for (int t = 0; t < 2; ++t)
+    for (int ss = 0; ss < SL; ++ss) {
+      const int sl = u * SL + ss;
+      uint32_t x[2][4];
+      i_ldm4(ld + sl * 32, x[0]);
+      i_ldm4(ld + 16 * kInRow + sl * 32, x[1]);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) w[t][i] = 0u;
+      for (int ah = 0; ah < 2; ++ah) {
+        const uint4 P = prm[(2 * sl + ah) * 4 + c4];
+        const float s0 = i_h_lo(P.x), z0 = i_h_hi(P.x), v0 = __uint_as_float(P.y);
+        const float s1 = i_h_lo(P.z), z1 = i_h_hi(P.z), v1 = __uint_as_float(P.w);
+        const int wi = BITS == 8 ? ah : 0;
 #pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    const int sl = k >> 1, ah = k & 1, src = 4 * k + c4;
-    const float s0 = __shfl_sync(kFullI, g0.s, src), z0 = __shfl_sync(kFullI, g0.z, src), v0 = __shfl_sync(kFullI, g0.inv, src);
-    const float s1 = __shfl_sync(kFullI, g1.s, src), z1 = __shfl_sync(kFullI, g1.z, src), v1 = __shfl_sync(kFullI, g1.inv, src);
-    // word index inside the lane's words of a tile: 8 bits: 2 sl + ah (8 words), 4 bits: sl (4), 2 bits: sl >> 1 (2)
-    const int wi = BITS == 8 ? (2 * sl + ah) & 3 : (BITS == 4 ? sl : sl >> 1);
+        for (int t = 0; t < 2; ++t) {
+          i_quant2<BITS>(x[t][2 * ah], s0, z0, v0, s1, z1, v1, i_bit<BITS>(ss, 2 * ah, 0), i_bit<BITS>(ss, 2 * ah, 1), w[t][wi],
+                         t == 0 ? e00 : e10, t == 0 ? f00 : f10);
+          i_quant2<BITS>(x[t][2 * ah + 1], s0, z0, v0, s1, z1, v1, i_bit<BITS>(ss, 2 * ah + 1, 0), i_bit<BITS>(ss, 2 * ah + 1, 1),
+                         w[t][wi], t == 0 ? e01 : e11, t == 0 ? f01 : f11);
+        }
+      }
+    }
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
-      i_quant2<BITS>(x[t][sl][2 * ah], s0, z0, v0, s1, z1, v1, i_bit<BITS>(sl, 2 * ah, 0), i_bit<BITS>(sl, 2 * ah, 1), w[t][wi],
-                     t == 0 ? e00 : e10, t == 0 ? f00 : f10);
-      i_quant2<BITS>(x[t][sl][2 * ah + 1], s0, z0, v0, s1, z1, v1, i_bit<BITS>(sl, 2 * ah + 1, 0), i_bit<BITS>(sl, 2 * ah + 1, 1),
-                     w[t][wi], t == 0 ? e01 : e11, t == 0 ? f01 : f11);
-    }
-    // a group of words is complete: take the magic constants off and store
-    const bool flush = BITS == 8 ? (k & 3) == 3 : k == 7;
-    if (flush) {
-#pragma unroll
-      for (int t = 0; t < 2; ++t) {
-        uint8_t* codes = half_base + off_kc(BITS, t);
-        if (BITS == 8) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) w[t][i] -= kMagicBits * 0x01010101u;
-          const int chunk = 2 * chh + (k >> 2);
-          *reinterpret_cast<uint4*>(codes + (chunk * 32 + lane) * 16) = make_uint4(w[t][0], w[t][1], w[t][2], w[t][3]);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) w[t][i] = 0u;
-        } else if (BITS == 4) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) w[t][i] -= kMagicBits * 0x11111111u;
-          *reinterpret_cast<uint4*>(codes + (chh * 32 + lane) * 16) = make_uint4(w[t][0], w[t][1], w[t][2], w[t][3]);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 2; ++i) w[t][i] -= kMagicBits * 0x55555555u;
-          *reinterpret_cast<uint2*>(codes + lane * 16 + chh * 8) = make_uint2(w[t][0], w[t][1]);
-        }
+      uint8_t* codes = half_base + off_kc(BITS, t);
+      if (BITS == 8) {          // words 8 chh + 2 u + {0, 1}
+        *reinterpret_cast<uint2*>(codes + ((2 * chh + (u >> 1)) * 32 + lane) * 16 + (u & 1) * 8) =
+            make_uint2(w[t][0] - kMagicBits * kOff, w[t][1] - kMagicBits * kOff);
+      } else if (BITS == 4) {   // word 4 chh + u
+        *reinterpret_cast<uint32_t*>(codes + (chh * 32 + lane) * 16 + u * 4) = w[t][0] - kMagicBits * kOff;
+      } else {                  // word 2 chh + u
+        *reinterpret_cast<uint32_t*>(codes + lane * 16 + chh * 8 + u * 4) = w[t][0] - kMagicBits * kOff;
       }
     }
   }
@@ -205,73 +214,97 @@ __device__ __forceinline__ bool ingest_keys(const uint32_t (&x)[2][4][4], uint8_
   return g0.range || g1.range;
 }
 
-// Values of one tile (16 tokens) x 128 channels: x[slice][a], channel 16 s + r + 8 (a & 1), token
-// 8 (a >> 1) + 2 c4 + {0, 1}.  Groups are 32 channels of one token: slices 2 g and 2 g + 1, a & 1 and the
-// eight lanes r.  Pair k = 2 g + (a >> 1) names the lane's tokens 8 (a >> 1) + 2 c4 + {0, 1} in group g.
-// e[a >> 1][0 / 1]: squared error of token 8 (a >> 1) + 2 c4 + {0, 1} over the lane's channels.
+// Values of one tile (16 tokens) x 128 channels.  ldmatrix.trans hands a lane, per slice of 16
+// channels, registers a = 0..3: channel 16 s + r + 8 (a & 1), tokens 8 (a >> 1) + 2 c4 + {0, 1}.  Groups
+// are 32 channels of one token: slices 2 g and 2 g + 1, a & 1 and the eight lanes r.  Pair
+// k = 2 g + (a >> 1) names the lane's two tokens in group g.
+// e[a >> 1][0 / 1], n[a >> 1][0 / 1]: squared error / squared norm of token 8 (a >> 1) + 2 c4 + {0, 1}
+// summed over the lane's channels.
 template <int BITS>
-__device__ __forceinline__ bool ingest_values(const uint32_t (&x)[8][4], uint8_t* vp, uint8_t* codes, int lane, float (&e)[2][2]) {
+__device__ __forceinline__ bool ingest_values(uint32_t ld, uint8_t* vp, uint8_t* codes, int lane, uint4* prm, float (&e)[2][2],
+                                              float (&n)[2][2]) {
   const int r = lane >> 2, c4 = lane & 3;
-  uint32_t mn[8], mx[8];
+  uint32_t my_mn = 0u, my_mx = 0u;
+#pragma unroll 1
+  for (int g = 0; g < 4; ++g) {
+    uint32_t x0[4], x1[4];
+    i_ldm4t(ld + g * 64, x0);
+    i_ldm4t(ld + g * 64 + 32, x1);
 #pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    const int g = k >> 1, ah = k & 1;
-    mn[k] = i_min2(i_min2(x[2 * g][2 * ah], x[2 * g][2 * ah + 1]), i_min2(x[2 * g + 1][2 * ah], x[2 * g + 1][2 * ah + 1]));
-    mx[k] = i_max2(i_max2(x[2 * g][2 * ah], x[2 * g][2 * ah + 1]), i_max2(x[2 * g + 1][2 * ah], x[2 * g + 1][2 * ah + 1]));
+    for (int ah = 0; ah < 2; ++ah) {
+      uint32_t mn = i_min2(i_min2(x0[2 * ah], x0[2 * ah + 1]), i_min2(x1[2 * ah], x1[2 * ah + 1]));
+      uint32_t mx = i_max2(i_max2(x0[2 * ah], x0[2 * ah + 1]), i_max2(x1[2 * ah], x1[2 * ah + 1]));
 #pragma unroll
-    for (int d = 4; d <= 16; d <<= 1) {
-      mn[k] = i_min2(mn[k], __shfl_xor_sync(kFullI, mn[k], d));
-      mx[k] = i_max2(mx[k], __shfl_xor_sync(kFullI, mx[k], d));
-    }
-  }
-  uint32_t my_mn = mn[0], my_mx = mx[0];
-#pragma unroll
-  for (int k = 1; k < 8; ++k) {
-    if (r == k) {
-      my_mn = mn[k];
-      my_mx = mx[k];
+      for (int d = 4; d <= 16; d <<= 1) {
+        mn = i_min2(mn, __shfl_xor_sync(kFullI, mn, d));
+        mx = i_max2(mx, __shfl_xor_sync(kFullI, mx, d));
+      }
+      if (r == 2 * g + ah) {
+        my_mn = mn;
+        my_mx = mx;
+      }
     }
   }
   const GroupParams g0 = i_params<BITS>(i_lo(my_mn), i_lo(my_mx)), g1 = i_params<BITS>(i_hi(my_mn), i_hi(my_mx));
   {
-    // scales [c4][group] = {tA0, tA1, tB0, tB1}, zeros [group][c4] likewise at fp16 index 64; pair r = (group, a >> 1)
+    // scales [c4][group] = {tA0, tA1, tB0, tB1}, zeros [group][c4] likewise from fp16 index 64; pair r = (group, a >> 1)
     const int g = r >> 1, ah = r & 1;
     uint16_t* p16 = reinterpret_cast<uint16_t*>(vp);
     *reinterpret_cast<uint32_t*>(p16 + (c4 * 4 + g) * 4 + ah * 2) = static_cast<uint32_t>(g0.s_bits) | (static_cast<uint32_t>(g1.s_bits) << 16);
     *reinterpret_cast<uint32_t*>(p16 + 64 + (g * 4 + c4) * 4 + ah * 2) = static_cast<uint32_t>(g0.z_bits) | (static_cast<uint32_t>(g1.z_bits) << 16);
   }
-  float e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f;      // [a >> 1][hlf]
-  uint32_t w[4] = {0u, 0u, 0u, 0u};
+  prm[r * 4 + c4] = i_pack_params(g0, g1);
+  __syncwarp();
+  constexpr uint32_t kOff = BITS == 8 ? 0x01010101u : (BITS == 4 ? 0x11111111u : 0x55555555u);
+  float e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f, n0 = 0.f, n1 = 0.f, n2 = 0.f, n3 = 0.f;
+#pragma unroll 1
+  for (int g = 0; g < 4; ++g) {
+    uint32_t x[2][4];
+    i_ldm4t(ld + g * 64, x[0]);
+    i_ldm4t(ld + g * 64 + 32, x[1]);
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    const int g = k >> 1, ah = k & 1, src = 4 * k + c4;
-    const float s0 = __shfl_sync(kFullI, g0.s, src), z0 = __shfl_sync(kFullI, g0.z, src), v0 = __shfl_sync(kFullI, g0.inv, src);
-    const float s1 = __shfl_sync(kFullI, g1.s, src), z1 = __shfl_sync(kFullI, g1.z, src), v1 = __shfl_sync(kFullI, g1.inv, src);
+    for (int ah = 0; ah < 2; ++ah) {
+      const uint4 P = prm[(2 * g + ah) * 4 + c4];
+      const float s0 = i_h_lo(P.x), z0 = i_h_hi(P.x), v0 = __uint_as_float(P.y);
+      const float s1 = i_h_lo(P.z), z1 = i_h_hi(P.z), v1 = __uint_as_float(P.w);
 #pragma unroll
-    for (int ss = 0; ss < 2; ++ss) {
-      const int s = 2 * g + ss;
-      // word of (s, a): 8 bits: 2 s + ah, 4 bits: s, 2 bits: s >> 1; index inside the 16-byte chunk being filled
-      const int wi = BITS == 8 ? (2 * s + ah) & 3 : (BITS == 4 ? s & 3 : s >> 1);
+      for (int ss = 0; ss < 2; ++ss) {
+        // word of (slice 2 g + ss, a): 8 bits: 4 g + 2 ss + (a >> 1), 4 bits: 2 g + ss, 2 bits: g
+        const int wi = BITS == 8 ? 2 * ss + ah : (BITS == 4 ? ss : 0);
 #pragma unroll
-      for (int al = 0; al < 2; ++al)
-        i_quant2<BITS>(x[s][2 * ah + al], s0, z0, v0, s1, z1, v1, i_bit<BITS>(s, 2 * ah + al, 0), i_bit<BITS>(s, 2 * ah + al, 1), w[wi],
-                       ah == 0 ? e0 : e2, ah == 0 ? e1 : e3);
+        for (int al = 0; al < 2; ++al) {
+          const uint32_t xv = x[ss][2 * ah + al];
+          i_quant2<BITS>(xv, s0, z0, v0, s1, z1, v1, i_bit<BITS>(ss, 2 * ah + al, 0), i_bit<BITS>(ss, 2 * ah + al, 1), w[wi],
+                         ah == 0 ? e0 : e2, ah == 0 ? e1 : e3);
+          const float x0f = i_lo(xv), x1f = i_hi(xv);
+          if (ah == 0) {
+            n0 = fmaf(x0f, x0f, n0);
+            n1 = fmaf(x1f, x1f, n1);
+          } else {
+            n2 = fmaf(x0f, x0f, n2);
+            n3 = fmaf(x1f, x1f, n3);
+          }
+        }
+      }
     }
-    const bool flush = BITS == 8 ? ah == 1 : (BITS == 4 ? (k & 3) == 3 : k == 7);
-    if (flush) {
-      constexpr uint32_t kOff = BITS == 8 ? 0x01010101u : (BITS == 4 ? 0x11111111u : 0x55555555u);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) w[i] -= kMagicBits * kOff;
-      const int chunk = BITS == 8 ? g : (BITS == 4 ? g >> 1 : 0);
-      *reinterpret_cast<uint4*>(codes + (chunk * 32 + lane) * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) w[i] = 0u;
+    if (BITS == 8) {
+      *reinterpret_cast<uint4*>(codes + (g * 32 + lane) * 16) =
+          make_uint4(w[0] - kMagicBits * kOff, w[1] - kMagicBits * kOff, w[2] - kMagicBits * kOff, w[3] - kMagicBits * kOff);
+    } else if (BITS == 4) {
+      *reinterpret_cast<uint2*>(codes + ((g >> 1) * 32 + lane) * 16 + (g & 1) * 8) = make_uint2(w[0] - kMagicBits * kOff, w[1] - kMagicBits * kOff);
+    } else {
+      *reinterpret_cast<uint32_t*>(codes + lane * 16 + g * 4) = w[0] - kMagicBits * kOff;
     }
   }
   e[0][0] = e0;
   e[0][1] = e1;
   e[1][0] = e2;
   e[1][1] = e3;
+  n[0][0] = n0;
+  n[0][1] = n1;
+  n[1][0] = n2;
+  n[1][1] = n3;
   return g0.range || g1.range;
 }
 
@@ -280,8 +313,10 @@ __global__ void __launch_bounds__(kInThreads, 3) ingest_kernel(const __grid_cons
   float* cen = reinterpret_cast<float*>(ism + 2 * kInBuf);      // [2][128] centroid of keys, of values
   float* kd2 = cen + 256;                                       // [2 channel halves][64 tokens]
   float* red = kd2 + 128;                                       // [4 value warps][2]: max error, max norm (squared)
+  uint4* prm_all = reinterpret_cast<uint4*>(red + 16);          // [8 warps][8 pairs][4 lanes c4]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int r = lane >> 2, c4 = lane & 3;
+  const int r = lane >> 2, c4 = lane & 3, mi = lane >> 3;
+  uint4* prm = prm_all + warp * 32;
   const uint32_t sbase = i_u32(ism);
   const size_t row_stride = static_cast<size_t>(p.n_kv_heads) * kD;      // elements between two tokens of a stream
 
@@ -340,34 +375,30 @@ __global__ void __launch_bounds__(kInThreads, 3) ingest_kernel(const __grid_cons
       // ---- keys: warp = (half of the block, half of the channels) ----
       const int half = warp >> 1, chh = warp & 1;
       float e[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-      if (L != 16) {
-        uint32_t x[2][4][4];
-        const int mi = lane >> 3;
+      uint8_t* half_base = dst + half * half_bytes(L);
+      if (L == 8) range = ingest_keys<8>(tile_s, half_base, half, chh, lane, prm, e);
+      else if (L == 4) range = ingest_keys<4>(tile_s, half_base, half, chh, lane, prm, e);
+      else if (L == 2) range = ingest_keys<2>(tile_s, half_base, half, chh, lane, prm, e);
+      else if (L == 1) {
+        // distance from the centroid
+        const uint32_t ld = tile_s + (32 * half + (mi & 1) * 8 + (lane & 7)) * kInRow + (64 * chh + (mi >> 1) * 8) * 2;
+#pragma unroll 1
+        for (int sl = 0; sl < 4; ++sl) {
+          uint32_t x[2][4];
+          i_ldm4(ld + sl * 32, x[0]);
+          i_ldm4(ld + 16 * kInRow + sl * 32, x[1]);
 #pragma unroll
-        for (int t = 0; t < 2; ++t)
+          for (int ah = 0; ah < 2; ++ah) {
+            const float2 cc = *reinterpret_cast<const float2*>(cen + 64 * chh + 16 * sl + 8 * ah + 2 * c4);
 #pragma unroll
-          for (int sl = 0; sl < 4; ++sl)
-            i_ldm4(tile_s + (32 * half + 16 * t + (mi & 1) * 8 + (lane & 7)) * kInRow + (64 * chh + 16 * sl + (mi >> 1) * 8) * 2, x[t][sl]);
-        uint8_t* half_base = dst + half * half_bytes(L);
-        if (L == 8) range = ingest_keys<8>(x, half_base, chh, lane, e);
-        else if (L == 4) range = ingest_keys<4>(x, half_base, chh, lane, e);
-        else if (L == 2) range = ingest_keys<2>(x, half_base, chh, lane, e);
-        else {
-          // distance from the centroid
+            for (int t = 0; t < 2; ++t)
 #pragma unroll
-          for (int sl = 0; sl < 4; ++sl)
-#pragma unroll
-            for (int ah = 0; ah < 2; ++ah) {
-              const float2 cc = *reinterpret_cast<const float2*>(cen + 64 * chh + 16 * sl + 8 * ah + 2 * c4);
-#pragma unroll
-              for (int t = 0; t < 2; ++t)
-#pragma unroll
-                for (int al = 0; al < 2; ++al) {
-                  const float d0 = i_lo(x[t][sl][2 * ah + al]) - cc.x, d1 = i_hi(x[t][sl][2 * ah + al]) - cc.y;
-                  e[t][al] = fmaf(d0, d0, e[t][al]);
-                  e[t][al] = fmaf(d1, d1, e[t][al]);
-                }
-            }
+              for (int al = 0; al < 2; ++al) {
+                const float d0 = i_lo(x[t][2 * ah + al]) - cc.x, d1 = i_hi(x[t][2 * ah + al]) - cc.y;
+                e[t][al] = fmaf(d0, d0, e[t][al]);
+                e[t][al] = fmaf(d1, d1, e[t][al]);
+              }
+          }
         }
       }
       // a token's sum over this warp's 64 channels: add the four lanes of its row
@@ -383,43 +414,38 @@ __global__ void __launch_bounds__(kInThreads, 3) ingest_kernel(const __grid_cons
     } else {
       // ---- values: warp = 16-token tile ----
       const int tile = warp - 4;
-      uint32_t x[8][4];
-      const int mi = lane >> 3;
-#pragma unroll
-      for (int s = 0; s < 8; ++s)
-        i_ldm4t(tile_s + kInTensor + (16 * tile + (mi >> 1) * 8 + (lane & 7)) * kInRow + (16 * s + (mi & 1) * 8) * 2, x[s]);
-      float e[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+      const uint32_t ld = tile_s + kInTensor + (16 * tile + (mi >> 1) * 8 + (lane & 7)) * kInRow + ((mi & 1) * 8) * 2;
+      float e[2][2] = {{0.f, 0.f}, {0.f, 0.f}}, n[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
       if (L != 16 && L != 1) {
         uint8_t* hb = dst + (tile >> 1) * half_bytes(L);
         uint8_t* vp = hb + off_vp(L, tile & 1);
         uint8_t* codes = hb + off_vc(L, tile & 1);
-        if (L == 8) range = ingest_values<8>(x, vp, codes, lane, e);
-        else if (L == 4) range = ingest_values<4>(x, vp, codes, lane, e);
-        else range = ingest_values<2>(x, vp, codes, lane, e);
-      } else if (L == 1) {
-#pragma unroll
-        for (int s = 0; s < 8; ++s)
+        if (L == 8) range = ingest_values<8>(ld, vp, codes, lane, prm, e, n);
+        else if (L == 4) range = ingest_values<4>(ld, vp, codes, lane, prm, e, n);
+        else range = ingest_values<2>(ld, vp, codes, lane, prm, e, n);
+      } else {
+        // squared norms of the rows; for a centroid block also the distance from the centroid
+#pragma unroll 1
+        for (int s = 0; s < 8; ++s) {
+          uint32_t x[4];
+          i_ldm4t(ld + s * 32, x);
 #pragma unroll
           for (int al = 0; al < 2; ++al) {
-            const float cc = cen[kD + 16 * s + r + 8 * al];
+            const float cc = L == 1 ? cen[kD + 16 * s + r + 8 * al] : 0.f;
 #pragma unroll
             for (int ah = 0; ah < 2; ++ah) {
-              const float d0 = i_lo(x[s][2 * ah + al]) - cc, d1 = i_hi(x[s][2 * ah + al]) - cc;
-              e[ah][0] = fmaf(d0, d0, e[ah][0]);
-              e[ah][1] = fmaf(d1, d1, e[ah][1]);
+              const float x0 = i_lo(x[2 * ah + al]), x1 = i_hi(x[2 * ah + al]);
+              n[ah][0] = fmaf(x0, x0, n[ah][0]);
+              n[ah][1] = fmaf(x1, x1, n[ah][1]);
+              if (L == 1) {
+                const float d0 = x0 - cc, d1 = x1 - cc;
+                e[ah][0] = fmaf(d0, d0, e[ah][0]);
+                e[ah][1] = fmaf(d1, d1, e[ah][1]);
+              }
             }
           }
-      }
-      // squared norms of the original value rows, same token layout
-      float n[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-#pragma unroll
-      for (int s = 0; s < 8; ++s)
-#pragma unroll
-        for (int a = 0; a < 4; ++a) {
-          const float x0 = i_lo(x[s][a]), x1 = i_hi(x[s][a]);
-          n[a >> 1][0] = fmaf(x0, x0, n[a >> 1][0]);
-          n[a >> 1][1] = fmaf(x1, x1, n[a >> 1][1]);
         }
+      }
       // a token's sums over all channels: add the eight lanes r; then the largest token of the tile
       float em = 0.f, nm = 0.f;
 #pragma unroll
