@@ -646,17 +646,61 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
     }
   }
 
-  // 3. slots + table mirror
-  for (int s = 0; s < ns; ++s) {
-    for (int b = 0; b <= n_closed; ++b) {
-      const int lvl = b < n_closed ? L.level[static_cast<size_t>(s) * c->max_blocks + b] : 16;
-      uint32_t off;
-      if (!c->heap.alloc(lvl, &off)) return GKV_ERR_ARENA_TOO_SMALL;
-      set_entry(c, L, s, b, off, lvl);
-      L.table_h[static_cast<size_t>(s) * c->table_stride + b].resmask = 0;
+  // 3. slots + table mirror.  The fast encoder takes its work from the table itself, so on its path
+  // the sequences go up in groups: slots of a group, its table rows, its encode launch, and the
+  // host allocates the next group's slots while the GPU encodes this one.
+  const bool has_res = cfg.residual_fraction > 0.f && token_mass && n_closed > 0;
+  const bool fast = n_closed > 0 && v_new &&
+                    ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new)) & 15u) == 0;
+  auto alloc_streams = [&](int s0, int s1) -> int {
+    for (int s = s0; s < s1; ++s) {
+      for (int b = 0; b <= n_closed; ++b) {
+        const int lvl = b < n_closed ? L.level[static_cast<size_t>(s) * c->max_blocks + b] : 16;
+        uint32_t off;
+        if (!c->heap.alloc(lvl, &off)) return GKV_ERR_ARENA_TOO_SMALL;
+        set_entry(c, L, s, b, off, lvl);
+        L.table_h[static_cast<size_t>(s) * c->table_stride + b].resmask = 0;
+      }
+      L.res_count_h[s] = 0;
+      L.res_idx[s].clear();
     }
-    L.res_count_h[s] = 0;
-    L.res_idx[s].clear();
+    return GKV_OK;
+  };
+  // table rows of streams [s0, s1) to the device, then every closed block of theirs encoded once at its planned level
+  auto encode_streams = [&](int s0, int s1) -> int {
+    const size_t row = static_cast<size_t>(c->table_stride);
+    int r2;
+    if ((r2 = upload(c, L.table_d + s0 * row, L.table_h + s0 * row, (s1 - s0) * row * sizeof(TableEntry), st, L.ev)) != GKV_OK) return r2;
+    EncodeParams ep{};
+    ep.arena = c->arena;
+    ep.jobs = nullptr;
+    ep.n_jobs = (s1 - s0) * n_closed;
+    ep.k_in = k_new;
+    ep.v_in = v_new;
+    ep.n_tok = n_new;
+    ep.n_kv_heads = cfg.n_kv_heads;
+    ep.status = c->status_d;
+    ep.err = L.err_d;
+    ep.err_stride = c->max_blocks;
+    ep.table = L.table_d;
+    ep.table_stride = c->table_stride;
+    ep.n_blocks = n_closed;
+    ep.first_seq = s0 / cfg.n_kv_heads;
+    CK(c, launch_ingest(ep, st));
+    return GKV_OK;
+  };
+  bool encoded = false;
+  if (fast && !has_res) {
+    const int per_seq = n_closed * cfg.n_kv_heads;
+    const int seqs = std::max(1, (4096 + per_seq - 1) / per_seq);       // at least ~4096 blocks per launch
+    for (int q0 = 0; q0 < cfg.batch; q0 += seqs) {
+      const int s0 = q0 * cfg.n_kv_heads, s1 = std::min(cfg.batch, q0 + seqs) * cfg.n_kv_heads;
+      if ((rc = alloc_streams(s0, s1)) != GKV_OK) return rc;
+      if ((rc = encode_streams(s0, s1)) != GKV_OK) return rc;
+    }
+    encoded = true;
+  } else if ((rc = alloc_streams(0, ns)) != GKV_OK) {
+    return rc;
   }
   L.has_tail_slot = true;
 
@@ -699,8 +743,10 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
     }
   }
 
-  // 5. uploads, then encode every closed block once at its planned level, copy the tail rows
-  if ((rc = upload(c, L.table_d, L.table_h, static_cast<size_t>(ns) * c->table_stride * sizeof(TableEntry), st, L.ev)) != GKV_OK) return rc;
+  // 5. uploads, then encode every closed block once at its planned level (unless done above), copy the tail rows
+  if (!encoded && !fast &&
+      (rc = upload(c, L.table_d, L.table_h, static_cast<size_t>(ns) * c->table_stride * sizeof(TableEntry), st, L.ev)) != GKV_OK)
+    return rc;
   if ((rc = upload(c, L.res_count_d, L.res_count_h, ns * sizeof(int32_t), st, L.ev)) != GKV_OK) return rc;
   if (L.res_count_d && cfg.residual_fraction > 0.f) {
     int max_k = 0;
@@ -709,14 +755,14 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
                                  L.res_count_d, L.res_off_d, max_k, ns, st));
   }
   const size_t n_jobs = static_cast<size_t>(ns) * n_closed;
-  if (n_jobs > 0) {
+  if (!encoded && fast) {
+    if ((rc = encode_streams(0, ns)) != GKV_OK) return rc;
+  } else if (!encoded && n_jobs > 0) {
+    // inputs that the fast encoder does not take (unaligned rows): the general block encoder, one job per block
     EncodeJob* jobs = reinterpret_cast<EncodeJob*>(stage + stage_off);
     size_t j = 0;
-    // order (sequence, block, KV head): CTAs that run at the same time read neighbouring rows
-    for (int sq = 0; sq < cfg.batch; ++sq)
-      for (int b = 0; b < n_closed; ++b)
-        for (int kvh = 0; kvh < cfg.n_kv_heads; ++kvh) {
-        const int s = sq * cfg.n_kv_heads + kvh;
+    for (int s = 0; s < ns; ++s)
+      for (int b = 0; b < n_closed; ++b) {
         EncodeJob& job = jobs[j++];
         job.src_off256 = 0;
         job.dst_off256 = L.table_h[static_cast<size_t>(s) * c->table_stride + b].off256;
@@ -738,9 +784,7 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
     ep.status = c->status_d;
     ep.err = L.err_d;
     ep.err_stride = c->max_blocks;
-    const bool aligned = ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new)) & 15u) == 0;
-    if (aligned && v_new) CK(c, launch_ingest(ep, st));
-    else CK(c, launch_encode(ep, st));
+    CK(c, launch_encode(ep, st));
   }
   CK(c, cudaEventRecord(c->ev_stage, st));
   CK(c, launch_append_rows(c->arena, L.table_d, c->table_stride, n_closed, ns, cfg.n_kv_heads, k_new, v_new, n_new,

@@ -320,8 +320,25 @@ __global__ void __launch_bounds__(kInThreads, 3) ingest_kernel(const __grid_cons
   const uint32_t sbase = i_u32(ism);
   const size_t row_stride = static_cast<size_t>(p.n_kv_heads) * kD;      // elements between two tokens of a stream
 
+  // work item -> (stream, block, slot, level): from the job list, or counted off in the order
+  // (sequence, block, KV head) with slot and level taken from the block table
+  auto job_of = [&](int item) -> EncodeJob {
+    if (p.jobs) return p.jobs[item];
+    const int per_seq = p.n_blocks * p.n_kv_heads;
+    const int sq = item / per_seq, rem = item - sq * per_seq;
+    EncodeJob job;
+    job.block = rem / p.n_kv_heads;
+    job.stream = (p.first_seq + sq) * p.n_kv_heads + (rem - job.block * p.n_kv_heads);
+    const TableEntry te = p.table[static_cast<size_t>(job.stream) * p.table_stride + job.block];
+    job.src_off256 = 0;
+    job.dst_off256 = te.off256;
+    job.src_level = 0;
+    job.dst_level = static_cast<int16_t>(te.level);
+    job.pad = 0;
+    return job;
+  };
   auto stage = [&](int item, int buf) {
-    const EncodeJob job = p.jobs[item];
+    const EncodeJob job = job_of(item);
     const int b = job.stream / p.n_kv_heads, kvh = job.stream - b * p.n_kv_heads;
     const size_t first = (static_cast<size_t>(b) * p.n_tok + static_cast<size_t>(job.block) * kBlock) * row_stride + static_cast<size_t>(kvh) * kD;
 #pragma unroll
@@ -337,7 +354,7 @@ __global__ void __launch_bounds__(kInThreads, 3) ingest_kernel(const __grid_cons
   if (item < p.n_jobs) stage(item, 0);
   i_commit();
   for (; item < p.n_jobs; item += gridDim.x, buf ^= 1) {
-    const EncodeJob job = p.jobs[item];
+    const EncodeJob job = job_of(item);
     i_wait_all();
     __syncthreads();                       // the block's rows are there; nobody still reads the other buffer
     if (item + static_cast<int>(gridDim.x) < p.n_jobs) stage(item + gridDim.x, buf ^ 1);
@@ -489,7 +506,7 @@ __global__ void __launch_bounds__(kInThreads, 3) ingest_kernel(const __grid_cons
 
 }  // namespace
 
-// All jobs read the bf16 input rows (src_level == 0).
+// All jobs read the bf16 input rows (src_level == 0); without a job list the work is counted off the block table.
 cudaError_t launch_ingest(const EncodeParams& p, cudaStream_t st) {
   if (p.n_jobs <= 0) return cudaSuccess;
   static bool configured = false;

@@ -140,6 +140,10 @@ struct EncodeParams {
   // offset and level of entry [stream][block], the residual mask stays).
   TableEntry* table;
   int32_t table_stride;
+  // Bulk ingest without a job list (jobs == nullptr): work item i is block (i / n_kv_heads) % n_blocks of
+  // KV head i % n_kv_heads of sequence first_seq + i / (n_blocks * n_kv_heads); its slot and level are read
+  // from the table (which is not written).
+  int32_t n_blocks, first_seq;
 };
 
 // Statistics of freshly closed blocks: page boxes, key range proxy, block mass.
