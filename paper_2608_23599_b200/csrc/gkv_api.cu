@@ -9,6 +9,7 @@
 #include <cstring>
 #include <new>
 #include <numeric>
+#include <thread>
 #include <vector>
 
 #include "../../include/gkv.h"
@@ -397,6 +398,33 @@ bool rd_allocate(const gkv_config& c, const float* mass, const float* range, int
   return budget_miss;
 }
 
+// The streams' allocations are independent: a handful of host threads share them (each stream's
+// plan depends only on its own masses and ranges, so the result does not depend on the thread count).
+// Returns true when some stream missed its budget.
+bool rd_allocate_streams(const gkv_config& c, const float* mass, const float* range, int n, int n_tail, int ns,
+                         const int8_t* prev, size_t prev_stride, int8_t* out, size_t out_stride) {
+  std::vector<char> miss(ns, 0);
+  auto run = [&](int s) {
+    miss[s] = rd_allocate(c, mass + static_cast<size_t>(s) * n, range + static_cast<size_t>(s) * n, n, n_tail,
+                          prev ? prev + static_cast<size_t>(s) * prev_stride : nullptr, out + static_cast<size_t>(s) * out_stride);
+  };
+  const unsigned hw = std::thread::hardware_concurrency();
+  const int n_thr = std::min({ns / 2, 8, static_cast<int>(hw ? hw : 1u)});
+  if (n_thr < 2 || static_cast<size_t>(ns) * n < 2048) {
+    for (int s = 0; s < ns; ++s) run(s);
+  } else {
+    std::vector<std::thread> pool;
+    pool.reserve(n_thr - 1);
+    for (int t = 1; t < n_thr; ++t)
+      pool.emplace_back([&, t] {
+        for (int s = t; s < ns; s += n_thr) run(s);
+      });
+    for (int s = 0; s < ns; s += n_thr) run(s);
+    for (std::thread& th : pool) th.join();
+  }
+  return std::find(miss.begin(), miss.end(), 1) != miss.end();
+}
+
 // ---- decode work split ---------------------------------------------------------------------------
 // Cost of one item for the work split: cycles a warp needs for it while the whole GPU runs the
 // mixed workload, measured on B200 by timing every step of individual warps of the config-2 launch
@@ -636,13 +664,9 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
     CK(c, cudaMemcpy2DAsync(L.range_d, static_cast<size_t>(c->max_blocks) * sizeof(float), c->range_d,
                             static_cast<size_t>(n_closed) * sizeof(float), static_cast<size_t>(n_closed) * sizeof(float), ns,
                             cudaMemcpyDeviceToDevice, st));
-    for (int s = 0; s < ns; ++s) {
-      const bool miss = rd_allocate(cfg, &mass[static_cast<size_t>(s) * n_closed], &range[static_cast<size_t>(s) * n_closed],
-                                    n_closed, n_tail, nullptr, &L.level[static_cast<size_t>(s) * c->max_blocks]);
-      if (miss) {
-        L.budget_flag = true;
-        warn = GKV_ERR_BUDGET;
-      }
+    if (rd_allocate_streams(cfg, mass.data(), range.data(), n_closed, n_tail, ns, nullptr, 0, L.level.data(), c->max_blocks)) {
+      L.budget_flag = true;
+      warn = GKV_ERR_BUDGET;
     }
   }
 
@@ -1354,13 +1378,9 @@ int gkv_rd_reallocate(gkv_cache* c, int32_t layer, void* stream) {
   CK(c, cudaStreamSynchronize(st));
   std::vector<int8_t> target(static_cast<size_t>(ns) * n);
   int warn = GKV_OK;
-  for (int s = 0; s < ns; ++s) {
-    const bool miss = rd_allocate(cfg, &mass[static_cast<size_t>(s) * n], &range[static_cast<size_t>(s) * n], n, L.n_tail,
-                                  &L.level[static_cast<size_t>(s) * c->max_blocks], &target[static_cast<size_t>(s) * n]);
-    if (miss) {
-      L.budget_flag = true;
-      warn = GKV_ERR_BUDGET;
-    }
+  if (rd_allocate_streams(cfg, mass.data(), range.data(), n, L.n_tail, ns, L.level.data(), c->max_blocks, target.data(), n)) {
+    L.budget_flag = true;
+    warn = GKV_ERR_BUDGET;
   }
   const int rc = demote_to_targets(c, L, target.data(), static_cast<size_t>(n), st);
   return rc != GKV_OK ? rc : warn;
