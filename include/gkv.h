@@ -18,6 +18,10 @@
  *    on the host before anything is launched; nothing traps or asserts on the device.
  *  - bf16 / fp16 data are raw 16-bit patterns.  Values must be finite and, for blocks
  *    below level 16 and for queries, within +-65504 (fp16 range).
+ *  - Alignment of device buffers: queries and attention outputs 16 bytes; new key / value
+ *    rows 4 bytes (16 bytes lets a bulk ingest take the fast encoder; other rows are
+ *    encoded by the general one, with the same bits); float and int32 arrays 4 bytes.
+ *    A pointer off these boundaries is refused with GKV_ERR_INVALID_ARG.
  */
 #ifndef GKV_H_
 #define GKV_H_

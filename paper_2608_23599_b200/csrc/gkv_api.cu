@@ -716,7 +716,7 @@ int bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* 
   bool encoded = false;
   if (fast && !has_res) {
     const int per_seq = n_closed * cfg.n_kv_heads;
-    const int seqs = std::max(1, (4096 + per_seq - 1) / per_seq);       // at least ~4096 blocks per launch
+    const int seqs = std::max(1, (8192 + per_seq - 1) / per_seq);       // at least ~8192 blocks per launch
     for (int q0 = 0; q0 < cfg.batch; q0 += seqs) {
       const int s0 = q0 * cfg.n_kv_heads, s1 = std::min(cfg.batch, q0 + seqs) * cfg.n_kv_heads;
       if ((rc = alloc_streams(s0, s1)) != GKV_OK) return rc;
@@ -1415,10 +1415,17 @@ int gkv_ctx_len(gkv_cache* c, int32_t layer, int32_t* ctx) {
   return GKV_OK;
 }
 
+namespace {
+// The kernels read queries, new rows and index lists and write results with 4- to 16-byte accesses:
+// a pointer off its natural boundary is refused here instead of faulting on the device.
+inline bool misaligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
+}  // namespace
+
 int gkv_append_demote(gkv_cache* c, int32_t layer, const void* k_new, const void* v_new, int32_t n_new,
                       const float* token_mass, const int8_t* level_plan, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || !k_new || n_new <= 0) return GKV_ERR_INVALID_ARG;
   if (is_mla(c->cfg) ? (v_new != nullptr) : (v_new == nullptr)) return GKV_ERR_INVALID_ARG;
+  if (misaligned(k_new, 4) || misaligned(v_new, 4) || misaligned(token_mass, 4)) return GKV_ERR_INVALID_ARG;
   LayerState& L = c->layers[layer];
   const int ctx = L.n_closed * kBlock + L.n_tail;
   if (static_cast<long long>(ctx) + n_new > c->cfg.max_ctx) return GKV_ERR_CTX_FULL;
@@ -1442,6 +1449,9 @@ int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_
                 bool observe, float* block_mass, float* certificate, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !out) return GKV_ERR_INVALID_ARG;
   if (!page_idx && n_sel != 0) return GKV_ERR_INVALID_ARG;
+  if (misaligned(q, 16) || misaligned(out, 16) || misaligned(lse, 4) || misaligned(page_idx, 4) || misaligned(block_mass, 4) ||
+      misaligned(certificate, 4))
+    return GKV_ERR_INVALID_ARG;
   LayerState& L = c->layers[layer];
   if (L.n_closed * kBlock + L.n_tail == 0) return GKV_ERR_BAD_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1593,6 +1603,7 @@ int gkv_quest_select(gkv_cache* c, int32_t layer, const void* q, int32_t budget_
                      int32_t* n_sel_out, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !page_idx_out || !n_sel_out || budget_tokens < 0)
     return GKV_ERR_INVALID_ARG;
+  if (misaligned(q, 16) || misaligned(page_idx_out, 4)) return GKV_ERR_INVALID_ARG;
   const gkv_config& cfg = c->cfg;
   if (cfg.page_tokens <= 0) return GKV_ERR_BAD_STATE;
   LayerState& L = c->layers[layer];
@@ -1612,6 +1623,7 @@ int gkv_quest_select_static(gkv_cache* c, int32_t layer, const void* q, int32_t 
                             int32_t* page_idx_out, int32_t* n_sel_out, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !page_idx_out || !n_sel_out || budget_tokens < 0)
     return GKV_ERR_INVALID_ARG;
+  if (misaligned(q, 16) || misaligned(page_idx_out, 4)) return GKV_ERR_INVALID_ARG;
   const gkv_config& cfg = c->cfg;
   if (cfg.page_tokens <= 0) return GKV_ERR_BAD_STATE;
   LayerState& L = c->layers[layer];

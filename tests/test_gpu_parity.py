@@ -53,6 +53,30 @@ def test_single_tier(level, T):
     gcache.close()
 
 
+def test_ingest_of_rows_that_are_not_16_byte_aligned():
+    """The bulk encoder wants 16-byte aligned rows; other inputs go through the general block encoder.
+    Same prompt, key / value tensors placed 4 bytes off a 16-byte boundary: same bits as the oracle."""
+    w = _tiny(456)
+    ocache, gcache = _pair(w)
+    data = W.make_layer(w, 0, "cpu")
+    ocache.append_demote(0, U.f32(data["k"]), U.f32(data["v"]))
+    dev = gcache.device
+
+    def shifted(t):
+        flat = torch.empty(t.numel() + 8, dtype=t.dtype, device=dev)
+        view = flat[2:2 + t.numel()].view(t.shape)
+        view.copy_(t.to(dev))
+        assert view.data_ptr() % 16 == 4
+        return view
+
+    k, v = shifted(data["k"]), shifted(data["v"])
+    gcache.gkv_append_demote(0, k, v)
+    U.assert_state_equal(ocache, gcache, 0)
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
+    U.assert_outputs_close(out, o_out, "unaligned ingest")
+    gcache.close()
+
+
 def test_tail_only_and_single_token():
     """Contexts shorter than one block: only the exact tail exists."""
     for T in (1, 17, 63):
@@ -285,6 +309,25 @@ def test_host_side_errors():
     with pytest.raises(B.GkvError) as e:
         full.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
     assert e.value.status == -3
+    # pointers off their natural boundary are refused before anything is launched
+    def off_by(t, n_elem):
+        flat = torch.empty(t.numel() + 16, dtype=t.dtype, device=dev)
+        view = flat[n_elem:n_elem + t.numel()].view(t.shape)
+        view.copy_(t.to(dev))
+        return view
+    qd = d2["q"].to(dev).to(torch.bfloat16)
+    out = torch.empty((w2.batch, w2.n_q_heads, w2.d_v), dtype=torch.float32, device=dev)
+    with pytest.raises(B.GkvError) as e:
+        full.gkv_decode_attn(0, off_by(qd, 1), out)            # query 2 bytes off
+    assert e.value.status == -1
+    with pytest.raises(B.GkvError) as e:
+        full.gkv_decode_attn(0, qd, off_by(out, 1))            # output 4 bytes off a 16-byte boundary
+    assert e.value.status == -1
+    fresh = B.Cache(B.config_from_workload(w2))
+    with pytest.raises(B.GkvError) as e:
+        fresh.gkv_append_demote(0, off_by(d2["k"], 1), d2["v"].to(dev))   # rows 2 bytes off
+    assert e.value.status == -1
+    fresh.close()
     full.close()
 
 
