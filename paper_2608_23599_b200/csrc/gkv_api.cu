@@ -1062,7 +1062,9 @@ int mla_bulk_ingest(gkv_cache* c, int layer, const uint16_t* k_new, int n_new, c
     ep.k_in = k_new;
     ep.n_tok = n_new;
     ep.status = c->status_d;
-    CK(c, launch_mla_encode(ep, st));
+    // 16-byte aligned rows take the bulk encoder; the general block encoder stores the same bits
+    if ((reinterpret_cast<uintptr_t>(k_new) & 15u) == 0) CK(c, launch_mla_ingest(ep, st));
+    else CK(c, launch_mla_encode(ep, st));
   }
   CK(c, cudaEventRecord(c->ev_stage, st));
   CK(c, launch_mla_append_rows(c->arena, L.table_d, c->table_stride, n_closed, ns, k_new, n_new, n_closed * kBlock, n_tail, 0, st));

@@ -22,6 +22,7 @@
 #include <cuda_fp16.h>
 
 #include "gkv_internal.h"
+#include "gkv_mla.h"
 
 namespace gkv {
 namespace {
@@ -504,6 +505,116 @@ __global__ void __launch_bounds__(kInThreads, 3) ingest_kernel(const __grid_cons
   }
 }
 
+// ---- latent-attention (MLA) streams -------------------------------------------------------------
+// One 576-wide row per token, quantised with the key rule (groups of 32 tokens of one channel);
+// codes are stored row-major, a chunk of 8 neighbouring channels of a token per 32-bit word (4 bits)
+// or pair of words (8 bits).  Thread = (half of the block, chunk): it owns the 8 groups of its
+// chunk, so nothing is exchanged between threads.  The block (73.7 KB, contiguous in the input) is
+// staged in shared memory with 16-byte cp.async copies; three CTAs per SM take turns loading and
+// encoding.
+constexpr int kMlaInThreads = 160;                       // 144 = 2 halves x 72 chunks work on quantised blocks
+constexpr int kMlaInTile = kBlock * kMlaRowBytes;         // 73728
+
+// code of x as an integer in the low mantissa bits of (clamped value + 1.5 * 2^23)
+template <int BITS>
+__device__ __forceinline__ uint32_t i_code(float x, float z, float inv) {
+  constexpr float qmax = static_cast<float>((1 << BITS) - 1);
+  return __float_as_uint(__fadd_rn(fminf(fmaxf(__fmul_rn(__fsub_rn(x, z), inv), 0.f), qmax), kMagic));
+}
+
+template <int BITS>
+__device__ __forceinline__ bool mla_ingest_quant(const uint8_t* tile, uint8_t* dst, int tid) {
+  const int half = tid / kMlaChunks, j = tid - half * kMlaChunks;
+  const uint8_t* rows = tile + (32 * half) * kMlaRowBytes + j * 16;
+  uint4 mn = *reinterpret_cast<const uint4*>(rows), mx = mn;
+#pragma unroll 4
+  for (int t = 1; t < kGroup; ++t) {
+    const uint4 v = *reinterpret_cast<const uint4*>(rows + t * kMlaRowBytes);
+    mn.x = i_min2(mn.x, v.x);
+    mn.y = i_min2(mn.y, v.y);
+    mn.z = i_min2(mn.z, v.z);
+    mn.w = i_min2(mn.w, v.w);
+    mx.x = i_max2(mx.x, v.x);
+    mx.y = i_max2(mx.y, v.y);
+    mx.z = i_max2(mx.z, v.z);
+    mx.w = i_max2(mx.w, v.w);
+  }
+  const uint32_t mnr[4] = {mn.x, mn.y, mn.z, mn.w}, mxr[4] = {mx.x, mx.y, mx.z, mx.w};
+  float z[8], inv[8];
+  uint32_t sb[4], zb[4];
+  bool range = false;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const GroupParams g0 = i_params<BITS>(i_lo(mnr[i]), i_lo(mxr[i])), g1 = i_params<BITS>(i_hi(mnr[i]), i_hi(mxr[i]));
+    z[2 * i] = g0.z;
+    z[2 * i + 1] = g1.z;
+    inv[2 * i] = g0.inv;
+    inv[2 * i + 1] = g1.inv;
+    sb[i] = static_cast<uint32_t>(g0.s_bits) | (static_cast<uint32_t>(g1.s_bits) << 16);
+    zb[i] = static_cast<uint32_t>(g0.z_bits) | (static_cast<uint32_t>(g1.z_bits) << 16);
+    range |= g0.range || g1.range;
+  }
+  uint8_t* hb = dst + half * mla_half_bytes(BITS);
+  // parameters of chunk j: eight fp16 scales, then eight fp16 zero points
+  *reinterpret_cast<uint4*>(hb + j * 32) = make_uint4(sb[0], sb[1], sb[2], sb[3]);
+  *reinterpret_cast<uint4*>(hb + j * 32 + 16) = make_uint4(zb[0], zb[1], zb[2], zb[3]);
+  uint8_t* codes = hb + mla_kp_bytes() + j * BITS;
+#pragma unroll 2
+  for (int t = 0; t < kGroup; ++t) {
+    const uint4 v = *reinterpret_cast<const uint4*>(rows + t * kMlaRowBytes);
+    const uint32_t u0 = i_code<BITS>(i_lo(v.x), z[0], inv[0]), u1 = i_code<BITS>(i_hi(v.x), z[1], inv[1]);
+    const uint32_t u2 = i_code<BITS>(i_lo(v.y), z[2], inv[2]), u3 = i_code<BITS>(i_hi(v.y), z[3], inv[3]);
+    const uint32_t u4 = i_code<BITS>(i_lo(v.z), z[4], inv[4]), u5 = i_code<BITS>(i_hi(v.z), z[5], inv[5]);
+    const uint32_t u6 = i_code<BITS>(i_lo(v.w), z[6], inv[6]), u7 = i_code<BITS>(i_hi(v.w), z[7], inv[7]);
+    if (BITS == 8) {
+      // channel c of a word's four sits at byte ((c & 3) >> 1) + 2 (c & 1)
+      const uint32_t w0 = u0 + (u2 << 8) + (u1 << 16) + (u3 << 24) - kMagicBits * 0x01010101u;
+      const uint32_t w1 = u4 + (u6 << 8) + (u5 << 16) + (u7 << 24) - kMagicBits * 0x01010101u;
+      *reinterpret_cast<uint2*>(codes + t * mla_code_row_bytes(8)) = make_uint2(w0, w1);
+    } else {
+      // channel c sits at bit 4 (c >> 1) + 16 (c & 1)
+      const uint32_t w0 = u0 + (u2 << 4) + (u4 << 8) + (u6 << 12) + (u1 << 16) + (u3 << 20) + (u5 << 24) + (u7 << 28) -
+                          kMagicBits * 0x11111111u;
+      *reinterpret_cast<uint32_t*>(codes + t * mla_code_row_bytes(4)) = w0;
+    }
+  }
+  return range;
+}
+
+__global__ void __launch_bounds__(kMlaInThreads, 3) mla_ingest_kernel(const __grid_constant__ MlaEncodeParams p) {
+  extern __shared__ __align__(16) uint8_t msm[];
+  const int tid = threadIdx.x;
+  const uint32_t sbase = i_u32(msm);
+  constexpr int kChunks = kMlaInTile / 16;               // 4608
+  for (int item = blockIdx.x; item < p.n_jobs; item += gridDim.x) {
+    const EncodeJob job = p.jobs[item];
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(
+        p.k_in + (static_cast<size_t>(job.stream) * p.n_tok + static_cast<size_t>(job.block) * kBlock) * kMlaDk);
+    __syncthreads();                                     // everybody is done with the previous block
+    for (int q = tid; q < kChunks; q += kMlaInThreads) i_cp16(sbase + q * 16, src + q * 16);
+    i_commit();
+    i_wait_all();
+    __syncthreads();
+    uint8_t* dst = p.arena + static_cast<size_t>(job.dst_off256) * 256;
+    const int L = job.dst_level;
+    if (L == 16) {
+      for (int q = tid; q < kChunks; q += kMlaInThreads)
+        *reinterpret_cast<uint4*>(dst + q * 16) = *reinterpret_cast<const uint4*>(msm + q * 16);
+    } else if (L == 1) {
+      for (int c = tid; c < kMlaDk; c += kMlaInThreads) {
+        const uint16_t* col = reinterpret_cast<const uint16_t*>(msm) + c;
+        float acc = 0.f;
+#pragma unroll 16
+        for (int t = 0; t < kBlock; ++t) acc = __fadd_rn(acc, __uint_as_float(static_cast<uint32_t>(col[t * kMlaDk]) << 16));
+        reinterpret_cast<uint16_t*>(dst)[c] = i_bf16(__fmul_rn(acc, 1.0f / kBlock));
+      }
+    } else if (tid < 2 * kMlaChunks) {
+      const bool range = L == 8 ? mla_ingest_quant<8>(msm, dst, tid) : mla_ingest_quant<4>(msm, dst, tid);
+      if (range) atomicOr(p.status, kStatusRange);
+    }
+  }
+}
+
 }  // namespace
 
 // All jobs read the bf16 input rows (src_level == 0); without a job list the work is counted off the block table.
@@ -520,4 +631,20 @@ cudaError_t launch_ingest(const EncodeParams& p, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+}  // namespace gkv
+
+namespace gkv {
+// Bulk ingest of latent-attention rows: every job reads the bf16 input (src_level == 0), rows 16-byte aligned.
+cudaError_t launch_mla_ingest(const MlaEncodeParams& p, cudaStream_t st) {
+  if (p.n_jobs <= 0) return cudaSuccess;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(mla_ingest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMlaInTile);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int grid = p.n_jobs < 148 * 3 ? p.n_jobs : 148 * 3;
+  mla_ingest_kernel<<<grid, kMlaInThreads, kMlaInTile, st>>>(p);
+  return cudaGetLastError();
+}
 }  // namespace gkv

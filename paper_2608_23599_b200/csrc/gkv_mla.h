@@ -27,6 +27,7 @@ struct MlaDecodeParams {
 };
 
 cudaError_t launch_mla_encode(const MlaEncodeParams& p, cudaStream_t st);
+cudaError_t launch_mla_ingest(const MlaEncodeParams& p, cudaStream_t st);   // all jobs from the bf16 input, 16-byte aligned
 cudaError_t launch_mla_append_rows(uint8_t* arena, const TableEntry* table, int table_stride, int tail_index, int n_streams,
                                    const uint16_t* k_in, int n_tok, int first_tok, int n_rows, int dst_row0, cudaStream_t st);
 cudaError_t launch_mla_export(const uint8_t* arena, uint32_t off256, int level, uint8_t* codes, uint16_t* scale,

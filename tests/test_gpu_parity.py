@@ -357,6 +357,26 @@ def test_mla_single_tier(level, T):
     gcache.close()
 
 
+def test_mla_ingest_of_rows_that_are_not_16_byte_aligned():
+    """Latent rows 4 bytes off a 16-byte boundary go through the general block encoder: same bits."""
+    T = 328
+    w = _mla(T, policy=W.POLICY_EXTERNAL)
+    ocache, gcache = _pair(w)
+    data = W.make_layer(w, 0, "cpu")
+    plan = np.tile(np.array([1, 4, 8, 4, 16], dtype=np.int8), (w.batch, 1, 1))
+    ocache.append_demote(0, U.f32(data["k"]), None, level_plan=plan)
+    dev = gcache.device
+    flat = torch.empty(data["k"].numel() + 8, dtype=data["k"].dtype, device=dev)
+    k = flat[2:2 + data["k"].numel()].view(data["k"].shape)
+    k.copy_(data["k"].to(dev))
+    assert k.data_ptr() % 16 == 4
+    gcache.gkv_append_demote(0, k, None, level_plan=plan)
+    U.assert_state_equal(ocache, gcache, 0)
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
+    U.assert_outputs_close(out, o_out, "mla unaligned ingest", scale=U.value_scale(data["k"][..., :512]))
+    gcache.close()
+
+
 def test_cfg4_small_mla_ladder_with_appends():
     """Config 4 structure at small size: exact newest rung, int8, int4, centroid for the oldest
     quarter (5.0 bits/value), then appends with staircase demotion."""
