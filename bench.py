@@ -194,14 +194,26 @@ def run_ours(args, rank, local, world):
     k_sel = wl.quest_budget_tokens // wl.page_tokens if quest else 0
     pages = torch.zeros((Bsz, Hkv, max(k_sel, 1)), dtype=torch.int32, device=device) if quest else None
 
+    # The loops below hand the library plain device addresses (worked out once, here) instead of a
+    # fresh tensor view per call, as a serving loop in C++ would: on the small workloads the per-call
+    # host time would otherwise be the bound.  The buffers are the tensors above.
+    cache.stream_handle = torch.cuda.current_stream().cuda_stream
+    k_stride, v_stride, q_stride, o_stride = Bsz * Hkv * d * 2, Bsz * Hkv * dv * 2, Bsz * Hq * d * 2, Bsz * Hq * dv * 4
+    k_at = lambda s_, l_: k_new.data_ptr() + (s_ * n_layers + l_) * k_stride
+    v_at = (lambda s_, l_: None) if alias else (lambda s_, l_: v_new.data_ptr() + (s_ * n_layers + l_) * v_stride)
+    q_at = lambda s_, l_: q_new.data_ptr() + (s_ * n_layers + l_) * q_stride
+    out_at = [out.data_ptr() + l_ * o_stride for l_ in range(n_layers)]
+    pages_at = pages.data_ptr() if quest else None
+    budget = wl.quest_budget_tokens
+
     def step_device(s):
         for l in range(n_layers):
-            cache.gkv_append_demote(l, k_new[s, l], None if alias else v_new[s, l])
+            cache.gkv_append_demote(l, k_at(s, l), v_at(s, l), n_new=1)
             if quest:
-                n_sel = cache.gkv_quest_select(l, q_new[s, l], wl.quest_budget_tokens, pages)
-                cache.gkv_decode_attn(l, q_new[s, l], out[l], page_idx=pages, n_sel=n_sel)
+                n_sel = cache.gkv_quest_select(l, q_at(s, l), budget, pages_at)
+                cache.gkv_decode_attn(l, q_at(s, l), out_at[l], page_idx=pages_at, n_sel=n_sel)
             else:
-                cache.gkv_decode_attn(l, q_new[s, l], out[l])
+                cache.gkv_decode_attn(l, q_at(s, l), out_at[l])
 
     # ---- device-resident timing -------------------------------------------------------------------
     s = 0
@@ -242,21 +254,32 @@ def run_ours(args, rank, local, world):
     reps = max(3, min(20, int(2e10 / max(algo_bytes * n_layers, 1))))
     for l in range(n_layers):
         if quest:
-            cache.gkv_decode_attn(l, q_new[0, l], out[l], page_idx=pages, n_sel=k_sel)
+            cache.gkv_decode_attn(l, q_at(0, l), out_at[l], page_idx=pages_at, n_sel=k_sel)
         else:
-            cache.gkv_decode_attn(l, q_new[0, l], out[l])
+            cache.gkv_decode_attn(l, q_at(0, l), out_at[l])
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for r in range(reps):
         for l in range(n_layers):
             if quest:
-                cache.gkv_decode_attn(l, q_new[r % total_steps, l], out[l], page_idx=pages, n_sel=k_sel)
+                cache.gkv_decode_attn(l, q_at(r % total_steps, l), out_at[l], page_idx=pages_at, n_sel=k_sel)
             else:
-                cache.gkv_decode_attn(l, q_new[r % total_steps, l], out[l])
+                cache.gkv_decode_attn(l, q_at(r % total_steps, l), out_at[l])
     e1.record()
     torch.cuda.synchronize()
     us_launch = e0.elapsed_time(e1) * 1e3 / (reps * n_layers)
+    # the same call on one layer back to back: its bytes stay in the 126 MB L2 when they fit (labelled warm)
+    w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0.record()
+    for r in range(20):
+        if quest:
+            cache.gkv_decode_attn(0, q_at(r % total_steps, 0), out_at[0], page_idx=pages_at, n_sel=k_sel)
+        else:
+            cache.gkv_decode_attn(0, q_at(r % total_steps, 0), out_at[0])
+    w1.record()
+    torch.cuda.synchronize()
+    us_launch_one_layer = w0.elapsed_time(w1) * 1e3 / 20
     achieved = algo_bytes / (us_launch * 1e-6) / 1e9
     peak, peak_kind = measured_hbm_peak()
     traffic = DRAM_TRAFFIC_PER_LAUNCH.get(wl.name)
@@ -267,7 +290,7 @@ def run_ours(args, rank, local, world):
         s0.record()
         for r in range(reps):
             for l in range(n_layers):
-                cache.gkv_quest_select(l, q_new[r % total_steps, l], wl.quest_budget_tokens, pages)
+                cache.gkv_quest_select(l, q_at(r % total_steps, l), budget, pages_at)
         s1.record()
         torch.cuda.synchronize()
         us_sel = s0.elapsed_time(s1) * 1e3 / (reps * n_layers)
@@ -281,18 +304,22 @@ def run_ours(args, rank, local, world):
     hout = torch.empty((n_layers, Bsz, Hq, dv), dtype=torch.float32).pin_memory()
     dk, dvv, dq = torch.empty_like(hk, device=device), torch.empty_like(hv, device=device), torch.empty_like(hq, device=device)
 
+    dk_at = [dk.data_ptr() + l_ * k_stride for l_ in range(n_layers)]
+    dv_at = [None if alias else dvv.data_ptr() + l_ * v_stride for l_ in range(n_layers)]
+    dq_at = [dq.data_ptr() + l_ * q_stride for l_ in range(n_layers)]
+
     def step_e2e():
         dk.copy_(hk, non_blocking=True)
         if not alias:
             dvv.copy_(hv, non_blocking=True)
         dq.copy_(hq, non_blocking=True)
         for l in range(n_layers):
-            cache.gkv_append_demote(l, dk[l], None if alias else dvv[l])
+            cache.gkv_append_demote(l, dk_at[l], dv_at[l], n_new=1)
             if quest:
-                n_sel = cache.gkv_quest_select(l, dq[l], wl.quest_budget_tokens, pages)
-                cache.gkv_decode_attn(l, dq[l], out[l], page_idx=pages, n_sel=n_sel)
+                n_sel = cache.gkv_quest_select(l, dq_at[l], budget, pages_at)
+                cache.gkv_decode_attn(l, dq_at[l], out_at[l], page_idx=pages_at, n_sel=n_sel)
             else:
-                cache.gkv_decode_attn(l, dq[l], out[l])
+                cache.gkv_decode_attn(l, dq_at[l], out_at[l])
         hout.copy_(out, non_blocking=True)
         torch.cuda.current_stream().synchronize()      # the caller consumes the step's result
 
@@ -334,6 +361,8 @@ def run_ours(args, rank, local, world):
                      "traffic": traffic, "peak_kind": peak_kind + " copy bandwidth",
                      "kernel": "decode_kernel (split-K partials merged in the same launch; timed per gkv_decode_attn call)",
                      "us_per_launch": us_launch, "algorithmic_bytes_per_launch": algo_bytes,
+                     "us_per_launch_same_layer_back_to_back": us_launch_one_layer,
+                     "same_layer_fits_l2": bool(algo_bytes < 100e6),
                      "frac_of_8TBs": achieved / NOMINAL_HBM_GBS},
         "ctx_tokens_per_s_per_layer_call": Bsz * ctx_start / (us_launch * 1e-6),
         # gkv_append_demote next to gkv_decode_attn: what a layer's append adds to its decode call in a

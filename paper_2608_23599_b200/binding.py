@@ -215,28 +215,36 @@ class Cache:
         except Exception:
             pass
 
-    def gkv_append_demote(self, layer, k_new, v_new, token_mass=None, level_plan=None):
+    stream_handle = None   # set to a cudaStream_t (int) to skip the per-call look-up of torch's current stream
+
+    def _st(self) -> int:
+        return self.stream_handle if self.stream_handle is not None else _stream()
+
+    def gkv_append_demote(self, layer, k_new, v_new, token_mass=None, level_plan=None, n_new=None):
         """k_new/v_new: cuda bf16 [B][n_new][Hkv][d]; token_mass cuda fp32 [B][Hkv][n_new];
-        level_plan: host int8 numpy [B][Hkv][n_new // 64]."""
-        n_new = k_new.shape[1]
+        level_plan: host int8 numpy [B][Hkv][n_new // 64].  Device buffers may be given as tensors or as
+        plain integer device addresses (then pass n_new): a serving loop that calls once per layer and step
+        keeps its addresses instead of building tensor views."""
+        if n_new is None:
+            n_new = k_new.shape[1]
         plan_ptr = None
         if level_plan is not None:
             self._plan_keep = level_plan = level_plan.astype("int8", copy=False)
             plan_ptr = level_plan.ctypes.data
         return _check(load().gkv_append_demote(self.handle, layer, _ptr(k_new), _ptr(v_new), n_new,
-                                               _ptr(token_mass), plan_ptr, _stream()),
+                                               _ptr(token_mass), plan_ptr, self._st()),
                       "gkv_append_demote", allow=(ERR_RANGE, ERR_BUDGET))
 
     def gkv_decode_attn(self, layer, q, out, lse=None, page_idx=None, n_sel=0):
         return _check(load().gkv_decode_attn(self.handle, layer, _ptr(q), _ptr(page_idx), n_sel, _ptr(out),
-                                             _ptr(lse), _stream()), "gkv_decode_attn")
+                                             _ptr(lse), self._st()), "gkv_decode_attn")
 
     def gkv_decode_attn_observe(self, layer, q, out, lse=None, block_mass=None, certificate=None):
         """Full-context decode that also observes the attention mass of every block and updates the
         cache's running masses (block_mass: device fp32 [batch][n_kv_heads][ceil(ctx / 64)] or None;
         certificate: device fp32 [batch][n_q_heads] or None, the error certificate of this query)."""
         return _check(load().gkv_decode_attn_observe(self.handle, layer, _ptr(q), _ptr(out), _ptr(lse), _ptr(block_mass),
-                                                     _ptr(certificate), _stream()), "gkv_decode_attn_observe")
+                                                     _ptr(certificate), self._st()), "gkv_decode_attn_observe")
 
     def gkv_debug_export_bounds(self, layer):
         """Per-block certificate bounds as numpy [batch][n_kv_heads][n_closed][4] (kappa, delta, max |v|, 0)."""
@@ -247,7 +255,7 @@ class Cache:
 
     def gkv_rd_reallocate(self, layer):
         """Decode-time re-allocation of an RD-policy layer from the running block masses."""
-        return _check(load().gkv_rd_reallocate(self.handle, layer, _stream()), "gkv_rd_reallocate",
+        return _check(load().gkv_rd_reallocate(self.handle, layer, self._st()), "gkv_rd_reallocate",
                       allow=(ERR_RANGE, ERR_BUDGET))
 
     def gkv_debug_export_mass(self, layer):
@@ -260,7 +268,7 @@ class Cache:
     def gkv_quest_select(self, layer, q, budget_tokens, page_idx_out) -> int:
         n = C.c_int32(0)
         _check(load().gkv_quest_select(self.handle, layer, _ptr(q), budget_tokens, _ptr(page_idx_out), C.byref(n),
-                                       _stream()), "gkv_quest_select")
+                                       self._st()), "gkv_quest_select")
         return n.value
 
     def gkv_quest_select_static(self, layer, q, budget_tokens, page_idx_out) -> int:
@@ -268,7 +276,7 @@ class Cache:
         that must not trigger any device allocation.  Same arguments and results."""
         n = C.c_int32(0)
         _check(load().gkv_quest_select_static(self.handle, layer, _ptr(q), budget_tokens, _ptr(page_idx_out),
-                                              C.byref(n), _stream()), "gkv_quest_select_static")
+                                              C.byref(n), self._st()), "gkv_quest_select_static")
         return n.value
 
     def gkv_bits_report(self, layer=-1) -> GkvBits:
