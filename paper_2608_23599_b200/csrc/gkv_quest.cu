@@ -110,6 +110,9 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 
 constexpr int kTopkThreads = 1024;
 
+// KEEP: n <= 4 * kTopkThreads, every thread keeps the keys of its (up to four) elements in registers
+// instead of reading the scores again in every pass.
+template <bool KEEP>
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restrict__ scores, int score_stride,
                                                             int n, const int32_t* __restrict__ k_per_stream,
                                                             int k_uniform, int32_t* __restrict__ idx_out,
@@ -130,6 +133,14 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
     s_prefix = 0;
     s_remaining = static_cast<uint32_t>(k);
   }
+  uint32_t kreg[4] = {0u, 0u, 0u, 0u};
+  if (KEEP) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = tid + j * kTopkThreads;
+      if (i < n) kreg[j] = score_key(sc[i]);
+    }
+  }
   // radix select, most significant byte first: find the key of the k-th largest score
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
@@ -137,9 +148,15 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
     __syncthreads();
     const uint32_t prefix = s_prefix;
     const uint32_t pmask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-    for (int i = tid; i < n; i += kTopkThreads) {
-      const uint32_t key = score_key(sc[i]);
-      if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    if (KEEP) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (tid + j * kTopkThreads < n && (kreg[j] & pmask) == prefix) atomicAdd(&hist[(kreg[j] >> shift) & 255u], 1u);
+    } else {
+      for (int i = tid; i < n; i += kTopkThreads) {
+        const uint32_t key = score_key(sc[i]);
+        if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      }
     }
     __syncthreads();
     // The digit of the k-th largest is the t with c[t] >= rem > c[t + 1], c[t] = sum_{j >= t} hist[j].
@@ -183,12 +200,14 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
   __syncthreads();
   // ordered compaction in index order
   const int lane = tid & 31, wid = tid >> 5;
-  for (int i0 = 0; i0 < n; i0 += kTopkThreads) {
+#pragma unroll 1
+  for (int i0 = 0, j = 0; i0 < n; i0 += kTopkThreads, ++j) {
     const int i = i0 + tid;
     uint32_t key = 0;
     bool gt = false, eq = false;
     if (i < n) {
-      key = score_key(sc[i]);
+      if (KEEP) key = j == 0 ? kreg[0] : (j == 1 ? kreg[1] : (j == 2 ? kreg[2] : kreg[3]));
+      else key = score_key(sc[i]);
       gt = key > thr;
       eq = key == thr;
     }
@@ -278,7 +297,9 @@ cudaError_t launch_topk(const float* scores, int score_stride, int n, const int3
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, topk_kernel, scores, score_stride, n, k_per_stream, k_uniform, idx_out, idx_stride);
+  if (n <= 4 * kTopkThreads)
+    return cudaLaunchKernelEx(&cfg, topk_kernel<true>, scores, score_stride, n, k_per_stream, k_uniform, idx_out, idx_stride);
+  return cudaLaunchKernelEx(&cfg, topk_kernel<false>, scores, score_stride, n, k_per_stream, k_uniform, idx_out, idx_stride);
 }
 
 }  // namespace gkv
