@@ -555,9 +555,9 @@ __device__ __forceinline__ bool mla_ingest_quant(const uint8_t* tile, uint8_t* d
     range |= g0.range || g1.range;
   }
   uint8_t* hb = dst + half * mla_half_bytes(BITS);
-  // parameters of chunk j: eight fp16 scales, then eight fp16 zero points
-  *reinterpret_cast<uint4*>(hb + j * 32) = make_uint4(sb[0], sb[1], sb[2], sb[3]);
-  *reinterpret_cast<uint4*>(hb + j * 32 + 16) = make_uint4(zb[0], zb[1], zb[2], zb[3]);
+  // parameters: the 576 fp16 scales, then the 576 fp16 zero points; chunk j owns piece j of each
+  *reinterpret_cast<uint4*>(hb + j * 16) = make_uint4(sb[0], sb[1], sb[2], sb[3]);
+  *reinterpret_cast<uint4*>(hb + kMlaZeroOff * 2 + j * 16) = make_uint4(zb[0], zb[1], zb[2], zb[3]);
   uint8_t* codes = hb + mla_kp_bytes() + j * BITS;
 #pragma unroll 2
   for (int t = 0; t < kGroup; ++t) {

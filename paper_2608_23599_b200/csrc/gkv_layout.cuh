@@ -127,8 +127,9 @@ GKV_HD int vp_zero_index(int t16, int grp) {
 // ---- latent-attention (MLA) streams: one 576-wide row per token, values = channels [0, 512) ----
 // The row is quantised once with the key rule (32 tokens x 1 channel per group).  A quantised slot
 // is two halves of 32 tokens: [params 2304 B][codes 32 rows x 72 chunks]; a chunk is 8 neighbouring
-// channels of one token (8 bytes at 8 bits, one 32-bit word at 4 bits).  The params of chunk j are
-// 32 bytes: eight fp16 scales, then eight fp16 zero points.  Inside a chunk the codes are placed so
+// channels of one token (8 bytes at 8 bits, one 32-bit word at 4 bits).  The params are the 576 fp16
+// scales, then the 576 fp16 zero points (a chunk's eight scales are one 16-byte piece, neighbouring
+// chunks neighbouring pieces: a warp reads them without gaps).  Inside a chunk the codes are placed so
 // that one "mask, or in an exponent" (4 bits) or one byte permute (8 bits) yields the fp16 pair
 // of two neighbouring channels: 4-bit channel c sits at bit 4 (c >> 1) + 16 (c & 1); 8-bit channel c
 // sits in word c >> 2 at byte ((c & 3) >> 1) + 2 (c & 1).
@@ -142,8 +143,9 @@ GKV_HD int mla_half_bytes(int bits) { return mla_kp_bytes() + 32 * mla_code_row_
 GKV_HD int mla_slot_bytes(int level) {
   return level == 16 ? kBlock * kMlaRowBytes : (level == 1 ? 1280 : 2 * mla_half_bytes(level));
 }
-// fp16 index of channel ch's scale inside a half's params; its zero point sits 8 entries later
-GKV_HD int mla_kp_index(int ch) { return (ch >> 3) * 16 + (ch & 7); }
+// fp16 index of channel ch's scale inside a half's params; its zero point sits kMlaZeroOff entries later
+GKV_HD int mla_kp_index(int ch) { return ch; }
+constexpr int kMlaZeroOff = kMlaDk;   // fp16 entries from a channel's scale to its zero point
 // position of the code of (token t32 of the half, channel ch): byte offset of its 32-bit word from
 // the start of the half's code rows, and the bit inside that word
 GKV_HD void mla_code_pos(int bits, int t32, int ch, int* byte_off, int* bit) {

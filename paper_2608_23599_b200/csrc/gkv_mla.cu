@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(256) mla_encode_kernel(const __grid_constant__
           const int code = mla_read_code(slot, bits, t, c);
           const uint16_t* kp = reinterpret_cast<const uint16_t*>(slot + (t >> 5) * mla_half_bytes(bits));
           const int idx = mla_kp_index(c);
-          tile[t * kMTileLd + c] = __fmaf_rn(static_cast<float>(code), hbits(kp[idx]), hbits(kp[idx + 8]));
+          tile[t * kMTileLd + c] = __fmaf_rn(static_cast<float>(code), hbits(kp[idx]), hbits(kp[idx + kMlaZeroOff]));
         }
       }
     }
@@ -102,7 +102,7 @@ __global__ void __launch_bounds__(256) mla_encode_kernel(const __grid_constant__
         uint16_t* kp = reinterpret_cast<uint16_t*>(dst + half * mla_half_bytes(L));
         const int idx = mla_kp_index(c);
         kp[idx] = sb;
-        kp[idx + 8] = zb;
+        kp[idx + kMlaZeroOff] = zb;
       }
       if (range) atomicOr(p.status, kStatusRange);
       __syncthreads();
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(256) mla_export_kernel(const uint8_t* arena, u
     const int half = g / kMlaDk, c = g % kMlaDk;
     const uint16_t* kp = reinterpret_cast<const uint16_t*>(slot + half * mla_half_bytes(level));
     scale[g] = kp[mla_kp_index(c)];
-    zero[g] = kp[mla_kp_index(c) + 8];
+    zero[g] = kp[mla_kp_index(c) + kMlaZeroOff];
   }
 }
 

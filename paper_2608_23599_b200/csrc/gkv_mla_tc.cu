@@ -304,7 +304,7 @@ __device__ __forceinline__ uint32_t tc_tile_addr(uint32_t tile, int row, int j) 
 // dequantise one half (32 tokens) of a quantised block: thread = (chunk j, 8 tokens)
 template <int BITS>
 __device__ __forceinline__ void tc_dequant_half(uint32_t raw, uint32_t tile, int half, int j, int tg) {
-  const uint4 sv = t_lds128(raw + j * 32), zv = t_lds128(raw + j * 32 + 16);
+  const uint4 sv = t_lds128(raw + j * 16), zv = t_lds128(raw + kMlaZeroOff * 2 + j * 16);
   const __half2 s0 = t_h2(sv.x), s1 = t_h2(sv.y), s2 = t_h2(sv.z), s3 = t_h2(sv.w);
   const __half2 z0 = t_h2(zv.x), z1 = t_h2(zv.y), z2 = t_h2(zv.z), z3 = t_h2(zv.w);
   const uint32_t codes = raw + mla_kp_bytes() + j * BITS + tg * 8 * (kMlaChunks * BITS);
