@@ -91,6 +91,7 @@ struct LayerState {
   std::vector<std::vector<int32_t>> res_idx;
   bool desc_dirty = true;
   bool desc_split = false;              // the work lists hold sub-block units (never for observing calls)
+  bool desc_allow_split = false;        // what the lists were built with
   int n_warps = 0;
   cudaEvent_t ev = nullptr;             // last upload from this layer's pinned table / residual mirrors
   cudaEvent_t ev_desc = nullptr;        // last upload from its pinned work lists (warps, units, parts)
@@ -124,6 +125,7 @@ struct gkv_cache {
   float scale = 0.f;
   SlotHeap heap;
   std::vector<LayerState> layers;
+  int desc_src = -1;                    // layer whose work lists were last built from scratch
   // shared device scratch
   uint32_t* status_d = nullptr;
   uint8_t* debug_d = nullptr;
@@ -451,6 +453,31 @@ size_t item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) 
 // walks its units in a mixed order (see below).
 void build_descs(gkv_cache* c, LayerState& L, bool allow_split) {
   const int ns = c->n_streams;
+  // The lists depend only on the streams' levels and residual counts.  Layers usually close a block
+  // in the same step and, under the staircase, with the same plan: a layer whose levels equal those
+  // of the layer built last takes a copy of that layer's lists instead of building its own.
+  const int self = static_cast<int>(&L - c->layers.data());
+  if (c->desc_src >= 0 && c->desc_src != self) {
+    const LayerState& S = c->layers[c->desc_src];
+    bool same = !S.desc_dirty && S.desc_allow_split == allow_split && S.n_closed == L.n_closed &&
+                std::memcmp(S.res_count_h, L.res_count_h, static_cast<size_t>(ns) * sizeof(int32_t)) == 0;
+    for (int s = 0; same && s < ns; ++s)
+      same = std::memcmp(S.level.data() + static_cast<size_t>(s) * c->max_blocks, L.level.data() + static_cast<size_t>(s) * c->max_blocks,
+                         static_cast<size_t>(L.n_closed)) == 0;
+    if (same) {
+      std::memcpy(L.warps_h, S.warps_h, static_cast<size_t>(S.n_warps) * sizeof(WarpDesc));
+      std::memcpy(L.units_h, S.units_h, static_cast<size_t>(S.n_units) * sizeof(uint32_t));
+      std::memcpy(L.parts_h, S.parts_h, static_cast<size_t>(ns) * sizeof(StreamParts));
+      L.n_warps = S.n_warps;
+      L.n_units = S.n_units;
+      L.desc_split = S.desc_split;
+      L.desc_allow_split = allow_split;
+      L.desc_dirty = false;
+      return;
+    }
+  }
+  c->desc_src = self;
+  L.desc_allow_split = allow_split;
   struct Unit { uint32_t word; uint32_t cost; };
   // Pass 1: the units of every stream and their total cost.  Streams with the same levels and the
   // same number of residual rows (all streams under the staircase policy) have the same units:
