@@ -393,12 +393,50 @@ def run_ours(args, rank, local, world):
                           **step_detail},
     }
     line["bulk_ingest"] = ingest
+    if rank == 0 and wl.config_id == 1 and n_layers > 1:
+        line["all_layers_in_one_launch"] = one_launch_figure(wl, n_layers, device)
     if scorer:
         line["quest_select"] = scorer
     if rank == 0:
         line["cpu_baseline"] = cpu_baseline(wl, n_layers, budget_s=args.cpu_seconds)
     cache.close()
     return line
+
+
+# --------------------------------------------------------------------------------------------------
+def one_launch_figure(w: W.Workload, n_layers: int, device):
+    """Config 1 reads ~5 MB per layer call and is bound by launch latency.  For scale: the same amount of
+    cache as all layers of a step, laid out as n_layers sequences of ONE layer, read by ONE decode launch.
+    This is not a model step (a layer's query depends on the layer before it); it shows what the kernel
+    does with the step's bytes when they come in one launch."""
+    from paper_2608_23599_b200 import binding as B
+    import dataclasses
+    wide = dataclasses.replace(w, batch=w.batch * n_layers, n_layers=1)
+    cache = B.Cache(B.config_from_workload(wide, 1), device=device)
+    data = W.make_layer(wide, 0, device)
+    cache.gkv_append_demote(0, data["k"], data.get("v"), token_mass=data.get("mass"))
+    q = data["q"]
+    out = torch.empty((wide.batch, wide.n_q_heads, wide.d_v), dtype=torch.float32, device=device)
+    for _ in range(3):
+        cache.gkv_decode_attn(0, q, out)
+    torch.cuda.synchronize()
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=device)      # larger than the 126 MB L2
+    times = []
+    for _ in range(10):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        cache.gkv_decode_attn(0, q, out)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) * 1e3)
+    rep = cache.gkv_bits_report(0)
+    nbytes = rep.last_read_bits / 8 + q.numel() * 2 + out.numel() * 4
+    us = sorted(times)[len(times) // 2]
+    cache.close()
+    return {"us": us, "bytes": nbytes, "GB/s": nbytes / (us * 1e-6) / 1e9, "sequences": wide.batch,
+            "l2": "flushed before every launch",
+            "note": "n_layers x batch sequences of one layer in one launch; not a model step"}
 
 
 # --------------------------------------------------------------------------------------------------
