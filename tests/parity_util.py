@@ -20,7 +20,10 @@ def value_scale(v):
     if v is None:
         return 1.0
     x = v.detach().float().cpu() if hasattr(v, "detach") else torch.as_tensor(np.asarray(v)).float()
-    sd = x.reshape(-1, x.shape[-1]).std(dim=0).numpy().astype(np.float64)
+    rows = x.reshape(-1, x.shape[-1])
+    if rows.shape[0] < 2:            # a single row has no spread
+        return np.ones(rows.shape[1], dtype=np.float64)
+    sd = rows.std(dim=0).numpy().astype(np.float64)
     return np.maximum(1.0, sd)
 
 
@@ -87,7 +90,8 @@ def assert_state_equal(ocache, gcache, layer, streams=None, blocks=None):
                     assert np.array_equal(ex["rows"][: st.n_tail], O.bf16_bits(st.tail_v))
 
 
-def assert_outputs_close(out_gpu, out_oracle, what="", scale=1.0):
+def assert_outputs_close(out_gpu, out_oracle, what="", scale=1.0, abs_tol=None):
+    """abs_tol: override of ABS_TOL (only the random-shape run uses one, see its docstring)."""
     g = out_gpu.detach().to("cpu").to(torch.float64).numpy()
     o = np.asarray(out_oracle, dtype=np.float64)
     assert g.shape == o.shape
@@ -95,8 +99,9 @@ def assert_outputs_close(out_gpu, out_oracle, what="", scale=1.0):
     scale = np.maximum(1.0, np.asarray(scale, dtype=np.float64))        # scalar or per channel
     nerr = (np.abs(g - o) / scale).max()
     err = np.abs(g - o).max()
-    assert nerr <= ABS_TOL, (f"{what}: max-abs error per unit of value scale {nerr:.3e} > {ABS_TOL} "
-                             f"(raw max-abs {err:.3e}, value scale up to {float(np.max(scale)):.2f})")
+    tol = ABS_TOL if abs_tol is None else abs_tol
+    assert nerr <= tol, (f"{what}: max-abs error per unit of value scale {nerr:.3e} > {tol} "
+                         f"(raw max-abs {err:.3e}, value scale up to {float(np.max(scale)):.2f})")
     num = np.linalg.norm(g - o, axis=-1)
     den = np.linalg.norm(o, axis=-1) + 1e-30
     rel = (num / den).max()
