@@ -368,7 +368,8 @@ def run_ours(args, rank, local, world):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 exact rows / int8-int4-int2 codes dequantised to f16, f32 accumulate",
+        "dtype": "f16",       # tensor-core operands; f32 accumulation
+        "dtype_detail": "bf16 exact rows / int8-int4-int2 codes dequantised to f16 operands, f32 accumulate",
         "data": "synthetic",
         "config": {"workload": wl.name, "batch": Bsz, "context": ctx_start, "n_layers": n_layers,
                    "n_q_heads": Hq, "n_kv_heads": Hkv, "head_dim": d, "resident_bpv": rep.bpv_resident,
