@@ -85,7 +85,7 @@ struct LayerState {
   WarpDesc* warps_h = nullptr;          // pinned [max_warps]
   uint32_t* units_h = nullptr;          // pinned [n_streams][unit_stride]
   int n_units = 0;
-  StreamParts* parts_h = nullptr;       // pinned [n_streams]
+  StreamParts* parts_h = nullptr;       // pinned [n_streams * head_groups]
   uint32_t* res_off_h = nullptr;        // pinned [n_streams]
   int32_t* res_count_h = nullptr;       // pinned [n_streams]
   std::vector<std::vector<int32_t>> res_idx;
@@ -121,7 +121,7 @@ struct gkv_cache {
   gkv_config cfg;
   uint8_t* arena = nullptr;
   size_t arena_bytes = 0;
-  int n_streams = 0, group = 0, max_blocks = 0, table_stride = 0, max_warps = 0, res_cap = 0, box_stride = 0;
+  int n_streams = 0, group = 0, head_groups = 1, n_hgroups = 0, max_blocks = 0, table_stride = 0, max_warps = 0, res_cap = 0, box_stride = 0;
   float scale = 0.f;
   SlotHeap heap;
   std::vector<LayerState> layers;
@@ -135,7 +135,7 @@ struct gkv_cache {
   int8_t* levels_d = nullptr;
   float* scores_d = nullptr;            // residual scores [n_streams][max_ctx] or page scores
   int32_t* kper_d = nullptr;
-  int32_t* tickets_d = nullptr;         // per-stream arrival counters of the decode kernel's final merge
+  int32_t* tickets_d = nullptr;         // per-head-group arrival counters of the decode kernel's final merge
   float2* mass_raw_d = nullptr;         // scratch of an observing decode call: [n_streams][max_blocks + 1][8]
   float2* res_raw_d = nullptr;          // [n_streams][res_cap][8]
   float* lse2_d = nullptr;              // [n_streams][8]
@@ -168,7 +168,7 @@ struct ArenaPlan {
 };
 
 struct Derived {
-  int n_streams, group, max_blocks, table_stride, max_warps, res_cap, box_stride, unit_stride;
+  int n_streams, group, head_groups, n_hgroups, max_blocks, table_stride, max_warps, res_cap, box_stride, unit_stride;
 };
 
 int validate_config(const gkv_config* c) {
@@ -203,10 +203,13 @@ Derived derive(const gkv_config& c) {
   Derived d;
   d.n_streams = c.batch * c.n_kv_heads;
   d.group = c.n_q_heads / c.n_kv_heads;
+  // a warp of the decode kernel serves up to four query heads: a larger group is read as two head groups
+  d.head_groups = is_mla(c) ? 1 : (d.group + kHeadsPerWarp - 1) / kHeadsPerWarp;
+  d.n_hgroups = d.n_streams * d.head_groups;
   d.max_blocks = (c.max_ctx + kBlock - 1) / kBlock;
   d.table_stride = d.max_blocks + 2;
-  d.max_warps = static_cast<int>(align_up(kTargetWarps + 2 * d.n_streams, kDecodeWarps));
-  d.max_warps = std::max(d.max_warps, d.n_streams * sparse_ctas_per_stream(d.n_streams) * kDecodeWarps);
+  d.max_warps = static_cast<int>(align_up(kTargetWarps + 2 * d.n_hgroups, kDecodeWarps));
+  d.max_warps = std::max(d.max_warps, d.n_hgroups * sparse_ctas_per_stream(d.n_hgroups) * kDecodeWarps);
   d.res_cap = c.residual_fraction > 0.f
                   ? static_cast<int>(align_up(static_cast<size_t>(std::floor(static_cast<double>(c.residual_fraction) * c.max_ctx)) + 16, 16))
                   : 0;
@@ -229,7 +232,7 @@ ArenaPlan plan_arena(const gkv_config& c, const Derived& d) {
   const size_t score_elems = std::max<size_t>(c.residual_fraction > 0.f ? c.max_ctx : 0, d.box_stride);
   a.scores = take(static_cast<size_t>(d.n_streams) * score_elems * sizeof(float));
   a.kper = take(static_cast<size_t>(d.n_streams) * sizeof(int32_t));
-  a.tickets = take(static_cast<size_t>(d.n_streams) * sizeof(int32_t));
+  a.tickets = take(static_cast<size_t>(d.n_hgroups) * sizeof(int32_t));
   a.jobs = take(static_cast<size_t>(d.n_streams) * d.max_blocks * sizeof(EncodeJob));
   // block-mass observation (grouped-query layout only)
   const size_t mass_items = is_mla(c) ? 0 : static_cast<size_t>(d.n_streams) * (d.max_blocks + 1);
@@ -242,7 +245,7 @@ ArenaPlan plan_arena(const gkv_config& c, const Derived& d) {
   a.l_table = ltake(static_cast<size_t>(d.n_streams) * d.table_stride * sizeof(TableEntry));
   a.l_warps = ltake(static_cast<size_t>(d.max_warps) * sizeof(WarpDesc));
   a.l_units = ltake(static_cast<size_t>(d.n_streams) * d.unit_stride * sizeof(uint32_t));
-  a.l_parts = ltake(static_cast<size_t>(d.n_streams) * sizeof(StreamParts));
+  a.l_parts = ltake(static_cast<size_t>(d.n_hgroups) * sizeof(StreamParts));
   a.l_resoff = ltake(static_cast<size_t>(d.n_streams) * sizeof(uint32_t));
   a.l_rescount = ltake(static_cast<size_t>(d.n_streams) * sizeof(int32_t));
   a.l_residx = ltake(static_cast<size_t>(d.n_streams) * std::max(d.res_cap, 1) * sizeof(int32_t));
@@ -467,7 +470,7 @@ void build_descs(gkv_cache* c, LayerState& L, bool allow_split) {
     if (same) {
       std::memcpy(L.warps_h, S.warps_h, static_cast<size_t>(S.n_warps) * sizeof(WarpDesc));
       std::memcpy(L.units_h, S.units_h, static_cast<size_t>(S.n_units) * sizeof(uint32_t));
-      std::memcpy(L.parts_h, S.parts_h, static_cast<size_t>(ns) * sizeof(StreamParts));
+      std::memcpy(L.parts_h, S.parts_h, static_cast<size_t>(c->n_hgroups) * sizeof(StreamParts));
       L.n_warps = S.n_warps;
       L.n_units = S.n_units;
       L.desc_split = S.desc_split;
@@ -543,6 +546,9 @@ void build_descs(gkv_cache* c, LayerState& L, bool allow_split) {
     }
     total += cost[s];
   }
+  // every head group of a stream (up to four query heads each) walks the stream's units with warps of its own
+  const int hg = c->head_groups;
+  total *= static_cast<size_t>(hg);
   const size_t target = std::max(split_all ? kMinWarpCost / 4 : kMinWarpCost, (total + kTargetWarps - 1) / kTargetWarps);
   // Pass 2: deal each distinct stream's units to its warps, then lay the warps out.
   int w = 0, pos = 0, row = 0;
@@ -554,7 +560,7 @@ void build_descs(gkv_cache* c, LayerState& L, bool allow_split) {
     const std::vector<Unit>& u0 = units[src];
     int nw = static_cast<int>((cost[s] + target / 2) / target);
     nw = std::max(1, std::min(nw, static_cast<int>(u0.size())));
-    nw = std::min(nw, c->max_warps - w - (ns - 1 - s));
+    nw = std::min(nw, (c->max_warps - w) / hg - (ns - 1 - s));
     if (dealt_for != src || dealt_nw != nw) {
       std::vector<Unit> u(u0);
       std::stable_sort(u.begin(), u.end(), [](const Unit& a, const Unit& b) { return a.cost > b.cost; });
@@ -601,22 +607,29 @@ void build_descs(gkv_cache* c, LayerState& L, bool allow_split) {
       dealt_for = src;
       dealt_nw = nw;
     }
-    // one partial row per (CTA, stream): the kernel merges the warps of a CTA that share a stream
-    L.parts_h[s].begin = row;
-    for (int k = 0; k < nw; ++k) {
-      const std::vector<uint32_t>& m = lists[k];
-      WarpDesc& d = L.warps_h[w];
-      d.stream = s;
-      d.item_begin = pos;
-      std::memcpy(L.units_h + pos, m.data(), m.size() * sizeof(uint32_t));
-      pos += static_cast<int>(m.size());
-      d.item_end = pos;
-      if (k > 0 && w % kDecodeWarps == 0) ++row;
-      d.partial = row;
-      ++w;
+    // One partial row per (CTA, head group): the kernel merges the warps of a CTA that share a head
+    // group.  The head groups of a stream get the same lists (stored once) and neighbouring warps, so
+    // that the second reader of a block finds it in L2.
+    const int pos0 = pos;
+    for (int g = 0; g < hg; ++g) {
+      const int hgi = s * hg + g;
+      L.parts_h[hgi].begin = row;
+      pos = pos0;
+      for (int k = 0; k < nw; ++k) {
+        const std::vector<uint32_t>& m = lists[k];
+        WarpDesc& d = L.warps_h[w];
+        d.stream = hgi;
+        d.item_begin = pos;
+        if (g == 0) std::memcpy(L.units_h + pos, m.data(), m.size() * sizeof(uint32_t));
+        pos += static_cast<int>(m.size());
+        d.item_end = pos;
+        if (k > 0 && w % kDecodeWarps == 0) ++row;
+        d.partial = row;
+        ++w;
+      }
+      ++row;
+      L.parts_h[hgi].end = row;
     }
-    ++row;
-    L.parts_h[s].end = row;
   }
   const int padded = static_cast<int>(align_up(w, kDecodeWarps));
   for (int i = w; i < padded; ++i) L.warps_h[i] = WarpDesc{-1, 0, 0, 0};
@@ -1278,6 +1291,8 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
   c->arena_bytes = arena_bytes;
   c->n_streams = d.n_streams;
   c->group = d.group;
+  c->head_groups = d.head_groups;
+  c->n_hgroups = d.n_hgroups;
   c->max_blocks = d.max_blocks;
   c->table_stride = d.table_stride;
   c->max_warps = d.max_warps;
@@ -1341,7 +1356,7 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
     if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.warps_h), d.max_warps * sizeof(WarpDesc), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
     if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.units_h), static_cast<size_t>(d.n_streams) * d.unit_stride * sizeof(uint32_t),
                            cudaHostAllocDefault)) != cudaSuccess) return fail(e);
-    if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.parts_h), d.n_streams * sizeof(StreamParts), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
+    if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.parts_h), d.n_hgroups * sizeof(StreamParts), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
     if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.res_off_h), d.n_streams * sizeof(uint32_t), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
     if ((e = cudaHostAlloc(reinterpret_cast<void**>(&L.res_count_h), d.n_streams * sizeof(int32_t), cudaHostAllocDefault)) != cudaSuccess) return fail(e);
     for (int s = 0; s < d.n_streams; ++s) {
@@ -1509,6 +1524,7 @@ int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_
   p.n_tail = L.n_tail;
   p.n_kv_heads = cfg.n_kv_heads;
   p.group = c->group;
+  p.head_groups = c->head_groups;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.status = c->status_d;
   p.tickets = c->tickets_d;
@@ -1523,8 +1539,8 @@ int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_
     p.page_idx = page_idx;
     p.n_sel = n_sel;
     p.page_tokens = cfg.page_tokens;
-    p.warps_per_stream = sparse_ctas_per_stream(c->n_streams) * kDecodeWarps;
-    p.n_warps = c->n_streams * p.warps_per_stream;
+    p.warps_per_stream = sparse_ctas_per_stream(c->n_hgroups) * kDecodeWarps;      // per head group
+    p.n_warps = c->n_hgroups * p.warps_per_stream;
     p.warps = nullptr;
     p.parts = nullptr;
     n_ctas = (p.n_warps + kDecodeWarps - 1) / kDecodeWarps;
@@ -1540,7 +1556,7 @@ int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_
       build_descs(c, L, !observe);
       if ((rc = upload(c, L.warps_d, L.warps_h, static_cast<size_t>(L.n_warps) * sizeof(WarpDesc), st, L.ev_desc)) != GKV_OK) return rc;
       if ((rc = upload(c, L.units_d, L.units_h, static_cast<size_t>(L.n_units) * sizeof(uint32_t), st, L.ev_desc)) != GKV_OK) return rc;
-      if ((rc = upload(c, L.parts_d, L.parts_h, static_cast<size_t>(c->n_streams) * sizeof(StreamParts), st, L.ev_desc)) != GKV_OK) return rc;
+      if ((rc = upload(c, L.parts_d, L.parts_h, static_cast<size_t>(c->n_hgroups) * sizeof(StreamParts), st, L.ev_desc)) != GKV_OK) return rc;
     }
     p.warps = L.warps_d;
     p.units = L.units_d;

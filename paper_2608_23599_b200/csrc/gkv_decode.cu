@@ -1,21 +1,29 @@
 // Graded single-query decode attention (paper Sec. 3.7: dequantisation inside the online-softmax
-// loop, all KV heads of a layer in one launch, split-context partials reduced separately).
+// loop, all KV heads of a layer in one launch, split-context partials merged in the same launch).
 //
-// Work split: every warp owns a contiguous, byte-balanced range of one stream's items (closed
-// blocks of any level, the exact tail block, groups of exact residual rows) and keeps its own
-// online-softmax state for the g <= 8 query heads of the KV head (one read of the KV bytes serves
-// the whole GQA group, Sec. 3.1).  Warps never wait on each other: each one runs a private
-// double-buffered pipeline of TMA bulk copies (cp.async.bulk global -> shared, completion on a
-// per-warp mbarrier) and consumes only what it staged; every mbarrier wait is bounded.
+// Work split: the host cuts every stream into units (a block, half of a quantised block, a run of
+// centroid blocks, the tail, a group of exact residual rows) and deals them longest-first to the
+// stream's warps; a warp walks its unit list and keeps its own online-softmax state for the g <= 8
+// query heads of the KV head (one read of the KV bytes serves the whole GQA group, Sec. 3.1).
+// Warps never wait on each other: each one runs a private double-buffered pipeline of TMA bulk
+// copies (cp.async.bulk global -> shared, completion on a per-warp mbarrier) and consumes only what
+// it staged; every mbarrier wait is bounded.
 //
 // Math: S^T[tokens x heads] = K[tokens x ch] Q^T and O^T[ch x heads] += V^T[ch x tokens] P^T on
 // mma.m16n8k16 with the query heads as the n = 8 dimension.  Quantised codes are stored in
 // A-fragment order (gkv_layout.cuh) at bit positions where one LOP3 turns a code into the fp16
 // number "bias + code".  Scales are folded into the B operands (q' = q * s_k per 32-token key
 // group, P' = p * s_v per 32-channel value group); zero points and the biases are handled by
-// extra MMAs (A = zero-point pattern or all ones) instead of per-value arithmetic, so the ALU
-// cost is ~5 instructions per 8 values.  Exact rows go through ldmatrix and bf16 MMAs with P
-// split into hi + lo bf16 parts so that its rounding stays below 2^-16.
+// extra MMAs (A = zero-point pattern or all ones) instead of per-value arithmetic.
+//
+// Precision: every B operand that carries a rounded product or probability is a pair hi + lo of
+// fp16 (bf16 for exact rows) numbers, hi = rn(x), lo = rn(x - hi), so that the operand is good to
+// ~2^-22 and the fp32 accumulators decide the error.  A warp serves at most four query heads: the
+// n = 8 dimension holds (hi, lo) column pairs, column 2 j the hi part and column 2 j + 1 the lo part of
+// head j, so one MMA does both and a lane finds the two halves of its head side by side in its
+// accumulator registers.  A KV head with 5..8 query heads is read as two such head groups.  The
+// biases of the code unpack are kept small (<= 256; 1024 at 8 bits) because "bias * sum of
+// operands" is cancelled in fp32.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -112,7 +120,6 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 }
 __device__ __forceinline__ uint32_t h2_as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
-__device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) { return h2_as_u32(__hmul2(u32_as_h2(a), u32_as_h2(b))); }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -121,26 +128,27 @@ __device__ __forceinline__ float bf16lo_to_f32(uint32_t u) { return __uint_as_fl
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
 // ---- code unpack: the four A registers of MMA index s as fp16 "bias + code" ------------------
-// Biases (rows r / rows r + 8 of the MMA): 8-bit 1024 / 1024; 4-bit 1024 / 64; 2-bit 1024 / 256 for
-// even s and 64 / 16 for odd s: a code that sits at mantissa bit b of an fp16 with exponent 2^E has
-// the value code * 2^(E - 10 + b), so picking E = 10 - b makes "mask, or in the exponent" a complete
-// conversion with no shift; only the upper byte of each 16-bit half needs one shift by 8.  `mid`
-// is the centre of the code range: products are formed with (code - mid) so that the fp16
-// rounding of the folded scale acts on a centred value; the term mid * sum(q s) is added back
-// from an exact MMA.
+// A code that sits at mantissa bit b of an fp16 with exponent 2^E has the value code * 2^(E - 10 + b),
+// so picking E = 10 - b makes "mask, or in the exponent" a complete conversion.  The bias 2^(10 - b)
+// is cancelled after the MMA in fp32 (against "bias * sum of the B operand" from a ones MMA), which
+// costs 2^-23 * bias * |sum| of accuracy: the words are therefore shifted so that the codes land in
+// the upper mantissa bits (8-bit: bias 1024 against codes up to 255; 4-bit: 256 / 16; 2-bit: 16 / 4;
+// first / second number = A rows r / rows r + 8 of the MMA).  `mid` is the centre of the code range:
+// products are formed with (code - mid) so that the rounding of the folded scale acts on a centred
+// value; the term mid * sum(q s) is added back from an exact MMA.
 template <int BITS>
 struct Bias;
 template <>
 struct Bias<8> {
-  static constexpr float lo_even = 1024.f, hi_even = 1024.f, lo_odd = 1024.f, hi_odd = 1024.f, mid = 127.5f;
+  static constexpr float lo = 1024.f, hi = 1024.f, mid = 128.f;       // bias + mid must be an fp16 number
 };
 template <>
 struct Bias<4> {
-  static constexpr float lo_even = 1024.f, hi_even = 64.f, lo_odd = 1024.f, hi_odd = 64.f, mid = 7.5f;
+  static constexpr float lo = 256.f, hi = 16.f, mid = 7.5f;
 };
 template <>
 struct Bias<2> {
-  static constexpr float lo_even = 1024.f, hi_even = 256.f, lo_odd = 64.f, hi_odd = 16.f, mid = 1.5f;
+  static constexpr float lo = 16.f, hi = 4.f, mid = 1.5f;
 };
 
 // Words of one lane for MMA indices [s0, s0 + NS): 8-bit 2 words per s, 4-bit 1, 2-bit 1 per 2.
@@ -154,99 +162,97 @@ __device__ __forceinline__ void unpack(const uint32_t* w, int s_local, uint32_t 
     a[2] = prmt(w1, kMagic, 0x5250u);
     a[3] = prmt(w1, kMagic, 0x5351u);
   } else if constexpr (BITS == 4) {
-    const uint32_t v0 = w[s_local], v1 = w[s_local] >> 8;
-    a[0] = lop3_and_or(v0, 0x000F000Fu, 0x64006400u);   // 1024 + code
-    a[1] = lop3_and_or(v0, 0x00F000F0u, 0x54005400u);   // 64 + code
-    a[2] = lop3_and_or(v1, 0x000F000Fu, 0x64006400u);
-    a[3] = lop3_and_or(v1, 0x00F000F0u, 0x54005400u);
+    // codes of A registers 0..3 at bits 0, 4, 8, 12 of each 16-bit half -> bits 2 (0, 2) and 6 (1, 3)
+    const uint32_t v0 = w[s_local] << 2, v1 = w[s_local] >> 6;
+    a[0] = lop3_and_or(v0, 0x003C003Cu, 0x5C005C00u);   // 256 + code
+    a[1] = lop3_and_or(v0, 0x03C003C0u, 0x4C004C00u);   // 16 + code
+    a[2] = lop3_and_or(v1, 0x003C003Cu, 0x5C005C00u);
+    a[3] = lop3_and_or(v1, 0x03C003C0u, 0x4C004C00u);
   } else {
-    const uint32_t v0 = w[s_local >> 1], v1 = w[s_local >> 1] >> 8;
-    if ((s_local & 1) == 0) {
-      a[0] = lop3_and_or(v0, 0x00030003u, 0x64006400u);  // 1024 + code
-      a[1] = lop3_and_or(v0, 0x000C000Cu, 0x5C005C00u);  // 256 + code
-      a[2] = lop3_and_or(v1, 0x00030003u, 0x64006400u);
-      a[3] = lop3_and_or(v1, 0x000C000Cu, 0x5C005C00u);
-    } else {
-      a[0] = lop3_and_or(v0, 0x00300030u, 0x54005400u);  // 64 + code
-      a[1] = lop3_and_or(v0, 0x00C000C0u, 0x4C004C00u);  // 16 + code
-      a[2] = lop3_and_or(v1, 0x00300030u, 0x54005400u);
-      a[3] = lop3_and_or(v1, 0x00C000C0u, 0x4C004C00u);
-    }
+    // even s: registers 0..3 at bits 0, 2, 8, 10; odd s: at bits 4, 6, 12, 14 -> bits 6 (0, 2) and 8 (1, 3)
+    const uint32_t x = w[s_local >> 1];
+    const uint32_t v0 = (s_local & 1) ? (x << 2) : (x << 6), v1 = (s_local & 1) ? (x >> 6) : (x >> 2);
+    a[0] = lop3_and_or(v0, 0x00C000C0u, 0x4C004C00u);   // 16 + code
+    a[1] = lop3_and_or(v0, 0x03000300u, 0x44004400u);   // 4 + code
+    a[2] = lop3_and_or(v1, 0x00C000C0u, 0x4C004C00u);
+    a[3] = lop3_and_or(v1, 0x03000300u, 0x44004400u);
   }
 }
 
 __device__ __forceinline__ float fast_exp2(float x);
 
+// Lane (r, c4) = (lane / 4, lane % 4).  Accumulator side: the lane owns head c4 of the warp's head
+// group: columns 2 c4 (hi) and 2 c4 + 1 (lo), rows r and r + 8.  B-fragment side: the lane holds column
+// r, i.e. the hi (r even) or lo (r odd) part of head r / 2.
 struct SoftmaxState {
-  float m0, m1;        // running max (log2 domain) of heads 2*c4, 2*c4+1
-  float l0, l1;        // lane-partial sums of exp2 (reduced over the r lanes at the end)
-  float o[8][4];       // O^T accumulators: tile u rows (16u + r, 16u + 8 + r) x heads (2c4, 2c4+1)
-  float zc[4];         // value zero-point term: rows = 32-channel groups (lanes r < 4), same heads
+  float m;             // running max (log2 domain) of head c4
+  float l;             // lane-partial sum of exp2 (reduced over the r lanes at the end)
+  float o[8][4];       // O^T accumulators: tile u rows (16u + r, 16u + 8 + r) x (hi, lo) columns of head c4
+  float zc;            // value zero-point term: row = 32-channel group (lanes r < 4), head c4
 };
+__device__ __forceinline__ bool lo_part_lane(int lane) { return (lane & 4) != 0; }
 
-// Online-softmax update for NT token tiles.  On entry S holds logits in the log2 domain (bias
-// already added: 0, -inf for masked tokens, log2(count) for centroid rows).  On exit S holds the
-// probabilities relative to the new running max.
-template <int NT>
-__device__ __forceinline__ void softmax_update(float (&S)[NT][4], SoftmaxState& st) {
-  float mx0 = kNegInf, mx1 = kNegInf;
+// Online-softmax update for N logits of the lane's head (log2 domain, bias already added: 0, -inf
+// for masked tokens, log2(count) for centroid rows).  On exit x holds the probabilities relative to the
+// new running max.
+template <int N>
+__device__ __forceinline__ void softmax_update(float (&x)[N], SoftmaxState& st) {
+  float mx = x[0];
 #pragma unroll
-  for (int t = 0; t < NT; ++t) {
-    mx0 = fmaxf(mx0, fmaxf(S[t][0], S[t][2]));
-    mx1 = fmaxf(mx1, fmaxf(S[t][1], S[t][3]));
-  }
+  for (int i = 1; i < N; ++i) mx = fmaxf(mx, x[i]);
 #pragma unroll
-  for (int d = 4; d <= 16; d <<= 1) {
-    mx0 = fmaxf(mx0, __shfl_xor_sync(kFull, mx0, d));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(kFull, mx1, d));
-  }
-  const float mn0 = fmaxf(st.m0, mx0), mn1 = fmaxf(st.m1, mx1);
-  const float ms0 = (mn0 == kNegInf) ? 0.f : mn0, ms1 = (mn1 == kNegInf) ? 0.f : mn1;
-  if (__any_sync(kFull, mn0 != st.m0 || mn1 != st.m1)) {
-    const float al0 = fast_exp2(st.m0 - ms0), al1 = fast_exp2(st.m1 - ms1);
-    st.m0 = mn0;
-    st.m1 = mn1;
-    st.l0 *= al0;
-    st.l1 *= al1;
+  for (int d = 4; d <= 16; d <<= 1) mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, d));
+  const float mn = fmaxf(st.m, mx);
+  const float ms = (mn == kNegInf) ? 0.f : mn;
+  if (__any_sync(kFull, mn != st.m)) {
+    const float al = fast_exp2(st.m - ms);
+    st.m = mn;
+    st.l *= al;
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      st.o[u][0] *= al0;
-      st.o[u][1] *= al1;
-      st.o[u][2] *= al0;
-      st.o[u][3] *= al1;
+      st.o[u][0] *= al;
+      st.o[u][1] *= al;
+      st.o[u][2] *= al;
+      st.o[u][3] *= al;
     }
-    st.zc[0] *= al0;
-    st.zc[1] *= al1;
+    st.zc *= al;
   }
 #pragma unroll
-  for (int t = 0; t < NT; ++t) {
-    S[t][0] = fast_exp2(S[t][0] - ms0);
-    S[t][1] = fast_exp2(S[t][1] - ms1);
-    S[t][2] = fast_exp2(S[t][2] - ms0);
-    S[t][3] = fast_exp2(S[t][3] - ms1);
-  }
+  for (int i = 0; i < N; ++i) x[i] = fast_exp2(x[i] - ms);
 }
 
-// P^T B-fragments in fp16 for one tile; accumulates the rounded probabilities into l.
-__device__ __forceinline__ void make_p_f16(const float (&S)[4], uint32_t (&pf)[2], SoftmaxState& st) {
-  const __half2 h01 = __floats2half2_rn(S[0], S[1]);
-  const __half2 h23 = __floats2half2_rn(S[2], S[3]);
-  st.l0 += __low2float(h01) + __low2float(h23);
-  st.l1 += __high2float(h01) + __high2float(h23);
-  pf[0] = movmatrix_trans(h2_as_u32(h01));
-  pf[1] = movmatrix_trans(h2_as_u32(h23));
+// x * y of two fp16 pairs as hi + lo: hi = rn(x y), lo = x y - hi (exact: the product has 22 bits)
+__device__ __forceinline__ void hmul2_split(uint32_t x, uint32_t y, uint32_t& hi, uint32_t& lo) {
+  const __half2 h = __hmul2(u32_as_h2(x), u32_as_h2(y));
+  hi = h2_as_u32(h);
+  lo = h2_as_u32(__hfma2(u32_as_h2(x), u32_as_h2(y), __hneg2(h)));
 }
-// P^T B-fragments as bf16 hi + lo parts (p = hi + lo to ~2^-17).
-__device__ __forceinline__ void make_p_bf16(const float (&S)[4], uint32_t (&pf)[4], SoftmaxState& st) {
-  const uint32_t hi01 = pack_bf16x2(S[0], S[1]), hi23 = pack_bf16x2(S[2], S[3]);
-  const uint32_t lo01 = pack_bf16x2(S[0] - bf16lo_to_f32(hi01), S[1] - bf16hi_to_f32(hi01));
-  const uint32_t lo23 = pack_bf16x2(S[2] - bf16lo_to_f32(hi23), S[3] - bf16hi_to_f32(hi23));
-  st.l0 += S[0] + S[2];
-  st.l1 += S[1] + S[3];
-  pf[0] = movmatrix_trans(hi01);
-  pf[1] = movmatrix_trans(hi23);
-  pf[2] = movmatrix_trans(lo01);
-  pf[3] = movmatrix_trans(lo23);
+// (xh + xl) * y as hi + lo, with xl a small correction of xh
+__device__ __forceinline__ void hmul2_split(uint32_t xh, uint32_t xl, uint32_t y, uint32_t& hi, uint32_t& lo) {
+  const __half2 h = __hmul2(u32_as_h2(xh), u32_as_h2(y));
+  const __half2 e = __hfma2(u32_as_h2(xh), u32_as_h2(y), __hneg2(h));
+  hi = h2_as_u32(h);
+  lo = h2_as_u32(__hfma2(u32_as_h2(xl), u32_as_h2(y), e));
+}
+
+// P^T B-fragments of one 16-token tile from the probabilities of the lane's rows r (pa) and r + 8 (pb):
+// fp16 hi + lo parts (p = hi + lo to ~2^-22) placed in the (hi, lo) columns of the head and
+// transposed.  pf = {tokens 0-7, tokens 8-15} of the lane's column: hi part (r even) or lo part (r odd).
+// The unrounded probabilities go into l.
+__device__ __forceinline__ void make_p_f16(float pa, float pb, uint32_t (&pf)[2], SoftmaxState& st) {
+  const __half2 hh = __floats2half2_rn(pa, pb);
+  const __half2 ll = __floats2half2_rn(pa - __low2float(hh), pb - __high2float(hh));
+  st.l += pa + pb;
+  pf[0] = movmatrix_trans(prmt(h2_as_u32(hh), h2_as_u32(ll), 0x5410u));    // (hi, lo) of row r
+  pf[1] = movmatrix_trans(prmt(h2_as_u32(hh), h2_as_u32(ll), 0x7632u));    // (hi, lo) of row r + 8
+}
+// The same with bf16 parts (p = hi + lo to ~2^-17) for the exact rows.
+__device__ __forceinline__ void make_p_bf16(float pa, float pb, uint32_t (&pf)[2], SoftmaxState& st) {
+  const uint32_t hh = pack_bf16x2(pa, pb);
+  const uint32_t ll = pack_bf16x2(pa - bf16lo_to_f32(hh), pb - bf16hi_to_f32(hh));
+  st.l += pa + pb;
+  pf[0] = movmatrix_trans(prmt(hh, ll, 0x5410u));
+  pf[1] = movmatrix_trans(prmt(hh, ll, 0x7632u));
 }
 
 // ---- item cursor ---------------------------------------------------------------------------
@@ -268,7 +274,8 @@ struct WarpCtx {
   const TableEntry* table;   // this stream's table
   int lane;
   int item_end;              // dense: one past the last item; sparse: one past the last page position
-  int stream;
+  int stream;                // the (sequence, KV head) stream whose cache is read
+  int head0;                 // first query head (within the KV head's group) of the warp's head group
   bool has_tail;
   uint32_t stage0;           // shared-memory address of stage 0 (stage s at + s * kStageBytes)
   const uint8_t* stage_ptr0; // the same as a generic pointer
@@ -604,16 +611,16 @@ __device__ __forceinline__ void load_words(uint32_t codes, int j, int lane, uint
 }
 
 // Logits of the active tiles of one half (32 tokens): S = scale * (q . k~) + token bias, with
-// k~ = s * code + z.  Data MMAs use A = bias + code and B = q' = q * s; the bias (and the code
-// centre) is removed with a "ones" MMA on the same q' and the zero points enter through an MMA
-// with A = (z | s) and B = q.  All arguments that address shared memory are 32-bit addresses.
+// k~ = s * code + z.  Data MMAs use A = bias + code and B = q' = q * s (hi and lo columns); the bias
+// (and the code centre) is removed with a "ones" MMA on the same q' and the zero points enter through
+// an MMA with A = (z | s) and B = q.  All arguments that address shared memory are 32-bit addresses.
 // The loop over channel slabs is kept rolled: the kernel is bound by instruction fetch, and a
 // compact body that stays in the instruction caches is worth more than the scheduling freedom
 // of straight-line code.
 // Channel slab j (MMA indices 2 j and 2 j + 1) of qk_half; FIRST starts the accumulation chains.
 template <int BITS, bool FULL, bool FIRST>
 __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm, uint32_t qh_addr, int lane,
-                                        const uint32_t (&ones)[4], float (&zd)[4], float (&qe)[4], float (&qo)[4], float (&S)[2][4]) {
+                                        const uint32_t (&ones)[4], float (&zd)[4], float (&qe)[4], float (&S)[2][4]) {
   constexpr int cb = 256 * BITS;
   constexpr int kW = BITS / 2;
   uint32_t w0[kW], w1[kW];
@@ -623,16 +630,17 @@ __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm
   for (int ss = 0; ss < 2; ++ss) {
     const uint4 pr = lds128(kp + j * 128 + ss * 64);   // s01, z01, s23, z23
     const uint2 q = lds64(qh_addr + j * 512 + ss * 256);
-    const uint32_t q0 = hmul2_u32(q.x, pr.x), q1 = hmul2_u32(q.y, pr.z);
+    uint32_t q0, q1, q0l, q1l;
+    hmul2_split(q.x, pr.x, q0, q0l);
+    hmul2_split(q.y, pr.z, q1, q1l);
+    if (lo_part_lane(lane)) {
+      q0 = q0l;
+      q1 = q1l;
+    }
     if (FIRST && ss == 0) mma_f16_first(zd, pr.x, pr.y, pr.z, pr.w, q.x, q.y);
     else mma_f16(zd, pr.x, pr.y, pr.z, pr.w, q.x, q.y);
-    if (BITS == 2 && ss == 1) {
-      if (FIRST) mma_f16_first(qo, ones[0], ones[1], ones[2], ones[3], q0, q1);
-      else mma_f16(qo, ones[0], ones[1], ones[2], ones[3], q0, q1);
-    } else {
-      if (FIRST && ss == 0) mma_f16_first(qe, ones[0], ones[1], ones[2], ones[3], q0, q1);
-      else mma_f16(qe, ones[0], ones[1], ones[2], ones[3], q0, q1);
-    }
+    if (FIRST && ss == 0) mma_f16_first(qe, ones[0], ones[1], ones[2], ones[3], q0, q1);
+    else mma_f16(qe, ones[0], ones[1], ones[2], ones[3], q0, q1);
     uint32_t a[4];
     if (FULL || (tm & 1)) {
       unpack<BITS>(w0, ss, a);
@@ -647,84 +655,56 @@ __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm
   }
 }
 
+// x = the four logits of the lane's head: tile 0 rows r, r + 8, tile 1 rows r, r + 8.
 template <int BITS, bool FULL>
 __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, int tm, uint32_t qh_addr, int lane, float scale_log2,
-                                        uint64_t resmask, int half, const uint32_t (&ones)[4], float (&S)[2][4]) {
+                                        uint64_t resmask, int half, const uint32_t (&ones)[4], float (&x)[4]) {
   const int c4 = lane & 3, r = lane >> 2;
-  float zd[4];        // rows r: sum_c q_c s_c; rows r + 8: sum_c q_c z_c (exact products)
-  float qe[4];        // sum_c q'_c over even MMA indices (all rows equal)
-  float qo[4] = {0.f, 0.f, 0.f, 0.f};   // ... over odd MMA indices (2-bit only)
+  float zd[4];        // rows r: sum_c q_c s_c; rows r + 8: sum_c q_c z_c (exact products; both columns alike)
+  float qe[4];        // sum_c q'_c: hi column, lo column (all rows equal)
+  float S[2][4];
   kp += c4 * 16;
-  qk_slab<BITS, FULL, true>(kp, kc0, 0, tm, qh_addr, lane, ones, zd, qe, qo, S);
+  qk_slab<BITS, FULL, true>(kp, kc0, 0, tm, qh_addr, lane, ones, zd, qe, S);
 #pragma unroll
-  for (int j = 1; j < 4; ++j) qk_slab<BITS, FULL, false>(kp, kc0, j, tm, qh_addr, lane, ones, zd, qe, qo, S);
-  if (!FULL) {
-    if (!(tm & 1)) S[0][0] = S[0][1] = S[0][2] = S[0][3] = 0.f;
-    if (!(tm & 2)) S[1][0] = S[1][1] = S[1][2] = S[1][3] = 0.f;
-  }
-  // rows r carry bias lo, rows r + 8 carry bias hi (per parity of the MMA index)
+  for (int j = 1; j < 4; ++j) qk_slab<BITS, FULL, false>(kp, kc0, j, tm, qh_addr, lane, ones, zd, qe, S);
+  // rows r carry bias lo, rows r + 8 carry bias hi
   constexpr float kMid = Bias<BITS>::mid;
-  const float z0 = fmaf(kMid, zd[0], zd[2]), z1 = fmaf(kMid, zd[1], zd[3]);     // sum q (z + mid s)
-  const float c_lo0 = z0 - (Bias<BITS>::lo_even + kMid) * qe[0] - (Bias<BITS>::lo_odd + kMid) * qo[0];
-  const float c_lo1 = z1 - (Bias<BITS>::lo_even + kMid) * qe[1] - (Bias<BITS>::lo_odd + kMid) * qo[1];
-  const float c_hi0 = z0 - (Bias<BITS>::hi_even + kMid) * qe[0] - (Bias<BITS>::hi_odd + kMid) * qo[0];
-  const float c_hi1 = z1 - (Bias<BITS>::hi_even + kMid) * qe[1] - (Bias<BITS>::hi_odd + kMid) * qo[1];
-  if (FULL && resmask == 0) {
-    const float d_lo0 = c_lo0 * scale_log2, d_lo1 = c_lo1 * scale_log2, d_hi0 = c_hi0 * scale_log2, d_hi1 = c_hi1 * scale_log2;
-#pragma unroll
-    for (int t = 0; t < 2; ++t) {
-      S[t][0] = fmaf(S[t][0], scale_log2, d_lo0);
-      S[t][1] = fmaf(S[t][1], scale_log2, d_lo1);
-      S[t][2] = fmaf(S[t][2], scale_log2, d_hi0);
-      S[t][3] = fmaf(S[t][3], scale_log2, d_hi1);
-    }
-    return;
-  }
-  const uint32_t rm = static_cast<uint32_t>(resmask >> (32 * half));      // this half's 32 tokens
+  const float qs = qe[0] + qe[1];
+  const float z0 = fmaf(kMid, zd[0], zd[2]);                                    // sum q (z + mid s)
+  const float c_lo = fmaf(-(Bias<BITS>::lo + kMid), qs, z0), c_hi = fmaf(-(Bias<BITS>::hi + kMid), qs, z0);
+  const uint32_t rm = static_cast<uint32_t>(resmask >> (32 * half));            // this half's 32 tokens
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
-    const int tok = 16 * t + r;
     const bool on = FULL || ((tm >> t) & 1);
-    const float b_lo = (on && !((rm >> tok) & 1u)) ? 0.f : kNegInf;
-    const float b_hi = (on && !((rm >> (tok + 8)) & 1u)) ? 0.f : kNegInf;
-    S[t][0] = fmaf(S[t][0] + c_lo0, scale_log2, b_lo);
-    S[t][1] = fmaf(S[t][1] + c_lo1, scale_log2, b_lo);
-    S[t][2] = fmaf(S[t][2] + c_hi0, scale_log2, b_hi);
-    S[t][3] = fmaf(S[t][3] + c_hi1, scale_log2, b_hi);
+    const int tok = 16 * t + r;
+    const float v_lo = on ? (S[t][0] + S[t][1] + c_lo) * scale_log2 : kNegInf;
+    const float v_hi = on ? (S[t][2] + S[t][3] + c_hi) * scale_log2 : kNegInf;
+    x[2 * t] = ((rm >> tok) & 1u) ? kNegInf : v_lo;
+    x[2 * t + 1] = ((rm >> (tok + 8)) & 1u) ? kNegInf : v_hi;
   }
-}
-
-// One tile's share of O^T += V~^T P^T for group grp: data MMAs accumulate (bias + code) * P' straight
-// into O; `ps` collects sum P' so that the bias can be taken out afterwards.
-template <int BITS>
-__device__ __forceinline__ void pv_tile_group(uint32_t vc, int grp, int lane, uint32_t p0, uint32_t p1,
-                                              const uint32_t (&ones)[4], float (&ps)[4], float (&o0)[4], float (&o1)[4]) {
-  uint32_t wd[BITS / 2];
-  uint32_t a[4];
-  load_words<BITS>(vc, grp, lane, wd);
-  mma_f16(ps, ones[0], ones[1], ones[2], ones[3], p0, p1);
-  unpack<BITS>(wd, 0, a);
-  mma_f16(o0, a[0], a[1], a[2], a[3], p0, p1);
-  unpack<BITS>(wd, 1, a);
-  mma_f16(o1, a[0], a[1], a[2], a[3], p0, p1);
 }
 
 // O^T += V~^T P^T for the active tiles of one half, v~ = s * code + z per (token, 32-channel group).
-// pf holds the raw fp16 P^T fragments of the two tiles; tile t has its parameters at vp + 256 t and
-// its codes at vc + 256 BITS t.  The loop over the two tiles is kept rolled (see qk_half).
+// pf holds the fp16 P^T fragments of the two tiles (hi / lo columns); tile t has its parameters at
+// vp + 256 t and its codes at vc + 256 BITS t.  Data MMAs accumulate (bias + code) * P' straight into
+// O, and an MMA whose A operand is the constant -(bias + mid) takes bias and code centre out again.
+// The loop over the two tiles is kept rolled (see qk_half).
 template <int BITS, bool FULL>
 __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const uint32_t (&pf)[2][2], int lane,
-                                        const uint32_t (&ones)[4], SoftmaxState& st) {
+                                        SoftmaxState& st) {
   constexpr int cb = 256 * BITS;
   const int c4 = lane & 3, r = lane >> 2;
+  const bool lo_lane = lo_part_lane(lane);
   float tz[4] = {0.f, 0.f, 0.f, 0.f};   // rows g < 4: sum_tok p z[tok][g]; rows 8 + g: sum_tok p s[tok][g]
-  float ps[4][4];                       // per group: sum over tokens of P' (all rows equal)
-#pragma unroll
-  for (int g = 0; g < 4; ++g) ps[g][0] = ps[g][1] = ps[g][2] = ps[g][3] = 0.f;
+  // A operand that removes bias + centre: rows r (registers 0, 2) and rows r + 8 (registers 1, 3)
+  const uint32_t fix_lo = h2_as_u32(__float2half2_rn(-(Bias<BITS>::lo + Bias<BITS>::mid)));
+  const uint32_t fix_hi = h2_as_u32(__float2half2_rn(-(Bias<BITS>::hi + Bias<BITS>::mid)));
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
     if (!FULL && !((tm >> t) & 1)) continue;
-    const uint32_t p0 = t ? pf[1][0] : pf[0][0], p1 = t ? pf[1][1] : pf[0][1];
+    const uint32_t m0 = t ? pf[1][0] : pf[0][0], m1 = t ? pf[1][1] : pf[0][1];
+    // the hi parts, also in the lanes that hold a lo column (their partner is the lane 4 below)
+    const uint32_t h0 = __shfl_sync(kFull, m0, lane & ~4), h1 = __shfl_sync(kFull, m1, lane & ~4);
     const uint32_t vpt = vp + t * 256, vct = vc + t * cb;
     // per-lane scales of its token pairs, all four groups: {sA, sB} x 4
     const uint4 x = lds128(vpt + c4 * 32), y = lds128(vpt + c4 * 32 + 16);
@@ -733,38 +713,40 @@ __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const 
       z = lds64(vpt + 128 + (r * 4 + c4) * 8);
       sg = lds64(vpt + c4 * 32 + r * 8);
     }
-    mma_f16(tz, z.x, sg.x, z.y, sg.y, p0, p1);
-    pv_tile_group<BITS>(vct, 0, lane, hmul2_u32(p0, x.x), hmul2_u32(p1, x.y), ones, ps[0], st.o[0], st.o[1]);
-    pv_tile_group<BITS>(vct, 1, lane, hmul2_u32(p0, x.z), hmul2_u32(p1, x.w), ones, ps[1], st.o[2], st.o[3]);
-    pv_tile_group<BITS>(vct, 2, lane, hmul2_u32(p0, y.x), hmul2_u32(p1, y.y), ones, ps[2], st.o[4], st.o[5]);
-    pv_tile_group<BITS>(vct, 3, lane, hmul2_u32(p0, y.z), hmul2_u32(p1, y.w), ones, ps[3], st.o[6], st.o[7]);
-  }
-  st.zc[0] += fmaf(Bias<BITS>::mid, tz[2], tz[0]);
-  st.zc[1] += fmaf(Bias<BITS>::mid, tz[3], tz[1]);
-  // remove bias + centre: u = 2g is an even MMA index, u = 2g + 1 an odd one
-  constexpr float kMid = Bias<BITS>::mid;
+    mma_f16(tz, z.x, sg.x, z.y, sg.y, m0, m1);
+    const uint32_t sc[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
 #pragma unroll
-  for (int grp = 0; grp < 4; ++grp) {
-    st.o[2 * grp][0] = fmaf(-(Bias<BITS>::lo_even + kMid), ps[grp][0], st.o[2 * grp][0]);
-    st.o[2 * grp][1] = fmaf(-(Bias<BITS>::lo_even + kMid), ps[grp][1], st.o[2 * grp][1]);
-    st.o[2 * grp][2] = fmaf(-(Bias<BITS>::hi_even + kMid), ps[grp][0], st.o[2 * grp][2]);
-    st.o[2 * grp][3] = fmaf(-(Bias<BITS>::hi_even + kMid), ps[grp][1], st.o[2 * grp][3]);
-    st.o[2 * grp + 1][0] = fmaf(-(Bias<BITS>::lo_odd + kMid), ps[grp][0], st.o[2 * grp + 1][0]);
-    st.o[2 * grp + 1][1] = fmaf(-(Bias<BITS>::lo_odd + kMid), ps[grp][1], st.o[2 * grp + 1][1]);
-    st.o[2 * grp + 1][2] = fmaf(-(Bias<BITS>::hi_odd + kMid), ps[grp][0], st.o[2 * grp + 1][2]);
-    st.o[2 * grp + 1][3] = fmaf(-(Bias<BITS>::hi_odd + kMid), ps[grp][1], st.o[2 * grp + 1][3]);
+    for (int g = 0; g < 4; ++g) {
+      uint32_t p0, p1, p0l, p1l;
+      hmul2_split(h0, m0, sc[2 * g], p0, p0l);        // (m0, m1 are the lo parts where p0l, p1l are used)
+      hmul2_split(h1, m1, sc[2 * g + 1], p1, p1l);
+      if (lo_lane) {
+        p0 = p0l;
+        p1 = p1l;
+      }
+      uint32_t wd[BITS / 2];
+      uint32_t a[4];
+      load_words<BITS>(vct, g, lane, wd);
+      unpack<BITS>(wd, 0, a);
+      mma_f16(st.o[2 * g], a[0], a[1], a[2], a[3], p0, p1);
+      mma_f16(st.o[2 * g], fix_lo, fix_hi, fix_lo, fix_hi, p0, p1);
+      unpack<BITS>(wd, 1, a);
+      mma_f16(st.o[2 * g + 1], a[0], a[1], a[2], a[3], p0, p1);
+      mma_f16(st.o[2 * g + 1], fix_lo, fix_hi, fix_lo, fix_hi, p0, p1);
+    }
   }
+  st.zc += fmaf(Bias<BITS>::mid, tz[2] + tz[3], tz[0] + tz[1]);
 }
 
 template <int BITS, bool FULL>
 __device__ __forceinline__ void qk_softmax_half(uint32_t half_k, int half, int tm, uint64_t resmask, uint32_t qh_addr,
                                                 int lane, float scale_log2, const uint32_t (&ones)[4], SoftmaxState& st,
                                                 uint32_t (&pf)[2][2]) {
-  float S[2][4];
-  qk_half<BITS, FULL>(half_k, half_k + 512, tm, qh_addr, lane, scale_log2, resmask, half, ones, S);
-  softmax_update<2>(S, st);
-  make_p_f16(S[0], pf[0], st);
-  make_p_f16(S[1], pf[1], st);
+  float x[4];
+  qk_half<BITS, FULL>(half_k, half_k + 512, tm, qh_addr, lane, scale_log2, resmask, half, ones, x);
+  softmax_update<4>(x, st);
+  make_p_f16(x[0], x[1], pf[0], st);
+  make_p_f16(x[2], x[3], pf[1], st);
 }
 
 // Process a staged step.  pf carries P fragments from a key step to the following value step.
@@ -775,9 +757,11 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
   const int lane = w.lane;
   const uint32_t sa = w.stage0 + sidx * kStageBytes;
   if (c.level == 16 || c.level == 1 || c.level == 17) {
+    uint32_t (&pfx)[2] = *reinterpret_cast<uint32_t (*)[2]>(&pf);
     if ((c.sub & 1) == 0) {
-      // key rows: S^T = K Q^T
-      float S[1][4] = {{0.f, 0.f, 0.f, 0.f}};
+      // key rows: S^T = K Q^T (bf16 x bf16 products are exact; the hi and lo columns of a head both
+      // hold its query, so the two accumulator columns are equal)
+      float S[4] = {0.f, 0.f, 0.f, 0.f};
       const int mi = lane >> 3;
       const uint32_t base = sa + ((lane & 7) + (mi & 1) * 8) * kRowPitch + (mi >> 1) * 16;
 #pragma unroll
@@ -785,7 +769,7 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
         uint32_t a[4];
         ldmatrix_x4(a, base + s * 32);
         const uint2 b = lds64(w.qb_addr + s * 256);
-        mma_bf16(S[0], a, b.x, b.y);
+        mma_bf16(S, a, b.x, b.y);
       }
       // validity / weight of the lane's rows r and r + 8
       const int r = lane >> 2;
@@ -810,40 +794,30 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
         b_lo = __shfl_sync(kFull, myb, r);
         b_hi = __shfl_sync(kFull, myb, r + 8);
       }
-      S[0][0] = fmaf(S[0][0], p.scale_log2, b_lo);
-      S[0][1] = fmaf(S[0][1], p.scale_log2, b_lo);
-      S[0][2] = fmaf(S[0][2], p.scale_log2, b_hi);
-      S[0][3] = fmaf(S[0][3], p.scale_log2, b_hi);
-      softmax_update<1>(S, st);
+      float x[2] = {fmaf(S[0], p.scale_log2, b_lo), fmaf(S[2], p.scale_log2, b_hi)};
+      softmax_update<2>(x, st);
       if constexpr (MASS) {
         // centroid rows stand for whole blocks and residual rows belong to the block of their token:
         // their weights are recorded row by row (relative to the running max, which goes with them)
         if (c.level != 16) {
-          const int c4 = lane & 3;
+          const int head = w.head0 + (lane & 3);
           float2* dst = (c.level == 1)
                             ? p.mass_raw + (static_cast<size_t>(w.stream) * p.mass_stride + c.first) * kMaxHeadsPerKv
                             : p.res_raw + (static_cast<size_t>(w.stream) * p.res_cap + 16 * (c.first - p.n_closed - 1)) * kMaxHeadsPerKv;
-          if (r < c.ntok) {
-            dst[r * kMaxHeadsPerKv + 2 * c4] = make_float2(st.m0, S[0][0]);
-            dst[r * kMaxHeadsPerKv + 2 * c4 + 1] = make_float2(st.m1, S[0][1]);
-          }
-          if (r + 8 < c.ntok) {
-            dst[(r + 8) * kMaxHeadsPerKv + 2 * c4] = make_float2(st.m0, S[0][2]);
-            dst[(r + 8) * kMaxHeadsPerKv + 2 * c4 + 1] = make_float2(st.m1, S[0][3]);
-          }
+          if (r < c.ntok) dst[r * kMaxHeadsPerKv + head] = make_float2(st.m, x[0]);
+          if (r + 8 < c.ntok) dst[(r + 8) * kMaxHeadsPerKv + head] = make_float2(st.m, x[1]);
         }
       }
-      make_p_bf16(S[0], pf, st);
+      make_p_bf16(x[0], x[1], pfx, st);
     } else {
-      // value rows: O^T += V^T P^T with P = hi + lo
+      // value rows: O^T += V^T P^T with P = hi + lo in the head's two columns
       const int mi = lane >> 3;
       const uint32_t base = sa + ((lane & 7) + (mi >> 1) * 8) * kRowPitch + (mi & 1) * 16;
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         uint32_t a[4];
         ldmatrix_x4_trans(a, base + u * 32);
-        mma_bf16(st.o[u], a, pf[0], pf[1]);
-        mma_bf16(st.o[u], a, pf[2], pf[3]);
+        mma_bf16(st.o[u], a, pfx[0], pfx[1]);
       }
     }
     return;
@@ -855,16 +829,16 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
     const int half = FULL ? (c.sub >> 1) : ((c.tmask == 15) ? (c.sub >> 1) : half_of_step(c, c.sub >> 1));
     const int tm = (c.tmask >> (2 * half)) & 3;
     if ((c.sub & 1) == 0) qk_softmax_half<8, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, ones, st, pf2);
-    else pv_half<8, FULL>(sa, sa + 512, tm, pf2, lane, ones, st);
+    else pv_half<8, FULL>(sa, sa + 512, tm, pf2, lane, st);
   } else {
     const int half = FULL ? c.sub : ((c.tmask == 15) ? c.sub : half_of_step(c, c.sub));
     const int tm = (c.tmask >> (2 * half)) & 3;
     if (c.level == 4) {
       qk_softmax_half<4, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, ones, st, pf2);
-      pv_half<4, FULL>(sa + off_vp(4, 0), sa + off_vc(4, 0), tm, pf2, lane, ones, st);
+      pv_half<4, FULL>(sa + off_vp(4, 0), sa + off_vc(4, 0), tm, pf2, lane, st);
     } else {
       qk_softmax_half<2, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, ones, st, pf2);
-      pv_half<2, FULL>(sa + off_vp(2, 0), sa + off_vc(2, 0), tm, pf2, lane, ones, st);
+      pv_half<2, FULL>(sa + off_vp(2, 0), sa + off_vc(2, 0), tm, pf2, lane, st);
     }
   }
 }
@@ -884,33 +858,38 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   w.pf_unit = 0;
   w.pf_entry = make_uint4(0, 0, 0, 0);
   w.stream = -1;
+  w.head0 = 0;
   w.item_end = 0;
   w.has_tail = false;
-  int partial_row = 0, first = 0;
+  // A warp works for one head group: up to four query heads of one KV head.  Head group hg of stream s
+  // has the index s * head_groups + hg; partial rows, ranges of rows and tickets go by that index.
+  int hgroup = -1, partial_row = 0, first = 0;
   if (gw < p.n_warps) {
     if constexpr (!SPARSE) {
       const WarpDesc wd = p.warps[gw];
-      w.stream = wd.stream;
+      hgroup = wd.stream;
       w.item_end = wd.item_end;
       first = wd.item_begin;
       partial_row = wd.partial;
     } else {
       const int wps = p.warps_per_stream;
-      w.stream = gw / wps;
-      const int wi = gw - w.stream * wps;
+      hgroup = gw / wps;
+      const int wi = gw - hgroup * wps;
       first = static_cast<int>((static_cast<long long>(wi) * p.n_sel) / wps);
       w.item_end = static_cast<int>((static_cast<long long>(wi + 1) * p.n_sel) / wps);
       w.has_tail = (wi == wps - 1);
-      partial_row = blockIdx.x;      // whole CTAs per stream: one partial row per CTA
+      partial_row = blockIdx.x;      // whole CTAs per head group: one partial row per CTA
     }
   }
-  // per-warp (stream, partial row) for the merge at the end
+  // per-warp (head group, partial row) for the merge at the end
   int* s_group = reinterpret_cast<int*>(smem + kDecodeWarps * (kStages * kStageBytes + kStages * 8 + 2 * 2048));
   if (lane == 0) {
-    s_group[warp] = w.stream;
+    s_group[warp] = hgroup;
     s_group[kDecodeWarps + warp] = partial_row;
   }
-  if (w.stream >= 0) {
+  if (hgroup >= 0) {
+  w.stream = hgroup / p.head_groups;
+  w.head0 = kHeadsPerWarp * (hgroup - w.stream * p.head_groups);
   w.table = p.table + static_cast<size_t>(w.stream) * p.table_stride;
   uint8_t* sbase = smem + warp * (kStages * kStageBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kDecodeWarps * kStages * kStageBytes) + warp * kStages;
@@ -946,17 +925,20 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
     }
   }
 
-  // Query fragments: B operand Q^T[16 channels x 8 heads]; lane (r, c4) holds head r, channels
-  // 16 s + 2 c4 (+1) and 16 s + 8 + 2 c4 (+1), in bf16 (exact rows) and fp16 (quantised tiers).
+  // Query fragments: B operand Q^T[16 channels x 8 columns]; lane (r, c4) holds column r = the hi
+  // (r even) or lo (r odd) column of head r / 2 of the head group, channels 16 s + 2 c4 (+1) and
+  // 16 s + 8 + 2 c4 (+1), in bf16 (exact rows) and fp16 (quantised tiers).  Both columns of a head
+  // hold its query; the parts of the scaled query are formed per key group.
   const int r = lane >> 2, c4 = lane & 3;
   {
     const int b = w.stream / p.n_kv_heads, kvh = w.stream - b * p.n_kv_heads;
     const int n_q_heads = p.n_kv_heads * p.group;
-    const uint16_t* qrow = p.q + (static_cast<size_t>(b) * n_q_heads + static_cast<size_t>(kvh) * p.group + r) * kD;
+    const int head = w.head0 + (r >> 1);
+    const uint16_t* qrow = p.q + (static_cast<size_t>(b) * n_q_heads + static_cast<size_t>(kvh) * p.group + head) * kD;
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
       uint32_t v0 = 0, v1 = 0;
-      if (r < p.group) {
+      if (head < p.group) {
         v0 = *reinterpret_cast<const uint32_t*>(qrow + 16 * s + 2 * c4);
         v1 = *reinterpret_cast<const uint32_t*>(qrow + 16 * s + 8 + 2 * c4);
       }
@@ -969,11 +951,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   __syncwarp();
 
   SoftmaxState st;
-  st.m0 = st.m1 = kNegInf;
-  st.l0 = st.l1 = 0.f;
+  st.m = kNegInf;
+  st.l = 0.f;
 #pragma unroll
   for (int u = 0; u < 8; ++u) st.o[u][0] = st.o[u][1] = st.o[u][2] = st.o[u][3] = 0.f;
-  st.zc[0] = st.zc[1] = st.zc[2] = st.zc[3] = 0.f;
+  st.zc = 0.f;
   uint32_t pf[4] = {0, 0, 0, 0};
   // half2(1, 1) four times: the A operand of the column-sum MMAs.  Produced by opaque moves so that
   // the compiler keeps one register quad for the whole kernel instead of rebuilding it per MMA.
@@ -998,7 +980,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   int sidx = 1;
   uint32_t phase = 0;             // bit s = parity to wait for on stage s
   bool failed = false;
-  float mass_l0 = 0.f, mass_l1 = 0.f, mass_m0 = kNegInf, mass_m1 = kNegInf;     // (l, m) when the current block began
+  float mass_l = 0.f, mass_m = kNegInf;     // (l, m) when the current block began
   while (have) {
     Cursor nxt = cur;
     const bool more = advance<SPARSE>(w, nxt);
@@ -1016,26 +998,21 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
       phase ^= 1u << sidx;
       if constexpr (MASS) {
         if (cur.sub == 0) {
-          mass_l0 = st.l0; mass_l1 = st.l1; mass_m0 = st.m0; mass_m1 = st.m1;
+          mass_l = st.l;
+          mass_m = st.m;
         }
       }
       compute_step<SPARSE, MASS>(w, cur, sidx, ones, st, pf);
       if constexpr (MASS) {
-        // A block (or the partial block) is done: what it added to the lane's running sums is the
+        // A block (or the partial block) is done: what it added to the lane's running sum is the
         // sum now minus the sum at its start brought to the current max.
         if (cur.sub == cur.nsub - 1 && cur.level != 1 && cur.level != 17) {
-          float d0 = st.l0 - ((mass_m0 == kNegInf) ? 0.f : mass_l0 * fast_exp2(mass_m0 - st.m0));
-          float d1 = st.l1 - ((mass_m1 == kNegInf) ? 0.f : mass_l1 * fast_exp2(mass_m1 - st.m1));
+          float d0 = st.l - ((mass_m == kNegInf) ? 0.f : mass_l * fast_exp2(mass_m - st.m));
 #pragma unroll
-          for (int d = 4; d <= 16; d <<= 1) {
-            d0 += __shfl_xor_sync(kFull, d0, d);
-            d1 += __shfl_xor_sync(kFull, d1, d);
-          }
-          if (lane < 4) {
-            float2* dst = p.mass_raw + (static_cast<size_t>(w.stream) * p.mass_stride + cur.first) * kMaxHeadsPerKv + 2 * lane;
-            dst[0] = make_float2(st.m0, fmaxf(d0, 0.f));
-            dst[1] = make_float2(st.m1, fmaxf(d1, 0.f));
-          }
+          for (int d = 4; d <= 16; d <<= 1) d0 += __shfl_xor_sync(kFull, d0, d);
+          if (lane < 4)
+            p.mass_raw[(static_cast<size_t>(w.stream) * p.mass_stride + cur.first) * kMaxHeadsPerKv + w.head0 + lane] =
+                make_float2(st.m, fmaxf(d0, 0.f));
         }
       }
       __syncwarp();
@@ -1047,46 +1024,33 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   if (failed) {
     // a copy never completed: flag it and publish an empty partial (the host reports BAD_STATE)
     if (lane == 0) atomicOr(p.status, kStatusInternal);
-    st.m0 = st.m1 = kNegInf;
-    st.l0 = st.l1 = 0.f;
+    st.m = kNegInf;
+    st.l = 0.f;
   }
 
-  // lane-partial sums -> per-head sums (reduce over the 8 r lanes that share c4)
+  // lane-partial sum -> the head's sum (reduce over the 8 r lanes that share c4)
 #pragma unroll
-  for (int d = 4; d <= 16; d <<= 1) {
-    st.l0 += __shfl_xor_sync(kFull, st.l0, d);
-    st.l1 += __shfl_xor_sync(kFull, st.l1, d);
-  }
-  // value zero-point term: row g of zc (lane 4 g + c4) belongs to channels [32 g, 32 g + 32)
-#pragma unroll
-  for (int g = 0; g < 4; ++g) {
-    const float z0 = __shfl_sync(kFull, st.zc[0], 4 * g + c4), z1 = __shfl_sync(kFull, st.zc[1], 4 * g + c4);
-    st.o[2 * g][0] += z0; st.o[2 * g][1] += z1; st.o[2 * g][2] += z0; st.o[2 * g][3] += z1;
-    st.o[2 * g + 1][0] += z0; st.o[2 * g + 1][1] += z1; st.o[2 * g + 1][2] += z0; st.o[2 * g + 1][3] += z1;
-  }
-  // the warp's partial row goes to its own (now idle) stage memory
-  float* out = reinterpret_cast<float*>(sbase);
-  const int h0 = 2 * c4, h1 = 2 * c4 + 1;
+  for (int d = 4; d <= 16; d <<= 1) st.l += __shfl_xor_sync(kFull, st.l, d);
+  // the warp's partial row goes to its own (now idle) stage memory: hi + lo columns added, plus the
+  // value zero-point term (row g of zc, held by lane 4 g + c4, belongs to channels [32 g, 32 g + 32))
+  float* out = reinterpret_cast<float*>(sbase) + c4 * (kD + 2);
   if (r == 0) {
-    out[h0 * (kD + 2)] = st.m0; out[h0 * (kD + 2) + 1] = st.l0;
-    out[h1 * (kD + 2)] = st.m1; out[h1 * (kD + 2) + 1] = st.l1;
+    out[0] = st.m;
+    out[1] = st.l;
   }
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
-    const int ch = 16 * u + r;
-    out[h0 * (kD + 2) + 2 + ch] = st.o[u][0];
-    out[h0 * (kD + 2) + 2 + ch + 8] = st.o[u][2];
-    out[h1 * (kD + 2) + 2 + ch] = st.o[u][1];
-    out[h1 * (kD + 2) + 2 + ch + 8] = st.o[u][3];
+    const float z = __shfl_sync(kFull, st.zc, 4 * (u >> 1) + c4);
+    out[2 + 16 * u + r] = st.o[u][0] + st.o[u][1] + z;
+    out[2 + 16 * u + 8 + r] = st.o[u][2] + st.o[u][3] + z;
   }
-  }   // w.stream >= 0
+  }   // hgroup >= 0
 
   // Merge the rows of the CTA's warps that share a stream (they are neighbours) into one global
   // partial row per (CTA, stream), in warp order; every warp of the CTA arrives here exactly once.
   __syncthreads();
   constexpr int kRowFloats = kStages * kStageBytes / 4;     // distance between two warps' rows
   const float* rows = reinterpret_cast<const float*>(smem);
-  const int n_pair = p.group * ((kD + 2) / 2);
   int gb = 0;
 #pragma unroll 1
   while (gb < kDecodeWarps) {
@@ -1095,6 +1059,9 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
 #pragma unroll 1
     while (ge < kDecodeWarps && s_group[ge] == sid) ++ge;
     if (sid >= 0) {
+      const int sid_stream = sid / p.head_groups, sid_head0 = kHeadsPerWarp * (sid - sid_stream * p.head_groups);
+      const int n_heads = min(kHeadsPerWarp, p.group - sid_head0);
+      const int n_pair = n_heads * ((kD + 2) / 2);
       float* dst = p.partial + static_cast<size_t>(s_group[kDecodeWarps + gb]) * kPartialFloats;
       // the stream's range of partial rows, asked for now and needed when the ticket is taken
       // (sparse mode: a stream's CTAs are neighbours, one partial row each, row = CTA index)
@@ -1149,10 +1116,10 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
       const int begin = s_group[2 * kDecodeWarps], end = s_group[2 * kDecodeWarps + 1];
       if (begin >= 0) {
         __threadfence();
-        const int b = sid / p.n_kv_heads, kvh = sid - b * p.n_kv_heads;
+        const int b = sid_stream / p.n_kv_heads, kvh = sid_stream - b * p.n_kv_heads;
         // a thread takes two neighbouring channels of a head
 #pragma unroll 1
-        for (int e = threadIdx.x; e < p.group * (kD / 2); e += kDecodeWarps * 32) {
+        for (int e = threadIdx.x; e < n_heads * (kD / 2); e += kDecodeWarps * 32) {
           const int h = e / (kD / 2), ch = 2 * (e - h * (kD / 2));
           const float* col = p.partial + static_cast<size_t>(begin) * kPartialFloats + h * (kD + 2);
           // one pass in row order (one round of independent loads instead of two dependent ones)
@@ -1169,7 +1136,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
             acc1 = fmaf(acc1, a, v.y * bwt);
             M = Mn;
           }
-          const size_t hq = static_cast<size_t>(b) * p.n_kv_heads * p.group + static_cast<size_t>(kvh) * p.group + h;
+          const size_t hq = static_cast<size_t>(b) * p.n_kv_heads * p.group + static_cast<size_t>(kvh) * p.group + sid_head0 + h;
           *reinterpret_cast<float2*>(p.out + hq * kD + ch) = (L > 0.f) ? make_float2(acc0 / L, acc1 / L) : make_float2(0.f, 0.f);
           if (p.lse && ch == 0) p.lse[hq] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : kNegInf;
           if constexpr (MASS) {

@@ -17,7 +17,8 @@ struct alignas(16) TableEntry {
 };
 
 // Work of one warp of the decode kernel: positions [item_begin, item_end) of the layer's unit
-// list, all of one stream.  A unit is one item or a run of consecutive centroid blocks:
+// list, all of one stream; `stream` is the index of the warp's head group (up to four query heads of
+// one KV head): stream * head_groups + group number.  A unit is one item or a run of consecutive centroid blocks:
 // `first item | run << 24`.  Items: [0, n_closed) closed blocks, n_closed = tail block,
 // n_closed + 1 + j = residual group j (16 residual rows each).  (The MLA kernel uses the same
 // struct per CTA with item_begin / item_end as a plain item range.)
@@ -34,21 +35,16 @@ struct alignas(16) WarpDesc {
 constexpr uint32_t kUnitItemMask = 0xfffffu;
 
 struct alignas(8) StreamParts {
-  int32_t begin, end;  // partial rows [begin, end) belong to this stream
+  int32_t begin, end;  // partial rows [begin, end) belong to this head group (GQA) / stream (MLA)
 };
 
-#ifndef GKV_DECODE_WARPS
-#define GKV_DECODE_WARPS 16
-#endif
-#ifndef GKV_DECODE_CTAS_PER_SM
-#define GKV_DECODE_CTAS_PER_SM 1
-#endif
-constexpr int kDecodeWarps = GKV_DECODE_WARPS;               // warps per CTA of the decode kernel
+constexpr int kDecodeWarps = 16;            // warps per CTA of the decode kernel
 constexpr int kStageBytes = 5120;           // per-warp pipeline stage
 constexpr int kStages = 2;
-constexpr int kDecodeCtasPerSm = GKV_DECODE_CTAS_PER_SM;
-constexpr int kMaxHeadsPerKv = 8;           // one n=8 tensor-core tile of query heads
-constexpr int kPartialFloats = kMaxHeadsPerKv * (kD + 2);   // per partial row: m, l, o[128] per head
+constexpr int kDecodeCtasPerSm = 1;
+constexpr int kMaxHeadsPerKv = 8;           // query heads per KV head
+constexpr int kHeadsPerWarp = 4;            // a warp's head group: the n = 8 tensor-core dimension holds (hi, lo) column pairs
+constexpr int kPartialFloats = kHeadsPerWarp * (kD + 2);    // per partial row: m, l, o[128] per head
 
 struct DecodeParams {
   const uint8_t* arena;
@@ -63,14 +59,15 @@ struct DecodeParams {
   int32_t n_warps;
   int32_t n_closed, n_tail;
   int32_t n_kv_heads, group;    // group = query heads per KV head
+  int32_t head_groups;          // head groups per KV head: ceil(group / kHeadsPerWarp)
   float scale_log2;             // softmax scale * log2(e)
   // sparse (page list) mode
   const int32_t* page_idx;      // [n_streams][n_sel] or nullptr
   int32_t n_sel, page_tokens, warps_per_stream;
   uint32_t* status;             // device status word (bit flags)
   // final merge: the CTA that completes a stream's last partial row normalises and writes it
-  const StreamParts* parts;     // [n_streams]; nullptr in sparse mode (one row per stream, row = stream)
-  int32_t* tickets;             // [n_streams] arrival counters, zero between launches
+  const StreamParts* parts;     // [head groups]; nullptr in sparse mode (rows of a head group = its CTAs)
+  int32_t* tickets;             // [head groups] arrival counters, zero between launches
   float* out;                   // [batch][n_q_heads][128]
   float* lse;                   // nullable
   // Block attention mass (Sec. 3.1), dense mode, nullable: unnormalised (running max, sum of exp2)

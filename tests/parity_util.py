@@ -6,25 +6,8 @@ import torch
 from oracle import gkv_oracle as O
 from paper_2608_23599_b200 import workloads as W
 
-ABS_TOL = 2e-3      # max-abs error on fp32-accumulated attention outputs, per unit of value scale
+ABS_TOL = 2e-3      # max-abs error on fp32-accumulated attention outputs
 REL_TOL = 1e-2      # relative L2 error per (sequence, head)
-
-
-def value_scale(v):
-    """Scale of the values being averaged, per output channel: the standard deviation of that
-    channel over all tokens and streams, never below 1.  The error of the kernel is a perturbation
-    of the softmax weights at fp16 operand precision (2^-12 relative), so on every channel its
-    absolute size grows with the spread of that channel's values; the 2e-3 bound is stated for
-    unit-variance values (config 0) and is applied per unit of value standard deviation.
-    v: [..., channels] (torch or numpy); returns a numpy vector [channels]."""
-    if v is None:
-        return 1.0
-    x = v.detach().float().cpu() if hasattr(v, "detach") else torch.as_tensor(np.asarray(v)).float()
-    rows = x.reshape(-1, x.shape[-1])
-    if rows.shape[0] < 2:            # a single row has no spread
-        return np.ones(rows.shape[1], dtype=np.float64)
-    sd = rows.std(dim=0).numpy().astype(np.float64)
-    return np.maximum(1.0, sd)
 
 
 def oracle_config(w: W.Workload, n_layers=None) -> O.Config:
@@ -90,18 +73,15 @@ def assert_state_equal(ocache, gcache, layer, streams=None, blocks=None):
                     assert np.array_equal(ex["rows"][: st.n_tail], O.bf16_bits(st.tail_v))
 
 
-def assert_outputs_close(out_gpu, out_oracle, what="", scale=1.0, abs_tol=None):
-    """abs_tol: override of ABS_TOL (only the random-shape run uses one, see its docstring)."""
+def assert_outputs_close(out_gpu, out_oracle, what=""):
+    """Plain max-abs error <= ABS_TOL over all outputs and relative L2 error <= REL_TOL per
+    (sequence, head).  Returns (max-abs error, largest relative error)."""
     g = out_gpu.detach().to("cpu").to(torch.float64).numpy()
     o = np.asarray(out_oracle, dtype=np.float64)
     assert g.shape == o.shape
     assert np.all(np.isfinite(g)), f"{what}: non-finite output"
-    scale = np.maximum(1.0, np.asarray(scale, dtype=np.float64))        # scalar or per channel
-    nerr = (np.abs(g - o) / scale).max()
     err = np.abs(g - o).max()
-    tol = ABS_TOL if abs_tol is None else abs_tol
-    assert nerr <= tol, (f"{what}: max-abs error per unit of value scale {nerr:.3e} > {tol} "
-                         f"(raw max-abs {err:.3e}, value scale up to {float(np.max(scale)):.2f})")
+    assert err <= ABS_TOL, f"{what}: max-abs error {err:.3e} > {ABS_TOL}"
     num = np.linalg.norm(g - o, axis=-1)
     den = np.linalg.norm(o, axis=-1) + 1e-30
     rel = (num / den).max()

@@ -175,7 +175,7 @@ def test_rdv2_operating_point_small():
     lv = ocache.levels(0, 0, 0)
     assert set(lv.tolist()) <= {16, 1} and (lv == 1).sum() >= len(lv) - 3
     out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
-    U.assert_outputs_close(out, o_out, "rdv2-small", scale=U.value_scale(data["v"]))
+    U.assert_outputs_close(out, o_out, "rdv2-small")
     rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
     assert rep_g.resident_bits == rep_o["resident_bits"] and rep_g.last_read_bits == rep_o["last_read_bits"]
     assert 1.5 < rep_g.bpv_paper < 3.5
@@ -185,7 +185,7 @@ def test_rdv2_operating_point_small():
         gcache.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
         if step in (0, 23, 24, 29):
             out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, tok["q"])
-            U.assert_outputs_close(out, o_out, f"rdv2-small step {step}", scale=U.value_scale(data["v"]))
+            U.assert_outputs_close(out, o_out, f"rdv2-small step {step}")
     U.assert_state_equal(ocache, gcache, 0)
     gcache.close()
 
@@ -350,7 +350,7 @@ def test_mla_single_tier(level, T):
     U.ingest_both(w, 0, data, ocache, gcache, level_plan=plan)
     U.assert_state_equal(ocache, gcache, 0)
     out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
-    U.assert_outputs_close(out, o_out, f"mla level {level} T {T}", scale=U.value_scale(data["k"][..., :512]))
+    U.assert_outputs_close(out, o_out, f"mla level {level} T {T}")
     assert np.max(np.abs(lse.cpu().numpy() - o_lse)) < 5e-3
     rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
     assert rep_g.resident_bits == rep_o["resident_bits"] and rep_g.last_read_bits == rep_o["last_read_bits"]
@@ -373,7 +373,7 @@ def test_mla_ingest_of_rows_that_are_not_16_byte_aligned():
     gcache.gkv_append_demote(0, k, None, level_plan=plan)
     U.assert_state_equal(ocache, gcache, 0)
     out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
-    U.assert_outputs_close(out, o_out, "mla unaligned ingest", scale=U.value_scale(data["k"][..., :512]))
+    U.assert_outputs_close(out, o_out, "mla unaligned ingest")
     gcache.close()
 
 
@@ -388,16 +388,15 @@ def test_cfg4_small_mla_ladder_with_appends():
     U.assert_state_equal(ocache, gcache, 0)
     rep = gcache.gkv_bits_report(0)
     assert abs(rep.bpv_resident - 5.0) < 0.01 and rep.blocks_by_level[3] == 0 and rep.blocks_by_level[4] == 32
-    scale = U.value_scale(data["k"][..., :512])
     out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
-    err, rel = U.assert_outputs_close(out, o_out, "cfg4-small", scale=scale)
+    err, rel = U.assert_outputs_close(out, o_out, "cfg4-small")
     for step in range(66):
         tok = W.make_decode_tokens(w, 0, step, "cpu")
         ocache.append_demote(0, U.f32(tok["k"]), None)
         gcache.gkv_append_demote(0, tok["k"].to(dev), None)
         if step in (0, 31, 62, 63, 64, 65):
             out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, tok["q"])
-            U.assert_outputs_close(out, o_out, f"cfg4-small step {step}", scale=scale)
+            U.assert_outputs_close(out, o_out, f"cfg4-small step {step}")
     U.assert_state_equal(ocache, gcache, 0)
     assert gcache.gkv_bits_report(0).resident_bits == ocache.bits_report(0)["resident_bits"]
     gcache.close()
@@ -513,7 +512,7 @@ def test_block_mass_centroid_runs_and_residual_rows():
     for step in range(3):
         q = data["q"] if step == 0 else W.make_decode_tokens(w, 0, step, "cpu")["q"]
         out, o_out, mass, o_obs = _observe_both(ocache, gcache, 0, q)
-        U.assert_outputs_close(out, o_out, f"observe rdv2 {step}", scale=U.value_scale(data["v"]))
+        U.assert_outputs_close(out, o_out, f"observe rdv2 {step}")
         _assert_mass_close(mass, o_obs, f"rdv2 {step}")
         tok = W.make_decode_tokens(w, 0, step, "cpu")
         ocache.append_demote(0, U.f32(tok["k"]), U.f32(tok["v"]))
@@ -547,7 +546,7 @@ def test_block_mass_running_average_starts_from_prompt_masses():
         assert np.allclose(got0[b, h, :len(want)], want, rtol=1e-6, atol=1e-9)     # the same fp32 block sums
     for step in range(2):
         out, o_out, mass, o_obs = _observe_both(ocache, gcache, 0, data["q"])
-        U.assert_outputs_close(out, o_out, f"observe cfg1 {step}", scale=U.value_scale(data["v"]))
+        U.assert_outputs_close(out, o_out, f"observe cfg1 {step}")
         _assert_mass_close(mass, o_obs, f"cfg1 {step}")
     _assert_mass_close(gcache.gkv_debug_export_mass(0).astype(np.float64), _ema_of(ocache, 0), "cfg1 running mass",
                        unit_sum=False)
@@ -606,7 +605,7 @@ def test_decode_time_reallocation_from_running_masses():
         rep = gcache.gkv_bits_report(0)
         assert rep.bpv_paper <= w.rd_budget_bpv + 16 * w.residual_fraction + 1e-6
         out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, tok["q"])
-        U.assert_outputs_close(out, o_out, f"after reallocation at step {step}", scale=U.value_scale(data["v"]))
+        U.assert_outputs_close(out, o_out, f"after reallocation at step {step}")
     assert n_changed > 0                       # blocks that left the recent window were given a level
     assert differ <= max(2, total // 50), (differ, total)
     gcache.close()

@@ -3,19 +3,9 @@ heads per KV head, batch 1-3, contexts from 1 to 3100 tokens, staircase plans wi
 widths / random external plans / the RD policy, exact residual rows, page sizes 0 / 16 / 32 / 64, up
 to 200 single-token appends with their demotions, page selection with a sparse read.
 
-What is held:
-  * the discrete state (levels, codes, scale / zero, centroids, exact rows, residual indices, selected
-    pages, resident bits) bit for bit, in every case;
-  * the attention outputs within 4e-3 per unit of value scale, and within the stated 2e-3 in at least
-    nine cases out of ten.
-
-Why the looser first bound here: the kernel's tensor-core operands are fp16.  A logit therefore
-carries an error of about 2^-12 of its largest per-channel product q_c * k_c; on the keys' outlier
-channels (x8 by the input recipe) that is ~0.02 before the softmax scale.  It shows in the output
-only when one such token holds about half of a head's attention mass and its value is far from the
-rest (error = w (1 - w) * logit error * value distance); with random rung widths a planted heavy
-token sometimes sits on the 2-bit rung in exactly that position.  Over 360 random cases 3 % exceeded
-2e-3, the worst at 3.3e-3; the benchmark configurations stay below 7.3e-4 (per unit of value scale).
+What is held: the discrete state (levels, codes, scale / zero, centroids, exact rows, residual indices,
+selected pages, resident bits) bit for bit and the attention outputs within the stated bounds
+(max-abs 2e-3, relative L2 1e-2), in every case.
 """
 import random
 
@@ -29,7 +19,6 @@ import parity_util as U
 
 pytestmark = pytest.mark.gpu
 
-LOOSE_TOL = 4e-3
 N_CASES = 36
 
 
@@ -55,7 +44,7 @@ def _draw(case):
 
 
 def _run_case(case, B):
-    """Returns the largest output error of the case per unit of value scale."""
+    """Returns the largest max-abs output error of the case."""
     w, pol, n_app = _draw(case)
     tag = (f"case {case}: {w.n_kv_heads} KV heads x {w.n_q_heads // w.n_kv_heads}, batch {w.batch}, T {w.ctx}, {pol}, "
            f"page {w.page_tokens}, residual {w.residual_fraction}, {n_app} appends, rungs {tuple(w.stair_tokens)}")
@@ -64,15 +53,13 @@ def _run_case(case, B):
     dev = gcache.device
     worst = 0.0
 
-    def check(out, o_out, what, scale):
+    def check(out, o_out, what):
         nonlocal worst
-        U.assert_outputs_close(out, o_out, what, scale=scale, abs_tol=LOOSE_TOL)
-        g = out.detach().cpu().to(torch.float64).numpy()
-        worst = max(worst, float((np.abs(g - o_out) / np.maximum(1.0, scale)).max()))
+        err, _ = U.assert_outputs_close(out, o_out, what)
+        worst = max(worst, float(err))
 
     try:
         data = W.make_layer(w, 0, "cpu", with_mass=(pol == "rd" or w.residual_fraction > 0))
-        scale = U.value_scale(data["v"])
         plan = None
         if pol == "ext":
             prs = np.random.RandomState(case)
@@ -80,14 +67,14 @@ def _run_case(case, B):
         U.ingest_both(w, 0, data, ocache, gcache, level_plan=plan)
         U.assert_state_equal(ocache, gcache, 0)
         out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
-        check(out, o_out, tag, scale)
+        check(out, o_out, tag)
         for step in range(n_app):
             tok = W.make_decode_tokens(w, 0, step, "cpu")
             ocache.append_demote(0, U.f32(tok["k"]), U.f32(tok["v"]))
             gcache.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
             if step in (0, n_app - 1) or (w.ctx + step + 1) % 64 in (0, 1):
                 out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, tok["q"])
-                check(out, o_out, tag + f", step {step}", scale)
+                check(out, o_out, tag + f", step {step}")
         if n_app:
             U.assert_state_equal(ocache, gcache, 0)
         assert gcache.gkv_bits_report(0).resident_bits == ocache.bits_report(0)["resident_bits"], tag
@@ -105,15 +92,14 @@ def _run_case(case, B):
                     assert np.array_equal(pg[b, h, :n_sel], sel_o[b][h]), f"{tag}: selected pages differ for stream {(b, h)}"
             out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"], page_idx_gpu=pages, n_sel=n_sel,
                                                    page_idx_oracle=sel_o)
-            check(out, o_out, tag + ", page-list read", scale)
+            check(out, o_out, tag + ", page-list read")
     finally:
         gcache.close()
     return worst
 
 
-def test_random_shapes_state_bit_exact_and_outputs_within_the_fp16_operand_bound():
+@pytest.mark.parametrize("case", range(N_CASES))
+def test_random_shape_state_bit_exact_and_outputs_within_bounds(case):
     from paper_2608_23599_b200 import binding as B
     B.build()
-    worst = [_run_case(case, B) for case in range(N_CASES)]
-    above = [(case, e) for case, e in enumerate(worst) if e > U.ABS_TOL]
-    assert len(above) * 10 <= N_CASES, f"cases above {U.ABS_TOL}: {above}"
+    _run_case(case, B)
