@@ -696,9 +696,16 @@ __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const 
   const int c4 = lane & 3, r = lane >> 2;
   const bool lo_lane = lo_part_lane(lane);
   float tz[4] = {0.f, 0.f, 0.f, 0.f};   // rows g < 4: sum_tok p z[tok][g]; rows 8 + g: sum_tok p s[tok][g]
-  // A operand that removes bias + centre: rows r (registers 0, 2) and rows r + 8 (registers 1, 3)
-  const uint32_t fix_lo = h2_as_u32(__float2half2_rn(-(Bias<BITS>::lo + Bias<BITS>::mid)));
-  const uint32_t fix_hi = h2_as_u32(__float2half2_rn(-(Bias<BITS>::hi + Bias<BITS>::mid)));
+  // A operand that removes bias + centre: rows r (registers 0, 2) and rows r + 8 (registers 1, 3).
+  // Produced by opaque moves so that the compiler keeps one register quad for the whole half
+  // instead of rebuilding it per MMA.
+  uint32_t fix[4];
+  {
+    const uint32_t f_lo = h2_as_u32(__float2half2_rn(-(Bias<BITS>::lo + Bias<BITS>::mid)));
+    const uint32_t f_hi = h2_as_u32(__float2half2_rn(-(Bias<BITS>::hi + Bias<BITS>::mid)));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) asm volatile("mov.b32 %0, %1;\n" : "=r"(fix[i]) : "r"((i & 1) ? f_hi : f_lo));
+  }
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
     if (!FULL && !((tm >> t) & 1)) continue;
@@ -729,10 +736,10 @@ __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const 
       load_words<BITS>(vct, g, lane, wd);
       unpack<BITS>(wd, 0, a);
       mma_f16(st.o[2 * g], a[0], a[1], a[2], a[3], p0, p1);
-      mma_f16(st.o[2 * g], fix_lo, fix_hi, fix_lo, fix_hi, p0, p1);
+      mma_f16(st.o[2 * g], fix[0], fix[1], fix[2], fix[3], p0, p1);
       unpack<BITS>(wd, 1, a);
       mma_f16(st.o[2 * g + 1], a[0], a[1], a[2], a[3], p0, p1);
-      mma_f16(st.o[2 * g + 1], fix_lo, fix_hi, fix_lo, fix_hi, p0, p1);
+      mma_f16(st.o[2 * g + 1], fix[0], fix[1], fix[2], fix[3], p0, p1);
     }
   }
   st.zc += fmaf(Bias<BITS>::mid, tz[2] + tz[3], tz[0] + tz[1]);

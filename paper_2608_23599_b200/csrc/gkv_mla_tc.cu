@@ -1,19 +1,24 @@
 // Decode attention for latent-attention (MLA) streams on the 5th-generation tensor cores
 // (Sec. 3.1 read path applied to a 576-wide latent row that is key and value at once).
 //
-// One CTA per SM walks a contiguous range of one stream's blocks.  Per 64-token tile:
-//   1. a producer thread stages the packed block (TMA bulk copies, two raw stages, mbarriers);
-//   2. nine warps dequantise it to fp16 (k~ = s * code + z, rounded once) into a 128-byte-swizzled
-//      shared-memory tile [9 panels of 64 channels][64 tokens][128 B];
-//   3. one thread issues tcgen05.mma: S[64 tokens x 16 heads] = K~ Q^T (A = the tile, K-major;
-//      B = the query, K-major; accumulator in tensor memory);
-//   4. four warps read S from tensor memory, run the online softmax and write P (fp16) to shared
-//      memory;
-//   5. the same thread issues O^T[512 channels x 16 heads] += V~^T P^T with A = the same tile read
-//      MN-major (channels are contiguous), four accumulators of 128 channels in tensor memory.
-// Tiles are double-buffered, so the dequantisation of tile i + 1 overlaps the tensor-core work of
-// tile i.  Every wait is bounded; on a time-out the CTA raises kStatusInternal and publishes an
-// empty partial.  Partials of the CTAs of a stream are merged by mla_combine_kernel in CTA order.
+// A quantised latent row is k~[c] = s[c] * code[c] + z[c] with one (s, z) pair per channel and
+// half block (32 tokens, Sec. 3.2).  fp16 operands hold 11 bits, too few for k~ itself, for the
+// query times a scale and for the probabilities, so nothing rounded ever becomes an operand:
+//   * the tile holds the integers code - mid (exact in fp16); exact and centroid rows are bf16 values
+//     (exact in fp16) with s = 1, z = 0;
+//   * the scales go into the query: Q'[half][head][c] = q[head][c] * s[half][c] as an fp16 pair
+//     hi + lo, so S[64 tokens x (2 halves x (hi | lo) x 16 heads)] = T Q'^T in one MMA chain and a
+//     token takes the 32 columns of its own half; sum_c q[c] (z[c] + mid s[c]) is added per (half, head);
+//   * O^T[512 x 16] += V~^T P^T runs per half block on the same tile (read MN-major) with P as an
+//     fp16 pair hi + lo (N = 32), into a per-half accumulator in tensor memory; four warps read it out,
+//     apply s[c] and z[c] in fp32 and add it to the running O^T (also in tensor memory), together with
+//     the rescaling of the online softmax.
+// One CTA per SM walks a contiguous range of one stream's blocks.  Nine warps convert packed
+// blocks (read straight from global memory, prefetched into L2 by a helper warp) into the
+// 128-byte-swizzled tile [9 panels of 64 channels][64 tokens][128 B] and prepare Q'; one warp
+// issues tcgen05.mma; four warps run the softmax and the read-out.  Tiles are double-buffered.
+// Every wait is bounded; on a time-out the CTA raises kStatusInternal and publishes an empty
+// partial.  Partials of the CTAs of a stream are merged by mla_combine_kernel in CTA order.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -27,48 +32,44 @@
 namespace gkv {
 namespace {
 
-constexpr int kTcDequantWarps = 9;                     // 288 threads = 72 chunks x 4 token groups
-constexpr int kTcFirstDequantWarp = 4;                 // warps 0-3 run the softmax
-constexpr int kTcProducerWarp = 13, kTcMmaWarp = 14;
+constexpr int kTcConvertWarps = 9;                     // 288 threads = 72 chunks x 4 token groups
+constexpr int kTcFirstConvertWarp = 4;                 // warps 0-3 run the softmax and the read-out
+constexpr int kTcPrefetchWarp = 13, kTcMmaWarp = 14;
 constexpr int kTcThreads = 15 * 32;
-constexpr int kTcPanelBytes = 64 * 128;                // 64 tokens x 64 channels fp16
-constexpr int kTcTileBytes = 9 * kTcPanelBytes;        // 73728
-constexpr int kTcQBytes = 9 * 16 * 128;                // 16 heads x 576 channels fp16, 9 panels
-constexpr int kTcPBytes = 16 * 128;                    // 16 heads x 64 tokens fp16
-constexpr int kTcRawBytes = 20736;                     // int8 half = 2304 + 32 x 576; 16 exact rows = 18432
+constexpr int kTcPanelBytes = 64 * 128;                // 64 rows x 64 channels fp16
+constexpr int kTcTileBytes = 9 * kTcPanelBytes;        // 73728: 64 rows x 576 channels
+constexpr int kTcPBytes = 2 * 64 * 32;                 // P: hi block and lo block, each 64 tokens x 16 heads fp16
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffTile = 0;
-constexpr int kOffQ = 2 * kTcTileBytes;                // 147456
-constexpr int kOffP = kOffQ + kTcQBytes;               // 165888
-constexpr int kOffRaw = kOffP + 2 * kTcPBytes;         // 169984
-constexpr int kOffMisc = kOffRaw + 2 * kTcRawBytes;    // 211456
-constexpr int kTcSmem = kOffMisc + 2048 + 1024;        // + misc + alignment slack
-// misc: 16 mbarriers (128 B) | tmem base (4 B) @128 | abort flag @132 | bias[2][64] floats @256 |
-//       head maxima [2][4 warps][16] floats @768, rescale flags [2][4] ints @1280 | row sums [4][16] @1344
-constexpr int kMiscTmem = 128, kMiscAbort = 132, kMiscBias = 256, kMiscMax = 768, kMiscSum = 1344;
-enum { kBarRawFull = 0, kBarRawEmpty = 2, kBarKtFull = 4, kBarSFull = 6, kBarPFull = 8, kBarPvDone = 10, kBarMax = 12, kBarSum = 14 };
+constexpr int kOffQp = 2 * kTcTileBytes;               // 147456: Q' of one block, laid out like a tile (row = column of S)
+constexpr int kOffP = kOffQp + kTcTileBytes;           // 221184
+constexpr int kOffMisc = kOffP + kTcPBytes;            // 225280
+constexpr int kTcSmem = kOffMisc + 4608 + 1024;        // + misc + alignment slack = 230912
+// misc: mbarriers (128 B) | tmem base @128 | abort flag @132 | tiles converted @136 | bias[2][64] floats @256 |
+//       head maxima [2][4 warps][16] @768 | row sums [4][16] @1280 | key constants [2 tiles][2 halves][16] @1536 |
+//       probability sums per warp [2 tiles][4][16] @1792 | parts of the key constants [2][2][9 warps][16] @2304
+constexpr int kMiscTmem = 128, kMiscAbort = 132, kMiscDone = 136, kMiscBias = 256, kMiscMax = 768, kMiscSum = 1280;
+constexpr int kMiscConst = 1536;                       // [2][2][16] floats = 256 B
+constexpr int kMiscHalfSum = 1792;                     // [2 tiles][4 warps][16] floats = 512 B: probability sums per warp
+constexpr int kMiscConstPart = 2304;                   // [2][2][9][16] floats = 2304 B, ends at 4608
+enum { kBarKtFull = 0, kBarQpFull = 2, kBarSFull = 4, kBarPFull = 6, kBarPvDone = 7, kBarRFree = 9 };
 constexpr int kTcWaitSpins = 1 << 20;
 constexpr float kNegInfT = -INFINITY;
 constexpr uint32_t kFullT = 0xffffffffu;
-constexpr uint32_t kTmemCols = 128;                    // S[2] at columns 0 / 16, O^T tiles at 32 + 16 i
-constexpr uint32_t kTmemS = 0, kTmemO = 32;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kTmemS = 0;                         // S[2]: 64 columns each
+constexpr uint32_t kTmemR = 128;                       // per-half accumulators: [2 halves][4 channel tiles][32 columns]
+constexpr uint32_t kTmemO = 384;                       // running O^T: [4 channel tiles][16 heads]
 constexpr float kRescaleSlack = 8.f;                   // keep a stale running max while logits stay within 2^8 of it
+constexpr int kPrefetchAhead = 4;                      // blocks the L2 prefetch runs ahead of the conversion
 
 __device__ __forceinline__ uint32_t t_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ void t_bar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ void t_fence_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
-__device__ __forceinline__ void t_bar_expect(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ void t_bar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void t_bulk(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
 }
 __device__ __forceinline__ bool t_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -97,21 +98,6 @@ __device__ __forceinline__ bool t_wait(uint32_t bar, uint32_t parity, volatile i
 // the same for a whole warp: the outcome is made uniform (lanes poll on their own)
 __device__ __forceinline__ bool t_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   return __all_sync(kFullT, t_wait(bar, parity, abort_flag));
-}
-__device__ __forceinline__ uint4 t_lds128(uint32_t a) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
-  return v;
-}
-__device__ __forceinline__ uint2 t_lds64(uint32_t a) {
-  uint2 v;
-  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(a));
-  return v;
-}
-__device__ __forceinline__ uint32_t t_lds32(uint32_t a) {
-  uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(a));
-  return v;
 }
 __device__ __forceinline__ void t_sts128(uint32_t a, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
   asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(a), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
@@ -267,101 +253,82 @@ __device__ __forceinline__ TableEntry tc_entry(const MlaDecodeParams& p, const T
   return table[min(it, p.n_closed)];
 }
 
-// producer warp: copies of stage s of tile t into raw buffer `raw`.  Lane 0 posts the byte count
-// and issues the contiguous copies; the rows of a centroid gather are issued by lanes 0-15, one
-// row each, so that their table look-ups run in parallel.
-__device__ __forceinline__ void tc_issue(const MlaDecodeParams& p, const TableEntry* table, const TcTile& t, int s, uint32_t raw,
-                                         uint32_t bar, int lane) {
-  const uint8_t* slot = p.arena + static_cast<size_t>(t.off256) * 256;
-  if (t.kind == 0) {
-    if (lane == 0) {
-      const uint32_t bytes = static_cast<uint32_t>(mla_half_bytes(t.level));
-      t_bar_expect(bar, bytes);
-      t_bulk(raw, slot + static_cast<size_t>(s) * bytes, bytes, bar);
-    }
-  } else if (t.kind == 1) {
-    if (lane == 0) {
-      const int n = min(16, t.nrows - 16 * s);
-      t_bar_expect(bar, static_cast<uint32_t>(n) * kMlaRowBytes);
-      t_bulk(raw, slot + static_cast<size_t>(16 * s) * kMlaRowBytes, static_cast<uint32_t>(n) * kMlaRowBytes, bar);
-    }
-  } else {
-    const int n = min(16, t.nrows - 16 * s);
-    const uint8_t* src = nullptr;
-    if (lane < n) src = p.arena + static_cast<size_t>(table[t.item + 16 * s + lane].off256) * 256;
-    if (lane == 0) t_bar_expect(bar, static_cast<uint32_t>(n) * kMlaRowBytes);
-    __syncwarp();
-    if (lane < n) t_bulk(raw + lane * kMlaRowBytes, src, kMlaRowBytes, bar);
-  }
-  __syncwarp();
-}
-
 // address of the 16-byte piece (row, chunk j of 8 channels) inside a swizzled tile
 __device__ __forceinline__ uint32_t tc_tile_addr(uint32_t tile, int row, int j) {
   return tile + (j >> 3) * kTcPanelBytes + row * 128 + ((((j & 7) ^ (row & 7))) << 4);
 }
+__device__ __forceinline__ uint32_t tc_bf2_to_h2(uint32_t u) {
+  return t_u(__floats2half2_rn(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)));
+}
+__device__ __forceinline__ uint2 t_ldg64(const void* p) { return __ldg(reinterpret_cast<const uint2*>(p)); }
+__device__ __forceinline__ uint4 t_ldg128(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
 
-// dequantise one half (32 tokens) of a quantised block: thread = (chunk j, 8 tokens)
+// centre of the code range that the tile subtracts (an integer, so that the tile holds integers)
+__device__ __forceinline__ float tc_mid(int level) { return level == 8 ? 128.f : 8.f; }
+
+// One half (32 tokens) of a quantised block -> rows [32 half, 32 half + 32) of the tile as the exact
+// integers code - mid.  Thread = (chunk j of 8 channels, 8 tokens); the packed codes come straight
+// from global memory (a token's chunk is 8 bytes at 8 bits, 4 bytes at 4 bits).
 template <int BITS>
-__device__ __forceinline__ void tc_dequant_half(uint32_t raw, uint32_t tile, int half, int j, int tg) {
-  const uint4 sv = t_lds128(raw + j * 16), zv = t_lds128(raw + kMlaZeroOff * 2 + j * 16);
-  const __half2 s0 = t_h2(sv.x), s1 = t_h2(sv.y), s2 = t_h2(sv.z), s3 = t_h2(sv.w);
-  const __half2 z0 = t_h2(zv.x), z1 = t_h2(zv.y), z2 = t_h2(zv.z), z3 = t_h2(zv.w);
-  const uint32_t codes = raw + mla_kp_bytes() + j * BITS + tg * 8 * (kMlaChunks * BITS);
-  // rows 32 half + 8 tg + i: row & 7 = i, so the swizzled 16-byte slot is (j & 7) ^ i
+__device__ __forceinline__ void tc_convert_half(const uint8_t* half_base, uint32_t tile, int half, int j, int tg) {
+  const uint8_t* codes = half_base + mla_kp_bytes() + static_cast<size_t>(8 * tg) * (kMlaChunks * BITS) + j * BITS;
   const uint32_t out = tile + (j >> 3) * kTcPanelBytes + (32 * half + 8 * tg) * 128;
   const uint32_t jx = (j & 7) << 4;
-  const __half2 b0 = __float2half2_rn(1024.f), b1 = __float2half2_rn(BITS == 4 ? 64.f : 1024.f);
+  uint2 w[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    if constexpr (BITS == 8) w[i] = t_ldg64(codes + i * (kMlaChunks * 8));
+    else w[i] = make_uint2(__ldg(reinterpret_cast<const uint32_t*>(codes + i * (kMlaChunks * 4))), 0u);
+  }
+  // bias + mid of the two code positions of a word (see gkv_layout.cuh for the positions)
+  const __half2 b0 = __float2half2_rn(BITS == 4 ? 1024.f + 8.f : 1024.f + 128.f);
+  const __half2 b1 = __float2half2_rn(BITS == 4 ? 64.f + 8.f : 1024.f + 128.f);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     uint32_t x0, x1, x2, x3;
     if constexpr (BITS == 4) {
-      const uint32_t w = t_lds32(codes + i * (kMlaChunks * 4));
-      const uint32_t v = w >> 8;
-      x0 = t_lop_ao(w, 0x000F000Fu, 0x64006400u);      // 1024 + code (channels 0, 1)
-      x1 = t_lop_ao(w, 0x00F000F0u, 0x54005400u);      // 64 + code   (channels 2, 3)
+      const uint32_t v = w[i].x >> 8;
+      x0 = t_lop_ao(w[i].x, 0x000F000Fu, 0x64006400u);      // 1024 + code (channels 0, 1)
+      x1 = t_lop_ao(w[i].x, 0x00F000F0u, 0x54005400u);      // 64 + code   (channels 2, 3)
       x2 = t_lop_ao(v, 0x000F000Fu, 0x64006400u);
       x3 = t_lop_ao(v, 0x00F000F0u, 0x54005400u);
     } else {
-      const uint2 w = t_lds64(codes + i * (kMlaChunks * 8));
-      x0 = t_prmt(w.x, 0x64006400u, 0x5250u);
-      x1 = t_prmt(w.x, 0x64006400u, 0x5351u);
-      x2 = t_prmt(w.y, 0x64006400u, 0x5250u);
-      x3 = t_prmt(w.y, 0x64006400u, 0x5351u);
+      x0 = t_prmt(w[i].x, 0x64006400u, 0x5250u);
+      x1 = t_prmt(w[i].x, 0x64006400u, 0x5351u);
+      x2 = t_prmt(w[i].y, 0x64006400u, 0x5250u);
+      x3 = t_prmt(w[i].y, 0x64006400u, 0x5351u);
     }
-    // code = x - bias exactly; k~ = code * s + z with one rounding
-    const uint32_t y0 = t_u(__hfma2(__hsub2(t_h2(x0), b0), s0, z0));
-    const uint32_t y1 = t_u(__hfma2(__hsub2(t_h2(x1), b1), s1, z1));
-    const uint32_t y2 = t_u(__hfma2(__hsub2(t_h2(x2), b0), s2, z2));
-    const uint32_t y3 = t_u(__hfma2(__hsub2(t_h2(x3), b1), s3, z3));
-    t_sts128(out + i * 128 + (jx ^ (i << 4)), y0, y1, y2, y3);
+    // rows 32 half + 8 tg + i: row & 7 = i, so the swizzled 16-byte slot is (j & 7) ^ i
+    t_sts128(out + i * 128 + (jx ^ (i << 4)), t_u(__hsub2(t_h2(x0), b0)), t_u(__hsub2(t_h2(x1), b1)), t_u(__hsub2(t_h2(x2), b0)),
+             t_u(__hsub2(t_h2(x3), b1)));
   }
 }
 
-__device__ __forceinline__ uint32_t tc_bf2_to_h2(uint32_t u) {
-  return t_u(__floats2half2_rn(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)));
-}
-// 16 bf16 rows of a raw stage -> fp16 rows [16 q, 16 q + 16) of the tile; rows >= n become zeros
-__device__ __forceinline__ void tc_rows_quarter(uint32_t raw, uint32_t tile, int q, int n, int tid) {
-  const int j = tid % kMlaChunks, rg = tid / kMlaChunks;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = rg * 4 + i;
+// bf16 rows -> fp16 rows of the tile (exact for the magnitudes a cache holds).  Thread = (chunk j, rows
+// 16 rg .. 16 rg + 15); rows >= n become zeros.  CENTROID: row r is the centroid row of block item + r.
+template <bool CENTROID>
+__device__ __forceinline__ void tc_convert_rows(const MlaDecodeParams& p, const TableEntry* table, const TcTile& t, uint32_t tile, int j,
+                                                int rg) {
+  const uint8_t* slot = p.arena + static_cast<size_t>(t.off256) * 256;
+#pragma unroll 4
+  for (int i = 0; i < 16; ++i) {
+    const int r = 16 * rg + i;
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (r < n) {
-      v = t_lds128(raw + r * kMlaRowBytes + j * 16);
+    if (r < t.nrows) {
+      const uint8_t* row = CENTROID ? p.arena + static_cast<size_t>(table[t.item + r].off256) * 256 : slot + static_cast<size_t>(r) * kMlaRowBytes;
+      v = t_ldg128(row + j * 16);
       v.x = tc_bf2_to_h2(v.x);
       v.y = tc_bf2_to_h2(v.y);
       v.z = tc_bf2_to_h2(v.z);
       v.w = tc_bf2_to_h2(v.w);
     }
-    t_sts128(tc_tile_addr(tile, 16 * q + r, j), v.x, v.y, v.z, v.w);
+    t_sts128(tc_tile_addr(tile, r, j), v.x, v.y, v.z, v.w);
   }
 }
 
 // ---- kernel ------------------------------------------------------------------------------------
-// Warp roles: 0-3 softmax (warp w owns tensor-memory lanes 32 w .. 32 w + 31), 4-12 dequantisation,
-// 13 producer, 14 tensor-core issue.
+// Warp roles: 0-3 softmax and read-out (warp w owns tensor-memory lanes 32 w .. 32 w + 31), 4-12
+// conversion and Q', 13 L2 prefetch, 14 tensor-core issue.
 __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __grid_constant__ MlaDecodeParams p) {
   extern __shared__ uint8_t tsm_raw[];
   const WarpDesc cd = p.ctas[blockIdx.x];
@@ -371,208 +338,322 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
   uint8_t* gbase = tsm_raw + (base - t_u32(tsm_raw));
   const uint32_t misc = base + kOffMisc;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + kOffMisc + kMiscAbort);
-  float* bias_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscBias);      // [2][64]
-  float* max_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscMax);        // [2][4][16]
-  float* sum_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscSum);        // [4][16]
+  volatile int* tiles_done = reinterpret_cast<volatile int*>(gbase + kOffMisc + kMiscDone);
+  float* bias_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscBias);            // [2][64]
+  float* max_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscMax);              // [2][4][16]
+  float* sum_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscSum);              // [4][16]
+  float* const_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscConst);          // [2][2][16]
+  float* hsum_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscHalfSum);         // [2][4][16]
+  float* cpart_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscConstPart);      // [2][2][9][16]
   const TableEntry* table = p.table + static_cast<size_t>(cd.stream) * p.table_stride;
   auto bar = [&](int which, int i) { return misc + 8u * static_cast<uint32_t>(which + i); };
 
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) {
-      t_bar_init(bar(kBarRawFull, i), 1);
-      t_bar_init(bar(kBarRawEmpty, i), kTcDequantWarps);
-      t_bar_init(bar(kBarKtFull, i), kTcDequantWarps);
+      t_bar_init(bar(kBarKtFull, i), kTcConvertWarps);
       t_bar_init(bar(kBarSFull, i), 1);
-      t_bar_init(bar(kBarPFull, i), 4);
+      t_bar_init(bar(kBarQpFull, i), kTcConvertWarps);
       t_bar_init(bar(kBarPvDone, i), 1);
-      t_bar_init(bar(kBarMax, i), 4);
     }
-    t_bar_init(bar(kBarSum, 0), 4);
+    t_bar_init(bar(kBarPFull, 0), 4);
+    t_bar_init(bar(kBarRFree, 0), 4);
     *abort_flag = 0;
+    *tiles_done = 0;
     t_fence_async();
   }
   if (warp == 0) t_tmem_alloc(misc + kMiscTmem, kTmemCols);
-  // query -> fp16, K-major swizzled panels [9][16 heads][128 B]
-  {
-    const uint16_t* q = p.q + static_cast<size_t>(cd.stream) * kMlaHeads * kMlaDk;
-    for (int i = tid; i < kMlaHeads * kMlaChunks; i += kTcThreads) {
-      const int h = i / kMlaChunks, j = i % kMlaChunks;
-      const uint4 v = *reinterpret_cast<const uint4*>(q + h * kMlaDk + 8 * j);
-      const uint32_t dst = base + kOffQ + (j >> 3) * (16 * 128) + h * 128 + ((((j & 7) ^ (h & 7))) << 4);
-      t_sts128(dst, tc_bf2_to_h2(v.x), tc_bf2_to_h2(v.y), tc_bf2_to_h2(v.z), tc_bf2_to_h2(v.w));
-    }
-  }
-  t_fence_async();
   t_fence_before();
   __syncthreads();
   t_fence_after();
   const uint32_t tmem = __shfl_sync(kFullT, *reinterpret_cast<volatile uint32_t*>(gbase + kOffMisc + kMiscTmem), 0);
+  const uint16_t* qg = p.q + static_cast<size_t>(cd.stream) * kMlaHeads * kMlaDk;
 
-  if (warp == kTcProducerWarp) {
-    // ---------------- producer: raw stages (lane 0 drives; lanes 0-15 share a centroid gather) ----------------
+  if (warp == kTcPrefetchWarp) {
+    // ---------------- L2 prefetch of the blocks ahead of the conversion ----------------
     TcTile t;
-    int it = cd.item_begin, sg = 0;
-    bool ok = true;
+    int it = cd.item_begin, n = 0, spins = 0;
     TableEntry pre = tc_entry(p, table, it);
-    while (ok && tc_next(p, table, cd.item_end, it, pre, t)) {
+    while (tc_next(p, table, cd.item_end, it, pre, t)) {
       pre = tc_entry(p, table, t.item + t.adv);
-      for (int s = 0; s < t.nstages && ok; ++s, ++sg) {
-        const int b = sg & 1;
-        ok = t_wait_warp(bar(kBarRawEmpty, b), ((sg >> 1) & 1) ^ 1, abort_flag);        // fresh barriers pass
-        if (ok) tc_issue(p, table, t, s, base + kOffRaw + b * kTcRawBytes, bar(kBarRawFull, b), lane);
+      while (n > *tiles_done + kPrefetchAhead && !*abort_flag && ++spins < kTcWaitSpins) __nanosleep(200);
+      if (t.kind != 2 && lane == 0) {
+        const uint8_t* slot = p.arena + static_cast<size_t>(t.off256) * 256;
+        const uint32_t bytes = t.kind == 0 ? 2u * static_cast<uint32_t>(mla_half_bytes(t.level))
+                                           : static_cast<uint32_t>(t.nrows) * kMlaRowBytes;
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(slot), "r"(bytes) : "memory");
       }
       it = t.item + t.adv;
+      ++n;
     }
   } else if (warp == kTcMmaWarp) {
     // ---------------- tensor-core issue (whole warp, one elected lane per instruction) ----------------
-    {
-      constexpr uint32_t kIdQK = t_idesc(64, 16, false), kIdPV = t_idesc(128, 16, true, true);
-      // descriptors differ only in the start-address field (16-byte units in the low word)
-      const uint64_t dq = t_desc(base + kOffQ, 16, 1024);
-      auto issue_qk = [&](int tg) {
-        const int b = tg & 1;
-        const uint64_t da = t_desc(base + kOffTile + b * kTcTileBytes, 16, 1024);
-        const uint32_t d = tmem + kTmemS + 16 * b;
+    constexpr uint32_t kIdQK = t_idesc(64, 64, false), kIdPV = t_idesc(128, 32, true, true);
+    // descriptors differ only in the start-address field (16-byte units in the low word)
+    const uint64_t dq = t_desc(base + kOffQp, 16, 1024);
+    // P: hi block | lo block, each [64 tokens][16 heads] fp16 with the heads contiguous (MN-major),
+    // 32-byte swizzle, 8-token groups of 256 B; the lo block is the second 16 columns (2048 B further)
+    const uint64_t dp = t_desc(base + kOffP, 2048, 256, 6);
+    auto issue_qk = [&](int tg) {
+      const int b = tg & 1;
+      const uint64_t da = t_desc(base + kOffTile + b * kTcTileBytes, 16, 1024);
+      const uint32_t d = tmem + kTmemS + 64 * b;
 #pragma unroll
-        for (int pn = 0; pn < 9; ++pn)
+      for (int pn = 0; pn < 9; ++pn)
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk)
-            t_mma_f16(d, da + ((pn * kTcPanelBytes + kk * 32) >> 4), dq + ((pn * 2048 + kk * 32) >> 4), kIdQK, (pn | kk) != 0);
-        t_commit(bar(kBarSFull, b));
-      };
-      auto issue_pv = [&](int tg) {
-        const int b = tg & 1;
-        const uint64_t da = t_desc(base + kOffTile + b * kTcTileBytes, kTcPanelBytes, 1024);
-        // P: [64 tokens][16 heads] fp16, heads contiguous (MN-major), 32-byte swizzle, 8-token groups of 256 B
-        const uint64_t dp = t_desc(base + kOffP + b * kTcPBytes, 256, 256, 6);
-        const uint32_t first = tg != 0;
+        for (int kk = 0; kk < 4; ++kk)
+          t_mma_f16(d, da + ((pn * kTcPanelBytes + kk * 32) >> 4), dq + ((pn * kTcPanelBytes + kk * 32) >> 4), kIdQK, (pn | kk) != 0);
+      t_commit(bar(kBarSFull, b));
+    };
+    auto issue_pv = [&](int tg) {
+      const int b = tg & 1;
+      const uint64_t da = t_desc(base + kOffTile + b * kTcTileBytes, kTcPanelBytes, 1024);
+#pragma unroll
+      for (int half = 0; half < 2; ++half)
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk)
-            t_mma_f16(tmem + kTmemO + 16 * i, da + ((2 * i * kTcPanelBytes + kk * 2048) >> 4), dp + ((kk * 512) >> 4), kIdPV,
-                      kk != 0 ? 1u : first);
-        t_commit(bar(kBarPvDone, b));
-      };
-      // Event-driven order: the value MMAs of tile pv go out as soon as its P is there, the key MMAs
-      // of tile qk as soon as its tile is there (qk runs at most two tiles ahead of pv: S and the
-      // tile buffers are double).  n_tiles is not known in advance: the iterator tells.
-      TcTile t;
-      int it = cd.item_begin;
-      TableEntry pre = tc_entry(p, table, it);
-      bool more_tiles = tc_next(p, table, cd.item_end, it, pre, t);
-      pre = tc_entry(p, table, t.item + t.adv);
-      int qk = 0, pv = 0, n_known = more_tiles ? 1 : 0;      // tiles [0, n_known) exist so far
-      bool ok = true;
-      int spins = 0;
-      while (ok && (pv < n_known || more_tiles)) {
-        bool progress = false;
-        // key MMAs of tile qk: S[qk & 1] is free once the softmax of tile qk - 2 has published its P
-        if (qk < n_known && qk < pv + 2) {
-          const bool ready = __all_sync(kFullT, t_try_wait(bar(kBarKtFull, qk & 1), (qk >> 1) & 1));
-          if (ready) {
-            t_fence_after();
-            issue_qk(qk);
-            ++qk;
-            // look one tile further
-            it = t.item + t.adv;
-            more_tiles = tc_next(p, table, cd.item_end, it, pre, t);
-            if (more_tiles) {
-              ++n_known;
-              pre = tc_entry(p, table, t.item + t.adv);
-            }
-            progress = true;
-          }
-        }
-        if (pv < qk) {
-          const bool ready = __all_sync(kFullT, t_try_wait(bar(kBarPFull, pv & 1), (pv >> 1) & 1));
-          if (ready) {
-            t_fence_after();
-            issue_pv(pv);
-            ++pv;
-            progress = true;
-          }
-        }
-        if (progress) spins = 0;
-        else if (++spins > kTcWaitSpins || *abort_flag) {
-          *abort_flag = 1;
-          ok = false;
-        }
-        ok = __all_sync(kFullT, ok);
-      }
-    }
-  } else if (warp >= kTcFirstDequantWarp) {
-    // ---------------- dequantisation ----------------
-    const int dt = tid - kTcFirstDequantWarp * 32;          // 0 .. 287
-    const int dj = dt % kMlaChunks, dg = dt / kMlaChunks;   // chunk of 8 channels, token group
+          for (int kk = 2 * half; kk < 2 * half + 2; ++kk)
+            t_mma_f16(tmem + kTmemR + 128 * half + 32 * i, da + ((2 * i * kTcPanelBytes + kk * 2048) >> 4), dp + ((kk * 512) >> 4), kIdPV,
+                      kk != 2 * half);
+      t_commit(bar(kBarPvDone, b));
+    };
+    // Event-driven order: the value MMAs of tile pv go out as soon as its P is there (and the
+    // accumulators of tile pv - 1 have been read out), the key MMAs of tile qk as soon as its tile and
+    // its Q' are there (qk runs at most two tiles ahead of pv: S and the tile buffers are double).
     TcTile t;
-    int it = cd.item_begin, tg = 0, sg = 0;
+    int it = cd.item_begin;
+    TableEntry pre = tc_entry(p, table, it);
+    bool more_tiles = tc_next(p, table, cd.item_end, it, pre, t);
+    pre = tc_entry(p, table, t.item + t.adv);
+    int qk = 0, pv = 0, n_known = more_tiles ? 1 : 0;      // tiles [0, n_known) exist so far
+    bool ok = true;
+    int spins = 0;
+    while (ok && (pv < n_known || more_tiles)) {
+      bool progress = false;
+      if (qk < n_known && qk < pv + 2) {
+        const bool ready = __all_sync(kFullT, t_try_wait(bar(kBarKtFull, qk & 1), (qk >> 1) & 1) && t_try_wait(bar(kBarQpFull, qk & 1), (qk >> 1) & 1));
+        if (ready) {
+          t_fence_after();
+          issue_qk(qk);
+          ++qk;
+          it = t.item + t.adv;
+          more_tiles = tc_next(p, table, cd.item_end, it, pre, t);
+          if (more_tiles) {
+            ++n_known;
+            pre = tc_entry(p, table, t.item + t.adv);
+          }
+          progress = true;
+        }
+      }
+      if (pv < qk) {
+        const bool ready = __all_sync(kFullT, t_try_wait(bar(kBarPFull, 0), pv & 1) && (pv == 0 || t_try_wait(bar(kBarRFree, 0), (pv - 1) & 1)));
+        if (ready) {
+          t_fence_after();
+          issue_pv(pv);
+          ++pv;
+          progress = true;
+        }
+      }
+      if (progress) spins = 0;
+      else if (++spins > kTcWaitSpins || *abort_flag) {
+        *abort_flag = 1;
+        ok = false;
+      }
+      ok = __all_sync(kFullT, ok);
+    }
+  } else if (warp >= kTcFirstConvertWarp) {
+    // ---------------- conversion of blocks into tiles, and Q' ----------------
+    const int dt = tid - kTcFirstConvertWarp * 32;          // 0 .. 287
+    const int dj = dt % kMlaChunks, dg = dt / kMlaChunks;   // tile conversion: chunk of 8 channels, token group
+    // Q': this thread scales the channels of chunk qj for the heads 4 qg .. 4 qg + 3
+    const int cw = warp - kTcFirstConvertWarp;              // = panel of 64 channels
+    const int qj = 8 * cw + (lane >> 2), qgd = lane & 3;
+    uint32_t qh[4][4];                                      // fp16 pairs of the query: [head][channel pair]
+#pragma unroll
+    for (int hh = 0; hh < 4; ++hh) {
+      const uint4 v = t_ldg128(qg + (4 * qgd + hh) * kMlaDk + 8 * qj);
+      qh[hh][0] = tc_bf2_to_h2(v.x);
+      qh[hh][1] = tc_bf2_to_h2(v.y);
+      qh[hh][2] = tc_bf2_to_h2(v.z);
+      qh[hh][3] = tc_bf2_to_h2(v.w);
+    }
+    TcTile t;
+    int it = cd.item_begin, tg = 0;
     bool ok = true;
     TableEntry pre = tc_entry(p, table, it);
     while (ok && tc_next(p, table, cd.item_end, it, pre, t)) {
       pre = tc_entry(p, table, t.item + t.adv);
       const int b = tg & 1;
       const uint32_t tile = base + kOffTile + b * kTcTileBytes;
+      const uint8_t* slot = p.arena + static_cast<size_t>(t.off256) * 256;
       // the tile buffer is free once the value MMAs of tile tg - 2 are done
       if (tg >= 2) ok = t_wait_warp(bar(kBarPvDone, b), ((tg - 2) >> 1) & 1, abort_flag);
       if (!ok) break;
       if (dt < 64) bias_sm[b * 64 + dt] = dt < t.nrows ? (t.kind == 2 ? 6.0f : 0.f) : kNegInfT;   // log2(64) per centroid row
-      const int nq = (t.kind == 0) ? 2 : 4;
-      for (int s = 0; s < nq && ok; ++s) {
-        if (s < t.nstages) {
-          const int rb = sg & 1;
-          ok = t_wait_warp(bar(kBarRawFull, rb), (sg >> 1) & 1, abort_flag);
-          if (!ok) break;
-          const uint32_t raw = base + kOffRaw + rb * kTcRawBytes;
-          if (t.kind == 0) {
-            if (t.level == 8) tc_dequant_half<8>(raw, tile, s, dj, dg);
-            else tc_dequant_half<4>(raw, tile, s, dj, dg);
-          } else {
-            tc_rows_quarter(raw, tile, s, min(16, t.nrows - 16 * s), dt);
-          }
-          __syncwarp();
-          if (lane == 0) t_bar_arrive(bar(kBarRawEmpty, rb));
-          ++sg;
+      if (t.kind == 0) {
+        const size_t hb = static_cast<size_t>(mla_half_bytes(t.level));
+        if (t.level == 8) {
+          tc_convert_half<8>(slot, tile, 0, dj, dg);
+          tc_convert_half<8>(slot + hb, tile, 1, dj, dg);
         } else {
-          tc_rows_quarter(0, tile, s, 0, dt);               // rows past the data: zeros
+          tc_convert_half<4>(slot, tile, 0, dj, dg);
+          tc_convert_half<4>(slot + hb, tile, 1, dj, dg);
         }
+      } else if (t.kind == 1) {
+        tc_convert_rows<false>(p, table, t, tile, dj, dg);
+      } else {
+        tc_convert_rows<true>(p, table, t, tile, dj, dg);
       }
-      if (!ok) break;
       t_fence_async();
       __syncwarp();
       if (lane == 0) t_bar_arrive(bar(kBarKtFull, b));
+      if (dt == 0) *tiles_done = tg + 1;
+      // Q' of this tile: the buffer is free once the key MMAs of tile tg - 1 are done
+      if (tg >= 1) ok = t_wait_warp(bar(kBarSFull, (tg - 1) & 1), ((tg - 1) >> 1) & 1, abort_flag);
+      if (!ok) break;
+      const uint32_t qp = base + kOffQp;
+      const float mid = tc_mid(t.level);
+#pragma unroll 1
+      for (int half = 0; half < 2; ++half) {
+        float cacc[4] = {0.f, 0.f, 0.f, 0.f};
+        uint4 sv = make_uint4(0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u);     // scales 1
+        if (t.kind == 0) {
+          const uint8_t* prm = slot + static_cast<size_t>(half) * mla_half_bytes(t.level);
+          sv = t_ldg128(prm + 16 * qj);
+          const uint4 zv = t_ldg128(prm + 2 * kMlaZeroOff + 16 * qj);
+          // z' = z + mid s per channel (fp32), and its product with the query summed over the chunk
+          const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w}, zw[4] = {zv.x, zv.y, zv.z, zv.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 sf = __half22float2(t_h2(sw[i])), zf = __half22float2(t_h2(zw[i]));
+            const float z0 = fmaf(mid, sf.x, zf.x), z1 = fmaf(mid, sf.y, zf.y);
+#pragma unroll
+            for (int hh = 0; hh < 4; ++hh) {
+              const float2 qf = __half22float2(t_h2(qh[hh][i]));
+              cacc[hh] = fmaf(qf.x, z0, cacc[hh]);
+              cacc[hh] = fmaf(qf.y, z1, cacc[hh]);
+            }
+          }
+        }
+        const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+        for (int hh = 0; hh < 4; ++hh) {
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const __half2 h = __hmul2(t_h2(qh[hh][i]), t_h2(sw[i]));
+            hi[i] = t_u(h);
+            lo[i] = t_u(__hfma2(t_h2(qh[hh][i]), t_h2(sw[i]), __hneg2(h)));
+          }
+          const int row = 32 * half + 4 * qgd + hh;           // column of S: half, (hi | lo), head
+          t_sts128(tc_tile_addr(qp, row, qj), hi[0], hi[1], hi[2], hi[3]);
+          t_sts128(tc_tile_addr(qp, row + 16, qj), lo[0], lo[1], lo[2], lo[3]);
+        }
+        // the warp's part of sum_c q[c] z'[c]: add the 8 chunks of the warp (lanes with the same head quad)
+#pragma unroll
+        for (int hh = 0; hh < 4; ++hh) {
+#pragma unroll
+          for (int d = 4; d <= 16; d <<= 1) cacc[hh] += __shfl_xor_sync(kFullT, cacc[hh], d);
+        }
+        if (lane < 4) {
+          float* dst = cpart_sm + ((b * 2 + half) * kTcConvertWarps + cw) * 16 + 4 * lane;
+          dst[0] = cacc[0]; dst[1] = cacc[1]; dst[2] = cacc[2]; dst[3] = cacc[3];
+        }
+      }
+      t_fence_async();
+      __syncwarp();
+      if (lane == 0) t_bar_arrive(bar(kBarQpFull, b));
       it = t.item + t.adv;
       ++tg;
     }
   } else {
-    // ---------------- softmax (warps 0-3) and the result ----------------
-    float m_run[16], l_part[16];
+    // ---------------- softmax, read-out (warps 0-3) and the result ----------------
+    float m_run[16], l_part[16], alpha[16];
 #pragma unroll
     for (int h = 0; h < 16; ++h) {
       m_run[h] = kNegInfT;
       l_part[h] = 0.f;
+      alpha[h] = 1.f;
     }
-    TcTile t;
-    int it = cd.item_begin, ts = 0, xph = 0;                // xph: exchanges done so far (phase of the exchange barrier)
-    bool ok = true;
     const uint32_t tlane = tmem + (static_cast<uint32_t>(32 * warp) << 16);
+    const int half = warp >> 1;                             // the half block of this warp's 16 token rows
+    bool ok = true;
+    // Read-out of tile `pt` (number pn): O^T <- (O^T + s[c] R[c] + z'[c] sum_t p) * alpha per half, then
+    // per head, for the 128 channels of each of the four channel tiles that this thread's lane holds.
+    auto read_out = [&](const TcTile& pt, int pn, bool scale) {
+      ok = t_wait_warp(bar(kBarPvDone, pn & 1), (pn >> 1) & 1, abort_flag) && ok;
+      t_fence_after();
+      const float* hs = hsum_sm + (pn & 1) * 64;            // [4 warps][16]
+      const float mid = tc_mid(pt.level);
+      const uint8_t* slot = p.arena + static_cast<size_t>(pt.off256) * 256;
+#pragma unroll 1
+      for (int i = 0; i < 4; ++i) {
+        const int c = 128 * i + tid;
+        float o[16];
+        if (pn > 0) {
+          t_ld16(tlane + kTmemO + 16 * i, o);
+        } else {
+#pragma unroll
+          for (int h = 0; h < 16; ++h) o[h] = 0.f;
+        }
+#pragma unroll 1
+        for (int hf = 0; hf < 2; ++hf) {
+          float sc = 1.f, zp = 0.f;
+          if (pt.kind == 0) {
+            const __half* prm = reinterpret_cast<const __half*>(slot + static_cast<size_t>(hf) * mla_half_bytes(pt.level));
+            sc = __half2float(__ldg(prm + c));
+            zp = fmaf(mid, sc, __half2float(__ldg(prm + kMlaZeroOff + c)));
+          }
+          float r[16], rl[16];
+          t_ld16(tlane + kTmemR + 128 * hf + 32 * i, r);
+          t_ld16(tlane + kTmemR + 128 * hf + 32 * i + 16, rl);
+#pragma unroll
+          for (int h = 0; h < 16; ++h) {
+            const float ps = hs[(2 * hf) * 16 + h] + hs[(2 * hf + 1) * 16 + h];       // sum of the half's probabilities
+            o[h] = fmaf(sc, r[h] + rl[h], fmaf(zp, ps, o[h]));
+          }
+        }
+        if (scale) {
+#pragma unroll
+          for (int h = 0; h < 16; ++h) o[h] *= alpha[h];
+        }
+        t_st16(tlane + kTmemO + 16 * i, o);
+      }
+      t_fence_before();
+      __syncwarp();
+      if (lane == 0) t_bar_arrive(bar(kBarRFree, 0));
+    };
+    TcTile t, prev;
+    prev.kind = 1; prev.level = 16; prev.off256 = 0; prev.item = 0; prev.adv = 0; prev.nrows = 0; prev.nstages = 0;
+    int it = cd.item_begin, ts = 0, xph = 0;                // xph: exchanges done so far (phase of the exchange buffers)
     TableEntry pre = tc_entry(p, table, it);
     while (tc_next(p, table, cd.item_end, it, pre, t)) {
       pre = tc_entry(p, table, t.item + t.adv);
       const int b = ts & 1;
+      ok = t_wait_warp(bar(kBarQpFull, b), (ts >> 1) & 1, abort_flag) && ok;   // the parts of the key constants are written
+      // key constants of the tile: (half, head) = thread 0..31 adds the nine parts in a fixed order
+      if (tid < 32) {
+        const float* cp = cpart_sm + ((b * 2 + (tid >> 4)) * kTcConvertWarps) * 16 + (tid & 15);
+        float c = 0.f;
+#pragma unroll
+        for (int w9 = 0; w9 < kTcConvertWarps; ++w9) c += cp[w9 * 16];
+        const_sm[b * 32 + tid] = t.kind == 0 ? c : 0.f;
+      }
       ok = t_wait_warp(bar(kBarSFull, b), (ts >> 1) & 1, abort_flag) && ok;
       t_fence_after();
-      float s[16];
-      t_ld16(tlane + kTmemS + 16 * b, s);
+      float s[16], sl[16];
+      t_ld16(tlane + kTmemS + 64 * b + 32 * half, s);
+      t_ld16(tlane + kTmemS + 64 * b + 32 * half + 16, sl);
+      asm volatile("bar.sync 1, 128;\n" ::: "memory");                    // const_sm is complete
       const int row = 16 * warp + (lane & 15);
       const float bs = (lane < 16) ? bias_sm[b * 64 + row] : kNegInfT;
       // Common case: no logit of the tile exceeds its head's running max by more than the slack;
       // then the (stale) max stays and nothing is reduced.  The four warps agree through one flag
-      // exchange; only when a flag is up are the head maxima reduced and O rescaled.
+      // exchange; only when a flag is up are the head maxima reduced and the sums rescaled.
       bool mine = false;
 #pragma unroll
       for (int h = 0; h < 16; ++h) {
-        s[h] = (bs == kNegInfT) ? kNegInfT : fmaf(s[h], p.scale_log2, bs);
+        s[h] = (bs == kNegInfT) ? kNegInfT : fmaf(s[h] + sl[h] + const_sm[b * 32 + half * 16 + h], p.scale_log2, bs);
         mine |= s[h] > m_run[h] + kRescaleSlack;            // also true for the first finite logit (max = -inf)
       }
       uint32_t need_u;
@@ -601,7 +682,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
           for (int h = 0; h < 16; ++h) mbuf[warp * 16 + h] = mx[h];
         }
         asm volatile("bar.sync 1, 128;\n" ::: "memory");
-        float alpha[16];
 #pragma unroll
         for (int h = 0; h < 16; ++h) {
           const float bm = fmaxf(fmaxf(mbuf[h], mbuf[16 + h]), fmaxf(mbuf[32 + h], mbuf[48 + h]));
@@ -611,48 +691,57 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
           l_part[h] *= alpha[h];
         }
         ++xph;
-        if (ts > 0) {                                       // O holds the tiles before ts: rescale it
-          ok = t_wait_warp(bar(kBarPvDone, (ts - 1) & 1), ((ts - 1) >> 1) & 1, abort_flag) && ok;
-          t_fence_after();
-#pragma unroll 1
-          for (int i = 0; i < 4; ++i) {
-            float o[16];
-            t_ld16(tlane + kTmemO + 16 * i, o);
-#pragma unroll
-            for (int h = 0; h < 16; ++h) o[h] *= alpha[h];
-            t_st16(tlane + kTmemO + 16 * i, o);
-          }
-        }
       }
-      // probabilities relative to the (possibly stale) running max; the rounded value is what is summed
+      // probabilities relative to the (possibly stale) running max as fp16 pairs hi + lo; the
+      // unrounded value is what is summed
+      float pr[16];
+#pragma unroll
+      for (int h = 0; h < 16; ++h) {
+        pr[h] = (lane < 16 && s[h] != kNegInfT) ? t_ex2(s[h] - m_run[h]) : 0.f;
+        l_part[h] += pr[h];
+      }
+      // the P buffer is free once the value MMAs of the tile before are done
+      if (ts > 0) ok = t_wait_warp(bar(kBarPvDone, (ts - 1) & 1), ((ts - 1) >> 1) & 1, abort_flag) && ok;
       if (lane < 16) {
-        uint32_t pk[8];
+        uint32_t pk[8], pl[8];
 #pragma unroll
         for (int h = 0; h < 16; h += 2) {
-          const float p0 = (s[h] == kNegInfT) ? 0.f : t_ex2(s[h] - m_run[h]);
-          const float p1 = (s[h + 1] == kNegInfT) ? 0.f : t_ex2(s[h + 1] - m_run[h + 1]);
-          const __half2 ph = __floats2half2_rn(p0, p1);
-          l_part[h] += __low2float(ph);
-          l_part[h + 1] += __high2float(ph);
+          const __half2 ph = __floats2half2_rn(pr[h], pr[h + 1]);
           pk[h >> 1] = t_u(ph);
+          pl[h >> 1] = t_u(__floats2half2_rn(pr[h] - __low2float(ph), pr[h + 1] - __high2float(ph)));
         }
         // row of 16 heads (32 B) of token `row`; 32-byte swizzle: the 16-byte halves swap on bit 7
-        const uint32_t prow = base + kOffP + b * kTcPBytes + row * 32;
+        const uint32_t prow = base + kOffP + row * 32;
         const uint32_t sw = ((row >> 2) & 1) << 4;
         t_sts128(prow + sw, pk[0], pk[1], pk[2], pk[3]);
         t_sts128(prow + (sw ^ 16), pk[4], pk[5], pk[6], pk[7]);
+        t_sts128(prow + 2048 + sw, pl[0], pl[1], pl[2], pl[3]);
+        t_sts128(prow + 2048 + (sw ^ 16), pl[4], pl[5], pl[6], pl[7]);
+      }
+      // sums of the warp's 16 rows per head (for the zero-point term of the read-out), fixed order
+#pragma unroll
+      for (int d = 8; d >= 1; d >>= 1)
+#pragma unroll
+        for (int h = 0; h < 16; ++h) pr[h] += __shfl_xor_sync(kFullT, pr[h], d);
+      if (lane == 0) {
+#pragma unroll
+        for (int h = 0; h < 16; ++h) hsum_sm[b * 64 + warp * 16 + h] = pr[h];
       }
       t_fence_async();
       t_fence_before();
       __syncwarp();
-      if (lane == 0) t_bar_arrive(bar(kBarPFull, b));
+      if (lane == 0) t_bar_arrive(bar(kBarPFull, 0));
+      // read-out of the tile before (its accumulators are complete: the wait above), rescaled when this
+      // tile moved the running max
+      if (ts > 0) read_out(prev, ts - 1, need);
+      prev = t;
       it = t.item + t.adv;
       ++ts;
     }
     // ---------------- result ----------------
+    asm volatile("bar.sync 1, 128;\n" ::: "memory");                      // hsum_sm of the last tile
+    if (ts > 0) read_out(prev, ts - 1, false);
     float* out = p.partial + static_cast<size_t>(cd.partial) * kMlaPartialFloats;
-    if (ts > 0) ok = t_wait_warp(bar(kBarPvDone, (ts - 1) & 1), ((ts - 1) >> 1) & 1, abort_flag) && ok;
-    t_fence_after();
 #pragma unroll
     for (int d = 8; d >= 1; d >>= 1)
 #pragma unroll
