@@ -24,6 +24,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <type_traits>
 
 #include "gkv_internal.h"
 #include "gkv_layout.cuh"
@@ -33,9 +34,10 @@ namespace gkv {
 namespace {
 
 constexpr int kTcConvertWarps = 9;                     // 288 threads = 72 chunks x 4 token groups
-constexpr int kTcFirstConvertWarp = 4;                 // warps 0-3 run the softmax and the read-out
-constexpr int kTcPrefetchWarp = 13, kTcMmaWarp = 14;
-constexpr int kTcThreads = 15 * 32;
+constexpr int kTcFirstConvertWarp = 8;                 // warps 0-3: softmax + read-out, warps 4-7: read-out
+constexpr int kTcMmaWarp = 17;
+constexpr int kTcThreads = 18 * 32;
+constexpr int kTcReadTiles0 = 0;                       // channel tiles (of 128) read out by warps 0-3 beside the softmax; warps 4-7 take the rest
 constexpr int kTcPanelBytes = 64 * 128;                // 64 rows x 64 channels fp16
 constexpr int kTcTileBytes = 9 * kTcPanelBytes;        // 73728: 64 rows x 576 channels
 constexpr int kTcPBytes = 2 * 64 * 32;                 // P: hi block and lo block, each 64 tokens x 16 heads fp16
@@ -44,15 +46,18 @@ constexpr int kOffTile = 0;
 constexpr int kOffQp = 2 * kTcTileBytes;               // 147456: Q' of one block, laid out like a tile (row = column of S)
 constexpr int kOffP = kOffQp + kTcTileBytes;           // 221184
 constexpr int kOffMisc = kOffP + kTcPBytes;            // 225280
-constexpr int kTcSmem = kOffMisc + 4608 + 1024;        // + misc + alignment slack = 230912
-// misc: mbarriers (128 B) | tmem base @128 | abort flag @132 | tiles converted @136 | bias[2][64] floats @256 |
+constexpr int kTcSmem = kOffMisc + 5120 + 1024;        // + misc + alignment slack = 231424
+// misc: mbarriers (128 B) | tmem base @128 | abort flag @132 | bias[2][64] floats @256 |
 //       head maxima [2][4 warps][16] @768 | row sums [4][16] @1280 | key constants [2 tiles][2 halves][16] @1536 |
-//       probability sums per warp [2 tiles][4][16] @1792 | parts of the key constants [2][2][9 warps][16] @2304
-constexpr int kMiscTmem = 128, kMiscAbort = 132, kMiscDone = 136, kMiscBias = 256, kMiscMax = 768, kMiscSum = 1280;
+//       probability sums per warp [2 tiles][4][16] @1792 | parts of the key constants [2][2][9 warps][16] @2304 |
+//       rescale factors [2][16] + flag [2] @4608
+constexpr int kMiscTmem = 128, kMiscAbort = 132, kMiscBias = 256, kMiscMax = 768, kMiscSum = 1280;
 constexpr int kMiscConst = 1536;                       // [2][2][16] floats = 256 B
 constexpr int kMiscHalfSum = 1792;                     // [2 tiles][4 warps][16] floats = 512 B: probability sums per warp
 constexpr int kMiscConstPart = 2304;                   // [2][2][9][16] floats = 2304 B, ends at 4608
-enum { kBarKtFull = 0, kBarQpFull = 2, kBarSFull = 4, kBarPFull = 6, kBarPvDone = 7, kBarRFree = 9 };
+constexpr int kMiscAlpha = 4608;                       // [2][16] floats, then [2] ints (1 = rescale): ends at 4744
+constexpr int kMiscHalfSum2 = 4864;                    // [2 tiles][2 halves][16] floats = 256 B: sums per half block
+enum { kBarKtFull = 0, kBarQpFull = 2, kBarSFull = 4, kBarPFull = 6, kBarPvDone = 7, kBarRFree = 9, kBarHsFull = 10 };
 constexpr int kTcWaitSpins = 1 << 20;
 constexpr float kNegInfT = -INFINITY;
 constexpr uint32_t kFullT = 0xffffffffu;
@@ -60,8 +65,8 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemS = 0;                         // S[2]: 64 columns each
 constexpr uint32_t kTmemR = 128;                       // per-half accumulators: [2 halves][4 channel tiles][32 columns]
 constexpr uint32_t kTmemO = 384;                       // running O^T: [4 channel tiles][16 heads]
+constexpr int kPrefetchAhead = 6;                      // tiles the L2 prefetch runs ahead of the key MMAs
 constexpr float kRescaleSlack = 8.f;                   // keep a stale running max while logits stay within 2^8 of it
-constexpr int kPrefetchAhead = 4;                      // blocks the L2 prefetch runs ahead of the conversion
 
 __device__ __forceinline__ uint32_t t_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ void t_bar_init(uint32_t bar, uint32_t count) {
@@ -80,14 +85,17 @@ __device__ __forceinline__ bool t_try_wait(uint32_t bar, uint32_t parity) {
       "selp.u32 %0, 1, 0, p;\n"
       "}\n"
       : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(2000)
+      : "r"(bar), "r"(parity), "r"(200)
       : "memory");
   return ok != 0;
 }
-// Bounded wait; a time-out raises the CTA's abort flag, which every other waiter also watches.
+// Bounded wait; a time-out raises the CTA's abort flag, which every other waiter also watches.  A
+// waiting thread backs off between polls: the polls of eighteen warps otherwise take a third of the
+// SM's issue slots from the warps that work.
 __device__ __forceinline__ bool t_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   int spins = 0;
   while (!t_try_wait(bar, parity)) {
+    __nanosleep(spins < 4 ? 64 : 256);
     if (++spins > kTcWaitSpins || *abort_flag) {
       *abort_flag = 1;
       return false;
@@ -163,6 +171,15 @@ __device__ __forceinline__ void t_ld16(uint32_t taddr, float (&v)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+// the same without the wait: several loads may be in flight; t_wait_ld() before the first use
+__device__ __forceinline__ void t_ld16_async(uint32_t taddr, float (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]), "=f"(v[8]),
+        "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void t_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void t_st16(uint32_t taddr, const float (&v)[16]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n" ::"r"(taddr),
@@ -260,47 +277,55 @@ __device__ __forceinline__ uint32_t tc_tile_addr(uint32_t tile, int row, int j) 
 __device__ __forceinline__ uint32_t tc_bf2_to_h2(uint32_t u) {
   return t_u(__floats2half2_rn(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)));
 }
-__device__ __forceinline__ uint2 t_ldg64(const void* p) { return __ldg(reinterpret_cast<const uint2*>(p)); }
 __device__ __forceinline__ uint4 t_ldg128(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
 
 // centre of the code range that the tile subtracts (an integer, so that the tile holds integers)
 __device__ __forceinline__ float tc_mid(int level) { return level == 8 ? 128.f : 8.f; }
 
-// One half (32 tokens) of a quantised block -> rows [32 half, 32 half + 32) of the tile as the exact
-// integers code - mid.  Thread = (chunk j of 8 channels, 8 tokens); the packed codes come straight
-// from global memory (a token's chunk is 8 bytes at 8 bits, 4 bytes at 4 bits).
-template <int BITS>
-__device__ __forceinline__ void tc_convert_half(const uint8_t* half_base, uint32_t tile, int half, int j, int tg) {
-  const uint8_t* codes = half_base + mla_kp_bytes() + static_cast<size_t>(8 * tg) * (kMlaChunks * BITS) + j * BITS;
-  const uint32_t out = tile + (j >> 3) * kTcPanelBytes + (32 * half + 8 * tg) * 128;
-  const uint32_t jx = (j & 7) << 4;
-  uint2 w[8];
+// A quantised block -> the tile as the exact integers code - mid.  Thread = (chunk j of 8 channels, 8
+// tokens of each half); the packed codes come straight from global memory (a token's chunk is 8
+// bytes at 8 bits, 4 bytes at 4 bits).  The loads are issued early (tc_load_block), while the
+// thread still waits for the tile buffer.
+__device__ __forceinline__ void tc_load_block(const uint8_t* slot, int bits, int j, int tg, uint2 (&w)[2][8]) {
+  const int row = kMlaChunks * bits;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    if constexpr (BITS == 8) w[i] = t_ldg64(codes + i * (kMlaChunks * 8));
-    else w[i] = make_uint2(__ldg(reinterpret_cast<const uint32_t*>(codes + i * (kMlaChunks * 4))), 0u);
+  for (int half = 0; half < 2; ++half) {
+    const uint8_t* codes = slot + static_cast<size_t>(half) * mla_half_bytes(bits) + mla_kp_bytes() + static_cast<size_t>(8 * tg) * row + j * bits;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (bits == 8) w[half][i] = __ldg(reinterpret_cast<const uint2*>(codes + i * row));
+      else w[half][i] = make_uint2(__ldg(reinterpret_cast<const uint32_t*>(codes + i * row)), 0u);
+    }
   }
+}
+template <int BITS>
+__device__ __forceinline__ void tc_store_block(const uint2 (&w)[2][8], uint32_t tile, int j, int tg) {
   // bias + mid of the two code positions of a word (see gkv_layout.cuh for the positions)
   const __half2 b0 = __float2half2_rn(BITS == 4 ? 1024.f + 8.f : 1024.f + 128.f);
   const __half2 b1 = __float2half2_rn(BITS == 4 ? 64.f + 8.f : 1024.f + 128.f);
+  const uint32_t jx = (j & 7) << 4;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    uint32_t x0, x1, x2, x3;
-    if constexpr (BITS == 4) {
-      const uint32_t v = w[i].x >> 8;
-      x0 = t_lop_ao(w[i].x, 0x000F000Fu, 0x64006400u);      // 1024 + code (channels 0, 1)
-      x1 = t_lop_ao(w[i].x, 0x00F000F0u, 0x54005400u);      // 64 + code   (channels 2, 3)
-      x2 = t_lop_ao(v, 0x000F000Fu, 0x64006400u);
-      x3 = t_lop_ao(v, 0x00F000F0u, 0x54005400u);
-    } else {
-      x0 = t_prmt(w[i].x, 0x64006400u, 0x5250u);
-      x1 = t_prmt(w[i].x, 0x64006400u, 0x5351u);
-      x2 = t_prmt(w[i].y, 0x64006400u, 0x5250u);
-      x3 = t_prmt(w[i].y, 0x64006400u, 0x5351u);
+  for (int half = 0; half < 2; ++half) {
+    const uint32_t out = tile + (j >> 3) * kTcPanelBytes + (32 * half + 8 * tg) * 128;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t x0, x1, x2, x3;
+      if constexpr (BITS == 4) {
+        const uint32_t v = w[half][i].x >> 8;
+        x0 = t_lop_ao(w[half][i].x, 0x000F000Fu, 0x64006400u);      // 1024 + code (channels 0, 1)
+        x1 = t_lop_ao(w[half][i].x, 0x00F000F0u, 0x54005400u);      // 64 + code   (channels 2, 3)
+        x2 = t_lop_ao(v, 0x000F000Fu, 0x64006400u);
+        x3 = t_lop_ao(v, 0x00F000F0u, 0x54005400u);
+      } else {
+        x0 = t_prmt(w[half][i].x, 0x64006400u, 0x5250u);
+        x1 = t_prmt(w[half][i].x, 0x64006400u, 0x5351u);
+        x2 = t_prmt(w[half][i].y, 0x64006400u, 0x5250u);
+        x3 = t_prmt(w[half][i].y, 0x64006400u, 0x5351u);
+      }
+      // rows 32 half + 8 tg + i: row & 7 = i, so the swizzled 16-byte slot is (j & 7) ^ i
+      t_sts128(out + i * 128 + (jx ^ (i << 4)), t_u(__hsub2(t_h2(x0), b0)), t_u(__hsub2(t_h2(x1), b1)), t_u(__hsub2(t_h2(x2), b0)),
+               t_u(__hsub2(t_h2(x3), b1)));
     }
-    // rows 32 half + 8 tg + i: row & 7 = i, so the swizzled 16-byte slot is (j & 7) ^ i
-    t_sts128(out + i * 128 + (jx ^ (i << 4)), t_u(__hsub2(t_h2(x0), b0)), t_u(__hsub2(t_h2(x1), b1)), t_u(__hsub2(t_h2(x2), b0)),
-             t_u(__hsub2(t_h2(x3), b1)));
   }
 }
 
@@ -327,8 +352,72 @@ __device__ __forceinline__ void tc_convert_rows(const MlaDecodeParams& p, const 
 }
 
 // ---- kernel ------------------------------------------------------------------------------------
-// Warp roles: 0-3 softmax and read-out (warp w owns tensor-memory lanes 32 w .. 32 w + 31), 4-12
-// conversion and Q', 13 L2 prefetch, 14 tensor-core issue.
+// Warp roles: 0-3 softmax + read-out of the first channel tile, 4-7 read-out of the other three
+// (warp w owns tensor-memory lanes 32 (w % 4) .. + 31), 8-16 conversion and Q', 17 tensor-core issue.
+
+// Read-out of the accumulators of tile `pt` (number pn) for the channel tiles [i0, i1): O^T *= alpha
+// when this tile moved the running max (O^T holds the tiles before it), then per half block
+// O^T <- O^T + s[c] R[c] + z'[c] sum_t p.  A thread owns channel 128 i + lt of every channel tile i (its
+// tensor-memory lane lt).  hs = [2 halves][16 heads] sums of the tile's probabilities.
+__device__ __forceinline__ bool tc_read_out(const MlaDecodeParams& p, const TcTile& pt, int pn, int i0, int i1, bool scale,
+                                            const float* alpha_sm, const float* hs, uint32_t tlane, int lt, uint32_t bar_pv,
+                                            volatile int* abort_flag) {
+  // scale and zero point of this thread's channels in both halves (asked for before the wait)
+  const float mid = tc_mid(pt.level);
+  const uint8_t* slot = p.arena + static_cast<size_t>(pt.off256) * 256;
+  __half sch[4][2], zph[4][2];
+  if (pt.kind == 0) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (i < i0 || i >= i1) continue;
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const __half* prm = reinterpret_cast<const __half*>(slot + static_cast<size_t>(hf) * mla_half_bytes(pt.level));
+        sch[i][hf] = __ldg(prm + 128 * i + lt);
+        zph[i][hf] = __ldg(prm + kMlaZeroOff + 128 * i + lt);
+      }
+    }
+  }
+  const bool ok = t_wait_warp(bar_pv, (pn >> 1) & 1, abort_flag);
+  t_fence_after();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    if (i < i0 || i >= i1) continue;
+    float o[16], r[16], rl[16];
+    if (pn > 0) {
+      t_ld16_async(tlane + kTmemO + 16 * i, o);
+    } else {
+#pragma unroll
+      for (int h = 0; h < 16; ++h) o[h] = 0.f;
+    }
+    t_ld16_async(tlane + kTmemR + 32 * i, r);
+    t_ld16_async(tlane + kTmemR + 32 * i + 16, rl);
+    t_wait_ld();
+    if (scale) {
+#pragma unroll
+      for (int h = 0; h < 16; ++h) o[h] *= alpha_sm[h];
+    }
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+      float sc = 1.f, zp = 0.f;
+      if (pt.kind == 0) {
+        sc = __half2float(sch[i][hf]);
+        zp = fmaf(mid, sc, __half2float(zph[i][hf]));
+      }
+#pragma unroll
+      for (int h = 0; h < 16; ++h) o[h] = fmaf(sc, r[h] + rl[h], fmaf(zp, hs[hf * 16 + h], o[h]));
+      if (hf == 0) {                                    // the second half's accumulators
+        t_ld16_async(tlane + kTmemR + 128 + 32 * i, r);
+        t_ld16_async(tlane + kTmemR + 128 + 32 * i + 16, rl);
+        t_wait_ld();
+      }
+    }
+    t_st16(tlane + kTmemO + 16 * i, o);
+  }
+  t_fence_before();
+  return ok;
+}
+
 __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __grid_constant__ MlaDecodeParams p) {
   extern __shared__ uint8_t tsm_raw[];
   const WarpDesc cd = p.ctas[blockIdx.x];
@@ -338,13 +427,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
   uint8_t* gbase = tsm_raw + (base - t_u32(tsm_raw));
   const uint32_t misc = base + kOffMisc;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + kOffMisc + kMiscAbort);
-  volatile int* tiles_done = reinterpret_cast<volatile int*>(gbase + kOffMisc + kMiscDone);
   float* bias_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscBias);            // [2][64]
   float* max_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscMax);              // [2][4][16]
   float* sum_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscSum);              // [4][16]
   float* const_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscConst);          // [2][2][16]
   float* hsum_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscHalfSum);         // [2][4][16]
   float* cpart_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscConstPart);      // [2][2][9][16]
+  float* alpha_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscAlpha);          // [2][16]
+  float* hsum2_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscHalfSum2);       // [2][2][16]
+  volatile int* need_sm = reinterpret_cast<volatile int*>(gbase + kOffMisc + kMiscAlpha + 128);   // [2]
   const TableEntry* table = p.table + static_cast<size_t>(cd.stream) * p.table_stride;
   auto bar = [&](int which, int i) { return misc + 8u * static_cast<uint32_t>(which + i); };
 
@@ -354,11 +445,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       t_bar_init(bar(kBarSFull, i), 1);
       t_bar_init(bar(kBarQpFull, i), kTcConvertWarps);
       t_bar_init(bar(kBarPvDone, i), 1);
+      t_bar_init(bar(kBarHsFull, i), 4);
     }
     t_bar_init(bar(kBarPFull, 0), 4);
-    t_bar_init(bar(kBarRFree, 0), 4);
+    t_bar_init(bar(kBarRFree, 0), kTcReadTiles0 > 0 ? 8 : 4);
     *abort_flag = 0;
-    *tiles_done = 0;
     t_fence_async();
   }
   if (warp == 0) t_tmem_alloc(misc + kMiscTmem, kTmemCols);
@@ -368,24 +459,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
   const uint32_t tmem = __shfl_sync(kFullT, *reinterpret_cast<volatile uint32_t*>(gbase + kOffMisc + kMiscTmem), 0);
   const uint16_t* qg = p.q + static_cast<size_t>(cd.stream) * kMlaHeads * kMlaDk;
 
-  if (warp == kTcPrefetchWarp) {
-    // ---------------- L2 prefetch of the blocks ahead of the conversion ----------------
-    TcTile t;
-    int it = cd.item_begin, n = 0, spins = 0;
-    TableEntry pre = tc_entry(p, table, it);
-    while (tc_next(p, table, cd.item_end, it, pre, t)) {
-      pre = tc_entry(p, table, t.item + t.adv);
-      while (n > *tiles_done + kPrefetchAhead && !*abort_flag && ++spins < kTcWaitSpins) __nanosleep(200);
-      if (t.kind != 2 && lane == 0) {
-        const uint8_t* slot = p.arena + static_cast<size_t>(t.off256) * 256;
-        const uint32_t bytes = t.kind == 0 ? 2u * static_cast<uint32_t>(mla_half_bytes(t.level))
-                                           : static_cast<uint32_t>(t.nrows) * kMlaRowBytes;
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(slot), "r"(bytes) : "memory");
-      }
-      it = t.item + t.adv;
-      ++n;
-    }
-  } else if (warp == kTcMmaWarp) {
+  if (warp == kTcMmaWarp) {
     // ---------------- tensor-core issue (whole warp, one elected lane per instruction) ----------------
     constexpr uint32_t kIdQK = t_idesc(64, 64, false), kIdPV = t_idesc(128, 32, true, true);
     // descriptors differ only in the start-address field (16-byte units in the low word)
@@ -417,6 +491,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
                       kk != 2 * half);
       t_commit(bar(kBarPvDone, b));
     };
+    // packed bytes of a tile that is about to be converted: ask for them in L2
+    auto prefetch = [&](const TcTile& t) {
+      if (t.kind != 2 && lane == 0) {
+        const uint8_t* slot = p.arena + static_cast<size_t>(t.off256) * 256;
+        const uint32_t bytes = t.kind == 0 ? 2u * static_cast<uint32_t>(mla_half_bytes(t.level)) : static_cast<uint32_t>(t.nrows) * kMlaRowBytes;
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(slot), "r"(bytes) : "memory");
+      }
+    };
     // Event-driven order: the value MMAs of tile pv go out as soon as its P is there (and the
     // accumulators of tile pv - 1 have been read out), the key MMAs of tile qk as soon as its tile and
     // its Q' are there (qk runs at most two tiles ahead of pv: S and the tile buffers are double).
@@ -426,6 +508,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     bool more_tiles = tc_next(p, table, cd.item_end, it, pre, t);
     pre = tc_entry(p, table, t.item + t.adv);
     int qk = 0, pv = 0, n_known = more_tiles ? 1 : 0;      // tiles [0, n_known) exist so far
+    // a second walk over the tiles runs kPrefetchAhead tiles in front and asks for their bytes in L2
+    TcTile tp;
+    int itp = cd.item_begin;
+    TableEntry prep = tc_entry(p, table, itp);
+    bool more_pf = true;
+    auto prefetch_step = [&]() {
+      if (!more_pf) return;
+      more_pf = tc_next(p, table, cd.item_end, itp, prep, tp);
+      if (more_pf) {
+        prefetch(tp);
+        itp = tp.item + tp.adv;
+        prep = tc_entry(p, table, itp);
+      }
+    };
+#pragma unroll 1
+    for (int i = 0; i < kPrefetchAhead; ++i) prefetch_step();
     bool ok = true;
     int spins = 0;
     while (ok && (pv < n_known || more_tiles)) {
@@ -442,6 +540,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
             ++n_known;
             pre = tc_entry(p, table, t.item + t.adv);
           }
+          prefetch_step();
           progress = true;
         }
       }
@@ -454,10 +553,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
           progress = true;
         }
       }
-      if (progress) spins = 0;
-      else if (++spins > kTcWaitSpins || *abort_flag) {
-        *abort_flag = 1;
-        ok = false;
+      if (progress) {
+        spins = 0;
+      } else {
+        __nanosleep(128);
+        if (++spins > kTcWaitSpins || *abort_flag) {
+          *abort_flag = 1;
+          ok = false;
+        }
       }
       ok = __all_sync(kFullT, ok);
     }
@@ -465,7 +568,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     // ---------------- conversion of blocks into tiles, and Q' ----------------
     const int dt = tid - kTcFirstConvertWarp * 32;          // 0 .. 287
     const int dj = dt % kMlaChunks, dg = dt / kMlaChunks;   // tile conversion: chunk of 8 channels, token group
-    // Q': this thread scales the channels of chunk qj for the heads 4 qg .. 4 qg + 3
+    // Q': this thread scales the channels of chunk qj for the heads 4 qgd .. 4 qgd + 3
     const int cw = warp - kTcFirstConvertWarp;              // = panel of 64 channels
     const int qj = 8 * cw + (lane >> 2), qgd = lane & 3;
     uint32_t qh[4][4];                                      // fp16 pairs of the query: [head][channel pair]
@@ -486,19 +589,32 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       const int b = tg & 1;
       const uint32_t tile = base + kOffTile + b * kTcTileBytes;
       const uint8_t* slot = p.arena + static_cast<size_t>(t.off256) * 256;
+      // everything a quantised block needs from global memory is asked for before the wait for the
+      // tile buffer: the packed codes of the thread's part of the tile, the scales and zero points of
+      // its Q' chunk
+      uint2 w[2][8];
+      uint4 svh[2], zvh[2];
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        svh[half] = make_uint4(0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u);    // scales 1
+        zvh[half] = make_uint4(0, 0, 0, 0);
+      }
+      if (t.kind == 0) {
+        tc_load_block(slot, t.level, dj, dg, w);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const uint8_t* prm = slot + static_cast<size_t>(half) * mla_half_bytes(t.level);
+          svh[half] = t_ldg128(prm + 16 * qj);
+          zvh[half] = t_ldg128(prm + 2 * kMlaZeroOff + 16 * qj);
+        }
+      }
       // the tile buffer is free once the value MMAs of tile tg - 2 are done
       if (tg >= 2) ok = t_wait_warp(bar(kBarPvDone, b), ((tg - 2) >> 1) & 1, abort_flag);
       if (!ok) break;
       if (dt < 64) bias_sm[b * 64 + dt] = dt < t.nrows ? (t.kind == 2 ? 6.0f : 0.f) : kNegInfT;   // log2(64) per centroid row
       if (t.kind == 0) {
-        const size_t hb = static_cast<size_t>(mla_half_bytes(t.level));
-        if (t.level == 8) {
-          tc_convert_half<8>(slot, tile, 0, dj, dg);
-          tc_convert_half<8>(slot + hb, tile, 1, dj, dg);
-        } else {
-          tc_convert_half<4>(slot, tile, 0, dj, dg);
-          tc_convert_half<4>(slot + hb, tile, 1, dj, dg);
-        }
+        if (t.level == 8) tc_store_block<8>(w, tile, dj, dg);
+        else tc_store_block<4>(w, tile, dj, dg);
       } else if (t.kind == 1) {
         tc_convert_rows<false>(p, table, t, tile, dj, dg);
       } else {
@@ -507,22 +623,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       t_fence_async();
       __syncwarp();
       if (lane == 0) t_bar_arrive(bar(kBarKtFull, b));
-      if (dt == 0) *tiles_done = tg + 1;
-      // Q' of this tile: the buffer is free once the key MMAs of tile tg - 1 are done
-      if (tg >= 1) ok = t_wait_warp(bar(kBarSFull, (tg - 1) & 1), ((tg - 1) >> 1) & 1, abort_flag);
-      if (!ok) break;
-      const uint32_t qp = base + kOffQp;
+      // Q' of this tile.  The key constants sum_c q[c] (z[c] + mid s[c]) are formed before the wait:
+      // only the stores need the Q' buffer, which is free once the key MMAs of tile tg - 1 are done.
       const float mid = tc_mid(t.level);
-#pragma unroll 1
+#pragma unroll
       for (int half = 0; half < 2; ++half) {
         float cacc[4] = {0.f, 0.f, 0.f, 0.f};
-        uint4 sv = make_uint4(0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u);     // scales 1
         if (t.kind == 0) {
-          const uint8_t* prm = slot + static_cast<size_t>(half) * mla_half_bytes(t.level);
-          sv = t_ldg128(prm + 16 * qj);
-          const uint4 zv = t_ldg128(prm + 2 * kMlaZeroOff + 16 * qj);
-          // z' = z + mid s per channel (fp32), and its product with the query summed over the chunk
-          const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w}, zw[4] = {zv.x, zv.y, zv.z, zv.w};
+          const uint32_t sw[4] = {svh[half].x, svh[half].y, svh[half].z, svh[half].w};
+          const uint32_t zw[4] = {zvh[half].x, zvh[half].y, zvh[half].z, zvh[half].w};
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const float2 sf = __half22float2(t_h2(sw[i])), zf = __half22float2(t_h2(zw[i]));
@@ -534,8 +643,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
               cacc[hh] = fmaf(qf.y, z1, cacc[hh]);
             }
           }
+          // the warp's part: add the 8 chunks of the warp (lanes with the same head quad), fixed order
+#pragma unroll
+          for (int hh = 0; hh < 4; ++hh) {
+#pragma unroll
+            for (int d = 4; d <= 16; d <<= 1) cacc[hh] += __shfl_xor_sync(kFullT, cacc[hh], d);
+          }
         }
-        const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
+        if (lane < 4) {
+          float* dst = cpart_sm + ((b * 2 + half) * kTcConvertWarps + cw) * 16 + 4 * lane;
+          dst[0] = cacc[0]; dst[1] = cacc[1]; dst[2] = cacc[2]; dst[3] = cacc[3];
+        }
+      }
+      if (tg >= 1) ok = t_wait_warp(bar(kBarSFull, (tg - 1) & 1), ((tg - 1) >> 1) & 1, abort_flag);
+      if (!ok) break;
+      const uint32_t qp = base + kOffQp;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const uint32_t sw[4] = {svh[half].x, svh[half].y, svh[half].z, svh[half].w};
 #pragma unroll
         for (int hh = 0; hh < 4; ++hh) {
           uint32_t hi[4], lo[4];
@@ -549,16 +674,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
           t_sts128(tc_tile_addr(qp, row, qj), hi[0], hi[1], hi[2], hi[3]);
           t_sts128(tc_tile_addr(qp, row + 16, qj), lo[0], lo[1], lo[2], lo[3]);
         }
-        // the warp's part of sum_c q[c] z'[c]: add the 8 chunks of the warp (lanes with the same head quad)
-#pragma unroll
-        for (int hh = 0; hh < 4; ++hh) {
-#pragma unroll
-          for (int d = 4; d <= 16; d <<= 1) cacc[hh] += __shfl_xor_sync(kFullT, cacc[hh], d);
-        }
-        if (lane < 4) {
-          float* dst = cpart_sm + ((b * 2 + half) * kTcConvertWarps + cw) * 16 + 4 * lane;
-          dst[0] = cacc[0]; dst[1] = cacc[1]; dst[2] = cacc[2]; dst[3] = cacc[3];
-        }
       }
       t_fence_async();
       __syncwarp();
@@ -566,65 +681,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       it = t.item + t.adv;
       ++tg;
     }
+  } else if (warp >= 4) {
+    // ---------------- read-out of the channel tiles [kTcReadTiles0, 4) (warps 4-7) ----------------
+    const int lt = tid - 128;                               // tensor-memory lane
+    const uint32_t tlane = tmem + (static_cast<uint32_t>(32 * (warp - 4)) << 16);
+    TcTile t;
+    int it = cd.item_begin, ts = 0;
+    bool ok = true;
+    TableEntry pre = tc_entry(p, table, it);
+    while (ok && tc_next(p, table, cd.item_end, it, pre, t)) {
+      pre = tc_entry(p, table, t.item + t.adv);
+      // what the softmax of tile ts published: the sums of its probabilities and whether it moved the running max
+      ok = t_wait_warp(bar(kBarHsFull, ts & 1), (ts >> 1) & 1, abort_flag) && ok;
+      ok = tc_read_out(p, t, ts, kTcReadTiles0, 4, need_sm[ts & 1] != 0, alpha_sm + (ts & 1) * 16, hsum2_sm + (ts & 1) * 32, tlane, lt,
+                       bar(kBarPvDone, ts & 1), abort_flag) && ok;
+      __syncwarp();
+      if (lane == 0) t_bar_arrive(bar(kBarRFree, 0));
+      it = t.item + t.adv;
+      ++ts;
+    }
   } else {
-    // ---------------- softmax, read-out (warps 0-3) and the result ----------------
-    float m_run[16], l_part[16], alpha[16];
+    // ---------------- softmax, read-out of the first channel tiles (warps 0-3) and the result ----------------
+    float m_run[16], l_part[16];
 #pragma unroll
     for (int h = 0; h < 16; ++h) {
       m_run[h] = kNegInfT;
       l_part[h] = 0.f;
-      alpha[h] = 1.f;
     }
     const uint32_t tlane = tmem + (static_cast<uint32_t>(32 * warp) << 16);
     const int half = warp >> 1;                             // the half block of this warp's 16 token rows
     bool ok = true;
-    // Read-out of tile `pt` (number pn): O^T <- (O^T + s[c] R[c] + z'[c] sum_t p) * alpha per half, then
-    // per head, for the 128 channels of each of the four channel tiles that this thread's lane holds.
-    auto read_out = [&](const TcTile& pt, int pn, bool scale) {
-      ok = t_wait_warp(bar(kBarPvDone, pn & 1), (pn >> 1) & 1, abort_flag) && ok;
-      t_fence_after();
-      const float* hs = hsum_sm + (pn & 1) * 64;            // [4 warps][16]
-      const float mid = tc_mid(pt.level);
-      const uint8_t* slot = p.arena + static_cast<size_t>(pt.off256) * 256;
-#pragma unroll 1
-      for (int i = 0; i < 4; ++i) {
-        const int c = 128 * i + tid;
-        float o[16];
-        if (pn > 0) {
-          t_ld16(tlane + kTmemO + 16 * i, o);
-        } else {
-#pragma unroll
-          for (int h = 0; h < 16; ++h) o[h] = 0.f;
-        }
-#pragma unroll 1
-        for (int hf = 0; hf < 2; ++hf) {
-          float sc = 1.f, zp = 0.f;
-          if (pt.kind == 0) {
-            const __half* prm = reinterpret_cast<const __half*>(slot + static_cast<size_t>(hf) * mla_half_bytes(pt.level));
-            sc = __half2float(__ldg(prm + c));
-            zp = fmaf(mid, sc, __half2float(__ldg(prm + kMlaZeroOff + c)));
-          }
-          float r[16], rl[16];
-          t_ld16(tlane + kTmemR + 128 * hf + 32 * i, r);
-          t_ld16(tlane + kTmemR + 128 * hf + 32 * i + 16, rl);
-#pragma unroll
-          for (int h = 0; h < 16; ++h) {
-            const float ps = hs[(2 * hf) * 16 + h] + hs[(2 * hf + 1) * 16 + h];       // sum of the half's probabilities
-            o[h] = fmaf(sc, r[h] + rl[h], fmaf(zp, ps, o[h]));
-          }
-        }
-        if (scale) {
-#pragma unroll
-          for (int h = 0; h < 16; ++h) o[h] *= alpha[h];
-        }
-        t_st16(tlane + kTmemO + 16 * i, o);
-      }
-      t_fence_before();
-      __syncwarp();
-      if (lane == 0) t_bar_arrive(bar(kBarRFree, 0));
-    };
-    TcTile t, prev;
-    prev.kind = 1; prev.level = 16; prev.off256 = 0; prev.item = 0; prev.adv = 0; prev.nrows = 0; prev.nstages = 0;
+    TcTile t;
     int it = cd.item_begin, ts = 0, xph = 0;                // xph: exchanges done so far (phase of the exchange buffers)
     TableEntry pre = tc_entry(p, table, it);
     while (tc_next(p, table, cd.item_end, it, pre, t)) {
@@ -642,8 +729,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       ok = t_wait_warp(bar(kBarSFull, b), (ts >> 1) & 1, abort_flag) && ok;
       t_fence_after();
       float s[16], sl[16];
-      t_ld16(tlane + kTmemS + 64 * b + 32 * half, s);
-      t_ld16(tlane + kTmemS + 64 * b + 32 * half + 16, sl);
+      t_ld16_async(tlane + kTmemS + 64 * b + 32 * half, s);
+      t_ld16_async(tlane + kTmemS + 64 * b + 32 * half + 16, sl);
+      t_wait_ld();
       asm volatile("bar.sync 1, 128;\n" ::: "memory");                    // const_sm is complete
       const int row = 16 * warp + (lane & 15);
       const float bs = (lane < 16) ? bias_sm[b * 64 + row] : kNegInfT;
@@ -686,12 +774,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
         for (int h = 0; h < 16; ++h) {
           const float bm = fmaxf(fmaxf(mbuf[h], mbuf[16 + h]), fmaxf(mbuf[32 + h], mbuf[48 + h]));
           const float mn = fmaxf(m_run[h], bm);
-          alpha[h] = (m_run[h] == kNegInfT) ? 0.f : t_ex2(m_run[h] - mn);
+          const float al = (m_run[h] == kNegInfT) ? 0.f : t_ex2(m_run[h] - mn);
           m_run[h] = mn;
-          l_part[h] *= alpha[h];
+          l_part[h] *= al;
+          if (tid == 0) alpha_sm[b * 16 + h] = al;          // what O^T (tiles before this one) is rescaled by
         }
         ++xph;
       }
+      if (tid == 0) need_sm[b] = need ? 1 : 0;
       // probabilities relative to the (possibly stale) running max as fp16 pairs hi + lo; the
       // unrounded value is what is summed
       float pr[16];
@@ -719,28 +809,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
         t_sts128(prow + 2048 + (sw ^ 16), pl[4], pl[5], pl[6], pl[7]);
       }
       // sums of the warp's 16 rows per head (for the zero-point term of the read-out), fixed order
+      // (reduce-scatter: after the step with distance d a lane keeps the heads whose bit d equals
+      // its own, so lane j < 16 ends with the sum of head j; lanes 16-31 hold zeros)
 #pragma unroll
-      for (int d = 8; d >= 1; d >>= 1)
+      for (int d = 8; d >= 1; d >>= 1) {
+        const bool up = (lane & d) != 0;
 #pragma unroll
-        for (int h = 0; h < 16; ++h) pr[h] += __shfl_xor_sync(kFullT, pr[h], d);
-      if (lane == 0) {
-#pragma unroll
-        for (int h = 0; h < 16; ++h) hsum_sm[b * 64 + warp * 16 + h] = pr[h];
+        for (int h = 0; h < d; ++h) {
+          const float give = up ? pr[h] : pr[h + d], keep = up ? pr[h + d] : pr[h];
+          pr[h] = keep + __shfl_xor_sync(kFullT, give, d);
+        }
       }
+      if (lane < 16) hsum_sm[b * 64 + warp * 16 + lane] = pr[0];
       t_fence_async();
       t_fence_before();
       __syncwarp();
       if (lane == 0) t_bar_arrive(bar(kBarPFull, 0));
-      // read-out of the tile before (its accumulators are complete: the wait above), rescaled when this
-      // tile moved the running max
-      if (ts > 0) read_out(prev, ts - 1, need);
-      prev = t;
+      // the sums of the tile per half block: the two warps of a half added in a fixed order
+      asm volatile("bar.sync 1, 128;\n" ::: "memory");
+      if (tid < 32) hsum2_sm[b * 32 + tid] = hsum_sm[b * 64 + (tid >> 4) * 32 + (tid & 15)] + hsum_sm[b * 64 + (tid >> 4) * 32 + 16 + (tid & 15)];
+      __syncwarp();
+      if (lane == 0) t_bar_arrive(bar(kBarHsFull, b));
+      if (kTcReadTiles0 > 0) {
+        asm volatile("bar.sync 1, 128;\n" ::: "memory");                  // the sums are complete
+        ok = tc_read_out(p, t, ts, 0, kTcReadTiles0, need, alpha_sm + b * 16, hsum2_sm + b * 32, tlane, tid, bar(kBarPvDone, b), abort_flag) && ok;
+        __syncwarp();
+        if (lane == 0) t_bar_arrive(bar(kBarRFree, 0));
+      }
       it = t.item + t.adv;
       ++ts;
     }
     // ---------------- result ----------------
-    asm volatile("bar.sync 1, 128;\n" ::: "memory");                      // hsum_sm of the last tile
-    if (ts > 0) read_out(prev, ts - 1, false);
     float* out = p.partial + static_cast<size_t>(cd.partial) * kMlaPartialFloats;
 #pragma unroll
     for (int d = 8; d >= 1; d >>= 1)
@@ -759,6 +858,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
         out[h * (kMlaDv + 2) + 1] = good ? sum_sm[h] + sum_sm[16 + h] + sum_sm[32 + h] + sum_sm[48 + h] : 0.f;
       }
     }
+  }
+  // the running O^T is complete once every read-out warp is here
+  t_fence_before();
+  __syncthreads();
+  t_fence_after();
+  if (warp < 4) {
+    const uint32_t tlane = tmem + (static_cast<uint32_t>(32 * warp) << 16);
+    float* out = p.partial + static_cast<size_t>(cd.partial) * kMlaPartialFloats;
+    const bool good = !*abort_flag;
 #pragma unroll 1
     for (int i = 0; i < 4; ++i) {
       float o[16];
