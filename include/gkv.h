@@ -63,7 +63,7 @@ typedef struct gkv_config {
   uint32_t struct_size;  /* sizeof(gkv_config) */
   uint32_t abi_version;  /* GKV_ABI_VERSION */
   int32_t n_layers, batch, n_q_heads, n_kv_heads; /* n_q_heads % n_kv_heads == 0 */
-  int32_t d_k, d_v;      /* head dims; this build: 128 / 128 */
+  int32_t d_k, d_v;      /* head dims: 128 / 128, or 576 / 512 with v_aliases_k */
   int32_t v_aliases_k;   /* 1: values are channels [0, d_v) of the key row (latent attention) */
   int32_t max_ctx;       /* capacity in tokens per sequence */
   int32_t block_tokens;  /* 64 (Sec. 3.2) */
@@ -126,12 +126,17 @@ GKV_API int gkv_append_demote(gkv_cache* c, int32_t layer, const void* k_new, co
                       const float* token_mass, const int8_t* level_plan, void* stream);
 
 /* Single-query attention of every query head over the graded cache of `layer`
- * (Sec. 3.7; Eq. 1 over the reconstructed keys/values; split-context partials reduced
- * separately).
+ * (Sec. 3.7; Eq. 1 over the reconstructed keys/values; split-context partials are merged inside
+ * the same launch, in a fixed order).
  *   q        device bf16 [batch][n_q_heads][d_k]
  *   page_idx device int32 [batch][n_kv_heads][n_sel] ascending closed-page indices, or NULL with
  *            n_sel = 0 for a full read.  With a list, only those pages and the partial tail block
- *            are read; every other token is hard-masked (Sec. 3.5)
+ *            are read; every other token is hard-masked (Sec. 3.5), exact residual tokens of
+ *            pages that are not listed included.  An entry outside [0, closed pages) is skipped
+ *            by the kernel (nothing is read through it) and the next gkv_bits_report returns
+ *            GKV_ERR_BAD_STATE.  The library keeps the pointer, not a copy: the list must stay
+ *            allocated and unchanged until the next gkv_bits_report of this layer if that report
+ *            is to count the bits the read touched (a later read of the layer replaces it)
  *   out      device fp32 [batch][n_q_heads][d_v]
  *   lse      device fp32 [batch][n_q_heads] natural-log sum of exp(logit), or NULL */
 GKV_API int gkv_decode_attn(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_idx, int32_t n_sel,
@@ -193,6 +198,20 @@ GKV_API int gkv_debug_export_mass(gkv_cache* c, int32_t layer, float* mass_out);
  *   n_sel_out    host int32, receives k */
 GKV_API int gkv_quest_select(gkv_cache* c, int32_t layer, const void* q, int32_t budget_tokens,
                      int32_t* page_idx_out, int32_t* n_sel_out, void* stream);
+
+/* Parity helpers of the page scorer (Sec. 3.5; both synchronise the device).
+ * gkv_debug_export_boxes: the exact per-page per-channel key minima and maxima of one stream, as
+ * recorded from the unquantised keys when each block closed.
+ *   lo / hi   HOST bf16 bits [n_pages][d_k] each, n_pages = closed blocks * (64 / page_tokens);
+ *             cap_pages is the room of the two arrays in pages, *n_pages receives the count
+ * gkv_debug_export_scores: the page scores that gkv_quest_select ranks, for every stream of `layer`
+ * and the query q (device bf16 [batch][n_q_heads][d_k]): per query head sum_d q_d * (q_d >= 0 ? max_d :
+ * min_d) added in ascending d in fp32, reduced over the KV head's query heads (cfg.quest_reduce).
+ *   scores    HOST fp32 [batch][n_kv_heads][n_pages]
+ * Both return GKV_ERR_BAD_STATE without a page scorer (page_tokens == 0). */
+GKV_API int gkv_debug_export_boxes(gkv_cache* c, int32_t layer, int32_t b, int32_t kv_head, uint16_t* lo, uint16_t* hi,
+                                   int32_t cap_pages, int32_t* n_pages);
+GKV_API int gkv_debug_export_scores(gkv_cache* c, int32_t layer, const void* q, float* scores, void* stream);
 
 /* The same page selection as gkv_quest_select for callers that cannot have any device memory
  * allocated on their behalf while they run: a plug-in that was handed a fixed arena by a serving

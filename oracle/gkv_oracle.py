@@ -455,7 +455,8 @@ class GradedCache:
                 for h in range(cfg.n_kv_heads):
                     self.streams[(l, b, h)] = Stream(cfg.d_k, cfg.d_v, self.alias)
         self.last_read_bits: Dict[int, int] = {}
-        self.last_box_bits: Dict[int, int] = {}
+        self.last_box_bits: Dict[int, int] = {}        # boxes scored by a quest_select that no read has used yet
+        self.last_read_box_bits: Dict[int, int] = {}   # boxes that count for the last read
 
     @property
     def scale(self) -> float:
@@ -664,6 +665,11 @@ class GradedCache:
                     if return_weights:
                         weights[(b, hq)] = w
         self.last_read_bits[layer] = read_bits
+        # Sec. 3.5: the read cost of a scored query is "all summaries + selected pages".  The boxes
+        # count for the page-list read that follows a quest_select; a later read with a list that
+        # was not scored (or a full read) did not look at them.
+        self.last_read_box_bits[layer] = self.last_box_bits.pop(layer, 0) if page_idx is not None else 0
+        self.last_box_bits.pop(layer, None)
         if return_weights:
             return out, lse, weights
         return out, lse
@@ -782,7 +788,8 @@ class GradedCache:
     def _read_bits(self, st: Stream, page_idx) -> int:
         """Bits of graded K/V a query touches: whole blocks for a full read; for a page list,
         per selected page its share of codes, its V params, and each touched 32-token K group's
-        params once.  Centroid and exact blocks: centroid rows once / exact rows per token."""
+        params once.  Centroid and exact blocks: centroid rows once / exact rows per token.
+        Residual rows: all of them in a full read, those of listed pages with a page list."""
         alias = self.alias
         dk, dv = st.d_k, st.d_v
         nval_tok = dk if alias else dk + dv
@@ -812,6 +819,9 @@ class GradedCache:
                     touched_groups.add(t0 // G)
         bits += len(touched_groups) * dk * 32                              # K params per touched group
         bits += len(touched_cent) * 16 * nval_tok
+        # exact residual rows of listed pages are read too (those of other pages are masked, Sec. 3.5)
+        listed = set(int(p) for p in page_idx)
+        bits += sum(1 for t in st.res_idx if int(t) // page in listed) * 16 * nval_tok
         # the current partial block is always read, exact
         bits += st.n_tail * 16 * nval_tok
         return bits
@@ -847,7 +857,7 @@ class GradedCache:
                                 + rep["box_bits"])
         rep["bpv_resident"] = rep["resident_bits"] / max(1, rep["values"])
         rep["bpv_paper"] = (rep["resident_bits"] - rep["residual_index_bits"]) / max(1, rep["values"])
-        rep["last_read_bits"] = self.last_read_bits.get(layer, 0) + self.last_box_bits.get(layer, 0)
+        rep["last_read_bits"] = self.last_read_bits.get(layer, 0) + self.last_read_box_bits.get(layer, 0)
         rep["bpv_read"] = rep["last_read_bits"] / max(1, rep["values"])
         return rep
 

@@ -27,7 +27,8 @@ EXPORTS = [
     "gkv_query_arena_bytes", "gkv_create", "gkv_destroy", "gkv_append_demote", "gkv_decode_attn",
     "gkv_decode_attn_observe", "gkv_debug_export_mass", "gkv_debug_export_bounds", "gkv_rd_reallocate",
     "gkv_debug_replan_levels",
-    "gkv_quest_select", "gkv_quest_select_static", "gkv_bits_report", "gkv_debug_export_block", "gkv_debug_export_residual",
+    "gkv_quest_select", "gkv_quest_select_static", "gkv_debug_export_boxes", "gkv_debug_export_scores", "gkv_bits_report",
+    "gkv_debug_export_block", "gkv_debug_export_residual",
     "gkv_debug_export_levels", "gkv_debug_plan_levels", "gkv_ctx_len", "gkv_strerror", "gkv_last_cuda_error",
 ]
 
@@ -89,6 +90,8 @@ def load():
     lib.gkv_debug_replan_levels.argtypes = [C.POINTER(GkvConfig), i32, i32, C.POINTER(C.c_float), C.POINTER(C.c_float),
                                             C.POINTER(C.c_int8), C.POINTER(C.c_int8), C.POINTER(i32)]
     lib.gkv_quest_select.argtypes = [vp, i32, vp, i32, vp, C.POINTER(i32), vp]
+    lib.gkv_debug_export_boxes.argtypes = [vp, i32, i32, i32, vp, vp, i32, C.POINTER(i32)]
+    lib.gkv_debug_export_scores.argtypes = [vp, i32, vp, vp, vp]
     lib.gkv_quest_select_static.argtypes = [vp, i32, vp, i32, vp, C.POINTER(i32), vp]
     lib.gkv_bits_report.argtypes = [vp, i32, C.POINTER(GkvBits)]
     lib.gkv_debug_export_block.argtypes = [vp, i32, i32, i32, i32, i32, C.POINTER(i32), vp, vp, vp, vp, C.POINTER(i32)]
@@ -133,7 +136,8 @@ def config_from_workload(w, n_layers: Optional[int] = None) -> GkvConfig:
                        v_aliases_k=w.v_aliases_k, page_tokens=w.page_tokens, policy=w.policy,
                        stair_tokens=tuple(w.stair_tokens), n_sink_blocks=w.n_sink_blocks,
                        retire_after=w.retire_after, rd_budget_bpv=w.rd_budget_bpv,
-                       residual_fraction=w.residual_fraction, softmax_scale=w.softmax_scale)
+                       residual_fraction=w.residual_fraction, quest_reduce=getattr(w, "quest_reduce", REDUCE_MAX),
+                       softmax_scale=w.softmax_scale)
 
 
 def _ptr(t) -> Optional[int]:
@@ -263,6 +267,26 @@ class Cache:
         n_items = (self.gkv_ctx_len(layer) + 63) // 64
         out = np.zeros((self.cfg.batch, self.cfg.n_kv_heads, n_items), dtype=np.float32)
         _check(load().gkv_debug_export_mass(self.handle, layer, out.ctypes.data_as(C.c_void_p)), "gkv_debug_export_mass")
+        return out
+
+    def gkv_debug_export_boxes(self, layer, b, kv_head):
+        """Page boxes of one stream: (lo, hi) uint16 arrays [n_pages][d_k] of bf16 bits."""
+        page = self.cfg.page_tokens
+        cap = (self.gkv_ctx_len(layer) // 64) * (64 // page) if page > 0 else 0
+        lo = np.zeros((max(cap, 1), self.cfg.d_k), dtype=np.uint16)
+        hi = np.zeros((max(cap, 1), self.cfg.d_k), dtype=np.uint16)
+        n = C.c_int32(0)
+        _check(load().gkv_debug_export_boxes(self.handle, layer, b, kv_head, lo.ctypes.data_as(C.c_void_p),
+                                             hi.ctypes.data_as(C.c_void_p), cap, C.byref(n)), "gkv_debug_export_boxes")
+        return lo[: n.value], hi[: n.value]
+
+    def gkv_debug_export_scores(self, layer, q):
+        """Page scores of every stream for query q: float32 [batch][n_kv_heads][n_pages]."""
+        page = self.cfg.page_tokens
+        n_pages = (self.gkv_ctx_len(layer) // 64) * (64 // page) if page > 0 else 0
+        out = np.zeros((self.cfg.batch, self.cfg.n_kv_heads, n_pages), dtype=np.float32)
+        _check(load().gkv_debug_export_scores(self.handle, layer, _ptr(q), out.ctypes.data_as(C.c_void_p), self._st()),
+               "gkv_debug_export_scores")
         return out
 
     def gkv_quest_select(self, layer, q, budget_tokens, page_idx_out) -> int:

@@ -111,7 +111,8 @@ struct LayerState {
   int last_mode = 0;                    // 0 none, 1 full, 2 page list
   const int32_t* last_pages = nullptr;
   int last_n_sel = 0;
-  bool quest_ran = false;
+  bool quest_ran = false;               // gkv_quest_select ran and no read has consumed its result yet
+  bool last_read_scored = false;        // the last page-list read followed a gkv_quest_select (its boxes count as read)
   bool budget_flag = false;
 };
 
@@ -888,16 +889,28 @@ int demote_to_targets(gkv_cache* c, LayerState& L, const int8_t* target, size_t 
   }
   if ((rc = wait_event(c, ev_jobs)) != GKV_OK) return rc;
   if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
+  // Phase 1: a destination slot for every job.  If the arena cannot hold them all, everything taken
+  // so far goes back and nothing else has changed: the host mirrors, the device table and the
+  // levels still describe the cache as it was, and the call can be repeated with a larger arena.
+  std::vector<uint32_t> dst(want_list.size());
+  for (size_t i = 0; i < want_list.size(); ++i) {
+    const int8_t want = target[static_cast<size_t>(want_list[i].first) * stride + want_list[i].second];
+    if (!c->heap.alloc(want, &dst[i])) {
+      for (size_t k = 0; k < i; ++k)
+        c->heap.release(target[static_cast<size_t>(want_list[k].first) * stride + want_list[k].second], dst[k]);
+      return GKV_ERR_ARENA_TOO_SMALL;
+    }
+  }
+  // Phase 2: the job list and the mirrors.
   size_t n_jobs = 0;
   std::vector<std::pair<int, uint32_t>> to_free;
   to_free.reserve(want_list.size());
-  for (const auto& sb : want_list) {
-    const int s = sb.first, b = sb.second;
+  for (size_t i = 0; i < want_list.size(); ++i) {
+    const int s = want_list[i].first, b = want_list[i].second;
     const int8_t want = target[static_cast<size_t>(s) * stride + b];
     int8_t& cur = L.level[static_cast<size_t>(s) * c->max_blocks + b];
     TableEntry& e = L.table_h[static_cast<size_t>(s) * c->table_stride + b];
-    uint32_t off;
-    if (!c->heap.alloc(want, &off)) return GKV_ERR_ARENA_TOO_SMALL;
+    const uint32_t off = dst[i];
     EncodeJob& job = jobs[n_jobs++];
     job.src_off256 = e.off256;
     job.dst_off256 = off;
@@ -934,14 +947,20 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
   LayerState& L = c->layers[layer];
   const int ns = c->n_streams;
   int rc;
-  const size_t table_bytes = static_cast<size_t>(ns) * c->table_stride * sizeof(TableEntry);
   if (!L.has_tail_slot) {
     // a new tail block starts: give every stream an exact slot for it
     if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
+    // all or nothing: when the arena cannot hold a slot for every stream, the slots taken so far go
+    // back and the layer is as it was
+    std::vector<uint32_t> slots(ns);
     for (int s = 0; s < ns; ++s) {
-      uint32_t off;
-      if (!c->heap.alloc(16, &off)) return GKV_ERR_ARENA_TOO_SMALL;
-      set_entry(c, L, s, L.n_closed, off, 16);
+      if (!c->heap.alloc(16, &slots[s])) {
+        for (int k = 0; k < s; ++k) c->heap.release(16, slots[k]);
+        return GKV_ERR_ARENA_TOO_SMALL;
+      }
+    }
+    for (int s = 0; s < ns; ++s) {
+      set_entry(c, L, s, L.n_closed, slots[s], 16);
       L.table_h[static_cast<size_t>(s) * c->table_stride + L.n_closed].resmask = 0;
     }
     L.has_tail_slot = true;
@@ -1123,10 +1142,15 @@ int mla_append_one(gkv_cache* c, int layer, const uint16_t* k_new, cudaStream_t 
   const size_t table_bytes = static_cast<size_t>(ns) * c->table_stride * sizeof(TableEntry);
   if (!L.has_tail_slot) {
     if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
+    std::vector<uint32_t> slots(ns);                     // all or nothing, as in append_one
     for (int s = 0; s < ns; ++s) {
-      uint32_t off;
-      if (!c->heap.alloc(16, &off)) return GKV_ERR_ARENA_TOO_SMALL;
-      set_entry(c, L, s, L.n_closed, off, 16);
+      if (!c->heap.alloc(16, &slots[s])) {
+        for (int k = 0; k < s; ++k) c->heap.release(16, slots[k]);
+        return GKV_ERR_ARENA_TOO_SMALL;
+      }
+    }
+    for (int s = 0; s < ns; ++s) {
+      set_entry(c, L, s, L.n_closed, slots[s], 16);
       L.table_h[static_cast<size_t>(s) * c->table_stride + L.n_closed].resmask = 0;
     }
     L.has_tail_slot = true;
@@ -1149,27 +1173,38 @@ int mla_append_one(gkv_cache* c, int layer, const uint16_t* k_new, cudaStream_t 
   if ((rc = wait_event(c, L.ev)) != GKV_OK) return rc;
   EncodeJob* jobs = reinterpret_cast<EncodeJob*>(c->stage_h);
   size_t n_jobs = 0;
-  std::vector<std::pair<int, uint32_t>> to_free;
+  // phase 1: a destination slot for every block that falls; on failure they all go back and the
+  // mirrors, the levels and the device table are untouched
+  std::vector<std::pair<int, int>> want_list;
   for (int s = 0; s < ns; ++s)
-    for (int b = 0; b < L.n_closed; ++b) {
-      int8_t& cur = L.level[static_cast<size_t>(s) * c->max_blocks + b];
-      if (target[b] >= cur) continue;
-      TableEntry& e = L.table_h[static_cast<size_t>(s) * c->table_stride + b];
-      uint32_t off;
-      if (!c->heap.alloc(target[b], &off)) return GKV_ERR_ARENA_TOO_SMALL;
-      EncodeJob& job = jobs[n_jobs++];
-      job.src_off256 = e.off256;
-      job.dst_off256 = off;
-      job.src_level = cur;
-      job.dst_level = target[b];
-      job.stream = s;
-      job.block = b;
-      job.pad = 0;
-      to_free.emplace_back(cur, e.off256);
-      e.off256 = off;
-      e.level = static_cast<uint32_t>(target[b]);
-      cur = target[b];
+    for (int b = 0; b < L.n_closed; ++b)
+      if (target[b] < L.level[static_cast<size_t>(s) * c->max_blocks + b]) want_list.emplace_back(s, b);
+  std::vector<uint32_t> dst(want_list.size());
+  for (size_t i = 0; i < want_list.size(); ++i) {
+    if (!c->heap.alloc(target[want_list[i].second], &dst[i])) {
+      for (size_t k = 0; k < i; ++k) c->heap.release(target[want_list[k].second], dst[k]);
+      return GKV_ERR_ARENA_TOO_SMALL;
     }
+  }
+  // phase 2: jobs and mirrors
+  std::vector<std::pair<int, uint32_t>> to_free;
+  for (size_t i = 0; i < want_list.size(); ++i) {
+    const int s = want_list[i].first, b = want_list[i].second;
+    int8_t& cur = L.level[static_cast<size_t>(s) * c->max_blocks + b];
+    TableEntry& e = L.table_h[static_cast<size_t>(s) * c->table_stride + b];
+    EncodeJob& job = jobs[n_jobs++];
+    job.src_off256 = e.off256;
+    job.dst_off256 = dst[i];
+    job.src_level = cur;
+    job.dst_level = target[b];
+    job.stream = s;
+    job.block = b;
+    job.pad = 0;
+    to_free.emplace_back(cur, e.off256);
+    e.off256 = dst[i];
+    e.level = static_cast<uint32_t>(target[b]);
+    cur = target[b];
+  }
   if (n_jobs > 0) {
     CK(c, cudaMemcpyAsync(c->jobs_d, jobs, n_jobs * sizeof(EncodeJob), cudaMemcpyHostToDevice, st));
     CK(c, cudaEventRecord(c->ev_stage, st));
@@ -1534,9 +1569,9 @@ int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_
   if (page_idx) {
     if (cfg.page_tokens <= 0) return GKV_ERR_BAD_STATE;
     if (n_sel < 0 || n_sel > L.n_closed * (kBlock / cfg.page_tokens)) return GKV_ERR_INVALID_ARG;
-    for (int s = 0; s < c->n_streams; ++s)
-      if (L.res_count_h[s] > 0) return GKV_ERR_UNSUPPORTED;
     p.page_idx = page_idx;
+    p.res_idx = L.res_idx_d;
+    p.res_cap = c->res_cap;
     p.n_sel = n_sel;
     p.page_tokens = cfg.page_tokens;
     p.warps_per_stream = sparse_ctas_per_stream(c->n_hgroups) * kDecodeWarps;      // per head group
@@ -1547,6 +1582,8 @@ int decode_impl(gkv_cache* c, int32_t layer, const void* q, const int32_t* page_
     L.last_mode = 2;
     L.last_pages = page_idx;
     L.last_n_sel = n_sel;
+    L.last_read_scored = L.quest_ran;     // a later read with a list of the caller's own does not inherit it
+    L.quest_ran = false;
   } else {
     if (L.desc_dirty || (observe && L.desc_split)) {      // an observing call needs whole-block units
       // the work lists have their own event: waiting for the table's would wait for copies that
@@ -1664,6 +1701,47 @@ int gkv_quest_select(gkv_cache* c, int32_t layer, const void* q, int32_t budget_
   return GKV_OK;
 }
 
+int gkv_debug_export_boxes(gkv_cache* c, int32_t layer, int32_t b, int32_t kv_head, uint16_t* lo, uint16_t* hi,
+                           int32_t cap_pages, int32_t* n_pages) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !lo || !hi || !n_pages) return GKV_ERR_INVALID_ARG;
+  const gkv_config& cfg = c->cfg;
+  if (b < 0 || b >= cfg.batch || kv_head < 0 || kv_head >= cfg.n_kv_heads) return GKV_ERR_INVALID_ARG;
+  if (cfg.page_tokens <= 0) return GKV_ERR_BAD_STATE;
+  LayerState& L = c->layers[layer];
+  const int np = L.n_closed * (kBlock / cfg.page_tokens);
+  *n_pages = np;
+  if (np > cap_pages) return GKV_ERR_INVALID_ARG;
+  if (np == 0) return GKV_OK;
+  CK(c, cudaDeviceSynchronize());
+  // device layout [stream][channel][min | max][page] -> [page][channel]
+  std::vector<uint16_t> raw(static_cast<size_t>(kD) * 2 * c->box_stride);
+  const int stream = b * cfg.n_kv_heads + kv_head;
+  CK(c, cudaMemcpy(raw.data(), L.boxes_d + static_cast<size_t>(stream) * kD * 2 * c->box_stride, raw.size() * sizeof(uint16_t),
+                   cudaMemcpyDeviceToHost));
+  for (int pg = 0; pg < np; ++pg)
+    for (int ch = 0; ch < kD; ++ch) {
+      lo[static_cast<size_t>(pg) * kD + ch] = raw[(static_cast<size_t>(ch) * 2) * c->box_stride + pg];
+      hi[static_cast<size_t>(pg) * kD + ch] = raw[(static_cast<size_t>(ch) * 2 + 1) * c->box_stride + pg];
+    }
+  return GKV_OK;
+}
+
+int gkv_debug_export_scores(gkv_cache* c, int32_t layer, const void* q, float* scores, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !scores || misaligned(q, 16)) return GKV_ERR_INVALID_ARG;
+  const gkv_config& cfg = c->cfg;
+  if (cfg.page_tokens <= 0) return GKV_ERR_BAD_STATE;
+  LayerState& L = c->layers[layer];
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int np = L.n_closed * (kBlock / cfg.page_tokens);
+  if (np == 0) return GKV_OK;
+  CK(c, launch_quest_scores(L.boxes_d, c->box_stride, np, static_cast<const uint16_t*>(q), c->n_streams, cfg.n_kv_heads, c->group,
+                            cfg.quest_reduce, c->scores_d, c->box_stride, st));
+  CK(c, cudaStreamSynchronize(st));
+  CK(c, cudaMemcpy2D(scores, static_cast<size_t>(np) * sizeof(float), c->scores_d, static_cast<size_t>(c->box_stride) * sizeof(float),
+                     static_cast<size_t>(np) * sizeof(float), c->n_streams, cudaMemcpyDeviceToHost));
+  return GKV_OK;
+}
+
 int gkv_quest_select_static(gkv_cache* c, int32_t layer, const void* q, int32_t budget_tokens,
                             int32_t* page_idx_out, int32_t* n_sel_out, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !page_idx_out || !n_sel_out || budget_tokens < 0)
@@ -1747,10 +1825,16 @@ int gkv_bits_report(gkv_cache* c, int32_t layer, gkv_bits* out) {
         }
         for (char g : group_seen) if (g) out->last_read_bits += static_cast<uint64_t>(cfg.d_k) * 32;
         for (char g : cent_seen) if (g) out->last_read_bits += 16ull * nval_tok;
+        // exact residual rows are read where the page of their token is listed
+        if (!L.res_idx.empty() && !L.res_idx[s].empty()) {
+          const int32_t* lb = pages.data() + static_cast<size_t>(s) * L.last_n_sel;
+          for (int32_t tok : L.res_idx[s])
+            if (std::binary_search(lb, lb + L.last_n_sel, tok / page)) out->last_read_bits += 16ull * nval_tok;
+        }
         out->last_read_bits += static_cast<uint64_t>(L.n_tail) * 16 * nval_tok;
       }
     }
-    if (L.quest_ran && L.last_mode == 2)
+    if (L.last_read_scored && L.last_mode == 2)
       out->last_read_bits += static_cast<uint64_t>(c->n_streams) * L.n_closed * (kBlock / cfg.page_tokens) * 2 * cfg.d_k * 16;
     if (L.budget_flag) warn = GKV_ERR_BUDGET;
   }

@@ -275,6 +275,7 @@ struct WarpCtx {
   int lane;
   int item_end;              // dense: one past the last item; sparse: one past the last page position
   int stream;                // the (sequence, KV head) stream whose cache is read
+  int sparse_rank;           // page-list reads: this warp's number among the warps of its head group
   int head0;                 // first query head (within the KV head's group) of the warp's head group
   bool has_tail;
   uint32_t stage0;           // shared-memory address of stage 0 (stage s at + s * kStageBytes)
@@ -379,29 +380,38 @@ __device__ __forceinline__ bool load_item_dense(WarpCtx& w, int pos, Cursor& c) 
 }
 
 // Sparse mode: position `pos` in the warp's slice of the ascending page list; pages that fall in
-// the same block are merged into one visit.  Position item_end stands for the tail block.
+// the same block are merged into one visit.  Position item_end stands for the tail block.  The list
+// is the caller's memory: an entry outside [0, closed pages) is skipped (nothing is read through it)
+// and raises kStatusInternal, which the next gkv_bits_report returns as GKV_ERR_BAD_STATE.
 __device__ __forceinline__ bool load_item_sparse(WarpCtx& w, int pos, Cursor& c) {
   const DecodeParams& p = *w.p;
   const int tiles_per_page = p.page_tokens >> 4;
   const int pages_per_block = kBlock / p.page_tokens;
-  if (pos < w.item_end) {
-    const int32_t* list = p.page_idx + static_cast<size_t>(w.stream) * p.n_sel;
+  const int n_pages = p.n_closed * pages_per_block;
+  const int32_t* list = p.page_idx + static_cast<size_t>(w.stream) * p.n_sel;
+  while (pos < w.item_end) {
     const int page = list[pos];
+    if (page < 0 || page >= n_pages) {
+      if (w.lane == 0) atomicOr(p.status, kStatusInternal);
+      ++pos;
+      continue;
+    }
     const int blk = page / pages_per_block;
     int mask = ((1 << tiles_per_page) - 1) << (tiles_per_page * (page % pages_per_block));
     int adv = 1;
     while (pos + adv < w.item_end) {
       const int pg = list[pos + adv];
-      if (pg / pages_per_block != blk) break;
+      if (pg < 0 || pg >= n_pages || pg / pages_per_block != blk) break;
       mask |= ((1 << tiles_per_page) - 1) << (tiles_per_page * (pg % pages_per_block));
       ++adv;
     }
     const TableEntry e = w.table[blk];
     c.item = pos;
+    c.first = page;              // the visit's first page (the centroid gather looks its block up again)
     c.sub = 0;
     c.adv = adv;
     c.off256 = e.off256;
-    c.resmask = 0;
+    c.resmask = e.resmask;       // tokens served from the residual pool: their stored copies are masked
     c.level = static_cast<int>(e.level);
     c.tmask = mask;
     c.ntok = kBlock;
@@ -414,6 +424,7 @@ __device__ __forceinline__ bool load_item_sparse(WarpCtx& w, int pos, Cursor& c)
     }
     return true;
   }
+  // pos == item_end (also after skipped entries): the tail
   if (pos == w.item_end && w.has_tail && p.n_tail > 0) {
     const TableEntry e = w.table[p.n_closed];
     c.item = pos;
@@ -428,7 +439,38 @@ __device__ __forceinline__ bool load_item_sparse(WarpCtx& w, int pos, Cursor& c)
     c.nsub = 2 * nt;
     return true;
   }
-  return false;
+  // Positions past the tail: the stream's groups of 16 exact residual rows, dealt round-robin to
+  // its warps.  Which rows of a group count (those whose page is listed) is decided when the
+  // group is computed.
+  const int n_res = p.res_count ? p.res_count[w.stream] : 0;
+  const int n_groups = (n_res + 15) >> 4;
+  const int k = max(pos - w.item_end - 1, 0);
+  const int j = w.sparse_rank + k * p.warps_per_stream;
+  if (j >= n_groups) return false;
+  c.item = w.item_end + 1 + k;
+  c.first = p.n_closed + 1 + j;
+  c.sub = 0;
+  c.adv = 1;
+  c.level = 17;
+  c.ntok = min(16, n_res - 16 * j);
+  c.nsub = 2;
+  c.tmask = 1;
+  c.off256 = p.res_off256[w.stream] + 32u * static_cast<uint32_t>(j);
+  c.resmask = 0;
+  return true;
+}
+
+// Page-list reads: is the page of token `tok` in the stream's ascending list?
+__device__ __forceinline__ bool page_listed(const DecodeParams& p, int stream, int tok) {
+  const int32_t* list = p.page_idx + static_cast<size_t>(stream) * p.n_sel;
+  const int page = tok / p.page_tokens;
+  int lo = 0, hi = p.n_sel;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (list[mid] < page) lo = mid + 1;
+    else hi = mid;
+  }
+  return lo < p.n_sel && list[lo] == page;
 }
 
 template <bool SPARSE>
@@ -500,7 +542,7 @@ __device__ __forceinline__ void issue_step(const WarpCtx& w, const Cursor& c, in
     const int nrows = c.ntok;
     if (lane < nrows) {
       int blk;
-      if constexpr (SPARSE) blk = p.page_idx[static_cast<size_t>(w.stream) * p.n_sel + c.item] / (kBlock / p.page_tokens);
+      if constexpr (SPARSE) blk = c.first / (kBlock / p.page_tokens);      // c.first = the visit's (range-checked) first page
       else blk = c.first + lane;
       src = p.arena + static_cast<size_t>(w.table[blk].off256) * 256 + (is_v ? kRowBytes : 0);
     }
@@ -787,15 +829,31 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
         b_lo = (t0 < c.ntok && !((c.resmask >> t0) & 1ull)) ? 0.f : kNegInf;
         b_hi = (t0 + 8 < c.ntok && !((c.resmask >> (t0 + 8)) & 1ull)) ? 0.f : kNegInf;
       } else if (c.level == 17) {
-        b_lo = (r < c.ntok) ? 0.f : kNegInf;
-        b_hi = (r + 8 < c.ntok) ? 0.f : kNegInf;
+        bool on_lo = r < c.ntok, on_hi = r + 8 < c.ntok;
+        if constexpr (SPARSE) {
+          // a residual row counts only when the page of its token is listed (Sec. 3.5: every token of
+          // a page that is not selected is masked, exact or not)
+          const int32_t* ri = p.res_idx + static_cast<size_t>(w.stream) * p.res_cap + 16 * (c.first - p.n_closed - 1);
+          on_lo = on_lo && page_listed(p, w.stream, ri[r]);
+          on_hi = on_hi && page_listed(p, w.stream, ri[r + 8]);
+        }
+        b_lo = on_lo ? 0.f : kNegInf;
+        b_hi = on_hi ? 0.f : kNegInf;
       } else {
         // centroid rows: each stands for the block's readable tokens -> add log2(count)
         float myb = kNegInf;
         if (lane < c.ntok) {
           int cnt;
-          if constexpr (SPARSE) cnt = 16 * popc4(c.tmask);
-          else cnt = kBlock - __popcll(w.table[c.first + lane].resmask);
+          if constexpr (SPARSE) {
+            // tokens of the selected pages that are not served from the residual pool
+            uint64_t sel = 0;
+#pragma unroll
+            for (int t4 = 0; t4 < 4; ++t4)
+              if ((c.tmask >> t4) & 1) sel |= 0xffffull << (16 * t4);
+            cnt = __popcll(sel & ~c.resmask);
+          } else {
+            cnt = kBlock - __popcll(w.table[c.first + lane].resmask);
+          }
           myb = cnt > 0 ? log2f(static_cast<float>(cnt)) : kNegInf;
         }
         b_lo = __shfl_sync(kFull, myb, r);
@@ -866,6 +924,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   w.pf_entry = make_uint4(0, 0, 0, 0);
   w.stream = -1;
   w.head0 = 0;
+  w.sparse_rank = 0;
   w.item_end = 0;
   w.has_tail = false;
   // A warp works for one head group: up to four query heads of one KV head.  Head group hg of stream s
@@ -885,6 +944,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
       first = static_cast<int>((static_cast<long long>(wi) * p.n_sel) / wps);
       w.item_end = static_cast<int>((static_cast<long long>(wi + 1) * p.n_sel) / wps);
       w.has_tail = (wi == wps - 1);
+      w.sparse_rank = wi;
       partial_row = blockIdx.x;      // whole CTAs per head group: one partial row per CTA
     }
   }

@@ -64,6 +64,7 @@ struct DecodeParams {
   // sparse (page list) mode
   const int32_t* page_idx;      // [n_streams][n_sel] or nullptr
   int32_t n_sel, page_tokens, warps_per_stream;
+  const int32_t* res_idx;       // sparse mode: [n_streams][res_cap] ascending token indices of the residual rows
   uint32_t* status;             // device status word (bit flags)
   // final merge: the CTA that completes a stream's last partial row normalises and writes it
   const StreamParts* parts;     // [head groups]; nullptr in sparse mode (rows of a head group = its CTAs)

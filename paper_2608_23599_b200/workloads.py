@@ -57,6 +57,7 @@ class Workload:
     softmax_scale: float = 0.0    # 0 -> 1/sqrt(d_k)
     decode_steps: int = 0
     quest_budget_tokens: int = 0
+    quest_reduce: int = 0         # page score over the KV head's query heads: 0 = max, 1 = sum
     # data recipe
     n_outlier: int = 4
     outlier_gain: float = 8.0

@@ -15,7 +15,7 @@ def oracle_config(w: W.Workload, n_layers=None) -> O.Config:
                     d_k=w.d_k, d_v=w.d_v, v_aliases_k=w.v_aliases_k, max_ctx=w.max_ctx, page_tokens=w.page_tokens,
                     policy=w.policy, stair_tokens=tuple(w.stair_tokens), n_sink_blocks=w.n_sink_blocks,
                     retire_after=w.retire_after, rd_budget_bpv=w.rd_budget_bpv,
-                    residual_fraction=w.residual_fraction, softmax_scale=w.softmax_scale)
+                    residual_fraction=w.residual_fraction, quest_reduce=w.quest_reduce, softmax_scale=w.softmax_scale)
 
 
 def f32(t):
@@ -71,6 +71,27 @@ def assert_state_equal(ocache, gcache, layer, streams=None, blocks=None):
                 if not cfg.v_aliases_k:
                     ex = gcache.gkv_debug_export_block(layer, b, h, st.n_closed, B.TENSOR_V)
                     assert np.array_equal(ex["rows"][: st.n_tail], O.bf16_bits(st.tail_v))
+
+
+def assert_boxes_and_scores_equal(ocache, gcache, layer, q_bf16, streams=None):
+    """Page boxes (exact per-page per-channel key minima / maxima) and page scores of every stream,
+    bit for bit against the oracle's."""
+    cfg = ocache.cfg
+    scores_g = gcache.gkv_debug_export_scores(layer, q_bf16.to(gcache.device))
+    scores_o = ocache.quest_scores(layer, f32(q_bf16))
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            if streams is not None and (b, h) not in streams:
+                continue
+            st = ocache.streams[(layer, b, h)]
+            n_pages = st.n_closed * (64 // cfg.page_tokens)
+            lo, hi = gcache.gkv_debug_export_boxes(layer, b, h)
+            assert lo.shape == (n_pages, cfg.d_k)
+            if n_pages:
+                assert np.array_equal(lo, O.bf16_bits(np.stack(st.box_lo[:n_pages]))), f"box minima of stream {(b, h)}"
+                assert np.array_equal(hi, O.bf16_bits(np.stack(st.box_hi[:n_pages]))), f"box maxima of stream {(b, h)}"
+            want = scores_o[(b, h)]
+            assert np.array_equal(scores_g[b, h].view(np.uint32), want.view(np.uint32)), f"page scores of stream {(b, h)}"
 
 
 def assert_outputs_close(out_gpu, out_oracle, what=""):

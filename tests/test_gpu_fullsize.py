@@ -192,6 +192,14 @@ def test_cfg3_full_size_quest_sampled():
     ocache.append_demote(0, k, v, token_mass=mass)
     for j, (b, h) in enumerate(streams):
         assert np.array_equal(gcache.gkv_debug_export_levels(0, b, h), ocache.levels(0, 0, j))
+    # boxes and page scores of the sampled streams, bit for bit (the oracle holds them as streams 0..2 of sequence 0)
+    scores_g = gcache.gkv_debug_export_scores(0, data["q"])
+    scores_o = ocache.quest_scores(0, q)
+    for j, (b, h) in enumerate(streams):
+        lo, hi = gcache.gkv_debug_export_boxes(0, b, h)
+        st = ocache.streams[(0, 0, j)]
+        assert np.array_equal(lo, O.bf16_bits(np.stack(st.box_lo))) and np.array_equal(hi, O.bf16_bits(np.stack(st.box_hi)))
+        assert np.array_equal(scores_g[b, h].view(np.uint32), scores_o[(0, j)].view(np.uint32)), f"page scores of stream {(b, h)}"
     k_sel = w.quest_budget_tokens // w.page_tokens
     pages = torch.full((w.batch, w.n_kv_heads, k_sel), -1, dtype=torch.int32, device=dev)
     n_sel = gcache.gkv_quest_select(0, data["q"], w.quest_budget_tokens, pages)

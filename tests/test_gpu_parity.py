@@ -199,6 +199,7 @@ def test_cfg3_small_quest_select_and_sparse_attention():
     data = W.make_layer(w, 0, "cpu")
     U.ingest_both(w, 0, data, ocache, gcache)
     U.assert_state_equal(ocache, gcache, 0)
+    U.assert_boxes_and_scores_equal(ocache, gcache, 0, data["q"])
     k = w.quest_budget_tokens // w.page_tokens
     pages = torch.full((w.batch, w.n_kv_heads, k), -1, dtype=torch.int32, device=dev)
     n_sel = gcache.gkv_quest_select(0, data["q"].to(dev), w.quest_budget_tokens, pages)
@@ -231,6 +232,7 @@ def test_quest_larger_pages(page):
     data = W.make_layer(w, 0, "cpu")
     U.ingest_both(w, 0, data, ocache, gcache)
     U.assert_state_equal(ocache, gcache, 0)
+    U.assert_boxes_and_scores_equal(ocache, gcache, 0, data["q"])
     k = w.quest_budget_tokens // page
     pages = torch.full((w.batch, w.n_kv_heads, k), -1, dtype=torch.int32, device=dev)
     n_sel = gcache.gkv_quest_select(0, data["q"].to(dev), w.quest_budget_tokens, pages)
@@ -246,6 +248,34 @@ def test_quest_larger_pages(page):
     U.assert_outputs_close(out, o_out, f"page {page} sparse")
     rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
     assert rep_g.resident_bits == rep_o["resident_bits"] and rep_g.last_read_bits == rep_o["last_read_bits"]
+    gcache.close()
+
+
+@pytest.mark.parametrize("group", [1, 3, 4, 8])
+def test_quest_sum_reduction_and_boxes_after_appends(group):
+    """The page score summed (instead of maximised) over the KV head's query heads, for several group
+    sizes; boxes and scores bit for bit, also after appends have closed further blocks."""
+    w = dataclasses.replace(W.config(3, "small"), n_q_heads=2 * group, quest_reduce=1, ctx=1000, max_ctx=1000 + 256)
+    ocache, gcache = _pair(w)
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    U.assert_boxes_and_scores_equal(ocache, gcache, 0, data["q"])
+    for step in range(70):
+        tok = W.make_decode_tokens(w, 0, step, "cpu")
+        ocache.append_demote(0, U.f32(tok["k"]), U.f32(tok["v"]))
+        gcache.gkv_append_demote(0, tok["k"].to(dev), tok["v"].to(dev))
+    U.assert_boxes_and_scores_equal(ocache, gcache, 0, data["q"])
+    k = 8
+    pages = torch.full((w.batch, w.n_kv_heads, k), -1, dtype=torch.int32, device=dev)
+    n_sel = gcache.gkv_quest_select(0, data["q"].to(dev), k * w.page_tokens, pages)
+    torch.cuda.synchronize()
+    sel_o = ocache.quest_select(0, U.f32(data["q"]), k * w.page_tokens)
+    assert n_sel == k
+    pg = pages.cpu().numpy()
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            assert np.array_equal(pg[b, h], sel_o[b][h])
     gcache.close()
 
 
@@ -734,3 +764,151 @@ def test_observe_and_reallocate_reject_what_they_do_not_cover():
         g.gkv_rd_reallocate(0)
     assert e.value.status == B.ERR_BAD_STATE
     g.close()
+
+
+# ---- page lists on layers that hold exact residual tokens (Sec. 3.4 + 3.5) ----------------------
+@pytest.mark.parametrize("group", [4, 8])
+def test_page_list_read_with_residual_tokens(group):
+    """RD-graded store with exact residual rows, read through a page list: residual tokens of pages
+    that are not listed are masked with their page, those of listed pages are served exact, centroid
+    pages count only their readable tokens.  Selected pages, outputs and read bits against the oracle."""
+    w = dataclasses.replace(W.config(1, "small"), n_q_heads=2 * group, page_tokens=16, residual_fraction=0.05, ctx=2048 + 40,
+                            max_ctx=2048 + 256, quest_budget_tokens=384)
+    ocache, gcache = _pair(w, 1)
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu", with_mass=True)
+    U.ingest_both(w, 0, data, ocache, gcache)
+    U.assert_state_equal(ocache, gcache, 0)
+    assert all(len(ocache.streams[(0, b, h)].res_idx) > 50 for b in range(w.batch) for h in range(w.n_kv_heads))
+    k = w.quest_budget_tokens // w.page_tokens
+    pages = torch.full((w.batch, w.n_kv_heads, k), -1, dtype=torch.int32, device=dev)
+    n_sel = gcache.gkv_quest_select(0, data["q"].to(dev), w.quest_budget_tokens, pages)
+    torch.cuda.synchronize()
+    sel_o = ocache.quest_select(0, U.f32(data["q"]), w.quest_budget_tokens)
+    pg = pages.cpu().numpy()
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            assert np.array_equal(pg[b, h, :n_sel], sel_o[b][h])
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"], page_idx_gpu=pages, n_sel=n_sel, page_idx_oracle=sel_o)
+    U.assert_outputs_close(out, o_out, "page list + residual rows")
+    assert np.max(np.abs(lse.cpu().numpy() - o_lse)) < 5e-3
+    rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
+    assert rep_g.resident_bits == rep_o["resident_bits"] and rep_g.last_read_bits == rep_o["last_read_bits"]
+    # a list of the caller's own choosing that covers pages with and without residual tokens, centroid blocks included
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            st = ocache.streams[(0, b, h)]
+            with_res = sorted(set(int(t) // 16 for t in st.res_idx))[:5]
+            own = sorted(set(with_res + [0, 1, 2, 3, 17, 40, 77, 101]))[:12]
+            own += [p for p in range(120, 128) if p not in own][: 12 - len(own)]
+            pg[b, h, :12] = sorted(own)
+    pages2 = torch.from_numpy(np.ascontiguousarray(pg[:, :, :12])).to(dev)
+    sel2 = [[pg[b, h, :12] for h in range(w.n_kv_heads)] for b in range(w.batch)]
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"], page_idx_gpu=pages2, n_sel=12, page_idx_oracle=sel2)
+    U.assert_outputs_close(out, o_out, "own page list + residual rows")
+    rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
+    assert rep_g.last_read_bits == rep_o["last_read_bits"]
+    # listing every page equals the full read
+    n_pages = (w.ctx // 64) * 4
+    all_pages = torch.arange(n_pages, dtype=torch.int32, device=dev).repeat(w.batch, w.n_kv_heads, 1).contiguous()
+    full = torch.empty((w.batch, w.n_q_heads, 128), dtype=torch.float32, device=dev)
+    gcache.gkv_decode_attn(0, data["q"].to(dev), full)
+    sparse = torch.empty_like(full)
+    gcache.gkv_decode_attn(0, data["q"].to(dev), sparse, page_idx=all_pages, n_sel=n_pages)
+    torch.cuda.synchronize()
+    assert float((full - sparse).abs().max()) < 1e-5
+    gcache.close()
+
+
+def test_page_list_entries_out_of_range_are_skipped_and_reported():
+    """A page list is the caller's memory: entries outside [0, closed pages) are skipped by the kernel
+    (no table entry and no byte is read through them), the output stays finite and equals the read of the
+    valid entries, and the next bits report returns GKV_ERR_BAD_STATE."""
+    B = _binding()
+    w = W.config(3, "small")
+    ocache, gcache = _pair(w)
+    dev = gcache.device
+    data = W.make_layer(w, 0, "cpu")
+    U.ingest_both(w, 0, data, ocache, gcache)
+    n_pages = (w.ctx // 64) * 4
+    good = np.array([3, 9, 10, 57, 100], dtype=np.int32)
+    bad = np.array([-5, 3, 9, 10, 57, 100, n_pages, 1 << 30], dtype=np.int32)      # ascending, three entries invalid
+    lists = torch.from_numpy(np.tile(bad, (w.batch, w.n_kv_heads, 1))).to(dev)
+    out = torch.empty((w.batch, w.n_q_heads, 128), dtype=torch.float32, device=dev)
+    gcache.gkv_decode_attn(0, data["q"].to(dev), out, page_idx=lists, n_sel=len(bad))
+    torch.cuda.synchronize()
+    assert torch.isfinite(out).all()
+    sel = [[good for _ in range(w.n_kv_heads)] for _ in range(w.batch)]
+    o_out, _ = ocache.decode_attn(0, U.f32(data["q"]), sel)
+    U.assert_outputs_close(out, o_out, "list with invalid entries")
+    with pytest.raises(B.GkvError) as e:
+        gcache.gkv_bits_report(0)
+    assert e.value.status == B.ERR_BAD_STATE
+    gcache.close()
+
+
+def test_arena_exhausted_by_a_demotion_step_leaves_the_cache_consistent():
+    """An arena that holds the ingested cache but not the slots of the next block-close demotions: the
+    append that closes the block reports GKV_ERR_ARENA_TOO_SMALL, and the cache stays what the host
+    mirror says it is (levels unchanged, attention still equal to the oracle with the same levels)."""
+    B = _binding()
+    w = dataclasses.replace(_tiny(1024 + 63, stair_tokens=(128, 256, 256, 256)), max_ctx=2048)
+    cfg = B.config_from_workload(w)
+    data = W.make_layer(w, 0, "cpu")
+    full_bytes = B.gkv_query_arena_bytes(cfg)
+
+    def try_ingest(nbytes):
+        try:
+            g = B.Cache(cfg, arena_bytes=nbytes)
+        except B.GkvError:
+            return None
+        try:
+            g.gkv_append_demote(0, data["k"].to(g.device), data["v"].to(g.device))
+        except B.GkvError:
+            g.close()
+            return None
+        return g
+
+    # the smallest arena (in steps of 4 KiB) that still holds the ingested cache
+    lo, hi = 0, full_bytes                                   # lo fails, hi succeeds
+    g = try_ingest(hi)
+    assert g is not None
+    g.close()
+    while hi - lo > 4096:
+        mid = (lo + hi) // 2 // 256 * 256
+        g = try_ingest(mid)
+        if g is None:
+            lo = mid
+        else:
+            g.close()
+            hi = mid
+    tok = W.make_decode_tokens(w, 0, 0, "cpu")
+    failed = None
+    for extra in range(0, 16):                               # the close needs ~35 KB of new slots before it frees the old ones
+        gcache = try_ingest(hi + extra * 2048)
+        assert gcache is not None
+        try:
+            gcache.gkv_append_demote(0, tok["k"].to(gcache.device), tok["v"].to(gcache.device))
+        except B.GkvError as e:
+            assert e.status == B.ERR_ARENA_TOO_SMALL
+            failed = gcache
+            break
+        gcache.close()
+    assert failed is not None, "no arena size found where only the demotion step runs out of slots"
+    gcache = failed
+    # the block closed (17 closed blocks, all levels as before the failed demotions, the new one exact)
+    lv = gcache.gkv_debug_export_levels(0, 0, 0)
+    assert len(lv) == 17 and lv[-1] == 16
+    ocfg = U.oracle_config(dataclasses.replace(w, policy=W.POLICY_EXTERNAL))
+    oc = O.GradedCache(ocfg)
+    kk = torch.cat([data["k"], tok["k"]], dim=1)
+    vv = torch.cat([data["v"], tok["v"]], dim=1)
+    plan = np.tile(lv.astype(np.int8), (w.batch, w.n_kv_heads, 1))
+    oc.append_demote(0, U.f32(kk), U.f32(vv), level_plan=plan)
+    out = torch.empty((w.batch, w.n_q_heads, 128), dtype=torch.float32, device=gcache.device)
+    gcache.gkv_decode_attn(0, tok["q"].to(gcache.device), out)
+    torch.cuda.synchronize()
+    o_out, _ = oc.decode_attn(0, U.f32(tok["q"]))
+    U.assert_outputs_close(out, o_out, "after a failed demotion step")
+    assert gcache.gkv_bits_report(0).resident_bits == oc.bits_report(0)["resident_bits"]
+    gcache.close()

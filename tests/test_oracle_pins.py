@@ -127,6 +127,10 @@ def test_accounting_identities_from_paper():
     assert len(sel[0][0]) == 33
     c.decode_attn(0, q, sel)
     assert c.bits_report(0)["bpv_read"] == g_quest_read
+    # the summaries count for the read that scored them: the same list read again, without a new
+    # scoring pass, costs the pages alone (12.5 % of the pages + the current page = 33 / 256 of 16 bits)
+    c.decode_attn(0, q, sel)
+    assert c.bits_report(0)["bpv_read"] == g_quest_read - g_box == 33 / 256 * 16
     # exact tokens cost 16 bits per value each, tail included: StreamingLLM / SnapKV rows
     for kept, want in ((4 + 2048, g_stream), (2304, g_snap)):
         c2 = O.GradedCache(cfg)
@@ -709,3 +713,134 @@ def test_certificate_is_zero_for_an_exact_cache_and_ignores_exact_residual_rows(
     for h in range(2):
         assert np.linalg.norm(o_true[0, h] - o_hat[0, h]) <= c_with[0, h]
     assert np.all(c_with > 0) and np.all(c_without > 0)
+
+
+# ---- Sec. 3.5 Eq. 8: bits a page-list read touches, written out by hand -------------------------
+def test_page_list_read_bits_by_hand():
+    """d_k = d_v = 32, 16-token pages, 64-token blocks, groups of 32: every term of the read cost of
+    a page list, counted by hand for one stream whose six closed blocks sit on known rungs."""
+    D = 32
+    cfg = small_cfg(n_q_heads=1, n_kv_heads=1, d_k=D, d_v=D, page_tokens=16, policy=O.POLICY_EXTERNAL)
+    T = 6 * 64 + 5                                    # six closed blocks and a partial block of 5 tokens
+    k, v, q = rand_kv(cfg, T)
+    plan = np.array([[[4, 1, 16, 8, 2, 1]]], dtype=np.int8)
+    c = O.GradedCache(cfg)
+    c.append_demote(0, k, v, level_plan=plan)
+    nval = 2 * D                                      # values per token
+    tail = 5 * 16 * nval                              # the partial block is always read, exact
+
+    def read(pages):
+        c.decode_attn(0, q, [[np.array(pages, dtype=np.int32)]])
+        return c.bits_report(0)["last_read_bits"]
+
+    codes4 = 16 * nval * 4                            # one page of 4-bit codes (keys and values)
+    vpar = 16 * (D // 32) * 32                        # value params: one group of 32 channels per token
+    kgrp = D * 32                                     # key params of one 32-token group: D channels x (scale + zero)
+    # one page of the int4 block 0
+    assert read([0]) == codes4 + vpar + kgrp + tail == 4096 + 512 + 1024 + tail
+    # pages 0 and 1 share one 32-token key group: its params are read once
+    assert read([0, 1]) == 2 * (codes4 + vpar) + kgrp + tail
+    # pages 0 and 2 lie in different halves of the block: two key groups
+    assert read([0, 2]) == 2 * (codes4 + vpar) + 2 * kgrp + tail
+    # a centroid block (block 1 = pages 4..7) costs its two centroid rows once, however many pages
+    cent = 16 * nval
+    assert read([4]) == cent + tail
+    assert read([4, 5, 7]) == cent + tail
+    # an exact block (block 2 = pages 8..11): 16 bits per value of the page, no params
+    assert read([9]) == 16 * nval * 16 + tail
+    # int8 block 3 (pages 12..15) and int2 block 4 (pages 16..19)
+    assert read([12]) == 16 * nval * 8 + vpar + kgrp + tail
+    assert read([16, 17, 18, 19]) == 4 * (16 * nval * 2 + vpar) + 2 * kgrp + tail
+    # everything mixed: the sum of the parts (block 5 is a second centroid block: pages 20..23)
+    assert read([0, 1, 5, 9, 12, 19, 22]) == (2 * (codes4 + vpar) + kgrp) + cent + 16 * nval * 16 + (16 * nval * 8 + vpar + kgrp) \
+        + (16 * nval * 2 + vpar + kgrp) + cent + tail
+    # selecting every page of a quantised block reads the whole block: codes + all params
+    whole4 = 64 * nval * 4 + (64 * nval // 32) * 32
+    assert read([0, 1, 2, 3]) == whole4 + tail
+    # an empty list reads the partial block only
+    assert read([]) == tail
+
+
+# ---- Sec. 3.5 page score with the sum over the KV head's query heads -----------------------------
+def test_quest_scores_sum_reduction():
+    """The flag variant of the page score (sum instead of max over the g query heads): scalar fp32
+    loops in the stated order (channels ascending, then heads ascending), the upper-bound property
+    head by head, and g = 1 where sum and max coincide."""
+    cfg_sum = small_cfg(n_q_heads=6, n_kv_heads=2, page_tokens=16, stair_tokens=(-1, 0, 0, 0), quest_reduce=O.REDUCE_SUM)
+    T = 330
+    k, v, q = rand_kv(cfg_sum, T)
+    c = O.GradedCache(cfg_sum)
+    c.append_demote(0, k, v)
+    scores = c.quest_scores(0, q)
+    g = 3
+    n_pages = (T // 64) * 4
+    f32 = np.float32
+    for (b, h), sc in scores.items():
+        assert len(sc) == n_pages and sc.dtype == np.float32
+        for p in range(n_pages):
+            page = k[b, 16 * p:16 * p + 16, h]                        # bf16 values
+            lo, hi = page.min(axis=0), page.max(axis=0)
+            total = None
+            bound = 0.0
+            for j in range(g):
+                qh = q[b, h * g + j]
+                acc = f32(0.0)
+                for d in range(cfg_sum.d_k):
+                    acc = f32(acc + f32(qh[d]) * f32(hi[d] if qh[d] >= 0 else lo[d]))     # the product is exact in fp32
+                total = acc if total is None else f32(total + acc)
+                bound += float(np.max(page.astype(np.float64) @ qh.astype(np.float64)))
+            assert sc[p] == total, (b, h, p)
+            assert sc[p] >= bound - 1e-4 * (1 + abs(bound))           # sum of per-head upper bounds
+    # one query head per KV head: nothing to reduce, sum == max
+    for red in (O.REDUCE_SUM, O.REDUCE_MAX):
+        cfg1 = small_cfg(n_q_heads=2, n_kv_heads=2, page_tokens=16, stair_tokens=(-1, 0, 0, 0), quest_reduce=red)
+        c1 = O.GradedCache(cfg1)
+        c1.append_demote(0, k, v)
+        s1 = c1.quest_scores(0, q[:, :2])
+        if red == O.REDUCE_SUM:
+            keep = s1
+        else:
+            for key in s1:
+                assert np.array_equal(s1[key], keep[key])
+    # the selection follows the summed score
+    sel = c.quest_select(0, q, 64)
+    for (b, h), sc in scores.items():
+        assert list(sel[b][h]) == sorted(np.argsort(-sc.astype(np.float64), kind="stable")[:4].tolist())
+
+
+def test_page_list_with_residual_tokens_masks_cold_pages_and_counts_listed_rows():
+    """Sec. 3.4 + 3.5 together: exact residual tokens of pages that are not listed are masked like
+    the rest of their page; those of listed pages are read exact.  Checked against dense attention
+    over hand-built rows, and the read bits against a count by hand."""
+    D = 32
+    cfg = small_cfg(n_q_heads=2, n_kv_heads=1, d_k=D, d_v=D, page_tokens=16, policy=O.POLICY_EXTERNAL, residual_fraction=0.05)
+    T = 4 * 64 + 3
+    k, v, q = rand_kv(cfg, T)
+    mass = RNG.random((1, 1, T)).astype(np.float32)
+    plan = np.array([[[4, 1, 2, 8]]], dtype=np.int8)
+    c = O.GradedCache(cfg)
+    c.append_demote(0, k, v, token_mass=mass, level_plan=plan)
+    st = c.streams[(0, 0, 0)]
+    res = [int(t) for t in st.res_idx]
+    assert len(res) == int(0.05 * T) and len(res) >= 8
+    pages = sorted(set([res[0] // 16, res[3] // 16, 5]))            # two pages holding residual tokens and page 5
+    out, _ = c.decode_attn(0, q, [[np.array(pages, dtype=np.int32)]])
+    # dense attention over exactly the readable rows: listed pages (residual tokens exact, the others
+    # reconstructed) and the partial block
+    K, V = c.reconstruct(st)
+    rows = [t for pg in pages for t in range(16 * pg, 16 * pg + 16)] + list(range(256, T))
+    for t in rows:
+        if t in res:
+            assert np.array_equal(K[t], k[0, t, 0].astype(np.float64)) and np.array_equal(V[t], v[0, t, 0].astype(np.float64))
+    for h in range(2):
+        w = np.exp(K[rows] @ q[0, h].astype(np.float64) * c.scale)      # the oracle's softmax scale (fp32 1/sqrt(d))
+        ref = (w[:, None] * V[rows]).sum(0) / w.sum()
+        assert np.abs(out[0, h] - ref).max() < 1e-12, np.abs(out[0, h] - ref).max()
+    # read bits: the pages' own cost plus 16 bits per value for every residual row on a listed page
+    n_listed = sum(1 for t in res if t // 16 in pages)
+    assert n_listed >= 2
+    with_res = c.bits_report(0)["last_read_bits"]
+    c2 = O.GradedCache(small_cfg(n_q_heads=2, n_kv_heads=1, d_k=D, d_v=D, page_tokens=16, policy=O.POLICY_EXTERNAL))
+    c2.append_demote(0, k, v, level_plan=plan)
+    c2.decode_attn(0, q, [[np.array(pages, dtype=np.int32)]])
+    assert with_res == c2.bits_report(0)["last_read_bits"] + n_listed * 16 * 2 * D
