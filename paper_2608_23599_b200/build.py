@@ -12,7 +12,7 @@ SOURCES = ["gkv_api.cu", "gkv_decode.cu", "gkv_pack.cu", "gkv_ingest.cu", "gkv_q
 HEADERS = ["gkv_internal.h", "gkv_layout.cuh", "gkv_mla.h", os.path.join("..", "..", "include", "gkv.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--use_fast_math=false",
+    "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
 ]
 
 
@@ -33,8 +33,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     objs = []
-    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
-    flags += os.environ.get("GKV_NVCC_DEFS", "").split()      # e.g. -DGKV_DECODE_WARPS=12 (tuning experiments)
+    flags = list(NVCC_FLAGS)
     procs = []
     for src in SOURCES:
         obj = os.path.join(CSRC, src.replace(".cu", ".o"))

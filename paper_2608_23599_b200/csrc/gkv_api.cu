@@ -8,6 +8,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <mutex>
 #include <numeric>
 #include <thread>
 #include <vector>
@@ -126,6 +127,7 @@ struct gkv_cache {
   float scale = 0.f;
   SlotHeap heap;
   std::vector<LayerState> layers;
+  int device = -1;                      // the device that owns the arena
   int desc_src = -1;                    // layer whose work lists were last built from scratch
   // shared device scratch
   uint32_t* status_d = nullptr;
@@ -1264,14 +1266,22 @@ constexpr int kMaxDevices = 64;
 static float* g_static_scores_ptr[kMaxDevices] = {};
 
 // In host code the array's name is only a handle; the device address has to be asked for, once
-// per device, with that device current.
+// per device, with that device current.  The device is the one that owns the cache's arena (not
+// whatever device the calling thread happens to have current), and the first look-up per device
+// is serialised between host threads.
+std::mutex g_static_scores_mutex;
 int static_scores_address(gkv_cache* c, float** out) {
-  int dev = -1;
-  CK(c, cudaGetDevice(&dev));
+  const int dev = c->device;
   if (dev < 0 || dev >= kMaxDevices) return GKV_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_scores_mutex);
   if (!g_static_scores_ptr[dev]) {
+    int cur = -1;
+    CK(c, cudaGetDevice(&cur));
+    if (cur != dev) CK(c, cudaSetDevice(dev));
     void* ptr = nullptr;
-    CK(c, cudaGetSymbolAddress(&ptr, g_static_scores));
+    const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scores);
+    if (cur != dev) cudaSetDevice(cur);
+    if (e != cudaSuccess) return cuda_fail(c, e);
     g_static_scores_ptr[dev] = static_cast<float*>(ptr);
   }
   *out = g_static_scores_ptr[dev];
@@ -1322,6 +1332,11 @@ int gkv_create(const gkv_config* cfg, void* arena, size_t arena_bytes, gkv_cache
   gkv_cache* c = new (std::nothrow) gkv_cache();
   if (!c) return GKV_ERR_INVALID_ARG;
   c->cfg = *cfg;
+  {
+    cudaPointerAttributes attr{};
+    if (cudaPointerGetAttributes(&attr, arena) == cudaSuccess && attr.type == cudaMemoryTypeDevice) c->device = attr.device;
+    else cudaGetDevice(&c->device);
+  }
   c->arena = static_cast<uint8_t*>(arena);
   c->arena_bytes = arena_bytes;
   c->n_streams = d.n_streams;

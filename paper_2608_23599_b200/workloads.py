@@ -70,8 +70,17 @@ class Workload:
         return self.n_q_heads // self.n_kv_heads
 
 
+# Bit budgets handed to the RD allocator.  The allocator snaps every block up to a ladder rung and
+# projects the plan onto the monotone staircase, so the rate it realises lies below its budget by
+# a data-dependent amount; the recipes name realised averages (config 1: 5 bits/value including the
+# 1 % exact residual, i.e. 4.84 for the graded part; config 3: 4 bits/value; config 6: 9.6), so the
+# budgets are fitted on the recipes' own data: `python -m oracle.fit_rd_budget CONFIG TARGET`.
+RD_BUDGET = {1: 5.3437, 3: 4.0, 6: 9.604}
+
+
 def config(cid: int, scale: str = "full") -> Workload:
-    """The five benchmark configurations (0-4) and the RD-V2 operating point (5); ``scale='small'`` keeps the structure
+    """The five benchmark configurations (0-4), the RD-V2 operating point (5) and the paper's own Quest
+    setting (6); ``scale='small'`` keeps the structure
     (every rung populated, ragged tail, several splits) at a size the CPU
     oracle finishes in seconds."""
     small = scale == "small"
@@ -83,7 +92,7 @@ def config(cid: int, scale: str = "full") -> Workload:
         T = 2048 if small else 16384
         return Workload("cfg1_qwen3b_rd5", 1, 2 if small else 36, 1, 16, 2, 128, 128, T, T + 128,
                         policy=POLICY_RD, retire_after=512 if not small else 128,
-                        rd_budget_bpv=4.84, residual_fraction=0.01, drift_std=0.05)
+                        rd_budget_bpv=4.84 if small else RD_BUDGET[1], residual_fraction=0.01, drift_std=0.05)
     if cid == 2:
         if small:
             return Workload("cfg2_llama8b_append_small", 2, 2, 2, 8, 2, 128, 128, 2048, 2048 + 256,
@@ -96,7 +105,7 @@ def config(cid: int, scale: str = "full") -> Workload:
                             page_tokens=16, policy=POLICY_RD, rd_budget_bpv=4.0, retire_after=64,
                             n_clusters=16, n_heavy=0, quest_budget_tokens=256)
         return Workload("cfg3_quest_llama8b", 3, 32, 4, 32, 8, 128, 128, 32768, 32768 + 128,
-                        page_tokens=16, policy=POLICY_RD, rd_budget_bpv=4.0, retire_after=64,
+                        page_tokens=16, policy=POLICY_RD, rd_budget_bpv=RD_BUDGET[3], retire_after=64,
                         n_clusters=64, n_heavy=0, quest_budget_tokens=2048)
     if cid == 4:
         T = 8192 if small else 1048576
@@ -121,6 +130,17 @@ def config(cid: int, scale: str = "full") -> Workload:
                             stair_tokens=(128, 0, 0, 0), residual_fraction=0.10, drift_std=0.05)
         return Workload("cfg5_rdv2", 5, 32, 8, 32, 8, 128, 128, 32768, 32768 + 128,
                         stair_tokens=(256, 0, 0, 0), residual_fraction=0.10, drift_std=0.05)
+    if cid == 6:
+        # not one of the five headline configurations: compressed-Quest as the paper sets it (Sec. 3.5 last
+        # paragraph, Table 2): page = block = 64 tokens, 12.5 % of the pages selected, a graded base of about
+        # 9.6 bits/value (resident 9.85 with the 0.25 bits/value of exact boxes), on the config-3 shapes and keys
+        if small:
+            return Workload("cfg6_quest_paper_small", 6, 1, 2, 8, 2, 128, 128, 2048 + 24, 2048 + 128,
+                            page_tokens=64, policy=POLICY_RD, rd_budget_bpv=RD_BUDGET[6], retire_after=64,
+                            n_clusters=16, n_heavy=0, quest_budget_tokens=256)
+        return Workload("cfg6_quest_paper", 6, 32, 4, 32, 8, 128, 128, 32768, 32768 + 128,
+                        page_tokens=64, policy=POLICY_RD, rd_budget_bpv=RD_BUDGET[6], retire_after=64,
+                        n_clusters=64, n_heavy=0, quest_budget_tokens=4096)
     raise ValueError(cid)
 
 

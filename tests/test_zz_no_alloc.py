@@ -1,8 +1,8 @@
 """The allocation-free page selection (gkv_quest_select_static) must return exactly what
 gkv_quest_select returns.  It exists for callers that cannot let the library's work depend on any
 device allocation (a fixed arena inside a fully committed memory pool, a no-allocation real-time
-loop), so its score scratch is a fixed array inside the library.  Collected last on purpose:
-a run that stops at the first failure has then already run every other test."""
+loop), so its score scratch is a fixed array inside the library.  Two calls in a row: the array
+keeps the first call's scores, and the second call must not be disturbed by them."""
 import dataclasses
 
 import pytest
