@@ -252,7 +252,11 @@ def test_cfg4_full_size_mla_one_million_tokens():
     (a) sampled blocks of every rung are bit-exact against the oracle's per-block encoder;
     (b) property that holds at any size: the million-token result equals the log-sum-exp merge of
         four quarter caches that hold the same blocks at the same levels;
-    (c) the newest quarter (exact + int8 rungs, 262,144 tokens, 4096 blocks) matches the oracle."""
+    (c) the newest quarter (exact + int8 rungs, 262,144 tokens, 4096 blocks) matches the oracle;
+    (d) the two rungs that hold three quarters of the context: a 65,536-token window of the int4 rung, one
+        of the centroid rung and one across the centroid / int4 border, read from caches that hold these
+        windows at the exported levels, match the oracle on the same rows (outputs and log-sum-exp), and the
+        merge of (b) ties the windows' quarters to the million-token result."""
     B = _binding()
     w = dataclasses.replace(W.config(4), n_layers=1)
     gcache = B.Cache(B.config_from_workload(w, 1))
@@ -320,4 +324,35 @@ def test_cfg4_full_size_mla_one_million_tokens():
     err, rel = U.assert_outputs_close(newest[0], o_out, "cfg4 newest quarter")
     assert np.max(np.abs(newest[1].cpu().numpy() - o_lse)) < 5e-3
     print(f"cfg4 full: quarter-merge gap {gap:.2e}, newest-quarter max-abs error {err:.2e}, relative L2 {rel:.2e}")
+    # (d) windows of the int4 and centroid rungs against the oracle
+    first4 = int(np.argmax(levels == 4)) * 64                        # first token of the int4 rung (the centroid rung ends here)
+    Wn = 65536
+    wwin = dataclasses.replace(w, ctx=Wn, max_ctx=Wn + 64, policy=W.POLICY_EXTERNAL)
+    for name, start in (("centroid rung", 1024 * 64), ("centroid / int4 border", first4 - Wn // 2), ("int4 rung", first4 + 2048 * 64)):
+        lv = levels[start // 64:(start + Wn) // 64].astype(np.int8)
+        assert set(np.unique(lv)) <= {1, 4}
+        plan = lv.reshape(1, 1, -1)
+        kw = k[:, start:start + Wn].contiguous()
+        wc = B.Cache(B.config_from_workload(wwin, 1))
+        wc.gkv_append_demote(0, kw, None, level_plan=plan)
+        o = torch.empty_like(out_full); l = torch.empty_like(lse_full)
+        wc.gkv_decode_attn(0, data["q"], o, l)
+        torch.cuda.synchronize()
+        oc = O.GradedCache(U.oracle_config(wwin, 1))
+        oc.append_demote(0, U.f32(kw.cpu()), None, level_plan=plan)
+        o_out, o_lse = oc.decode_attn(0, U.f32(data["q"]))
+        err, rel = U.assert_outputs_close(o, o_out, f"cfg4 window in the {name}")
+        assert np.max(np.abs(l.cpu().numpy() - o_lse)) < 5e-3
+        # a few blocks of the window, bit for bit
+        st = oc.streams[(0, 0, 0)]
+        for i in (0, 511, 1023):
+            ex = wc.gkv_debug_export_block(0, 0, 0, i, B.TENSOR_K)
+            blk = st.blocks[i]
+            assert ex["level"] == blk.level
+            if blk.level == 1:
+                assert np.array_equal(ex["rows"][0], O.bf16_bits(blk.k_cent))
+            else:
+                assert np.array_equal(ex["codes"], blk.k_codes) and np.array_equal(ex["scale"], blk.k_scale.view(np.uint16))
+        print(f"cfg4 full: window in the {name}: max-abs error {err:.2e}, relative L2 {rel:.2e}")
+        wc.close()
     gcache.close()
