@@ -14,7 +14,7 @@
 // A-fragment order (gkv_layout.cuh) at bit positions where one LOP3 turns a code into the fp16
 // number "bias + code".  Scales are folded into the B operands (q' = q * s_k per 32-token key
 // group, P' = p * s_v per 32-channel value group); zero points and the biases are handled by
-// extra MMAs (A = zero-point pattern or all ones) instead of per-value arithmetic.
+// extra MMAs (A = scale / zero-point pattern or a constant) instead of per-value arithmetic.
 //
 // Precision: every B operand that carries a rounded product or probability is a pair hi + lo of
 // fp16 (bf16 for exact rows) numbers, hi = rn(x), lo = rn(x - hi), so that the operand is good to
@@ -37,7 +37,6 @@ namespace {
 constexpr unsigned kFull = 0xffffffffu;
 constexpr float kNegInf = -__builtin_huge_valf();
 constexpr int kRowPitch = kRowBytes + 16;       // staged exact rows: 272 B pitch -> conflict-free ldmatrix
-constexpr uint32_t kOnesH2 = 0x3C003C00u;       // half2(1, 1)
 constexpr int kWaitSpins = 1 << 20;             // bound of every mbarrier wait (each poll may sleep up to the hint)
 constexpr uint32_t kWaitHintNs = 2000;          // suspend-time hint of one mbarrier poll, nanoseconds
 
@@ -130,7 +129,7 @@ __device__ __forceinline__ float bf16hi_to_f32(uint32_t u) { return __uint_as_fl
 // ---- code unpack: the four A registers of MMA index s as fp16 "bias + code" ------------------
 // A code that sits at mantissa bit b of an fp16 with exponent 2^E has the value code * 2^(E - 10 + b),
 // so picking E = 10 - b makes "mask, or in the exponent" a complete conversion.  The bias 2^(10 - b)
-// is cancelled after the MMA in fp32 (against "bias * sum of the B operand" from a ones MMA), which
+// is cancelled after the MMA in fp32 (against "bias * sum of the B operand"), which
 // costs 2^-23 * bias * |sum| of accuracy: the words are therefore shifted so that the codes land in
 // the upper mantissa bits (8-bit: bias 1024 against codes up to 255; 4-bit: 256 / 16; 2-bit: 16 / 4;
 // first / second number = A rows r / rows r + 8 of the MMA).  `mid` is the centre of the code range:
@@ -653,16 +652,13 @@ __device__ __forceinline__ void load_words(uint32_t codes, int j, int lane, uint
 }
 
 // Logits of the active tiles of one half (32 tokens): S = scale * (q . k~) + token bias, with
-// k~ = s * code + z.  Data MMAs use A = bias + code and B = q' = q * s (hi and lo columns); the bias
-// (and the code centre) is removed with a "ones" MMA on the same q' and the zero points enter through
-// an MMA with A = (z | s) and B = q.  All arguments that address shared memory are 32-bit addresses.
-// The loop over channel slabs is kept rolled: the kernel is bound by instruction fetch, and a
-// compact body that stays in the instruction caches is worth more than the scheduling freedom
-// of straight-line code.
+// k~ = s * code + z.  Data MMAs use A = bias + code and B = q' = q * s (hi and lo columns); an MMA with
+// A = (s | z) and B = q gives sum q s, which is what the bias multiplies (q' is an exact split of q s),
+// and sum q z.  All arguments that address shared memory are 32-bit addresses.
 // Channel slab j (MMA indices 2 j and 2 j + 1) of qk_half; FIRST starts the accumulation chains.
 template <int BITS, bool FULL, bool FIRST>
 __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm, uint32_t qh_addr, int lane,
-                                        const uint32_t (&ones)[4], float (&zd)[4], float (&qe)[4], float (&S)[2][4]) {
+                                        float (&zd)[4], float (&S)[2][4]) {
   constexpr int cb = 256 * BITS;
   constexpr int kW = BITS / 2;
   uint32_t w0[kW], w1[kW];
@@ -681,8 +677,6 @@ __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm
     }
     if (FIRST && ss == 0) mma_f16_first(zd, pr.x, pr.y, pr.z, pr.w, q.x, q.y);
     else mma_f16(zd, pr.x, pr.y, pr.z, pr.w, q.x, q.y);
-    if (FIRST && ss == 0) mma_f16_first(qe, ones[0], ones[1], ones[2], ones[3], q0, q1);
-    else mma_f16(qe, ones[0], ones[1], ones[2], ones[3], q0, q1);
     uint32_t a[4];
     if (FULL || (tm & 1)) {
       unpack<BITS>(w0, ss, a);
@@ -700,20 +694,21 @@ __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm
 // x = the four logits of the lane's head: tile 0 rows r, r + 8, tile 1 rows r, r + 8.
 template <int BITS, bool FULL>
 __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, int tm, uint32_t qh_addr, int lane, float scale_log2,
-                                        uint64_t resmask, int half, const uint32_t (&ones)[4], float (&x)[4]) {
+                                        uint64_t resmask, int half, float (&x)[4]) {
   const int c4 = lane & 3, r = lane >> 2;
-  float zd[4];        // rows r: sum_c q_c s_c; rows r + 8: sum_c q_c z_c (exact products; both columns alike)
-  float qe[4];        // sum_c q'_c: hi column, lo column (all rows equal)
+  // rows r: sum_c q_c s_c; rows r + 8: sum_c q_c z_c (exact products; both columns alike).  The first is
+  // also the sum of q' over its hi and lo columns (q' = q s is split exactly), i.e. what the bias of the
+  // data MMAs multiplies.
+  float zd[4];
   float S[2][4];
   kp += c4 * 16;
-  qk_slab<BITS, FULL, true>(kp, kc0, 0, tm, qh_addr, lane, ones, zd, qe, S);
+  qk_slab<BITS, FULL, true>(kp, kc0, 0, tm, qh_addr, lane, zd, S);
 #pragma unroll
-  for (int j = 1; j < 4; ++j) qk_slab<BITS, FULL, false>(kp, kc0, j, tm, qh_addr, lane, ones, zd, qe, S);
+  for (int j = 1; j < 4; ++j) qk_slab<BITS, FULL, false>(kp, kc0, j, tm, qh_addr, lane, zd, S);
   // rows r carry bias lo, rows r + 8 carry bias hi
   constexpr float kMid = Bias<BITS>::mid;
-  const float qs = qe[0] + qe[1];
-  const float z0 = fmaf(kMid, zd[0], zd[2]);                                    // sum q (z + mid s)
-  const float c_lo = fmaf(-(Bias<BITS>::lo + kMid), qs, z0), c_hi = fmaf(-(Bias<BITS>::hi + kMid), qs, z0);
+  (void)kMid;                                                                  // (code - mid) s + (z + mid s)
+  const float c_lo = fmaf(-Bias<BITS>::lo, zd[0], zd[2]), c_hi = fmaf(-Bias<BITS>::hi, zd[0], zd[2]);
   const uint32_t rm = static_cast<uint32_t>(resmask >> (32 * half));            // this half's 32 tokens
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
@@ -789,10 +784,10 @@ __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const 
 
 template <int BITS, bool FULL>
 __device__ __forceinline__ void qk_softmax_half(uint32_t half_k, int half, int tm, uint64_t resmask, uint32_t qh_addr,
-                                                int lane, float scale_log2, const uint32_t (&ones)[4], SoftmaxState& st,
+                                                int lane, float scale_log2, SoftmaxState& st,
                                                 uint32_t (&pf)[2][2]) {
   float x[4];
-  qk_half<BITS, FULL>(half_k, half_k + 512, tm, qh_addr, lane, scale_log2, resmask, half, ones, x);
+  qk_half<BITS, FULL>(half_k, half_k + 512, tm, qh_addr, lane, scale_log2, resmask, half, x);
   softmax_update<4>(x, st);
   make_p_f16(x[0], x[1], pf[0], st);
   make_p_f16(x[2], x[3], pf[1], st);
@@ -800,7 +795,7 @@ __device__ __forceinline__ void qk_softmax_half(uint32_t half_k, int half, int t
 
 // Process a staged step.  pf carries P fragments from a key step to the following value step.
 template <bool SPARSE, bool MASS>
-__device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, int sidx, const uint32_t (&ones)[4],
+__device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, int sidx,
                                              SoftmaxState& st, uint32_t (&pf)[4]) {
   const DecodeParams& p = *w.p;
   const int lane = w.lane;
@@ -893,16 +888,16 @@ __device__ __forceinline__ void compute_step(const WarpCtx& w, const Cursor& c, 
   if (c.level == 8) {
     const int half = FULL ? (c.sub >> 1) : ((c.tmask == 15) ? (c.sub >> 1) : half_of_step(c, c.sub >> 1));
     const int tm = (c.tmask >> (2 * half)) & 3;
-    if ((c.sub & 1) == 0) qk_softmax_half<8, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, ones, st, pf2);
+    if ((c.sub & 1) == 0) qk_softmax_half<8, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
     else pv_half<8, FULL>(sa, sa + 512, tm, pf2, lane, st);
   } else {
     const int half = FULL ? c.sub : ((c.tmask == 15) ? c.sub : half_of_step(c, c.sub));
     const int tm = (c.tmask >> (2 * half)) & 3;
     if (c.level == 4) {
-      qk_softmax_half<4, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, ones, st, pf2);
+      qk_softmax_half<4, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
       pv_half<4, FULL>(sa + off_vp(4, 0), sa + off_vc(4, 0), tm, pf2, lane, st);
     } else {
-      qk_softmax_half<2, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, ones, st, pf2);
+      qk_softmax_half<2, FULL>(sa, half, tm, c.resmask, qh, lane, p.scale_log2, st, pf2);
       pv_half<2, FULL>(sa + off_vp(2, 0), sa + off_vc(2, 0), tm, pf2, lane, st);
     }
   }
@@ -1024,11 +1019,6 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
   for (int u = 0; u < 8; ++u) st.o[u][0] = st.o[u][1] = st.o[u][2] = st.o[u][3] = 0.f;
   st.zc = 0.f;
   uint32_t pf[4] = {0, 0, 0, 0};
-  // half2(1, 1) four times: the A operand of the column-sum MMAs.  Produced by opaque moves so that
-  // the compiler keeps one register quad for the whole kernel instead of rebuilding it per MMA.
-  uint32_t ones[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) asm volatile("mov.b32 %0, %1;\n" : "=r"(ones[i]) : "r"(kOnesH2));
 
   // Software pipeline over steps: while step k is computed, step k + 1 is in flight.  The loop
   // starts on an empty pseudo-unit (level 0) so that the cursor and copy code exists once.
@@ -1069,7 +1059,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
           mass_m = st.m;
         }
       }
-      compute_step<SPARSE, MASS>(w, cur, sidx, ones, st, pf);
+      compute_step<SPARSE, MASS>(w, cur, sidx, st, pf);
       if constexpr (MASS) {
         // A block (or the partial block) is done: what it added to the lane's running sum is the
         // sum now minus the sum at its start brought to the current max.
