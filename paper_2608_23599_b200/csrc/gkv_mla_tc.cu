@@ -46,7 +46,11 @@ constexpr int kOffTile = 0;
 constexpr int kOffQp = 2 * kTcTileBytes;               // 147456: Q' of one block, laid out like a tile (row = column of S)
 constexpr int kOffP = kOffQp + kTcTileBytes;           // 221184
 constexpr int kOffMisc = kOffP + kTcPBytes;            // 225280
+#ifdef GKV_MLA_PROF
+constexpr int kTcSmem = kOffMisc + 5120 + 1024 + 128;
+#else
 constexpr int kTcSmem = kOffMisc + 5120 + 1024;        // + misc + alignment slack = 231424
+#endif
 // misc: mbarriers (128 B) | tmem base @128 | abort flag @132 | bias[2][64] floats @256 |
 //       head maxima [2][4 warps][16] @768 | row sums [4][16] @1280 | key constants [2 tiles][2 halves][16] @1536 |
 //       probability sums per warp [2 tiles][4][16] @1792 | parts of the key constants [2][2][9 warps][16] @2304 |
@@ -67,6 +71,16 @@ constexpr uint32_t kTmemR = 128;                       // per-half accumulators:
 constexpr uint32_t kTmemO = 384;                       // running O^T: [4 channel tiles][16 heads]
 constexpr int kPrefetchAhead = 6;                      // tiles the L2 prefetch runs ahead of the key MMAs
 constexpr float kRescaleSlack = 8.f;                   // keep a stale running max while logits stay within 2^8 of it
+
+#ifdef GKV_MLA_PROF
+// development aid: cycles per role and phase, kept in shared memory by one lane per role
+__device__ unsigned long long g_prof[148 * 32];
+#define PROF_DECL(basei) uint32_t* const pbase = prof_sm + (basei); uint32_t pt0 = clock()
+#define PROF_LAP(i) do { const uint32_t pt1 = clock(); if (prof_lane) pbase[i] += pt1 - pt0; pt0 = pt1; } while (0)
+#else
+#define PROF_DECL(basei)
+#define PROF_LAP(i)
+#endif
 
 __device__ __forceinline__ uint32_t t_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ void t_bar_init(uint32_t bar, uint32_t count) {
@@ -103,17 +117,32 @@ __device__ __forceinline__ bool t_wait(uint32_t bar, uint32_t parity, volatile i
   }
   return true;
 }
-// the same for a whole warp: the outcome is made uniform (lanes poll on their own)
-__device__ __forceinline__ bool t_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  return __all_sync(kFullT, t_wait(bar, parity, abort_flag));
+// Wait of a whole warp role (n threads on named barrier `id`): the role's first warp polls the
+// mbarrier, the others block on the named barrier and spend no issue slots; the outcome (false after a
+// time-out or an abort) reaches every thread through the barrier's reduction, so the role leaves its
+// loop as one.
+__device__ __forceinline__ bool t_role_sync(int id, int n, bool ok_in) {
+  const uint32_t ok = ok_in ? 1u : 0u;
+  uint32_t all;
+  asm volatile(
+      "{\n"
+      ".reg .pred pi, po;\n"
+      "setp.ne.u32 pi, %1, 0;\n"
+      "bar.red.and.pred po, %2, %3, pi;\n"
+      "selp.u32 %0, 1, 0, po;\n"
+      "}\n"
+      : "=r"(all)
+      : "r"(ok), "r"(id), "r"(n)
+      : "memory");
+  return all != 0;
+}
+__device__ __forceinline__ bool t_wait_role(bool leader, uint32_t bar, uint32_t parity, int id, int n, volatile int* abort_flag) {
+  bool ok = true;
+  if (leader) ok = t_wait(bar, parity, abort_flag);
+  return t_role_sync(id, n, ok);
 }
 __device__ __forceinline__ void t_sts128(uint32_t a, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
   asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(a), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
-}
-__device__ __forceinline__ uint32_t t_lop_ao(uint32_t x, uint32_t mask, uint32_t orv) {
-  uint32_t r;
-  asm("lop3.b32 %0, %1, %2, %3, 0xEA;\n" : "=r"(r) : "r"(x), "r"(mask), "r"(orv));
-  return r;
 }
 __device__ __forceinline__ uint32_t t_prmt(uint32_t a, uint32_t b, uint32_t sel) {
   uint32_t r;
@@ -223,7 +252,7 @@ struct TcTile {
 };
 
 // `e` is the caller's copy of table[it] (it fetches the next one while a tile is being worked on).
-__device__ __noinline__ bool tc_next(const MlaDecodeParams& p, const TableEntry* table, int item_end, int it, const TableEntry e,
+__device__ __forceinline__ bool tc_next(const MlaDecodeParams& p, const TableEntry* table, int item_end, int it, const TableEntry e,
                                      TcTile& t) {
   if (it >= item_end) return false;
   t.item = it;
@@ -277,32 +306,47 @@ __device__ __forceinline__ uint32_t tc_tile_addr(uint32_t tile, int row, int j) 
 __device__ __forceinline__ uint32_t tc_bf2_to_h2(uint32_t u) {
   return t_u(__floats2half2_rn(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)));
 }
-__device__ __forceinline__ uint4 t_ldg128(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+// Streaming loads bypass L1: what little of it the shared-memory carve-out leaves is kept for the
+// threads' stack slots.
+__device__ __forceinline__ uint4 t_ldg128(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint2 t_ldg64(const void* p) {
+  uint2 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint32_t t_ldg32(const void* p) {
+  uint32_t v;
+  asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];\n" : "=r"(v) : "l"(p));
+  return v;
+}
 
-// centre of the code range that the tile subtracts (an integer, so that the tile holds integers)
-__device__ __forceinline__ float tc_mid(int level) { return level == 8 ? 128.f : 8.f; }
+// A code in the mantissa of an fp16 with a zero exponent field is the number code * 2^(b - 24), b the
+// code's lowest bit: no bias to take out again.  8-bit codes sit at b = 0; 4-bit codes at b = 0
+// (channels with (c & 2) == 0) or b = 4.  The logits of a quantised tile therefore come out of the
+// tensor cores scaled by 2^-24 (8 bits) or 2^-20 (4 bits, whose b = 0 channels get 16 s in Q'), and a
+// value channel by 2^(b - 24).
+__device__ __forceinline__ float tc_logit_scale(const int kind, const int level) {
+  return kind != 0 ? 1.f : (level == 8 ? 16777216.f : 1048576.f);
+}
 
-// A quantised block -> the tile as the exact integers code - mid.  Thread = (chunk j of 8 channels, 8
+// A quantised block -> the tile as the codes themselves (scaled by a power of two).  Thread = (chunk j of 8 channels, 8
 // tokens of each half); the packed codes come straight from global memory (a token's chunk is 8
-// bytes at 8 bits, 4 bytes at 4 bits).  The loads are issued early (tc_load_block), while the
-// thread still waits for the tile buffer.
-__device__ __forceinline__ void tc_load_block(const uint8_t* slot, int bits, int j, int tg, uint2 (&w)[2][8]) {
+// bytes at 8 bits, 4 bytes at 4 bits).  The loads are issued a tile ahead (tc_load_half).
+__device__ __forceinline__ void tc_load_half(const uint8_t* slot, int bits, int half, int j, int tg, uint2 (&w)[8]) {
   const int row = kMlaChunks * bits;
+  const uint8_t* codes = slot + static_cast<size_t>(half) * mla_half_bytes(bits) + mla_kp_bytes() + static_cast<size_t>(8 * tg) * row + j * bits;
 #pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    const uint8_t* codes = slot + static_cast<size_t>(half) * mla_half_bytes(bits) + mla_kp_bytes() + static_cast<size_t>(8 * tg) * row + j * bits;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if (bits == 8) w[half][i] = __ldg(reinterpret_cast<const uint2*>(codes + i * row));
-      else w[half][i] = make_uint2(__ldg(reinterpret_cast<const uint32_t*>(codes + i * row)), 0u);
-    }
+  for (int i = 0; i < 8; ++i) {
+    if (bits == 8) w[i] = t_ldg64(codes + i * row);
+    else w[i] = make_uint2(t_ldg32(codes + i * row), 0u);
   }
 }
 template <int BITS>
 __device__ __forceinline__ void tc_store_block(const uint2 (&w)[2][8], uint32_t tile, int j, int tg) {
-  // bias + mid of the two code positions of a word (see gkv_layout.cuh for the positions)
-  const __half2 b0 = __float2half2_rn(BITS == 4 ? 1024.f + 8.f : 1024.f + 128.f);
-  const __half2 b1 = __float2half2_rn(BITS == 4 ? 64.f + 8.f : 1024.f + 128.f);
   const uint32_t jx = (j & 7) << 4;
 #pragma unroll
   for (int half = 0; half < 2; ++half) {
@@ -312,19 +356,18 @@ __device__ __forceinline__ void tc_store_block(const uint2 (&w)[2][8], uint32_t 
       uint32_t x0, x1, x2, x3;
       if constexpr (BITS == 4) {
         const uint32_t v = w[half][i].x >> 8;
-        x0 = t_lop_ao(w[half][i].x, 0x000F000Fu, 0x64006400u);      // 1024 + code (channels 0, 1)
-        x1 = t_lop_ao(w[half][i].x, 0x00F000F0u, 0x54005400u);      // 64 + code   (channels 2, 3)
-        x2 = t_lop_ao(v, 0x000F000Fu, 0x64006400u);
-        x3 = t_lop_ao(v, 0x00F000F0u, 0x54005400u);
+        x0 = w[half][i].x & 0x000F000Fu;      // channels 0, 1: b = 0
+        x1 = w[half][i].x & 0x00F000F0u;      // channels 2, 3: b = 4
+        x2 = v & 0x000F000Fu;
+        x3 = v & 0x00F000F0u;
       } else {
-        x0 = t_prmt(w[half][i].x, 0x64006400u, 0x5250u);
-        x1 = t_prmt(w[half][i].x, 0x64006400u, 0x5351u);
-        x2 = t_prmt(w[half][i].y, 0x64006400u, 0x5250u);
-        x3 = t_prmt(w[half][i].y, 0x64006400u, 0x5351u);
+        x0 = t_prmt(w[half][i].x, 0u, 0x4240u);
+        x1 = t_prmt(w[half][i].x, 0u, 0x4341u);
+        x2 = t_prmt(w[half][i].y, 0u, 0x4240u);
+        x3 = t_prmt(w[half][i].y, 0u, 0x4341u);
       }
       // rows 32 half + 8 tg + i: row & 7 = i, so the swizzled 16-byte slot is (j & 7) ^ i
-      t_sts128(out + i * 128 + (jx ^ (i << 4)), t_u(__hsub2(t_h2(x0), b0)), t_u(__hsub2(t_h2(x1), b1)), t_u(__hsub2(t_h2(x2), b0)),
-               t_u(__hsub2(t_h2(x3), b1)));
+      t_sts128(out + i * 128 + (jx ^ (i << 4)), x0, x1, x2, x3);
     }
   }
 }
@@ -361,9 +404,13 @@ __device__ __forceinline__ void tc_convert_rows(const MlaDecodeParams& p, const 
 // tensor-memory lane lt).  hs = [2 halves][16 heads] sums of the tile's probabilities.
 __device__ __forceinline__ bool tc_read_out(const MlaDecodeParams& p, const TcTile& pt, int pn, int i0, int i1, bool scale,
                                             const float* alpha_sm, const float* hs, uint32_t tlane, int lt, uint32_t bar_pv,
-                                            volatile int* abort_flag) {
+                                            bool leader, int role_bar, volatile int* abort_flag
+#ifdef GKV_MLA_PROF
+                                            , uint32_t* prof_sm
+#endif
+) {
   // scale and zero point of this thread's channels in both halves (asked for before the wait)
-  const float mid = tc_mid(pt.level);
+  const float unscale = (pt.level == 4 && (lt & 2)) ? 1048576.f : 16777216.f;      // 2^(24 - b) of the thread's channels
   const uint8_t* slot = p.arena + static_cast<size_t>(pt.off256) * 256;
   __half sch[4][2], zph[4][2];
   if (pt.kind == 0) {
@@ -378,7 +425,13 @@ __device__ __forceinline__ bool tc_read_out(const MlaDecodeParams& p, const TcTi
       }
     }
   }
-  const bool ok = t_wait_warp(bar_pv, (pn >> 1) & 1, abort_flag);
+#ifdef GKV_MLA_PROF
+  const uint32_t rw0 = clock();
+#endif
+  const bool ok = t_wait_role(leader, bar_pv, (pn >> 1) & 1, role_bar, 128, abort_flag);
+#ifdef GKV_MLA_PROF
+  if (threadIdx.x == 128) prof_sm[20] += clock() - rw0;
+#endif
   t_fence_after();
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -395,17 +448,29 @@ __device__ __forceinline__ bool tc_read_out(const MlaDecodeParams& p, const TcTi
     t_wait_ld();
     if (scale) {
 #pragma unroll
-      for (int h = 0; h < 16; ++h) o[h] *= alpha_sm[h];
+      for (int h4 = 0; h4 < 4; ++h4) {
+        const float4 a = reinterpret_cast<const float4*>(alpha_sm)[h4];
+        o[4 * h4] *= a.x;
+        o[4 * h4 + 1] *= a.y;
+        o[4 * h4 + 2] *= a.z;
+        o[4 * h4 + 3] *= a.w;
+      }
     }
 #pragma unroll
     for (int hf = 0; hf < 2; ++hf) {
       float sc = 1.f, zp = 0.f;
       if (pt.kind == 0) {
-        sc = __half2float(sch[i][hf]);
-        zp = fmaf(mid, sc, __half2float(zph[i][hf]));
+        sc = __half2float(sch[i][hf]) * unscale;
+        zp = __half2float(zph[i][hf]);
       }
 #pragma unroll
-      for (int h = 0; h < 16; ++h) o[h] = fmaf(sc, r[h] + rl[h], fmaf(zp, hs[hf * 16 + h], o[h]));
+      for (int h4 = 0; h4 < 4; ++h4) {
+        const float4 w = reinterpret_cast<const float4*>(hs)[hf * 4 + h4];
+        o[4 * h4] = fmaf(sc, r[4 * h4] + rl[4 * h4], fmaf(zp, w.x, o[4 * h4]));
+        o[4 * h4 + 1] = fmaf(sc, r[4 * h4 + 1] + rl[4 * h4 + 1], fmaf(zp, w.y, o[4 * h4 + 1]));
+        o[4 * h4 + 2] = fmaf(sc, r[4 * h4 + 2] + rl[4 * h4 + 2], fmaf(zp, w.z, o[4 * h4 + 2]));
+        o[4 * h4 + 3] = fmaf(sc, r[4 * h4 + 3] + rl[4 * h4 + 3], fmaf(zp, w.w, o[4 * h4 + 3]));
+      }
       if (hf == 0) {                                    // the second half's accumulators
         t_ld16_async(tlane + kTmemR + 128 + 32 * i, r);
         t_ld16_async(tlane + kTmemR + 128 + 32 * i + 16, rl);
@@ -436,6 +501,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
   float* alpha_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscAlpha);          // [2][16]
   float* hsum2_sm = reinterpret_cast<float*>(gbase + kOffMisc + kMiscHalfSum2);       // [2][2][16]
   volatile int* need_sm = reinterpret_cast<volatile int*>(gbase + kOffMisc + kMiscAlpha + 128);   // [2]
+#ifdef GKV_MLA_PROF
+  uint32_t* prof_sm = reinterpret_cast<uint32_t*>(gbase + kOffMisc + 5120);
+  const bool prof_lane = (lane == 0) && (warp == 0 || warp == 4 || warp == kTcFirstConvertWarp || warp == kTcMmaWarp);
+  if (tid < 32) prof_sm[tid] = 0;
+#endif
   const TableEntry* table = p.table + static_cast<size_t>(cd.stream) * p.table_stride;
   auto bar = [&](int which, int i) { return misc + 8u * static_cast<uint32_t>(which + i); };
 
@@ -471,24 +541,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       const int b = tg & 1;
       const uint64_t da = t_desc(base + kOffTile + b * kTcTileBytes, 16, 1024);
       const uint32_t d = tmem + kTmemS + 64 * b;
+      // (the loops stay rolled: the issue warp's code competes with the working warps for the instruction cache)
+#pragma unroll 1
+      for (int pn = 0; pn < 9; ++pn) {
+        const uint32_t o16 = static_cast<uint32_t>(pn * kTcPanelBytes) >> 4;
 #pragma unroll
-      for (int pn = 0; pn < 9; ++pn)
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
-          t_mma_f16(d, da + ((pn * kTcPanelBytes + kk * 32) >> 4), dq + ((pn * kTcPanelBytes + kk * 32) >> 4), kIdQK, (pn | kk) != 0);
+        for (int kk = 0; kk < 4; ++kk) t_mma_f16(d, da + o16 + 2 * kk, dq + o16 + 2 * kk, kIdQK, (pn | kk) != 0);
+      }
       t_commit(bar(kBarSFull, b));
     };
     auto issue_pv = [&](int tg) {
       const int b = tg & 1;
       const uint64_t da = t_desc(base + kOffTile + b * kTcTileBytes, kTcPanelBytes, 1024);
-#pragma unroll
-      for (int half = 0; half < 2; ++half)
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-          for (int kk = 2 * half; kk < 2 * half + 2; ++kk)
-            t_mma_f16(tmem + kTmemR + 128 * half + 32 * i, da + ((2 * i * kTcPanelBytes + kk * 2048) >> 4), dp + ((kk * 512) >> 4), kIdPV,
-                      kk != 2 * half);
+#pragma unroll 1
+      for (int hi = 0; hi < 8; ++hi) {
+        const int half = hi >> 2, i = hi & 3;
+        const uint32_t oa = static_cast<uint32_t>(2 * i * kTcPanelBytes + 2 * half * 2048) >> 4, ob = static_cast<uint32_t>(2 * half * 512) >> 4;
+        const uint32_t d = tmem + kTmemR + 128 * half + 32 * i;
+        t_mma_f16(d, da + oa, dp + ob, kIdPV, 0);
+        t_mma_f16(d, da + oa + (2048 >> 4), dp + ob + (512 >> 4), kIdPV, 1);
+      }
       t_commit(bar(kBarPvDone, b));
     };
     // packed bytes of a tile that is about to be converted: ask for them in L2
@@ -526,13 +598,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     for (int i = 0; i < kPrefetchAhead; ++i) prefetch_step();
     bool ok = true;
     int spins = 0;
+    PROF_DECL(24);
     while (ok && (pv < n_known || more_tiles)) {
       bool progress = false;
       if (qk < n_known && qk < pv + 2) {
         const bool ready = __all_sync(kFullT, t_try_wait(bar(kBarKtFull, qk & 1), (qk >> 1) & 1) && t_try_wait(bar(kBarQpFull, qk & 1), (qk >> 1) & 1));
         if (ready) {
           t_fence_after();
+          PROF_LAP(0);
           issue_qk(qk);
+          PROF_LAP(1);
           ++qk;
           it = t.item + t.adv;
           more_tiles = tc_next(p, table, cd.item_end, it, pre, t);
@@ -548,7 +623,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
         const bool ready = __all_sync(kFullT, t_try_wait(bar(kBarPFull, 0), pv & 1) && (pv == 0 || t_try_wait(bar(kBarRFree, 0), (pv - 1) & 1)));
         if (ready) {
           t_fence_after();
+          PROF_LAP(0);
           issue_pv(pv);
+          PROF_LAP(2);
           ++pv;
           progress = true;
         }
@@ -580,37 +657,42 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       qh[hh][2] = tc_bf2_to_h2(v.z);
       qh[hh][3] = tc_bf2_to_h2(v.w);
     }
-    TcTile t;
-    int it = cd.item_begin, tg = 0;
+    // The packed codes of a tile's quantised block (w) and the scales and zero points of the
+    // thread's Q' chunk (svh, zvh) are asked for one tile ahead: the codes of the next tile as soon as
+    // this tile is stored, its parameters once this tile's Q' is written.
+    TcTile t, tn;
+    int tg = 0;
     bool ok = true;
-    TableEntry pre = tc_entry(p, table, it);
-    while (ok && tc_next(p, table, cd.item_end, it, pre, t)) {
-      pre = tc_entry(p, table, t.item + t.adv);
-      const int b = tg & 1;
-      const uint32_t tile = base + kOffTile + b * kTcTileBytes;
-      const uint8_t* slot = p.arena + static_cast<size_t>(t.off256) * 256;
-      // everything a quantised block needs from global memory is asked for before the wait for the
-      // tile buffer: the packed codes of the thread's part of the tile, the scales and zero points of
-      // its Q' chunk
-      uint2 w[2][8];
-      uint4 svh[2], zvh[2];
+    uint2 w[2][8];
+    uint4 svh[2], zvh[2];
+    auto load_params = [&](const TcTile& x) {
+      const uint8_t* slot = p.arena + static_cast<size_t>(x.off256) * 256;
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
-        svh[half] = make_uint4(0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u);    // scales 1
-        zvh[half] = make_uint4(0, 0, 0, 0);
+        const uint8_t* prm = slot + static_cast<size_t>(half) * mla_half_bytes(x.level);
+        svh[half] = t_ldg128(prm + 16 * qj);
+        zvh[half] = t_ldg128(prm + 2 * kMlaZeroOff + 16 * qj);
       }
-      if (t.kind == 0) {
-        tc_load_block(slot, t.level, dj, dg, w);
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const uint8_t* prm = slot + static_cast<size_t>(half) * mla_half_bytes(t.level);
-          svh[half] = t_ldg128(prm + 16 * qj);
-          zvh[half] = t_ldg128(prm + 2 * kMlaZeroOff + 16 * qj);
-        }
-      }
+    };
+    TableEntry pre = tc_entry(p, table, cd.item_begin);
+    bool have = tc_next(p, table, cd.item_end, cd.item_begin, pre, t);
+    if (have && t.kind == 0) {
+      tc_load_half(p.arena + static_cast<size_t>(t.off256) * 256, t.level, 0, dj, dg, w[0]);
+      tc_load_half(p.arena + static_cast<size_t>(t.off256) * 256, t.level, 1, dj, dg, w[1]);
+      load_params(t);
+    }
+    if (have) pre = tc_entry(p, table, t.item + t.adv);
+    PROF_DECL(0);
+    while (ok && have) {
+      const int b = tg & 1;
+      const uint32_t tile = base + kOffTile + b * kTcTileBytes;
+      const bool have_n = tc_next(p, table, cd.item_end, t.item + t.adv, pre, tn);
+      if (have_n) pre = tc_entry(p, table, tn.item + tn.adv);
+      PROF_LAP(0);
       // the tile buffer is free once the value MMAs of tile tg - 2 are done
-      if (tg >= 2) ok = t_wait_warp(bar(kBarPvDone, b), ((tg - 2) >> 1) & 1, abort_flag);
+      if (tg >= 2) ok = t_wait_role(cw == 0, bar(kBarPvDone, b), ((tg - 2) >> 1) & 1, 2, kTcConvertWarps * 32, abort_flag);
       if (!ok) break;
+      PROF_LAP(1);
       if (dt < 64) bias_sm[b * 64 + dt] = dt < t.nrows ? (t.kind == 2 ? 6.0f : 0.f) : kNegInfT;   // log2(64) per centroid row
       if (t.kind == 0) {
         if (t.level == 8) tc_store_block<8>(w, tile, dj, dg);
@@ -620,47 +702,60 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       } else {
         tc_convert_rows<true>(p, table, t, tile, dj, dg);
       }
+      PROF_LAP(2);
       t_fence_async();
       __syncwarp();
       if (lane == 0) t_bar_arrive(bar(kBarKtFull, b));
-      // Q' of this tile.  The key constants sum_c q[c] (z[c] + mid s[c]) are formed before the wait:
-      // only the stores need the Q' buffer, which is free once the key MMAs of tile tg - 1 are done.
-      const float mid = tc_mid(t.level);
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        float cacc[4] = {0.f, 0.f, 0.f, 0.f};
+      PROF_LAP(3);
+      // Key constants sum_c q[c] z[c] per (half, head): this thread's chunk, then the warp's eight chunks
+      // (lanes with the same head quad) in a fixed order.  Formed before the wait for the Q' buffer.
+      {
+        float cacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
         if (t.kind == 0) {
-          const uint32_t sw[4] = {svh[half].x, svh[half].y, svh[half].z, svh[half].w};
-          const uint32_t zw[4] = {zvh[half].x, zvh[half].y, zvh[half].z, zvh[half].w};
+          const uint32_t zw[2][4] = {{zvh[0].x, zvh[0].y, zvh[0].z, zvh[0].w}, {zvh[1].x, zvh[1].y, zvh[1].z, zvh[1].w}};
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const float2 sf = __half22float2(t_h2(sw[i])), zf = __half22float2(t_h2(zw[i]));
-            const float z0 = fmaf(mid, sf.x, zf.x), z1 = fmaf(mid, sf.y, zf.y);
+            const float2 za = __half22float2(t_h2(zw[0][i])), zb = __half22float2(t_h2(zw[1][i]));
 #pragma unroll
             for (int hh = 0; hh < 4; ++hh) {
               const float2 qf = __half22float2(t_h2(qh[hh][i]));
-              cacc[hh] = fmaf(qf.x, z0, cacc[hh]);
-              cacc[hh] = fmaf(qf.y, z1, cacc[hh]);
+              cacc[0][hh] = fmaf(qf.y, za.y, fmaf(qf.x, za.x, cacc[0][hh]));
+              cacc[1][hh] = fmaf(qf.y, zb.y, fmaf(qf.x, zb.x, cacc[1][hh]));
             }
           }
-          // the warp's part: add the 8 chunks of the warp (lanes with the same head quad), fixed order
 #pragma unroll
-          for (int hh = 0; hh < 4; ++hh) {
+          for (int d = 4; d <= 16; d <<= 1) {
 #pragma unroll
-            for (int d = 4; d <= 16; d <<= 1) cacc[hh] += __shfl_xor_sync(kFullT, cacc[hh], d);
+            for (int hh = 0; hh < 4; ++hh) {
+              cacc[0][hh] += __shfl_xor_sync(kFullT, cacc[0][hh], d);
+              cacc[1][hh] += __shfl_xor_sync(kFullT, cacc[1][hh], d);
+            }
           }
         }
         if (lane < 4) {
-          float* dst = cpart_sm + ((b * 2 + half) * kTcConvertWarps + cw) * 16 + 4 * lane;
-          dst[0] = cacc[0]; dst[1] = cacc[1]; dst[2] = cacc[2]; dst[3] = cacc[3];
+#pragma unroll
+          for (int half = 0; half < 2; ++half)
+            *reinterpret_cast<float4*>(cpart_sm + ((b * 2 + half) * kTcConvertWarps + cw) * 16 + 4 * lane) =
+                make_float4(cacc[half][0], cacc[half][1], cacc[half][2], cacc[half][3]);
         }
       }
-      if (tg >= 1) ok = t_wait_warp(bar(kBarSFull, (tg - 1) & 1), ((tg - 1) >> 1) & 1, abort_flag);
+      // the next tile's codes: the first half block now, the second once this tile's Q' is written (the
+      // registers they need are free by then)
+      if (have_n && tn.kind == 0) tc_load_half(p.arena + static_cast<size_t>(tn.off256) * 256, tn.level, 0, dj, dg, w[0]);
+      PROF_LAP(4);
+      // the Q' buffer is free once the key MMAs of tile tg - 1 are done
+      if (tg >= 1) ok = t_wait_role(cw == 0, bar(kBarSFull, (tg - 1) & 1), ((tg - 1) >> 1) & 1, 2, kTcConvertWarps * 32, abort_flag);
       if (!ok) break;
+      PROF_LAP(5);
       const uint32_t qp = base + kOffQp;
+      const bool quant = t.kind == 0;
+      const __half2 f16 = __float2half2_rn((quant && t.level == 4) ? 16.f : 1.f);     // the b = 0 channel pairs of a 4-bit chunk
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
-        const uint32_t sw[4] = {svh[half].x, svh[half].y, svh[half].z, svh[half].w};
+        uint32_t sw[4] = {svh[half].x, svh[half].y, svh[half].z, svh[half].w};
+        if (!quant) sw[0] = sw[1] = sw[2] = sw[3] = 0x3C003C00u;                      // exact and centroid rows: scale 1
+        sw[0] = t_u(__hmul2(t_h2(sw[0]), f16));
+        sw[2] = t_u(__hmul2(t_h2(sw[2]), f16));
 #pragma unroll
         for (int hh = 0; hh < 4; ++hh) {
           uint32_t hi[4], lo[4];
@@ -677,9 +772,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       }
       t_fence_async();
       __syncwarp();
+      PROF_LAP(6);
       if (lane == 0) t_bar_arrive(bar(kBarQpFull, b));
-      it = t.item + t.adv;
+      if (have_n && tn.kind == 0) {
+        tc_load_half(p.arena + static_cast<size_t>(tn.off256) * 256, tn.level, 1, dj, dg, w[1]);
+        load_params(tn);
+      }
+      t = tn;
+      have = have_n;
       ++tg;
+      PROF_LAP(7);
     }
   } else if (warp >= 4) {
     // ---------------- read-out of the channel tiles [kTcReadTiles0, 4) (warps 4-7) ----------------
@@ -689,16 +791,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     int it = cd.item_begin, ts = 0;
     bool ok = true;
     TableEntry pre = tc_entry(p, table, it);
+    PROF_DECL(16);
     while (ok && tc_next(p, table, cd.item_end, it, pre, t)) {
       pre = tc_entry(p, table, t.item + t.adv);
+      PROF_LAP(0);
       // what the softmax of tile ts published: the sums of its probabilities and whether it moved the running max
-      ok = t_wait_warp(bar(kBarHsFull, ts & 1), (ts >> 1) & 1, abort_flag) && ok;
+      ok = t_wait_role(warp == 4, bar(kBarHsFull, ts & 1), (ts >> 1) & 1, 3, 128, abort_flag) && ok;
+      PROF_LAP(1);
       ok = tc_read_out(p, t, ts, kTcReadTiles0, 4, need_sm[ts & 1] != 0, alpha_sm + (ts & 1) * 16, hsum2_sm + (ts & 1) * 32, tlane, lt,
-                       bar(kBarPvDone, ts & 1), abort_flag) && ok;
+                       bar(kBarPvDone, ts & 1), warp == 4, 3, abort_flag
+#ifdef GKV_MLA_PROF
+                       , prof_sm
+#endif
+                       ) && ok;
       __syncwarp();
       if (lane == 0) t_bar_arrive(bar(kBarRFree, 0));
       it = t.item + t.adv;
       ++ts;
+      PROF_LAP(2);
     }
   } else {
     // ---------------- softmax, read-out of the first channel tiles (warps 0-3) and the result ----------------
@@ -714,34 +824,43 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     TcTile t;
     int it = cd.item_begin, ts = 0, xph = 0;                // xph: exchanges done so far (phase of the exchange buffers)
     TableEntry pre = tc_entry(p, table, it);
+    PROF_DECL(8);
     while (tc_next(p, table, cd.item_end, it, pre, t)) {
       pre = tc_entry(p, table, t.item + t.adv);
       const int b = ts & 1;
-      ok = t_wait_warp(bar(kBarQpFull, b), (ts >> 1) & 1, abort_flag) && ok;   // the parts of the key constants are written
-      // key constants of the tile: (half, head) = thread 0..31 adds the nine parts in a fixed order
-      if (tid < 32) {
-        const float* cp = cpart_sm + ((b * 2 + (tid >> 4)) * kTcConvertWarps) * 16 + (tid & 15);
-        float c = 0.f;
+      PROF_LAP(0);
+      {
+        // warp 0 waits for the parts of the key constants (written before Q' is published), adds the
+        // nine parts per (half, head) in a fixed order, then waits for the logits; the role barrier
+        // releases the other three warps and publishes the constants to them
+        bool okl = true;
+        if (warp == 0) {
+          okl = t_wait(bar(kBarQpFull, b), (ts >> 1) & 1, abort_flag);
+          const float* cp = cpart_sm + ((b * 2 + (tid >> 4)) * kTcConvertWarps) * 16 + (tid & 15);
+          float c = 0.f;
 #pragma unroll
-        for (int w9 = 0; w9 < kTcConvertWarps; ++w9) c += cp[w9 * 16];
-        const_sm[b * 32 + tid] = t.kind == 0 ? c : 0.f;
+          for (int w9 = 0; w9 < kTcConvertWarps; ++w9) c += cp[w9 * 16];
+          const_sm[b * 32 + tid] = t.kind == 0 ? c : 0.f;
+          okl = t_wait(bar(kBarSFull, b), (ts >> 1) & 1, abort_flag) && okl;
+        }
+        ok = t_role_sync(1, 128, okl) && ok;
       }
-      ok = t_wait_warp(bar(kBarSFull, b), (ts >> 1) & 1, abort_flag) && ok;
+      PROF_LAP(1);
       t_fence_after();
       float s[16], sl[16];
       t_ld16_async(tlane + kTmemS + 64 * b + 32 * half, s);
       t_ld16_async(tlane + kTmemS + 64 * b + 32 * half + 16, sl);
       t_wait_ld();
-      asm volatile("bar.sync 1, 128;\n" ::: "memory");                    // const_sm is complete
       const int row = 16 * warp + (lane & 15);
       const float bs = (lane < 16) ? bias_sm[b * 64 + row] : kNegInfT;
+      const float ks = tc_logit_scale(t.kind, t.level);
       // Common case: no logit of the tile exceeds its head's running max by more than the slack;
       // then the (stale) max stays and nothing is reduced.  The four warps agree through one flag
       // exchange; only when a flag is up are the head maxima reduced and the sums rescaled.
       bool mine = false;
 #pragma unroll
       for (int h = 0; h < 16; ++h) {
-        s[h] = (bs == kNegInfT) ? kNegInfT : fmaf(s[h] + sl[h] + const_sm[b * 32 + half * 16 + h], p.scale_log2, bs);
+        s[h] = (bs == kNegInfT) ? kNegInfT : fmaf(fmaf(s[h] + sl[h], ks, const_sm[b * 32 + half * 16 + h]), p.scale_log2, bs);
         mine |= s[h] > m_run[h] + kRescaleSlack;            // also true for the first finite logit (max = -inf)
       }
       uint32_t need_u;
@@ -791,7 +910,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
         l_part[h] += pr[h];
       }
       // the P buffer is free once the value MMAs of the tile before are done
-      if (ts > 0) ok = t_wait_warp(bar(kBarPvDone, (ts - 1) & 1), ((ts - 1) >> 1) & 1, abort_flag) && ok;
+      PROF_LAP(2);
+      if (ts > 0) ok = t_wait_role(warp == 0, bar(kBarPvDone, (ts - 1) & 1), ((ts - 1) >> 1) & 1, 1, 128, abort_flag) && ok;
+      PROF_LAP(3);
       if (lane < 16) {
         uint32_t pk[8], pl[8];
 #pragma unroll
@@ -832,13 +953,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       if (lane == 0) t_bar_arrive(bar(kBarHsFull, b));
       if (kTcReadTiles0 > 0) {
         asm volatile("bar.sync 1, 128;\n" ::: "memory");                  // the sums are complete
-        ok = tc_read_out(p, t, ts, 0, kTcReadTiles0, need, alpha_sm + b * 16, hsum2_sm + b * 32, tlane, tid, bar(kBarPvDone, b), abort_flag) && ok;
+        ok = tc_read_out(p, t, ts, 0, kTcReadTiles0, need, alpha_sm + b * 16, hsum2_sm + b * 32, tlane, tid, bar(kBarPvDone, b), warp == 0, 1, abort_flag
+#ifdef GKV_MLA_PROF
+                       , prof_sm
+#endif
+                       ) && ok;
         __syncwarp();
         if (lane == 0) t_bar_arrive(bar(kBarRFree, 0));
       }
       it = t.item + t.adv;
       ++ts;
+      PROF_LAP(4);
     }
+#ifdef GKV_MLA_PROF
+    if (tid == 0) prof_sm[13] += ts;
+#endif
     // ---------------- result ----------------
     float* out = p.partial + static_cast<size_t>(cd.partial) * kMlaPartialFloats;
 #pragma unroll
@@ -883,6 +1012,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
   }
   t_fence_before();
   __syncthreads();
+#ifdef GKV_MLA_PROF
+  if (tid < 32) g_prof[blockIdx.x * 32 + tid] += prof_sm[tid];
+#endif
   if (tid == 0 && *abort_flag) atomicOr(p.status, kStatusInternal);
   if (warp == 0) t_tmem_dealloc(tmem, kTmemCols);
 }
@@ -963,3 +1095,14 @@ cudaError_t launch_mla_decode(const MlaDecodeParams& p, int n_ctas, const Stream
 }
 
 }  // namespace gkv
+
+#ifdef GKV_MLA_PROF
+extern "C" __attribute__((visibility("default"))) void gkv_x_prof_read(unsigned long long* buf, int reset) {
+  if (reset) {
+    static unsigned long long z[148 * 32];
+    cudaMemcpyToSymbol(gkv::g_prof, z, sizeof(z));
+  } else {
+    cudaMemcpyFromSymbol(buf, gkv::g_prof, sizeof(unsigned long long) * 148 * 32);
+  }
+}
+#endif
