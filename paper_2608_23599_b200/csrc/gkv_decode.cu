@@ -178,6 +178,56 @@ __device__ __forceinline__ void unpack(const uint32_t* w, int s_local, uint32_t 
   }
 }
 
+// Value codes need no bias: with a zero exponent field the fp16 number is code * 2^(p - 24), p the
+// code's lowest mantissa bit, and the value MMAs accumulate V^T P' directly (no correction MMA, no
+// cancellation in the accumulators).  The fields of a word are arranged (gkv_layout.cuh) so that p depends
+// on the token half only: registers 0, 1 (tokens 0-7 of the tile) at p_lo, registers 2, 3 (tokens 8-15) at
+// p_hi = 6; P' of the first half is multiplied by 2^(p_hi - p_lo) (VScale::lo), 8-bit codes (p = 0
+// everywhere) by 2^6 in both halves, so that every product carries the common factor 2^-18, which the
+// exact rows put into P and the final row takes out again.
+template <int BITS>
+struct VScale;
+template <>
+struct VScale<8> {
+  static constexpr float lo = 64.f, hi = 64.f;
+};
+template <>
+struct VScale<4> {
+  static constexpr float lo = 16.f, hi = 1.f;
+};
+template <>
+struct VScale<2> {
+  static constexpr float lo = 4.f, hi = 1.f;
+};
+constexpr float kVUnit = 1.f / 262144.f;          // 2^-18: weight of a value product in the accumulators
+constexpr float kVUnitInv = 262144.f;
+
+template <int BITS>
+__device__ __forceinline__ void unpack_v(const uint32_t* w, int s_local, uint32_t (&a)[4]) {
+  if constexpr (BITS == 8) {
+    const uint32_t w0 = w[2 * s_local], w1 = w[2 * s_local + 1];
+    a[0] = prmt(w0, 0u, 0x4240u);
+    a[1] = prmt(w0, 0u, 0x4341u);
+    a[2] = prmt(w1, 0u, 0x4240u);
+    a[3] = prmt(w1, 0u, 0x4341u);
+  } else if constexpr (BITS == 4) {
+    // fields at bits 0, 4 (registers 0, 2) and 8, 12 (registers 1, 3) of each 16-bit half -> bits 2 and 6
+    const uint32_t v0 = w[s_local] << 2, v1 = w[s_local] >> 6;
+    a[0] = v0 & 0x003C003Cu;
+    a[2] = v0 & 0x03C003C0u;
+    a[1] = v1 & 0x003C003Cu;
+    a[3] = v1 & 0x03C003C0u;
+  } else {
+    // even s: fields at bits 0, 2 (registers 0, 2) and 8, 10 (registers 1, 3); odd s: 4 further -> bits 4 and 6
+    const uint32_t x = w[s_local >> 1];
+    const uint32_t v0 = (s_local & 1) ? x : (x << 4), v1 = (s_local & 1) ? (x >> 8) : (x >> 4);
+    a[0] = v0 & 0x00300030u;
+    a[2] = v0 & 0x00C000C0u;
+    a[1] = v1 & 0x00300030u;
+    a[3] = v1 & 0x00C000C0u;
+  }
+}
+
 __device__ __forceinline__ float fast_exp2(float x);
 
 // Lane (r, c4) = (lane / 4, lane % 4).  Accumulator side: the lane owns head c4 of the warp's head
@@ -245,11 +295,13 @@ __device__ __forceinline__ void make_p_f16(float pa, float pb, uint32_t (&pf)[2]
   pf[0] = movmatrix_trans(prmt(h2_as_u32(hh), h2_as_u32(ll), 0x5410u));    // (hi, lo) of row r
   pf[1] = movmatrix_trans(prmt(h2_as_u32(hh), h2_as_u32(ll), 0x7632u));    // (hi, lo) of row r + 8
 }
-// The same with bf16 parts (p = hi + lo to ~2^-17) for the exact rows.
+// The same with bf16 parts (p = hi + lo to ~2^-17) for the exact rows, in the accumulators' unit 2^-18.
 __device__ __forceinline__ void make_p_bf16(float pa, float pb, uint32_t (&pf)[2], SoftmaxState& st) {
+  st.l += pa + pb;
+  pa *= kVUnit;
+  pb *= kVUnit;
   const uint32_t hh = pack_bf16x2(pa, pb);
   const uint32_t ll = pack_bf16x2(pa - bf16lo_to_f32(hh), pb - bf16hi_to_f32(hh));
-  st.l += pa + pb;
   pf[0] = movmatrix_trans(prmt(hh, ll, 0x5410u));
   pf[1] = movmatrix_trans(prmt(hh, ll, 0x7632u));
 }
@@ -723,8 +775,8 @@ __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, int tm, uint3
 
 // O^T += V~^T P^T for the active tiles of one half, v~ = s * code + z per (token, 32-channel group).
 // pf holds the fp16 P^T fragments of the two tiles (hi / lo columns); tile t has its parameters at
-// vp + 256 t and its codes at vc + 256 BITS t.  Data MMAs accumulate (bias + code) * P' straight into
-// O, and an MMA whose A operand is the constant -(bias + mid) takes bias and code centre out again.
+// vp + 256 t and its codes at vc + 256 BITS t.  The data MMAs accumulate code * P' (bias-free codes,
+// see unpack_v) straight into O; the zero points go through one MMA per tile into zc.
 // The loop over the two tiles is kept rolled (see qk_half).
 template <int BITS, bool FULL>
 __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const uint32_t (&pf)[2][2], int lane,
@@ -732,17 +784,8 @@ __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const 
   constexpr int cb = 256 * BITS;
   const int c4 = lane & 3, r = lane >> 2;
   const bool lo_lane = lo_part_lane(lane);
-  float tz[4] = {0.f, 0.f, 0.f, 0.f};   // rows g < 4: sum_tok p z[tok][g]; rows 8 + g: sum_tok p s[tok][g]
-  // A operand that removes bias + centre: rows r (registers 0, 2) and rows r + 8 (registers 1, 3).
-  // Produced by opaque moves so that the compiler keeps one register quad for the whole half
-  // instead of rebuilding it per MMA.
-  uint32_t fix[4];
-  {
-    const uint32_t f_lo = h2_as_u32(__float2half2_rn(-(Bias<BITS>::lo + Bias<BITS>::mid)));
-    const uint32_t f_hi = h2_as_u32(__float2half2_rn(-(Bias<BITS>::hi + Bias<BITS>::mid)));
-#pragma unroll
-    for (int i = 0; i < 4; ++i) asm volatile("mov.b32 %0, %1;\n" : "=r"(fix[i]) : "r"((i & 1) ? f_hi : f_lo));
-  }
+  float tz[4] = {0.f, 0.f, 0.f, 0.f};   // rows g < 4: sum_tok p z[tok][g] (rows 8 + g: sum_tok p s[tok][g], not used)
+  const __half2 f_lo = __float2half2_rn(VScale<BITS>::lo), f_hi = __float2half2_rn(VScale<BITS>::hi);
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
     if (!FULL && !((tm >> t) & 1)) continue;
@@ -761,9 +804,12 @@ __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const 
     const uint32_t sc[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
+      // the scales in the accumulators' unit: tokens 0-7 (sA) and 8-15 (sB) of the tile
+      const uint32_t sa = h2_as_u32(__hmul2(u32_as_h2(sc[2 * g]), f_lo));
+      const uint32_t sb = VScale<BITS>::hi == 1.f ? sc[2 * g + 1] : h2_as_u32(__hmul2(u32_as_h2(sc[2 * g + 1]), f_hi));
       uint32_t p0, p1, p0l, p1l;
-      hmul2_split(h0, m0, sc[2 * g], p0, p0l);        // (m0, m1 are the lo parts where p0l, p1l are used)
-      hmul2_split(h1, m1, sc[2 * g + 1], p1, p1l);
+      hmul2_split(h0, m0, sa, p0, p0l);        // (m0, m1 are the lo parts where p0l, p1l are used)
+      hmul2_split(h1, m1, sb, p1, p1l);
       if (lo_lane) {
         p0 = p0l;
         p1 = p1l;
@@ -771,15 +817,13 @@ __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const 
       uint32_t wd[BITS / 2];
       uint32_t a[4];
       load_words<BITS>(vct, g, lane, wd);
-      unpack<BITS>(wd, 0, a);
+      unpack_v<BITS>(wd, 0, a);
       mma_f16(st.o[2 * g], a[0], a[1], a[2], a[3], p0, p1);
-      mma_f16(st.o[2 * g], fix[0], fix[1], fix[2], fix[3], p0, p1);
-      unpack<BITS>(wd, 1, a);
+      unpack_v<BITS>(wd, 1, a);
       mma_f16(st.o[2 * g + 1], a[0], a[1], a[2], a[3], p0, p1);
-      mma_f16(st.o[2 * g + 1], fix[0], fix[1], fix[2], fix[3], p0, p1);
     }
   }
-  st.zc += fmaf(Bias<BITS>::mid, tz[2] + tz[3], tz[0] + tz[1]);
+  st.zc += tz[0] + tz[1];
 }
 
 template <int BITS, bool FULL>
@@ -1098,8 +1142,8 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
     const float z = __shfl_sync(kFull, st.zc, 4 * (u >> 1) + c4);
-    out[2 + 16 * u + r] = st.o[u][0] + st.o[u][1] + z;
-    out[2 + 16 * u + 8 + r] = st.o[u][2] + st.o[u][3] + z;
+    out[2 + 16 * u + r] = fmaf(st.o[u][0] + st.o[u][1], kVUnitInv, z);
+    out[2 + 16 * u + 8 + r] = fmaf(st.o[u][2] + st.o[u][3], kVUnitInv, z);
   }
   }   // hgroup >= 0
 

@@ -93,10 +93,15 @@ __device__ __forceinline__ GroupParams i_params(float mn, float mx) {
   return g;
 }
 
-// bit position of code (slice s, register a, half hlf) inside its 32-bit word
+// bit position of code (slice s, register a, half hlf) inside its 32-bit word (value codes: the fields
+// of registers 1 and 2 change places, see gkv_layout.cuh)
 template <int BITS>
 __device__ __forceinline__ constexpr int i_bit(int s, int a, int hlf) {
   return BITS == 8 ? 8 * (a & 1) + 16 * hlf : (BITS == 4 ? 4 * a + 16 * hlf : 4 * (s & 1) + 2 * (a & 1) + 8 * (a >> 1) + 16 * hlf);
+}
+template <int BITS>
+__device__ __forceinline__ constexpr int i_bit_v(int s, int a, int hlf) {
+  return i_bit<BITS>(s, BITS == 8 ? a : ((a >> 1) | ((a & 1) << 1)), hlf);
 }
 
 // Quantise the two values of a register (low half: params 0, high half: params 1), add the codes to
@@ -276,7 +281,7 @@ __device__ __forceinline__ bool ingest_values(uint32_t ld, uint8_t* vp, uint8_t*
 #pragma unroll
         for (int al = 0; al < 2; ++al) {
           const uint32_t xv = x[ss][2 * ah + al];
-          i_quant2<BITS>(xv, s0, z0, v0, s1, z1, v1, i_bit<BITS>(ss, 2 * ah + al, 0), i_bit<BITS>(ss, 2 * ah + al, 1), w[wi],
+          i_quant2<BITS>(xv, s0, z0, v0, s1, z1, v1, i_bit_v<BITS>(ss, 2 * ah + al, 0), i_bit_v<BITS>(ss, 2 * ah + al, 1), w[wi],
                          ah == 0 ? e0 : e2, ah == 0 ? e1 : e3);
           const float x0f = i_lo(xv), x1f = i_hi(xv);
           if (ah == 0) {

@@ -28,7 +28,11 @@
 //   2-bit: word = s >> 1;         pair at bit 4 (s & 1) + 2 (a & 1) + 8 (a >> 1)
 //                                 bias 256 / 64 (s even, a even / odd), 16 / 4 (s odd)
 // so that within one MMA the bias depends only on the A-row half (a & 1) and can be removed after
-// the MMA with one extra "ones" MMA.  Word w of a lane lives at byte ((w/4)*32 + lane)*16 + (w%4)*4
+// the MMA.  Value codes (V role) swap the fields of registers 1 and 2 (field f = (a >> 1) | ((a & 1) << 1)
+// takes the place of a in the 4-bit and 2-bit positions): the kernel reads them as the bias-free
+// numbers code * 2^(p - 24) (a code in the mantissa of an fp16 with a zero exponent field), whose
+// weight then depends only on the token half a >> 1 and is evened out in the probabilities.
+// Word w of a lane lives at byte ((w/4)*32 + lane)*16 + (w%4)*4
 // of the tile's code region (chunk-major: 512 contiguous bytes per warp-wide 16-byte load).
 #pragma once
 #include <stdint.h>
@@ -63,17 +67,19 @@ GKV_HD int off_vc(int bits, int t) { return 1024 + (2 + t) * code_bytes_per_tile
 
 // Where code (lane, s, a, hlf) of a tile sits: byte offset of its 32-bit word inside the tile's
 // code region, and the bit position inside the word.
-GKV_HD void code_pos(int bits, int lane, int s, int a, int hlf, int* byte_off, int* bit) {
+GKV_HD int code_field(bool is_v, int a) { return is_v ? ((a >> 1) | ((a & 1) << 1)) : a; }
+GKV_HD void code_pos(int bits, bool is_v, int lane, int s, int a, int hlf, int* byte_off, int* bit) {
   int w, b;
   if (bits == 8) {
     w = 2 * s + (a >> 1);
     b = 8 * (a & 1);
   } else if (bits == 4) {
     w = s;
-    b = 4 * a;
+    b = 4 * code_field(is_v, a);
   } else {
+    const int f = code_field(is_v, a);
     w = s >> 1;
-    b = 4 * (s & 1) + 2 * (a & 1) + 8 * (a >> 1);
+    b = 4 * (s & 1) + 2 * (f & 1) + 8 * (f >> 1);
   }
   *byte_off = ((w >> 2) * 32 + lane) * 16 + (w & 3) * 4;
   *bit = b + 16 * hlf;

@@ -37,7 +37,7 @@ __device__ __forceinline__ int read_code(const uint8_t* slot, int bits, bool is_
   if (is_v) v_coord(tok, ch, &tile, &lane, &s, &a, &hlf);
   else k_coord(tok, ch, &tile, &lane, &s, &a, &hlf);
   int boff, bit;
-  code_pos(bits, lane, s, a, hlf, &boff, &bit);
+  code_pos(bits, is_v, lane, s, a, hlf, &boff, &bit);
   const int half = tile >> 1, t = tile & 1;
   const uint8_t* region = slot + half * half_bytes(bits) + (is_v ? off_vc(bits, t) : off_kc(bits, t));
   const uint32_t w = *reinterpret_cast<const uint32_t*>(region + boff);
@@ -131,7 +131,7 @@ __device__ void pack_codes(uint8_t* slot, const uint8_t* codes, int bits, bool i
         hlf = q >> 3;
       }
       int boff, bit;
-      code_pos(bits, lane, s, a, hlf, &boff, &bit);
+      code_pos(bits, is_v, lane, s, a, hlf, &boff, &bit);
       int tok, ch;
       if (!is_v) {
         tok = 16 * tile + r + 8 * (a & 1);
