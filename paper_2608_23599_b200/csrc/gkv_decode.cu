@@ -1218,15 +1218,21 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
       if (begin >= 0) {
         __threadfence();
         const int b = sid_stream / p.n_kv_heads, kvh = sid_stream - b * p.n_kv_heads;
-        // a thread takes two neighbouring channels of a head
-#pragma unroll 1
-        for (int e = threadIdx.x; e < n_heads * (kD / 2); e += kDecodeWarps * 32) {
-          const int h = e / (kD / 2), ch = 2 * (e - h * (kD / 2));
+        // a thread takes two neighbouring channels of a head and one half of the rows; the second half's
+        // aggregate joins the first's through shared memory (warp 0's stage memory behind its row), so
+        // the order of summation stays fixed whichever CTA does it
+        float4* s_half = reinterpret_cast<float4*>(smem + 5120);
+        const int e = threadIdx.x & 255, part = threadIdx.x >> 8;
+        const int n = end - begin, n0 = (n + 1) >> 1;
+        const bool on = e < n_heads * (kD / 2);
+        const int h = e / (kD / 2), ch = 2 * (e - h * (kD / 2));
+        float M = kNegInf, L = 0.f, acc0 = 0.f, acc1 = 0.f;
+        if (on) {
+          const int i0 = part ? n0 : 0, i1 = part ? n : n0;
           const float* col = p.partial + static_cast<size_t>(begin) * kPartialFloats + h * (kD + 2);
-          // one pass in row order (one round of independent loads instead of two dependent ones)
-          float M = kNegInf, L = 0.f, acc0 = 0.f, acc1 = 0.f;
-#pragma unroll 4
-          for (int i = 0; i < end - begin; ++i) {
+          // one pass in row order (rounds of independent loads; only the short rescaling chain is serial)
+#pragma unroll 8
+          for (int i = i0; i < i1; ++i) {
             const float* row = col + static_cast<size_t>(i) * kPartialFloats;
             const float2 ml = __ldcg(reinterpret_cast<const float2*>(row));
             const float2 v = __ldcg(reinterpret_cast<const float2*>(row + 2 + ch));
@@ -1237,6 +1243,17 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, kDecodeCtasPerSm) decode_ke
             acc1 = fmaf(acc1, a, v.y * bwt);
             M = Mn;
           }
+          if (part) s_half[e] = make_float4(M, L, acc0, acc1);
+        }
+        __syncthreads();
+        if (on && part == 0) {
+          const float4 o2 = s_half[e];
+          const float Mn = fmaxf(M, o2.x);
+          const float a = (M == kNegInf) ? 0.f : exp2f(M - Mn), bwt = (o2.x == kNegInf) ? 0.f : exp2f(o2.x - Mn);
+          L = fmaf(L, a, o2.y * bwt);
+          acc0 = fmaf(acc0, a, o2.z * bwt);
+          acc1 = fmaf(acc1, a, o2.w * bwt);
+          M = Mn;
           const size_t hq = static_cast<size_t>(b) * p.n_kv_heads * p.group + static_cast<size_t>(kvh) * p.group + sid_head0 + h;
           *reinterpret_cast<float2*>(p.out + hq * kD + ch) = (L > 0.f) ? make_float2(acc0 / L, acc1 / L) : make_float2(0.f, 0.f);
           if (p.lse && ch == 0) p.lse[hq] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : kNegInf;
