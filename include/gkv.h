@@ -176,10 +176,22 @@ GKV_API int gkv_debug_export_bounds(gkv_cache* c, int32_t layer, float* bounds_o
  * proxies recorded when each block closed, at the budget rd_budget_bpv of the current context.
  * The temporal constraint of Sec. 3.2 holds: no level rises, sink blocks and the newest
  * retire_after tokens' blocks stay at 16 bits; blocks whose level falls are requantised from their
- * current representation.  Reads the masses back to the host, so it synchronises `stream` once;
- * meant to be called when a block has closed (every 64 tokens), not every step.
+ * current representation.  The plan is made on the device (the threshold search of Eq. 4 over the
+ * sorted breakpoints, one thread block per stream; up to 4095 closed blocks, beyond that on the host
+ * from masses read back); the host reads the plan back - one byte per block - to do the slot
+ * bookkeeping, so the call synchronises `stream` once.  Meant to be called when a block has closed
+ * (every 64 tokens), not every step.
  * May return GKV_ERR_BUDGET / GKV_ERR_RANGE as warnings after completing the work. */
 GKV_API int gkv_rd_reallocate(gkv_cache* c, int32_t layer, void* stream);
+
+/* Parity only: the plan gkv_rd_reallocate would apply now, made the way it makes it (on the device),
+ * without applying it, together with the numbers it was made from.  Synchronises `stream`.
+ *   levels_out  HOST int8 [batch][n_kv_heads][n_closed]
+ *   mass_out    HOST fp32 [batch][n_kv_heads][n_closed] running masses m_b, or NULL
+ *   range_out   HOST fp32 [batch][n_kv_heads][n_closed] range proxies e_b, or NULL
+ * Returns GKV_ERR_BUDGET (with the plan written) when a stream cannot meet the budget. */
+GKV_API int gkv_debug_device_plan(gkv_cache* c, int32_t layer, int8_t* levels_out, float* mass_out, float* range_out,
+                                  void* stream);
 
 /* Host-only (no device work): the plan gkv_rd_reallocate decides for one stream.  mass / range
  * fp32 [n_closed]; prev int8 [n_closed] current levels; levels int8 [n_closed] out. */

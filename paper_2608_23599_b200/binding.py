@@ -25,7 +25,7 @@ ERR_RANGE, ERR_BUDGET, ERR_CUDA = -6, -7, -8
 
 EXPORTS = [
     "gkv_query_arena_bytes", "gkv_create", "gkv_destroy", "gkv_append_demote", "gkv_decode_attn",
-    "gkv_decode_attn_observe", "gkv_debug_export_mass", "gkv_debug_export_bounds", "gkv_rd_reallocate",
+    "gkv_decode_attn_observe", "gkv_debug_export_mass", "gkv_debug_export_bounds", "gkv_rd_reallocate", "gkv_debug_device_plan",
     "gkv_debug_replan_levels",
     "gkv_quest_select", "gkv_quest_select_static", "gkv_debug_export_boxes", "gkv_debug_export_scores", "gkv_bits_report",
     "gkv_debug_export_block", "gkv_debug_export_residual",
@@ -87,6 +87,7 @@ def load():
     lib.gkv_debug_export_bounds.argtypes = [vp, i32, vp]
     lib.gkv_debug_export_mass.argtypes = [vp, i32, vp]
     lib.gkv_rd_reallocate.argtypes = [vp, i32, vp]
+    lib.gkv_debug_device_plan.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.gkv_debug_replan_levels.argtypes = [C.POINTER(GkvConfig), i32, i32, C.POINTER(C.c_float), C.POINTER(C.c_float),
                                             C.POINTER(C.c_int8), C.POINTER(C.c_int8), C.POINTER(i32)]
     lib.gkv_quest_select.argtypes = [vp, i32, vp, i32, vp, C.POINTER(i32), vp]
@@ -256,6 +257,17 @@ class Cache:
         out = np.zeros((self.cfg.batch, self.cfg.n_kv_heads, n, 4), dtype=np.float32)
         _check(load().gkv_debug_export_bounds(self.handle, layer, out.ctypes.data_as(C.c_void_p)), "gkv_debug_export_bounds")
         return out
+
+    def gkv_debug_device_plan(self, layer):
+        """(levels int8, mass fp32, range fp32) as numpy [batch][n_kv_heads][n_closed]: the plan the device
+        allocator makes now and the numbers it was made from; flag: a stream missed the budget."""
+        n = self.gkv_ctx_len(layer) // 64
+        shp = (self.cfg.batch, self.cfg.n_kv_heads, n)
+        lv, ms, rg = np.zeros(shp, np.int8), np.zeros(shp, np.float32), np.zeros(shp, np.float32)
+        rc = load().gkv_debug_device_plan(self.handle, layer, lv.ctypes.data_as(C.c_void_p), ms.ctypes.data_as(C.c_void_p),
+                                          rg.ctypes.data_as(C.c_void_p), self._st())
+        _check(rc, "gkv_debug_device_plan", allow=(ERR_BUDGET,))
+        return lv, ms, rg, rc == ERR_BUDGET
 
     def gkv_rd_reallocate(self, layer):
         """Decode-time re-allocation of an RD-policy layer from the running block masses."""

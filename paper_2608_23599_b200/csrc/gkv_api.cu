@@ -1454,14 +1454,49 @@ int gkv_debug_replan_levels(const gkv_config* cfg, int32_t n_closed, int32_t n_t
   return GKV_OK;
 }
 
-int gkv_rd_reallocate(gkv_cache* c, int32_t layer, void* stream) {
-  if (!c || layer < 0 || layer >= c->cfg.n_layers) return GKV_ERR_INVALID_ARG;
+namespace {
+// Largest number of closed blocks whose breakpoints the device allocator sorts in shared memory.
+constexpr int kRdPlanMaxBlocks = 4095;
+
+// Level plan of every stream of a layer from its running masses and range proxies: on the device when
+// the breakpoints fit (one small launch and n bytes per stream back instead of 8 n and the host's
+// sort), else on the host.  target: [n_streams][n].  *missed: some stream cannot meet the budget.
+int rd_plan_layer(gkv_cache* c, LayerState& L, int8_t* target, bool* missed, cudaStream_t st) {
   const gkv_config& cfg = c->cfg;
-  if (cfg.policy != GKV_POLICY_RD || is_mla(cfg)) return GKV_ERR_BAD_STATE;
-  LayerState& L = c->layers[layer];
   const int n = L.n_closed, ns = c->n_streams;
-  if (n == 0) return GKV_OK;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  *missed = false;
+  if (n <= kRdPlanMaxBlocks) {
+    const long long nval_tok = cfg.d_k + cfg.d_v;
+    const long long T = static_cast<long long>(n) * kBlock + L.n_tail;
+    RdPlanParams p{};
+    p.mass = L.ema_d;
+    p.range = L.range_d;
+    p.table = L.table_d;
+    p.levels_out = c->levels_d;
+    p.miss_flag = reinterpret_cast<uint32_t*>(c->mass_d);        // ingest scratch, idle here
+    p.n = n;
+    p.mass_stride = c->max_blocks + 1;
+    p.range_stride = c->max_blocks;
+    p.table_stride = c->table_stride;
+    p.out_stride = c->max_blocks;
+    rd_plan_smem_bytes(n, &p.m_pad);
+    p.n_sink_blocks = cfg.n_sink_blocks;
+    p.retire_after = cfg.retire_after;
+    p.monotone = cfg.monotone_in_age != 0;
+    p.use_prev = 1;
+    p.nval_tok = static_cast<unsigned long long>(nval_tok);
+    p.budget_bits = static_cast<unsigned long long>(std::floor(static_cast<double>(cfg.rd_budget_bpv) * static_cast<double>(T * nval_tok)));
+    p.tail_bits = static_cast<unsigned long long>(L.n_tail) * 16ull * static_cast<unsigned long long>(nval_tok);
+    uint32_t flag = 0;
+    CK(c, cudaMemsetAsync(p.miss_flag, 0, sizeof(uint32_t), st));
+    CK(c, launch_rd_plan(p, ns, st));
+    CK(c, cudaMemcpy2DAsync(target, static_cast<size_t>(n), c->levels_d, static_cast<size_t>(c->max_blocks), static_cast<size_t>(n), ns,
+                            cudaMemcpyDeviceToHost, st));
+    CK(c, cudaMemcpyAsync(&flag, p.miss_flag, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    CK(c, cudaStreamSynchronize(st));
+    *missed = flag != 0;
+    return GKV_OK;
+  }
   std::vector<float> mass(static_cast<size_t>(ns) * n), range(static_cast<size_t>(ns) * n);
   CK(c, cudaMemcpy2DAsync(mass.data(), static_cast<size_t>(n) * sizeof(float), L.ema_d,
                           static_cast<size_t>(c->max_blocks + 1) * sizeof(float), static_cast<size_t>(n) * sizeof(float), ns,
@@ -1470,14 +1505,50 @@ int gkv_rd_reallocate(gkv_cache* c, int32_t layer, void* stream) {
                           static_cast<size_t>(c->max_blocks) * sizeof(float), static_cast<size_t>(n) * sizeof(float), ns,
                           cudaMemcpyDeviceToHost, st));
   CK(c, cudaStreamSynchronize(st));
+  *missed = rd_allocate_streams(cfg, mass.data(), range.data(), n, L.n_tail, ns, L.level.data(), c->max_blocks, target, n);
+  return GKV_OK;
+}
+}  // namespace
+
+int gkv_rd_reallocate(gkv_cache* c, int32_t layer, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return GKV_ERR_INVALID_ARG;
+  const gkv_config& cfg = c->cfg;
+  if (cfg.policy != GKV_POLICY_RD || is_mla(cfg)) return GKV_ERR_BAD_STATE;
+  LayerState& L = c->layers[layer];
+  const int n = L.n_closed, ns = c->n_streams;
+  if (n == 0) return GKV_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
   std::vector<int8_t> target(static_cast<size_t>(ns) * n);
+  bool missed = false;
+  int rc = rd_plan_layer(c, L, target.data(), &missed, st);
+  if (rc != GKV_OK) return rc;
   int warn = GKV_OK;
-  if (rd_allocate_streams(cfg, mass.data(), range.data(), n, L.n_tail, ns, L.level.data(), c->max_blocks, target.data(), n)) {
+  if (missed) {
     L.budget_flag = true;
     warn = GKV_ERR_BUDGET;
   }
-  const int rc = demote_to_targets(c, L, target.data(), static_cast<size_t>(n), st);
+  rc = demote_to_targets(c, L, target.data(), static_cast<size_t>(n), st);
   return rc != GKV_OK ? rc : warn;
+}
+
+int gkv_debug_device_plan(gkv_cache* c, int32_t layer, int8_t* levels_out, float* mass_out, float* range_out, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !levels_out) return GKV_ERR_INVALID_ARG;
+  const gkv_config& cfg = c->cfg;
+  if (cfg.policy != GKV_POLICY_RD || is_mla(cfg)) return GKV_ERR_BAD_STATE;
+  LayerState& L = c->layers[layer];
+  const int n = L.n_closed, ns = c->n_streams;
+  if (n == 0) return GKV_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bool missed = false;
+  const int rc = rd_plan_layer(c, L, levels_out, &missed, st);
+  if (rc != GKV_OK) return rc;
+  if (mass_out)
+    CK(c, cudaMemcpy2D(mass_out, static_cast<size_t>(n) * sizeof(float), L.ema_d, static_cast<size_t>(c->max_blocks + 1) * sizeof(float),
+                       static_cast<size_t>(n) * sizeof(float), ns, cudaMemcpyDeviceToHost));
+  if (range_out)
+    CK(c, cudaMemcpy2D(range_out, static_cast<size_t>(n) * sizeof(float), L.range_d, static_cast<size_t>(c->max_blocks) * sizeof(float),
+                       static_cast<size_t>(n) * sizeof(float), ns, cudaMemcpyDeviceToHost));
+  return missed ? GKV_ERR_BUDGET : GKV_OK;
 }
 
 int gkv_destroy(gkv_cache* c) {

@@ -173,6 +173,22 @@ cudaError_t launch_certificate(const CertificateParams& p, cudaStream_t st);
 cudaError_t launch_encode(const EncodeParams& p, cudaStream_t st);
 cudaError_t launch_ingest(const EncodeParams& p, cudaStream_t st);   // every job reads the bf16 input rows; 16-byte aligned inputs
 cudaError_t launch_stats(const StatsParams& p, cudaStream_t st);
+
+// RD allocator on the device (Sec. 3.3; gkv_rdplan.cu): one level plan per stream from block masses
+// and range proxies, identical to the host allocator's on the same numbers.
+struct RdPlanParams {
+  const float* mass;            // [n_streams][mass_stride] running block mass m_b
+  const float* range;           // [n_streams][range_stride] range proxy e_b
+  const TableEntry* table;      // [n_streams][table_stride]: the blocks' present levels
+  int8_t* levels_out;           // [n_streams][out_stride]
+  uint32_t* miss_flag;          // set to 1 when a stream cannot meet the budget (its plan is still written)
+  int32_t n, mass_stride, range_stride, table_stride, out_stride;
+  int32_t m_pad;                // power of two >= 4 n + 1 (rd_plan_smem_bytes)
+  int32_t n_sink_blocks, retire_after, monotone, use_prev;
+  unsigned long long nval_tok, budget_bits, tail_bits;
+};
+size_t rd_plan_smem_bytes(int n, int* m_pad_out);
+cudaError_t launch_rd_plan(const RdPlanParams& p, int n_streams, cudaStream_t st);
 cudaError_t launch_append_rows(uint8_t* arena, const TableEntry* table, int table_stride, int tail_index,
                                int n_streams, int n_kv_heads, const uint16_t* k_in, const uint16_t* v_in,
                                int n_tok, int first_tok, int n_rows, int dst_row0, cudaStream_t st);

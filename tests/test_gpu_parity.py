@@ -618,7 +618,15 @@ def test_decode_time_reallocation_from_running_masses():
         if gcache.gkv_ctx_len(0) % 64 != 0:
             continue
         before = {(b, h): gcache.gkv_debug_export_levels(0, b, h).copy() for b in range(cfg.batch) for h in range(cfg.n_kv_heads)}
+        # the plan is made on the device: bit for bit the host allocator's plan on the same masses and ranges
+        B = _binding()
+        lv_dev, ms, rg, _ = gcache.gkv_debug_device_plan(0)
+        for (b, h), old in before.items():
+            lv_host, _ = B.gkv_debug_replan_levels(gcache.cfg, gcache.gkv_ctx_len(0) % 64, ms[b, h], rg[b, h], old)
+            assert np.array_equal(lv_dev[b, h], lv_host), f"device and host plans differ for stream {(b, h)} at step {step}"
         gcache.gkv_rd_reallocate(0)
+        for (b, h) in before:
+            assert np.array_equal(gcache.gkv_debug_export_levels(0, b, h), lv_dev[b, h])
         free_plan = ofree.rd_reallocate(0)
         recent = w.retire_after // 64
         for (b, h), old in before.items():
@@ -912,3 +920,37 @@ def test_arena_exhausted_by_a_demotion_step_leaves_the_cache_consistent():
     U.assert_outputs_close(out, o_out, "after a failed demotion step")
     assert gcache.gkv_bits_report(0).resident_bits == oc.bits_report(0)["resident_bits"]
     gcache.close()
+
+
+@pytest.mark.parametrize("budget", [2.5, 4.84, 9.0, 0.05])
+def test_device_allocator_equals_host_allocator(budget):
+    """The threshold search on the device (gkv_rd_reallocate's planner) against the host allocator on
+    the same masses, ranges and present levels: 127 closed blocks per stream, several budgets (the last one
+    cannot be met: both report it and agree on the plan), after observed queries have moved the masses."""
+    w = dataclasses.replace(W.config(1, "small"), ctx=8192 - 37, max_ctx=8192 + 256, rd_budget_bpv=budget)
+    B = _binding()
+    g = B.Cache(B.config_from_workload(w, 1))
+    dev = g.device
+    data = W.make_layer(w, 0, "cpu")
+    g.gkv_append_demote(0, data["k"].to(dev), data["v"].to(dev), token_mass=data["mass"].to(dev).contiguous())
+    out = torch.empty((w.batch, w.n_q_heads, w.d_v), dtype=torch.float32, device=dev)
+    for step in range(5):
+        tok = W.make_decode_tokens(w, 0, step, "cpu")
+        g.gkv_decode_attn_observe(0, tok["q"].to(dev), out)
+    torch.cuda.synchronize()
+    lv_dev, ms, rg, miss_dev = g.gkv_debug_device_plan(0)
+    assert lv_dev.shape[2] == 127 and np.all(ms >= 0) and np.all(rg >= 0)
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            prev = g.gkv_debug_export_levels(0, b, h)
+            lv_host, miss_host = B.gkv_debug_replan_levels(g.cfg, g.gkv_ctx_len(0) % 64, ms[b, h], rg[b, h], prev)
+            assert np.array_equal(lv_dev[b, h], lv_host), (budget, b, h)
+            assert np.all(lv_dev[b, h] <= prev)
+            if miss_host:
+                assert miss_dev
+            # and the oracle's allocator (Sec. 3.3) on the same fp32 numbers
+            want, _tau, flag = O.rd_allocate(ms[b, h], rg[b, h], w.d_k, w.d_v, 0, g.gkv_ctx_len(0) % 64, budget, w.n_sink_blocks,
+                                             w.retire_after, prev.astype(np.int32), 1)
+            assert np.array_equal(lv_dev[b, h].astype(np.int32), np.asarray(want, dtype=np.int32))
+            assert bool(flag) == miss_host
+    g.close()
