@@ -317,8 +317,9 @@ class Cache:
 
     def gkv_bits_report(self, layer=-1) -> GkvBits:
         out = GkvBits()
-        _check(load().gkv_bits_report(self.handle, layer, C.byref(out)), "gkv_bits_report",
-               allow=(ERR_RANGE, ERR_BUDGET))
+        # the warnings (a saturated or oversized scale, a missed budget) do not fail the call; the last one is kept
+        self.last_report_status = _check(load().gkv_bits_report(self.handle, layer, C.byref(out)), "gkv_bits_report",
+                                         allow=(ERR_RANGE, ERR_BUDGET))
         return out
 
     def gkv_ctx_len(self, layer) -> int:

@@ -311,7 +311,7 @@ __device__ __forceinline__ bool ingest_values(uint32_t ld, uint8_t* vp, uint8_t*
   n[0][1] = n1;
   n[1][0] = n2;
   n[1][1] = n3;
-  return g0.range || g1.range;
+  return g0.range || g1.range || g0.s > v_scale_limit(BITS) || g1.s > v_scale_limit(BITS);
 }
 
 __global__ void __launch_bounds__(kInThreads, 3) ingest_kernel(const __grid_constant__ EncodeParams p) {

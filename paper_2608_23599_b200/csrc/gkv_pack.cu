@@ -219,8 +219,8 @@ __global__ void __launch_bounds__(256) encode_kernel(const __grid_constant__ Enc
             mx = fmaxf(mx, x);
           }
           const QuantOut q = quant_params(mn, mx, L);
-          range = q.range;
           const float s32 = fp16_bits_to_f32(q.s_bits), z32 = fp16_bits_to_f32(q.z_bits);
+          range = q.range || s32 > v_scale_limit(L);
           const float inv = s32 > 0.f ? __fdiv_rn(1.f, s32) : 0.f;
           for (int c = 0; c < kGroup; ++c)
             codes[t * kD + 32 * g + c] = quant_code(tile[t * kTileLd + 32 * g + c], s32, z32, inv, qmax);

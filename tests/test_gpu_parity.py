@@ -954,3 +954,34 @@ def test_device_allocator_equals_host_allocator(budget):
             assert np.array_equal(lv_dev[b, h].astype(np.int32), np.asarray(want, dtype=np.int32))
             assert bool(flag) == miss_host
     g.close()
+
+
+@pytest.mark.parametrize("level,ok_span,bad_span", [(8, 2.0e5, 3.0e5), (4, 5.0e4, 7.0e4), (2, 4.0e4, 6.0e4)])
+@pytest.mark.parametrize("aligned", [True, False])
+def test_value_scale_beyond_the_read_path_is_reported(level, ok_span, bad_span, aligned):
+    """A 32-channel value group whose span makes the fp16 scale larger than the read path takes
+    (1023 / 4094 / 16376 at 8 / 4 / 2 bits) is stored as the quantiser defines it and reported as
+    GKV_ERR_RANGE by the next bits report, by the bulk encoder (16-byte aligned rows) and by the general
+    one alike; a span just below the limit is not."""
+    B = _binding()
+    w = _tiny(128, policy=W.POLICY_EXTERNAL)
+    plan = np.full((w.batch, w.n_kv_heads, 2), level, dtype=np.int8)
+    for span, want in ((ok_span, B.OK), (bad_span, B.ERR_RANGE)):
+        g = B.Cache(B.config_from_workload(w))
+        dev = g.device
+        data = W.make_layer(w, 0, "cpu")
+        v = data["v"].clone()
+        v[0, 5, 0, 1] = span              # the group's minimum stays near zero: the zero point does not saturate
+
+        def place(t):
+            if aligned:
+                return t.to(dev).contiguous()
+            flat = torch.empty(t.numel() + 8, dtype=t.dtype, device=dev)
+            view = flat[2:2 + t.numel()].view(t.shape)
+            view.copy_(t.to(dev))
+            return view
+
+        g.gkv_append_demote(0, place(data["k"]), place(v), level_plan=plan)
+        g.gkv_bits_report(0)
+        assert g.last_report_status == want, (level, span, g.last_report_status)
+        g.close()
