@@ -48,7 +48,7 @@ typedef enum gkv_status {
   GKV_ERR_BAD_STATE = -4,       /* e.g. page selection without page_tokens, ingest on a non-empty stream */
   GKV_ERR_UNSUPPORTED = -5,     /* shape or combination not compiled */
   GKV_ERR_RANGE = -6,           /* a scale/zero saturated at +-65504, or a value scale exceeds what the read path
-                                   takes (1023 / 4094 / 16376 at 8 / 4 / 2 bits); result stored, flag returned */
+                                   takes (4094); result stored, flag returned */
   GKV_ERR_BUDGET = -7,          /* RD budget unreachable even with every free block at centroid (plan applied) */
   GKV_ERR_CUDA = -8             /* CUDA runtime error; see gkv_last_cuda_error */
 } gkv_status;

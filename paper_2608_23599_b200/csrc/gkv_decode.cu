@@ -11,19 +11,18 @@
 //
 // Math: S^T[tokens x heads] = K[tokens x ch] Q^T and O^T[ch x heads] += V^T[ch x tokens] P^T on
 // mma.m16n8k16 with the query heads as the n = 8 dimension.  Quantised codes are stored in
-// A-fragment order (gkv_layout.cuh) at bit positions where one LOP3 turns a code into the fp16
-// number "bias + code".  Scales are folded into the B operands (q' = q * s_k per 32-token key
-// group, P' = p * s_v per 32-channel value group); zero points and the biases are handled by
-// extra MMAs (A = scale / zero-point pattern or a constant) instead of per-value arithmetic.
+// A-fragment order (gkv_layout.cuh) and become A operands by masking: a code in the mantissa of an
+// fp16 with a zero exponent field is the number code * 2^(p - 24), bias-free.  Scales are folded into the
+// B operands (q' = q * s_k per 32-token key group, P' = p * s_v per 32-channel value group); zero
+// points are handled by extra MMAs (A = zero-point pattern) instead of per-value arithmetic, the
+// powers of two of the code fields in fp32 after the key MMAs and in P' before the value MMAs.
 //
 // Precision: every B operand that carries a rounded product or probability is a pair hi + lo of
 // fp16 (bf16 for exact rows) numbers, hi = rn(x), lo = rn(x - hi), so that the operand is good to
 // ~2^-22 and the fp32 accumulators decide the error.  A warp serves at most four query heads: the
 // n = 8 dimension holds (hi, lo) column pairs, column 2 j the hi part and column 2 j + 1 the lo part of
 // head j, so one MMA does both and a lane finds the two halves of its head side by side in its
-// accumulator registers.  A KV head with 5..8 query heads is read as two such head groups.  The
-// biases of the code unpack are kept small (<= 256; 1024 at 8 bits) because "bias * sum of
-// operands" is cancelled in fp32.
+// accumulator registers.  A KV head with 5..8 query heads is read as two such head groups.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -126,70 +125,36 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
-// ---- code unpack: the four A registers of MMA index s as fp16 "bias + code" ------------------
-// A code that sits at mantissa bit b of an fp16 with exponent 2^E has the value code * 2^(E - 10 + b),
-// so picking E = 10 - b makes "mask, or in the exponent" a complete conversion.  The bias 2^(10 - b)
-// is cancelled after the MMA in fp32 (against "bias * sum of the B operand"), which
-// costs 2^-23 * bias * |sum| of accuracy: the words are therefore shifted so that the codes land in
-// the upper mantissa bits (8-bit: bias 1024 against codes up to 255; 4-bit: 256 / 16; 2-bit: 16 / 4;
-// first / second number = A rows r / rows r + 8 of the MMA).  `mid` is the centre of the code range:
-// products are formed with (code - mid) so that the rounding of the folded scale acts on a centred
-// value; the term mid * sum(q s) is added back from an exact MMA.
+// ---- code unpack: the four A registers of MMA index s as bias-free fp16 numbers --------------------
+// A code that sits at mantissa bit p of an fp16 whose exponent field is zero is the number
+// code * 2^(p - 24): masking the packed word is a complete conversion, there is no bias to cancel in the
+// accumulators afterwards and no precision is lost to one.  The fields of a word are read where they are
+// (one shift per word brings the second pair of fields down), so p differs between the fields:
+//   keys    (field = A register a: rows r / r + 8 of the MMA for a & 1 = 0 / 1): the two row classes of an
+//           MMA come out with the weights 2^-24 and 2^(p1 - 24) (KScale), evened out in fp32 after it;
+//   values  (fields ordered by token half, gkv_layout.cuh): registers 0, 1 (tokens 0-7 of the tile) at
+//           p = 0, registers 2, 3 (tokens 8-15) at p1; P' is multiplied by 2^(4 - p) (VScale), so that
+//           every product carries the common factor 2^-20, which the exact rows put into P and the final
+//           row takes out again.
 template <int BITS>
-struct Bias;
+struct KScale;                     // 2^(24 - p) of the rows r (lo) and r + 8 (hi)
 template <>
-struct Bias<8> {
-  static constexpr float lo = 1024.f, hi = 1024.f, mid = 128.f;       // bias + mid must be an fp16 number
+struct KScale<8> {
+  static constexpr float lo = 16777216.f, hi = 16777216.f;
 };
 template <>
-struct Bias<4> {
-  static constexpr float lo = 256.f, hi = 16.f, mid = 7.5f;
+struct KScale<4> {
+  static constexpr float lo = 16777216.f, hi = 1048576.f;
 };
 template <>
-struct Bias<2> {
-  static constexpr float lo = 16.f, hi = 4.f, mid = 1.5f;
+struct KScale<2> {
+  static constexpr float lo = 16777216.f, hi = 4194304.f;
 };
-
-// Words of one lane for MMA indices [s0, s0 + NS): 8-bit 2 words per s, 4-bit 1, 2-bit 1 per 2.
 template <int BITS>
-__device__ __forceinline__ void unpack(const uint32_t* w, int s_local, uint32_t (&a)[4]) {
-  if constexpr (BITS == 8) {
-    constexpr uint32_t kMagic = 0x64006400u;            // selector 5 picks the 0x64 byte
-    const uint32_t w0 = w[2 * s_local], w1 = w[2 * s_local + 1];
-    a[0] = prmt(w0, kMagic, 0x5250u);
-    a[1] = prmt(w0, kMagic, 0x5351u);
-    a[2] = prmt(w1, kMagic, 0x5250u);
-    a[3] = prmt(w1, kMagic, 0x5351u);
-  } else if constexpr (BITS == 4) {
-    // codes of A registers 0..3 at bits 0, 4, 8, 12 of each 16-bit half -> bits 2 (0, 2) and 6 (1, 3)
-    const uint32_t v0 = w[s_local] << 2, v1 = w[s_local] >> 6;
-    a[0] = lop3_and_or(v0, 0x003C003Cu, 0x5C005C00u);   // 256 + code
-    a[1] = lop3_and_or(v0, 0x03C003C0u, 0x4C004C00u);   // 16 + code
-    a[2] = lop3_and_or(v1, 0x003C003Cu, 0x5C005C00u);
-    a[3] = lop3_and_or(v1, 0x03C003C0u, 0x4C004C00u);
-  } else {
-    // even s: registers 0..3 at bits 0, 2, 8, 10; odd s: at bits 4, 6, 12, 14 -> bits 6 (0, 2) and 8 (1, 3)
-    const uint32_t x = w[s_local >> 1];
-    const uint32_t v0 = (s_local & 1) ? (x << 2) : (x << 6), v1 = (s_local & 1) ? (x >> 6) : (x >> 2);
-    a[0] = lop3_and_or(v0, 0x00C000C0u, 0x4C004C00u);   // 16 + code
-    a[1] = lop3_and_or(v0, 0x03000300u, 0x44004400u);   // 4 + code
-    a[2] = lop3_and_or(v1, 0x00C000C0u, 0x4C004C00u);
-    a[3] = lop3_and_or(v1, 0x03000300u, 0x44004400u);
-  }
-}
-
-// Value codes need no bias: with a zero exponent field the fp16 number is code * 2^(p - 24), p the
-// code's lowest mantissa bit, and the value MMAs accumulate V^T P' directly (no correction MMA, no
-// cancellation in the accumulators).  The fields of a word are arranged (gkv_layout.cuh) so that p depends
-// on the token half only: registers 0, 1 (tokens 0-7 of the tile) at p_lo, registers 2, 3 (tokens 8-15) at
-// p_hi = 6; P' of the first half is multiplied by 2^(p_hi - p_lo) (VScale::lo), 8-bit codes (p = 0
-// everywhere) by 2^6 in both halves, so that every product carries the common factor 2^-18, which the
-// exact rows put into P and the final row takes out again.
-template <int BITS>
-struct VScale;
+struct VScale;                     // 2^(4 - p) of the tokens 0-7 (lo) and 8-15 (hi) of a tile
 template <>
 struct VScale<8> {
-  static constexpr float lo = 64.f, hi = 64.f;
+  static constexpr float lo = 16.f, hi = 16.f;
 };
 template <>
 struct VScale<4> {
@@ -197,13 +162,16 @@ struct VScale<4> {
 };
 template <>
 struct VScale<2> {
-  static constexpr float lo = 4.f, hi = 1.f;
+  static constexpr float lo = 16.f, hi = 4.f;
 };
-constexpr float kVUnit = 1.f / 262144.f;          // 2^-18: weight of a value product in the accumulators
-constexpr float kVUnitInv = 262144.f;
+constexpr float kVUnit = 1.f / 1048576.f;         // 2^-20: weight of a value product in the accumulators
+constexpr float kVUnitInv = 1048576.f;
 
-template <int BITS>
-__device__ __forceinline__ void unpack_v(const uint32_t* w, int s_local, uint32_t (&a)[4]) {
+// Words of one lane for MMA indices [s0, s0 + NS): 8-bit 2 words per s, 4-bit 1, 2-bit 1 per 2.
+// Keys: field f of a word belongs to register f.  Values: fields 0, 1 / 2, 3 belong to registers 0, 2 / 1, 3.
+template <int BITS, bool IS_V>
+__device__ __forceinline__ void unpack(const uint32_t* w, int s_local, uint32_t (&a)[4]) {
+  constexpr int i1 = IS_V ? 2 : 1, i2 = IS_V ? 1 : 2;      // registers of fields 1 and 2
   if constexpr (BITS == 8) {
     const uint32_t w0 = w[2 * s_local], w1 = w[2 * s_local + 1];
     a[0] = prmt(w0, 0u, 0x4240u);
@@ -211,20 +179,20 @@ __device__ __forceinline__ void unpack_v(const uint32_t* w, int s_local, uint32_
     a[2] = prmt(w1, 0u, 0x4240u);
     a[3] = prmt(w1, 0u, 0x4341u);
   } else if constexpr (BITS == 4) {
-    // fields at bits 0, 4 (registers 0, 2) and 8, 12 (registers 1, 3) of each 16-bit half -> bits 2 and 6
-    const uint32_t v0 = w[s_local] << 2, v1 = w[s_local] >> 6;
-    a[0] = v0 & 0x003C003Cu;
-    a[2] = v0 & 0x03C003C0u;
-    a[1] = v1 & 0x003C003Cu;
-    a[3] = v1 & 0x03C003C0u;
+    // fields at bits 0, 4, 8, 12 of each 16-bit half
+    const uint32_t v0 = w[s_local], v1 = v0 >> 8;
+    a[0] = v0 & 0x000F000Fu;
+    a[i1] = v0 & 0x00F000F0u;
+    a[i2] = v1 & 0x000F000Fu;
+    a[3] = v1 & 0x00F000F0u;
   } else {
-    // even s: fields at bits 0, 2 (registers 0, 2) and 8, 10 (registers 1, 3); odd s: 4 further -> bits 4 and 6
+    // even s: fields at bits 0, 2, 8, 10; odd s: 4 further
     const uint32_t x = w[s_local >> 1];
-    const uint32_t v0 = (s_local & 1) ? x : (x << 4), v1 = (s_local & 1) ? (x >> 8) : (x >> 4);
-    a[0] = v0 & 0x00300030u;
-    a[2] = v0 & 0x00C000C0u;
-    a[1] = v1 & 0x00300030u;
-    a[3] = v1 & 0x00C000C0u;
+    const uint32_t v0 = (s_local & 1) ? (x >> 4) : x, v1 = (s_local & 1) ? (x >> 12) : (x >> 8);
+    a[0] = v0 & 0x00030003u;
+    a[i1] = v0 & 0x000C000Cu;
+    a[i2] = v1 & 0x00030003u;
+    a[3] = v1 & 0x000C000Cu;
   }
 }
 
@@ -704,9 +672,8 @@ __device__ __forceinline__ void load_words(uint32_t codes, int j, int lane, uint
 }
 
 // Logits of the active tiles of one half (32 tokens): S = scale * (q . k~) + token bias, with
-// k~ = s * code + z.  Data MMAs use A = bias + code and B = q' = q * s (hi and lo columns); an MMA with
-// A = (s | z) and B = q gives sum q s, which is what the bias multiplies (q' is an exact split of q s),
-// and sum q z.  All arguments that address shared memory are 32-bit addresses.
+// k~ = s * code + z.  Data MMAs use A = code * 2^(p - 24) and B = q' = q * s (hi and lo columns); an MMA with
+// A = (s | z) and B = q gives sum q z.  All arguments that address shared memory are 32-bit addresses.
 // Channel slab j (MMA indices 2 j and 2 j + 1) of qk_half; FIRST starts the accumulation chains.
 template <int BITS, bool FULL, bool FIRST>
 __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm, uint32_t qh_addr, int lane,
@@ -731,12 +698,12 @@ __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm
     else mma_f16(zd, pr.x, pr.y, pr.z, pr.w, q.x, q.y);
     uint32_t a[4];
     if (FULL || (tm & 1)) {
-      unpack<BITS>(w0, ss, a);
+      unpack<BITS, false>(w0, ss, a);
       if (FIRST && ss == 0) mma_f16_first(S[0], a[0], a[1], a[2], a[3], q0, q1);
       else mma_f16(S[0], a[0], a[1], a[2], a[3], q0, q1);
     }
     if (FULL || (tm & 2)) {
-      unpack<BITS>(w1, ss, a);
+      unpack<BITS, false>(w1, ss, a);
       if (FIRST && ss == 0) mma_f16_first(S[1], a[0], a[1], a[2], a[3], q0, q1);
       else mma_f16(S[1], a[0], a[1], a[2], a[3], q0, q1);
     }
@@ -748,26 +715,22 @@ template <int BITS, bool FULL>
 __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, int tm, uint32_t qh_addr, int lane, float scale_log2,
                                         uint64_t resmask, int half, float (&x)[4]) {
   const int c4 = lane & 3, r = lane >> 2;
-  // rows r: sum_c q_c s_c; rows r + 8: sum_c q_c z_c (exact products; both columns alike).  The first is
-  // also the sum of q' over its hi and lo columns (q' = q s is split exactly), i.e. what the bias of the
-  // data MMAs multiplies.
+  // rows r + 8: sum_c q_c z_c (exact products; both columns alike; rows r, sum_c q_c s_c, are not needed)
   float zd[4];
   float S[2][4];
   kp += c4 * 16;
   qk_slab<BITS, FULL, true>(kp, kc0, 0, tm, qh_addr, lane, zd, S);
 #pragma unroll
   for (int j = 1; j < 4; ++j) qk_slab<BITS, FULL, false>(kp, kc0, j, tm, qh_addr, lane, zd, S);
-  // rows r carry bias lo, rows r + 8 carry bias hi
-  constexpr float kMid = Bias<BITS>::mid;
-  (void)kMid;                                                                  // (code - mid) s + (z + mid s)
-  const float c_lo = fmaf(-Bias<BITS>::lo, zd[0], zd[2]), c_hi = fmaf(-Bias<BITS>::hi, zd[0], zd[2]);
+  // rows r and rows r + 8 carry the weights of their code fields (KScale)
+  const float k_lo = KScale<BITS>::lo * scale_log2, k_hi = KScale<BITS>::hi * scale_log2, zs = zd[2] * scale_log2;
   const uint32_t rm = static_cast<uint32_t>(resmask >> (32 * half));            // this half's 32 tokens
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
     const bool on = FULL || ((tm >> t) & 1);
     const int tok = 16 * t + r;
-    const float v_lo = on ? (S[t][0] + S[t][1] + c_lo) * scale_log2 : kNegInf;
-    const float v_hi = on ? (S[t][2] + S[t][3] + c_hi) * scale_log2 : kNegInf;
+    const float v_lo = on ? fmaf(S[t][0] + S[t][1], k_lo, zs) : kNegInf;
+    const float v_hi = on ? fmaf(S[t][2] + S[t][3], k_hi, zs) : kNegInf;
     x[2 * t] = ((rm >> tok) & 1u) ? kNegInf : v_lo;
     x[2 * t + 1] = ((rm >> (tok + 8)) & 1u) ? kNegInf : v_hi;
   }
@@ -776,7 +739,7 @@ __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, int tm, uint3
 // O^T += V~^T P^T for the active tiles of one half, v~ = s * code + z per (token, 32-channel group).
 // pf holds the fp16 P^T fragments of the two tiles (hi / lo columns); tile t has its parameters at
 // vp + 256 t and its codes at vc + 256 BITS t.  The data MMAs accumulate code * P' (bias-free codes,
-// see unpack_v) straight into O; the zero points go through one MMA per tile into zc.
+// see unpack) straight into O; the zero points go through one MMA per tile into zc.
 // The loop over the two tiles is kept rolled (see qk_half).
 template <int BITS, bool FULL>
 __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const uint32_t (&pf)[2][2], int lane,
@@ -817,9 +780,9 @@ __device__ __forceinline__ void pv_half(uint32_t vp, uint32_t vc, int tm, const 
       uint32_t wd[BITS / 2];
       uint32_t a[4];
       load_words<BITS>(vct, g, lane, wd);
-      unpack_v<BITS>(wd, 0, a);
+      unpack<BITS, true>(wd, 0, a);
       mma_f16(st.o[2 * g], a[0], a[1], a[2], a[3], p0, p1);
-      unpack_v<BITS>(wd, 1, a);
+      unpack<BITS, true>(wd, 1, a);
       mma_f16(st.o[2 * g + 1], a[0], a[1], a[2], a[3], p0, p1);
     }
   }

@@ -68,10 +68,9 @@ GKV_HD int off_vc(int bits, int t) { return 1024 + (2 + t) * code_bytes_per_tile
 // Where code (lane, s, a, hlf) of a tile sits: byte offset of its 32-bit word inside the tile's
 // code region, and the bit position inside the word.
 // Largest value scale the read path takes: the kernel multiplies the probabilities by the scale and by the
-// power of two that evens out the fields' weights (2^6 / 2^4 / 2^2 at 8 / 4 / 2 bits) in fp16.  A larger
-// scale (a 32-channel value group spanning more than 2.6e5 / 6.1e4 / 4.9e4) is reported like a
-// saturated one.
-GKV_HD float v_scale_limit(int bits) { return bits == 8 ? 1023.f : (bits == 4 ? 4094.f : 16376.f); }
+// power of two that evens out the fields' weights (up to 2^4) in fp16.  A larger scale (a 32-channel
+// value group spanning more than 1.0e6 / 6.1e4 / 1.2e4 at 8 / 4 / 2 bits) is reported like a saturated one.
+GKV_HD float v_scale_limit(int bits) { (void)bits; return 4094.f; }
 GKV_HD int code_field(bool is_v, int a) { return is_v ? ((a >> 1) | ((a & 1) << 1)) : a; }
 GKV_HD void code_pos(int bits, bool is_v, int lane, int s, int a, int hlf, int* byte_off, int* bit) {
   int w, b;
