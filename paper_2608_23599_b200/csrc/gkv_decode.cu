@@ -673,7 +673,7 @@ __device__ __forceinline__ void load_words(uint32_t codes, int j, int lane, uint
 
 // Logits of the active tiles of one half (32 tokens): S = scale * (q . k~) + token bias, with
 // k~ = s * code + z.  Data MMAs use A = code * 2^(p - 24) and B = q' = q * s (hi and lo columns); an MMA with
-// A = (s | z) and B = q gives sum q z.  All arguments that address shared memory are 32-bit addresses.
+// A = zero points and B = q gives sum q z.  All arguments that address shared memory are 32-bit addresses.
 // Channel slab j (MMA indices 2 j and 2 j + 1) of qk_half; FIRST starts the accumulation chains.
 template <int BITS, bool FULL, bool FIRST>
 __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm, uint32_t qh_addr, int lane,
@@ -683,19 +683,26 @@ __device__ __forceinline__ void qk_slab(uint32_t kp, uint32_t kc0, int j, int tm
   uint32_t w0[kW], w1[kW];
   if (FULL || (tm & 1)) load_words<BITS>(kc0, j, lane, w0);
   if (FULL || (tm & 2)) load_words<BITS>(kc0 + cb, j, lane, w1);
+  // zero points and scales of the slab's two MMA indices: {s0: c0 c1, s1: c0 c1, s0: c2 c3, s1: c2 c3}
+  const uint4 zp = lds128(kp + j * 128), sp = lds128(kp + j * 128 + 16);
+  {
+    // sum q z of both MMA indices in one MMA: rows r carry the zero points of index s0, rows r + 8 those of
+    // s1; the hi column of a head carries the query slice of s0, its lo column that of s1.  The wanted
+    // products sit in the accumulator registers 0 (row r, hi column) and 3 (row r + 8, lo column).
+    const uint2 qz = lds64(qh_addr + j * 512 + (lo_part_lane(lane) ? 256 : 0));
+    if (FIRST) mma_f16_first(zd, zp.x, zp.y, zp.z, zp.w, qz.x, qz.y);
+    else mma_f16(zd, zp.x, zp.y, zp.z, zp.w, qz.x, qz.y);
+  }
 #pragma unroll
   for (int ss = 0; ss < 2; ++ss) {
-    const uint4 pr = lds128(kp + j * 128 + ss * 64);   // s01, z01, s23, z23
     const uint2 q = lds64(qh_addr + j * 512 + ss * 256);
     uint32_t q0, q1, q0l, q1l;
-    hmul2_split(q.x, pr.x, q0, q0l);
-    hmul2_split(q.y, pr.z, q1, q1l);
+    hmul2_split(q.x, ss ? sp.y : sp.x, q0, q0l);
+    hmul2_split(q.y, ss ? sp.w : sp.z, q1, q1l);
     if (lo_part_lane(lane)) {
       q0 = q0l;
       q1 = q1l;
     }
-    if (FIRST && ss == 0) mma_f16_first(zd, pr.x, pr.y, pr.z, pr.w, q.x, q.y);
-    else mma_f16(zd, pr.x, pr.y, pr.z, pr.w, q.x, q.y);
     uint32_t a[4];
     if (FULL || (tm & 1)) {
       unpack<BITS, false>(w0, ss, a);
@@ -715,15 +722,15 @@ template <int BITS, bool FULL>
 __device__ __forceinline__ void qk_half(uint32_t kp, uint32_t kc0, int tm, uint32_t qh_addr, int lane, float scale_log2,
                                         uint64_t resmask, int half, float (&x)[4]) {
   const int c4 = lane & 3, r = lane >> 2;
-  // rows r + 8: sum_c q_c z_c (exact products; both columns alike; rows r, sum_c q_c s_c, are not needed)
+  // sum_c q_c z_c = zd[0] + zd[3] (exact products, see qk_slab)
   float zd[4];
   float S[2][4];
-  kp += c4 * 16;
+  kp += c4 * 32;
   qk_slab<BITS, FULL, true>(kp, kc0, 0, tm, qh_addr, lane, zd, S);
 #pragma unroll
   for (int j = 1; j < 4; ++j) qk_slab<BITS, FULL, false>(kp, kc0, j, tm, qh_addr, lane, zd, S);
   // rows r and rows r + 8 carry the weights of their code fields (KScale)
-  const float k_lo = KScale<BITS>::lo * scale_log2, k_hi = KScale<BITS>::hi * scale_log2, zs = zd[2] * scale_log2;
+  const float k_lo = KScale<BITS>::lo * scale_log2, k_hi = KScale<BITS>::hi * scale_log2, zs = (zd[0] + zd[3]) * scale_log2;
   const uint32_t rm = static_cast<uint32_t>(resmask >> (32 * half));            // this half's 32 tokens
 #pragma unroll
   for (int t = 0; t < 2; ++t) {

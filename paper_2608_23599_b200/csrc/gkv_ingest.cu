@@ -164,12 +164,12 @@ __device__ __forceinline__ bool ingest_keys(uint32_t tile_k, uint8_t* half_base,
   }
   const GroupParams g0 = i_params<BITS>(i_lo(my_mn), i_lo(my_mx)), g1 = i_params<BITS>(i_hi(my_mn), i_hi(my_mx));
   {
-    // record [slice][c4] = {scale c0, scale c1, zero c0, zero c1, then the same for c0 + 8, c1 + 8}
+    // per (slab, c4) a record of zero points and one of scales, each {s0: c0 c1, s1: c0 c1, s0: c2 c3, s1: c2 c3}
+    // (gkv_layout.cuh); this lane holds the pair (c0, c1) or (c2, c3) (r & 1) of MMA index s_glob
     const int s_glob = 4 * chh + (r >> 1);
-    uint2 rec;
-    rec.x = static_cast<uint32_t>(g0.s_bits) | (static_cast<uint32_t>(g1.s_bits) << 16);
-    rec.y = static_cast<uint32_t>(g0.z_bits) | (static_cast<uint32_t>(g1.z_bits) << 16);
-    *reinterpret_cast<uint2*>(half_base + off_kp() + (s_glob * 4 + c4) * 16 + (r & 1) * 8) = rec;
+    uint32_t* rec = reinterpret_cast<uint32_t*>(half_base + off_kp() + ((s_glob >> 1) * 4 + c4) * 32) + (r & 1) * 2 + (s_glob & 1);
+    rec[0] = static_cast<uint32_t>(g0.z_bits) | (static_cast<uint32_t>(g1.z_bits) << 16);
+    rec[4] = static_cast<uint32_t>(g0.s_bits) | (static_cast<uint32_t>(g1.s_bits) << 16);
   }
   prm[r * 4 + c4] = i_pack_params(g0, g1);
   __syncwarp();

@@ -109,15 +109,19 @@ GKV_HD void v_coord(int tok, int ch, int* tile, int* lane, int* s, int* a, int* 
   *a = (c16 >> 3) | ((t16 >> 3) << 1);
   *hlf = t16 & 1;
 }
-// Key params of a half: 16-byte records [s][c4] = {scale c0, scale c1, zero c0, zero c1,
-// scale c2, scale c3, zero c2, zero c3} with c0 = 16 s + 2 c4, c1 = c0 + 1, c2 = c0 + 8, c3 = c2 + 1.
-// Returns the index (in fp16 units) of channel ch's scale inside the 512-byte record array;
-// its zero sits 2 entries later.
+// Key params of a half: 32 bytes per (channel slab j of 32 channels, c4): a 16-byte record of zero points,
+// then one of scales, each {s0: c0 c1, s1: c0 c1, s0: c2 c3, s1: c2 c3} for the slab's two MMA indices
+// s0 = 2 j, s1 = 2 j + 1 and the lane's channel pairs c0 = 16 s + 2 c4, c1 = c0 + 1, c2 = c0 + 8,
+// c3 = c2 + 1.  The zero-point record is the A operand of the one MMA per slab that forms sum q z for both
+// MMA indices (rows r from s0, rows r + 8 from s1); the scale record feeds q' = q s of both.
+// Returns the index (in fp16 units) of channel ch's scale inside the 512-byte array; its zero point
+// sits 8 entries before.
 GKV_HD int kp_index(int ch) {
   const int s = ch >> 4, c16 = ch & 15;
   const int c4 = (c16 & 7) >> 1;
-  return (s * 4 + c4) * 8 + (c16 >> 3) * 4 + (c16 & 1);
+  return ((s >> 1) * 4 + c4) * 16 + 8 + ((c16 >> 3) * 2 + (s & 1)) * 2 + (c16 & 1);
 }
+GKV_HD int kp_zero_index(int ch) { return kp_index(ch) - 8; }
 // Value params of a tile (256 B): scales first, then zeros, both as fp16 pairs of the lane's
 // token pairs tA = (2 c4, 2 c4 + 1) and tB = (8 + 2 c4, 9 + 2 c4):
 //   scales [c4][group] = {s tA0, s tA1, s tB0, s tB1}   (one lane reads its 4 groups as 32 contiguous bytes)

@@ -73,7 +73,7 @@ __device__ void load_tile(float* tile, const uint8_t* arena, const EncodeParams&
       const uint16_t* kp = reinterpret_cast<const uint16_t*>(hb + off_kp());
       const int idx = kp_index(c);
       s = fp16_bits_to_f32(kp[idx]);
-      z = fp16_bits_to_f32(kp[idx + 2]);
+      z = fp16_bits_to_f32(kp[kp_zero_index(c)]);
     } else {
       const uint16_t* vp = reinterpret_cast<const uint16_t*>(hb + off_vp(bits, (t >> 4) & 1));
       s = fp16_bits_to_f32(vp[vp_scale_index(t & 15, c >> 5)]);
@@ -206,7 +206,7 @@ __global__ void __launch_bounds__(256) encode_kernel(const __grid_constant__ Enc
           uint16_t* kp = reinterpret_cast<uint16_t*>(dst + half * half_bytes(L) + off_kp());
           const int idx = kp_index(c);
           kp[idx] = q.s_bits;
-          kp[idx + 2] = q.z_bits;
+          kp[kp_zero_index(c)] = q.z_bits;
           ps[tid] = s32;                 // index = half * 128 + channel
           pz[tid] = z32;
         } else {
@@ -491,7 +491,7 @@ __global__ void __launch_bounds__(256) export_kernel(const uint8_t* arena, uint3
     const int half = tid >> 7, c = tid & (kD - 1);
     const uint16_t* kp = reinterpret_cast<const uint16_t*>(slot + half * half_bytes(level) + off_kp());
     scale[half * kD + c] = kp[kp_index(c)];
-    zero[half * kD + c] = kp[kp_index(c) + 2];
+    zero[half * kD + c] = kp[kp_zero_index(c)];
   } else {
     // [64][4]
     const int t = tid >> 2, g = tid & 3;
