@@ -180,6 +180,12 @@ __device__ __forceinline__ void t_mma_f16(uint32_t d_tmem, uint64_t a_desc, uint
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// legacy warp-level MMA (m16n8k16, fp16 operands, fp32 accumulators) for the small key-constant products
+__device__ __forceinline__ void t_mma_sync_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ void t_commit(uint32_t bar) {
   asm volatile(
       "{\n"
@@ -645,17 +651,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     // ---------------- conversion of blocks into tiles, and Q' ----------------
     const int dt = tid - kTcFirstConvertWarp * 32;          // 0 .. 287
     const int dj = dt % kMlaChunks, dg = dt / kMlaChunks;   // tile conversion: chunk of 8 channels, token group
-    // Q': this thread scales the channels of chunk qj for the heads 4 qgd .. 4 qgd + 3
-    const int cw = warp - kTcFirstConvertWarp;              // = panel of 64 channels
-    const int qj = 8 * cw + (lane >> 2), qgd = lane & 3;
-    uint32_t qh[4][4];                                      // fp16 pairs of the query: [head][channel pair]
+    // Q' and the key constants: warp cw owns the panel of 64 channels cw; lane (n, c4) = (lane / 4, lane % 4)
+    // holds the heads n and n + 8 on the 16 channels 64 cw + 16 c4 .. + 15 (chunks qj0 and qj0 + 1) as fp16
+    // pairs.  That is at once the B-fragment layout of mma.m16n8k16 for a contraction over the panel's
+    // channels taken in the order "k-step ks, index k = 2 c4 + e (+ 8)  <->  channel 16 c4 + 4 ks + e (+ 2)":
+    // the key constants sum_c q[c] z[c] come from eight legacy MMAs per warp (A rows 0, 1 = the zero points of
+    // the two half blocks), and the same registers times the scales give the Q' rows.
+    const int cw = warp - kTcFirstConvertWarp;
+    const int qn = lane >> 2, qc4 = lane & 3;
+    const int qj0 = 8 * cw + 2 * qc4;
+    uint32_t qf[2][8];                                      // [head n + 8 t][channel pair i of the lane's 16 channels]
 #pragma unroll
-    for (int hh = 0; hh < 4; ++hh) {
-      const uint4 v = t_ldg128(qg + (4 * qgd + hh) * kMlaDk + 8 * qj);
-      qh[hh][0] = tc_bf2_to_h2(v.x);
-      qh[hh][1] = tc_bf2_to_h2(v.y);
-      qh[hh][2] = tc_bf2_to_h2(v.z);
-      qh[hh][3] = tc_bf2_to_h2(v.w);
+    for (int tq = 0; tq < 2; ++tq) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const uint4 v = t_ldg128(qg + (qn + 8 * tq) * kMlaDk + 8 * (qj0 + e));
+        qf[tq][4 * e + 0] = tc_bf2_to_h2(v.x);
+        qf[tq][4 * e + 1] = tc_bf2_to_h2(v.y);
+        qf[tq][4 * e + 2] = tc_bf2_to_h2(v.z);
+        qf[tq][4 * e + 3] = tc_bf2_to_h2(v.w);
+      }
     }
     // The packed codes of a tile's quantised block (w) and the scales and zero points of the
     // thread's Q' chunk (svh, zvh) are asked for one tile ahead: the codes of the next tile as soon as
@@ -664,15 +679,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
     int tg = 0;
     bool ok = true;
     uint2 w[2][8];
-    uint4 svh[2], zvh[2];
+    uint4 svh[2][2], zvh[2];        // scales [half][chunk of the lane]; zero points of half (n & 1), both chunks
     auto load_params = [&](const TcTile& x) {
       const uint8_t* slot = p.arena + static_cast<size_t>(x.off256) * 256;
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         const uint8_t* prm = slot + static_cast<size_t>(half) * mla_half_bytes(x.level);
-        svh[half] = t_ldg128(prm + 16 * qj);
-        zvh[half] = t_ldg128(prm + 2 * kMlaZeroOff + 16 * qj);
+        svh[half][0] = t_ldg128(prm + 16 * qj0);
+        svh[half][1] = t_ldg128(prm + 16 * qj0 + 16);
       }
+      const uint8_t* zp = slot + static_cast<size_t>(qn & 1) * mla_half_bytes(x.level) + 2 * kMlaZeroOff + 16 * qj0;
+      zvh[0] = t_ldg128(zp);
+      zvh[1] = t_ldg128(zp + 16);
     };
     TableEntry pre = tc_entry(p, table, cd.item_begin);
     bool have = tc_next(p, table, cd.item_end, cd.item_begin, pre, t);
@@ -707,36 +725,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       __syncwarp();
       if (lane == 0) t_bar_arrive(bar(kBarKtFull, b));
       PROF_LAP(3);
-      // Key constants sum_c q[c] z[c] per (half, head): this thread's chunk, then the warp's eight chunks
-      // (lanes with the same head quad) in a fixed order.  Formed before the wait for the Q' buffer.
+      // Key constants sum_c q[c] z[c] per (half, head) over the warp's panel: D[half][head] = Z Q^T on the
+      // legacy tensor-core path (products of two fp16 numbers are exact, the sums are fp32).  Row r of A is
+      // the zero-point row of half r & 1 (only rows 0 and 1 are read back), so the lanes 0-3 end up with
+      // half 0 and the lanes 4-7 with half 1, heads 2 c4, 2 c4 + 1 (+ 8).  Formed before the wait for the
+      // Q' buffer.
       {
-        float cacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
         if (t.kind == 0) {
-          const uint32_t zw[2][4] = {{zvh[0].x, zvh[0].y, zvh[0].z, zvh[0].w}, {zvh[1].x, zvh[1].y, zvh[1].z, zvh[1].w}};
+          const uint32_t zr[8] = {zvh[0].x, zvh[0].y, zvh[0].z, zvh[0].w, zvh[1].x, zvh[1].y, zvh[1].z, zvh[1].w};
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 za = __half22float2(t_h2(zw[0][i])), zb = __half22float2(t_h2(zw[1][i]));
-#pragma unroll
-            for (int hh = 0; hh < 4; ++hh) {
-              const float2 qf = __half22float2(t_h2(qh[hh][i]));
-              cacc[0][hh] = fmaf(qf.y, za.y, fmaf(qf.x, za.x, cacc[0][hh]));
-              cacc[1][hh] = fmaf(qf.y, zb.y, fmaf(qf.x, zb.x, cacc[1][hh]));
-            }
-          }
-#pragma unroll
-          for (int d = 4; d <= 16; d <<= 1) {
-#pragma unroll
-            for (int hh = 0; hh < 4; ++hh) {
-              cacc[0][hh] += __shfl_xor_sync(kFullT, cacc[0][hh], d);
-              cacc[1][hh] += __shfl_xor_sync(kFullT, cacc[1][hh], d);
-            }
+          for (int ks = 0; ks < 4; ++ks) {
+            t_mma_sync_f16(c0, zr[2 * ks], zr[2 * ks], zr[2 * ks + 1], zr[2 * ks + 1], qf[0][2 * ks], qf[0][2 * ks + 1]);
+            t_mma_sync_f16(c1, zr[2 * ks], zr[2 * ks], zr[2 * ks + 1], zr[2 * ks + 1], qf[1][2 * ks], qf[1][2 * ks + 1]);
           }
         }
-        if (lane < 4) {
-#pragma unroll
-          for (int half = 0; half < 2; ++half)
-            *reinterpret_cast<float4*>(cpart_sm + ((b * 2 + half) * kTcConvertWarps + cw) * 16 + 4 * lane) =
-                make_float4(cacc[half][0], cacc[half][1], cacc[half][2], cacc[half][3]);
+        if (lane < 8) {
+          float* dst = cpart_sm + ((b * 2 + qn) * kTcConvertWarps + cw) * 16 + 2 * qc4;
+          *reinterpret_cast<float2*>(dst) = make_float2(c0[0], c0[1]);
+          *reinterpret_cast<float2*>(dst + 8) = make_float2(c1[0], c1[1]);
         }
       }
       // the next tile's codes: the first half block now, the second once this tile's Q' is written (the
@@ -752,22 +759,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) mla_tc_decode_kernel(const __gr
       const __half2 f16 = __float2half2_rn((quant && t.level == 4) ? 16.f : 1.f);     // the b = 0 channel pairs of a 4-bit chunk
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
-        uint32_t sw[4] = {svh[half].x, svh[half].y, svh[half].z, svh[half].w};
-        if (!quant) sw[0] = sw[1] = sw[2] = sw[3] = 0x3C003C00u;                      // exact and centroid rows: scale 1
-        sw[0] = t_u(__hmul2(t_h2(sw[0]), f16));
-        sw[2] = t_u(__hmul2(t_h2(sw[2]), f16));
 #pragma unroll
-        for (int hh = 0; hh < 4; ++hh) {
-          uint32_t hi[4], lo[4];
+        for (int e = 0; e < 2; ++e) {
+          uint32_t sw[4] = {svh[half][e].x, svh[half][e].y, svh[half][e].z, svh[half][e].w};
+          if (!quant) sw[0] = sw[1] = sw[2] = sw[3] = 0x3C003C00u;                      // exact and centroid rows: scale 1
+          sw[0] = t_u(__hmul2(t_h2(sw[0]), f16));
+          sw[2] = t_u(__hmul2(t_h2(sw[2]), f16));
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const __half2 h = __hmul2(t_h2(qh[hh][i]), t_h2(sw[i]));
-            hi[i] = t_u(h);
-            lo[i] = t_u(__hfma2(t_h2(qh[hh][i]), t_h2(sw[i]), __hneg2(h)));
+          for (int tq = 0; tq < 2; ++tq) {
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const __half2 h = __hmul2(t_h2(qf[tq][4 * e + i]), t_h2(sw[i]));
+              hi[i] = t_u(h);
+              lo[i] = t_u(__hfma2(t_h2(qf[tq][4 * e + i]), t_h2(sw[i]), __hneg2(h)));
+            }
+            const int row = 32 * half + qn + 8 * tq;          // column of S: half, (hi | lo), head
+            t_sts128(tc_tile_addr(qp, row, qj0 + e), hi[0], hi[1], hi[2], hi[3]);
+            t_sts128(tc_tile_addr(qp, row + 16, qj0 + e), lo[0], lo[1], lo[2], lo[3]);
           }
-          const int row = 32 * half + 4 * qgd + hh;           // column of S: half, (hi | lo), head
-          t_sts128(tc_tile_addr(qp, row, qj), hi[0], hi[1], hi[2], hi[3]);
-          t_sts128(tc_tile_addr(qp, row + 16, qj), lo[0], lo[1], lo[2], lo[3]);
         }
       }
       t_fence_async();
