@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgkv.so")
-SOURCES = ["gkv_api.cu", "gkv_decode.cu", "gkv_pack.cu", "gkv_ingest.cu", "gkv_quest.cu", "gkv_rdplan.cu", "gkv_mla.cu", "gkv_mla_tc.cu"]
+SOURCES = ["gkv_api.cu", "gkv_decode.cu", "gkv_pack.cu", "gkv_ingest.cu", "gkv_quest.cu", "gkv_rdplan.cu", "gkv_mla.cu", "gkv_mla_decode.cu"]
 HEADERS = ["gkv_internal.h", "gkv_layout.cuh", "gkv_mla.h", os.path.join("..", "..", "include", "gkv.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

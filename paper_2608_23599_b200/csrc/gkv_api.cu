@@ -1042,6 +1042,7 @@ void mla_build_descs(gkv_cache* c, LayerState& L) {
     total += cost[s];
   }
   const size_t target = std::max<size_t>(800, (total + kMlaTargetCtas - 1) / kMlaTargetCtas);
+  std::vector<WarpDesc> cta(static_cast<size_t>(kMlaTargetCtas) + 2 * ns);
   int w = 0;
   for (int s = 0; s < ns; ++s) {
     int nw = static_cast<int>((cost[s] + target / 2) / target);
@@ -1058,11 +1059,28 @@ void mla_build_descs(gkv_cache* c, LayerState& L) {
         acc += mla_item_cost(c, L, s, item);
         ++item;
       } while (item < max_end && acc < limit);
-      L.warps_h[w] = WarpDesc{s, begin, item, w};
+      cta[w] = WarpDesc{s, begin, item, w};
       ++w;
     }
-    L.warps_h[w - 1].item_end = n_items;
+    cta[w - 1].item_end = n_items;
     L.parts_h[s].end = w;
+  }
+  // a CTA's range is cut once more, by cost, into the contiguous ranges of its quads (descriptor
+  // kMlaQuads * cta + quad; all of them name the CTA's partial row)
+  for (int i = 0; i < w; ++i) {
+    size_t tot = 0;
+    for (int it = cta[i].item_begin; it < cta[i].item_end; ++it) tot += mla_item_cost(c, L, cta[i].stream, it);
+    size_t acc = 0;
+    int item = cta[i].item_begin;
+    for (int qd = 0; qd < kMlaQuads; ++qd) {
+      const size_t limit = tot * (qd + 1) / kMlaQuads;
+      const int begin = item;
+      while (item < cta[i].item_end && (qd == kMlaQuads - 1 || acc + mla_item_cost(c, L, cta[i].stream, item) / 2 < limit)) {
+        acc += mla_item_cost(c, L, cta[i].stream, item);
+        ++item;
+      }
+      L.warps_h[kMlaQuads * i + qd] = WarpDesc{cta[i].stream, begin, item, cta[i].partial};
+    }
   }
   L.n_warps = w;                  // here: number of CTAs
   L.desc_dirty = false;
@@ -1227,7 +1245,7 @@ int mla_decode(gkv_cache* c, LayerState& L, const void* q, float* out, float* ls
     int rc = wait_event(c, L.ev_desc);
     if (rc != GKV_OK) return rc;
     mla_build_descs(c, L);
-    if ((rc = upload(c, L.warps_d, L.warps_h, static_cast<size_t>(L.n_warps) * sizeof(WarpDesc), st, L.ev_desc)) != GKV_OK) return rc;
+    if ((rc = upload(c, L.warps_d, L.warps_h, static_cast<size_t>(L.n_warps) * kMlaQuads * sizeof(WarpDesc), st, L.ev_desc)) != GKV_OK) return rc;
     if ((rc = upload(c, L.parts_d, L.parts_h, static_cast<size_t>(c->n_streams) * sizeof(StreamParts), st, L.ev_desc)) != GKV_OK) return rc;
   }
   MlaDecodeParams p{};

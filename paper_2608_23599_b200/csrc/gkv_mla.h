@@ -5,6 +5,7 @@
 namespace gkv {
 
 constexpr int kMlaPartialFloats = kMlaHeads * (kMlaDv + 2);   // per CTA partial: m, l, o[512] per head
+constexpr int kMlaQuads = 3;                                  // groups of four warps per CTA of the decode kernel, each with a block range of its own
 
 struct MlaEncodeParams {
   uint8_t* arena;
@@ -18,7 +19,7 @@ struct MlaEncodeParams {
 struct MlaDecodeParams {
   const uint8_t* arena;
   const TableEntry* table;  // [n_streams][table_stride]
-  const WarpDesc* ctas;     // one descriptor per CTA: a contiguous item range of one stream
+  const WarpDesc* ctas;     // kMlaQuads descriptors per CTA: contiguous item ranges of one stream, one partial row
   const uint16_t* q;        // bf16 [batch][16][576]
   float* partial;           // [n_ctas][kMlaPartialFloats]
   int32_t table_stride, n_closed, n_tail;

@@ -1,0 +1,839 @@
+// Decode attention for latent-attention (MLA) streams (Sec. 3.1 read path applied to a 576-wide
+// latent row that is key and value at once), on warp-level tensor-core instructions.
+//
+// A quantised latent row is k~[c] = s[c] * code[c] + z[c] with one (s, z) pair per channel and
+// half block (32 tokens, Sec. 3.2).  Nothing rounded ever becomes a tensor-core operand:
+//   * codes are used as they are stored: a code in the mantissa of an fp16 with a zero exponent
+//     field is the number code * 2^(b - 24), b its lowest bit (8-bit codes b = 0; 4-bit codes b = 0
+//     or 4), taken out of the packed words with byte permutes and masks only;
+//   * the scales go into the query, Q'[c][head] = q[c][head] * s[c] as an fp16 pair hi + lo (the
+//     product of an 8-bit and an 11-bit mantissa has 19 bits), formed in registers in the
+//     B-fragment layout once per half block; sum_c q[c] z[c] comes from one more MMA per channel
+//     slab whose A rows all hold the zero points;
+//   * O^T[512 x 16] += V~^T P^T reads the same packed codes a second time with tokens along k and
+//     channels along m; the probabilities are an fp16 pair hi + lo; the per-channel scale and the
+//     zero point (times the half block's probability sum) are applied in fp32 to the half block's
+//     accumulator before it is added to the running O^T, which stays in registers;
+//   * exact rows, the tail and centroid rows (one row per block, +log2(64) on the logit) are bf16
+//     operands of bf16 MMAs, the probabilities a bf16 pair hi + lo.
+//
+// Work split: a CTA is three groups of four warps ("quads").  A quad walks its own contiguous range
+// of the stream's blocks in units of one half block (quantised) or 16 rows (exact, tail, centroid
+// runs); a unit is staged by one bulk copy (or one per row) into the quad's two-stage ring.  Inside
+// a quad warp w owns the value channels [128 w, 128 w + 128) and the rope channels
+// [512 + 16 w, 512 + 16 w + 16): it computes the partial logits of its 144 channels for all tokens
+// and heads of the unit, the four partials are exchanged through shared memory (added in warp
+// order, so all four warps hold the same logits bit for bit), every warp runs the same online
+// softmax, and then accumulates its own 128 rows of O^T.  A lane group g = lane / 4 owns the 16
+// channels 128 w + 16 g .. + 15: M-tile mu of the value MMAs has row g = channel 2 mu and row
+// g + 8 = channel 2 mu + 1 of them, for every kind of unit.
+//
+// At the end the quads' (m, l, O^T) are merged in shared memory into the CTA's partial row; the
+// partial rows of a stream's CTAs are merged by mla_combine_kernel in CTA order.  Every wait is
+// bounded; on a time-out the CTA raises kStatusInternal and publishes an empty partial.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "gkv_internal.h"
+#include "gkv_layout.cuh"
+#include "gkv_mla.h"
+
+namespace gkv {
+namespace {
+
+constexpr int kMThreads = kMlaQuads * 128;
+constexpr int kMStageBytes = 20736;                    // one 8-bit half block: params 2304 + 32 x 576
+constexpr int kMStages = 2;
+constexpr int kMRowPitch = kMlaRowBytes + 16;          // bf16 rows staged at this pitch (conflict-free ldmatrix)
+constexpr int kMQPitch = kMlaRowBytes + 16;            // query rows in shared memory (fp16 and bf16 copies)
+constexpr int kMXPitch = 40;                           // floats per (warp, head) row of the exchange buffer
+constexpr int kMXBytes = 4 * kMlaHeads * kMXPitch * 4; // 10240
+constexpr int kMOffQ16 = 0;
+constexpr int kMOffQbf = kMlaHeads * kMQPitch;         // 18688
+constexpr int kMOffQuad = 2 * kMlaHeads * kMQPitch;    // 37376
+constexpr int kMQuadBytes = kMStages * kMStageBytes + kMXBytes + 64;   // stages | exchange | mbarriers
+constexpr int kMOffFlag = kMOffQuad + kMlaQuads * kMQuadBytes;
+constexpr int kMSmem = kMOffFlag + 16;
+constexpr int kMOutPitch = kMlaDv + 2;                 // floats per head row of a quad's result in shared memory
+constexpr int kMWaitSpins = 1 << 22;
+constexpr float kMNegInf = -INFINITY;
+constexpr float kMSlack = 8.f;                         // keep a stale running max while logits stay within 2^8 of it
+constexpr uint32_t kMFull = 0xffffffffu;
+static_assert(kMStageBytes >= 16 * kMRowPitch, "a stage holds 16 staged rows");
+static_assert(kMStages * kMStageBytes >= kMlaHeads * kMOutPitch * 4 + 128, "a quad's result fits its stages");
+
+// ---- PTX helpers -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t m_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void m_bar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void m_fence_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+__device__ __forceinline__ void m_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void m_bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ bool m_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// bounded wait; false after kMWaitSpins failed polls
+__device__ __forceinline__ bool m_wait(uint32_t bar, uint32_t parity) {
+  for (int i = 0; i < kMWaitSpins; ++i) {
+    if (m_try_wait(bar, parity)) return true;
+    if (i > 64) __nanosleep(64);
+  }
+  return false;
+}
+__device__ __forceinline__ void m_quad_sync(int quad) { asm volatile("bar.sync %0, 128;\n" ::"r"(quad + 1) : "memory"); }
+__device__ __forceinline__ uint4 m_lds128(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint2 m_lds64(uint32_t a) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint32_t m_lds32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ float2 m_ldsf2(uint32_t a) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];\n" : "=f"(v.x), "=f"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void m_stsf(uint32_t a, float v) { asm volatile("st.shared.f32 [%0], %1;\n" ::"r"(a), "f"(v) : "memory"); }
+__device__ __forceinline__ void m_stsf2(uint32_t a, float x, float y) {
+  asm volatile("st.shared.v2.f32 [%0], {%1,%2};\n" ::"r"(a), "f"(x), "f"(y) : "memory");
+}
+__device__ __forceinline__ void m_sts128(uint32_t a, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+  asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"r"(a), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ uint32_t m_prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t r;
+  asm("prmt.b32 %0, %1, %2, %3;\n" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+  return r;
+}
+__device__ __forceinline__ float m_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ __half2 m_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
+__device__ __forceinline__ uint32_t m_u(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
+__device__ __forceinline__ uint32_t m_ubf(__nv_bfloat162 h) { return *reinterpret_cast<uint32_t*>(&h); }
+__device__ __forceinline__ void m_mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void m_mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void m_ldmatrix4(uint32_t a, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+// q * s as an fp16 pair: hi = the rounded product, lo = the exact remainder
+__device__ __forceinline__ void m_split(uint32_t q, uint32_t s, uint32_t& hi, uint32_t& lo) {
+  const __half2 h = __hmul2(m_h2(q), m_h2(s));
+  hi = m_u(h);
+  lo = m_u(__hfma2(m_h2(q), m_h2(s), __hneg2(h)));
+}
+__device__ __forceinline__ uint32_t m_bf2_to_h2(uint32_t u) {
+  return m_u(__floats2half2_rn(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)));
+}
+// 4-bit field n of both 16-bit halves of a packed word, left where it is (weight 2^(4 (n & 1)))
+template <int N>
+__device__ __forceinline__ uint32_t m_fld4(uint32_t w) {
+  const uint32_t v = (N & 2) ? (w >> 8) : w;
+  return v & ((N & 1) ? 0x00F000F0u : 0x000F000Fu);
+}
+__device__ __forceinline__ float m_h2f(uint32_t pair, int hi) {
+  return hi ? __high2float(m_h2(pair)) : __low2float(m_h2(pair));
+}
+
+// ---- units -------------------------------------------------------------------------------------
+// A quad's range of blocks is walked in units: one half block of a quantised block (kind 0), 16 rows
+// of an exact block or of the tail (kind 1), or a run of up to 16 neighbouring centroid blocks, one
+// row each (kind 2).  (m_load is called by whole, converged warps: the run is found with a ballot.)
+struct MWalk {
+  int it, sub, nsub;     // item, unit inside the item, units of the item
+  int kind, level;
+  int nrows;             // rows of the item (kind 1) or of the run (kind 2)
+  int run;               // blocks the item covers
+  uint32_t off256;
+};
+
+__device__ __forceinline__ bool m_load(const MlaDecodeParams& p, const TableEntry* table, int item_end, MWalk& w) {
+  if (w.it >= item_end) return false;
+  const TableEntry e = table[min(w.it, p.n_closed)];
+  w.off256 = e.off256;
+  w.level = static_cast<int>(e.level);
+  w.sub = 0;
+  w.run = 1;
+  if (w.it == p.n_closed) {                        // the tail: exact rows, the last item of the stream
+    if (p.n_tail == 0) return false;
+    w.kind = 1;
+    w.nrows = p.n_tail;
+    w.nsub = (p.n_tail + 15) >> 4;
+    return true;
+  }
+  if (w.level == 16) {
+    w.kind = 1;
+    w.nrows = kBlock;
+    w.nsub = 4;
+  } else if (w.level == 1) {
+    const int lim = min(min(item_end, p.n_closed) - w.it, 16);
+    const int ln = static_cast<int>(threadIdx.x & 31);
+    const bool c = ln < lim && table[w.it + ln].level == 1u;
+    const uint32_t b = __ballot_sync(kMFull, c);
+    w.run = __ffs(~b) - 1;                         // first lane that is not a centroid block (lanes >= 16 never are)
+    w.kind = 2;
+    w.nrows = w.run;
+    w.nsub = 1;
+  } else {
+    w.kind = 0;
+    w.nrows = kBlock;
+    w.nsub = 2;
+  }
+  return true;
+}
+__device__ __forceinline__ bool m_advance(const MlaDecodeParams& p, const TableEntry* table, int item_end, MWalk& w) {
+  if (++w.sub < w.nsub) return true;
+  w.it += w.run;
+  return m_load(p, table, item_end, w);
+}
+// valid rows of the current unit of a walk of kind 1 or 2
+__device__ __forceinline__ int m_unit_rows(const MWalk& w) { return min(16, w.nrows - 16 * w.sub); }
+
+// Start the copies of a unit into a stage (one warp, converged).  Rows past the end of a row unit
+// are written as zeros so that 0 * garbage never produces a NaN.
+__device__ __forceinline__ void m_issue(const MlaDecodeParams& p, const TableEntry* table, const MWalk& w, uint32_t st, uint32_t bar,
+                                        int lane) {
+  if (w.kind == 0) {
+    if (lane == 0) {
+      const uint32_t bytes = static_cast<uint32_t>(mla_half_bytes(w.level));
+      m_expect_tx(bar, bytes);
+      m_bulk_g2s(st, p.arena + static_cast<size_t>(w.off256) * 256 + static_cast<size_t>(w.sub) * bytes, bytes, bar);
+    }
+    return;
+  }
+  const int n = m_unit_rows(w);
+  if (lane == 0) m_expect_tx(bar, static_cast<uint32_t>(n) * kMlaRowBytes);
+  __syncwarp();
+  if (lane < n) {
+    const uint8_t* src = (w.kind == 2) ? p.arena + static_cast<size_t>(table[w.it + lane].off256) * 256
+                                       : p.arena + static_cast<size_t>(w.off256) * 256 + static_cast<size_t>(16 * w.sub + lane) * kMlaRowBytes;
+    m_bulk_g2s(st + lane * kMRowPitch, src, kMlaRowBytes, bar);
+  }
+  if (n < 16) {
+    for (int idx = lane; idx < (16 - n) * (kMlaRowBytes / 16); idx += 32) {
+      const int r = n + idx / (kMlaRowBytes / 16), piece = idx % (kMlaRowBytes / 16);
+      m_sts128(st + r * kMRowPitch + piece * 16, 0u, 0u, 0u, 0u);
+    }
+    m_fence_async();
+  }
+}
+
+// ---- softmax -------------------------------------------------------------------------------------
+// The four warps' partial logits -> this lane's share of the unit's probabilities.  A lane holds, for
+// the heads g and g + 8, the tokens 16 ks + 8 j + 2 c4 + e: the B-fragment layout of the value MMAs.
+// The running maximum may stay stale by up to kMSlack (then nothing is rescaled); when it moves, the
+// running sums and O^T are rescaled.  Outputs: the probabilities as a pair hi + lo (fp16 or bf16) and
+// the unit's probability sums of the heads 2 c4 + e (+ 8 hg), the columns of the lane's O^T registers.
+template <int NKS, bool BF16>
+__device__ __forceinline__ void m_softmax(uint32_t xb, int g, int c4, float scale_log2, float bias, int nvalid, float (&O)[8][2][4],
+                                          float (&m_run)[2], float (&l_run)[2], uint32_t (&ph)[2][NKS][2], uint32_t (&pl)[2][NKS][2],
+                                          float (&psc)[2][2]) {
+  float x[2][NKS][2][2];
+  float mloc[2];
+#pragma unroll
+  for (int hg = 0; hg < 2; ++hg) {
+    mloc[hg] = kMNegInf;
+#pragma unroll
+    for (int ks = 0; ks < NKS; ++ks) {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const uint32_t a = xb + (((g + 8 * hg) * kMXPitch) + 16 * ks + 8 * j + 2 * c4) * 4;
+        float2 acc = m_ldsf2(a);
+#pragma unroll
+        for (int w = 1; w < 4; ++w) {
+          const float2 v = m_ldsf2(a + w * kMlaHeads * kMXPitch * 4);
+          acc.x += v.x;
+          acc.y += v.y;
+        }
+        const int tok = 16 * ks + 8 * j + 2 * c4;
+        x[hg][ks][j][0] = tok < nvalid ? fmaf(acc.x, scale_log2, bias) : kMNegInf;
+        x[hg][ks][j][1] = tok + 1 < nvalid ? fmaf(acc.y, scale_log2, bias) : kMNegInf;
+        mloc[hg] = fmaxf(mloc[hg], fmaxf(x[hg][ks][j][0], x[hg][ks][j][1]));
+      }
+    }
+    mloc[hg] = fmaxf(mloc[hg], __shfl_xor_sync(kMFull, mloc[hg], 1));
+    mloc[hg] = fmaxf(mloc[hg], __shfl_xor_sync(kMFull, mloc[hg], 2));
+  }
+  const bool mine = mloc[0] > m_run[0] + kMSlack || mloc[1] > m_run[1] + kMSlack;   // also the first finite logit (max = -inf)
+  if (__any_sync(kMFull, mine)) {
+    float al[2];
+#pragma unroll
+    for (int hg = 0; hg < 2; ++hg) {
+      const float mn = fmaxf(m_run[hg], mloc[hg]);
+      al[hg] = (m_run[hg] == kMNegInf) ? 0.f : m_ex2(m_run[hg] - mn);
+      m_run[hg] = mn;
+      l_run[hg] *= al[hg];
+    }
+    // the factors of the heads 2 c4 + e + 8 hg sit in the lanes whose g is 2 c4 + e
+    float ac[2][2];
+#pragma unroll
+    for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) ac[hg][e] = __shfl_sync(kMFull, al[hg], 4 * (2 * c4 + e));
+#pragma unroll
+    for (int mu = 0; mu < 8; ++mu)
+#pragma unroll
+      for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) O[mu][hg][i] *= ac[hg][i & 1];
+  }
+  float ps[2];
+#pragma unroll
+  for (int hg = 0; hg < 2; ++hg) {
+    ps[hg] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < NKS; ++ks) {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const float p0 = x[hg][ks][j][0] == kMNegInf ? 0.f : m_ex2(x[hg][ks][j][0] - m_run[hg]);
+        const float p1 = x[hg][ks][j][1] == kMNegInf ? 0.f : m_ex2(x[hg][ks][j][1] - m_run[hg]);
+        ps[hg] += p0 + p1;
+        if constexpr (BF16) {
+          const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+          ph[hg][ks][j] = m_ubf(h);
+          pl[hg][ks][j] = m_ubf(__floats2bfloat162_rn(p0 - __low2float(h), p1 - __high2float(h)));
+        } else {
+          const __half2 h = __floats2half2_rn(p0, p1);
+          ph[hg][ks][j] = m_u(h);
+          pl[hg][ks][j] = m_u(__floats2half2_rn(p0 - __low2float(h), p1 - __high2float(h)));
+        }
+      }
+    }
+    l_run[hg] += ps[hg];
+    ps[hg] += __shfl_xor_sync(kMFull, ps[hg], 1);
+    ps[hg] += __shfl_xor_sync(kMFull, ps[hg], 2);
+  }
+#pragma unroll
+  for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) psc[hg][e] = __shfl_sync(kMFull, ps[hg], 4 * (2 * c4 + e));
+}
+
+// ---- a quantised half block ---------------------------------------------------------------------
+// Key MMAs of one channel slab (16 channels = the four lanes' four channels each).  a[mt] = the A
+// fragments of the two token tiles; (s0, s1) the scales, (z0, z1) the zero points and (q0, q1) the
+// query entries (per head group) of the lane's channel pairs k = 2 c4, 2 c4 + 1 and k = 2 c4 + 8, 2 c4 + 9.
+__device__ __forceinline__ void m_slab(const uint32_t (&a)[2][4], uint32_t s0, uint32_t s1, uint32_t z0, uint32_t z1, const uint32_t (&q0)[2],
+                                       const uint32_t (&q1)[2], float (&S)[2][2][4], float (&Z)[2][4]) {
+#pragma unroll
+  for (int hg = 0; hg < 2; ++hg) {
+    m_mma_f16(Z[hg], z0, z0, z1, z1, q0[hg], q1[hg]);
+    uint32_t h0, l0, h1, l1;
+    m_split(q0[hg], s0, h0, l0);
+    m_split(q1[hg], s1, h1, l1);
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      m_mma_f16(S[mt][hg], a[mt][0], a[mt][1], a[mt][2], a[mt][3], h0, h1);
+      m_mma_f16(S[mt][hg], a[mt][0], a[mt][1], a[mt][2], a[mt][3], l0, l1);
+    }
+  }
+}
+
+template <int BITS>
+__device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t xb, int quad, int wq, int g, int c4, float scale_log2,
+                                             float (&O)[8][2][4], float (&m_run)[2], float (&l_run)[2]) {
+  constexpr int RB = kMlaChunks * BITS;                    // bytes per token row of codes
+  const uint32_t codes = st + mla_kp_bytes();
+  const uint32_t zbase = st + 2 * kMlaZeroOff;
+  const uint32_t x16 = 0x4C004C00u;                        // fp16 pair (16, 16)
+  float S[2][2][4], Z[2][4];
+#pragma unroll
+  for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) Z[hg][i] = S[0][hg][i] = S[1][hg][i] = 0.f;
+  // ---- keys: four steps of 32 value channels (8 per lane = two slabs), then the rope slab ----
+#pragma unroll
+  for (int step = 0; step < 4; ++step) {
+    const int cb = 128 * wq + 32 * step + 8 * c4;          // the lane's 8 channels
+    uint32_t w[4][2];
+#pragma unroll
+    for (int tt = 0; tt < 4; ++tt) {
+      if constexpr (BITS == 8) {
+        const uint2 v = m_lds64(codes + (g + 8 * tt) * RB + cb);
+        w[tt][0] = v.x;
+        w[tt][1] = v.y;
+      } else {
+        w[tt][0] = m_lds32(codes + (g + 8 * tt) * RB + (cb >> 1));
+        w[tt][1] = 0u;
+      }
+    }
+    const uint4 s4 = m_lds128(st + 2 * cb), z4 = m_lds128(zbase + 2 * cb);
+    const uint4 qa = m_lds128(q16 + g * kMQPitch + 2 * cb), qb = m_lds128(q16 + (g + 8) * kMQPitch + 2 * cb);
+    const uint32_t sr[4] = {s4.x, s4.y, s4.z, s4.w}, zr[4] = {z4.x, z4.y, z4.z, z4.w};
+    const uint32_t qr[2][4] = {{qa.x, qa.y, qa.z, qa.w}, {qb.x, qb.y, qb.z, qb.w}};
+#pragma unroll
+    for (int sl = 0; sl < 2; ++sl) {
+      // 8-bit: slab sl = channels 4 sl .. 4 sl + 3 (word sl, bytes c0 c2 c1 c3); 4-bit: channels 2 sl, 2 sl + 1
+      // (field sl, b = 4 sl) and 2 sl + 4, 2 sl + 5 (field sl + 2)
+      const int i0 = BITS == 8 ? 2 * sl : sl, i1 = BITS == 8 ? 2 * sl + 1 : sl + 2;
+      uint32_t s0 = sr[i0], s1 = sr[i1];
+      if (BITS == 4 && sl == 0) {                          // the b = 0 fields weigh 2^-24, the b = 4 fields 2^-20
+        s0 = m_u(__hmul2(m_h2(s0), m_h2(x16)));
+        s1 = m_u(__hmul2(m_h2(s1), m_h2(x16)));
+      }
+      uint32_t a[2][4];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        if constexpr (BITS == 8) {
+          a[mt][0] = m_prmt(w[2 * mt][sl], 0u, 0x4240u);
+          a[mt][1] = m_prmt(w[2 * mt + 1][sl], 0u, 0x4240u);
+          a[mt][2] = m_prmt(w[2 * mt][sl], 0u, 0x4341u);
+          a[mt][3] = m_prmt(w[2 * mt + 1][sl], 0u, 0x4341u);
+        } else {
+          a[mt][0] = sl ? m_fld4<1>(w[2 * mt][0]) : m_fld4<0>(w[2 * mt][0]);
+          a[mt][1] = sl ? m_fld4<1>(w[2 * mt + 1][0]) : m_fld4<0>(w[2 * mt + 1][0]);
+          a[mt][2] = sl ? m_fld4<3>(w[2 * mt][0]) : m_fld4<2>(w[2 * mt][0]);
+          a[mt][3] = sl ? m_fld4<3>(w[2 * mt + 1][0]) : m_fld4<2>(w[2 * mt + 1][0]);
+        }
+      }
+      const uint32_t q0[2] = {qr[0][i0], qr[1][i0]}, q1[2] = {qr[0][i1], qr[1][i1]};
+      m_slab(a, s0, s1, zr[i0], zr[i1], q0, q1, S, Z);
+    }
+  }
+  {
+    // the rope slab: 16 channels of the warp, four per lane
+    uint32_t a[2][4], s0, s1, z0, z1, q0[2], q1[2];
+    if constexpr (BITS == 8) {
+      const int cb = kMlaDv + 16 * wq + 4 * c4;
+      uint32_t w[4];
+#pragma unroll
+      for (int tt = 0; tt < 4; ++tt) w[tt] = m_lds32(codes + (g + 8 * tt) * RB + cb);
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        a[mt][0] = m_prmt(w[2 * mt], 0u, 0x4240u);
+        a[mt][1] = m_prmt(w[2 * mt + 1], 0u, 0x4240u);
+        a[mt][2] = m_prmt(w[2 * mt], 0u, 0x4341u);
+        a[mt][3] = m_prmt(w[2 * mt + 1], 0u, 0x4341u);
+      }
+      const uint2 s2 = m_lds64(st + 2 * cb), z2 = m_lds64(zbase + 2 * cb);
+      const uint2 qa = m_lds64(q16 + g * kMQPitch + 2 * cb), qb = m_lds64(q16 + (g + 8) * kMQPitch + 2 * cb);
+      s0 = s2.x; s1 = s2.y; z0 = z2.x; z1 = z2.y;
+      q0[0] = qa.x; q0[1] = qb.x; q1[0] = qa.y; q1[1] = qb.y;
+    } else {
+      // the lane's word is chunk c4 / 2 of the warp's two; its fields sl = c4 & 1 (channels 2 sl, 2 sl + 1)
+      // and sl + 2 (channels 2 sl + 4, 2 sl + 5)
+      const int sl = c4 & 1;
+      const int cbase = kMlaDv + 16 * wq + 8 * (c4 >> 1);
+      const uint32_t mask = sl ? 0x00F000F0u : 0x000F000Fu;
+      uint32_t w[4];
+#pragma unroll
+      for (int tt = 0; tt < 4; ++tt) w[tt] = m_lds32(codes + (g + 8 * tt) * RB + (cbase >> 1));
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        a[mt][0] = w[2 * mt] & mask;
+        a[mt][1] = w[2 * mt + 1] & mask;
+        a[mt][2] = (w[2 * mt] >> 8) & mask;
+        a[mt][3] = (w[2 * mt + 1] >> 8) & mask;
+      }
+      const int ca = cbase + 2 * sl, cbb = ca + 4;
+      const __half2 f = __float2half2_rn(sl ? 1.f : 16.f);
+      s0 = m_u(__hmul2(m_h2(m_lds32(st + 2 * ca)), f));
+      s1 = m_u(__hmul2(m_h2(m_lds32(st + 2 * cbb)), f));
+      z0 = m_lds32(zbase + 2 * ca);
+      z1 = m_lds32(zbase + 2 * cbb);
+      q0[0] = m_lds32(q16 + g * kMQPitch + 2 * ca);
+      q0[1] = m_lds32(q16 + (g + 8) * kMQPitch + 2 * ca);
+      q1[0] = m_lds32(q16 + g * kMQPitch + 2 * cbb);
+      q1[1] = m_lds32(q16 + (g + 8) * kMQPitch + 2 * cbb);
+    }
+    m_slab(a, s0, s1, z0, z1, q0, q1, S, Z);
+  }
+  // partial logits of the warp's channels -> the exchange buffer [warp][head][token]
+  {
+    const float ks = BITS == 8 ? 16777216.f : 1048576.f;
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int head = 8 * hg + 2 * c4 + (i & 1), tok = 16 * mt + g + 8 * (i >> 1);
+          m_stsf(xb + ((wq * kMlaHeads + head) * kMXPitch + tok) * 4, fmaf(S[mt][hg][i], ks, Z[hg][i]));
+        }
+  }
+  m_quad_sync(quad);
+  uint32_t ph[2][2][2], pl[2][2][2];
+  float psc[2][2];
+  m_softmax<2, false>(xb, g, c4, scale_log2, 0.f, 32, O, m_run, l_run, ph, pl, psc);
+  // ---- values: the warp's 128 channels, 16 per lane group; two passes of four M-tiles ----
+#pragma unroll
+  for (int hp = 0; hp < 2; ++hp) {
+    const int cv = 128 * wq + 16 * g + 8 * hp;               // channels of this pass
+    uint32_t w[2][4][2];                                     // [k-step][token 2 c4, 2 c4 + 1, 2 c4 + 8, 2 c4 + 9][word]
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int tok = 16 * ks + 2 * c4 + (i & 1) + 8 * (i >> 1);
+        if constexpr (BITS == 8) {
+          const uint2 v = m_lds64(codes + tok * RB + cv);
+          w[ks][i][0] = v.x;
+          w[ks][i][1] = v.y;
+        } else {
+          w[ks][i][0] = m_lds32(codes + tok * RB + (cv >> 1));
+          w[ks][i][1] = 0u;
+        }
+      }
+    const uint4 s4 = m_lds128(st + 2 * cv), z4 = m_lds128(zbase + 2 * cv);
+    const uint32_t sr[4] = {s4.x, s4.y, s4.z, s4.w}, zr[4] = {z4.x, z4.y, z4.z, z4.w};
+    uint32_t lo01[2], hi01[2], lo23[2], hi23[2];             // 4-bit: the token pairs' low and high halves
+    if constexpr (BITS == 4) {
+#pragma unroll
+      for (int ks = 0; ks < 2; ++ks) {
+        lo01[ks] = m_prmt(w[ks][0][0], w[ks][1][0], 0x5410u);
+        hi01[ks] = m_prmt(w[ks][0][0], w[ks][1][0], 0x7632u);
+        lo23[ks] = m_prmt(w[ks][2][0], w[ks][3][0], 0x5410u);
+        hi23[ks] = m_prmt(w[ks][2][0], w[ks][3][0], 0x7632u);
+      }
+    }
+#pragma unroll
+    for (int m4 = 0; m4 < 4; ++m4) {
+      // M-tile mu = 4 hp + m4: row g = channel cv + 2 m4, row g + 8 = channel cv + 2 m4 + 1
+      const int mu = 4 * hp + m4;
+      float T[2][4];
+#pragma unroll
+      for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) T[hg][i] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < 2; ++ks) {
+        uint32_t a0, a1, a2, a3;
+        if constexpr (BITS == 8) {
+          // word m4 / 2 holds the channels 4 (m4 / 2) + (0, 2, 1, 3); the pair 2 (m4 & 1), 2 (m4 & 1) + 1 sits in the
+          // bytes (m4 & 1) and (m4 & 1) + 2
+          const uint32_t sel = (m4 & 1) ? 0x7531u : 0x6420u;
+          const uint32_t y01 = m_prmt(w[ks][0][m4 >> 1], w[ks][1][m4 >> 1], sel);
+          const uint32_t y23 = m_prmt(w[ks][2][m4 >> 1], w[ks][3][m4 >> 1], sel);
+          a0 = y01 & 0x00FF00FFu;
+          a1 = (y01 >> 8) & 0x00FF00FFu;
+          a2 = y23 & 0x00FF00FFu;
+          a3 = (y23 >> 8) & 0x00FF00FFu;
+        } else {
+          a0 = m4 == 0 ? m_fld4<0>(lo01[ks]) : (m4 == 1 ? m_fld4<1>(lo01[ks]) : (m4 == 2 ? m_fld4<2>(lo01[ks]) : m_fld4<3>(lo01[ks])));
+          a1 = m4 == 0 ? m_fld4<0>(hi01[ks]) : (m4 == 1 ? m_fld4<1>(hi01[ks]) : (m4 == 2 ? m_fld4<2>(hi01[ks]) : m_fld4<3>(hi01[ks])));
+          a2 = m4 == 0 ? m_fld4<0>(lo23[ks]) : (m4 == 1 ? m_fld4<1>(lo23[ks]) : (m4 == 2 ? m_fld4<2>(lo23[ks]) : m_fld4<3>(lo23[ks])));
+          a3 = m4 == 0 ? m_fld4<0>(hi23[ks]) : (m4 == 1 ? m_fld4<1>(hi23[ks]) : (m4 == 2 ? m_fld4<2>(hi23[ks]) : m_fld4<3>(hi23[ks])));
+        }
+#pragma unroll
+        for (int hg = 0; hg < 2; ++hg) {
+          m_mma_f16(T[hg], a0, a1, a2, a3, ph[hg][ks][0], ph[hg][ks][1]);
+          m_mma_f16(T[hg], a0, a1, a2, a3, pl[hg][ks][0], pl[hg][ks][1]);
+        }
+      }
+      const float un = (BITS == 4 && (m4 & 1)) ? 1048576.f : 16777216.f;   // 2^(24 - b)
+      const float sa = m_h2f(sr[m4], 0) * un, sb = m_h2f(sr[m4], 1) * un;
+      const float za = m_h2f(zr[m4], 0), zb = m_h2f(zr[m4], 1);
+#pragma unroll
+      for (int hg = 0; hg < 2; ++hg) {
+        O[mu][hg][0] = fmaf(T[hg][0], sa, fmaf(za, psc[hg][0], O[mu][hg][0]));
+        O[mu][hg][1] = fmaf(T[hg][1], sa, fmaf(za, psc[hg][1], O[mu][hg][1]));
+        O[mu][hg][2] = fmaf(T[hg][2], sb, fmaf(zb, psc[hg][0], O[mu][hg][2]));
+        O[mu][hg][3] = fmaf(T[hg][3], sb, fmaf(zb, psc[hg][1], O[mu][hg][3]));
+      }
+    }
+  }
+}
+
+// ---- 16 bf16 rows (an exact tile, the tail, a run of centroid rows) ---------------------------------
+__device__ __forceinline__ void m_unit_rows16(uint32_t st, uint32_t qbf, uint32_t xb, int quad, int wq, int lane, float scale_log2,
+                                              float bias, int nvalid, float (&O)[8][2][4], float (&m_run)[2], float (&l_run)[2]) {
+  const int g = lane >> 2, c4 = lane & 3;
+  float S[2][4];
+#pragma unroll
+  for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) S[hg][i] = 0.f;
+  const uint32_t arow = st + (lane & 15) * kMRowPitch + 16 * (lane >> 4);
+#pragma unroll
+  for (int sl = 0; sl < 9; ++sl) {
+    const int ch0 = sl < 8 ? 128 * wq + 16 * sl : kMlaDv + 16 * wq;
+    uint32_t a[4];
+    m_ldmatrix4(arow + 2 * ch0, a);
+#pragma unroll
+    for (int hg = 0; hg < 2; ++hg) {
+      const uint32_t b0 = m_lds32(qbf + (g + 8 * hg) * kMQPitch + 2 * (ch0 + 2 * c4));
+      const uint32_t b1 = m_lds32(qbf + (g + 8 * hg) * kMQPitch + 2 * (ch0 + 8 + 2 * c4));
+      m_mma_bf16(S[hg], a[0], a[1], a[2], a[3], b0, b1);
+    }
+  }
+#pragma unroll
+  for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int head = 8 * hg + 2 * c4 + (i & 1), tok = g + 8 * (i >> 1);
+      m_stsf(xb + ((wq * kMlaHeads + head) * kMXPitch + tok) * 4, S[hg][i]);
+    }
+  m_quad_sync(quad);
+  uint32_t ph[2][1][2], pl[2][1][2];
+  float psc[2][2];
+  m_softmax<1, true>(xb, g, c4, scale_log2, bias, nvalid, O, m_run, l_run, ph, pl, psc);
+  // values: channel pairs (2 mu, 2 mu + 1) of the lane group's 16 channels from the tokens 2 c4, 2 c4 + 1, 2 c4 + 8, 2 c4 + 9
+#pragma unroll
+  for (int hp = 0; hp < 2; ++hp) {
+    uint32_t w[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int tok = 2 * c4 + (i & 1) + 8 * (i >> 1);
+      const uint4 v = m_lds128(st + tok * kMRowPitch + 2 * (128 * wq + 16 * g + 8 * hp));
+      w[i][0] = v.x; w[i][1] = v.y; w[i][2] = v.z; w[i][3] = v.w;
+    }
+#pragma unroll
+    for (int m4 = 0; m4 < 4; ++m4) {
+      const int mu = 4 * hp + m4;
+      const uint32_t a0 = m_prmt(w[0][m4], w[1][m4], 0x5410u), a1 = m_prmt(w[0][m4], w[1][m4], 0x7632u);
+      const uint32_t a2 = m_prmt(w[2][m4], w[3][m4], 0x5410u), a3 = m_prmt(w[2][m4], w[3][m4], 0x7632u);
+#pragma unroll
+      for (int hg = 0; hg < 2; ++hg) {
+        m_mma_bf16(O[mu][hg], a0, a1, a2, a3, ph[hg][0][0], ph[hg][0][1]);
+        m_mma_bf16(O[mu][hg], a0, a1, a2, a3, pl[hg][0][0], pl[hg][0][1]);
+      }
+    }
+  }
+}
+
+// ---- kernel --------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kMThreads, 1) mla_decode_kernel(const __grid_constant__ MlaDecodeParams p) {
+  extern __shared__ __align__(128) uint8_t msm[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int quad = warp >> 2, wq = warp & 3, g = lane >> 2, c4 = lane & 3;
+  const WarpDesc cd = p.ctas[blockIdx.x * kMlaQuads + quad];
+  if (p.ctas[blockIdx.x * kMlaQuads].stream < 0) return;        // uniform for the CTA
+  const uint32_t base = m_u32(msm);
+  const uint32_t q16 = base + kMOffQ16, qbf = base + kMOffQbf;
+  const uint32_t qd = base + kMOffQuad + quad * kMQuadBytes;
+  const uint32_t xb = qd + kMStages * kMStageBytes, bars = xb + kMXBytes;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(msm + kMOffFlag);
+  const TableEntry* table = p.table + static_cast<size_t>(cd.stream) * p.table_stride;
+
+  if (tid == 0) *abort_flag = 0;
+  if (wq == 0 && lane == 0) {
+    m_bar_init(bars, 1);
+    m_bar_init(bars + 8, 1);
+    m_fence_async();
+  }
+  {
+    // the query: a bf16 copy (bf16 MMAs of exact rows) and an fp16 copy (exact for the magnitudes a query has)
+    const uint16_t* qg = p.q + static_cast<size_t>(cd.stream) * kMlaHeads * kMlaDk;
+    for (int idx = tid; idx < kMlaHeads * kMlaChunks; idx += kMThreads) {
+      const int head = idx / kMlaChunks, piece = idx % kMlaChunks;
+      const uint4 v = *reinterpret_cast<const uint4*>(qg + head * kMlaDk + 8 * piece);
+      m_sts128(qbf + head * kMQPitch + 16 * piece, v.x, v.y, v.z, v.w);
+      m_sts128(q16 + head * kMQPitch + 16 * piece, m_bf2_to_h2(v.x), m_bf2_to_h2(v.y), m_bf2_to_h2(v.z), m_bf2_to_h2(v.w));
+    }
+  }
+  __syncthreads();
+
+  float O[8][2][4];
+#pragma unroll
+  for (int mu = 0; mu < 8; ++mu)
+#pragma unroll
+    for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) O[mu][hg][i] = 0.f;
+  float m_run[2] = {kMNegInf, kMNegInf}, l_run[2] = {0.f, 0.f};
+
+  MWalk wc, wl;
+  wc.it = cd.item_begin;
+  bool have_c = m_load(p, table, cd.item_end, wc);
+  wl = wc;
+  bool have_l = have_c;
+  // the first two units' copies
+#pragma unroll 1
+  for (int i = 0; i < kMStages; ++i) {
+    if (have_l) {
+      if (wq == 0) m_issue(p, table, wl, qd + i * kMStageBytes, bars + 8 * i, lane);
+      have_l = m_advance(p, table, cd.item_end, wl);
+    }
+  }
+  int k = 0;
+#pragma unroll 1
+  while (have_c) {
+    const int s = k & 1;
+    const uint32_t st = qd + s * kMStageBytes;
+    // after a time-out nothing waits any more: the remaining units run through on whatever the stages hold
+    if (!*abort_flag && !m_wait(bars + 8 * s, (k >> 1) & 1)) *abort_flag = 1;
+    if (wc.kind == 0) {
+      if (wc.level == 8) m_unit_quant<8>(st, q16, xb, quad, wq, g, c4, p.scale_log2, O, m_run, l_run);
+      else m_unit_quant<4>(st, q16, xb, quad, wq, g, c4, p.scale_log2, O, m_run, l_run);
+    } else {
+      m_unit_rows16(st, qbf, xb, quad, wq, lane, p.scale_log2, wc.kind == 2 ? 6.0f : 0.f, m_unit_rows(wc), O, m_run, l_run);
+    }
+    // the stage and the exchange buffer are free once all four warps are here
+    m_quad_sync(quad);
+    if (have_l) {
+      if (wq == 0) m_issue(p, table, wl, st, bars + 8 * s, lane);
+      have_l = m_advance(p, table, cd.item_end, wl);
+    }
+    have_c = m_advance(p, table, cd.item_end, wc);
+    ++k;
+  }
+
+  // ---- the quad's result into its (now idle) stages: O^T as [head][channel], then m and l ----
+  {
+    float l[2];
+#pragma unroll
+    for (int hg = 0; hg < 2; ++hg) {
+      l[hg] = l_run[hg] + __shfl_xor_sync(kMFull, l_run[hg], 1);
+      l[hg] += __shfl_xor_sync(kMFull, l[hg], 2);
+    }
+#pragma unroll
+    for (int mu = 0; mu < 8; ++mu)
+#pragma unroll
+      for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int head = 8 * hg + 2 * c4 + e, ch = 128 * wq + 16 * g + 2 * mu;
+          m_stsf2(qd + (head * kMOutPitch + ch) * 4, O[mu][hg][e], O[mu][hg][e + 2]);
+        }
+    if (wq == 0 && c4 == 0) {
+#pragma unroll
+      for (int hg = 0; hg < 2; ++hg) {
+        m_stsf(qd + (kMlaHeads * kMOutPitch + g + 8 * hg) * 4, m_run[hg]);
+        m_stsf(qd + (kMlaHeads * kMOutPitch + 16 + g + 8 * hg) * 4, l[hg]);
+      }
+    }
+  }
+  __syncthreads();
+  // ---- merge of the quads in quad order -> the CTA's partial row ----
+  {
+    const bool good = !*abort_flag;
+    float* out = p.partial + static_cast<size_t>(cd.partial) * kMlaPartialFloats;
+    const float* sm = reinterpret_cast<const float*>(msm + kMOffQuad);
+    constexpr int kQF = kMQuadBytes / 4;                      // floats between two quads' results
+    for (int idx = tid; idx < kMlaHeads * kMlaDv; idx += kMThreads) {
+      const int head = idx / kMlaDv, ch = idx % kMlaDv;
+      float M = kMNegInf;
+#pragma unroll
+      for (int qn = 0; qn < kMlaQuads; ++qn) M = fmaxf(M, sm[qn * kQF + kMlaHeads * kMOutPitch + head]);
+      float acc = 0.f, L = 0.f;
+#pragma unroll
+      for (int qn = 0; qn < kMlaQuads; ++qn) {
+        const float mq = sm[qn * kQF + kMlaHeads * kMOutPitch + head];
+        const float wgt = (mq == kMNegInf) ? 0.f : exp2f(mq - M);
+        acc = fmaf(wgt, sm[qn * kQF + head * kMOutPitch + ch], acc);
+        L = fmaf(wgt, sm[qn * kQF + kMlaHeads * kMOutPitch + 16 + head], L);
+      }
+      out[head * (kMlaDv + 2) + 2 + ch] = good ? acc : 0.f;
+      if (ch == 0) {
+        out[head * (kMlaDv + 2)] = good ? M : kMNegInf;
+        out[head * (kMlaDv + 2) + 1] = good ? L : 0.f;
+      }
+    }
+  }
+  if (tid == 0 && *abort_flag) atomicOr(p.status, kStatusInternal);
+}
+
+// Merge the partial rows of a stream's CTAs.  One block per (stream, head, slice of 64 value
+// channels); its 512 threads are 8 row groups x 64 channels, row group g sums rows g, g + 8, ...
+// in that order and the 8 sums are added in group order, so the result is bitwise reproducible.
+constexpr int kCombSlice = 64, kCombGroups = 8, kCombThreads = kCombSlice * kCombGroups;
+__global__ void __launch_bounds__(kCombThreads) mla_combine_kernel(const float* partial, const StreamParts* parts, float* out,
+                                                                   float* lse) {
+  __shared__ float sm_m[kCombThreads], sm_w[kCombThreads], sm_acc[kCombGroups][kCombSlice];
+  const int stream = blockIdx.x, h = blockIdx.y, slice = blockIdx.z, tid = threadIdx.x;
+  const int c = tid % kCombSlice, g = tid / kCombSlice;
+  const int begin = parts[stream].begin, end = parts[stream].end;
+  const float* base = partial + h * (kMlaDv + 2);
+  // pass 1: the maximum of the rows' maxima (one row per thread, then a shared-memory sweep)
+  float M = kMNegInf;
+  for (int c0 = begin; c0 < end; c0 += kCombThreads) {
+    const int n = min(kCombThreads, end - c0);
+    __syncthreads();
+    sm_m[tid] = tid < n ? __ldcg(base + static_cast<size_t>(c0 + tid) * kMlaPartialFloats) : kMNegInf;
+    __syncthreads();
+#pragma unroll 8
+    for (int i = 0; i < n; ++i) M = fmaxf(M, sm_m[i]);
+  }
+  // pass 2: weights per row in shared memory, then every thread sums its channel over its rows
+  float L = 0.f, acc = 0.f;
+  for (int c0 = begin; c0 < end; c0 += kCombThreads) {
+    const int n = min(kCombThreads, end - c0);
+    __syncthreads();
+    if (tid < n) {
+      const float* row = base + static_cast<size_t>(c0 + tid) * kMlaPartialFloats;
+      const float m = __ldcg(row);
+      const float w = (m == kMNegInf) ? 0.f : exp2f(m - M);
+      sm_w[tid] = w;
+      sm_m[tid] = w * __ldcg(row + 1);
+    }
+    __syncthreads();
+    const float* col = base + static_cast<size_t>(c0) * kMlaPartialFloats + 2 + slice * kCombSlice + c;
+#pragma unroll 8
+    for (int i = g; i < n; i += kCombGroups) acc = fmaf(sm_w[i], __ldcg(col + static_cast<size_t>(i) * kMlaPartialFloats), acc);
+    if (g == 0 && c == 0)
+      for (int i = 0; i < n; ++i) L += sm_m[i];
+  }
+  sm_acc[g][c] = acc;
+  __syncthreads();
+  if (g == 0) {
+    if (c == 0) sm_m[0] = L;
+  }
+  __syncthreads();
+  L = sm_m[0];
+  if (g == 0) {
+    float tot = 0.f;
+#pragma unroll
+    for (int k = 0; k < kCombGroups; ++k) tot += sm_acc[k][c];
+    const size_t hq = static_cast<size_t>(stream) * kMlaHeads + h;
+    out[hq * kMlaDv + slice * kCombSlice + c] = (L > 0.f) ? tot / L : 0.f;
+    if (lse && slice == 0 && c == 0) lse[hq] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : kMNegInf;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_mla_decode(const MlaDecodeParams& p, int n_ctas, const StreamParts* parts, int n_streams, float* out,
+                              float* lse, cudaStream_t st) {
+  if (n_ctas <= 0) return cudaSuccess;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(mla_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMSmem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  mla_decode_kernel<<<n_ctas, kMThreads, kMSmem, st>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  mla_combine_kernel<<<dim3(n_streams, kMlaHeads, kMlaDv / kCombSlice), kCombThreads, 0, st>>>(p.partial, parts, out, lse);
+  return cudaGetLastError();
+}
+
+}  // namespace gkv
