@@ -1017,16 +1017,15 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
 // One stream per sequence; staircase or external plans only.  The block table, slot heap and
 // staging are shared with the GQA path; the kernels are those of gkv_mla.cu.
 size_t mla_item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) {
-  // Cost of a block for the split of a stream over the CTAs, in units where a 4-bit block is 1000:
-  // measured on B200 as the time of a call over a cache that holds one rung only (262,144 tokens:
-  // 40.7 ns per 4-bit block, 48.9 per 8-bit block, 79.9 per exact block, 6.0 per centroid block -
-  // a tile of 64 centroid rows is gathered from 64 slots through the block table).
+  // Cost of a block for the split of a stream over the CTAs and their quads, in units where a 4-bit
+  // block is 1000: measured on B200 as the time of a call over a cache that holds one rung only
+  // (262,144 tokens), less the call's fixed part.
   if (item < L.n_closed) {
     switch (L.level[static_cast<size_t>(stream) * c->max_blocks + item]) {
-      case 16: return 1960;
-      case 8: return 1200;
+      case 16: return 1330;
+      case 8: return 1100;
       case 4: return 1000;
-      default: return 147;
+      default: return 180;
     }
   }
   return 900;                     // tail

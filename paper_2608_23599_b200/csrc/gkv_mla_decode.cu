@@ -142,14 +142,20 @@ __device__ __forceinline__ __half2 m_h2(uint32_t u) { return *reinterpret_cast<_
 __device__ __forceinline__ uint32_t m_u(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ __forceinline__ uint32_t m_ubf(__nv_bfloat162 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ __forceinline__ void m_mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// D = A B (no accumulator input: the first MMA of a chain)
+__device__ __forceinline__ void m_mma_f16_first(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};\n"
+      : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
 __device__ __forceinline__ void m_mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void m_ldmatrix4(uint32_t a, uint32_t (&r)[4]) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
@@ -178,64 +184,63 @@ __device__ __forceinline__ float m_h2f(uint32_t pair, int hi) {
 // of an exact block or of the tail (kind 1), or a run of up to 16 neighbouring centroid blocks, one
 // row each (kind 2).  (m_load is called by whole, converged warps: the run is found with a ballot.)
 struct MWalk {
-  int it, sub, nsub;     // item, unit inside the item, units of the item
-  int kind, level;
-  int nrows;             // rows of the item (kind 1) or of the run (kind 2)
-  int run;               // blocks the item covers
+  int it;                // item (block index; n_closed = the tail)
+  uint32_t meta;         // sub | nsub << 4 | kind << 8 | level << 12 | run << 20 | nrows << 25
   uint32_t off256;
+  __device__ __forceinline__ int sub() const { return static_cast<int>(meta & 15u); }        // unit inside the item
+  __device__ __forceinline__ int nsub() const { return static_cast<int>((meta >> 4) & 15u); }
+  __device__ __forceinline__ int kind() const { return static_cast<int>((meta >> 8) & 15u); }
+  __device__ __forceinline__ int level() const { return static_cast<int>((meta >> 12) & 255u); }
+  __device__ __forceinline__ int run() const { return static_cast<int>((meta >> 20) & 31u); }   // blocks the item covers
+  __device__ __forceinline__ int nrows() const { return static_cast<int>(meta >> 25); }         // rows of the item (kind 1) or run (kind 2)
 };
+__device__ __forceinline__ uint32_t m_meta(int nsub, int kind, int level, int run, int nrows) {
+  return static_cast<uint32_t>(nsub) << 4 | static_cast<uint32_t>(kind) << 8 | static_cast<uint32_t>(level) << 12 |
+         static_cast<uint32_t>(run) << 20 | static_cast<uint32_t>(nrows) << 25;
+}
 
 __device__ __forceinline__ bool m_load(const MlaDecodeParams& p, const TableEntry* table, int item_end, MWalk& w) {
   if (w.it >= item_end) return false;
   const TableEntry e = table[min(w.it, p.n_closed)];
   w.off256 = e.off256;
-  w.level = static_cast<int>(e.level);
-  w.sub = 0;
-  w.run = 1;
+  const int level = static_cast<int>(e.level);
   if (w.it == p.n_closed) {                        // the tail: exact rows, the last item of the stream
     if (p.n_tail == 0) return false;
-    w.kind = 1;
-    w.nrows = p.n_tail;
-    w.nsub = (p.n_tail + 15) >> 4;
+    w.meta = m_meta((p.n_tail + 15) >> 4, 1, 16, 1, p.n_tail);
     return true;
   }
-  if (w.level == 16) {
-    w.kind = 1;
-    w.nrows = kBlock;
-    w.nsub = 4;
-  } else if (w.level == 1) {
+  if (level == 16) {
+    w.meta = m_meta(4, 1, 16, 1, kBlock);
+  } else if (level == 1) {
     const int lim = min(min(item_end, p.n_closed) - w.it, 16);
     const int ln = static_cast<int>(threadIdx.x & 31);
     const bool c = ln < lim && table[w.it + ln].level == 1u;
     const uint32_t b = __ballot_sync(kMFull, c);
-    w.run = __ffs(~b) - 1;                         // first lane that is not a centroid block (lanes >= 16 never are)
-    w.kind = 2;
-    w.nrows = w.run;
-    w.nsub = 1;
+    const int run = __ffs(~b) - 1;                 // first lane that is not a centroid block (lanes >= 16 never are)
+    w.meta = m_meta(1, 2, 1, run, run);
   } else {
-    w.kind = 0;
-    w.nrows = kBlock;
-    w.nsub = 2;
+    w.meta = m_meta(2, 0, level, 1, kBlock);
   }
   return true;
 }
 __device__ __forceinline__ bool m_advance(const MlaDecodeParams& p, const TableEntry* table, int item_end, MWalk& w) {
-  if (++w.sub < w.nsub) return true;
-  w.it += w.run;
+  ++w.meta;                                        // sub + 1 (never carries: nsub <= 4)
+  if (w.sub() < w.nsub()) return true;
+  w.it += w.run();
   return m_load(p, table, item_end, w);
 }
 // valid rows of the current unit of a walk of kind 1 or 2
-__device__ __forceinline__ int m_unit_rows(const MWalk& w) { return min(16, w.nrows - 16 * w.sub); }
+__device__ __forceinline__ int m_unit_rows(const MWalk& w) { return min(16, w.nrows() - 16 * w.sub()); }
 
 // Start the copies of a unit into a stage (one warp, converged).  Rows past the end of a row unit
 // are written as zeros so that 0 * garbage never produces a NaN.
 __device__ __forceinline__ void m_issue(const MlaDecodeParams& p, const TableEntry* table, const MWalk& w, uint32_t st, uint32_t bar,
                                         int lane) {
-  if (w.kind == 0) {
+  if (w.kind() == 0) {
     if (lane == 0) {
-      const uint32_t bytes = static_cast<uint32_t>(mla_half_bytes(w.level));
+      const uint32_t bytes = static_cast<uint32_t>(mla_half_bytes(w.level()));
       m_expect_tx(bar, bytes);
-      m_bulk_g2s(st, p.arena + static_cast<size_t>(w.off256) * 256 + static_cast<size_t>(w.sub) * bytes, bytes, bar);
+      m_bulk_g2s(st, p.arena + static_cast<size_t>(w.off256) * 256 + static_cast<size_t>(w.sub()) * bytes, bytes, bar);
     }
     return;
   }
@@ -243,8 +248,8 @@ __device__ __forceinline__ void m_issue(const MlaDecodeParams& p, const TableEnt
   if (lane == 0) m_expect_tx(bar, static_cast<uint32_t>(n) * kMlaRowBytes);
   __syncwarp();
   if (lane < n) {
-    const uint8_t* src = (w.kind == 2) ? p.arena + static_cast<size_t>(table[w.it + lane].off256) * 256
-                                       : p.arena + static_cast<size_t>(w.off256) * 256 + static_cast<size_t>(16 * w.sub + lane) * kMlaRowBytes;
+    const uint8_t* src = (w.kind() == 2) ? p.arena + static_cast<size_t>(table[w.it + lane].off256) * 256
+                                       : p.arena + static_cast<size_t>(w.off256) * 256 + static_cast<size_t>(16 * w.sub() + lane) * kMlaRowBytes;
     m_bulk_g2s(st + lane * kMRowPitch, src, kMlaRowBytes, bar);
   }
   if (n < 16) {
@@ -351,20 +356,32 @@ __device__ __forceinline__ void m_softmax(uint32_t xb, int g, int c4, float scal
 // Key MMAs of one channel slab (16 channels = the four lanes' four channels each).  a[mt] = the A
 // fragments of the two token tiles; (s0, s1) the scales, (z0, z1) the zero points and (q0, q1) the
 // query entries (per head group) of the lane's channel pairs k = 2 c4, 2 c4 + 1 and k = 2 c4 + 8, 2 c4 + 9.
+// sum_c q[c] z[c] takes one MMA for all sixteen heads: the query registers are at once the A fragment
+// of Q^T (rows = heads g and g + 8), the zero points fill every column of B, and Zt[0] / Zt[2] end up as
+// the sums of the heads g / g + 8.
+template <bool FIRST>
 __device__ __forceinline__ void m_slab(const uint32_t (&a)[2][4], uint32_t s0, uint32_t s1, uint32_t z0, uint32_t z1, const uint32_t (&q0)[2],
-                                       const uint32_t (&q1)[2], float (&S)[2][2][4], float (&Z)[2][4]) {
+                                       const uint32_t (&q1)[2], float (&S)[2][2][4], float (&Zt)[4]) {
+  uint32_t h0[2], l0[2], h1[2], l1[2];
 #pragma unroll
   for (int hg = 0; hg < 2; ++hg) {
-    m_mma_f16(Z[hg], z0, z0, z1, z1, q0[hg], q1[hg]);
-    uint32_t h0, l0, h1, l1;
-    m_split(q0[hg], s0, h0, l0);
-    m_split(q1[hg], s1, h1, l1);
+    m_split(q0[hg], s0, h0[hg], l0[hg]);
+    m_split(q1[hg], s1, h1[hg], l1[hg]);
+  }
+  if (FIRST) m_mma_f16_first(Zt, q0[0], q0[1], q1[0], q1[1], z0, z1);
+  else m_mma_f16(Zt, q0[0], q0[1], q1[0], q1[1], z0, z1);
+  // four accumulator chains; the two MMAs of a chain are kept four apart
+#pragma unroll
+  for (int hg = 0; hg < 2; ++hg)
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
-      m_mma_f16(S[mt][hg], a[mt][0], a[mt][1], a[mt][2], a[mt][3], h0, h1);
-      m_mma_f16(S[mt][hg], a[mt][0], a[mt][1], a[mt][2], a[mt][3], l0, l1);
+      if (FIRST) m_mma_f16_first(S[mt][hg], a[mt][0], a[mt][1], a[mt][2], a[mt][3], h0[hg], h1[hg]);
+      else m_mma_f16(S[mt][hg], a[mt][0], a[mt][1], a[mt][2], a[mt][3], h0[hg], h1[hg]);
     }
-  }
+#pragma unroll
+  for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) m_mma_f16(S[mt][hg], a[mt][0], a[mt][1], a[mt][2], a[mt][3], l0[hg], l1[hg]);
 }
 
 template <int BITS>
@@ -374,11 +391,7 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
   const uint32_t codes = st + mla_kp_bytes();
   const uint32_t zbase = st + 2 * kMlaZeroOff;
   const uint32_t x16 = 0x4C004C00u;                        // fp16 pair (16, 16)
-  float S[2][2][4], Z[2][4];
-#pragma unroll
-  for (int hg = 0; hg < 2; ++hg)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) Z[hg][i] = S[0][hg][i] = S[1][hg][i] = 0.f;
+  float S[2][2][4], Zt[4];
   // ---- keys: four steps of 32 value channels (8 per lane = two slabs), then the rope slab ----
 #pragma unroll
   for (int step = 0; step < 4; ++step) {
@@ -425,7 +438,8 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
         }
       }
       const uint32_t q0[2] = {qr[0][i0], qr[1][i0]}, q1[2] = {qr[0][i1], qr[1][i1]};
-      m_slab(a, s0, s1, zr[i0], zr[i1], q0, q1, S, Z);
+      if (step == 0 && sl == 0) m_slab<true>(a, s0, s1, zr[i0], zr[i1], q0, q1, S, Zt);
+      else m_slab<false>(a, s0, s1, zr[i0], zr[i1], q0, q1, S, Zt);
     }
   }
   {
@@ -474,19 +488,25 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
       q1[0] = m_lds32(q16 + g * kMQPitch + 2 * cbb);
       q1[1] = m_lds32(q16 + (g + 8) * kMQPitch + 2 * cbb);
     }
-    m_slab(a, s0, s1, z0, z1, q0, q1, S, Z);
+    m_slab<false>(a, s0, s1, z0, z1, q0, q1, S, Zt);
   }
   // partial logits of the warp's channels -> the exchange buffer [warp][head][token]
   {
     const float ks = BITS == 8 ? 16777216.f : 1048576.f;
+    // sum q z of the heads 2 c4 + e + 8 hg sits in the lanes whose g is 2 c4 + e (registers 0 and 2)
+    float Z[2][2];
+#pragma unroll
+    for (int hg = 0; hg < 2; ++hg)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) Z[hg][e] = __shfl_sync(kMFull, Zt[2 * hg], 4 * (2 * c4 + e));
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
       for (int hg = 0; hg < 2; ++hg)
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int head = 8 * hg + 2 * c4 + (i & 1), tok = 16 * mt + g + 8 * (i >> 1);
-          m_stsf(xb + ((wq * kMlaHeads + head) * kMXPitch + tok) * 4, fmaf(S[mt][hg][i], ks, Z[hg][i]));
+          const int head = 8 * hg + 2 * c4 + (i & 1);
+          m_stsf(xb + ((wq * kMlaHeads + head) * kMXPitch + 16 * mt + g + 8 * (i >> 1)) * 4, fmaf(S[mt][hg][i], ks, Z[hg][i & 1]));
         }
   }
   m_quad_sync(quad);
@@ -530,10 +550,6 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
       const int mu = 4 * hp + m4;
       float T[2][4];
 #pragma unroll
-      for (int hg = 0; hg < 2; ++hg)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) T[hg][i] = 0.f;
-#pragma unroll
       for (int ks = 0; ks < 2; ++ks) {
         uint32_t a0, a1, a2, a3;
         if constexpr (BITS == 8) {
@@ -542,10 +558,10 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
           const uint32_t sel = (m4 & 1) ? 0x7531u : 0x6420u;
           const uint32_t y01 = m_prmt(w[ks][0][m4 >> 1], w[ks][1][m4 >> 1], sel);
           const uint32_t y23 = m_prmt(w[ks][2][m4 >> 1], w[ks][3][m4 >> 1], sel);
-          a0 = y01 & 0x00FF00FFu;
-          a1 = (y01 >> 8) & 0x00FF00FFu;
-          a2 = y23 & 0x00FF00FFu;
-          a3 = (y23 >> 8) & 0x00FF00FFu;
+          a0 = m_prmt(y01, 0u, 0x4240u);
+          a1 = m_prmt(y01, 0u, 0x4341u);
+          a2 = m_prmt(y23, 0u, 0x4240u);
+          a3 = m_prmt(y23, 0u, 0x4341u);
         } else {
           a0 = m4 == 0 ? m_fld4<0>(lo01[ks]) : (m4 == 1 ? m_fld4<1>(lo01[ks]) : (m4 == 2 ? m_fld4<2>(lo01[ks]) : m_fld4<3>(lo01[ks])));
           a1 = m4 == 0 ? m_fld4<0>(hi01[ks]) : (m4 == 1 ? m_fld4<1>(hi01[ks]) : (m4 == 2 ? m_fld4<2>(hi01[ks]) : m_fld4<3>(hi01[ks])));
@@ -554,9 +570,11 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
         }
 #pragma unroll
         for (int hg = 0; hg < 2; ++hg) {
-          m_mma_f16(T[hg], a0, a1, a2, a3, ph[hg][ks][0], ph[hg][ks][1]);
-          m_mma_f16(T[hg], a0, a1, a2, a3, pl[hg][ks][0], pl[hg][ks][1]);
+          if (ks == 0) m_mma_f16_first(T[hg], a0, a1, a2, a3, ph[hg][ks][0], ph[hg][ks][1]);
+          else m_mma_f16(T[hg], a0, a1, a2, a3, ph[hg][ks][0], ph[hg][ks][1]);
         }
+#pragma unroll
+        for (int hg = 0; hg < 2; ++hg) m_mma_f16(T[hg], a0, a1, a2, a3, pl[hg][ks][0], pl[hg][ks][1]);
       }
       const float un = (BITS == 4 && (m4 & 1)) ? 1048576.f : 16777216.f;   // 2^(24 - b)
       const float sa = m_h2f(sr[m4], 0) * un, sb = m_h2f(sr[m4], 1) * un;
@@ -598,8 +616,8 @@ __device__ __forceinline__ void m_unit_rows16(uint32_t st, uint32_t qbf, uint32_
   for (int hg = 0; hg < 2; ++hg)
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const int head = 8 * hg + 2 * c4 + (i & 1), tok = g + 8 * (i >> 1);
-      m_stsf(xb + ((wq * kMlaHeads + head) * kMXPitch + tok) * 4, S[hg][i]);
+      const int head = 8 * hg + 2 * c4 + (i & 1);
+      m_stsf(xb + ((wq * kMlaHeads + head) * kMXPitch + g + 8 * (i >> 1)) * 4, S[hg][i]);
     }
   m_quad_sync(quad);
   uint32_t ph[2][1][2], pl[2][1][2];
@@ -690,11 +708,11 @@ __global__ void __launch_bounds__(kMThreads, 1) mla_decode_kernel(const __grid_c
     const uint32_t st = qd + s * kMStageBytes;
     // after a time-out nothing waits any more: the remaining units run through on whatever the stages hold
     if (!*abort_flag && !m_wait(bars + 8 * s, (k >> 1) & 1)) *abort_flag = 1;
-    if (wc.kind == 0) {
-      if (wc.level == 8) m_unit_quant<8>(st, q16, xb, quad, wq, g, c4, p.scale_log2, O, m_run, l_run);
+    if (wc.kind() == 0) {
+      if (wc.level() == 8) m_unit_quant<8>(st, q16, xb, quad, wq, g, c4, p.scale_log2, O, m_run, l_run);
       else m_unit_quant<4>(st, q16, xb, quad, wq, g, c4, p.scale_log2, O, m_run, l_run);
     } else {
-      m_unit_rows16(st, qbf, xb, quad, wq, lane, p.scale_log2, wc.kind == 2 ? 6.0f : 0.f, m_unit_rows(wc), O, m_run, l_run);
+      m_unit_rows16(st, qbf, xb, quad, wq, lane, p.scale_log2, wc.kind() == 2 ? 6.0f : 0.f, m_unit_rows(wc), O, m_run, l_run);
     }
     // the stage and the exchange buffer are free once all four warps are here
     m_quad_sync(quad);
