@@ -48,12 +48,11 @@ constexpr int kMThreads = kMlaQuads * 128;
 constexpr int kMStageBytes = 20736;                    // one 8-bit half block: params 2304 + 32 x 576
 constexpr int kMStages = 2;
 constexpr int kMRowPitch = kMlaRowBytes + 16;          // bf16 rows staged at this pitch (conflict-free ldmatrix)
-constexpr int kMQPitch = kMlaRowBytes + 16;            // query rows in shared memory (fp16 and bf16 copies)
-constexpr int kMXPitch = 40;                           // floats per (warp, head) row of the exchange buffer
-constexpr int kMXBytes = 4 * kMlaHeads * kMXPitch * 4; // 10240
+constexpr int kMQPitch = 2 * kMlaRowBytes + 16;        // a head pair's row of the query copies: (q[g][c c+1], q[g + 8][c c+1]) per channel pair
+constexpr int kMXBytes = 4 * 4 * 32 * 16;              // exchange buffer [warp][token group][lane] x 16 B = 8192
 constexpr int kMOffQ16 = 0;
-constexpr int kMOffQbf = kMlaHeads * kMQPitch;         // 18688
-constexpr int kMOffQuad = 2 * kMlaHeads * kMQPitch;    // 37376
+constexpr int kMOffQbf = 8 * kMQPitch;                 // 18560
+constexpr int kMOffQuad = 2 * 8 * kMQPitch;            // 37120
 constexpr int kMQuadBytes = kMStages * kMStageBytes + kMXBytes + 64;   // stages | exchange | mbarriers
 constexpr int kMOffFlag = kMOffQuad + kMlaQuads * kMQuadBytes;
 constexpr int kMSmem = kMOffFlag + 16;
@@ -120,6 +119,14 @@ __device__ __forceinline__ float2 m_ldsf2(uint32_t a) {
   float2 v;
   asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];\n" : "=f"(v.x), "=f"(v.y) : "r"(a));
   return v;
+}
+__device__ __forceinline__ float4 m_ldsf4(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void m_stsf4(uint32_t a, float x, float y, float z, float w) {
+  asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};\n" ::"r"(a), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
 }
 __device__ __forceinline__ void m_stsf(uint32_t a, float v) { asm volatile("st.shared.f32 [%0], %1;\n" ::"r"(a), "f"(v) : "memory"); }
 __device__ __forceinline__ void m_stsf2(uint32_t a, float x, float y) {
@@ -268,32 +275,37 @@ __device__ __forceinline__ void m_issue(const MlaDecodeParams& p, const TableEnt
 // running sums and O^T are rescaled.  Outputs: the probabilities as a pair hi + lo (fp16 or bf16) and
 // the unit's probability sums of the heads 2 c4 + e (+ 8 hg), the columns of the lane's O^T registers.
 template <int NKS, bool BF16>
-__device__ __forceinline__ void m_softmax(uint32_t xb, int g, int c4, float scale_log2, float bias, int nvalid, float (&O)[8][2][4],
+__device__ __forceinline__ void m_softmax(uint32_t xb, int lane, float scale_log2, float bias, int nvalid, float (&O)[8][2][4],
                                           float (&m_run)[2], float (&l_run)[2], uint32_t (&ph)[2][NKS][2], uint32_t (&pl)[2][NKS][2],
                                           float (&psc)[2][2]) {
+  const int c4 = lane & 3;
+  // token group j4 (tokens 8 j4 .. 8 j4 + 7) of every warp's partial is one 16-byte piece per lane:
+  // heads g (x, y) and g + 8 (z, w), tokens 8 j4 + 2 c4, + 1
   float x[2][NKS][2][2];
-  float mloc[2];
+  float mloc[2] = {kMNegInf, kMNegInf};
+#pragma unroll
+  for (int j4 = 0; j4 < 2 * NKS; ++j4) {
+    const uint32_t a = xb + (j4 * 32 + lane) * 16;
+    float4 acc = m_ldsf4(a);
+#pragma unroll
+    for (int w = 1; w < 4; ++w) {
+      const float4 v = m_ldsf4(a + w * 4 * 32 * 16);
+      acc.x += v.x;
+      acc.y += v.y;
+      acc.z += v.z;
+      acc.w += v.w;
+    }
+    const int tok = 8 * j4 + 2 * c4;
+    const int ks = j4 >> 1, j = j4 & 1;
+    x[0][ks][j][0] = tok < nvalid ? fmaf(acc.x, scale_log2, bias) : kMNegInf;
+    x[0][ks][j][1] = tok + 1 < nvalid ? fmaf(acc.y, scale_log2, bias) : kMNegInf;
+    x[1][ks][j][0] = tok < nvalid ? fmaf(acc.z, scale_log2, bias) : kMNegInf;
+    x[1][ks][j][1] = tok + 1 < nvalid ? fmaf(acc.w, scale_log2, bias) : kMNegInf;
+    mloc[0] = fmaxf(mloc[0], fmaxf(x[0][ks][j][0], x[0][ks][j][1]));
+    mloc[1] = fmaxf(mloc[1], fmaxf(x[1][ks][j][0], x[1][ks][j][1]));
+  }
 #pragma unroll
   for (int hg = 0; hg < 2; ++hg) {
-    mloc[hg] = kMNegInf;
-#pragma unroll
-    for (int ks = 0; ks < NKS; ++ks) {
-#pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        const uint32_t a = xb + (((g + 8 * hg) * kMXPitch) + 16 * ks + 8 * j + 2 * c4) * 4;
-        float2 acc = m_ldsf2(a);
-#pragma unroll
-        for (int w = 1; w < 4; ++w) {
-          const float2 v = m_ldsf2(a + w * kMlaHeads * kMXPitch * 4);
-          acc.x += v.x;
-          acc.y += v.y;
-        }
-        const int tok = 16 * ks + 8 * j + 2 * c4;
-        x[hg][ks][j][0] = tok < nvalid ? fmaf(acc.x, scale_log2, bias) : kMNegInf;
-        x[hg][ks][j][1] = tok + 1 < nvalid ? fmaf(acc.y, scale_log2, bias) : kMNegInf;
-        mloc[hg] = fmaxf(mloc[hg], fmaxf(x[hg][ks][j][0], x[hg][ks][j][1]));
-      }
-    }
     mloc[hg] = fmaxf(mloc[hg], __shfl_xor_sync(kMFull, mloc[hg], 1));
     mloc[hg] = fmaxf(mloc[hg], __shfl_xor_sync(kMFull, mloc[hg], 2));
   }
@@ -353,35 +365,30 @@ __device__ __forceinline__ void m_softmax(uint32_t xb, int g, int c4, float scal
 }
 
 // ---- a quantised half block ---------------------------------------------------------------------
-// Key MMAs of one channel slab (16 channels = the four lanes' four channels each).  a[mt] = the A
-// fragments of the two token tiles; (s0, s1) the scales, (z0, z1) the zero points and (q0, q1) the
-// query entries (per head group) of the lane's channel pairs k = 2 c4, 2 c4 + 1 and k = 2 c4 + 8, 2 c4 + 9.
-// sum_c q[c] z[c] takes one MMA for all sixteen heads: the query registers are at once the A fragment
-// of Q^T (rows = heads g and g + 8), the zero points fill every column of B, and Zt[0] / Zt[2] end up as
-// the sums of the heads g / g + 8.
+// Key MMAs of one channel slab (16 channels = the four lanes' four channels each), heads along the rows:
+// S^T[head][token] += Q'^T K^T.  qa = the query entries (q[g][k0 k0+1], q[g + 8][k0 k0+1], q[g][k1 k1+1],
+// q[g + 8][k1 k1+1]) of the lane's channel pairs k0 = 2 c4 and k1 = 2 c4 + 8: times the scales (s0, s1) they are
+// the A fragment of Q'^T, as they are the A fragment of Q^T for sum_c q[c] z[c] (zero points (z0, z1) in
+// every column of B; Zt[0] / Zt[2] = the sums of the heads g / g + 8).  a[mt] = the code registers of the
+// two 16-token tiles (tokens g and g + 8, channel pairs k0 and k1): B fragments of the four 8-token groups.
 template <bool FIRST>
-__device__ __forceinline__ void m_slab(const uint32_t (&a)[2][4], uint32_t s0, uint32_t s1, uint32_t z0, uint32_t z1, const uint32_t (&q0)[2],
-                                       const uint32_t (&q1)[2], float (&S)[2][2][4], float (&Zt)[4]) {
-  uint32_t h0[2], l0[2], h1[2], l1[2];
-#pragma unroll
-  for (int hg = 0; hg < 2; ++hg) {
-    m_split(q0[hg], s0, h0[hg], l0[hg]);
-    m_split(q1[hg], s1, h1[hg], l1[hg]);
-  }
-  if (FIRST) m_mma_f16_first(Zt, q0[0], q0[1], q1[0], q1[1], z0, z1);
-  else m_mma_f16(Zt, q0[0], q0[1], q1[0], q1[1], z0, z1);
+__device__ __forceinline__ void m_slab(const uint32_t (&a)[2][4], uint32_t s0, uint32_t s1, uint32_t z0, uint32_t z1, const uint32_t (&qa)[4],
+                                       float (&S)[4][4], float (&Zt)[4]) {
+  uint32_t h[4], l[4];
+  m_split(qa[0], s0, h[0], l[0]);
+  m_split(qa[1], s0, h[1], l[1]);
+  m_split(qa[2], s1, h[2], l[2]);
+  m_split(qa[3], s1, h[3], l[3]);
+  if (FIRST) m_mma_f16_first(Zt, qa[0], qa[1], qa[2], qa[3], z0, z1);
+  else m_mma_f16(Zt, qa[0], qa[1], qa[2], qa[3], z0, z1);
   // four accumulator chains; the two MMAs of a chain are kept four apart
 #pragma unroll
-  for (int hg = 0; hg < 2; ++hg)
+  for (int j4 = 0; j4 < 4; ++j4) {
+    if (FIRST) m_mma_f16_first(S[j4], h[0], h[1], h[2], h[3], a[j4 >> 1][j4 & 1], a[j4 >> 1][(j4 & 1) + 2]);
+    else m_mma_f16(S[j4], h[0], h[1], h[2], h[3], a[j4 >> 1][j4 & 1], a[j4 >> 1][(j4 & 1) + 2]);
+  }
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt) {
-      if (FIRST) m_mma_f16_first(S[mt][hg], a[mt][0], a[mt][1], a[mt][2], a[mt][3], h0[hg], h1[hg]);
-      else m_mma_f16(S[mt][hg], a[mt][0], a[mt][1], a[mt][2], a[mt][3], h0[hg], h1[hg]);
-    }
-#pragma unroll
-  for (int hg = 0; hg < 2; ++hg)
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt) m_mma_f16(S[mt][hg], a[mt][0], a[mt][1], a[mt][2], a[mt][3], l0[hg], l1[hg]);
+  for (int j4 = 0; j4 < 4; ++j4) m_mma_f16(S[j4], l[0], l[1], l[2], l[3], a[j4 >> 1][j4 & 1], a[j4 >> 1][(j4 & 1) + 2]);
 }
 
 template <int BITS>
@@ -391,8 +398,11 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
   const uint32_t codes = st + mla_kp_bytes();
   const uint32_t zbase = st + 2 * kMlaZeroOff;
   const uint32_t x16 = 0x4C004C00u;                        // fp16 pair (16, 16)
-  float S[2][2][4], Zt[4];
+  const uint32_t qrow = q16 + g * kMQPitch;                // (q[g], q[g + 8]) interleaved per channel pair
+  float S[4][4], Zt[4];
   // ---- keys: four steps of 32 value channels (8 per lane = two slabs), then the rope slab ----
+  // A slab takes four neighbouring channels of the lane: 8-bit word sl (bytes c0 c2 c1 c3); 4-bit fields 2 sl
+  // (b = 0: weight 2^-24, its scale is taken times 16) and 2 sl + 1 (b = 4: weight 2^-20).
 #pragma unroll
   for (int step = 0; step < 4; ++step) {
     const int cb = 128 * wq + 32 * step + 8 * c4;          // the lane's 8 channels
@@ -409,19 +419,13 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
       }
     }
     const uint4 s4 = m_lds128(st + 2 * cb), z4 = m_lds128(zbase + 2 * cb);
-    const uint4 qa = m_lds128(q16 + g * kMQPitch + 2 * cb), qb = m_lds128(q16 + (g + 8) * kMQPitch + 2 * cb);
+    const uint4 q4a = m_lds128(qrow + 4 * cb), q4b = m_lds128(qrow + 4 * cb + 16);
     const uint32_t sr[4] = {s4.x, s4.y, s4.z, s4.w}, zr[4] = {z4.x, z4.y, z4.z, z4.w};
-    const uint32_t qr[2][4] = {{qa.x, qa.y, qa.z, qa.w}, {qb.x, qb.y, qb.z, qb.w}};
+    const uint32_t qr[2][4] = {{q4a.x, q4a.y, q4a.z, q4a.w}, {q4b.x, q4b.y, q4b.z, q4b.w}};
 #pragma unroll
     for (int sl = 0; sl < 2; ++sl) {
-      // 8-bit: slab sl = channels 4 sl .. 4 sl + 3 (word sl, bytes c0 c2 c1 c3); 4-bit: channels 2 sl, 2 sl + 1
-      // (field sl, b = 4 sl) and 2 sl + 4, 2 sl + 5 (field sl + 2)
-      const int i0 = BITS == 8 ? 2 * sl : sl, i1 = BITS == 8 ? 2 * sl + 1 : sl + 2;
-      uint32_t s0 = sr[i0], s1 = sr[i1];
-      if (BITS == 4 && sl == 0) {                          // the b = 0 fields weigh 2^-24, the b = 4 fields 2^-20
-        s0 = m_u(__hmul2(m_h2(s0), m_h2(x16)));
-        s1 = m_u(__hmul2(m_h2(s1), m_h2(x16)));
-      }
+      uint32_t s0 = sr[2 * sl];
+      if (BITS == 4) s0 = m_u(__hmul2(m_h2(s0), m_h2(x16)));
       uint32_t a[2][4];
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt) {
@@ -431,22 +435,22 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
           a[mt][2] = m_prmt(w[2 * mt][sl], 0u, 0x4341u);
           a[mt][3] = m_prmt(w[2 * mt + 1][sl], 0u, 0x4341u);
         } else {
-          a[mt][0] = sl ? m_fld4<1>(w[2 * mt][0]) : m_fld4<0>(w[2 * mt][0]);
-          a[mt][1] = sl ? m_fld4<1>(w[2 * mt + 1][0]) : m_fld4<0>(w[2 * mt + 1][0]);
-          a[mt][2] = sl ? m_fld4<3>(w[2 * mt][0]) : m_fld4<2>(w[2 * mt][0]);
-          a[mt][3] = sl ? m_fld4<3>(w[2 * mt + 1][0]) : m_fld4<2>(w[2 * mt + 1][0]);
+          a[mt][0] = sl ? m_fld4<2>(w[2 * mt][0]) : m_fld4<0>(w[2 * mt][0]);
+          a[mt][1] = sl ? m_fld4<2>(w[2 * mt + 1][0]) : m_fld4<0>(w[2 * mt + 1][0]);
+          a[mt][2] = sl ? m_fld4<3>(w[2 * mt][0]) : m_fld4<1>(w[2 * mt][0]);
+          a[mt][3] = sl ? m_fld4<3>(w[2 * mt + 1][0]) : m_fld4<1>(w[2 * mt + 1][0]);
         }
       }
-      const uint32_t q0[2] = {qr[0][i0], qr[1][i0]}, q1[2] = {qr[0][i1], qr[1][i1]};
-      if (step == 0 && sl == 0) m_slab<true>(a, s0, s1, zr[i0], zr[i1], q0, q1, S, Zt);
-      else m_slab<false>(a, s0, s1, zr[i0], zr[i1], q0, q1, S, Zt);
+      if (step == 0 && sl == 0) m_slab<true>(a, s0, sr[2 * sl + 1], zr[2 * sl], zr[2 * sl + 1], qr[sl], S, Zt);
+      else m_slab<false>(a, s0, sr[2 * sl + 1], zr[2 * sl], zr[2 * sl + 1], qr[sl], S, Zt);
     }
   }
   {
     // the rope slab: 16 channels of the warp, four per lane
-    uint32_t a[2][4], s0, s1, z0, z1, q0[2], q1[2];
+    uint32_t a[2][4], s0, s1, z0, z1, qa[4];
+    int cb;
     if constexpr (BITS == 8) {
-      const int cb = kMlaDv + 16 * wq + 4 * c4;
+      cb = kMlaDv + 16 * wq + 4 * c4;
       uint32_t w[4];
 #pragma unroll
       for (int tt = 0; tt < 4; ++tt) w[tt] = m_lds32(codes + (g + 8 * tt) * RB + cb);
@@ -457,62 +461,44 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
         a[mt][2] = m_prmt(w[2 * mt], 0u, 0x4341u);
         a[mt][3] = m_prmt(w[2 * mt + 1], 0u, 0x4341u);
       }
-      const uint2 s2 = m_lds64(st + 2 * cb), z2 = m_lds64(zbase + 2 * cb);
-      const uint2 qa = m_lds64(q16 + g * kMQPitch + 2 * cb), qb = m_lds64(q16 + (g + 8) * kMQPitch + 2 * cb);
-      s0 = s2.x; s1 = s2.y; z0 = z2.x; z1 = z2.y;
-      q0[0] = qa.x; q0[1] = qb.x; q1[0] = qa.y; q1[1] = qb.y;
     } else {
-      // the lane's word is chunk c4 / 2 of the warp's two; its fields sl = c4 & 1 (channels 2 sl, 2 sl + 1)
-      // and sl + 2 (channels 2 sl + 4, 2 sl + 5)
-      const int sl = c4 & 1;
-      const int cbase = kMlaDv + 16 * wq + 8 * (c4 >> 1);
-      const uint32_t mask = sl ? 0x00F000F0u : 0x000F000Fu;
+      // the lane's word is chunk c4 / 2 of the warp's two; its fields 2 (c4 & 1) and 2 (c4 & 1) + 1
+      cb = kMlaDv + 16 * wq + 8 * (c4 >> 1) + 4 * (c4 & 1);
       uint32_t w[4];
 #pragma unroll
-      for (int tt = 0; tt < 4; ++tt) w[tt] = m_lds32(codes + (g + 8 * tt) * RB + (cbase >> 1));
+      for (int tt = 0; tt < 4; ++tt) {
+        w[tt] = m_lds32(codes + (g + 8 * tt) * RB + ((kMlaDv + 16 * wq + 8 * (c4 >> 1)) >> 1));
+        if (c4 & 1) w[tt] >>= 8;
+      }
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt) {
-        a[mt][0] = w[2 * mt] & mask;
-        a[mt][1] = w[2 * mt + 1] & mask;
-        a[mt][2] = (w[2 * mt] >> 8) & mask;
-        a[mt][3] = (w[2 * mt + 1] >> 8) & mask;
+        a[mt][0] = w[2 * mt] & 0x000F000Fu;
+        a[mt][1] = w[2 * mt + 1] & 0x000F000Fu;
+        a[mt][2] = w[2 * mt] & 0x00F000F0u;
+        a[mt][3] = w[2 * mt + 1] & 0x00F000F0u;
       }
-      const int ca = cbase + 2 * sl, cbb = ca + 4;
-      const __half2 f = __float2half2_rn(sl ? 1.f : 16.f);
-      s0 = m_u(__hmul2(m_h2(m_lds32(st + 2 * ca)), f));
-      s1 = m_u(__hmul2(m_h2(m_lds32(st + 2 * cbb)), f));
-      z0 = m_lds32(zbase + 2 * ca);
-      z1 = m_lds32(zbase + 2 * cbb);
-      q0[0] = m_lds32(q16 + g * kMQPitch + 2 * ca);
-      q0[1] = m_lds32(q16 + (g + 8) * kMQPitch + 2 * ca);
-      q1[0] = m_lds32(q16 + g * kMQPitch + 2 * cbb);
-      q1[1] = m_lds32(q16 + (g + 8) * kMQPitch + 2 * cbb);
     }
-    m_slab<false>(a, s0, s1, z0, z1, q0, q1, S, Zt);
+    const uint2 s2 = m_lds64(st + 2 * cb), z2 = m_lds64(zbase + 2 * cb);
+    const uint4 q4 = m_lds128(qrow + 4 * cb);
+    s0 = BITS == 4 ? m_u(__hmul2(m_h2(s2.x), m_h2(x16))) : s2.x;
+    s1 = s2.y; z0 = z2.x; z1 = z2.y;
+    qa[0] = q4.x; qa[1] = q4.y; qa[2] = q4.z; qa[3] = q4.w;
+    m_slab<false>(a, s0, s1, z0, z1, qa, S, Zt);
   }
-  // partial logits of the warp's channels -> the exchange buffer [warp][head][token]
+  // partial logits of the warp's channels -> the exchange buffer [warp][token group][lane]: heads g and
+  // g + 8, tokens 8 j4 + 2 c4, + 1
   {
     const float ks = BITS == 8 ? 16777216.f : 1048576.f;
-    // sum q z of the heads 2 c4 + e + 8 hg sits in the lanes whose g is 2 c4 + e (registers 0 and 2)
-    float Z[2][2];
+    const int lane = 4 * g + c4;
 #pragma unroll
-    for (int hg = 0; hg < 2; ++hg)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) Z[hg][e] = __shfl_sync(kMFull, Zt[2 * hg], 4 * (2 * c4 + e));
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-      for (int hg = 0; hg < 2; ++hg)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int head = 8 * hg + 2 * c4 + (i & 1);
-          m_stsf(xb + ((wq * kMlaHeads + head) * kMXPitch + 16 * mt + g + 8 * (i >> 1)) * 4, fmaf(S[mt][hg][i], ks, Z[hg][i & 1]));
-        }
+    for (int j4 = 0; j4 < 4; ++j4)
+      m_stsf4(xb + ((wq * 4 + j4) * 32 + lane) * 16, fmaf(S[j4][0], ks, Zt[0]), fmaf(S[j4][1], ks, Zt[0]), fmaf(S[j4][2], ks, Zt[2]),
+              fmaf(S[j4][3], ks, Zt[2]));
   }
   m_quad_sync(quad);
   uint32_t ph[2][2][2], pl[2][2][2];
   float psc[2][2];
-  m_softmax<2, false>(xb, g, c4, scale_log2, 0.f, 32, O, m_run, l_run, ph, pl, psc);
+  m_softmax<2, false>(xb, 4 * g + c4, scale_log2, 0.f, 32, O, m_run, l_run, ph, pl, psc);
   // ---- values: the warp's 128 channels, 16 per lane group; two passes of four M-tiles ----
 #pragma unroll
   for (int hp = 0; hp < 2; ++hp) {
@@ -594,35 +580,30 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
 __device__ __forceinline__ void m_unit_rows16(uint32_t st, uint32_t qbf, uint32_t xb, int quad, int wq, int lane, float scale_log2,
                                               float bias, int nvalid, float (&O)[8][2][4], float (&m_run)[2], float (&l_run)[2]) {
   const int g = lane >> 2, c4 = lane & 3;
+  // keys, heads along the rows: the A fragment is the query (bf16), the ldmatrix registers are the B fragments
+  // of the two 8-token groups
   float S[2][4];
 #pragma unroll
-  for (int hg = 0; hg < 2; ++hg)
+  for (int j4 = 0; j4 < 2; ++j4)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) S[hg][i] = 0.f;
+    for (int i = 0; i < 4; ++i) S[j4][i] = 0.f;
   const uint32_t arow = st + (lane & 15) * kMRowPitch + 16 * (lane >> 4);
+  const uint32_t qrow = qbf + g * kMQPitch + 8 * c4;
 #pragma unroll
   for (int sl = 0; sl < 9; ++sl) {
     const int ch0 = sl < 8 ? 128 * wq + 16 * sl : kMlaDv + 16 * wq;
     uint32_t a[4];
     m_ldmatrix4(arow + 2 * ch0, a);
-#pragma unroll
-    for (int hg = 0; hg < 2; ++hg) {
-      const uint32_t b0 = m_lds32(qbf + (g + 8 * hg) * kMQPitch + 2 * (ch0 + 2 * c4));
-      const uint32_t b1 = m_lds32(qbf + (g + 8 * hg) * kMQPitch + 2 * (ch0 + 8 + 2 * c4));
-      m_mma_bf16(S[hg], a[0], a[1], a[2], a[3], b0, b1);
-    }
+    const uint2 q0 = m_lds64(qrow + 4 * ch0), q1 = m_lds64(qrow + 4 * ch0 + 32);
+    m_mma_bf16(S[0], q0.x, q0.y, q1.x, q1.y, a[0], a[2]);
+    m_mma_bf16(S[1], q0.x, q0.y, q1.x, q1.y, a[1], a[3]);
   }
 #pragma unroll
-  for (int hg = 0; hg < 2; ++hg)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int head = 8 * hg + 2 * c4 + (i & 1);
-      m_stsf(xb + ((wq * kMlaHeads + head) * kMXPitch + g + 8 * (i >> 1)) * 4, S[hg][i]);
-    }
+  for (int j4 = 0; j4 < 2; ++j4) m_stsf4(xb + ((wq * 4 + j4) * 32 + lane) * 16, S[j4][0], S[j4][1], S[j4][2], S[j4][3]);
   m_quad_sync(quad);
   uint32_t ph[2][1][2], pl[2][1][2];
   float psc[2][2];
-  m_softmax<1, true>(xb, g, c4, scale_log2, bias, nvalid, O, m_run, l_run, ph, pl, psc);
+  m_softmax<1, true>(xb, lane, scale_log2, bias, nvalid, O, m_run, l_run, ph, pl, psc);
   // values: channel pairs (2 mu, 2 mu + 1) of the lane group's 16 channels from the tokens 2 c4, 2 c4 + 1, 2 c4 + 8, 2 c4 + 9
 #pragma unroll
   for (int hp = 0; hp < 2; ++hp) {
@@ -668,13 +649,18 @@ __global__ void __launch_bounds__(kMThreads, 1) mla_decode_kernel(const __grid_c
     m_fence_async();
   }
   {
-    // the query: a bf16 copy (bf16 MMAs of exact rows) and an fp16 copy (exact for the magnitudes a query has)
+    // the query: a bf16 copy (bf16 MMAs of exact rows) and an fp16 copy (exact for the magnitudes a query has),
+    // both with the heads g and g + 8 interleaved per channel pair
     const uint16_t* qg = p.q + static_cast<size_t>(cd.stream) * kMlaHeads * kMlaDk;
-    for (int idx = tid; idx < kMlaHeads * kMlaChunks; idx += kMThreads) {
-      const int head = idx / kMlaChunks, piece = idx % kMlaChunks;
-      const uint4 v = *reinterpret_cast<const uint4*>(qg + head * kMlaDk + 8 * piece);
-      m_sts128(qbf + head * kMQPitch + 16 * piece, v.x, v.y, v.z, v.w);
-      m_sts128(q16 + head * kMQPitch + 16 * piece, m_bf2_to_h2(v.x), m_bf2_to_h2(v.y), m_bf2_to_h2(v.z), m_bf2_to_h2(v.w));
+    for (int idx = tid; idx < 8 * kMlaChunks; idx += kMThreads) {
+      const int hp = idx / kMlaChunks, piece = idx % kMlaChunks;
+      const uint4 v0 = *reinterpret_cast<const uint4*>(qg + hp * kMlaDk + 8 * piece);
+      const uint4 v1 = *reinterpret_cast<const uint4*>(qg + (hp + 8) * kMlaDk + 8 * piece);
+      const uint32_t d = hp * kMQPitch + 32 * piece;
+      m_sts128(qbf + d, v0.x, v1.x, v0.y, v1.y);
+      m_sts128(qbf + d + 16, v0.z, v1.z, v0.w, v1.w);
+      m_sts128(q16 + d, m_bf2_to_h2(v0.x), m_bf2_to_h2(v1.x), m_bf2_to_h2(v0.y), m_bf2_to_h2(v1.y));
+      m_sts128(q16 + d + 16, m_bf2_to_h2(v0.z), m_bf2_to_h2(v1.z), m_bf2_to_h2(v0.w), m_bf2_to_h2(v1.w));
     }
   }
   __syncthreads();
