@@ -1022,10 +1022,10 @@ size_t mla_item_cost(const gkv_cache* c, const LayerState& L, int stream, int it
   // (262,144 tokens), less the call's fixed part.
   if (item < L.n_closed) {
     switch (L.level[static_cast<size_t>(stream) * c->max_blocks + item]) {
-      case 16: return 1180;
-      case 8: return 1015;
+      case 16: return 1065;
+      case 8: return 1005;
       case 4: return 1000;
-      default: return 155;
+      default: return 215;
     }
   }
   return 900;                     // tail

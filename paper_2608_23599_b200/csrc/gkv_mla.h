@@ -5,7 +5,7 @@
 namespace gkv {
 
 constexpr int kMlaPartialFloats = kMlaHeads * (kMlaDv + 2);   // per CTA partial: m, l, o[512] per head
-constexpr int kMlaQuads = 3;                                  // groups of four warps per CTA of the decode kernel, each with a block range of its own
+constexpr int kMlaQuads = 4;                                  // groups of four warps per CTA of the decode kernel, each with a block range of its own
 
 struct MlaEncodeParams {
   uint8_t* arena;

@@ -51,11 +51,12 @@ constexpr int kMRowPitch = kMlaRowBytes + 16;          // bf16 rows staged at th
 constexpr int kMQPitch = 2 * kMlaRowBytes + 16;        // a head pair's row of the query copies: (q[g][c c+1], q[g + 8][c c+1]) per channel pair
 constexpr int kMXBytes = 4 * 4 * 32 * 16;              // exchange buffer [warp][token group][lane] x 16 B = 8192
 constexpr int kMOffQ16 = 0;
-constexpr int kMOffQbf = 8 * kMQPitch;                 // 18560
-constexpr int kMOffQuad = 2 * 8 * kMQPitch;            // 37120
+constexpr int kMOffQuad = 8 * kMQPitch;                // 18560
 constexpr int kMQuadBytes = kMStages * kMStageBytes + kMXBytes + 64;   // stages | exchange | mbarriers
 constexpr int kMOffFlag = kMOffQuad + kMlaQuads * kMQuadBytes;
-constexpr int kMSmem = kMOffFlag + 16;
+constexpr int kMSmem = kMOffFlag + 16;                 // abort flag, tensor-memory base
+constexpr uint32_t kMTmemCols = 512;                   // per warp 64 columns of O^T and 36 of bf16 query fragments, four warps per lane quarter
+constexpr uint32_t kMTmemQ = 256;                      // first column of the query fragments
 constexpr int kMOutPitch = kMlaDv + 2;                 // floats per head row of a quad's result in shared memory
 constexpr int kMWaitSpins = 1 << 22;
 constexpr float kMNegInf = -INFINITY;
@@ -167,6 +168,41 @@ __device__ __forceinline__ void m_mma_bf16(float (&c)[4], uint32_t a0, uint32_t 
 __device__ __forceinline__ void m_ldmatrix4(uint32_t a, uint32_t (&r)[4]) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
 }
+// ---- tensor memory as the home of the running O^T (64 fp32 per thread: column 8 mu + 4 hg + i of the thread's lane) ----
+__device__ __forceinline__ void m_tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_dst), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void m_tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void m_tfence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void m_tfence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+// eight columns of the thread's lane; m_twait_ld() before the first use
+__device__ __forceinline__ void m_tld8(uint32_t taddr, float (&v)[2][4]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];\n"
+               : "=f"(v[0][0]), "=f"(v[0][1]), "=f"(v[0][2]), "=f"(v[0][3]), "=f"(v[1][0]), "=f"(v[1][1]), "=f"(v[1][2]), "=f"(v[1][3])
+               : "r"(taddr));
+}
+__device__ __forceinline__ void m_tld4(uint32_t taddr, uint32_t (&v)[4]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(taddr));
+}
+__device__ __forceinline__ void m_tst4(uint32_t taddr, const uint32_t (&v)[4]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]) : "memory");
+}
+__device__ __forceinline__ void m_twait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void m_tst8(uint32_t taddr, const float (&v)[2][4]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n" ::"r"(taddr), "f"(v[0][0]), "f"(v[0][1]),
+               "f"(v[0][2]), "f"(v[0][3]), "f"(v[1][0]), "f"(v[1][1]), "f"(v[1][2]), "f"(v[1][3])
+               : "memory");
+}
+__device__ __forceinline__ void m_twait_st() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ uint32_t m_ldg32(const void* p) {
+  uint32_t v;
+  asm volatile("ld.global.nc.u32 %0, [%1];\n" : "=r"(v) : "l"(p));
+  return v;
+}
+
 // q * s as an fp16 pair: hi = the rounded product, lo = the exact remainder
 __device__ __forceinline__ void m_split(uint32_t q, uint32_t s, uint32_t& hi, uint32_t& lo) {
   const __half2 h = __hmul2(m_h2(q), m_h2(s));
@@ -275,7 +311,7 @@ __device__ __forceinline__ void m_issue(const MlaDecodeParams& p, const TableEnt
 // running sums and O^T are rescaled.  Outputs: the probabilities as a pair hi + lo (fp16 or bf16) and
 // the unit's probability sums of the heads 2 c4 + e (+ 8 hg), the columns of the lane's O^T registers.
 template <int NKS, bool BF16>
-__device__ __forceinline__ void m_softmax(uint32_t xb, int lane, float scale_log2, float bias, int nvalid, float (&O)[8][2][4],
+__device__ __forceinline__ void m_softmax(uint32_t xb, int lane, float scale_log2, float bias, int nvalid, uint32_t ot,
                                           float (&m_run)[2], float (&l_run)[2], uint32_t (&ph)[2][NKS][2], uint32_t (&pl)[2][NKS][2],
                                           float (&psc)[2][2]) {
   const int c4 = lane & 3;
@@ -325,12 +361,18 @@ __device__ __forceinline__ void m_softmax(uint32_t xb, int lane, float scale_log
     for (int hg = 0; hg < 2; ++hg)
 #pragma unroll
       for (int e = 0; e < 2; ++e) ac[hg][e] = __shfl_sync(kMFull, al[hg], 4 * (2 * c4 + e));
-#pragma unroll
-    for (int mu = 0; mu < 8; ++mu)
+#pragma unroll 2
+    for (int mu = 0; mu < 8; ++mu) {
+      float o[2][4];
+      m_tld8(ot + 8 * mu, o);
+      m_twait_ld();
 #pragma unroll
       for (int hg = 0; hg < 2; ++hg)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) O[mu][hg][i] *= ac[hg][i & 1];
+        for (int i = 0; i < 4; ++i) o[hg][i] *= ac[hg][i & 1];
+      m_tst8(ot + 8 * mu, o);
+    }
+    m_twait_st();
   }
   float ps[2];
 #pragma unroll
@@ -393,7 +435,7 @@ __device__ __forceinline__ void m_slab(const uint32_t (&a)[2][4], uint32_t s0, u
 
 template <int BITS>
 __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t xb, int quad, int wq, int g, int c4, float scale_log2,
-                                             float (&O)[8][2][4], float (&m_run)[2], float (&l_run)[2]) {
+                                             uint32_t ot, float (&m_run)[2], float (&l_run)[2]) {
   constexpr int RB = kMlaChunks * BITS;                    // bytes per token row of codes
   const uint32_t codes = st + mla_kp_bytes();
   const uint32_t zbase = st + 2 * kMlaZeroOff;
@@ -498,7 +540,7 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
   m_quad_sync(quad);
   uint32_t ph[2][2][2], pl[2][2][2];
   float psc[2][2];
-  m_softmax<2, false>(xb, 4 * g + c4, scale_log2, 0.f, 32, O, m_run, l_run, ph, pl, psc);
+  m_softmax<2, false>(xb, 4 * g + c4, scale_log2, 0.f, 32, ot, m_run, l_run, ph, pl, psc);
   // ---- values: the warp's 128 channels, 16 per lane group; two passes of four M-tiles ----
 #pragma unroll
   for (int hp = 0; hp < 2; ++hp) {
@@ -534,7 +576,8 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
     for (int m4 = 0; m4 < 4; ++m4) {
       // M-tile mu = 4 hp + m4: row g = channel cv + 2 m4, row g + 8 = channel cv + 2 m4 + 1
       const int mu = 4 * hp + m4;
-      float T[2][4];
+      float T[2][4], o[2][4];
+      m_tld8(ot + 8 * mu, o);                                // this M-tile's rows of O^T, asked for before the MMAs
 #pragma unroll
       for (int ks = 0; ks < 2; ++ks) {
         uint32_t a0, a1, a2, a3;
@@ -565,20 +608,23 @@ __device__ __forceinline__ void m_unit_quant(uint32_t st, uint32_t q16, uint32_t
       const float un = (BITS == 4 && (m4 & 1)) ? 1048576.f : 16777216.f;   // 2^(24 - b)
       const float sa = m_h2f(sr[m4], 0) * un, sb = m_h2f(sr[m4], 1) * un;
       const float za = m_h2f(zr[m4], 0), zb = m_h2f(zr[m4], 1);
+      m_twait_ld();
 #pragma unroll
       for (int hg = 0; hg < 2; ++hg) {
-        O[mu][hg][0] = fmaf(T[hg][0], sa, fmaf(za, psc[hg][0], O[mu][hg][0]));
-        O[mu][hg][1] = fmaf(T[hg][1], sa, fmaf(za, psc[hg][1], O[mu][hg][1]));
-        O[mu][hg][2] = fmaf(T[hg][2], sb, fmaf(zb, psc[hg][0], O[mu][hg][2]));
-        O[mu][hg][3] = fmaf(T[hg][3], sb, fmaf(zb, psc[hg][1], O[mu][hg][3]));
+        o[hg][0] = fmaf(T[hg][0], sa, fmaf(za, psc[hg][0], o[hg][0]));
+        o[hg][1] = fmaf(T[hg][1], sa, fmaf(za, psc[hg][1], o[hg][1]));
+        o[hg][2] = fmaf(T[hg][2], sb, fmaf(zb, psc[hg][0], o[hg][2]));
+        o[hg][3] = fmaf(T[hg][3], sb, fmaf(zb, psc[hg][1], o[hg][3]));
       }
+      m_tst8(ot + 8 * mu, o);
     }
   }
+  m_twait_st();
 }
 
 // ---- 16 bf16 rows (an exact tile, the tail, a run of centroid rows) ---------------------------------
-__device__ __forceinline__ void m_unit_rows16(uint32_t st, uint32_t qbf, uint32_t xb, int quad, int wq, int lane, float scale_log2,
-                                              float bias, int nvalid, float (&O)[8][2][4], float (&m_run)[2], float (&l_run)[2]) {
+__device__ __forceinline__ void m_unit_rows16(uint32_t st, uint32_t qt, uint32_t xb, int quad, int wq, int lane, float scale_log2,
+                                              float bias, int nvalid, uint32_t ot, float (&m_run)[2], float (&l_run)[2]) {
   const int g = lane >> 2, c4 = lane & 3;
   // keys, heads along the rows: the A fragment is the query (bf16), the ldmatrix registers are the B fragments
   // of the two 8-token groups
@@ -588,22 +634,25 @@ __device__ __forceinline__ void m_unit_rows16(uint32_t st, uint32_t qbf, uint32_
 #pragma unroll
     for (int i = 0; i < 4; ++i) S[j4][i] = 0.f;
   const uint32_t arow = st + (lane & 15) * kMRowPitch + 16 * (lane >> 4);
-  const uint32_t qrow = qbf + g * kMQPitch + 8 * c4;
+  // (the bf16 query fragments of the warp's nine slabs wait in tensor memory)
+  uint32_t qa[9][4];
+#pragma unroll
+  for (int sl = 0; sl < 9; ++sl) m_tld4(qt + 4 * sl, qa[sl]);
+  m_twait_ld();
 #pragma unroll
   for (int sl = 0; sl < 9; ++sl) {
     const int ch0 = sl < 8 ? 128 * wq + 16 * sl : kMlaDv + 16 * wq;
     uint32_t a[4];
     m_ldmatrix4(arow + 2 * ch0, a);
-    const uint2 q0 = m_lds64(qrow + 4 * ch0), q1 = m_lds64(qrow + 4 * ch0 + 32);
-    m_mma_bf16(S[0], q0.x, q0.y, q1.x, q1.y, a[0], a[2]);
-    m_mma_bf16(S[1], q0.x, q0.y, q1.x, q1.y, a[1], a[3]);
+    m_mma_bf16(S[0], qa[sl][0], qa[sl][1], qa[sl][2], qa[sl][3], a[0], a[2]);
+    m_mma_bf16(S[1], qa[sl][0], qa[sl][1], qa[sl][2], qa[sl][3], a[1], a[3]);
   }
 #pragma unroll
   for (int j4 = 0; j4 < 2; ++j4) m_stsf4(xb + ((wq * 4 + j4) * 32 + lane) * 16, S[j4][0], S[j4][1], S[j4][2], S[j4][3]);
   m_quad_sync(quad);
   uint32_t ph[2][1][2], pl[2][1][2];
   float psc[2][2];
-  m_softmax<1, true>(xb, lane, scale_log2, bias, nvalid, O, m_run, l_run, ph, pl, psc);
+  m_softmax<1, true>(xb, lane, scale_log2, bias, nvalid, ot, m_run, l_run, ph, pl, psc);
   // values: channel pairs (2 mu, 2 mu + 1) of the lane group's 16 channels from the tokens 2 c4, 2 c4 + 1, 2 c4 + 8, 2 c4 + 9
 #pragma unroll
   for (int hp = 0; hp < 2; ++hp) {
@@ -619,13 +668,18 @@ __device__ __forceinline__ void m_unit_rows16(uint32_t st, uint32_t qbf, uint32_
       const int mu = 4 * hp + m4;
       const uint32_t a0 = m_prmt(w[0][m4], w[1][m4], 0x5410u), a1 = m_prmt(w[0][m4], w[1][m4], 0x7632u);
       const uint32_t a2 = m_prmt(w[2][m4], w[3][m4], 0x5410u), a3 = m_prmt(w[2][m4], w[3][m4], 0x7632u);
+      float o[2][4];
+      m_tld8(ot + 8 * mu, o);
+      m_twait_ld();
 #pragma unroll
       for (int hg = 0; hg < 2; ++hg) {
-        m_mma_bf16(O[mu][hg], a0, a1, a2, a3, ph[hg][0][0], ph[hg][0][1]);
-        m_mma_bf16(O[mu][hg], a0, a1, a2, a3, pl[hg][0][0], pl[hg][0][1]);
+        m_mma_bf16(o[hg], a0, a1, a2, a3, ph[hg][0][0], ph[hg][0][1]);
+        m_mma_bf16(o[hg], a0, a1, a2, a3, pl[hg][0][0], pl[hg][0][1]);
       }
+      m_tst8(ot + 8 * mu, o);
     }
   }
+  m_twait_st();
 }
 
 // ---- kernel --------------------------------------------------------------------------------------
@@ -636,11 +690,12 @@ __global__ void __launch_bounds__(kMThreads, 1) mla_decode_kernel(const __grid_c
   const WarpDesc cd = p.ctas[blockIdx.x * kMlaQuads + quad];
   if (p.ctas[blockIdx.x * kMlaQuads].stream < 0) return;        // uniform for the CTA
   const uint32_t base = m_u32(msm);
-  const uint32_t q16 = base + kMOffQ16, qbf = base + kMOffQbf;
+  const uint32_t q16 = base + kMOffQ16;
   const uint32_t qd = base + kMOffQuad + quad * kMQuadBytes;
   const uint32_t xb = qd + kMStages * kMStageBytes, bars = xb + kMXBytes;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(msm + kMOffFlag);
   const TableEntry* table = p.table + static_cast<size_t>(cd.stream) * p.table_stride;
+  const uint16_t* qg = p.q + static_cast<size_t>(cd.stream) * kMlaHeads * kMlaDk;
 
   if (tid == 0) *abort_flag = 0;
   if (wq == 0 && lane == 0) {
@@ -648,30 +703,43 @@ __global__ void __launch_bounds__(kMThreads, 1) mla_decode_kernel(const __grid_c
     m_bar_init(bars + 8, 1);
     m_fence_async();
   }
+  if (warp == 0) m_tmem_alloc(base + kMOffFlag + 4, kMTmemCols);
   {
-    // the query: a bf16 copy (bf16 MMAs of exact rows) and an fp16 copy (exact for the magnitudes a query has),
-    // both with the heads g and g + 8 interleaved per channel pair
-    const uint16_t* qg = p.q + static_cast<size_t>(cd.stream) * kMlaHeads * kMlaDk;
+    // the query as fp16 (exact for the magnitudes a query has), the heads g and g + 8 interleaved per channel pair
     for (int idx = tid; idx < 8 * kMlaChunks; idx += kMThreads) {
       const int hp = idx / kMlaChunks, piece = idx % kMlaChunks;
       const uint4 v0 = *reinterpret_cast<const uint4*>(qg + hp * kMlaDk + 8 * piece);
       const uint4 v1 = *reinterpret_cast<const uint4*>(qg + (hp + 8) * kMlaDk + 8 * piece);
       const uint32_t d = hp * kMQPitch + 32 * piece;
-      m_sts128(qbf + d, v0.x, v1.x, v0.y, v1.y);
-      m_sts128(qbf + d + 16, v0.z, v1.z, v0.w, v1.w);
       m_sts128(q16 + d, m_bf2_to_h2(v0.x), m_bf2_to_h2(v1.x), m_bf2_to_h2(v0.y), m_bf2_to_h2(v1.y));
       m_sts128(q16 + d + 16, m_bf2_to_h2(v0.z), m_bf2_to_h2(v1.z), m_bf2_to_h2(v0.w), m_bf2_to_h2(v1.w));
     }
   }
+  m_tfence_before();
   __syncthreads();
-
-  float O[8][2][4];
+  m_tfence_after();
+  // this warp's 64 columns of its lane quarter: the running O^T, zero to begin with
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(msm + kMOffFlag + 4);
+  const uint32_t ot = tmem + (static_cast<uint32_t>(32 * wq) << 16) + 64u * static_cast<uint32_t>(quad);
+  {
+    const float zero[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-  for (int mu = 0; mu < 8; ++mu)
-#pragma unroll
-    for (int hg = 0; hg < 2; ++hg)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) O[mu][hg][i] = 0.f;
+    for (int mu = 0; mu < 8; ++mu) m_tst8(ot + 8 * mu, zero);
+    m_twait_st();
+  }
+  // the bf16 query as the A fragments of the warp's nine channel slabs (rows = heads g and g + 8), for the units of
+  // exact and centroid rows
+  const uint32_t qt = tmem + (static_cast<uint32_t>(32 * wq) << 16) + kMTmemQ + 36u * static_cast<uint32_t>(quad);
+  {
+    const uint16_t* qa = qg + g * kMlaDk + 2 * c4;
+#pragma unroll 3
+    for (int sl = 0; sl < 9; ++sl) {
+      const int ch0 = sl < 8 ? 128 * wq + 16 * sl : kMlaDv + 16 * wq;
+      const uint32_t f[4] = {m_ldg32(qa + ch0), m_ldg32(qa + 8 * kMlaDk + ch0), m_ldg32(qa + ch0 + 8), m_ldg32(qa + 8 * kMlaDk + ch0 + 8)};
+      m_tst4(qt + 4 * sl, f);
+    }
+    m_twait_st();
+  }
   float m_run[2] = {kMNegInf, kMNegInf}, l_run[2] = {0.f, 0.f};
 
   MWalk wc, wl;
@@ -695,10 +763,10 @@ __global__ void __launch_bounds__(kMThreads, 1) mla_decode_kernel(const __grid_c
     // after a time-out nothing waits any more: the remaining units run through on whatever the stages hold
     if (!*abort_flag && !m_wait(bars + 8 * s, (k >> 1) & 1)) *abort_flag = 1;
     if (wc.kind() == 0) {
-      if (wc.level() == 8) m_unit_quant<8>(st, q16, xb, quad, wq, g, c4, p.scale_log2, O, m_run, l_run);
-      else m_unit_quant<4>(st, q16, xb, quad, wq, g, c4, p.scale_log2, O, m_run, l_run);
+      if (wc.level() == 8) m_unit_quant<8>(st, q16, xb, quad, wq, g, c4, p.scale_log2, ot, m_run, l_run);
+      else m_unit_quant<4>(st, q16, xb, quad, wq, g, c4, p.scale_log2, ot, m_run, l_run);
     } else {
-      m_unit_rows16(st, qbf, xb, quad, wq, lane, p.scale_log2, wc.kind() == 2 ? 6.0f : 0.f, m_unit_rows(wc), O, m_run, l_run);
+      m_unit_rows16(st, qt, xb, quad, wq, lane, p.scale_log2, wc.kind() == 2 ? 6.0f : 0.f, m_unit_rows(wc), ot, m_run, l_run);
     }
     // the stage and the exchange buffer are free once all four warps are here
     m_quad_sync(quad);
@@ -718,15 +786,19 @@ __global__ void __launch_bounds__(kMThreads, 1) mla_decode_kernel(const __grid_c
       l[hg] = l_run[hg] + __shfl_xor_sync(kMFull, l_run[hg], 1);
       l[hg] += __shfl_xor_sync(kMFull, l[hg], 2);
     }
-#pragma unroll
-    for (int mu = 0; mu < 8; ++mu)
+#pragma unroll 2
+    for (int mu = 0; mu < 8; ++mu) {
+      float o[2][4];
+      m_tld8(ot + 8 * mu, o);
+      m_twait_ld();
 #pragma unroll
       for (int hg = 0; hg < 2; ++hg)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const int head = 8 * hg + 2 * c4 + e, ch = 128 * wq + 16 * g + 2 * mu;
-          m_stsf2(qd + (head * kMOutPitch + ch) * 4, O[mu][hg][e], O[mu][hg][e + 2]);
+          m_stsf2(qd + (head * kMOutPitch + ch) * 4, o[hg][e], o[hg][e + 2]);
         }
+    }
     if (wq == 0 && c4 == 0) {
 #pragma unroll
       for (int hg = 0; hg < 2; ++hg) {
@@ -763,6 +835,9 @@ __global__ void __launch_bounds__(kMThreads, 1) mla_decode_kernel(const __grid_c
     }
   }
   if (tid == 0 && *abort_flag) atomicOr(p.status, kStatusInternal);
+  m_tfence_before();
+  __syncthreads();
+  if (warp == 0) m_tmem_dealloc(tmem, kMTmemCols);
 }
 
 // Merge the partial rows of a stream's CTAs.  One block per (stream, head, slice of 64 value
