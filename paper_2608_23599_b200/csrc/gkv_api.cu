@@ -163,7 +163,7 @@ namespace {
 inline bool is_mla(const gkv_config& c) { return c.v_aliases_k != 0; }
 inline int geo_slot_bytes(const gkv_config& c, int level) { return is_mla(c) ? mla_slot_bytes(level) : slot_bytes(level); }
 inline uint64_t nval_per_token(const gkv_config& c) { return is_mla(c) ? c.d_k : c.d_k + c.d_v; }
-constexpr int kMlaTargetCtas = 148;          // one CTA per SM (213 KB of shared memory, tensor memory)
+constexpr int kMlaTargetCtas = 148;          // one CTA per SM (212 KB of shared memory, all of tensor memory)
 
 struct ArenaPlan {
   size_t status, debug, partial, range, mass, levels, scores, kper, tickets, jobs, mass_raw, res_raw, lse2, per_layer, heap_begin, total_meta;

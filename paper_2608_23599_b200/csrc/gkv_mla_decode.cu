@@ -1,23 +1,26 @@
 // Decode attention for latent-attention (MLA) streams (Sec. 3.1 read path applied to a 576-wide
-// latent row that is key and value at once), on warp-level tensor-core instructions.
+// latent row that is key and value at once), on warp-level tensor-core instructions with the
+// running output in tensor memory.
 //
 // A quantised latent row is k~[c] = s[c] * code[c] + z[c] with one (s, z) pair per channel and
 // half block (32 tokens, Sec. 3.2).  Nothing rounded ever becomes a tensor-core operand:
 //   * codes are used as they are stored: a code in the mantissa of an fp16 with a zero exponent
 //     field is the number code * 2^(b - 24), b its lowest bit (8-bit codes b = 0; 4-bit codes b = 0
 //     or 4), taken out of the packed words with byte permutes and masks only;
-//   * the scales go into the query, Q'[c][head] = q[c][head] * s[c] as an fp16 pair hi + lo (the
-//     product of an 8-bit and an 11-bit mantissa has 19 bits), formed in registers in the
-//     B-fragment layout once per half block; sum_c q[c] z[c] comes from one more MMA per channel
-//     slab whose A rows all hold the zero points;
-//   * O^T[512 x 16] += V~^T P^T reads the same packed codes a second time with tokens along k and
-//     channels along m; the probabilities are an fp16 pair hi + lo; the per-channel scale and the
+//   * keys, heads along the MMA rows: S^T[16 heads x 32 tokens] = Q'^T K^T.  The scales go into the
+//     query, Q'[c][head] = q[c][head] * s[c] as an fp16 pair hi + lo (the product of an 8-bit and an
+//     11-bit mantissa has 19 bits), formed in registers once per half block: a lane's query registers
+//     (heads g and g + 8, its four channels of the slab) times the scales are the A fragment, the code
+//     registers the B fragments of the four 8-token groups.  sum_c q[c] z[c] is one more MMA per
+//     channel slab with the unscaled query as A and the zero points in every column of B;
+//   * values: O^T[512 x 16] += V~^T P^T reads the same packed codes a second time with tokens along k
+//     and channels along m; the probabilities are an fp16 pair hi + lo; the per-channel scale and the
 //     zero point (times the half block's probability sum) are applied in fp32 to the half block's
-//     accumulator before it is added to the running O^T, which stays in registers;
+//     accumulator before it is added to the running O^T;
 //   * exact rows, the tail and centroid rows (one row per block, +log2(64) on the logit) are bf16
 //     operands of bf16 MMAs, the probabilities a bf16 pair hi + lo.
 //
-// Work split: a CTA is three groups of four warps ("quads").  A quad walks its own contiguous range
+// Work split: a CTA is four groups of four warps ("quads").  A quad walks its own contiguous range
 // of the stream's blocks in units of one half block (quantised) or 16 rows (exact, tail, centroid
 // runs); a unit is staged by one bulk copy (or one per row) into the quad's two-stage ring.  Inside
 // a quad warp w owns the value channels [128 w, 128 w + 128) and the rope channels
@@ -27,6 +30,11 @@
 // softmax, and then accumulates its own 128 rows of O^T.  A lane group g = lane / 4 owns the 16
 // channels 128 w + 16 g .. + 15: M-tile mu of the value MMAs has row g = channel 2 mu and row
 // g + 8 = channel 2 mu + 1 of them, for every kind of unit.
+//
+// Tensor memory holds what 128 registers per thread cannot: a warp's piece of the running O^T (64
+// fp32 per thread; the eight of an M-tile are loaded before its MMAs and stored after its update)
+// and the bf16 query fragments of its nine channel slabs for the row units.  Each warp touches only
+// its own columns of its own lane quarter, so no tensor-memory access needs a barrier.
 //
 // At the end the quads' (m, l, O^T) are merged in shared memory into the CTA's partial row; the
 // partial rows of a stream's CTAs are merged by mla_combine_kernel in CTA order.  Every wait is
@@ -48,7 +56,7 @@ constexpr int kMThreads = kMlaQuads * 128;
 constexpr int kMStageBytes = 20736;                    // one 8-bit half block: params 2304 + 32 x 576
 constexpr int kMStages = 2;
 constexpr int kMRowPitch = kMlaRowBytes + 16;          // bf16 rows staged at this pitch (conflict-free ldmatrix)
-constexpr int kMQPitch = 2 * kMlaRowBytes + 16;        // a head pair's row of the query copies: (q[g][c c+1], q[g + 8][c c+1]) per channel pair
+constexpr int kMQPitch = 2 * kMlaRowBytes + 16;        // a head pair's row of the fp16 query: (q[g][c c+1], q[g + 8][c c+1]) per channel pair
 constexpr int kMXBytes = 4 * 4 * 32 * 16;              // exchange buffer [warp][token group][lane] x 16 B = 8192
 constexpr int kMOffQ16 = 0;
 constexpr int kMOffQuad = 8 * kMQPitch;                // 18560
