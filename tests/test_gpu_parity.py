@@ -407,6 +407,32 @@ def test_mla_ingest_of_rows_that_are_not_16_byte_aligned():
     gcache.close()
 
 
+def test_mla_runs_of_mixed_levels_inside_one_warp_group_range():
+    """65,541 tokens per sequence under an external plan of short runs (1-8 blocks) of random levels: every
+    CTA of the read kernel gets several blocks, so the block ranges of its warp groups mix exact, 8-bit, 4-bit
+    and centroid units, cut centroid runs at range ends and switch between the unit kinds while the running
+    output stays in place."""
+    T = 65536 + 5
+    w = _mla(T, policy=W.POLICY_EXTERNAL)
+    ocache, gcache = _pair(w)
+    data = W.make_layer(w, 0, "cpu")
+    rs = np.random.RandomState(4242)
+    plan = np.empty((w.batch, 1, T // 64), dtype=np.int8)
+    for b in range(w.batch):
+        i = 0
+        while i < T // 64:
+            n = int(rs.randint(1, 9))
+            plan[b, 0, i:i + n] = rs.choice(np.array([16, 8, 4, 1], dtype=np.int8))
+            i += n
+    U.ingest_both(w, 0, data, ocache, gcache, level_plan=plan)
+    out, lse, o_out, o_lse = U.decode_both(ocache, gcache, 0, data["q"])
+    U.assert_outputs_close(out, o_out, "mla mixed runs")
+    assert np.max(np.abs(lse.cpu().numpy() - o_lse)) < 5e-3
+    rep_g, rep_o = gcache.gkv_bits_report(0), ocache.bits_report(0)
+    assert rep_g.resident_bits == rep_o["resident_bits"] and rep_g.last_read_bits == rep_o["last_read_bits"]
+    gcache.close()
+
+
 def test_cfg4_small_mla_ladder_with_appends():
     """Config 4 structure at small size: exact newest rung, int8, int4, centroid for the oldest
     quarter (5.0 bits/value), then appends with staircase demotion."""
