@@ -471,6 +471,9 @@ def run_ours(args, rank, local, world):
                      "ms_per_step_median_of_layers_run": m["ms_per_step_median"],
                      "ms_per_step_scaled_to_workload": m["ms_per_step"] * wc.n_layers / m["config"]["n_layers"],
                      "ms_per_step_median_scaled_to_workload": m["ms_per_step_median"] * wc.n_layers / m["config"]["n_layers"],
+                     # the median over the steps that close no block (the medians above count every step)
+                     "ms_plain_step_median_scaled_to_workload": (m["append_demote"]["ms_median_step_without_block_fill"] or m["ms_per_step_median"])
+                     * wc.n_layers / m["config"]["n_layers"],
                      "resident_bpv": m["workload_state"]["resident_bpv"], "bpv_paper": m["workload_state"]["bpv_paper"],
                      "block_fills_in_timed_region": m["workload_state"]["block_fills_in_timed_region"],
                      "ms_block_fill_steps": m["append_demote"]["ms_block_fill_steps"],
