@@ -124,11 +124,6 @@ __device__ __forceinline__ uint32_t m_lds32(uint32_t a) {
   asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(a));
   return v;
 }
-__device__ __forceinline__ float2 m_ldsf2(uint32_t a) {
-  float2 v;
-  asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];\n" : "=f"(v.x), "=f"(v.y) : "r"(a));
-  return v;
-}
 __device__ __forceinline__ float4 m_ldsf4(uint32_t a) {
   float4 v;
   asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
