@@ -1018,14 +1018,15 @@ int append_one(gkv_cache* c, int layer, const uint16_t* k_new, const uint16_t* v
 // staging are shared with the GQA path; the kernels are those of gkv_mla.cu.
 size_t mla_item_cost(const gkv_cache* c, const LayerState& L, int stream, int item) {
   // Cost of a block for the split of a stream over the CTAs and their quads, in units where a 4-bit
-  // block is 1000: measured on B200 as the time of a call over a cache that holds one rung only
-  // (262,144 tokens), less the call's fixed part, then adjusted on the 1M-token staircase.
+  // block is 1000.  Exact, 8-bit and 4-bit blocks: measured on B200 as the time of a call over a cache that
+  // holds one rung only (262,144 tokens), less the call's fixed part.  A centroid block is one row of a
+  // 16-row unit: swept on the 1M-token staircase (a call over centroid blocks only is all fixed cost).
   if (item < L.n_closed) {
     switch (L.level[static_cast<size_t>(stream) * c->max_blocks + item]) {
       case 16: return 1100;
       case 8: return 1030;
       case 4: return 1000;
-      default: return 125;
+      default: return 24;
     }
   }
   return 900;                     // tail
