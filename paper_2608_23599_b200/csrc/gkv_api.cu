@@ -1024,7 +1024,7 @@ size_t mla_item_cost(const gkv_cache* c, const LayerState& L, int stream, int it
   if (item < L.n_closed) {
     switch (L.level[static_cast<size_t>(stream) * c->max_blocks + item]) {
       case 16: return 1100;
-      case 8: return 1030;
+      case 8: return 1005;
       case 4: return 1000;
       default: return 24;
     }
