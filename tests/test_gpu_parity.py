@@ -496,6 +496,30 @@ def test_decode_is_bitwise_reproducible():
         assert np.array_equal(o, outs[0][0]) and np.array_equal(l, outs[0][1])
 
 
+@pytest.mark.gpu
+def test_mla_decode_is_bitwise_reproducible():
+    """Latent streams: the partial logits of a warp group are added in warp order, its warps' results and
+    the CTAs' rows are merged in a fixed order, so the same call twice and a second handle on the same rows
+    give identical bits.  The context is long enough for every warp group of every CTA to have blocks."""
+    w = _mla(148 * 4 * 3 * 64 + 17, batch=1, policy=W.POLICY_STAIRCASE, stair_tokens=(4096, 32768, 49152, 0))
+    outs = []
+    for _ in range(2):
+        _, gcache = _pair(w)
+        dev = gcache.device
+        data = W.make_layer(w, 0, "cpu")
+        gcache.gkv_append_demote(0, data["k"].to(dev), None)
+        q = data["q"].to(dev)
+        for _rep in range(3):
+            out = torch.empty((w.batch, w.n_q_heads, w.d_v), dtype=torch.float32, device=dev)
+            lse = torch.empty((w.batch, w.n_q_heads), dtype=torch.float32, device=dev)
+            gcache.gkv_decode_attn(0, q, out, lse=lse)
+            torch.cuda.synchronize()
+            outs.append((out.cpu().numpy().copy(), lse.cpu().numpy().copy()))
+        gcache.close()
+    for o, l in outs[1:]:
+        assert np.array_equal(o, outs[0][0]) and np.array_equal(l, outs[0][1])
+
+
 # ---- block attention mass observed by the decode pass (Sec. 3.1) -------------------------------
 MASS_RTOL, MASS_ATOL = 1e-2, 2e-6     # weights carry the logit error of fp16 operands (about 1e-3 relative)
 
