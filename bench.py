@@ -46,7 +46,7 @@ FALLBACK_HBM_GBS = 6650.0
 # capture (profiles/ holds the summaries); None = not captured for that workload.
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (ncu captures
 # summarised under profiles/): config 2 330.0 MB read + 3.8 MB written, config 4 386.4 + 6.7 MB
-DRAM_TRAFFIC_PER_LAUNCH = {"cfg2_llama8b_append": 333.8e6, "cfg4_mla_1m": 383.7e6}
+DRAM_TRAFFIC_PER_LAUNCH = {"cfg2_llama8b_append": 333.8e6, "cfg4_mla_1m": 382.3e6}
 
 
 def dominant_kernel(w) -> str:
