@@ -700,6 +700,10 @@ __global__ void __launch_bounds__(kMThreads, 1) mla_decode_kernel(const __grid_c
   const TableEntry* table = p.table + static_cast<size_t>(cd.stream) * p.table_stride;
   const uint16_t* qg = p.q + static_cast<size_t>(cd.stream) * kMlaHeads * kMlaDk;
 
+  // (launched with programmatic stream serialisation as well: nothing above reads what an earlier kernel of the
+  // stream may have written; the table, the query and the cache are touched after this wait)
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
   if (tid == 0) *abort_flag = 0;
   if (wq == 0 && lane == 0) {
     m_bar_init(bars, 1);
@@ -850,6 +854,10 @@ constexpr int kCombSlice = 64, kCombGroups = 8, kCombThreads = kCombSlice * kCom
 __global__ void __launch_bounds__(kCombThreads) mla_combine_kernel(const float* partial, const StreamParts* parts, float* out,
                                                                    float* lse) {
   __shared__ float sm_m[kCombThreads], sm_w[kCombThreads], sm_acc[kCombGroups][kCombSlice];
+  // launched with programmatic stream serialisation: the launch overlaps the decode kernel's tail, the
+  // partial rows are touched only after that kernel has completed
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
   const int stream = blockIdx.x, h = blockIdx.y, slice = blockIdx.z, tid = threadIdx.x;
   const int c = tid % kCombSlice, g = tid / kCombSlice;
   const int begin = parts[stream].begin, end = parts[stream].end;
@@ -911,11 +919,25 @@ cudaError_t launch_mla_decode(const MlaDecodeParams& p, int n_ctas, const Stream
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  mla_decode_kernel<<<n_ctas, kMThreads, kMSmem, st>>>(p);
-  cudaError_t e = cudaGetLastError();
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_ctas);
+  cfg.blockDim = dim3(kMThreads);
+  cfg.dynamicSmemBytes = kMSmem;
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, mla_decode_kernel, p);
   if (e != cudaSuccess) return e;
-  mla_combine_kernel<<<dim3(n_streams, kMlaHeads, kMlaDv / kCombSlice), kCombThreads, 0, st>>>(p.partial, parts, out, lse);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cc = {};
+  cc.gridDim = dim3(n_streams, kMlaHeads, kMlaDv / kCombSlice);
+  cc.blockDim = dim3(kCombThreads);
+  cc.stream = st;
+  cc.attrs = attr;
+  cc.numAttrs = 1;
+  return cudaLaunchKernelEx(&cc, mla_combine_kernel, static_cast<const float*>(p.partial), parts, out, lse);
 }
 
 }  // namespace gkv
