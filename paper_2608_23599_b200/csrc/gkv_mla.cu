@@ -127,6 +127,10 @@ __global__ void __launch_bounds__(256) mla_encode_kernel(const __grid_constant__
 __global__ void __launch_bounds__(288) mla_append_rows_kernel(uint8_t* arena, const TableEntry* table, int table_stride,
                                                               int tail_index, const uint16_t* k_in, int n_tok,
                                                               int first_tok, int dst_row0) {
+  // launched with programmatic stream serialisation: returns once the previous kernel of the stream has
+  // completed (the launch itself overlaps that kernel's tail)
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
   const int stream = blockIdx.x, row = blockIdx.y;
   const TableEntry e = table[static_cast<size_t>(stream) * table_stride + tail_index];
   const uint32_t* src = reinterpret_cast<const uint32_t*>(k_in + (static_cast<size_t>(stream) * n_tok + first_tok + row) * kMlaDk);
@@ -171,9 +175,16 @@ cudaError_t launch_mla_encode(const MlaEncodeParams& p, cudaStream_t st) {
 cudaError_t launch_mla_append_rows(uint8_t* arena, const TableEntry* table, int table_stride, int tail_index, int n_streams,
                                    const uint16_t* k_in, int n_tok, int first_tok, int n_rows, int dst_row0, cudaStream_t st) {
   if (n_rows <= 0) return cudaSuccess;
-  mla_append_rows_kernel<<<dim3(n_streams, n_rows), kMlaDk / 2, 0, st>>>(arena, table, table_stride, tail_index, k_in, n_tok,
-                                                                         first_tok, dst_row0);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_streams, n_rows);
+  cfg.blockDim = dim3(kMlaDk / 2);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, mla_append_rows_kernel, arena, table, table_stride, tail_index, k_in, n_tok, first_tok, dst_row0);
 }
 
 cudaError_t launch_mla_export(const uint8_t* arena, uint32_t off256, int level, uint8_t* codes, uint16_t* scale,
